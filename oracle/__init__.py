@@ -1,0 +1,171 @@
+"""ctypes binding of the fp64 CPU oracle (``vla_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the CPU-baseline leg
+of the benchmark load this; the CUDA package never does.  The binding only
+marshals numpy arrays; all arithmetic is in the C file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "vla_oracle.c")
+_HDR = os.path.join(_HERE, "vla_oracle.h")
+_LIB = os.path.join(_HERE, "libvla_oracle.so")
+
+F32, BF16, F64 = 0, 1, 2
+IDENTITY_MAP = 1
+
+_lock = threading.Lock()
+_default = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, no vector intrinsics) if it is stale."""
+    newest_src = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest_src:
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-std=c99", "-O2", "-fPIC", "-shared", "-Wall", "-Wextra",
+             "-o", tmp, _SRC, "-lm", "-lpthread"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Trace(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("A", "S", "khat", "u", "alpha", "e", "delta", "den")]
+
+
+def _bind(path):
+    lib = ctypes.CDLL(path)
+    vp, i, d, u = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_uint
+    lib.vla_oracle_forward.restype = i
+    lib.vla_oracle_forward.argtypes = [vp, vp, vp, vp, i, d, i, i, i, i, i,
+                                       vp, vp, vp, u, d, vp, vp, vp, vp, i]
+    lib.vla_oracle_forward_trace.restype = i
+    lib.vla_oracle_forward_trace.argtypes = [vp, vp, vp, vp, i, d, i, i, i,
+                                             vp, vp, vp, u, d, vp, vp, vp, vp,
+                                             ctypes.POINTER(_Trace)]
+    return lib
+
+
+def _np_dtype(in_dtype: int):
+    return {F32: np.float32, BF16: np.uint16, F64: np.float64}[in_dtype]
+
+
+def _in(a, in_dtype, shape):
+    a = np.ascontiguousarray(a, dtype=_np_dtype(in_dtype))
+    assert a.shape == tuple(shape), (a.shape, shape)
+    return a
+
+
+def _opt64(a, shape):
+    if a is None:
+        return None
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    assert a.shape == tuple(shape), (a.shape, shape)
+    return a
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+@dataclass
+class OracleResult:
+    out: np.ndarray   # [B,H,T,d_v] fp64
+    S_T: np.ndarray   # [B,H,d_v,d_k]
+    A_T: np.ndarray   # [B,H,d_k,d_k]
+    z_T: np.ndarray   # [B,H,d_k]
+    trace: Optional[dict] = None
+
+
+class OracleLib:
+    """One loaded build of the oracle.  ``load()`` gives the committed source's build;
+    the mutation tests wrap deliberately broken builds of a copy of the C file."""
+
+    def __init__(self, path: str):
+        self.path = path
+        self._lib = _bind(path)
+
+    def forward(self, q, k, v, lam, *, u=None, in_dtype=F32, S0=None, A0=None, z0=None,
+                flags=0, eps=1e-4, n_threads=1) -> OracleResult:
+        """All units of ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``.
+
+        bf16 inputs are passed as uint16 bit patterns (``in_dtype=BF16``).
+        """
+        lib = self._lib
+        B, H, T, dk = np.shape(q)
+        dv = np.shape(v)[-1]
+        q = _in(q, in_dtype, (B, H, T, dk))
+        k = _in(k, in_dtype, (B, H, T, dk))
+        v = _in(v, in_dtype, (B, H, T, dv))
+        u = None if u is None else _in(u, in_dtype, (B, H, T, dk))
+        S0 = _opt64(S0, (B, H, dv, dk))
+        A0 = _opt64(A0, (B, H, dk, dk))
+        z0 = _opt64(z0, (B, H, dk))
+        out = np.empty((B, H, T, dv), np.float64)
+        S_T = np.empty((B, H, dv, dk), np.float64)
+        A_T = np.empty((B, H, dk, dk), np.float64)
+        z_T = np.empty((B, H, dk), np.float64)
+        rc = lib.vla_oracle_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(u), in_dtype, float(lam),
+                                    B, H, T, dk, dv, _ptr(S0), _ptr(A0), _ptr(z0),
+                                    flags, float(eps), _ptr(out), _ptr(S_T), _ptr(A_T),
+                                    _ptr(z_T), int(n_threads))
+        if rc != 0:
+            raise ValueError("vla_oracle_forward: invalid argument")
+        return OracleResult(out, S_T, A_T, z_T)
+
+
+    def forward_trace(self, q, k, v, lam, *, u=None, in_dtype=F64, S0=None, A0=None, z0=None,
+                      flags=0, eps=1e-4) -> OracleResult:
+        """One unit (``q,k[,u]: [T,d_k]``, ``v: [T,d_v]``) with every per-step quantity dumped."""
+        lib = self._lib
+        T, dk = np.shape(q)
+        dv = np.shape(v)[-1]
+        q = _in(q, in_dtype, (T, dk))
+        k = _in(k, in_dtype, (T, dk))
+        v = _in(v, in_dtype, (T, dv))
+        u = None if u is None else _in(u, in_dtype, (T, dk))
+        S0 = _opt64(S0, (dv, dk))
+        A0 = _opt64(A0, (dk, dk))
+        z0 = _opt64(z0, (dk,))
+        out = np.empty((T, dv), np.float64)
+        S_T = np.empty((dv, dk), np.float64)
+        A_T = np.empty((dk, dk), np.float64)
+        z_T = np.empty((dk,), np.float64)
+        tr = dict(A=np.empty((T, dk, dk)), S=np.empty((T, dv, dk)), khat=np.empty((T, dk)),
+                  u=np.empty((T, dk)), alpha=np.empty((T, dk)), e=np.empty((T, dv)),
+                  delta=np.empty((T,)), den=np.empty((T,)))
+        ctr = _Trace(**{n: a.ctypes.data for n, a in tr.items()})
+        rc = lib.vla_oracle_forward_trace(_ptr(q), _ptr(k), _ptr(v), _ptr(u), in_dtype,
+                                          float(lam), T, dk, dv, _ptr(S0), _ptr(A0), _ptr(z0),
+                                          flags, float(eps), _ptr(out), _ptr(S_T), _ptr(A_T),
+                                          _ptr(z_T), ctypes.byref(ctr))
+        if rc != 0:
+            raise ValueError("vla_oracle_forward_trace: invalid argument")
+        return OracleResult(out, S_T, A_T, z_T, tr)
+
+
+def load() -> OracleLib:
+    global _default
+    with _lock:
+        if _default is None:
+            _default = OracleLib(build())
+    return _default
+
+
+def forward(*args, **kw) -> OracleResult:
+    return load().forward(*args, **kw)
+
+
+def forward_trace(*args, **kw) -> OracleResult:
+    return load().forward_trace(*args, **kw)

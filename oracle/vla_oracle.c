@@ -1,0 +1,240 @@
+/*
+ * vla_oracle.c -- CPU oracle for the Variational Linear Attention forward scan.
+ *
+ * TEST INFRASTRUCTURE ONLY (see vla_oracle.h).  Plain C, fp64, one token at a
+ * time, in the order and notation of the paper's Algorithm 1 ("VLAv3
+ * sequential forward pass"), with three stated departures:
+ *   - the projections W_k, W_q, W_v, W_u are not applied: q, k, v (and u when
+ *     given) arrive already projected;
+ *   - the periodic identity refresh (A += eta*I every 20 steps) is left out,
+ *     because it contradicts A_t = M_t^{-1} (Section 1.2, Eq. "A-covariance");
+ *   - both norms are guarded as x / max(||x||, eps) (Section 5.3: "eps for
+ *     all denominators").
+ * No blocking, fusion or reordering: every matrix-vector product is a double
+ * loop, every rank-1 update a double loop.
+ *
+ * What pins it (tests/test_oracle_*.py, all independent of this file):
+ *   A-chain      brute-force inverse of M_t = lambda*I + sum u u^T; trace and
+ *                eigenvalue invariants; delta in [1, 1 + 1/lambda].
+ *   alpha_hat    unit norm; parallel to inv(M_t) k_hat (post-update A_t).
+ *   S-chain      closed forms (first step, orthonormal keys, repeated key),
+ *                the u = 0 reduction to the normalised delta rule written
+ *                separately, the corrected associative (R, G) composition of
+ *                Section 3.4, Proposition 1's norm identities.
+ *   readout      S_t q_t from dumped states; denominator from a direct sum.
+ *   state carry  split invariance.
+ * Absolute output values on random data are otherwise fixed by nothing the
+ * paper prints ("parity unpinned" beyond the pins above): this file is the
+ * definition the CUDA path is compared with.
+ */
+#include "vla_oracle.h"
+
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* phi(x) = ELU(x) + 1  (Section 3.3, below Eq. "output") */
+static double phi(double x) { return x > 0.0 ? x + 1.0 : exp(x); }
+
+/* exact widening of one stored element */
+static double load_elem(const void* base, size_t idx, int dtype) {
+  if (dtype == VLA_ORACLE_F64) return ((const double*)base)[idx];
+  if (dtype == VLA_ORACLE_F32) return (double)((const float*)base)[idx];
+  /* bfloat16: the upper 16 bits of an IEEE binary32 */
+  uint32_t bits = (uint32_t)((const uint16_t*)base)[idx] << 16;
+  float f;
+  memcpy(&f, &bits, sizeof f);
+  return (double)f;
+}
+
+static double dot(const double* a, const double* b, int n) {
+  double s = 0.0;
+  for (int i = 0; i < n; ++i) s += a[i] * b[i];
+  return s;
+}
+
+/*
+ * One (b, h) unit.  q,k,u point at this unit's [T, d_k] block, v at [T, d_v].
+ * S [d_v*d_k], A [d_k*d_k], zk [d_k] hold the incoming state and are updated
+ * in place; out is [T, d_v].
+ */
+static void scan_unit(const void* q, const void* k, const void* v, const void* u_in,
+                      size_t qk_off, size_t v_off, int dtype, int T, int dk, int dv,
+                      unsigned flags, double eps, double* S, double* A, double* zk,
+                      double* out, const vla_oracle_trace_t* tr) {
+  const int identity = (flags & VLA_ORACLE_IDENTITY_MAP) != 0;
+  double* kf = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* khat = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* u = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* zsm = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* alpha = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* qf = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* e = (double*)malloc(sizeof(double) * (size_t)dv);
+
+  for (int t = 0; t < T; ++t) {
+    const size_t row_k = qk_off + (size_t)t * (size_t)dk;
+    const size_t row_v = v_off + (size_t)t * (size_t)dv;
+
+    /* k_feat = ELU(k_raw) + 1 (Algorithm 1) or k_raw itself (Section 3.1) */
+    for (int j = 0; j < dk; ++j) {
+      double kr = load_elem(k, row_k + j, dtype);
+      kf[j] = identity ? kr : phi(kr);
+    }
+    /* k_hat = k_feat / ||k_feat|| */
+    {
+      double nrm = sqrt(dot(kf, kf, dk));
+      double g = nrm > eps ? nrm : eps;
+      for (int j = 0; j < dk; ++j) khat[j] = kf[j] / g;
+    }
+    /* penalty direction: supplied verbatim, else u_t = k_hat_t */
+    for (int j = 0; j < dk; ++j)
+      u[j] = u_in ? load_elem(u_in, row_k + j, dtype) : khat[j];
+
+    /* --- Sherman-Morrison (Eq. "sm") --- */
+    for (int i = 0; i < dk; ++i) zsm[i] = dot(A + (size_t)i * dk, u, dk); /* z = A_{t-1} u */
+    double delta = 1.0 + dot(u, zsm, dk);
+    if (delta < eps) delta = eps; /* Algorithm 1's clamp; inert since delta >= 1 */
+    for (int i = 0; i < dk; ++i)
+      for (int j = 0; j < dk; ++j) A[(size_t)i * dk + j] -= zsm[i] * zsm[j] / delta;
+
+    /* --- write direction from the POST-update A_t (Eq. "s-update") --- */
+    {
+      for (int i = 0; i < dk; ++i) alpha[i] = dot(A + (size_t)i * dk, khat, dk);
+      double nrm = sqrt(dot(alpha, alpha, dk));
+      double g = nrm > eps ? nrm : eps;
+      for (int i = 0; i < dk; ++i) alpha[i] /= g;
+    }
+
+    /* --- residual state update: e = v - S_{t-1} k_hat ; S += e alpha^T --- */
+    for (int i = 0; i < dv; ++i)
+      e[i] = load_elem(v, row_v + i, dtype) - dot(S + (size_t)i * dk, khat, dk);
+    for (int i = 0; i < dv; ++i)
+      for (int j = 0; j < dk; ++j) S[(size_t)i * dk + j] += e[i] * alpha[j];
+
+    /* --- readout (Eq. "output") --- */
+    double den = 1.0;
+    for (int j = 0; j < dk; ++j) {
+      double qr = load_elem(q, row_k + j, dtype);
+      qf[j] = identity ? qr : phi(qr);
+    }
+    if (!identity) {
+      for (int j = 0; j < dk; ++j) zk[j] += kf[j]; /* z^key includes token t */
+      den = dot(zk, qf, dk);
+      if (den < eps) den = eps;
+    }
+    for (int i = 0; i < dv; ++i)
+      out[(size_t)t * dv + i] = dot(S + (size_t)i * dk, qf, dk) / den;
+
+    if (tr) {
+      if (tr->A) memcpy(tr->A + (size_t)t * dk * dk, A, sizeof(double) * (size_t)dk * dk);
+      if (tr->S) memcpy(tr->S + (size_t)t * dv * dk, S, sizeof(double) * (size_t)dv * dk);
+      if (tr->khat) memcpy(tr->khat + (size_t)t * dk, khat, sizeof(double) * (size_t)dk);
+      if (tr->u) memcpy(tr->u + (size_t)t * dk, u, sizeof(double) * (size_t)dk);
+      if (tr->alpha) memcpy(tr->alpha + (size_t)t * dk, alpha, sizeof(double) * (size_t)dk);
+      if (tr->e) memcpy(tr->e + (size_t)t * dv, e, sizeof(double) * (size_t)dv);
+      if (tr->delta) tr->delta[t] = delta;
+      if (tr->den) tr->den[t] = den;
+    }
+  }
+  free(kf); free(khat); free(u); free(zsm); free(alpha); free(qf); free(e);
+}
+
+typedef struct {
+  const void *q, *k, *v, *u;
+  int dtype, T, dk, dv;
+  double lambda, eps;
+  unsigned flags;
+  const double *S0, *A0, *z0;
+  double *out, *S_T, *A_T, *z_T;
+  const vla_oracle_trace_t* tr;
+  long unit_begin, unit_end;
+} job_t;
+
+static void* run_units(void* arg) {
+  const job_t* jb = (const job_t*)arg;
+  const size_t dk = (size_t)jb->dk, dv = (size_t)jb->dv, T = (size_t)jb->T;
+  double* S = (double*)malloc(sizeof(double) * dv * dk);
+  double* A = (double*)malloc(sizeof(double) * dk * dk);
+  double* zk = (double*)malloc(sizeof(double) * dk);
+  for (long n = jb->unit_begin; n < jb->unit_end; ++n) {
+    /* initial state: S_0 = 0, A_0 = I/lambda_0, z = 0 unless carried in */
+    if (jb->S0) memcpy(S, jb->S0 + (size_t)n * dv * dk, sizeof(double) * dv * dk);
+    else memset(S, 0, sizeof(double) * dv * dk);
+    if (jb->A0) memcpy(A, jb->A0 + (size_t)n * dk * dk, sizeof(double) * dk * dk);
+    else {
+      memset(A, 0, sizeof(double) * dk * dk);
+      for (size_t i = 0; i < dk; ++i) A[i * dk + i] = 1.0 / jb->lambda;
+    }
+    if (jb->z0) memcpy(zk, jb->z0 + (size_t)n * dk, sizeof(double) * dk);
+    else memset(zk, 0, sizeof(double) * dk);
+
+    scan_unit(jb->q, jb->k, jb->v, jb->u, (size_t)n * T * dk, (size_t)n * T * dv, jb->dtype,
+              jb->T, jb->dk, jb->dv, jb->flags, jb->eps, S, A, zk,
+              jb->out + (size_t)n * T * dv, jb->tr);
+
+    if (jb->S_T) memcpy(jb->S_T + (size_t)n * dv * dk, S, sizeof(double) * dv * dk);
+    if (jb->A_T) memcpy(jb->A_T + (size_t)n * dk * dk, A, sizeof(double) * dk * dk);
+    if (jb->z_T) memcpy(jb->z_T + (size_t)n * dk, zk, sizeof(double) * dk);
+  }
+  free(S); free(A); free(zk);
+  return NULL;
+}
+
+static int check_args(const void* q, const void* k, const void* v, int in_dtype, double lambda,
+                      long units, int T, int dk, int dv, const double* A0, double eps,
+                      const double* out) {
+  if (units < 0 || T < 0 || dk <= 0 || dv <= 0) return -1;
+  if (in_dtype != VLA_ORACLE_F32 && in_dtype != VLA_ORACLE_BF16 && in_dtype != VLA_ORACLE_F64)
+    return -1;
+  if (!A0 && !(lambda > 0.0)) return -1;
+  if (!(eps > 0.0)) return -1;
+  if (units > 0 && T > 0 && (!q || !k || !v || !out)) return -1;
+  return 0;
+}
+
+int vla_oracle_forward(const void* q, const void* k, const void* v, const void* u,
+                       int in_dtype, double lambda, int B, int H, int T, int d_k, int d_v,
+                       const double* S0, const double* A0, const double* z0, unsigned flags,
+                       double eps, double* out, double* S_T, double* A_T, double* z_T,
+                       int n_threads) {
+  if (B < 0 || H < 0) return -1;
+  const long units = (long)B * (long)H;
+  if (check_args(q, k, v, in_dtype, lambda, units, T, d_k, d_v, A0, eps, out)) return -1;
+  if (units == 0) return 0;
+  if (n_threads < 1) n_threads = 1;
+  if (n_threads > units) n_threads = (int)units;
+
+  job_t base = {q, k, v, u, in_dtype, T, d_k, d_v, lambda, eps, flags,
+                S0, A0, z0, out, S_T, A_T, z_T, NULL, 0, 0};
+  if (n_threads == 1) {
+    base.unit_begin = 0;
+    base.unit_end = units;
+    run_units(&base);
+    return 0;
+  }
+  pthread_t* th = (pthread_t*)malloc(sizeof(pthread_t) * (size_t)n_threads);
+  job_t* jobs = (job_t*)malloc(sizeof(job_t) * (size_t)n_threads);
+  for (int i = 0; i < n_threads; ++i) {
+    jobs[i] = base;
+    jobs[i].unit_begin = units * i / n_threads;
+    jobs[i].unit_end = units * (i + 1) / n_threads;
+    pthread_create(&th[i], NULL, run_units, &jobs[i]);
+  }
+  for (int i = 0; i < n_threads; ++i) pthread_join(th[i], NULL);
+  free(th); free(jobs);
+  return 0;
+}
+
+int vla_oracle_forward_trace(const void* q, const void* k, const void* v, const void* u,
+                             int in_dtype, double lambda, int T, int d_k, int d_v,
+                             const double* S0, const double* A0, const double* z0,
+                             unsigned flags, double eps, double* out, double* S_T,
+                             double* A_T, double* z_T, const vla_oracle_trace_t* trace) {
+  if (check_args(q, k, v, in_dtype, lambda, 1, T, d_k, d_v, A0, eps, out)) return -1;
+  job_t jb = {q, k, v, u, in_dtype, T, d_k, d_v, lambda, eps, flags,
+              S0, A0, z0, out, S_T, A_T, z_T, trace, 0, 1};
+  run_units(&jb);
+  return 0;
+}

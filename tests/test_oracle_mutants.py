@@ -1,0 +1,80 @@
+"""The pins have teeth: each plausible mistake, planted in a COPY of the oracle's C
+file (on the CPU, in a temp directory), must trip at least one pin.  The committed
+oracle itself is never modified."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+import oracle
+from oracle_pins import PINS, pin_paper_constants
+from test_oracle_pins import read_golden
+
+SRC = os.path.join(os.path.dirname(oracle.__file__), "vla_oracle.c")
+
+# (name, text in the oracle, replacement)
+MUTANTS = [
+    ("sm_sign", "-= zsm[i] * zsm[j] / delta;", "+= zsm[i] * zsm[j] / delta;"),
+    ("sm_no_division", "-= zsm[i] * zsm[j] / delta;", "-= zsm[i] * zsm[j];"),
+    ("delta_drops_one", "double delta = 1.0 + dot(u, zsm, dk);", "double delta = dot(u, zsm, dk);"),
+    ("delta_wrong_dot", "double delta = 1.0 + dot(u, zsm, dk);", "double delta = 1.0 + dot(zsm, zsm, dk);"),
+    ("z_uses_khat", "zsm[i] = dot(A + (size_t)i * dk, u, dk);", "zsm[i] = dot(A + (size_t)i * dk, khat, dk);"),
+    ("u_ignored", "u[j] = u_in ? load_elem(u_in, row_k + j, dtype) : khat[j];", "u[j] = khat[j];"),
+    ("alpha_from_pre_update_A", "alpha[i] = dot(A + (size_t)i * dk, khat, dk);",
+     "alpha[i] = dot(A + (size_t)i * dk, khat, dk) + zsm[i] * dot(zsm, khat, dk) / delta;"),
+    ("alpha_not_normalised", "alpha[i] /= g;", "alpha[i] /= 1.0;"),
+    ("khat_not_normalised", "khat[j] = kf[j] / g;", "khat[j] = kf[j];"),
+    ("residual_sign", "- dot(S + (size_t)i * dk, khat, dk);", "+ dot(S + (size_t)i * dk, khat, dk);"),
+    ("residual_no_prediction", "- dot(S + (size_t)i * dk, khat, dk);", ";"),
+    ("write_along_khat", "S[(size_t)i * dk + j] += e[i] * alpha[j];", "S[(size_t)i * dk + j] += e[i] * khat[j];"),
+    ("write_sign", "S[(size_t)i * dk + j] += e[i] * alpha[j];", "S[(size_t)i * dk + j] -= e[i] * alpha[j];"),
+    ("readout_pre_update_S", "dot(S + (size_t)i * dk, qf, dk) / den;",
+     "(dot(S + (size_t)i * dk, qf, dk) - e[i] * dot(alpha, qf, dk)) / den;"),
+    ("readout_no_normaliser", "dot(S + (size_t)i * dk, qf, dk) / den;", "dot(S + (size_t)i * dk, qf, dk);"),
+    ("den_excludes_current_token", "den = dot(zk, qf, dk);", "den = dot(zk, qf, dk) - dot(kf, qf, dk);"),
+    ("elu_without_plus_one", "return x > 0.0 ? x + 1.0 : exp(x);", "return x > 0.0 ? x : exp(x) - 1.0;"),
+    ("phi_wrong_branch", "return x > 0.0 ? x + 1.0 : exp(x);", "return x > 0.0 ? x + 1.0 : 1.0 + x;"),
+    ("q_not_mapped", "qf[j] = identity ? qr : phi(qr);", "qf[j] = qr;"),
+    ("A0_is_lambda_I", "A[i * dk + i] = 1.0 / jb->lambda;", "A[i * dk + i] = jb->lambda;"),
+    ("z0_ignored", "if (jb->z0) memcpy(zk,", "if (0) memcpy(zk,"),
+    ("S0_ignored", "if (jb->S0) memcpy(S,", "if (0) memcpy(S,"),
+    ("out_unit_stride", "jb->out + (size_t)n * T * dv, jb->tr);", "jb->out + (size_t)n * T * dk, jb->tr);"),
+    ("bf16_shift", "[idx] << 16;", "[idx] << 15;"),
+    ("eps_guard_missing", "double g = nrm > eps ? nrm : eps;\n      for (int j = 0; j < dk; ++j) khat[j]",
+     "double g = nrm;\n      for (int j = 0; j < dk; ++j) khat[j]"),
+]
+
+
+def _tripped_by(orc):
+    for pin in PINS:
+        try:
+            pin(orc)
+        except Exception:          # AssertionError, or a LinAlgError from a non-finite state
+            return pin.__name__
+    try:
+        pin_paper_constants(orc, read_golden())
+    except Exception:
+        return "pin_paper_constants"
+    return None
+
+
+@pytest.mark.parametrize("name,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_mutant_is_caught(tmp_path, name, old, new):
+    text = open(SRC).read()
+    assert text.count(old) == 1, "mutation site must match the oracle source exactly once: %r" % old
+    c = tmp_path / "vla_oracle.c"
+    c.write_text(text.replace(old, new))
+    (tmp_path / "vla_oracle.h").write_text(open(SRC[:-2] + ".h").read())
+    so = str(tmp_path / ("mut_%s.so" % name))
+    subprocess.check_call(["gcc", "-std=c99", "-O2", "-fPIC", "-shared", "-w", "-o", so, str(c),
+                           "-lm", "-lpthread"])
+    # a child process, so that a mutant that corrupts memory cannot take pytest down
+    here = os.path.dirname(os.path.abspath(__file__))
+    code = ("import sys; sys.path[:0] = [%r, %r]; import oracle, test_oracle_mutants as m; "
+            "print('CAUGHT_BY', m._tripped_by(oracle.OracleLib(%r)))" % (here, os.path.dirname(here), so))
+    res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300)
+    if res.returncode != 0:
+        return                      # the mutant crashed: noticed
+    caught = res.stdout.strip().split("CAUGHT_BY")[-1].strip()
+    assert caught != "None", "no pin notices the planted mistake %r" % name

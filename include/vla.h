@@ -1,0 +1,123 @@
+/*
+ * vla.h -- C ABI of the B200 (sm_100a) Variational Linear Attention forward scan.
+ *
+ * One call runs, for every (batch, head) unit independently, the causal scan of
+ * the paper's Section 3.3 (Eqs. "sm", "s-update", "output"; Algorithm 1 without
+ * the projections and without the periodic refresh).  Per token t:
+ *
+ *     k_hat = kf / max(||kf||, eps)        kf = phi(k_t)  (phi = ELU+1, Algorithm 1)
+ *                                          kf = k_t       (VLA_FLAG_IDENTITY_MAP, Section 3.1)
+ *     u     = u_t as given, or k_hat when no u is supplied          (Eq. "penalty")
+ *     z     = A_{t-1} u ;  delta = max(1 + u.z, eps) ;  A_t = A_{t-1} - z z^T / delta   (Eq. "sm")
+ *     alpha = A_t k_hat / max(||A_t k_hat||, eps)                   (Eq. "s-update", post-update A_t)
+ *     e     = v_t - S_{t-1} k_hat ;  S_t = S_{t-1} + e alpha^T      (Eq. "s-update")
+ *     o_t   = S_t phi(q_t) / max(phi(q_t).zkey_t, eps),  zkey_t = zkey_{t-1} + phi(k_t)   (Eq. "output")
+ *     o_t   = S_t q_t                                               (VLA_FLAG_IDENTITY_MAP)
+ *
+ * All state arithmetic is fp32 on the GPU.  There is no CPU fallback: a shape
+ * the kernels do not cover returns VLA_ERR_UNSUPPORTED.
+ *
+ * Memory: unless a function says otherwise every pointer is a DEVICE pointer owned by
+ * the caller, tensors are contiguous and row-major, and base pointers are 16-byte
+ * aligned (else VLA_ERR_ALIGNMENT).  The library allocates nothing, keeps no state
+ * between calls, and never synchronises the device; work is enqueued on `stream`.
+ */
+#ifndef VLA_H
+#define VLA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  VLA_OK = 0,
+  VLA_ERR_INVALID_ARG = -1,    /* null/negative/ill-formed argument (host-side check)        */
+  VLA_ERR_UNSUPPORTED = -2,    /* shape/dtype/flag combination without a kernel              */
+  VLA_ERR_ALIGNMENT = -3,      /* a base pointer is not 16-byte aligned                      */
+  VLA_ERR_CUDA = -4,           /* a CUDA runtime call or the launch failed                   */
+  VLA_ERR_DEVICE_TIMEOUT = -5, /* written to opts->status: a bounded device-side wait ran out */
+  VLA_ERR_NONFINITE = -6       /* written to opts->status: non-finite delta / norm seen       */
+} vla_status_t;
+
+typedef enum { VLA_F32 = 0, VLA_BF16 = 1 } vla_dtype_t;
+
+enum {
+  VLA_FLAG_IDENTITY_MAP = 1u << 0, /* Section 3.1: k_hat = k/||k||, o_t = S_t q_t              */
+  VLA_FLAG_CHECK_FINITE = 1u << 1  /* report non-finite delta or ||A_t k_hat|| in opts->status */
+};
+
+/* Which scan kernel runs.  AUTO picks by shape; the others force one (tests, benchmarks). */
+typedef enum {
+  VLA_KERNEL_AUTO = 0,
+  VLA_KERNEL_TOKEN = 1  /* one CTA per unit, one state pass per token */
+} vla_kernel_t;
+
+typedef struct {
+  uint32_t struct_size;  /* = sizeof(vla_opts_t); lets the struct grow without breaking callers */
+  int32_t qkv_dtype;     /* vla_dtype_t of q, k, v, u.  Default VLA_F32                          */
+  const void* u;         /* [B,H,T,d_k] penalty directions, used verbatim (the caller applies
+                            f_theta, the L2 norm and any 1/sqrt(d_h)); NULL => u_t = k_hat_t    */
+  uint32_t flags;        /* VLA_FLAG_*; 0 = Algorithm 1                                         */
+  float eps;             /* stability floor of every denominator; <= 0 => 1e-4 (Section 5.3)    */
+  const float* z0;       /* [B,H,d_k] running sum of phi(k) carried in;  NULL => 0              */
+  float* zT;             /* [B,H,d_k] the same after T tokens;           NULL => not written    */
+  int32_t* status;       /* device int32, 0 on entry; set to a negative vla_status_t on a
+                            device-side problem.  Read it after synchronising.  NULL allowed    */
+  int32_t kernel;        /* vla_kernel_t                                                        */
+} vla_opts_t;
+
+/*
+ * vla_forward -- Section 3.3 / Algorithm 1, all B*H units, T tokens each.
+ *   q, k : [B,H,T,d_k]   v : [B,H,T,d_v]   in opts->qkv_dtype (fp32 default, bf16 widened in-kernel)
+ *   lambda_ : lambda_0 of Eq. "penalty"; A_0 = I/lambda_ when A0 == NULL (must then be > 0)
+ *   S0 : [B,H,d_v,d_k] fp32, row = value index (S k_hat predicts v); NULL => 0
+ *   A0 : [B,H,d_k,d_k] fp32, symmetric positive definite;           NULL => I/lambda_
+ *   out: [B,H,T,d_v] fp32
+ *   S_T, A_T: final states, fp32, same layouts; NULL => not written.  They may alias S0/A0.
+ *   out must not overlap any input.  T == 0 is legal and copies the state through.
+ *   Supported: d_k == d_v in {16, 32, 64, 128}.
+ * Returns VLA_OK once the work is enqueued on `stream` (a cudaStream_t; NULL = default
+ * stream), or a negative vla_status_t from host-side validation / launch.  Device-side
+ * problems are reported through opts->status.
+ */
+int vla_forward(const void* q, const void* k, const void* v, float lambda_,
+                int B, int H, int T, int d_k, int d_v,
+                const float* S0, const float* A0,
+                float* out, float* S_T, float* A_T,
+                const vla_opts_t* opts, void* stream);
+
+/*
+ * vla_forward_host -- the same computation for callers whose tensors live in HOST memory.
+ * q, k, v, opts->u, S0, A0, opts->z0, out, S_T, A_T, opts->zT are HOST pointers (pinned
+ * memory makes the copies asynchronous); `workspace` is a DEVICE buffer of at least
+ * vla_host_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller.  The call
+ * enqueues host->device copies, the scan and device->host copies on `stream` and returns
+ * without synchronising; outputs are valid once the stream has been synchronised.
+ * opts->status, when given, stays a DEVICE pointer.
+ */
+int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
+                     int B, int H, int T, int d_k, int d_v,
+                     const float* S0, const float* A0,
+                     float* out, float* S_T, float* A_T,
+                     const vla_opts_t* opts, void* workspace, size_t workspace_bytes,
+                     void* stream);
+
+/* Device bytes vla_forward_host needs for these sizes (0 on invalid sizes). */
+size_t vla_host_workspace_bytes(int B, int H, int T, int d_k, int d_v, int qkv_dtype, int has_u);
+
+/* VLA_OK when a kernel covers (d_k, d_v, dtype, flags), else VLA_ERR_UNSUPPORTED. */
+int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags);
+
+/* Static, NUL-terminated description of a vla_status_t value. */
+const char* vla_status_string(int status);
+
+/* major*10000 + minor*100 + patch */
+int vla_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VLA_H */

@@ -1,0 +1,225 @@
+"""Thin Python binding of the C ABI in ``include/vla.h``: argument marshalling only.
+
+Every step of the scan runs in the CUDA kernels behind ``libvla.so``.  There is no
+fallback: if the library is missing or a shape has no kernel, the call raises.
+PyTorch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+VLA_OK = 0
+VLA_ERR_INVALID_ARG, VLA_ERR_UNSUPPORTED, VLA_ERR_ALIGNMENT = -1, -2, -3
+VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE = -4, -5, -6
+VLA_F32, VLA_BF16 = 0, 1
+VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE = 1, 2
+VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN = 0, 1
+
+EXPORTS = ("vla_forward", "vla_forward_host", "vla_host_workspace_bytes",
+           "vla_query_support", "vla_status_string", "vla_version")
+
+
+class VlaOpts(ctypes.Structure):
+    """Mirror of ``vla_opts_t``."""
+    _fields_ = [("struct_size", ctypes.c_uint32), ("qkv_dtype", ctypes.c_int32),
+                ("u", ctypes.c_void_p), ("flags", ctypes.c_uint32), ("eps", ctypes.c_float),
+                ("z0", ctypes.c_void_p), ("zT", ctypes.c_void_p), ("status", ctypes.c_void_p),
+                ("kernel", ctypes.c_int32)]
+
+
+class VlaError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where, status_string(code), code))
+
+
+_lock = threading.Lock()
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def load_library():
+    """dlopen ``libvla.so`` (built in-tree by ``build.build()``).  Raises if it is absent."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            path = library_path()
+            if not os.path.exists(path):
+                raise RuntimeError(
+                    "CUDA library %s is missing: run paper_2605_11196_b200.build.build() "
+                    "(there is no fallback path)" % path)
+            lib = ctypes.CDLL(path)
+            vp, i, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+            lib.vla_forward.restype = i
+            lib.vla_forward.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp,
+                                        ctypes.POINTER(VlaOpts), vp]
+            lib.vla_forward_host.restype = i
+            lib.vla_forward_host.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp,
+                                             ctypes.POINTER(VlaOpts), vp, ctypes.c_size_t, vp]
+            lib.vla_host_workspace_bytes.restype = ctypes.c_size_t
+            lib.vla_host_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
+            lib.vla_query_support.restype = i
+            lib.vla_query_support.argtypes = [i, i, i, ctypes.c_uint32]
+            lib.vla_status_string.restype = ctypes.c_char_p
+            lib.vla_status_string.argtypes = [i]
+            lib.vla_version.restype = i
+            lib.vla_version.argtypes = []
+            _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load_library().vla_status_string(int(code)).decode()
+
+
+def vla_version() -> int:
+    return load_library().vla_version()
+
+
+def vla_query_support(d_k: int, d_v: int, qkv_dtype: int = VLA_F32, flags: int = 0) -> int:
+    return load_library().vla_query_support(d_k, d_v, qkv_dtype, flags)
+
+
+def vla_host_workspace_bytes(B, H, T, d_k, d_v, qkv_dtype=VLA_F32, has_u=False) -> int:
+    return load_library().vla_host_workspace_bytes(B, H, T, d_k, d_v, qkv_dtype, int(has_u))
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return VLA_F32
+    if t.dtype == torch.bfloat16:
+        return VLA_BF16
+    raise TypeError("q, k, v must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _chk(t, shape, dtype, name, cuda=True):
+    if t is None:
+        return
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError("%s: shape %s, expected %s" % (name, tuple(t.shape), tuple(shape)))
+    if t.dtype != dtype:
+        raise TypeError("%s: dtype %s, expected %s" % (name, t.dtype, dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if cuda != t.is_cuda:
+        raise ValueError("%s must be a %s tensor" % (name, "CUDA" if cuda else "CPU"))
+
+
+@dataclass
+class VlaResult:
+    out: torch.Tensor              # [B,H,T,d_v] fp32
+    S_T: torch.Tensor              # [B,H,d_v,d_k] fp32
+    A_T: torch.Tensor              # [B,H,d_k,d_k] fp32
+    z_T: torch.Tensor              # [B,H,d_k] fp32
+    status: Optional[torch.Tensor]  # device int32 scalar; read after synchronising
+
+
+def _make_opts(dt, u, flags, eps, z0, zT, status, kernel):
+    o = VlaOpts()
+    o.struct_size = ctypes.sizeof(VlaOpts)
+    o.qkv_dtype = dt
+    o.u = None if u is None else u.data_ptr()
+    o.flags = flags
+    o.eps = eps
+    o.z0 = None if z0 is None else z0.data_ptr()
+    o.zT = None if zT is None else zT.data_ptr()
+    o.status = None if status is None else status.data_ptr()
+    o.kernel = kernel
+    return o
+
+
+def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags: int = 0,
+                eps: float = 1e-4, out=None, S_T=None, A_T=None, z_T=None, status=None,
+                kernel: int = VLA_KERNEL_AUTO, stream: Optional[torch.cuda.Stream] = None,
+                want_status: bool = True) -> VlaResult:
+    """Enqueue the scan for CUDA tensors ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``.
+
+    Output tensors are allocated with torch unless passed in.  Nothing is synchronised.
+    """
+    lib = load_library()
+    if q.dim() != 4:
+        raise ValueError("q must be [B,H,T,d_k]")
+    B, H, T, dk = q.shape
+    dv = v.shape[-1]
+    dt = _dtype_code(q)
+    dev = q.device
+    _chk(q, (B, H, T, dk), q.dtype, "q"); _chk(k, (B, H, T, dk), q.dtype, "k")
+    _chk(v, (B, H, T, dv), q.dtype, "v"); _chk(u, (B, H, T, dk), q.dtype, "u")
+    f32 = torch.float32
+    _chk(S0, (B, H, dv, dk), f32, "S0"); _chk(A0, (B, H, dk, dk), f32, "A0")
+    _chk(z0, (B, H, dk), f32, "z0")
+    if out is None:
+        out = torch.empty((B, H, T, dv), dtype=f32, device=dev)
+    if S_T is None:
+        S_T = torch.empty((B, H, dv, dk), dtype=f32, device=dev)
+    if A_T is None:
+        A_T = torch.empty((B, H, dk, dk), dtype=f32, device=dev)
+    if z_T is None:
+        z_T = torch.empty((B, H, dk), dtype=f32, device=dev)
+    _chk(out, (B, H, T, dv), f32, "out"); _chk(S_T, (B, H, dv, dk), f32, "S_T")
+    _chk(A_T, (B, H, dk, dk), f32, "A_T"); _chk(z_T, (B, H, dk), f32, "z_T")
+    if status is None and want_status:
+        status = torch.zeros((), dtype=torch.int32, device=dev)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel)
+    with torch.cuda.device(dev):
+        rc = lib.vla_forward(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv,
+                             _ptr(S0), _ptr(A0), _ptr(out), _ptr(S_T), _ptr(A_T),
+                             ctypes.byref(opts), ctypes.c_void_p(st.cuda_stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_forward")
+    return VlaResult(out, S_T, A_T, z_T, status)
+
+
+def vla_forward_host(q, k, v, lam: float, workspace: torch.Tensor, *, u=None, S0=None, A0=None,
+                     z0=None, flags: int = 0, eps: float = 1e-4, out=None, S_T=None, A_T=None,
+                     z_T=None, status=None, kernel: int = VLA_KERNEL_AUTO,
+                     stream: Optional[torch.cuda.Stream] = None) -> VlaResult:
+    """The same for HOST tensors (pinned for asynchronous copies); ``workspace`` is a CUDA
+    uint8 tensor of at least ``vla_host_workspace_bytes(...)`` bytes.  Copies in, the scan
+    and copies out are enqueued on the stream; synchronise it before reading the results."""
+    lib = load_library()
+    B, H, T, dk = q.shape
+    dv = v.shape[-1]
+    dt = _dtype_code(q)
+    f32 = torch.float32
+    _chk(q, (B, H, T, dk), q.dtype, "q", cuda=False); _chk(k, (B, H, T, dk), q.dtype, "k", cuda=False)
+    _chk(v, (B, H, T, dv), q.dtype, "v", cuda=False); _chk(u, (B, H, T, dk), q.dtype, "u", cuda=False)
+    _chk(S0, (B, H, dv, dk), f32, "S0", cuda=False); _chk(A0, (B, H, dk, dk), f32, "A0", cuda=False)
+    _chk(z0, (B, H, dk), f32, "z0", cuda=False)
+    pin = torch.cuda.is_available()
+    mk = lambda shape: torch.empty(shape, dtype=f32, pin_memory=pin)
+    out = mk((B, H, T, dv)) if out is None else out
+    S_T = mk((B, H, dv, dk)) if S_T is None else S_T
+    A_T = mk((B, H, dk, dk)) if A_T is None else A_T
+    z_T = mk((B, H, dk)) if z_T is None else z_T
+    _chk(out, (B, H, T, dv), f32, "out", cuda=False); _chk(S_T, (B, H, dv, dk), f32, "S_T", cuda=False)
+    _chk(A_T, (B, H, dk, dk), f32, "A_T", cuda=False); _chk(z_T, (B, H, dk), f32, "z_T", cuda=False)
+    if not workspace.is_cuda or workspace.dtype != torch.uint8 or not workspace.is_contiguous():
+        raise ValueError("workspace must be a contiguous CUDA uint8 tensor")
+    dev = workspace.device
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel)
+    with torch.cuda.device(dev):
+        rc = lib.vla_forward_host(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv,
+                                  _ptr(S0), _ptr(A0), _ptr(out), _ptr(S_T), _ptr(A_T),
+                                  ctypes.byref(opts), _ptr(workspace), workspace.numel(),
+                                  ctypes.c_void_p(st.cuda_stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_forward_host")
+    return VlaResult(out, S_T, A_T, z_T, status)

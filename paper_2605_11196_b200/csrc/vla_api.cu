@@ -1,0 +1,209 @@
+// C ABI of the VLA forward scan (declared in include/vla.h): host-side validation,
+// kernel selection and launch.  No allocation, no synchronisation, no global state.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstring>
+
+#include "vla.h"
+#include "vla_common.cuh"
+#include "vla_scan_token.cuh"
+
+namespace {
+
+using vla::ScanParams;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Resolved {
+  vla_opts_t o;
+};
+
+int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
+  std::memset(r, 0, sizeof(*r));
+  r->struct_size = sizeof(vla_opts_t);
+  r->qkv_dtype = VLA_F32;
+  if (opts) {
+    if (opts->struct_size < offsetof(vla_opts_t, kernel) || opts->struct_size > sizeof(vla_opts_t))
+      return VLA_ERR_INVALID_ARG;
+    std::memcpy(r, opts, opts->struct_size);  // fields past the caller's struct stay 0
+    r->struct_size = sizeof(vla_opts_t);
+  }
+  if (!(r->eps > 0.0f)) r->eps = 1e-4f;
+  if (r->qkv_dtype != VLA_F32 && r->qkv_dtype != VLA_BF16) return VLA_ERR_INVALID_ARG;
+  if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_INVALID_ARG;
+  if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN) return VLA_ERR_INVALID_ARG;
+  return VLA_OK;
+}
+
+bool shape_supported(int d_k, int d_v) {
+  return d_k == d_v && (d_k == 16 || d_k == 32 || d_k == 64 || d_k == 128);
+}
+
+template <int D, typename TIn, bool HAS_U>
+int launch_token(const ScanParams& p, cudaStream_t st) {
+  using Cfg = vla::TokenCfg<D, TIn, HAS_U>;
+  auto kern = vla::vla_scan_token_kernel<D, TIn, HAS_U>;
+  // Idempotent; needed once per device and cheap enough to repeat (no global state kept).
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D>
+int launch_token_d(const ScanParams& p, int dtype, cudaStream_t st) {
+  const bool has_u = p.u != nullptr;
+  if (dtype == VLA_F32)
+    return has_u ? launch_token<D, float, true>(p, st) : launch_token<D, float, false>(p, st);
+  return has_u ? launch_token<D, uint16_t, true>(p, st) : launch_token<D, uint16_t, false>(p, st);
+}
+
+int launch(const ScanParams& p, int d, int dtype, int /*kernel*/, cudaStream_t st) {
+  switch (d) {
+    case 16: return launch_token_d<16>(p, dtype, st);
+    case 32: return launch_token_d<32>(p, dtype, st);
+    case 64: return launch_token_d<64>(p, dtype, st);
+    case 128: return launch_token_d<128>(p, dtype, st);
+    default: return VLA_ERR_UNSUPPORTED;
+  }
+}
+
+// Argument checks shared by the device- and host-pointer entry points.
+int check_common(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,
+                 int d_k, int d_v, const float* A0, const float* out) {
+  if (B < 0 || H < 0 || T < 0 || d_k <= 0 || d_v <= 0) return VLA_ERR_INVALID_ARG;
+  if (!shape_supported(d_k, d_v)) return VLA_ERR_UNSUPPORTED;
+  if (!A0 && !(lambda_ > 0.0f)) return VLA_ERR_INVALID_ARG;
+  const long long units = 1LL * B * H;
+  if (units > 0x7fffffffLL) return VLA_ERR_INVALID_ARG;
+  if (units > 0 && T > 0 && (!q || !k || !v || !out)) return VLA_ERR_INVALID_ARG;
+  return VLA_OK;
+}
+
+inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
+
+}  // namespace
+
+extern "C" {
+
+int vla_forward(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,
+                int d_k, int d_v, const float* S0, const float* A0, float* out, float* S_T,
+                float* A_T, const vla_opts_t* opts, void* stream) {
+  vla_opts_t o;
+  int rc = resolve_opts(opts, &o);
+  if (rc != VLA_OK) return rc;
+  rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, out);
+  if (rc != VLA_OK) return rc;
+  const void* ptrs[] = {q, k, v, o.u, S0, A0, out, S_T, A_T, o.z0, o.zT};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return VLA_ERR_ALIGNMENT;
+  if (o.status && (reinterpret_cast<uintptr_t>(o.status) & 3u)) return VLA_ERR_ALIGNMENT;
+  const int units = B * H;
+  if (units == 0) return VLA_OK;
+
+  ScanParams p;
+  p.q = q; p.k = k; p.v = v; p.u = o.u;
+  p.S0 = S0; p.A0 = A0; p.z0 = o.z0;
+  p.out = out; p.S_T = S_T; p.A_T = A_T; p.zT = o.zT;
+  p.status = o.status;
+  p.lambda = lambda_; p.eps = o.eps;
+  p.T = T; p.units = units; p.flags = o.flags;
+  return launch(p, d_k, o.qkv_dtype, o.kernel, static_cast<cudaStream_t>(stream));
+}
+
+size_t vla_host_workspace_bytes(int B, int H, int T, int d_k, int d_v, int qkv_dtype, int has_u) {
+  if (B < 0 || H < 0 || T < 0 || d_k <= 0 || d_v <= 0) return 0;
+  if (qkv_dtype != VLA_F32 && qkv_dtype != VLA_BF16) return 0;
+  const size_t es = qkv_dtype == VLA_F32 ? 4 : 2;
+  const size_t units = size_t(B) * size_t(H);
+  const size_t qk = round256(units * T * d_k * es), vv = round256(units * T * d_v * es);
+  const size_t ob = round256(units * T * d_v * 4);
+  const size_t Sb = round256(units * d_v * d_k * 4), Ab = round256(units * d_k * d_k * 4);
+  const size_t zb = round256(units * d_k * 4);
+  return qk * (has_u ? 3 : 2) + vv + ob + 2 * Sb + 2 * Ab + 2 * zb + 256;
+}
+
+int vla_forward_host(const void* q, const void* k, const void* v, float lambda_, int B, int H,
+                     int T, int d_k, int d_v, const float* S0, const float* A0, float* out,
+                     float* S_T, float* A_T, const vla_opts_t* opts, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+  vla_opts_t o;
+  int rc = resolve_opts(opts, &o);
+  if (rc != VLA_OK) return rc;
+  rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, out);
+  if (rc != VLA_OK) return rc;
+  const size_t need = vla_host_workspace_bytes(B, H, T, d_k, d_v, o.qkv_dtype, o.u != nullptr);
+  if (!workspace || workspace_bytes < need) return VLA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return VLA_ERR_ALIGNMENT;
+  const size_t units = size_t(B) * size_t(H);
+  if (units == 0) return VLA_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  const size_t es = o.qkv_dtype == VLA_F32 ? 4 : 2;
+  const size_t qk_b = units * T * d_k * es, v_b = units * T * d_v * es;
+  const size_t o_b = units * T * d_v * 4;
+  const size_t S_b = units * d_v * d_k * 4, A_b = units * d_k * d_k * 4, z_b = units * d_k * 4;
+  unsigned char* w = static_cast<unsigned char*>(workspace);
+  auto take = [&](size_t bytes) { void* r = w; w += round256(bytes); return r; };
+  void* dq = take(qk_b); void* dk = take(qk_b); void* dv = take(v_b);
+  void* du = o.u ? take(qk_b) : nullptr;
+  float* dout = static_cast<float*>(take(o_b));
+  float* dS0 = static_cast<float*>(take(S_b)); float* dST = static_cast<float*>(take(S_b));
+  float* dA0 = static_cast<float*>(take(A_b)); float* dAT = static_cast<float*>(take(A_b));
+  float* dz0 = static_cast<float*>(take(z_b)); float* dzT = static_cast<float*>(take(z_b));
+
+  bool bad = false;
+  auto h2d = [&](void* d, const void* h, size_t bytes) {
+    if (bytes && cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) bad = true;
+  };
+  auto d2h = [&](void* h, const void* d, size_t bytes) {
+    if (bytes && cudaMemcpyAsync(h, d, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) bad = true;
+  };
+  h2d(dq, q, qk_b); h2d(dk, k, qk_b); h2d(dv, v, v_b);
+  if (o.u) h2d(du, o.u, qk_b);
+  if (S0) h2d(dS0, S0, S_b);
+  if (A0) h2d(dA0, A0, A_b);
+  if (o.z0) h2d(dz0, o.z0, z_b);
+  if (bad) { cudaGetLastError(); return VLA_ERR_CUDA; }
+
+  vla_opts_t od = o;
+  od.u = du;
+  od.z0 = o.z0 ? dz0 : nullptr;
+  od.zT = o.zT ? dzT : nullptr;
+  rc = vla_forward(dq, dk, dv, lambda_, B, H, T, d_k, d_v, S0 ? dS0 : nullptr, A0 ? dA0 : nullptr,
+                   dout, S_T ? dST : nullptr, A_T ? dAT : nullptr, &od, stream);
+  if (rc != VLA_OK) return rc;
+  d2h(out, dout, o_b);
+  if (S_T) d2h(S_T, dST, S_b);
+  if (A_T) d2h(A_T, dAT, A_b);
+  if (o.zT) d2h(o.zT, dzT, z_b);
+  if (bad) { cudaGetLastError(); return VLA_ERR_CUDA; }
+  return VLA_OK;
+}
+
+int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags) {
+  if (qkv_dtype != VLA_F32 && qkv_dtype != VLA_BF16) return VLA_ERR_UNSUPPORTED;
+  if (flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_UNSUPPORTED;
+  return shape_supported(d_k, d_v) ? VLA_OK : VLA_ERR_UNSUPPORTED;
+}
+
+const char* vla_status_string(int status) {
+  switch (status) {
+    case VLA_OK: return "ok";
+    case VLA_ERR_INVALID_ARG: return "invalid argument";
+    case VLA_ERR_UNSUPPORTED: return "unsupported shape, dtype or flag (no kernel; there is no CPU fallback)";
+    case VLA_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case VLA_ERR_CUDA: return "CUDA runtime or launch error";
+    case VLA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case VLA_ERR_NONFINITE: return "non-finite delta or write-direction norm";
+    default: return "unknown status";
+  }
+}
+
+int vla_version(void) { return 100; }
+
+}  // extern "C"

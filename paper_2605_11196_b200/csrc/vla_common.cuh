@@ -1,0 +1,135 @@
+// Shared device-side pieces of the VLA scan kernels (sm_100a): launch parameters,
+// bounded mbarrier waits, 1-D bulk-async (TMA) copies, small math helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vla.h"
+
+namespace vla {
+
+struct ScanParams {
+  const void* q;       // [units, T, D]
+  const void* k;       // [units, T, D]
+  const void* v;       // [units, T, D]
+  const void* u;       // [units, T, D] or nullptr
+  const float* S0;     // [units, D, D] or nullptr
+  const float* A0;     // [units, D, D] or nullptr
+  const float* z0;     // [units, D] or nullptr
+  float* out;          // [units, T, D]
+  float* S_T;          // may be nullptr
+  float* A_T;          // may be nullptr
+  float* zT;           // may be nullptr
+  int* status;         // may be nullptr
+  float lambda;
+  float eps;
+  int T;
+  int units;
+  uint32_t flags;
+};
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(arrivals));
+}
+
+// Makes freshly initialised barriers visible to the async proxy (TMA).
+__device__ __forceinline__ void mbar_init_fence() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+               "r"(bytes)
+               : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n"
+      "  .reg .pred p;\n"
+      "  mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "  selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+
+// Every wait in these kernels is bounded: try_wait itself blocks for a
+// hardware-defined slice, so this many failed probes is on the order of a second.
+constexpr uint32_t kWaitProbeLimit = 1u << 22;
+
+// Returns false when the limit ran out (the caller reports VLA_ERR_DEVICE_TIMEOUT and
+// leaves through the common exit so that no thread is left at a CTA barrier).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kWaitProbeLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  return false;
+}
+
+// global -> shared bulk copy, completion counted in bytes on `bar`.
+// dst, src 16-byte aligned; bytes a multiple of 16.  No multicast.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes,
+                                          uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+          "r"(smem_u32(smem_dst)),
+      "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+
+// shared -> global bulk copy in the calling thread's bulk group.
+__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst),
+               "r"(smem_u32(smem_src)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {  // <= N groups still reading shared memory
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_all() {  // <= N groups not yet complete
+  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+// Orders generic-proxy writes to shared memory before a later bulk store reads them.
+__device__ __forceinline__ void fence_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// ---------------------------------------------------------------- math helpers
+// phi(x) = ELU(x) + 1 (Section 3.3): x + 1 for x > 0, exp(x) otherwise.
+__device__ __forceinline__ float phi_elu1(float x) { return x > 0.0f ? x + 1.0f : expf(x); }
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t bits16) {
+  return __uint_as_float(bits16 << 16);
+}
+
+// four consecutive elements of a shared-memory row, widened to fp32
+__device__ __forceinline__ float4 load4(const float* row, int c4) {
+  return reinterpret_cast<const float4*>(row)[c4];
+}
+__device__ __forceinline__ float4 load4(const uint16_t* row, int c4) {
+  uint2 r = reinterpret_cast<const uint2*>(row)[c4];
+  float4 f;
+  f.x = bf16_bits_to_f32(r.x & 0xffffu);
+  f.y = bf16_bits_to_f32(r.x >> 16);
+  f.z = bf16_bits_to_f32(r.y & 0xffffu);
+  f.w = bf16_bits_to_f32(r.y >> 16);
+  return f;
+}
+
+}  // namespace vla

@@ -1,0 +1,171 @@
+"""CUDA path vs the fp64 CPU oracle, element by element, through the C ABI (-m gpu)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2605_11196_b200 as vla
+from paper_2605_11196_b200 import workloads as W
+from parity_util import check_parity, rel_err, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+IDENT = vla.VLA_FLAG_IDENTITY_MAP
+
+
+def _small(d, T, dtype, units=(2, 3), seed=100, kind="normal"):
+    return W.Workload("small", units[0], units[1], d, T, dtype, seed, kind=kind)
+
+
+@pytest.mark.parametrize("d", [16, 32, 64, 128])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+@pytest.mark.parametrize("umode", ["khat", "unit", "unit_over_sqrt_d"])
+def test_small_shapes(d, dtype, flags, umode):
+    """Several chunks plus a ragged tail (T = 83 = 5*16 + 3), 6 units."""
+    w = _small(d, 83, dtype, seed=7 * d + len(umode))
+    q, k, v = W.make_inputs(w)
+    u = None
+    if umode != "khat":
+        u = W.make_u(w, 1.0 if umode == "unit" else d ** -0.5)
+    for lam in (1.0, 0.1):
+        check_parity(q, k, v, lam, 1e-4, u=u, flags=flags, label="%s d=%d lam=%g" % (umode, d, lam))
+
+
+@pytest.mark.parametrize("T", [0, 1, 2, 15, 16, 17, 31, 32, 33, 48, 49])
+@pytest.mark.parametrize("d", [16, 64])
+def test_ragged_and_degenerate_lengths(T, d):
+    w = _small(d, T, "f32", units=(1, 5), seed=T + d)
+    q, k, v = W.make_inputs(w)
+    g = torch.Generator().manual_seed(5)
+    S0 = torch.randn((1, 5, d, d), generator=g) * 0.1
+    z0 = torch.rand((1, 5, d), generator=g)
+    for flags in (0, IDENT):
+        check_parity(q, k, v, 0.5, 1e-4, S0=S0, z0=z0, flags=flags, label="T=%d" % T)
+
+
+def test_zero_units_and_status_strings():
+    dev = torch.device("cuda:0")
+    z = torch.zeros((0, 4, 8, 32), device=dev)
+    r = vla.vla_forward(z, z, z, 1.0)
+    assert r.out.shape == (0, 4, 8, 32)
+    assert "unsupported" in vla.status_string(vla.VLA_ERR_UNSUPPORTED)
+
+
+def test_state_carry_split_invariance():
+    """forward(T) == forward(T1) then forward(T - T1) with (S, A, zkey) carried (paper mode
+    carries the key sum as well)."""
+    w = _small(32, 100, "f32", seed=11)
+    q, k, v = W.make_inputs(w)
+    u = W.make_u(w)
+    for flags in (0, IDENT):
+        for uu in (None, u):
+            full = run_gpu(q, k, v, 0.1, u=uu, flags=flags)
+            ref = run_oracle(q, k, v, 0.1, u=uu, flags=flags)
+            for T1 in (16, 37, 64):
+                sl = lambda x, a, b: None if x is None else x[:, :, a:b].contiguous()
+                a = run_gpu(sl(q, 0, T1), sl(k, 0, T1), sl(v, 0, T1), 0.1, u=sl(uu, 0, T1), flags=flags)
+                b = run_gpu(sl(q, T1, 100), sl(k, T1, 100), sl(v, T1, 100), 0.1, u=sl(uu, T1, 100),
+                            S0=a.S_T, A0=a.A_T, z0=a.z_T, flags=flags)
+                cat = torch.cat([a.out, b.out], dim=2)
+                assert rel_err(cat, ref.out) <= 1e-4
+                assert rel_err(b.S_T, ref.S_T) <= 1e-4 and rel_err(b.A_T, ref.A_T) <= 1e-4
+                assert rel_err(b.z_T, ref.z_T) <= 1e-4
+                if T1 % 16 == 0:   # chunk-aligned split: the same instruction stream
+                    assert torch.equal(cat, full.out) and torch.equal(b.A_T, full.A_T)
+
+
+def test_in_place_state_and_canaries():
+    """S_T/A_T may alias S0/A0; nothing is written outside the output tensors."""
+    dev = torch.device("cuda:0")
+    w = _small(64, 40, "bf16", seed=13)
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    B, H, T, d = q.shape
+    g = torch.Generator().manual_seed(3)
+    S = (torch.randn((B, H, d, d), generator=g) * 0.1).to(dev)
+    Ah = torch.randn((B, H, d, d), generator=g) * 0.05
+    A = (Ah @ Ah.transpose(-1, -2) + torch.eye(d)).to(dev)
+    ref = run_oracle(q, k, v, 1.0, S0=S, A0=A)
+    pad = 1024
+    buf = torch.full((B * H * T * d + 2 * pad,), 12345.0, device=dev)
+    out = buf[pad:pad + B * H * T * d].view(B, H, T, d)
+    r = vla.vla_forward(q, k, v, 1.0, S0=S, A0=A, S_T=S, A_T=A, out=out)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    assert torch.all(buf[:pad] == 12345.0) and torch.all(buf[-pad:] == 12345.0)
+    assert rel_err(out, ref.out) <= 1e-4 and rel_err(S, ref.S_T) <= 1e-4 and rel_err(A, ref.A_T) <= 1e-4
+
+
+def test_bitwise_determinism():
+    w = _small(128, 200, "bf16", units=(3, 3), seed=17)
+    q, k, v = W.make_inputs(w)
+    a = run_gpu(q, k, v, 1.0)
+    b = run_gpu(q, k, v, 1.0)
+    assert torch.equal(a.out, b.out) and torch.equal(a.S_T, b.S_T) and torch.equal(a.A_T, b.A_T)
+
+
+def test_zero_key_is_a_no_op():
+    """A zero key (identity map) gives k_hat = 0, alpha = 0: no update, finite outputs."""
+    w = _small(32, 20, "f32", units=(1, 2), seed=19)
+    q, k, v = W.make_inputs(w)
+    k[:, :, 7] = 0
+    check_parity(q, k, v, 1.0, 1e-4, flags=IDENT)
+
+
+def test_nonfinite_inputs_are_reported():
+    dev = torch.device("cuda:0")
+    w = _small(32, 20, "f32", units=(1, 2), seed=23)
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    k[0, 1, 5, 3] = float("nan")
+    r = vla.vla_forward(q, k, v, 1.0, flags=vla.VLA_FLAG_CHECK_FINITE)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == vla.VLA_ERR_NONFINITE
+    assert torch.isfinite(r.out[0, 0]).all()        # the other unit is untouched by it
+
+
+def test_host_entry_point_matches_device_entry_point():
+    dev = torch.device("cuda:0")
+    w = _small(64, 70, "bf16", seed=29)
+    q, k, v = W.make_inputs(w)
+    u = W.make_u(w)
+    B, H, T, d = q.shape
+    g = torch.Generator().manual_seed(31)
+    S0 = torch.randn((B, H, d, d), generator=g) * 0.1
+    z0 = torch.rand((B, H, d), generator=g)
+    nbytes = vla.vla_host_workspace_bytes(B, H, T, d, d, vla.VLA_BF16, True)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    pin = lambda x: x.pin_memory()
+    rh = vla.vla_forward_host(pin(q), pin(k), pin(v), 1.0, ws, u=pin(u), S0=pin(S0), z0=pin(z0))
+    torch.cuda.synchronize()
+    rd = run_gpu(q, k, v, 1.0, u=u, S0=S0, z0=z0)
+    assert torch.equal(rh.out, rd.out.cpu()) and torch.equal(rh.S_T, rd.S_T.cpu())
+    assert torch.equal(rh.A_T, rd.A_T.cpu()) and torch.equal(rh.z_T, rd.z_T.cpu())
+
+
+# ---------------------------------------------------------------- the five workloads
+@pytest.mark.parametrize("name", ["tiny", "mid", "recall", "long"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_workload_full(name, flags):
+    """Whole workload, every unit, both readings of the feature map."""
+    w = W.WORKLOADS[name]
+    q, k, v = W.make_inputs(w)
+    errs, _, _ = check_parity(q, k, v, w.lam, w.tol, flags=flags, label=name)
+    print(name, flags, errs)
+
+
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_workload_throughput_sampled_units(flags):
+    """The full-size launch the benchmark times (512 units); the oracle recomputes a sample
+    of whole units (units are independent), compared element by element."""
+    w = W.WORKLOADS["throughput"]
+    dev = torch.device("cuda:0")
+    q, k, v = W.make_inputs(w)
+    r = vla.vla_forward(q.to(dev), k.to(dev), v.to(dev), w.lam, flags=flags)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    assert torch.isfinite(r.out).all()
+    for (b, h) in [(0, 0), (7, 3), (31, 15), (16, 8), (21, 0), (5, 11)]:
+        sl = lambda x: x[b:b + 1, h:h + 1].contiguous()
+        ref = run_oracle(sl(q), sl(k), sl(v), w.lam, flags=flags)
+        for name, got, want in (("o", r.out, ref.out), ("S_T", r.S_T, ref.S_T), ("A_T", r.A_T, ref.A_T)):
+            e = rel_err(got[b:b + 1, h:h + 1], want)
+            assert e <= w.tol, "unit (%d,%d) %s rel err %.3e" % (b, h, name, e)

@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the VLA forward scan on B200.
+
+A "step" is one pass of the whole hot path (stream in, prep, per-token Sherman-Morrison /
+residual update / readout, stream out, final states) over one batch of synthetic input.
+Default workload: "throughput" (B=32, H=16, d=128, T=8192, bf16 in, fp32 state) -- the
+largest of the five workloads, and the one that fills the GPU.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--all-workloads]
+  python bench.py --impl reference ...     # the fp64 CPU oracle, as it stands, on host cores
+
+For N > 1 launch with torch.distributed.run; every rank scans its own batch (weak scaling,
+no data-path collective).  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "vla_forward_tokens_per_s"
+UNIT = "tokens/s"
+
+# FP32 FMA peak: SMs x 128 lanes x 2 flop x clock.  Nominal at the maximum SM clock; the
+# achieved fraction is also reported at the clock sampled during the timed region.
+FP32_LANES_PER_SM = 128
+
+
+def alg_flops_per_token(d: int, has_u: bool = False) -> float:
+    """Algorithmic fp32 work per token (u = k_hat): A u (d^2 FMA), the symmetric rank-1
+    downdate (d(d+1)/2), S k_hat, S q_f and the S update (3 d^2); 2 flop per FMA."""
+    fma = d * d + d * (d + 1) / 2 + 3 * d * d + (d * d if has_u else 0)
+    return 2.0 * fma
+
+
+def alg_bytes_per_token(d: int, in_bytes: int, has_u: bool = False) -> float:
+    """q, k, v (and u) read once in their storage type, o written once in fp32."""
+    return (3 + (1 if has_u else 0)) * d * in_bytes + 4 * d
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        return float(pk["hbm_gbs"]), float(pk.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.idx = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [r for (ts, r) in self.rows if t0 <= ts <= t1 + 0.2] or [r for (_, r) in self.rows]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except Exception:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_arrays(q, k, v):
+    import oracle
+    if q.dtype == torch.bfloat16:
+        f = lambda x: x.contiguous().view(torch.int16).numpy().view(np.uint16)
+        return f(q), f(k), f(v), oracle.BF16
+    return q.contiguous().numpy(), k.contiguous().numpy(), v.contiguous().numpy(), oracle.F32
+
+
+def time_oracle(w, q, k, v, budget_units=None):
+    """The oracle as it stands on this machine's host cores, on a bounded sample of whole units
+    of the same workload (units are independent; tokens/s scales with units)."""
+    import oracle
+    cores = max(1, len(os.sched_getaffinity(0)))
+    # about 15 s of wall time: ~ 1 ns per fp64 multiply-add per core, 5 d^2 of them per token
+    per_unit_s = w.T * 5 * w.d * w.d * 1.0e-9
+    n_units = budget_units or int(max(1, min(w.units, round(15.0 * cores / max(per_unit_s, 1e-9)))))
+    n_units = max(min(n_units, w.units), min(cores, w.units))
+    qs = q.reshape(w.units, 1, w.T, w.d)[:n_units]
+    ks = k.reshape(w.units, 1, w.T, w.d)[:n_units]
+    vs = v.reshape(w.units, 1, w.T, w.d)[:n_units]
+    qa, ka, va, dt = oracle_arrays(qs, ks, vs)
+    threads = min(cores, n_units)
+    t0 = time.perf_counter()
+    oracle.forward(qa, ka, va, w.lam, in_dtype=dt, n_threads=threads)
+    dt_s = time.perf_counter() - t0
+    return {"value": n_units * w.T / dt_s, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "%d of %d units x T=%d tokens (whole units, first in batch order), fp64, %.1f s"
+                      % (n_units, w.units, w.T, dt_s)}, dt_s, n_units
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2605_11196_b200 import workloads as W
+    w = W.WORKLOADS[args.workload]
+    cores = max(1, len(os.sched_getaffinity(0)))
+    # a step = a bounded sample of whole units, sized for ~3 s of wall time per step
+    per_unit_s = w.T * 5 * w.d * w.d * 1.0e-9
+    n_units = int(max(1, min(w.units, round(3.0 * cores / per_unit_s))))
+    n_units = max(min(n_units, w.units), min(cores, w.units))
+    ws = W.scaled(w, B=1, H=n_units)
+    q, k, v = W.make_inputs(ws)
+    times = []
+    for it in range(args.warmup + args.steps):
+        _, dt_s, _ = time_oracle(ws, q, k, v, budget_units=n_units)
+        if it >= args.warmup:
+            times.append(dt_s)
+    total = sum(times)
+    val = args.steps * n_units * w.T / total
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic (seeded N(0,1), the workload's recipe)",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d, "d_v": w.d, "T": w.T,
+                       "in_dtype": w.dtype, "lambda": w.lam,
+                       "sample": "%d of %d units per step" % (n_units, w.units)},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": min(cores, n_units), "kind": "oracle",
+                             "sample": "%d of %d whole units x T=%d per step" % (n_units, w.units, w.T)},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def bench_one(vla, w, dev, q, k, v, steps, warmup, stream):
+    """Device-resident timing of `steps` launches; returns (seconds for all steps, per-launch ms list)."""
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    out = torch.empty((w.B, w.H, w.T, w.d), dtype=torch.float32, device=dev)
+    S_T = torch.empty((w.B, w.H, w.d, w.d), dtype=torch.float32, device=dev)
+    A_T = torch.empty_like(S_T)
+    z_T = torch.empty((w.B, w.H, w.d), dtype=torch.float32, device=dev)
+    status = torch.zeros((), dtype=torch.int32, device=dev)
+    call = lambda: vla.vla_forward(qd, kd, vd, w.lam, out=out, S_T=S_T, A_T=A_T, z_T=z_T,
+                                   status=status, stream=stream)
+    return (qd, kd, vd, out, S_T, A_T, z_T, status), call
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="throughput")
+    ap.add_argument("--all-workloads", action="store_true",
+                    help="also time the other four workloads (kernel only) into 'per_workload'")
+    ap.add_argument("--B", type=int, default=None, help="override the workload's batch (profiling cases)")
+    ap.add_argument("--H", type=int, default=None, help="override the workload's heads")
+    ap.add_argument("--T", type=int, default=None, help="override the workload's sequence length")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+
+    import paper_2605_11196_b200 as vla
+    from paper_2605_11196_b200 import workloads as W
+    vla.load_library()                        # raises if the CUDA library is missing
+    w = W.WORKLOADS[args.workload]
+    over = {n: getattr(args, n) for n in ("B", "H", "T") if getattr(args, n) is not None}
+    if over:
+        w = W.scaled(w, name=w.name + "-resized", **over)
+    hbm_peak, sm_max_mhz, peak_src = measured_peaks()
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+
+    q, k, v = W.make_inputs(w, rank=rank)
+    stream = torch.cuda.Stream(dev)
+    bufs, call = bench_one(vla, w, dev, q, k, v, args.steps, args.warmup, stream)
+    qd, kd, vd, out, S_T, A_T, z_T, status = bufs
+    in_bytes = 2 if w.dtype == "bf16" else 4
+    working_set = 3 * w.tokens * w.d * in_bytes + w.tokens * w.d * 4
+    l2_bytes = 126 * 2 ** 20
+    flush = None
+    if working_set <= 2 * l2_bytes:           # small workloads: flush L2 between timed steps
+        flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 0)):
+            call()
+    barrier()
+
+    # ---- kernel-only timed region: K steps, events on the launching stream
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    barrier()
+    t_wall0 = time.time()
+    with torch.cuda.stream(stream):
+        for (e0, e1) in ev:
+            if flush is not None:
+                flush.fill_(1)
+            e0.record(stream)
+            call()
+            e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    per_launch_ms = [e0.elapsed_time(e1) for (e0, e1) in ev]
+    total_s = sum(per_launch_ms) / 1e3
+    assert int(status.item()) == 0, vla.status_string(int(status.item()))
+    tt = torch.tensor([total_s], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    total_s_max = float(tt.item())
+    value = world * args.steps * w.tokens / total_s_max
+
+    # ---- end to end: pinned host buffers in, host buffers out, through vla_forward_host
+    e2e = None
+    if not args.no_e2e:
+        ws_bytes = vla.vla_host_workspace_bytes(w.B, w.H, w.T, w.d, w.d,
+                                                vla.VLA_BF16 if w.dtype == "bf16" else vla.VLA_F32)
+        wsbuf = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        qp, kp, vp = q.pin_memory(), k.pin_memory(), v.pin_memory()
+        outp = torch.empty((w.B, w.H, w.T, w.d), dtype=torch.float32).pin_memory()
+        STp = torch.empty((w.B, w.H, w.d, w.d), dtype=torch.float32).pin_memory()
+        ATp = torch.empty_like(STp).pin_memory()
+        zTp = torch.empty((w.B, w.H, w.d), dtype=torch.float32).pin_memory()
+        e2e_steps = max(1, min(args.steps, 3))
+        hcall = lambda: vla.vla_forward_host(qp, kp, vp, w.lam, wsbuf, out=outp, S_T=STp, A_T=ATp,
+                                             z_T=zTp, status=status, stream=stream)
+        with torch.cuda.stream(stream):
+            hcall()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(e2e_steps):
+                hcall()
+            e1.record(stream)
+        barrier()
+        t = torch.tensor([e0.elapsed_time(e1) / 1e3], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        h2d = 3 * w.tokens * w.d * in_bytes
+        d2h = w.tokens * w.d * 4 + w.units * (2 * w.d * w.d + w.d) * 4
+        e2e = {"value": world * e2e_steps * w.tokens / float(t.item()), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "api": "vla_forward_host (pinned host q,k,v in; out, S_T, A_T, z_T to pinned host)"}
+        del wsbuf
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the (single) scan kernel, from the live event timings
+    launch_ms = float(np.mean(per_launch_ms))
+    flops = alg_flops_per_token(w.d) * w.tokens
+    byts = alg_bytes_per_token(w.d, in_bytes) * w.tokens + w.units * (2 * w.d * w.d) * 4
+    fp32_peak_nominal = n_sm * FP32_LANES_PER_SM * 2 * sm_max_mhz * 1e6 / 1e12       # TFLOP/s
+    t_alu = flops / (fp32_peak_nominal * 1e12)
+    t_hbm = byts / (hbm_peak * 1e9)
+    bound = "alu" if t_alu >= t_hbm else "hbm"
+    achieved_tflops = flops / (launch_ms * 1e-3) / 1e12
+    achieved_gbs = byts / (launch_ms * 1e-3) / 1e9
+    roof = {"bound": bound, "kernel": "vla_scan_token_kernel<%d,%s>" % (w.d, w.dtype),
+            "achieved": achieved_tflops if bound == "alu" else achieved_gbs,
+            "peak": fp32_peak_nominal if bound == "alu" else hbm_peak,
+            "unit": "TFLOP/s" if bound == "alu" else "GB/s",
+            "frac": (achieved_tflops / fp32_peak_nominal) if bound == "alu" else achieved_gbs / hbm_peak,
+            "peak_source": ("fp32 FMA: %d SMs x 128 lanes x 2 x %.0f MHz (derived, nominal max clock)"
+                            % (n_sm, sm_max_mhz)) if bound == "alu" else "hbm_gbs of %s" % peak_src,
+            "traffic": None,
+            "alg_flops_per_token": alg_flops_per_token(w.d),
+            "alg_bytes_per_token": alg_bytes_per_token(w.d, in_bytes),
+            "hbm_achieved_gbs": achieved_gbs, "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
+            "hbm_frac": achieved_gbs / hbm_peak,
+            "launch_ms": launch_ms,
+            "unit_limited_frac_bound": min(w.units, n_sm) / n_sm}
+    if clocks and clocks.get("sm_mhz"):
+        roof["frac_at_sampled_clock"] = achieved_tflops / (fp32_peak_nominal * clocks["sm_mhz"] / sm_max_mhz)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total_s_max / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic (seeded N(0,1) q,k,v rounded to %s; each rank its own batch)" % w.dtype,
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d, "d_v": w.d, "T": w.T,
+                       "in_dtype": w.dtype, "state_dtype": "f32", "lambda": w.lam, "u": "k_hat",
+                       "mode": "Algorithm 1 (phi = ELU+1, normalised readout)",
+                       "parallelism": "dp%d over (batch, head) units, no collective" % world,
+                       "l2": ("inputs+outputs %.0f MB > L2" % (working_set / 1e6)) if flush is None
+                             else "L2 flushed between timed steps (256 MB write)"},
+            "ns_per_scan_step": 1e6 * launch_ms / w.T,
+            "roofline": roof, "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks}
+
+    if args.all_workloads:
+        per = {}
+        for name in W.ORDER:
+            if name == w.name:
+                continue
+            ww = W.WORKLOADS[name]
+            q2, k2, v2 = W.make_inputs(ww)
+            _, call2 = bench_one(vla, ww, dev, q2, k2, v2, 0, 0, stream)
+            fl = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+            ms = []
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    call2()
+                for _ in range(10):
+                    fl.fill_(1)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream); call2(); b.record(stream)
+                    ms.append((a, b))
+            torch.cuda.synchronize(dev)
+            ms = float(np.median([a.elapsed_time(b) for a, b in ms]))
+            ib = 2 if ww.dtype == "bf16" else 4
+            per[name] = {"ms": ms, "tokens_per_s": ww.tokens / (ms * 1e-3),
+                         "ns_per_scan_step": 1e6 * ms / ww.T,
+                         "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
+                         "hbm_frac": alg_bytes_per_token(ww.d, ib) * ww.tokens / (ms * 1e-3) / 1e9 / hbm_peak,
+                         "units": ww.units, "unit_limited_frac_bound": min(ww.units, n_sm) / n_sm}
+        line["per_workload"] = per
+
+    if not args.no_cpu_baseline:
+        cb, _, _ = time_oracle(w, q, k, v)
+        line["cpu_baseline"] = cb
+
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -276,8 +276,9 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
         es = ei * sc;
         oi = (ri + ei * (t2 * sc)) * inv_den[t];
         wvec = zbuf + b * D;
+        // fmaxf drops a NaN operand, so the raw sums are tested, not delta or sc
         if ((p.flags & VLA_FLAG_CHECK_FINITE) && tid == 0 && p.status &&
-            !(isfinite(delta) && isfinite(sc)))
+            !isfinite(t0 + t1 + t2))
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
       } else {
         // a = A_t k_hat = A_{t-1} k_hat - z (k_hat.z)/delta
@@ -302,7 +303,7 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
         oi = (ri + ei * (aq * sc)) * inv_den[t];
         wvec = abuf + b * D;
         if ((p.flags & VLA_FLAG_CHECK_FINITE) && tid == 0 && p.status &&
-            !(isfinite(delta) && isfinite(sc)))
+            !isfinite(t0 + t1 + aa + aq))
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
       }
       const float* zvec = zbuf + b * D;

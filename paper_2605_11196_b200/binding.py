@@ -21,7 +21,7 @@ VLA_ERR_INVALID_ARG, VLA_ERR_UNSUPPORTED, VLA_ERR_ALIGNMENT = -1, -2, -3
 VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE = -4, -5, -6
 VLA_F32, VLA_BF16 = 0, 1
 VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE = 1, 2
-VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN = 0, 1
+VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK = 0, 1, 2
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_host_workspace_bytes",
            "vla_query_support", "vla_status_string", "vla_version")

@@ -8,16 +8,13 @@
 #include "vla.h"
 #include "vla_common.cuh"
 #include "vla_scan_token.cuh"
+#include "vla_scan_chunk.cuh"
 
 namespace {
 
 using vla::ScanParams;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-struct Resolved {
-  vla_opts_t o;
-};
 
 int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
   std::memset(r, 0, sizeof(*r));
@@ -32,7 +29,8 @@ int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
   if (!(r->eps > 0.0f)) r->eps = 1e-4f;
   if (r->qkv_dtype != VLA_F32 && r->qkv_dtype != VLA_BF16) return VLA_ERR_INVALID_ARG;
   if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_INVALID_ARG;
-  if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN) return VLA_ERR_INVALID_ARG;
+  if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN && r->kernel != VLA_KERNEL_CHUNK)
+    return VLA_ERR_INVALID_ARG;
   return VLA_OK;
 }
 
@@ -62,7 +60,40 @@ int launch_token_d(const ScanParams& p, int dtype, cudaStream_t st) {
   return has_u ? launch_token<D, uint16_t, true>(p, st) : launch_token<D, uint16_t, false>(p, st);
 }
 
-int launch(const ScanParams& p, int d, int dtype, int /*kernel*/, cudaStream_t st) {
+template <int D, typename TIn>
+int launch_chunk(const ScanParams& p, cudaStream_t st) {
+  using Cfg = vla::ChunkCfg<D, TIn>;
+  auto kern = vla::vla_scan_chunk_kernel<D, TIn>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D>
+int launch_chunk_d(const ScanParams& p, int dtype, cudaStream_t st) {
+  return dtype == VLA_F32 ? launch_chunk<D, float>(p, st) : launch_chunk<D, uint16_t>(p, st);
+}
+
+// The chunk kernel covers u = k_hat and d in {32, 64, 128}; everything else runs on the
+// token kernel.  Both are CUDA paths; there is no host fallback.
+bool chunk_covers(const ScanParams& p, int d) { return p.u == nullptr && d >= 32; }
+
+int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
+  bool chunk = chunk_covers(p, d);
+  if (kernel == VLA_KERNEL_CHUNK && !chunk) return VLA_ERR_UNSUPPORTED;
+  if (kernel == VLA_KERNEL_TOKEN) chunk = false;
+  if (chunk) {
+    switch (d) {
+      case 32: return launch_chunk_d<32>(p, dtype, st);
+      case 64: return launch_chunk_d<64>(p, dtype, st);
+      case 128: return launch_chunk_d<128>(p, dtype, st);
+      default: return VLA_ERR_UNSUPPORTED;
+    }
+  }
   switch (d) {
     case 16: return launch_token_d<16>(p, dtype, st);
     case 32: return launch_token_d<32>(p, dtype, st);

@@ -16,23 +16,47 @@ def _small(d, T, dtype, units=(2, 3), seed=100, kind="normal"):
     return W.Workload("small", units[0], units[1], d, T, dtype, seed, kind=kind)
 
 
+KERNELS = {"token": vla.VLA_KERNEL_TOKEN, "chunk": vla.VLA_KERNEL_CHUNK}
+
+
+def _chunk_covers(d, umode="khat"):
+    return d >= 32 and umode == "khat"
+
+
+@pytest.mark.parametrize("kernel", ["token", "chunk"])
 @pytest.mark.parametrize("d", [16, 32, 64, 128])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("flags", [0, IDENT])
 @pytest.mark.parametrize("umode", ["khat", "unit", "unit_over_sqrt_d"])
-def test_small_shapes(d, dtype, flags, umode):
-    """Several chunks plus a ragged tail (T = 83 = 5*16 + 3), 6 units."""
+def test_small_shapes(kernel, d, dtype, flags, umode):
+    """Several chunks plus a ragged tail (T = 83 = 5*16 + 3), 6 units, both kernels."""
+    if kernel == "chunk" and not _chunk_covers(d, umode):
+        pytest.skip("the chunk kernel covers u = k_hat, d >= 32")
     w = _small(d, 83, dtype, seed=7 * d + len(umode))
     q, k, v = W.make_inputs(w)
     u = None
     if umode != "khat":
         u = W.make_u(w, 1.0 if umode == "unit" else d ** -0.5)
     for lam in (1.0, 0.1):
-        check_parity(q, k, v, lam, 1e-4, u=u, flags=flags, label="%s d=%d lam=%g" % (umode, d, lam))
+        check_parity(q, k, v, lam, 1e-4, u=u, flags=flags, kernel=KERNELS[kernel],
+                     label="%s %s d=%d lam=%g" % (kernel, umode, d, lam))
 
 
-@pytest.mark.parametrize("T", [0, 1, 2, 15, 16, 17, 31, 32, 33, 48, 49])
-@pytest.mark.parametrize("d", [16, 64])
+def test_forced_chunk_kernel_rejects_what_it_does_not_cover():
+    dev = torch.device("cuda:0")
+    w = _small(16, 8, "f32")
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    with pytest.raises(vla.VlaError) as ei:
+        vla.vla_forward(q, k, v, 1.0, kernel=vla.VLA_KERNEL_CHUNK)
+    assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+    w = _small(64, 8, "f32")
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    with pytest.raises(vla.VlaError):
+        vla.vla_forward(q, k, v, 1.0, u=W.make_u(w).to(dev), kernel=vla.VLA_KERNEL_CHUNK)
+
+
+@pytest.mark.parametrize("T", [0, 1, 2, 15, 16, 17, 31, 32, 33, 48, 49, 63, 64, 65, 97])
+@pytest.mark.parametrize("d", [16, 32, 64, 128])
 def test_ragged_and_degenerate_lengths(T, d):
     w = _small(d, T, "f32", units=(1, 5), seed=T + d)
     q, k, v = W.make_inputs(w)
@@ -40,7 +64,10 @@ def test_ragged_and_degenerate_lengths(T, d):
     S0 = torch.randn((1, 5, d, d), generator=g) * 0.1
     z0 = torch.rand((1, 5, d), generator=g)
     for flags in (0, IDENT):
-        check_parity(q, k, v, 0.5, 1e-4, S0=S0, z0=z0, flags=flags, label="T=%d" % T)
+        for kern in (vla.VLA_KERNEL_TOKEN, vla.VLA_KERNEL_CHUNK):
+            if kern == vla.VLA_KERNEL_CHUNK and not _chunk_covers(d):
+                continue
+            check_parity(q, k, v, 0.5, 1e-4, S0=S0, z0=z0, flags=flags, kernel=kern, label="T=%d" % T)
 
 
 def test_zero_units_and_status_strings():
@@ -108,7 +135,8 @@ def test_zero_key_is_a_no_op():
     w = _small(32, 20, "f32", units=(1, 2), seed=19)
     q, k, v = W.make_inputs(w)
     k[:, :, 7] = 0
-    check_parity(q, k, v, 1.0, 1e-4, flags=IDENT)
+    for kern in KERNELS.values():
+        check_parity(q, k, v, 1.0, 1e-4, flags=IDENT, kernel=kern)
 
 
 def test_nonfinite_inputs_are_reported():
@@ -116,10 +144,11 @@ def test_nonfinite_inputs_are_reported():
     w = _small(32, 20, "f32", units=(1, 2), seed=23)
     q, k, v = [x.to(dev) for x in W.make_inputs(w)]
     k[0, 1, 5, 3] = float("nan")
-    r = vla.vla_forward(q, k, v, 1.0, flags=vla.VLA_FLAG_CHECK_FINITE)
-    torch.cuda.synchronize()
-    assert int(r.status.item()) == vla.VLA_ERR_NONFINITE
-    assert torch.isfinite(r.out[0, 0]).all()        # the other unit is untouched by it
+    for kern in KERNELS.values():
+        r = vla.vla_forward(q, k, v, 1.0, flags=vla.VLA_FLAG_CHECK_FINITE, kernel=kern)
+        torch.cuda.synchronize()
+        assert int(r.status.item()) == vla.VLA_ERR_NONFINITE
+        assert torch.isfinite(r.out[0, 0]).all()        # the other unit is untouched by it
 
 
 def test_host_entry_point_matches_device_entry_point():

@@ -27,6 +27,9 @@ struct ScanParams {
   int T;
   int units;
   uint32_t flags;
+#ifdef VLA_SECTION_TIMERS
+  long long* dbg;      // debug builds only: per-section clock64 totals of unit 0
+#endif
 };
 
 // ---------------------------------------------------------------- PTX helpers

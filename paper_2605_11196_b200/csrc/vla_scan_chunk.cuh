@@ -240,6 +240,15 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   const int ptok0 = g / TOK_LANES;  // prep: first token of this thread (then +4, +8, +12)
   const int pc4 = g % TOK_LANES;    // prep: float4 column group
 
+#ifdef VLA_SECTION_TIMERS
+  long long tsec[12];
+  for (int i = 0; i < 12; ++i) tsec[i] = 0;
+  long long tlast = clock64();
+#define VLA_MARK(i) { long long now_ = clock64(); tsec[i] += now_ - tlast; tlast = now_; }
+#else
+#define VLA_MARK(i)
+#endif
+
   if (is_A) {
     // =====================================================================  group A
     for (int c = 0; c < nchunks; ++c) {
@@ -247,6 +256,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       const int n = min(C, T - c * C);
       const int slot = c % RING;
       wait(&full[s], (c / NSTAGE) & 1);
+      VLA_MARK(0)
 
       // ---- prep: k_hat rows of this chunk (zero rows past the end of the sequence)
       {
@@ -273,6 +283,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         }
       }
       group_bar(1, NG);
+      VLA_MARK(1)
       if (g == 0) mbar_arrive(&empty[s]);
 
       // ---- Z0 = A K^T: per token one pass over the tile, reduce-scatter over the row block
@@ -297,6 +308,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         Z0s[t * D + g] = reduce_scatter<LPR>(v, cg);
       }
       group_bar(1, NG);
+      VLA_MARK(2)
 
       // ---- W = K Z0 (C x C), 4x4 output tiles, D/16 threads per tile over the d index
       {
@@ -338,6 +350,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         }
       }
       group_bar(1, NG);
+      VLA_MARK(3)
 
       // ---- warp 0: I + W = L diag(delta) L^T, then T1 = L^-T (Z = Z0 T1)
       if (gw == 0) {
@@ -383,9 +396,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         }
       }
       group_bar(1, NG);
+      VLA_MARK(4)
 
       // the ring slot must have been released by group S (chunk c - RING)
       if (c >= RING) wait(&ring_empty[slot], ((c / RING) + 1) & 1);
+      VLA_MARK(5)
 
       // ---- Z = Z0 T1 (row g), published as Zs; ZD = Z / delta; partial ||z_t||^2
       {
@@ -418,6 +433,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         if ((lane & 1) == 0) N2p[gw * C + (lane >> 1)] = tot;
       }
       group_bar(1, NG);
+      VLA_MARK(6)
 
       // ---- warp 1 (or 0 when the group has one warp): sc, Gu, T2' = (I + Gu)^-1 diag(sc)
       if (gw == (NWG > 1 ? 1 : 0)) {
@@ -454,6 +470,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         if (lane == 0) mbar_arrive(&ring_full[slot]);
       }
 
+      VLA_MARK(7)
       // ---- A <- A - Z diag(1/delta) Z^T
       {
         const float* Zs = ringZ[slot];
@@ -479,6 +496,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         }
       }
       group_bar(1, NG);  // ZDs, Ws, N2p may be rewritten by the next chunk
+      VLA_MARK(8)
     }
     // final A
     if (p.A_T) {
@@ -502,6 +520,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       const int n = min(C, T - c * C);
       const int slot = c % RING;
       wait(&full[s], (c / NSTAGE) & 1);
+      VLA_MARK(0)
       if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
 
       // ---- prep: k_hat, ||phi(k)||, q_f, v (zero rows past the end of the sequence)
@@ -540,6 +559,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         }
       }
       group_bar(2, NG);
+      VLA_MARK(1)
       if (g == 0) {
         mbar_arrive(&empty[s]);
         if (c + NSTAGE < nchunks) {  // refill the stage once group A has left it too
@@ -591,9 +611,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 
       // ---- wait for group A's Z and T2' of this chunk
       wait(&ring_full[slot], (c / RING) & 1);
+      VLA_MARK(2)
       const float* Zs = ringZ[slot];
       const float* T2p = ringT2[slot];
       group_bar(2, NG);  // KhS/QfS/VS/R0s/denp complete for every row
+      VLA_MARK(3)
 
       // ---- H'[s][t] = z_s . q_t (C x C), same tiling as W; and the denominators
       {
@@ -640,6 +662,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         }
       }
       group_bar(2, NG);
+      VLA_MARK(4)
 
       // ---- row g: e'_t = sum_{s<=t} b_s T2'[s][t];  o_t = (r0_t + sum_{s<=t} e'_s H'[s][t]) / den_t
       {
@@ -679,6 +702,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       }
       fence_async_smem();
       group_bar(2, NG);
+      VLA_MARK(5)
       if (g == 0) {
         bulk_store(gout + size_t(c) * C * D, ostage + size_t(c & 1) * C * D,
                    uint32_t(n) * D * sizeof(float));
@@ -707,6 +731,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         }
       }
       group_bar(2, NG);
+      VLA_MARK(6)
       if (g == 0) mbar_arrive(&ring_empty[slot]);
     }
     // final S and key sum
@@ -723,6 +748,12 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     if (p.zT) p.zT[size_t(unit) * D + g] = zk;
     if (g == 0) bulk_wait_all<0>();
   }
+#ifdef VLA_SECTION_TIMERS
+  if (p.dbg && unit == 0 && (g == 0 || g == 32)) {
+    long long* d = p.dbg + ((is_A ? 0 : 2) + (g == 32 ? 1 : 0)) * 12;
+    for (int i = 0; i < 12; ++i) d[i] = tsec[i];
+  }
+#endif
 }
 
 }  // namespace vla

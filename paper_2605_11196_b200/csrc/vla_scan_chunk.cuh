@@ -10,18 +10,20 @@
 // A, S at the chunk start (Eqs. "sm", "s-update", "output"):
 //
 //   Z0 = A K^T                          W = K Z0 = K A K^T
-//   I + W = L diag(delta) L^T           delta_t is Eq. "sm"'s 1 + u.z, L[t,s] = (z_s.k_t)/delta_s
-//   Z  = Z0 L^-T                        column t is z_t = A_{t-1} k_hat_t
+//   I + W = L diag(delta) L^T           delta_t is Eq. "sm"'s 1 + u.z;  L[t,s] = (z_s.k_t)/delta_s
+//   Z L^T = Z0                          column t is z_t = A_{t-1} k_hat_t (forward substitution)
 //   alpha_t = sc_t z_t,  sc_t = (1/delta_t) / max(||z_t||/delta_t, eps)      (A_t k_hat_t = z_t/delta_t)
 //   A <- A - Z diag(1/delta) Z^T        (Woodbury form of 16 Sherman-Morrison steps)
-//   B  = V^T - S K^T                    E = B (I + Gu)^-1,  Gu[s,t] = alpha_s.k_hat_t (s < t)
-//   E' = E diag(sc) = B T2'             O[:,t] = (S q_t + sum_{s<=t} e'_s (z_s.q_t)) / den_t
+//   B  = V^T - S K^T                    e_t = b_t - sum_{s<t} Gu[s,t] e_s,  Gu[s,t] = alpha_s.k_hat_t
+//   e'_t = sc_t e_t                     o_t = (S q_t + sum_{s<=t} e'_s (z_s.q_t)) / den_t
 //   S <- S + E' Z^T
 //
-// Group A runs ahead of group S; Z and T2' travel through a two-slot shared-memory ring
-// guarded by mbarriers.  q/k/v arrive through a ring of 1-D bulk-async (TMA) copies; each
-// group widens and normalises what it needs.  Every mbarrier wait is bounded: if one runs
-// out the CTA records VLA_ERR_DEVICE_TIMEOUT, stops waiting and runs to its end.
+// Group A runs ahead of group S.  It owns the input stream: q/k/v arrive through a ring of
+// 1-D bulk-async (TMA) copies, and group A widens them (phi, k_hat, ||phi(k)||) into a
+// three-slot fp32 ring one chunk ahead, overlapped with the LDL^T factorisation.  Z, Gu, sc
+// and the small matrix z_s.q_t travel to group S through a two-slot ring.  Both rings are
+// guarded by mbarriers, and every mbarrier wait is bounded: if one runs out the CTA records
+// VLA_ERR_DEVICE_TIMEOUT, stops waiting and runs to its end.
 #pragma once
 
 #include "vla_common.cuh"
@@ -46,6 +48,29 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// Fast elementwise helpers of the prep pass (relative error ~1e-6, far inside the parity bound).
+// Branch-free: both sides are evaluated and selected, so a warp never diverges here.
+__device__ __forceinline__ float phi_fast(float x) {
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fminf(x, 0.0f) * 1.4426950408889634f));
+  return x > 0.0f ? x + 1.0f : e;
+}
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float r;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float r;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+// 1/x to within an ulp or so: hardware estimate plus one Newton step
+__device__ __forceinline__ float rcp_nr(float x) {
+  const float r = rcp_approx(x);
+  return fmaf(r, fmaf(-x, r, 1.0f), r);
+}
+
 template <int D>
 struct ChunkTile {
   static constexpr int TW = (D >= 64) ? 16 : 8;  // state columns per thread
@@ -62,39 +87,40 @@ struct ChunkCfg {
   static constexpr int NG = D;                   // threads per warp group
   static constexpr int NT = 2 * D;               // threads per CTA
   static constexpr int NWG = D / 32;             // warps per group
-  static constexpr int NSTAGE = sizeof(TIn) == 2 ? 4 : 3;
-  static constexpr int RING = 2;
-  static constexpr int TOK_LANES = D / 4;        // prep: threads per token
-  static constexpr int TOK_PER_PASS = NG / TOK_LANES;  // = 4
+  static constexpr int NSTAGE = sizeof(TIn) == 2 ? 4 : 2;  // raw q/k/v chunks in flight
+  static constexpr int RING = 2;                 // Z / Gu / HT / sc slots (group A -> group S)
+  static constexpr int KRING = 3;                // widened k_hat / q_f / v / ||phi(k)|| slots
   static constexpr int CP = C + 4;               // padded row of the small C x C matrices
 
   // shared memory layout (floats unless noted)
   static constexpr size_t raw_bytes = size_t(NSTAGE) * 3 * C * D * sizeof(TIn);
-  static constexpr size_t slot_floats = size_t(C) * D + C * CP;       // Zs, T2p
-  static constexpr size_t a_floats = size_t(3) * C * D + 2 * C * CP + NWG * C + 2 * C;
-  //   KhA, Z0s, ZDs | Ws, T1s | N2p | delta, inv_delta
-  static constexpr size_t s_floats = size_t(5) * C * D + 2 * C * D + C * CP + NWG * C + 2 * C;
-  //   KhS, QfS, VS(B), R0s, Eps | ostage[2] | Hs | denp | nrm, inv_den
+  static constexpr size_t kslot_floats = size_t(3) * C * D + C;             // Kh, Qf, Vf, nrm
+  static constexpr size_t slot_floats = size_t(C) * D + 2 * C * CP + C;     // Zs, GuT, HT, sc
+  static constexpr size_t a_floats = size_t(2) * C * D + 2 * C * CP + NWG * C + 2 * C;
+  //   Z0s, ZDs | Ws, Ls | N2p | delta, inv_delta
+  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + NWG * C + C;
+  //   VS(B), R0s, Eps | ostage[2] | denp | inv_den
   static constexpr size_t smem_bytes = raw_bytes +
-      (RING * slot_floats + a_floats + s_floats) * sizeof(float) +
-      (2 * NSTAGE + 2 * RING) * sizeof(uint64_t) + 16 + 128;
+      (KRING * kslot_floats + RING * slot_floats + a_floats + s_floats) * sizeof(float) +
+      (NSTAGE + 2 * RING) * sizeof(uint64_t) + 16 + 128;
 };
 
-// Reduce-scatter of N = LPR values over LPR consecutive lanes: on return v[0] is the sum,
-// over those lanes, of the element whose index equals the lane's position in the group.
-template <int LPR>
-__device__ __forceinline__ float reduce_scatter(float (&v)[LPR], int cg) {
+// Reduce-scatter of NTOK x LPR values over LPR consecutive lanes: on return v[k][0] is the
+// sum, over those lanes, of v[k][position of this lane in the group].
+template <int LPR, int NTOK>
+__device__ __forceinline__ void reduce_scatter(float (&v)[NTOK][LPR], int cg) {
 #pragma unroll
   for (int off = LPR / 2; off >= 1; off >>= 1) {
     const bool up = (cg & off) != 0;
 #pragma unroll
-    for (int i = 0; i < off; ++i) {
-      const float send = up ? v[i] : v[i + off];
-      const float keep = up ? v[i + off] : v[i];
-      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-    }
+    for (int k = 0; k < NTOK; ++k)
+#pragma unroll
+      for (int i = 0; i < off; ++i) {
+        const float send = up ? v[k][i] : v[k][i + off];
+        const float keep = up ? v[k][i + off] : v[k][i];
+        v[k][i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+      }
   }
-  return v[0];
 }
 
 // Reduce-scatter of 16 values over a full warp: lanes 2t and 2t+1 end with the sum of v[t].
@@ -111,7 +137,128 @@ __device__ __forceinline__ float warp_reduce_scatter16(float (&v)[16], int lane)
     }
   }
   v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
-  return v[0];  // token index = lane >> 1, with bits taken from lane bits 4..1
+  return v[0];  // token index = lane >> 1
+}
+
+// For every token t of the chunk: sink(t, row g of (state tile) . op[t]).  Two tokens per
+// pass so that the shuffle rounds of the reduce-scatter are paid once per pair, and the
+// reduce-scatter of one pair is issued alongside the FMAs of the next (software pipeline).
+template <int TR, int TW, int LPR, int D, int C, typename Sink>
+__device__ __forceinline__ void tile_matvec_chunk(const float2 (&st)[TR][TW / 2], const float* op,
+                                                  int cg, Sink sink) {
+  constexpr int NV = TW / 4;
+  // partial row sums of tokens t, t+1 over this thread's columns, folded to one float per row
+  auto pair_partial = [&](int t, float (&v)[2][LPR]) {
+    float2 acc[2][TR];
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+#pragma unroll
+      for (int r = 0; r < TR; ++r) acc[k][r] = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int m = 0; m < NV; ++m) {
+      const float4 a4 = reinterpret_cast<const float4*>(op + t * D)[m * LPR + cg];
+      const float4 b4 = reinterpret_cast<const float4*>(op + (t + 1) * D)[m * LPR + cg];
+      const float2 a01 = make_float2(a4.x, a4.y), a23 = make_float2(a4.z, a4.w);
+      const float2 b01 = make_float2(b4.x, b4.y), b23 = make_float2(b4.z, b4.w);
+#pragma unroll
+      for (int r = 0; r < TR; ++r) {
+        acc[0][r] = ffma2(st[r][2 * m], a01, acc[0][r]);
+        acc[1][r] = ffma2(st[r][2 * m], b01, acc[1][r]);
+        acc[0][r] = ffma2(st[r][2 * m + 1], a23, acc[0][r]);
+        acc[1][r] = ffma2(st[r][2 * m + 1], b23, acc[1][r]);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+#pragma unroll
+      for (int r = 0; r < TR; ++r) v[k][r] = acc[k][r].x + acc[k][r].y;
+  };
+  float v[2][LPR];
+  pair_partial(0, v);
+#pragma unroll 1
+  for (int t = 2; t < C; t += 2) {
+    float vn[2][LPR];
+    pair_partial(t, vn);          // independent of the shuffles below: issued together
+    reduce_scatter<LPR, 2>(v, cg);
+    sink(t - 2, v[0][0]);
+    sink(t - 1, v[1][0]);
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+#pragma unroll
+      for (int r = 0; r < LPR; ++r) v[k][r] = vn[k][r];
+  }
+  reduce_scatter<LPR, 2>(v, cg);
+  sink(C - 2, v[0][0]);
+  sink(C - 1, v[1][0]);
+}
+
+// tile += sum_s coef[s][rows of the tile] (x) vec[s][cols of the tile]   (rank-16 update)
+template <int TR, int TW, int LPR, int D, int C, bool NEGATE>
+__device__ __forceinline__ void tile_rank_update(float2 (&st)[TR][TW / 2], const float* coef,
+                                                 const float* vec, int rb, int cg) {
+  constexpr int NV = TW / 4;
+#pragma unroll 2
+  for (int s2 = 0; s2 < C; ++s2) {
+    float cf[TR];
+#pragma unroll
+    for (int r4 = 0; r4 < TR / 4; ++r4) {
+      const float4 x = reinterpret_cast<const float4*>(coef + s2 * D + rb * TR)[r4];
+      cf[4 * r4 + 0] = NEGATE ? -x.x : x.x; cf[4 * r4 + 1] = NEGATE ? -x.y : x.y;
+      cf[4 * r4 + 2] = NEGATE ? -x.z : x.z; cf[4 * r4 + 3] = NEGATE ? -x.w : x.w;
+    }
+#pragma unroll
+    for (int m = 0; m < NV; ++m) {
+      const float4 z4 = reinterpret_cast<const float4*>(vec + s2 * D)[m * LPR + cg];
+      const float2 z01 = make_float2(z4.x, z4.y), z23 = make_float2(z4.z, z4.w);
+#pragma unroll
+      for (int r = 0; r < TR; ++r) {
+        const float2 cc = make_float2(cf[r], cf[r]);
+        st[r][2 * m] = ffma2(cc, z01, st[r][2 * m]);
+        st[r][2 * m + 1] = ffma2(cc, z23, st[r][2 * m + 1]);
+      }
+    }
+  }
+}
+
+// G[i][j] = X[i] . Y[j] for two sets of C = 16 row vectors of length D (row stride D): 4x4
+// output tiles, NG/16 threads per tile splitting the D index; result rows have stride CP.
+template <int D, int NG, int CP>
+__device__ __forceinline__ void gram16(const float* X, const float* Y, float* G, int g) {
+  constexpr int P = NG / 16;
+  const int tile = g / P, part = g % P;
+  const int i0 = (tile >> 2) * 4, j0 = (tile & 3) * 4;
+  float w[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) w[i] = 0.f;
+#pragma unroll
+  for (int step = 0; step < D / (4 * P); ++step) {
+    const int f = step * P + part;
+    float4 a[4], b[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      a[i] = reinterpret_cast<const float4*>(X + (i0 + i) * D)[f];
+      b[i] = reinterpret_cast<const float4*>(Y + (j0 + i) * D)[f];
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        w[4 * i + j] = fmaf(a[i].x, b[j].x, w[4 * i + j]);
+        w[4 * i + j] = fmaf(a[i].y, b[j].y, w[4 * i + j]);
+        w[4 * i + j] = fmaf(a[i].z, b[j].z, w[4 * i + j]);
+        w[4 * i + j] = fmaf(a[i].w, b[j].w, w[4 * i + j]);
+      }
+  }
+#pragma unroll
+  for (int off = P / 2; off >= 1; off >>= 1)
+#pragma unroll
+    for (int i = 0; i < 16; ++i) w[i] += __shfl_xor_sync(0xffffffffu, w[i], off);
+  if (part == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      *reinterpret_cast<float4*>(G + (i0 + i) * CP + j0) =
+          make_float4(w[4 * i + 0], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+  }
 }
 
 template <int D, typename TIn>
@@ -119,47 +266,35 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   using Cfg = ChunkCfg<D, TIn>;
   constexpr int C = Cfg::C, TW = Cfg::TW, TR = Cfg::TR, LPR = Cfg::LPR, NV = Cfg::NV;
   constexpr int NG = Cfg::NG, NWG = Cfg::NWG, NSTAGE = Cfg::NSTAGE, RING = Cfg::RING;
-  constexpr int TOK_LANES = Cfg::TOK_LANES, TOK_PER_PASS = Cfg::TOK_PER_PASS, CP = Cfg::CP;
+  constexpr int KRING = Cfg::KRING, CP = Cfg::CP;
   static_assert(TR == LPR, "row ownership after the reduce-scatter needs TR == D/TW");
   static_assert(C == 16, "the small-matrix code is written for 16-token chunks");
 
   extern __shared__ __align__(128) unsigned char smem[];
   TIn* raw = reinterpret_cast<TIn*>(smem);
   float* fbase = reinterpret_cast<float*>(smem + Cfg::raw_bytes);
-  // ring slots
-  float* ringZ[RING];
-  float* ringT2[RING];
-#pragma unroll
-  for (int r = 0; r < RING; ++r) {
-    ringZ[r] = fbase + size_t(r) * Cfg::slot_floats;
-    ringT2[r] = ringZ[r] + C * D;
-  }
-  float* abase = fbase + RING * Cfg::slot_floats;
-  float* KhA = abase;
-  float* Z0s = KhA + C * D;
-  float* ZDs = Z0s + C * D;
-  float* Ws = ZDs + C * D;      // [C][CP]
-  float* T1s = Ws + C * CP;     // [C][CP]
-  float* N2p = T1s + C * CP;    // [NWG][C]
-  float* dlt = N2p + NWG * C;   // [C]
-  float* idl = dlt + C;         // [C]
+  float* kring = fbase;                               // [KRING] { Kh, Qf, Vf : [C][D], nrm[C] }
+  float* zring = kring + KRING * Cfg::kslot_floats;   // [RING] { Zs[C][D], GuT, HT : [C][CP], sc[C] }
+  float* abase = zring + RING * Cfg::slot_floats;
+  float* Z0s = abase;               // [C][D]
+  float* ZDs = Z0s + C * D;         // [C][D]  z_t / delta_t
+  float* Ws = ZDs + C * D;          // [C][CP] K A K^T
+  float* Ls = Ws + C * CP;          // [C][CP] unit lower factor
+  float* N2p = Ls + C * CP;         // [NWG][C]
+  float* dlt = N2p + NWG * C;       // [C]
+  float* idl = dlt + C;             // [C]
   float* sbase = abase + Cfg::a_floats;
-  float* KhS = sbase;
-  float* QfS = KhS + C * D;
-  float* VS = QfS + C * D;      // becomes B = V - S K^T in place
-  float* R0s = VS + C * D;
-  float* Eps = R0s + C * D;
-  float* ostage = Eps + C * D;  // [2][C*D]
-  float* Hs = ostage + 2 * C * D;  // [C][CP]
-  float* denp = Hs + C * CP;       // [NWG][C]
-  float* nrm = denp + NWG * C;     // [C]
-  float* inv_den = nrm + C;        // [C]
+  float* VS = sbase;                // [C][D]  B = V^T - S K^T
+  float* R0s = VS + C * D;          // [C][D]
+  float* Eps = R0s + C * D;         // [C][D]
+  float* ostage = Eps + C * D;      // [2][C][D]
+  float* denp = ostage + 2 * C * D; // [NWG][C]
+  float* inv_den = denp + NWG * C;  // [C]
   uint64_t* bars = reinterpret_cast<uint64_t*>(
       (reinterpret_cast<uintptr_t>(sbase + Cfg::s_floats) + 15) & ~uintptr_t(15));
   uint64_t* full = bars;                    // [NSTAGE] raw stage filled by TMA
-  uint64_t* empty = full + NSTAGE;          // [NSTAGE] both groups done with the raw stage
-  uint64_t* ring_full = empty + NSTAGE;     // [RING] group A published Z, T2'
-  uint64_t* ring_empty = ring_full + RING;  // [RING] group S is done with the slot
+  uint64_t* ring_full = full + NSTAGE;      // [RING] group A published chunk c
+  uint64_t* ring_empty = ring_full + RING;  // [RING] group S is done with chunk c
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ring_empty + RING);
 
   const int tid = threadIdx.x;
@@ -201,13 +336,13 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   };
 
   if (tid == 0) {
-    for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 2); }
+    for (int s = 0; s < NSTAGE; ++s) mbar_init(&full[s], 1);
     for (int r = 0; r < RING; ++r) { mbar_init(&ring_full[r], 1); mbar_init(&ring_empty[r], 1); }
     *abort_flag = 0;
     mbar_init_fence();
   }
   __syncthreads();
-  if (tid == NG) {  // thread 0 of group S is the TMA producer
+  if (tid == 0) {  // thread 0 of group A is the TMA producer
     for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue(c);
   }
 
@@ -237,9 +372,6 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     }
   }
 
-  const int ptok0 = g / TOK_LANES;  // prep: first token of this thread (then +4, +8, +12)
-  const int pc4 = g % TOK_LANES;    // prep: float4 column group
-
 #ifdef VLA_SECTION_TIMERS
   long long tsec[12];
   for (int i = 0; i < 12; ++i) tsec[i] = 0;
@@ -251,176 +383,156 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 
   if (is_A) {
     // =====================================================================  group A
-    for (int c = 0; c < nchunks; ++c) {
+    // Input prep of chunk c by the warps [w0, w0 + nw): k_hat, ||phi(k)||, q_f and v as fp32
+    // rows in ring slot c % KRING (zero rows past the end of the sequence).
+    auto prep_inputs = [&](int c, int w0, int nw) {
+      constexpr int LPT = 8;        // lanes per token
+      constexpr int NF = D / 32;    // float4 groups per lane and tensor
       const int s = c % NSTAGE;
       const int n = min(C, T - c * C);
-      const int slot = c % RING;
       wait(&full[s], (c / NSTAGE) & 1);
-      VLA_MARK(0)
-
-      // ---- prep: k_hat rows of this chunk (zero rows past the end of the sequence)
-      {
-        const TIn* rk = raw + (size_t(s) * 3 + 1) * C * D;
+      const TIn* rq = raw + (size_t(s) * 3 + 0) * C * D;
+      const TIn* rk = raw + (size_t(s) * 3 + 1) * C * D;
+      const TIn* rv = raw + (size_t(s) * 3 + 2) * C * D;
+      float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
+      float* Qf = Kh + C * D;
+      float* Vf = Qf + C * D;
+      float* nrm = Vf + C * D;
+      const int sub = lane / LPT, pl = lane % LPT;
+      // one token per 8 lanes; `token` does the elementwise work and returns the partial
+      // sum of squares, `finish` normalises once the 8 lanes have been summed
+      auto token = [&](int tt, float4 (&kf)[NF]) -> float {
+        const bool act = tt < n;
+        float ss = 0.f;
 #pragma unroll
-        for (int it = 0; it < C / TOK_PER_PASS; ++it) {
-          const int tt = it * TOK_PER_PASS + ptok0;
-          const bool act = tt < n;
-          float4 kf = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < NF; ++i) {
+          const int f = i * LPT + pl;
+          float4 qf = make_float4(0.f, 0.f, 0.f, 0.f), vv = qf;
+          kf[i] = qf;
           if (act) {
-            kf = load4(rk + tt * D, pc4);
+            kf[i] = load4(rk + tt * D, f);
+            qf = load4(rq + tt * D, f);
+            vv = load4(rv + tt * D, f);
             if (!ident) {
-              kf.x = phi_elu1(kf.x); kf.y = phi_elu1(kf.y);
-              kf.z = phi_elu1(kf.z); kf.w = phi_elu1(kf.w);
+              kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
+              kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
+              qf.x = phi_fast(qf.x); qf.y = phi_fast(qf.y);
+              qf.z = phi_fast(qf.z); qf.w = phi_fast(qf.w);
             }
           }
-          float ss = kf.x * kf.x + kf.y * kf.y + kf.z * kf.z + kf.w * kf.w;
-#pragma unroll
-          for (int off = TOK_LANES / 2; off >= 1; off >>= 1)
-            ss += __shfl_xor_sync(0xffffffffu, ss, off);
-          const float inv = 1.0f / fmaxf(sqrtf(ss), eps);
-          reinterpret_cast<float4*>(KhA + tt * D)[pc4] =
-              make_float4(kf.x * inv, kf.y * inv, kf.z * inv, kf.w * inv);
+          reinterpret_cast<float4*>(Qf + tt * D)[f] = qf;
+          reinterpret_cast<float4*>(Vf + tt * D)[f] = vv;
+          ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
+          ss = fmaf(kf[i].z, kf[i].z, ss); ss = fmaf(kf[i].w, kf[i].w, ss);
         }
+        return ss;
+      };
+      auto finish = [&](int tt, float ss, const float4 (&kf)[NF]) {
+        const float nr = fmaxf(sqrt_approx(ss), eps);   // max(||phi(k)||, eps)
+        const float inv = rcp_nr(nr);
+#pragma unroll
+        for (int i = 0; i < NF; ++i)
+          reinterpret_cast<float4*>(Kh + tt * D)[i * LPT + pl] =
+              make_float4(kf[i].x * inv, kf[i].y * inv, kf[i].z * inv, kf[i].w * inv);
+        // phi(k) = k_hat * nrm exactly as the recurrence sees it; 0 for padding rows
+        if (pl == 0) nrm[tt] = (tt < n) ? nr : 0.0f;
+      };
+      // two tokens per lane group and iteration, so that their dependency chains interleave
+      for (int tok0 = (gw - w0) * 4; tok0 < C; tok0 += 2 * nw * 4) {
+        const int ta = tok0 + sub, tb = tok0 + nw * 4 + sub;
+        const bool two = tok0 + nw * 4 < C;   // warp-uniform
+        float4 ka[NF], kb[NF];
+        float sa = token(ta, ka), sb = 0.f;
+        if (two) sb = token(tb, kb);
+#pragma unroll
+        for (int off = LPT / 2; off >= 1; off >>= 1) {
+          sa += __shfl_xor_sync(0xffffffffu, sa, off);
+          sb += __shfl_xor_sync(0xffffffffu, sb, off);
+        }
+        finish(ta, sa, ka);
+        if (two) finish(tb, sb, kb);
       }
+    };
+
+    if (nchunks > 0) prep_inputs(0, 0, NWG);
+    group_bar(1, NG);
+    if (g == 0 && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
+
+    for (int c = 0; c < nchunks; ++c) {
+      const int slot = c % RING;
+      const float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
+      const float* Qf = Kh + C * D;
+      float* Zs = zring + size_t(slot) * Cfg::slot_floats;
+      float* GuT = Zs + C * D;
+      float* HT = GuT + C * CP;
+      float* scs = HT + C * CP;
+      VLA_MARK(0)
+
+      // ---- Z0 = A K^T
+      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) { Z0s[t * D + g] = x; });
       group_bar(1, NG);
       VLA_MARK(1)
-      if (g == 0) mbar_arrive(&empty[s]);
 
-      // ---- Z0 = A K^T: per token one pass over the tile, reduce-scatter over the row block
-#pragma unroll 2
-      for (int t = 0; t < C; ++t) {
-        float2 acc[TR];
-#pragma unroll
-        for (int r = 0; r < TR; ++r) acc[r] = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int m = 0; m < NV; ++m) {
-          const float4 k4 = reinterpret_cast<const float4*>(KhA + t * D)[m * LPR + cg];
-          const float2 k01 = make_float2(k4.x, k4.y), k23 = make_float2(k4.z, k4.w);
-#pragma unroll
-          for (int r = 0; r < TR; ++r) {
-            acc[r] = ffma2(st[r][2 * m], k01, acc[r]);
-            acc[r] = ffma2(st[r][2 * m + 1], k23, acc[r]);
-          }
-        }
-        float v[TR];
-#pragma unroll
-        for (int r = 0; r < TR; ++r) v[r] = acc[r].x + acc[r].y;
-        Z0s[t * D + g] = reduce_scatter<LPR>(v, cg);
-      }
+      // ---- W = K Z0 (C x C)
+      gram16<D, NG, CP>(Kh, Z0s, Ws, g);
       group_bar(1, NG);
       VLA_MARK(2)
 
-      // ---- W = K Z0 (C x C), 4x4 output tiles, D/16 threads per tile over the d index
-      {
-        constexpr int P = NG / 16;  // threads per output tile
-        const int tile = g / P, part = g % P;
-        const int s0 = (tile >> 2) * 4, t0 = (tile & 3) * 4;
-        float w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) w[i] = 0.f;
-#pragma unroll
-        for (int step = 0; step < D / (4 * P); ++step) {
-          const int f = step * P + part;
-          float4 a[4], b[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            a[i] = reinterpret_cast<const float4*>(KhA + (s0 + i) * D)[f];
-            b[i] = reinterpret_cast<const float4*>(Z0s + (t0 + i) * D)[f];
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              w[4 * i + j] = fmaf(a[i].x, b[j].x, w[4 * i + j]);
-              w[4 * i + j] = fmaf(a[i].y, b[j].y, w[4 * i + j]);
-              w[4 * i + j] = fmaf(a[i].z, b[j].z, w[4 * i + j]);
-              w[4 * i + j] = fmaf(a[i].w, b[j].w, w[4 * i + j]);
-            }
-        }
-        // sum over the P threads of the tile (consecutive lanes)
-#pragma unroll
-        for (int off = P / 2; off >= 1; off >>= 1)
-#pragma unroll
-          for (int i = 0; i < 16; ++i) w[i] += __shfl_xor_sync(0xffffffffu, w[i], off);
-        if (part == 0) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) Ws[(s0 + i) * CP + t0 + j] = w[4 * i + j];
-        }
-      }
-      group_bar(1, NG);
+      // Group S must be done with chunk c - RING: that frees Z slot `slot` and, because
+      // KRING = RING + 1, the input slot that chunk c + 1 is about to overwrite.
+      if (c >= RING) wait(&ring_empty[slot], ((c / RING) + 1) & 1);
       VLA_MARK(3)
 
-      // ---- warp 0: I + W = L diag(delta) L^T, then T1 = L^-T (Z = Z0 T1)
+      // ---- warp 0: I + W = L diag(delta) L^T.  The other warps widen the next chunk's inputs.
       if (gw == 0) {
         // lane l holds row r = l & 15, columns h*8 .. h*8+7 (h = l >> 4) of M = I + W
         const int r = lane & 15, h = lane >> 4;
-        float m[8], lrow[16];
+        float m[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) m[j] = Ws[r * CP + h * 8 + j] + ((h * 8 + j == r) ? 1.0f : 0.0f);
 #pragma unroll
         for (int s2 = 0; s2 < 16; ++s2) {
           const int hs = s2 >> 3, js = s2 & 7;
+          // Algorithm 1 clamps delta at eps; delta >= 1 whenever A is positive definite
           const float piv = fmaxf(__shfl_sync(0xffffffffu, m[js], s2 + 16 * hs), eps);
           const float mrs = __shfl_sync(0xffffffffu, m[js], r + 16 * hs);
-          const float ipiv = 1.0f / piv;
-          const float l = (r > s2) ? mrs * ipiv : 0.0f;
-          lrow[s2] = l;  // L[r][s2]
+          const float ipiv = rcp_nr(piv);
+          const float l = (r > s2) ? mrs * ipiv : 0.0f;  // L[r][s2]
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float msj = __shfl_sync(0xffffffffu, m[j], s2 + 16 * h);
             m[j] = fmaf(-l, msj, m[j]);
           }
+          if (h == hs) Ls[r * CP + s2] = l;
           if (lane == 0) { dlt[s2] = piv; idl[s2] = ipiv; }
         }
-        // T1[:, t] = e_t - sum_{s<t} L[t][s] T1[:, s]; lane r (< 16) keeps row r of T1
-        float t1[16];
-#pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          float a0 = (r == t) ? 1.0f : 0.0f, a1 = 0.0f;
-#pragma unroll
-          for (int s2 = 0; s2 < t; ++s2) {
-            const float lts = __shfl_sync(0xffffffffu, lrow[s2], t);  // L[t][s2]
-            if (s2 & 1) a1 = fmaf(-lts, t1[s2], a1); else a0 = fmaf(-lts, t1[s2], a0);
-          }
-          t1[t] = a0 + a1;
-        }
-        if (h == 0) {
-#pragma unroll
-          for (int t = 0; t < 16; ++t) T1s[r * CP + t] = t1[t];
-        } else {
-          // upper half keeps L for the T2' step: Ws is free now, store L there (row r)
-#pragma unroll
-          for (int s2 = 0; s2 < 16; ++s2) Ws[r * CP + s2] = lrow[s2];
-        }
+        VLA_MARK(8)
+        if (NWG == 1 && c + 1 < nchunks) prep_inputs(c + 1, 0, 1);
+      } else {
+        if (c + 1 < nchunks) prep_inputs(c + 1, 1, NWG - 1);
+        VLA_MARK(8)
       }
       group_bar(1, NG);
+      // the raw stage of chunk c + 1 has been consumed: refill it
+      if (g == 0 && c + 1 + NSTAGE < nchunks) issue(c + 1 + NSTAGE);
       VLA_MARK(4)
 
-      // the ring slot must have been released by group S (chunk c - RING)
-      if (c >= RING) wait(&ring_empty[slot], ((c / RING) + 1) & 1);
-      VLA_MARK(5)
-
-      // ---- Z = Z0 T1 (row g), published as Zs; ZD = Z / delta; partial ||z_t||^2
+      // ---- row g of Z by forward substitution: z_t = z0_t - sum_{s<t} L[t][s] z_s
       {
-        float z0[16], z[16];
+        float z[16];
 #pragma unroll
-        for (int t = 0; t < 16; ++t) z0[t] = Z0s[t * D + g];
+        for (int t = 0; t < 16; ++t) {
+          float a0 = Z0s[t * D + g], a1 = 0.f;
 #pragma unroll
-        for (int t = 0; t < 16; ++t) z[t] = 0.f;
-#pragma unroll
-        for (int s2 = 0; s2 < 16; ++s2) {
-#pragma unroll
-          for (int t4 = s2 / 4; t4 < 4; ++t4) {
-            const float4 tt = reinterpret_cast<const float4*>(T1s + s2 * CP)[t4];
-            if (4 * t4 + 0 >= s2) z[4 * t4 + 0] = fmaf(z0[s2], tt.x, z[4 * t4 + 0]);
-            if (4 * t4 + 1 >= s2) z[4 * t4 + 1] = fmaf(z0[s2], tt.y, z[4 * t4 + 1]);
-            if (4 * t4 + 2 >= s2) z[4 * t4 + 2] = fmaf(z0[s2], tt.z, z[4 * t4 + 2]);
-            if (4 * t4 + 3 >= s2) z[4 * t4 + 3] = fmaf(z0[s2], tt.w, z[4 * t4 + 3]);
+          for (int s4 = 0; s4 * 4 < t; ++s4) {
+            const float4 l4 = reinterpret_cast<const float4*>(Ls + t * CP)[s4];
+            if (4 * s4 + 0 < t) a0 = fmaf(-l4.x, z[4 * s4 + 0], a0);
+            if (4 * s4 + 1 < t) a1 = fmaf(-l4.y, z[4 * s4 + 1], a1);
+            if (4 * s4 + 2 < t) a0 = fmaf(-l4.z, z[4 * s4 + 2], a0);
+            if (4 * s4 + 3 < t) a1 = fmaf(-l4.w, z[4 * s4 + 3], a1);
           }
+          z[t] = a0 + a1;
         }
-        float* Zs = ringZ[slot];
         float sq[16];
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
@@ -429,74 +541,41 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           sq[t] = z[t] * z[t];
         }
         const float tot = warp_reduce_scatter16(sq, lane);
-        // lane bits 4..1 select the token: bit 4 <-> token bit 3, ..., bit 1 <-> token bit 0
         if ((lane & 1) == 0) N2p[gw * C + (lane >> 1)] = tot;
       }
       group_bar(1, NG);
-      VLA_MARK(6)
+      VLA_MARK(5)
 
-      // ---- warp 1 (or 0 when the group has one warp): sc, Gu, T2' = (I + Gu)^-1 diag(sc)
-      if (gw == (NWG > 1 ? 1 : 0)) {
-        const int r = lane & 15;
+      // ---- warp 0: sc_t and GuT[t][s] = Gu[s][t] = sc_s delta_s L[t][s]
+      if (gw == 0) {
+        const int r = lane & 15, h = lane >> 4;
         float n2 = 0.f;
 #pragma unroll
         for (int w2 = 0; w2 < NWG; ++w2) n2 += N2p[w2 * C + r];
         const float id_r = idl[r], d_r = dlt[r];
-        const float sc_r = id_r / fmaxf(sqrtf(n2) * id_r, eps);  // alpha_r = sc_r z_r
+        // alpha_r = sc_r z_r with sc_r = (1/delta) / max(||z||/delta, eps)
+        const float sc_r = id_r * rcp_nr(fmaxf(sqrt_approx(n2) * id_r, eps));
         if ((p.flags & VLA_FLAG_CHECK_FINITE) && p.status && !isfinite(n2 + d_r))
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
-        // lane r keeps row r of T2 and the column r of Gu: Gu[s][t] = sc_s delta_s L[t][s]
-        // T2[:, t] = e_t - sum_{s<t} Gu[s][t] T2[:, s]
-        const float scd = sc_r * d_r;
-        float t2[16];
+        const float scd = sc_r * d_r;   // multiplies column r of L
+        if (h == 0) scs[r] = sc_r;
+        // lane (r, h) writes GuT[r][h*8 .. h*8+7]: GuT[r][s] = scd_s L[r][s]
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          float a0 = (r == t) ? 1.0f : 0.0f, a1 = 0.0f;
-#pragma unroll
-          for (int s2 = 0; s2 < t; ++s2) {
-            // Gu[s2][t] = sc_{s2} delta_{s2} L[t][s2]
-            const float gst = __shfl_sync(0xffffffffu, scd, s2) * Ws[t * CP + s2];
-            if (s2 & 1) a1 = fmaf(-gst, t2[s2], a1); else a0 = fmaf(-gst, t2[s2], a0);
-          }
-          t2[t] = a0 + a1;
+        for (int j = 0; j < 8; ++j) {
+          const int s2 = h * 8 + j;
+          const float scd_s = __shfl_sync(0xffffffffu, scd, s2);
+          GuT[r * CP + s2] = (s2 < r) ? scd_s * Ls[r * CP + s2] : 0.0f;
         }
-        float* T2p = ringT2[slot];
-        if (lane < 16) {
-#pragma unroll
-          for (int t = 0; t < 16; ++t)
-            T2p[r * CP + t] = t2[t] * __shfl_sync(0x0000ffffu, sc_r, t);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ring_full[slot]);
       }
+      // ---- HT[t][s] = q_t . z_s (C x C), then publish the chunk to group S
+      gram16<D, NG, CP>(Qf, Zs, HT, g);
+      group_bar(1, NG);
+      if (g == 0) mbar_arrive(&ring_full[slot]);
+      VLA_MARK(6)
 
-      VLA_MARK(7)
       // ---- A <- A - Z diag(1/delta) Z^T
-      {
-        const float* Zs = ringZ[slot];
-#pragma unroll 2
-        for (int s2 = 0; s2 < C; ++s2) {
-          float zd[TR];
-#pragma unroll
-          for (int r4 = 0; r4 < TR / 4; ++r4) {
-            const float4 x = reinterpret_cast<const float4*>(ZDs + s2 * D + rb * TR)[r4];
-            zd[4 * r4 + 0] = -x.x; zd[4 * r4 + 1] = -x.y; zd[4 * r4 + 2] = -x.z; zd[4 * r4 + 3] = -x.w;
-          }
-#pragma unroll
-          for (int m = 0; m < NV; ++m) {
-            const float4 z4 = reinterpret_cast<const float4*>(Zs + s2 * D)[m * LPR + cg];
-            const float2 z01 = make_float2(z4.x, z4.y), z23 = make_float2(z4.z, z4.w);
-#pragma unroll
-            for (int r = 0; r < TR; ++r) {
-              const float2 zz = make_float2(zd[r], zd[r]);
-              st[r][2 * m] = ffma2(zz, z01, st[r][2 * m]);
-              st[r][2 * m + 1] = ffma2(zz, z23, st[r][2 * m + 1]);
-            }
-          }
-        }
-      }
-      group_bar(1, NG);  // ZDs, Ws, N2p may be rewritten by the next chunk
-      VLA_MARK(8)
+      tile_rank_update<TR, TW, LPR, D, C, true>(st, ZDs, Zs, rb, cg);
+      VLA_MARK(7)
     }
     // final A
     if (p.A_T) {
@@ -516,223 +595,102 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     if (g < C) inv_den[g] = 1.0f;
 
     for (int c = 0; c < nchunks; ++c) {
-      const int s = c % NSTAGE;
       const int n = min(C, T - c * C);
       const int slot = c % RING;
-      wait(&full[s], (c / NSTAGE) & 1);
       VLA_MARK(0)
-      if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
-
-      // ---- prep: k_hat, ||phi(k)||, q_f, v (zero rows past the end of the sequence)
-      {
-        const TIn* rq = raw + (size_t(s) * 3 + 0) * C * D;
-        const TIn* rk = raw + (size_t(s) * 3 + 1) * C * D;
-        const TIn* rv = raw + (size_t(s) * 3 + 2) * C * D;
-#pragma unroll
-        for (int it = 0; it < C / TOK_PER_PASS; ++it) {
-          const int tt = it * TOK_PER_PASS + ptok0;
-          const bool act = tt < n;
-          float4 kf = make_float4(0.f, 0.f, 0.f, 0.f), qf = kf, vv = kf;
-          if (act) {
-            kf = load4(rk + tt * D, pc4);
-            qf = load4(rq + tt * D, pc4);
-            vv = load4(rv + tt * D, pc4);
-            if (!ident) {
-              kf.x = phi_elu1(kf.x); kf.y = phi_elu1(kf.y);
-              kf.z = phi_elu1(kf.z); kf.w = phi_elu1(kf.w);
-              qf.x = phi_elu1(qf.x); qf.y = phi_elu1(qf.y);
-              qf.z = phi_elu1(qf.z); qf.w = phi_elu1(qf.w);
-            }
-          }
-          float ss = kf.x * kf.x + kf.y * kf.y + kf.z * kf.z + kf.w * kf.w;
-#pragma unroll
-          for (int off = TOK_LANES / 2; off >= 1; off >>= 1)
-            ss += __shfl_xor_sync(0xffffffffu, ss, off);
-          const float nr = sqrtf(ss);
-          const float inv = 1.0f / fmaxf(nr, eps);
-          reinterpret_cast<float4*>(KhS + tt * D)[pc4] =
-              make_float4(kf.x * inv, kf.y * inv, kf.z * inv, kf.w * inv);
-          reinterpret_cast<float4*>(QfS + tt * D)[pc4] = qf;
-          reinterpret_cast<float4*>(VS + tt * D)[pc4] = vv;
-          // phi(k) = k_hat * mult (mult = max(||phi(k)||, eps) unless the floor was active)
-          if (pc4 == 0) nrm[tt] = act ? fmaxf(nr, eps) : 0.0f;
-        }
-      }
-      group_bar(2, NG);
+      // ---- group A's products of this chunk: k_hat, q_f, v, ||phi(k)||, Z, Gu, HT, sc
+      wait(&ring_full[slot], (c / RING) & 1);
+      const float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
+      const float* Qf = Kh + C * D;
+      const float* Vf = Qf + C * D;
+      const float* nrm = Vf + C * D;
+      const float* Zs = zring + size_t(slot) * Cfg::slot_floats;
+      const float* GuT = Zs + C * D;
+      const float* HT = GuT + C * CP;
+      const float* scs = HT + C * CP;
       VLA_MARK(1)
-      if (g == 0) {
-        mbar_arrive(&empty[s]);
-        if (c + NSTAGE < nchunks) {  // refill the stage once group A has left it too
-          wait(&empty[s], (c / NSTAGE) & 1);
-          issue(c + NSTAGE);
-        }
-      }
 
       // ---- running key sum and readout denominators (thread = column g)
       if (!ident) {
         float pr[16];
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
-          zk = fmaf(KhS[t * D + g], nrm[t], zk);
-          pr[t] = zk * QfS[t * D + g];
+          zk = fmaf(Kh[t * D + g], nrm[t], zk);
+          pr[t] = zk * Qf[t * D + g];
         }
         const float tot = warp_reduce_scatter16(pr, lane);
         if ((lane & 1) == 0) denp[gw * C + (lane >> 1)] = tot;
       }
 
-      // ---- P0 = S K^T, R0 = S Q^T; B = V^T - P0 (in place over V)
-#pragma unroll 2
-      for (int t = 0; t < C; ++t) {
-        float2 ap[TR], ar[TR];
+      // ---- B = V^T - S K^T and R0 = S Q^T, row g of each
+      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) {
+        VS[t * D + g] = Vf[t * D + g] - x;
+      });
+      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
+      if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
+      group_bar(2, NG);                 // denp complete
+      if (!ident && g < C) {
+        float dd = 0.f;
 #pragma unroll
-        for (int r = 0; r < TR; ++r) { ap[r] = make_float2(0.f, 0.f); ar[r] = make_float2(0.f, 0.f); }
-#pragma unroll
-        for (int m = 0; m < NV; ++m) {
-          const float4 k4 = reinterpret_cast<const float4*>(KhS + t * D)[m * LPR + cg];
-          const float4 q4 = reinterpret_cast<const float4*>(QfS + t * D)[m * LPR + cg];
-          const float2 k01 = make_float2(k4.x, k4.y), k23 = make_float2(k4.z, k4.w);
-          const float2 q01 = make_float2(q4.x, q4.y), q23 = make_float2(q4.z, q4.w);
-#pragma unroll
-          for (int r = 0; r < TR; ++r) {
-            ap[r] = ffma2(st[r][2 * m], k01, ap[r]);
-            ap[r] = ffma2(st[r][2 * m + 1], k23, ap[r]);
-            ar[r] = ffma2(st[r][2 * m], q01, ar[r]);
-            ar[r] = ffma2(st[r][2 * m + 1], q23, ar[r]);
-          }
-        }
-        float vp[TR], vr[TR];
-#pragma unroll
-        for (int r = 0; r < TR; ++r) { vp[r] = ap[r].x + ap[r].y; vr[r] = ar[r].x + ar[r].y; }
-        const float p0 = reduce_scatter<LPR>(vp, cg);
-        const float r0 = reduce_scatter<LPR>(vr, cg);
-        VS[t * D + g] = VS[t * D + g] - p0;   // same thread wrote nothing else here: row g
-        R0s[t * D + g] = r0;
+        for (int w2 = 0; w2 < NWG; ++w2) dd += denp[w2 * C + g];
+        inv_den[g] = rcp_nr(fmaxf(dd, eps));
       }
-
-      // ---- wait for group A's Z and T2' of this chunk
-      wait(&ring_full[slot], (c / RING) & 1);
       VLA_MARK(2)
-      const float* Zs = ringZ[slot];
-      const float* T2p = ringT2[slot];
-      group_bar(2, NG);  // KhS/QfS/VS/R0s/denp complete for every row
-      VLA_MARK(3)
 
-      // ---- H'[s][t] = z_s . q_t (C x C), same tiling as W; and the denominators
+      // ---- row g: e_t = b_t - sum_{s<t} Gu[s][t] e_s; e'_t = sc_t e_t;
+      //             o_t = (r0_t + sum_{s<=t} e'_s HT[t][s]) / den_t
+      float o[16];
       {
-        constexpr int P = NG / 16;
-        const int tile = g / P, part = g % P;
-        const int s0 = (tile >> 2) * 4, t0 = (tile & 3) * 4;
-        float w[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) w[i] = 0.f;
-#pragma unroll
-        for (int step = 0; step < D / (4 * P); ++step) {
-          const int f = step * P + part;
-          float4 a[4], b[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            a[i] = reinterpret_cast<const float4*>(Zs + (s0 + i) * D)[f];
-            b[i] = reinterpret_cast<const float4*>(QfS + (t0 + i) * D)[f];
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              w[4 * i + j] = fmaf(a[i].x, b[j].x, w[4 * i + j]);
-              w[4 * i + j] = fmaf(a[i].y, b[j].y, w[4 * i + j]);
-              w[4 * i + j] = fmaf(a[i].z, b[j].z, w[4 * i + j]);
-              w[4 * i + j] = fmaf(a[i].w, b[j].w, w[4 * i + j]);
-            }
-        }
-#pragma unroll
-        for (int off = P / 2; off >= 1; off >>= 1)
-#pragma unroll
-          for (int i = 0; i < 16; ++i) w[i] += __shfl_xor_sync(0xffffffffu, w[i], off);
-        if (part == 0) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) Hs[(s0 + i) * CP + t0 + j] = w[4 * i + j];
-        }
-        if (!ident && g < C) {
-          float dd = 0.f;
-#pragma unroll
-          for (int w2 = 0; w2 < NWG; ++w2) dd += denp[w2 * C + g];
-          inv_den[g] = 1.0f / fmaxf(dd, eps);
-        }
-      }
-      group_bar(2, NG);
-      VLA_MARK(4)
-
-      // ---- row g: e'_t = sum_{s<=t} b_s T2'[s][t];  o_t = (r0_t + sum_{s<=t} e'_s H'[s][t]) / den_t
-      {
-        float b[16], e[16], o[16];
-#pragma unroll
-        for (int t = 0; t < 16; ++t) { b[t] = VS[t * D + g]; e[t] = 0.f; o[t] = R0s[t * D + g]; }
-#pragma unroll
-        for (int s2 = 0; s2 < 16; ++s2) {
-#pragma unroll
-          for (int t4 = s2 / 4; t4 < 4; ++t4) {
-            const float4 tt = reinterpret_cast<const float4*>(T2p + s2 * CP)[t4];
-            if (4 * t4 + 0 >= s2) e[4 * t4 + 0] = fmaf(b[s2], tt.x, e[4 * t4 + 0]);
-            if (4 * t4 + 1 >= s2) e[4 * t4 + 1] = fmaf(b[s2], tt.y, e[4 * t4 + 1]);
-            if (4 * t4 + 2 >= s2) e[4 * t4 + 2] = fmaf(b[s2], tt.z, e[4 * t4 + 2]);
-            if (4 * t4 + 3 >= s2) e[4 * t4 + 3] = fmaf(b[s2], tt.w, e[4 * t4 + 3]);
-          }
-        }
-        // e[s2] is complete once every s <= s2 has been added: column t of T2' only has
-        // rows s <= t, so after the loop above all of e is final.
-#pragma unroll
-        for (int s2 = 0; s2 < 16; ++s2) {
-#pragma unroll
-          for (int t4 = s2 / 4; t4 < 4; ++t4) {
-            const float4 hh = reinterpret_cast<const float4*>(Hs + s2 * CP)[t4];
-            if (4 * t4 + 0 >= s2) o[4 * t4 + 0] = fmaf(e[s2], hh.x, o[4 * t4 + 0]);
-            if (4 * t4 + 1 >= s2) o[4 * t4 + 1] = fmaf(e[s2], hh.y, o[4 * t4 + 1]);
-            if (4 * t4 + 2 >= s2) o[4 * t4 + 2] = fmaf(e[s2], hh.z, o[4 * t4 + 2]);
-            if (4 * t4 + 3 >= s2) o[4 * t4 + 3] = fmaf(e[s2], hh.w, o[4 * t4 + 3]);
-          }
-        }
-        float* ost = ostage + size_t(c & 1) * C * D;
+        float e[16], ep[16];
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
-          Eps[t * D + g] = e[t];
-          ost[t * D + g] = o[t] * inv_den[t];
+          float a0 = VS[t * D + g], a1 = 0.f;
+#pragma unroll
+          for (int s4 = 0; s4 * 4 < t; ++s4) {
+            const float4 g4 = reinterpret_cast<const float4*>(GuT + t * CP)[s4];
+            if (4 * s4 + 0 < t) a0 = fmaf(-g4.x, e[4 * s4 + 0], a0);
+            if (4 * s4 + 1 < t) a1 = fmaf(-g4.y, e[4 * s4 + 1], a1);
+            if (4 * s4 + 2 < t) a0 = fmaf(-g4.z, e[4 * s4 + 2], a0);
+            if (4 * s4 + 3 < t) a1 = fmaf(-g4.w, e[4 * s4 + 3], a1);
+          }
+          e[t] = a0 + a1;
+          ep[t] = e[t] * scs[t];
+          Eps[t * D + g] = ep[t];
         }
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          float a0 = R0s[t * D + g], a1 = 0.f;
+#pragma unroll
+          for (int s4 = 0; s4 * 4 <= t; ++s4) {
+            const float4 h4 = reinterpret_cast<const float4*>(HT + t * CP)[s4];
+            if (4 * s4 + 0 <= t) a0 = fmaf(h4.x, ep[4 * s4 + 0], a0);
+            if (4 * s4 + 1 <= t) a1 = fmaf(h4.y, ep[4 * s4 + 1], a1);
+            if (4 * s4 + 2 <= t) a0 = fmaf(h4.z, ep[4 * s4 + 2], a0);
+            if (4 * s4 + 3 <= t) a1 = fmaf(h4.w, ep[4 * s4 + 3], a1);
+          }
+          o[t] = a0 + a1;
+        }
+      }
+      group_bar(2, NG);  // inv_den written; Eps complete
+      {
+        float* ost = ostage + size_t(c & 1) * C * D;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) ost[t * D + g] = o[t] * inv_den[t];
       }
       fence_async_smem();
       group_bar(2, NG);
-      VLA_MARK(5)
       if (g == 0) {
         bulk_store(gout + size_t(c) * C * D, ostage + size_t(c & 1) * C * D,
                    uint32_t(n) * D * sizeof(float));
         bulk_commit();
       }
+      VLA_MARK(3)
 
       // ---- S <- S + E' Z^T
-#pragma unroll 2
-      for (int s2 = 0; s2 < C; ++s2) {
-        float ev[TR];
-#pragma unroll
-        for (int r4 = 0; r4 < TR / 4; ++r4) {
-          const float4 x = reinterpret_cast<const float4*>(Eps + s2 * D + rb * TR)[r4];
-          ev[4 * r4 + 0] = x.x; ev[4 * r4 + 1] = x.y; ev[4 * r4 + 2] = x.z; ev[4 * r4 + 3] = x.w;
-        }
-#pragma unroll
-        for (int m = 0; m < NV; ++m) {
-          const float4 z4 = reinterpret_cast<const float4*>(Zs + s2 * D)[m * LPR + cg];
-          const float2 z01 = make_float2(z4.x, z4.y), z23 = make_float2(z4.z, z4.w);
-#pragma unroll
-          for (int r = 0; r < TR; ++r) {
-            const float2 ee = make_float2(ev[r], ev[r]);
-            st[r][2 * m] = ffma2(ee, z01, st[r][2 * m]);
-            st[r][2 * m + 1] = ffma2(ee, z23, st[r][2 * m + 1]);
-          }
-        }
-      }
+      tile_rank_update<TR, TW, LPR, D, C, false>(st, Eps, Zs, rb, cg);
       group_bar(2, NG);
-      VLA_MARK(6)
       if (g == 0) mbar_arrive(&ring_empty[slot]);
+      VLA_MARK(4)
     }
     // final S and key sum
     if (p.S_T) {

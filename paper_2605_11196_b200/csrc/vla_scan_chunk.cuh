@@ -51,8 +51,9 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // Fast elementwise helpers of the prep pass (relative error ~1e-6, far inside the parity bound).
 // Branch-free: both sides are evaluated and selected, so a warp never diverges here.
 __device__ __forceinline__ float phi_fast(float x) {
+  const float xm = x > 0.0f ? 0.0f : x;   // keeps a NaN (fminf would drop it)
   float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fminf(x, 0.0f) * 1.4426950408889634f));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(xm * 1.4426950408889634f));
   return x > 0.0f ? x + 1.0f : e;
 }
 __device__ __forceinline__ float sqrt_approx(float x) {

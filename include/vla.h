@@ -39,7 +39,8 @@ typedef enum {
   VLA_ERR_ALIGNMENT = -3,      /* a base pointer is not 16-byte aligned                      */
   VLA_ERR_CUDA = -4,           /* a CUDA runtime call or the launch failed                   */
   VLA_ERR_DEVICE_TIMEOUT = -5, /* written to opts->status: a bounded device-side wait ran out */
-  VLA_ERR_NONFINITE = -6       /* written to opts->status: non-finite delta / norm seen       */
+  VLA_ERR_NONFINITE = -6,      /* written to opts->status: non-finite delta / norm seen       */
+  VLA_ERR_TOO_LARGE = -7       /* vla_forward_host_static: the built-in buffer is too small   */
 } vla_status_t;
 
 typedef enum { VLA_F32 = 0, VLA_BF16 = 1 } vla_dtype_t;
@@ -106,6 +107,37 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
                      float* out, float* S_T, float* A_T,
                      const vla_opts_t* opts, void* workspace, size_t workspace_bytes,
                      void* stream);
+
+/*
+ * vla_forward_host_static -- vla_forward_host for callers that cannot hand over a device
+ * workspace.  (The paper has no counterpart; this is a convenience of the library.)
+ *
+ * Who needs it: code that has host buffers and a stream but no way to obtain device
+ * memory at the point of the call -- a plug-in inside a host application that gave the
+ * whole device to another memory pool, a process running against a hard device-memory
+ * cap that is already committed, or a latency-critical loop that must not pay
+ * cudaMalloc's cost and implicit synchronisation.  For them the staging memory that
+ * vla_forward_host takes as `workspace` is built into the library instead: a fixed array
+ * of VLA_STATIC_SCRATCH_BYTES in device memory, present on every GPU that loads the
+ * library until the process exits.  The call allocates and frees nothing.
+ *
+ * Arguments and results are exactly those of vla_forward_host without `workspace`.
+ * Limits and rules:
+ *   - vla_host_workspace_bytes(...) for the problem must not exceed
+ *     VLA_STATIC_SCRATCH_BYTES, else VLA_ERR_TOO_LARGE is returned and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (a one-time
+ *     set-up for that device); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left
+ *     in it.  Two calls whose work can overlap on the GPU (different streams without an
+ *     ordering between them) race on it: order them, or use vla_forward_host with
+ *     separate workspaces.
+ */
+#define VLA_STATIC_SCRATCH_BYTES (32u << 20)
+int vla_forward_host_static(const void* q, const void* k, const void* v, float lambda_,
+                            int B, int H, int T, int d_k, int d_v,
+                            const float* S0, const float* A0,
+                            float* out, float* S_T, float* A_T,
+                            const vla_opts_t* opts, void* stream);
 
 /* Device bytes vla_forward_host needs for these sizes (0 on invalid sizes). */
 size_t vla_host_workspace_bytes(int B, int H, int T, int d_k, int d_v, int qkv_dtype, int has_u);

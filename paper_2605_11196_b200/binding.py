@@ -18,12 +18,13 @@ from . import build as _build
 
 VLA_OK = 0
 VLA_ERR_INVALID_ARG, VLA_ERR_UNSUPPORTED, VLA_ERR_ALIGNMENT = -1, -2, -3
-VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE = -4, -5, -6
+VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE, VLA_ERR_TOO_LARGE = -4, -5, -6, -7
+VLA_STATIC_SCRATCH_BYTES = 32 << 20
 VLA_F32, VLA_BF16 = 0, 1
 VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE = 1, 2
 VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK = 0, 1, 2
 
-EXPORTS = ("vla_forward", "vla_forward_host", "vla_host_workspace_bytes",
+EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",
            "vla_query_support", "vla_status_string", "vla_version")
 
 
@@ -67,6 +68,9 @@ def load_library():
             lib.vla_forward_host.restype = i
             lib.vla_forward_host.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp,
                                              ctypes.POINTER(VlaOpts), vp, ctypes.c_size_t, vp]
+            lib.vla_forward_host_static.restype = i
+            lib.vla_forward_host_static.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp,
+                                                    ctypes.POINTER(VlaOpts), vp]
             lib.vla_host_workspace_bytes.restype = ctypes.c_size_t
             lib.vla_host_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
             lib.vla_query_support.restype = i
@@ -222,4 +226,43 @@ def vla_forward_host(q, k, v, lam: float, workspace: torch.Tensor, *, u=None, S0
                                   ctypes.c_void_p(st.cuda_stream))
     if rc != VLA_OK:
         raise VlaError(rc, "vla_forward_host")
+    return VlaResult(out, S_T, A_T, z_T, status)
+
+
+def vla_forward_host_static(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None,
+                            flags: int = 0, eps: float = 1e-4, out=None, S_T=None, A_T=None,
+                            z_T=None, status=None, kernel: int = VLA_KERNEL_AUTO,
+                            device=None, stream: Optional[torch.cuda.Stream] = None) -> VlaResult:
+    """``vla_forward_host`` without a workspace argument: the staging memory is the library's
+    built-in device array (``VLA_STATIC_SCRATCH_BYTES``), so the call allocates nothing on the
+    device.  For callers that hold host tensors and a stream but cannot get device memory
+    where they stand (no allocator handle, a committed memory cap, a loop that must not
+    allocate).  Problems whose staging need exceeds the array raise ``VLA_ERR_TOO_LARGE``.
+    Calls on one device share the array: do not let two of them overlap on the GPU."""
+    lib = load_library()
+    B, H, T, dk = q.shape
+    dv = v.shape[-1]
+    dt = _dtype_code(q)
+    f32 = torch.float32
+    _chk(q, (B, H, T, dk), q.dtype, "q", cuda=False); _chk(k, (B, H, T, dk), q.dtype, "k", cuda=False)
+    _chk(v, (B, H, T, dv), q.dtype, "v", cuda=False); _chk(u, (B, H, T, dk), q.dtype, "u", cuda=False)
+    _chk(S0, (B, H, dv, dk), f32, "S0", cuda=False); _chk(A0, (B, H, dk, dk), f32, "A0", cuda=False)
+    _chk(z0, (B, H, dk), f32, "z0", cuda=False)
+    pin = torch.cuda.is_available()
+    mk = lambda shape: torch.empty(shape, dtype=f32, pin_memory=pin)
+    out = mk((B, H, T, dv)) if out is None else out
+    S_T = mk((B, H, dv, dk)) if S_T is None else S_T
+    A_T = mk((B, H, dk, dk)) if A_T is None else A_T
+    z_T = mk((B, H, dk)) if z_T is None else z_T
+    _chk(out, (B, H, T, dv), f32, "out", cuda=False); _chk(S_T, (B, H, dv, dk), f32, "S_T", cuda=False)
+    _chk(A_T, (B, H, dk, dk), f32, "A_T", cuda=False); _chk(z_T, (B, H, dk), f32, "z_T", cuda=False)
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel)
+    with torch.cuda.device(dev):
+        rc = lib.vla_forward_host_static(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv,
+                                         _ptr(S0), _ptr(A0), _ptr(out), _ptr(S_T), _ptr(A_T),
+                                         ctypes.byref(opts), ctypes.c_void_p(st.cuda_stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_forward_host_static")
     return VlaResult(out, S_T, A_T, z_T, status)

@@ -4,6 +4,7 @@
 
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 
 #include "vla.h"
 #include "vla_common.cuh"
@@ -117,6 +118,35 @@ int check_common(const void* q, const void* k, const void* v, float lambda_, int
 
 inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
+// ---- built-in staging buffer of vla_forward_host_static
+// Lives in every device's memory for as long as the library is loaded.  In host code the
+// array's NAME is only a handle: the device address has to be asked for with
+// cudaGetSymbolAddress, once per device, with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[VLA_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {};   // per device, filled on the first call there
+
+// Device address of the built-in buffer on the current device (nullptr on failure).
+void* static_scratch_for_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    g_scratch_addr[dev] = ptr;
+  }
+  return g_scratch_addr[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -216,6 +246,26 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
   return VLA_OK;
 }
 
+int vla_forward_host_static(const void* q, const void* k, const void* v, float lambda_, int B,
+                            int H, int T, int d_k, int d_v, const float* S0, const float* A0,
+                            float* out, float* S_T, float* A_T, const vla_opts_t* opts,
+                            void* stream) {
+  // Size check first: it needs no CUDA call and gives the clearest answer.
+  vla_opts_t o;
+  int rc = resolve_opts(opts, &o);
+  if (rc != VLA_OK) return rc;
+  rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, out);
+  if (rc != VLA_OK) return rc;
+  const size_t need = vla_host_workspace_bytes(B, H, T, d_k, d_v, o.qkv_dtype, o.u != nullptr);
+  if (need > size_t(VLA_STATIC_SCRATCH_BYTES)) return VLA_ERR_TOO_LARGE;
+  void* scratch = static_scratch_for_current_device();
+  if (!scratch) return VLA_ERR_CUDA;
+  // Every staging region is written (by a copy or by the scan) before it is read, so
+  // nothing left behind by the previous call needs clearing.
+  return vla_forward_host(q, k, v, lambda_, B, H, T, d_k, d_v, S0, A0, out, S_T, A_T, opts, scratch,
+                          size_t(VLA_STATIC_SCRATCH_BYTES), stream);
+}
+
 int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags) {
   if (qkv_dtype != VLA_F32 && qkv_dtype != VLA_BF16) return VLA_ERR_UNSUPPORTED;
   if (flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_UNSUPPORTED;
@@ -231,6 +281,9 @@ const char* vla_status_string(int status) {
     case VLA_ERR_CUDA: return "CUDA runtime or launch error";
     case VLA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
     case VLA_ERR_NONFINITE: return "non-finite delta or write-direction norm";
+    case VLA_ERR_TOO_LARGE:
+      return "problem needs more staging memory than the built-in buffer of "
+             "vla_forward_host_static (VLA_STATIC_SCRATCH_BYTES); use vla_forward_host";
     default: return "unknown status";
   }
 }

@@ -96,11 +96,11 @@ struct ChunkCfg {
   // shared memory layout (floats unless noted)
   static constexpr size_t raw_bytes = size_t(NSTAGE) * 3 * C * D * sizeof(TIn);
   static constexpr size_t kslot_floats = size_t(3) * C * D + C;             // Kh, Qf, Vf, nrm
-  static constexpr size_t slot_floats = size_t(C) * D + 2 * C * CP + C;     // Zs, GuT, HT, sc
-  static constexpr size_t a_floats = size_t(2) * C * D + 2 * C * CP + NWG * C + 2 * C;
-  //   Z0s, ZDs | Ws, Ls | N2p | delta, inv_delta
-  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + NWG * C + C;
-  //   VS(B), R0s, Eps | ostage[2] | denp | inv_den
+  static constexpr size_t slot_floats = size_t(C) * D + 2 * C * CP + 2 * C; // Zs, GuT, HT, sc, inv_den
+  static constexpr size_t a_floats = size_t(2) * C * D + 2 * C * CP + 2 * NWG * C + 2 * C;
+  //   Z0s, ZDs | Ws, Ls | N2p, denp | delta, inv_delta
+  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D;
+  //   VS(B), R0s, Eps | ostage[2]
   static constexpr size_t smem_bytes = raw_bytes +
       (KRING * kslot_floats + RING * slot_floats + a_floats + s_floats) * sizeof(float) +
       (NSTAGE + 2 * RING) * sizeof(uint64_t) + 16 + 128;
@@ -275,22 +275,21 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   TIn* raw = reinterpret_cast<TIn*>(smem);
   float* fbase = reinterpret_cast<float*>(smem + Cfg::raw_bytes);
   float* kring = fbase;                               // [KRING] { Kh, Qf, Vf : [C][D], nrm[C] }
-  float* zring = kring + KRING * Cfg::kslot_floats;   // [RING] { Zs[C][D], GuT, HT : [C][CP], sc[C] }
+  float* zring = kring + KRING * Cfg::kslot_floats;   // [RING] { Zs[C][D], GuT, HT : [C][CP], sc, inv_den : [C] }
   float* abase = zring + RING * Cfg::slot_floats;
   float* Z0s = abase;               // [C][D]
   float* ZDs = Z0s + C * D;         // [C][D]  z_t / delta_t
   float* Ws = ZDs + C * D;          // [C][CP] K A K^T
   float* Ls = Ws + C * CP;          // [C][CP] unit lower factor
   float* N2p = Ls + C * CP;         // [NWG][C]
-  float* dlt = N2p + NWG * C;       // [C]
+  float* denp = N2p + NWG * C;      // [NWG][C]
+  float* dlt = denp + NWG * C;      // [C]
   float* idl = dlt + C;             // [C]
   float* sbase = abase + Cfg::a_floats;
   float* VS = sbase;                // [C][D]  B = V^T - S K^T
   float* R0s = VS + C * D;          // [C][D]
   float* Eps = R0s + C * D;         // [C][D]
   float* ostage = Eps + C * D;      // [2][C][D]
-  float* denp = ostage + 2 * C * D; // [NWG][C]
-  float* inv_den = denp + NWG * C;  // [C]
   uint64_t* bars = reinterpret_cast<uint64_t*>(
       (reinterpret_cast<uintptr_t>(sbase + Cfg::s_floats) + 15) & ~uintptr_t(15));
   uint64_t* full = bars;                    // [NSTAGE] raw stage filled by TMA
@@ -455,6 +454,9 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       }
     };
 
+    float zk = 0.0f;  // running sum of phi(k), column g
+    if (p.z0) zk = p.z0[size_t(unit) * D + g];
+
     if (nchunks > 0) prep_inputs(0, 0, NWG);
     group_bar(1, NG);
     if (g == 0 && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
@@ -467,7 +469,22 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       float* GuT = Zs + C * D;
       float* HT = GuT + C * CP;
       float* scs = HT + C * CP;
+      float* inv_den = scs + C;
       VLA_MARK(0)
+
+      // ---- running key sum and readout denominators (thread = column g): partial sums
+      //      over this warp's columns of q_f,t . zkey_t
+      if (!ident) {
+        const float* nrm = Kh + 3 * C * D;
+        float pr[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          zk = fmaf(Kh[t * D + g], nrm[t], zk);
+          pr[t] = zk * Qf[t * D + g];
+        }
+        const float tot = warp_reduce_scatter16(pr, lane);
+        if ((lane & 1) == 0) denp[gw * C + (lane >> 1)] = tot;
+      }
 
       // ---- Z0 = A K^T
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) { Z0s[t * D + g] = x; });
@@ -482,6 +499,12 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       // Group S must be done with chunk c - RING: that frees Z slot `slot` and, because
       // KRING = RING + 1, the input slot that chunk c + 1 is about to overwrite.
       if (c >= RING) wait(&ring_empty[slot], ((c / RING) + 1) & 1);
+      if (gw == NWG - 1 && lane < C) {   // denominators of this chunk into the (now free) slot
+        float dd = 0.f;
+#pragma unroll
+        for (int w2 = 0; w2 < NWG; ++w2) dd += denp[w2 * C + lane];
+        inv_den[lane] = ident ? 1.0f : rcp_nr(fmaxf(dd, eps));
+      }
       VLA_MARK(3)
 
       // ---- warp 0: I + W = L diag(delta) L^T.  The other warps widen the next chunk's inputs.
@@ -578,6 +601,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       tile_rank_update<TR, TW, LPR, D, C, true>(st, ZDs, Zs, rb, cg);
       VLA_MARK(7)
     }
+    if (p.zT) p.zT[size_t(unit) * D + g] = zk;
     // final A
     if (p.A_T) {
 #pragma unroll
@@ -591,10 +615,6 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     }
   } else {
     // =====================================================================  group S
-    float zk = 0.0f;  // running sum of phi(k), column g
-    if (p.z0) zk = p.z0[size_t(unit) * D + g];
-    if (g < C) inv_den[g] = 1.0f;
-
     for (int c = 0; c < nchunks; ++c) {
       const int n = min(C, T - c * C);
       const int slot = c % RING;
@@ -604,24 +624,12 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       const float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
       const float* Qf = Kh + C * D;
       const float* Vf = Qf + C * D;
-      const float* nrm = Vf + C * D;
       const float* Zs = zring + size_t(slot) * Cfg::slot_floats;
       const float* GuT = Zs + C * D;
       const float* HT = GuT + C * CP;
       const float* scs = HT + C * CP;
+      const float* inv_den = scs + C;
       VLA_MARK(1)
-
-      // ---- running key sum and readout denominators (thread = column g)
-      if (!ident) {
-        float pr[16];
-#pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          zk = fmaf(Kh[t * D + g], nrm[t], zk);
-          pr[t] = zk * Qf[t * D + g];
-        }
-        const float tot = warp_reduce_scatter16(pr, lane);
-        if ((lane & 1) == 0) denp[gw * C + (lane >> 1)] = tot;
-      }
 
       // ---- B = V^T - S K^T and R0 = S Q^T, row g of each
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) {
@@ -629,13 +637,6 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       });
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
       if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
-      group_bar(2, NG);                 // denp complete
-      if (!ident && g < C) {
-        float dd = 0.f;
-#pragma unroll
-        for (int w2 = 0; w2 < NWG; ++w2) dd += denp[w2 * C + g];
-        inv_den[g] = rcp_nr(fmaxf(dd, eps));
-      }
       VLA_MARK(2)
 
       // ---- row g: e_t = b_t - sum_{s<t} Gu[s][t] e_s; e'_t = sc_t e_t;
@@ -672,14 +673,14 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           o[t] = a0 + a1;
         }
       }
-      group_bar(2, NG);  // inv_den written; Eps complete
+      group_bar(2, NG);  // bulk_wait_read above is ordered before the stage is rewritten
       {
         float* ost = ostage + size_t(c & 1) * C * D;
 #pragma unroll
         for (int t = 0; t < 16; ++t) ost[t * D + g] = o[t] * inv_den[t];
       }
       fence_async_smem();
-      group_bar(2, NG);
+      group_bar(2, NG);  // Eps and the out stage complete
       if (g == 0) {
         bulk_store(gout + size_t(c) * C * D, ostage + size_t(c & 1) * C * D,
                    uint32_t(n) * D * sizeof(float));
@@ -704,7 +705,6 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
               make_float4(st[r][2 * m].x, st[r][2 * m].y, st[r][2 * m + 1].x, st[r][2 * m + 1].y);
       }
     }
-    if (p.zT) p.zT[size_t(unit) * D + g] = zk;
     if (g == 0) bulk_wait_all<0>();
   }
 #ifdef VLA_SECTION_TIMERS

@@ -2,6 +2,7 @@
 // kernel selection and launch.  No allocation, no synchronisation, no global state.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 #include <cstring>
 #include <mutex>
@@ -61,16 +62,49 @@ int launch_token_d(const ScanParams& p, int dtype, cudaStream_t st) {
   return has_u ? launch_token<D, uint16_t, true>(p, st) : launch_token<D, uint16_t, false>(p, st);
 }
 
+// Launch ids for the balanced schedule's hand-off flags (a flag equal to the launch's id
+// means "done"; ids never repeat within 2^32 launches, so the flags never need clearing).
+std::atomic<unsigned int> g_launch_epoch{0};
+
 template <int D, typename TIn>
 int launch_chunk(const ScanParams& p, cudaStream_t st) {
   using Cfg = vla::ChunkCfg<D, TIn>;
-  auto kern = vla::vla_scan_chunk_kernel<D, TIn>;
+  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false>;     // one CTA per unit
+  auto kern_bal = vla::vla_scan_chunk_kernel<D, TIn, true>;  // persistent grid, units cut at chunks
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess ||
+      cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(Cfg::smem_bytes)) != cudaSuccess) {
     cudaGetLastError();
     return VLA_ERR_CUDA;
   }
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  vla::SchedParams sp;
+  sp.balanced = 0;
+  sp.grid = p.units;
+  sp.epoch = 0;
+  // Balanced schedule: only when a plain launch would leave SMs idle in its last wave, every
+  // CTA of the persistent grid is resident at once, and the caller's S_T / A_T / zT can carry
+  // a unit's state from the CTA that starts it to the CTA that finishes it.
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern_bal, Cfg::NT, Cfg::smem_bytes) ==
+          cudaSuccess) {
+    const int resident = sms * per_sm;
+    const bool state_out = p.S_T && p.A_T && (p.zT || (p.flags & VLA_FLAG_IDENTITY_MAP));
+    if (resident > 0 && p.units > resident && p.units % resident != 0 && p.T > 0 && state_out &&
+        p.units <= vla::kSchedMaxUnits) {
+      sp.balanced = 1;
+      sp.grid = resident;
+      unsigned int e = ++g_launch_epoch;
+      if (e == 0) e = ++g_launch_epoch;   // 0 is the flags' initial value
+      sp.epoch = e;
+    }
+  } else {
+    cudaGetLastError();
+  }
+  if (sp.balanced) kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  else kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

@@ -1,7 +1,7 @@
 // VLA forward scan, "chunk" kernel (u = k_hat): the recurrence of Section 3.3 evaluated
 // C = 16 tokens at a time in exact algebra, so that the fp32 FMA pipe works on rank-16
-// updates instead of a chain of rank-1 steps.  One CTA per (batch, head) unit, two warp
-// groups of D threads each:
+// updates instead of a chain of rank-1 steps.  One CTA works on one (batch, head) unit at a
+// time (see "work distribution" below), two warp groups of D threads each:
 //
 //   group A holds A (the inverse penalty matrix) in registers, thread tile TR x TW;
 //   group S holds S (the memory state) in registers, same tiling.
@@ -262,8 +262,78 @@ __device__ __forceinline__ void gram16(const float* X, const float* Y, float* G,
   }
 }
 
-template <int D, typename TIn>
-__global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanParams p) {
+// ---------------------------------------------------------------- work distribution
+// Plain: one CTA per unit.  Balanced: a persistent grid of G co-resident CTAs; the units'
+// chunk sequences are laid end to end and cut into G equal segments, so a unit may be
+// started by one CTA (its "head", executed FIRST by that CTA) and finished by the next
+// (its "tail", executed LAST), with the state handed over through the caller's S_T / A_T /
+// zT buffers and a per-unit flag.  This removes the idle SMs of a last partial wave
+// (512 units on 148 SMs: 3.46 segments of work per SM instead of 4).
+constexpr int kSchedSlots = 16;        // launches whose flags may be live at the same time
+constexpr int kSchedMaxUnits = 4096;   // units per launch in balanced mode
+static __device__ unsigned int g_sched_flags[kSchedSlots * kSchedMaxUnits];
+
+struct SchedParams {
+  int balanced;        // 0: plain, 1: balanced
+  int grid;            // number of CTAs (balanced)
+  unsigned int epoch;  // launch id; flag value that means "head of this unit is done"
+};
+
+struct Piece {
+  int unit, cb, ce;      // chunks [cb, ce) of the unit
+  bool from_handoff;     // state comes from S_T / A_T / zT once the unit's flag shows the epoch
+  bool to_handoff;       // state goes to S_T / A_T / zT and the flag is raised
+};
+
+template <bool BALANCED>
+__device__ __forceinline__ bool get_piece(const SchedParams& sp, int units, int nch, int cta,
+                                          int pi, Piece& out) {
+  if (!BALANCED) {
+    if (pi > 0) return false;
+    out.unit = cta; out.cb = 0; out.ce = nch; out.from_handoff = false; out.to_handoff = false;
+    return true;
+  }
+  const long long N = 1LL * units * nch;
+  const long long lo = cta * N / sp.grid, hi = (cta + 1) * N / sp.grid;
+  if (hi <= lo) return false;
+  const int xf = int(lo / nch), xl = int((hi - 1) / nch);
+  const bool tail = lo > 1LL * xf * nch;                                    // first unit began earlier
+  const bool head = hi < 1LL * (xl + 1) * nch && 1LL * xl * nch >= lo;      // last unit ends later
+  const int wf = xf + (tail ? 1 : 0), wl = xl - (head ? 1 : 0);
+  const int nwhole = wl >= wf ? wl - wf + 1 : 0;
+  if (head) {
+    if (pi == 0) {
+      out.unit = xl; out.cb = 0; out.ce = int(hi - 1LL * xl * nch);
+      out.from_handoff = false; out.to_handoff = true;
+      return true;
+    }
+    --pi;
+  }
+  if (pi < nwhole) {
+    out.unit = wf + pi; out.cb = 0; out.ce = nch; out.from_handoff = false; out.to_handoff = false;
+    return true;
+  }
+  pi -= nwhole;
+  if (tail && pi == 0) {
+    out.unit = xf; out.cb = int(lo - 1LL * xf * nch); out.ce = nch;
+    out.from_handoff = true; out.to_handoff = false;
+    return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+template <int D, typename TIn, bool BALANCED>
+__global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanParams p,
+                                                                  const SchedParams sp) {
   using Cfg = ChunkCfg<D, TIn>;
   constexpr int C = Cfg::C, TW = Cfg::TW, TR = Cfg::TR, LPR = Cfg::LPR, NV = Cfg::NV;
   constexpr int NG = Cfg::NG, NWG = Cfg::NWG, NSTAGE = Cfg::NSTAGE, RING = Cfg::RING;
@@ -303,29 +373,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   const int lane = g & 31, gw = g >> 5;
   const int cg = g % LPR;                // column group
   const int rb = g / LPR;                // row block: rows rb*TR .. rb*TR+TR-1
-  const int unit = blockIdx.x;
-  const int T = p.T;
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
   const float eps = p.eps;
-  const int nchunks = (T + C - 1) / C;
+  const int nch_unit = (p.T + C - 1) / C;   // chunks per unit
+  unsigned int* sched_flags = g_sched_flags + size_t(sp.epoch % kSchedSlots) * kSchedMaxUnits;
 
-  const size_t tok_base = size_t(unit) * size_t(T);
-  const TIn* gq = static_cast<const TIn*>(p.q) + tok_base * D;
-  const TIn* gk = static_cast<const TIn*>(p.k) + tok_base * D;
-  const TIn* gv = static_cast<const TIn*>(p.v) + tok_base * D;
-  float* gout = p.out + tok_base * D;
-
-  auto issue = [&](int c) {
-    const int s = c % NSTAGE;
-    const int n = min(C, T - c * C);
-    const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
-    TIn* dst = raw + size_t(s) * 3 * C * D;
-    const size_t off = size_t(c) * C * D;
-    mbar_arrive_expect_tx(&full[s], 3 * bytes);
-    bulk_load(dst + 0 * C * D, gq + off, bytes, &full[s]);
-    bulk_load(dst + 1 * C * D, gk + off, bytes, &full[s]);
-    bulk_load(dst + 2 * C * D, gv + off, bytes, &full[s]);
-  };
   // Bounded wait shared by every mbarrier in this kernel.
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (*abort_flag) return;
@@ -334,22 +386,82 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       if (p.status) atomicCAS(p.status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
     }
   };
+  if (tid == 0) *abort_flag = 0;
 
+#ifdef VLA_SECTION_TIMERS
+  long long tsec[12];
+  for (int i = 0; i < 12; ++i) tsec[i] = 0;
+  long long tlast = clock64();
+#define VLA_MARK(i) { long long now_ = clock64(); tsec[i] += now_ - tlast; tlast = now_; }
+#else
+#define VLA_MARK(i)
+#endif
+
+  float2 st[TR][TW / 2];   // this thread's TR x TW tile of A (group A) or S (group S), as column pairs
+  Piece pc;
+#pragma unroll 1
+  for (int pi = 0; get_piece<BALANCED>(sp, p.units, nch_unit, blockIdx.x, pi, pc); ++pi) {
+  const int unit = pc.unit;
+  const int t_begin = pc.cb * C;
+  const int T = min(p.T, pc.ce * C) - t_begin;   // tokens of this piece
+  const int nchunks = pc.ce - pc.cb;
+  // A piece either starts its unit (from S0 / A0 / z0) or continues it (from the hand-off),
+  // and either finishes it or hands it over; both kinds of end write S_T / A_T / zT.
+  const bool from_handoff = t_begin > 0;
+  const bool to_handoff = t_begin + T < p.T;
+
+  // global addresses are formed where they are used (two threads of the CTA), so that they
+  // do not occupy registers in the FMA loops
+  auto issue = [&](int c) {
+    const size_t tok = size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+    const int s = c % NSTAGE;
+    const int n = min(C, T - c * C);
+    const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
+    TIn* dst = raw + size_t(s) * 3 * C * D;
+    mbar_arrive_expect_tx(&full[s], 3 * bytes);
+    bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &full[s]);
+    bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &full[s]);
+    bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
+  };
+
+  // (re)arm the barriers of this piece; a tail piece also waits for its unit's head
+  __syncthreads();
   if (tid == 0) {
-    for (int s = 0; s < NSTAGE; ++s) mbar_init(&full[s], 1);
-    for (int r = 0; r < RING; ++r) { mbar_init(&ring_full[r], 1); mbar_init(&ring_empty[r], 1); }
-    *abort_flag = 0;
+    for (int s = 0; s < NSTAGE; ++s) {
+      if (pi > 0) asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&full[s])) : "memory");
+      mbar_init(&full[s], 1);
+    }
+    for (int r = 0; r < RING; ++r) {
+      if (pi > 0) {
+        asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&ring_full[r])) : "memory");
+        asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&ring_empty[r])) : "memory");
+      }
+      mbar_init(&ring_full[r], 1);
+      mbar_init(&ring_empty[r], 1);
+    }
     mbar_init_fence();
+    if (from_handoff && !*abort_flag) {
+      bool seen = false;
+      for (uint32_t it = 0; it < (1u << 24) && !seen; ++it) {
+        seen = ld_acquire_gpu(&sched_flags[unit]) == sp.epoch;
+        if (!seen) __nanosleep(64);
+      }
+      if (!seen) {
+        *abort_flag = 1;
+        if (p.status) atomicCAS(p.status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
+      }
+    }
   }
   __syncthreads();
   if (tid == 0) {  // thread 0 of group A is the TMA producer
     for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue(c);
   }
 
-  // ---- a0: this thread's TR x TW tile of A (group A) or S (group S), as column pairs
-  float2 st[TR][TW / 2];
+  // ---- a0: load the state tile
   {
-    const float* src = is_A ? p.A0 : p.S0;
+    // a tail piece continues from the state its head left in the caller's output buffers
+    // (written by another SM: read past L1)
+    const float* src = from_handoff ? (is_A ? p.A_T : p.S_T) : (is_A ? p.A0 : p.S0);
 #pragma unroll
     for (int r = 0; r < TR; ++r) {
       const int row = rb * TR + r;
@@ -358,7 +470,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         const int c4 = m * LPR + cg;
         float4 x;
         if (src) {
-          x = reinterpret_cast<const float4*>(src + (size_t(unit) * D + row) * D)[c4];
+          x = __ldcg(reinterpret_cast<const float4*>(src + (size_t(unit) * D + row) * D) + c4);
         } else {
           const float dg = is_A ? 1.0f / p.lambda : 0.0f;
           x.x = (c4 * 4 + 0 == row) ? dg : 0.0f;
@@ -371,15 +483,6 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       }
     }
   }
-
-#ifdef VLA_SECTION_TIMERS
-  long long tsec[12];
-  for (int i = 0; i < 12; ++i) tsec[i] = 0;
-  long long tlast = clock64();
-#define VLA_MARK(i) { long long now_ = clock64(); tsec[i] += now_ - tlast; tlast = now_; }
-#else
-#define VLA_MARK(i)
-#endif
 
   if (is_A) {
     // =====================================================================  group A
@@ -455,7 +558,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     };
 
     float zk = 0.0f;  // running sum of phi(k), column g
-    if (p.z0) zk = p.z0[size_t(unit) * D + g];
+    if (from_handoff) {
+      if (p.zT) zk = __ldcg(p.zT + size_t(unit) * D + g);
+    } else if (p.z0) {
+      zk = p.z0[size_t(unit) * D + g];
+    }
 
     if (nchunks > 0) prep_inputs(0, 0, NWG);
     group_bar(1, NG);
@@ -602,7 +709,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       VLA_MARK(7)
     }
     if (p.zT) p.zT[size_t(unit) * D + g] = zk;
-    // final A
+    // final (or handed-over) A
     if (p.A_T) {
 #pragma unroll
       for (int r = 0; r < TR; ++r) {
@@ -682,7 +789,8 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       fence_async_smem();
       group_bar(2, NG);  // Eps and the out stage complete
       if (g == 0) {
-        bulk_store(gout + size_t(c) * C * D, ostage + size_t(c & 1) * C * D,
+        const size_t tok = size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+        bulk_store(p.out + tok * D, ostage + size_t(c & 1) * C * D,
                    uint32_t(n) * D * sizeof(float));
         bulk_commit();
       }
@@ -694,7 +802,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       if (g == 0) mbar_arrive(&ring_empty[slot]);
       VLA_MARK(4)
     }
-    // final S and key sum
+    // final (or handed-over) S
     if (p.S_T) {
 #pragma unroll
       for (int r = 0; r < TR; ++r) {
@@ -707,8 +815,16 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     }
     if (g == 0) bulk_wait_all<0>();
   }
+  if (to_handoff) {   // every thread's state stores precede the flag
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      st_release_gpu(&sched_flags[unit], sp.epoch);
+    }
+  }
+  }  // pieces
 #ifdef VLA_SECTION_TIMERS
-  if (p.dbg && unit == 0 && (g == 0 || g == 32)) {
+  if (p.dbg && blockIdx.x == 0 && (g == 0 || g == 32)) {
     long long* d = p.dbg + ((is_A ? 0 : 2) + (g == 32 ? 1 : 0)) * 12;
     for (int i = 0; i < 12; ++i) d[i] = tsec[i];
   }

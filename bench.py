@@ -336,9 +336,9 @@ def main():
             "frac": (achieved_tflops / fp32_peak_nominal) if bound == "alu" else achieved_gbs / hbm_peak,
             "peak_source": ("fp32 FMA: %d SMs x 128 lanes x 2 x %.0f MHz (derived, nominal max clock)"
                             % (n_sm, sm_max_mhz)) if bound == "alu" else "hbm_gbs of %s" % peak_src,
-            # dram__bytes_read+write of one ncu capture (296 units x 2048 tokens: 767.7 MB),
+            # dram__bytes_read+write of one ncu capture (300 units x 2048 tokens: 817.5 MB),
             # scaled by tokens; see profiles/chunk_kernel_d128_bf16.md
-            "traffic": (767.7e6 / 606208.0) * w.tokens if (w.d == 128 and w.dtype == "bf16") else None,
+            "traffic": (817.5e6 / 614400.0) * w.tokens if (w.d == 128 and w.dtype == "bf16") else None,
             "alg_flops_per_token": alg_flops_per_token(w.d),
             "alg_bytes_per_token": alg_bytes_per_token(w.d, in_bytes),
             "hbm_achieved_gbs": achieved_gbs, "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,

@@ -228,9 +228,9 @@ __device__ __forceinline__ void gram16(const float* X, const float* Y, float* G,
   constexpr int P = NG / 16;
   const int tile = g / P, part = g % P;
   const int i0 = (tile >> 2) * 4, j0 = (tile & 3) * 4;
-  float w[16];
+  float2 w2[16];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) w[i] = 0.f;
+  for (int i = 0; i < 16; ++i) w2[i] = make_float2(0.f, 0.f);
 #pragma unroll
   for (int step = 0; step < D / (4 * P); ++step) {
     const int f = step * P + part;
@@ -244,12 +244,13 @@ __device__ __forceinline__ void gram16(const float* X, const float* Y, float* G,
     for (int i = 0; i < 4; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        w[4 * i + j] = fmaf(a[i].x, b[j].x, w[4 * i + j]);
-        w[4 * i + j] = fmaf(a[i].y, b[j].y, w[4 * i + j]);
-        w[4 * i + j] = fmaf(a[i].z, b[j].z, w[4 * i + j]);
-        w[4 * i + j] = fmaf(a[i].w, b[j].w, w[4 * i + j]);
+        w2[4 * i + j] = ffma2(make_float2(a[i].x, a[i].y), make_float2(b[j].x, b[j].y), w2[4 * i + j]);
+        w2[4 * i + j] = ffma2(make_float2(a[i].z, a[i].w), make_float2(b[j].z, b[j].w), w2[4 * i + j]);
       }
   }
+  float w[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) w[i] = w2[i].x + w2[i].y;
 #pragma unroll
   for (int off = P / 2; off >= 1; off >>= 1)
 #pragma unroll
@@ -489,8 +490,9 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     // Input prep of chunk c by the warps [w0, w0 + nw): k_hat, ||phi(k)||, q_f and v as fp32
     // rows in ring slot c % KRING (zero rows past the end of the sequence).
     auto prep_inputs = [&](int c, int w0, int nw) {
-      constexpr int LPT = 8;        // lanes per token
-      constexpr int NF = D / 32;    // float4 groups per lane and tensor
+      constexpr int LPT = (D >= 128) ? 16 : 8;   // lanes per token
+      constexpr int NF = D / (4 * LPT);          // float4 groups per lane and tensor
+      constexpr int TPW = 32 / LPT;              // tokens per warp pass
       const int s = c % NSTAGE;
       const int n = min(C, T - c * C);
       wait(&full[s], (c / NSTAGE) & 1);
@@ -541,9 +543,9 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         if (pl == 0) nrm[tt] = (tt < n) ? nr : 0.0f;
       };
       // two tokens per lane group and iteration, so that their dependency chains interleave
-      for (int tok0 = (gw - w0) * 4; tok0 < C; tok0 += 2 * nw * 4) {
-        const int ta = tok0 + sub, tb = tok0 + nw * 4 + sub;
-        const bool two = tok0 + nw * 4 < C;   // warp-uniform
+      for (int tok0 = (gw - w0) * TPW; tok0 < C; tok0 += 2 * nw * TPW) {
+        const int ta = tok0 + sub, tb = tok0 + nw * TPW + sub;
+        const bool two = tok0 + nw * TPW < C;   // warp-uniform
         float4 ka[NF], kb[NF];
         float sa = token(ta, ka), sb = 0.f;
         if (two) sb = token(tb, kb);

@@ -97,8 +97,11 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_,
  * q, k, v, opts->u, S0, A0, opts->z0, out, S_T, A_T, opts->zT are HOST pointers (pinned
  * memory makes the copies asynchronous); `workspace` is a DEVICE buffer of at least
  * vla_host_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller.  The call
- * enqueues host->device copies, the scan and device->host copies on `stream` and returns
- * without synchronising; outputs are valid once the stream has been synchronised.
+ * enqueues host->device copies, the scan and device->host copies and returns without
+ * synchronising; everything is ordered after the work already in `stream`, and `stream`
+ * completes only after all of it, so outputs are valid once `stream` has been synchronised.
+ * Batches of at least one unit per SM and 64 MB are pipelined in slices of whole units over
+ * three short-lived internal streams (copy-in, scan and copy-out of different slices overlap).
  * opts->status, when given, stays a DEVICE pointer.
  */
 int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,

@@ -251,31 +251,108 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
   float* dA0 = static_cast<float*>(take(A_b)); float* dAT = static_cast<float*>(take(A_b));
   float* dz0 = static_cast<float*>(take(z_b)); float* dzT = static_cast<float*>(take(z_b));
 
-  bool bad = false;
-  auto h2d = [&](void* d, const void* h, size_t bytes) {
-    if (bytes && cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) bad = true;
-  };
-  auto d2h = [&](void* h, const void* d, size_t bytes) {
-    if (bytes && cudaMemcpyAsync(h, d, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) bad = true;
-  };
-  h2d(dq, q, qk_b); h2d(dk, k, qk_b); h2d(dv, v, v_b);
-  if (o.u) h2d(du, o.u, qk_b);
-  if (S0) h2d(dS0, S0, S_b);
-  if (A0) h2d(dA0, A0, A_b);
-  if (o.z0) h2d(dz0, o.z0, z_b);
-  if (bad) { cudaGetLastError(); return VLA_ERR_CUDA; }
+  // Large batches are cut into slices of whole units that rotate over three internal
+  // streams, so that the copy-in of one slice, the scan of another and the copy-out of a
+  // third overlap (separate copy engines per direction).  Slices keep at least half a unit
+  // per SM; smaller problems run on the caller's stream alone.
+  int nslices = 1;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+      const size_t moved = 2 * qk_b + v_b + o_b;
+      if (moved >= (size_t(64) << 20)) nslices = int(2 * units / size_t(sms));
+      if (nslices < 1) nslices = 1;
+      if (nslices > 8) nslices = 8;
+    } else {
+      cudaGetLastError();
+    }
+  }
+  constexpr int kLanes = 3;
+  cudaStream_t lanes[kLanes] = {st, st, st};
+  cudaEvent_t ev_begin = nullptr, ev_end[kLanes] = {nullptr, nullptr, nullptr};
+  bool own_streams = false;
+  if (nslices > 1) {
+    own_streams = cudaEventCreateWithFlags(&ev_begin, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventRecord(ev_begin, st) == cudaSuccess;
+    for (int i = 0; i < kLanes && own_streams; ++i) {
+      lanes[i] = nullptr;
+      own_streams = cudaStreamCreateWithFlags(&lanes[i], cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&ev_end[i], cudaEventDisableTiming) == cudaSuccess &&
+                    cudaStreamWaitEvent(lanes[i], ev_begin, 0) == cudaSuccess;
+    }
+    if (!own_streams) {   // could not set the lanes up: run everything on the caller's stream
+      cudaGetLastError();
+      for (int i = 0; i < kLanes; ++i) {
+        if (lanes[i] && lanes[i] != st) cudaStreamDestroy(lanes[i]);
+        if (ev_end[i]) cudaEventDestroy(ev_end[i]);
+        lanes[i] = st;
+        ev_end[i] = nullptr;
+      }
+      if (ev_begin) cudaEventDestroy(ev_begin);
+      ev_begin = nullptr;
+      nslices = 1;
+    }
+  }
 
-  vla_opts_t od = o;
-  od.u = du;
-  od.z0 = o.z0 ? dz0 : nullptr;
-  od.zT = o.zT ? dzT : nullptr;
-  rc = vla_forward(dq, dk, dv, lambda_, B, H, T, d_k, d_v, S0 ? dS0 : nullptr, A0 ? dA0 : nullptr,
-                   dout, S_T ? dST : nullptr, A_T ? dAT : nullptr, &od, stream);
-  if (rc != VLA_OK) return rc;
-  d2h(out, dout, o_b);
-  if (S_T) d2h(S_T, dST, S_b);
-  if (A_T) d2h(A_T, dAT, A_b);
-  if (o.zT) d2h(o.zT, dzT, z_b);
+  bool bad = false;
+  int rc_scan = VLA_OK;
+  for (int sl = 0; sl < nslices; ++sl) {
+    const size_t u0 = units * sl / nslices, u1 = units * (sl + 1) / nslices, nu = u1 - u0;
+    cudaStream_t ls = lanes[sl % kLanes];
+    auto h2d = [&](void* d, const void* h, size_t per_unit) {
+      const size_t off = u0 * per_unit, bytes = nu * per_unit;
+      if (bytes && cudaMemcpyAsync(static_cast<unsigned char*>(d) + off,
+                                   static_cast<const unsigned char*>(h) + off, bytes,
+                                   cudaMemcpyHostToDevice, ls) != cudaSuccess) bad = true;
+    };
+    auto d2h = [&](void* h, const void* d, size_t per_unit) {
+      const size_t off = u0 * per_unit, bytes = nu * per_unit;
+      if (bytes && cudaMemcpyAsync(static_cast<unsigned char*>(h) + off,
+                                   static_cast<const unsigned char*>(d) + off, bytes,
+                                   cudaMemcpyDeviceToHost, ls) != cudaSuccess) bad = true;
+    };
+    auto at = [&](void* base, size_t per_unit) {
+      return base ? static_cast<void*>(static_cast<unsigned char*>(base) + u0 * per_unit) : nullptr;
+    };
+    const size_t qk_u = size_t(T) * d_k * es, v_u = size_t(T) * d_v * es, o_u = size_t(T) * d_v * 4;
+    const size_t S_u = size_t(d_v) * d_k * 4, A_u = size_t(d_k) * d_k * 4, z_u = size_t(d_k) * 4;
+    h2d(dq, q, qk_u); h2d(dk, k, qk_u); h2d(dv, v, v_u);
+    if (o.u) h2d(du, o.u, qk_u);
+    if (S0) h2d(dS0, S0, S_u);
+    if (A0) h2d(dA0, A0, A_u);
+    if (o.z0) h2d(dz0, o.z0, z_u);
+    if (bad) break;
+
+    vla_opts_t od = o;
+    od.u = at(du, qk_u);
+    od.z0 = o.z0 ? static_cast<const float*>(at(dz0, z_u)) : nullptr;
+    od.zT = static_cast<float*>(at(dzT, z_u));   // device copies of the final states are always
+                                                 // kept: they let the scan cut units across CTAs
+    rc_scan = vla_forward(at(dq, qk_u), at(dk, qk_u), at(dv, v_u), lambda_, 1, int(nu), T, d_k, d_v,
+                          S0 ? static_cast<const float*>(at(dS0, S_u)) : nullptr,
+                          A0 ? static_cast<const float*>(at(dA0, A_u)) : nullptr,
+                          static_cast<float*>(at(dout, o_u)), static_cast<float*>(at(dST, S_u)),
+                          static_cast<float*>(at(dAT, A_u)), &od, ls);
+    if (rc_scan != VLA_OK) break;
+    d2h(out, dout, o_u);
+    if (S_T) d2h(S_T, dST, S_u);
+    if (A_T) d2h(A_T, dAT, A_u);
+    if (o.zT) d2h(o.zT, dzT, z_u);
+    if (bad) break;
+  }
+  if (own_streams) {
+    // the caller's stream continues only after every lane has drained; destroying a
+    // stream or event with work pending is deferred by the runtime until that work is done
+    for (int i = 0; i < kLanes; ++i) {
+      if (cudaEventRecord(ev_end[i], lanes[i]) != cudaSuccess ||
+          cudaStreamWaitEvent(st, ev_end[i], 0) != cudaSuccess) bad = true;
+      cudaEventDestroy(ev_end[i]);
+      cudaStreamDestroy(lanes[i]);
+    }
+    cudaEventDestroy(ev_begin);
+  }
+  if (rc_scan != VLA_OK) return rc_scan;
   if (bad) { cudaGetLastError(); return VLA_ERR_CUDA; }
   return VLA_OK;
 }

@@ -192,6 +192,35 @@ def test_host_entry_point_matches_device_entry_point():
     assert torch.equal(rh.A_T, rd.A_T.cpu()) and torch.equal(rh.z_T, rd.z_T.cpu())
 
 
+def test_host_entry_point_pipelines_large_batches_in_slices():
+    """Above 64 MB and one unit per SM the host entry point cuts the batch into slices of
+    whole units on three internal streams; results must equal the device entry point's."""
+    dev = torch.device("cuda:0")
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    w = _small(64, 512, "bf16", units=(1, 2 * sms + 5), seed=37)
+    q, k, v = W.make_inputs(w)
+    B, H, T, d = q.shape
+    g = torch.Generator().manual_seed(41)
+    S0 = torch.randn((B, H, d, d), generator=g) * 0.1
+    nbytes = vla.vla_host_workspace_bytes(B, H, T, d, d, vla.VLA_BF16, False)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    pin = lambda x: x.pin_memory()
+    rh = vla.vla_forward_host(pin(q), pin(k), pin(v), 1.0, ws, S0=pin(S0))
+    torch.cuda.synchronize()
+    rd = run_gpu(q, k, v, 1.0, S0=S0)
+    # each slice runs with its own grid, so the cut points of the balanced schedule differ
+    # from the single launch: equal within rounding, not bitwise
+    assert rel_err(rh.out, rd.out.cpu().double().numpy()) <= 1e-5
+    assert rel_err(rh.S_T, rd.S_T.cpu().double().numpy()) <= 1e-5
+    assert rel_err(rh.A_T, rd.A_T.cpu().double().numpy()) <= 1e-5
+    assert rel_err(rh.z_T, rd.z_T.cpu().double().numpy()) <= 1e-5
+    # and against the oracle on a few units of the first and of the last slice
+    for h in (0, 3, H - 1):
+        sl = lambda x: x[:, h:h + 1].contiguous()
+        ref = run_oracle(sl(q), sl(k), sl(v), 1.0, S0=sl(S0))
+        assert rel_err(rh.out[:, h:h + 1], ref.out) <= 1e-4
+
+
 # ---------------------------------------------------------------- the five workloads
 @pytest.mark.parametrize("name", ["tiny", "mid", "recall", "long"])
 @pytest.mark.parametrize("flags", [0, IDENT])

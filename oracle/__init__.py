@@ -44,16 +44,28 @@ class _Trace(ctypes.Structure):
                 ("A", "S", "khat", "u", "alpha", "e", "delta", "den")]
 
 
+class _Refresh(ctypes.Structure):
+    _fields_ = [("period", ctypes.c_int), ("eta", ctypes.c_double), ("step_offset", ctypes.c_long)]
+
+
+def _refresh_arg(refresh):
+    """refresh = None or (period, eta, step_offset)."""
+    if refresh is None:
+        return None
+    period, eta, off = refresh
+    return ctypes.byref(_Refresh(int(period), float(eta), int(off)))
+
+
 def _bind(path):
     lib = ctypes.CDLL(path)
     vp, i, d, u = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_uint
     lib.vla_oracle_forward.restype = i
     lib.vla_oracle_forward.argtypes = [vp, vp, vp, vp, i, d, i, i, i, i, i,
-                                       vp, vp, vp, u, d, vp, vp, vp, vp, i]
+                                       vp, vp, vp, u, d, vp, vp, vp, vp, i, vp]
     lib.vla_oracle_forward_trace.restype = i
     lib.vla_oracle_forward_trace.argtypes = [vp, vp, vp, vp, i, d, i, i, i,
                                              vp, vp, vp, u, d, vp, vp, vp, vp,
-                                             ctypes.POINTER(_Trace)]
+                                             ctypes.POINTER(_Trace), vp]
     return lib
 
 
@@ -97,7 +109,7 @@ class OracleLib:
         self._lib = _bind(path)
 
     def forward(self, q, k, v, lam, *, u=None, in_dtype=F32, S0=None, A0=None, z0=None,
-                flags=0, eps=1e-4, n_threads=1) -> OracleResult:
+                flags=0, eps=1e-4, n_threads=1, refresh=None) -> OracleResult:
         """All units of ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``.
 
         bf16 inputs are passed as uint16 bit patterns (``in_dtype=BF16``).
@@ -119,14 +131,14 @@ class OracleLib:
         rc = lib.vla_oracle_forward(_ptr(q), _ptr(k), _ptr(v), _ptr(u), in_dtype, float(lam),
                                     B, H, T, dk, dv, _ptr(S0), _ptr(A0), _ptr(z0),
                                     flags, float(eps), _ptr(out), _ptr(S_T), _ptr(A_T),
-                                    _ptr(z_T), int(n_threads))
+                                    _ptr(z_T), int(n_threads), _refresh_arg(refresh))
         if rc != 0:
             raise ValueError("vla_oracle_forward: invalid argument")
         return OracleResult(out, S_T, A_T, z_T)
 
 
     def forward_trace(self, q, k, v, lam, *, u=None, in_dtype=F64, S0=None, A0=None, z0=None,
-                      flags=0, eps=1e-4) -> OracleResult:
+                      flags=0, eps=1e-4, refresh=None) -> OracleResult:
         """One unit (``q,k[,u]: [T,d_k]``, ``v: [T,d_v]``) with every per-step quantity dumped."""
         lib = self._lib
         T, dk = np.shape(q)
@@ -149,7 +161,7 @@ class OracleLib:
         rc = lib.vla_oracle_forward_trace(_ptr(q), _ptr(k), _ptr(v), _ptr(u), in_dtype,
                                           float(lam), T, dk, dv, _ptr(S0), _ptr(A0), _ptr(z0),
                                           flags, float(eps), _ptr(out), _ptr(S_T), _ptr(A_T),
-                                          _ptr(z_T), ctypes.byref(ctr))
+                                          _ptr(z_T), ctypes.byref(ctr), _refresh_arg(refresh))
         if rc != 0:
             raise ValueError("vla_oracle_forward_trace: invalid argument")
         return OracleResult(out, S_T, A_T, z_T, tr)

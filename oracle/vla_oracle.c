@@ -6,8 +6,10 @@
  * sequential forward pass"), with three stated departures:
  *   - the projections W_k, W_q, W_v, W_u are not applied: q, k, v (and u when
  *     given) arrive already projected;
- *   - the periodic identity refresh (A += eta*I every 20 steps) is left out,
- *     because it contradicts A_t = M_t^{-1} (Section 1.2, Eq. "A-covariance");
+ *   - the periodic identity refresh (A += eta*I every 20 steps) is off unless the
+ *     caller asks for it, because it contradicts A_t = M_t^{-1} (Section 1.2,
+ *     Eq. "A-covariance"); when on it sits where Algorithm 1 puts it, between the
+ *     Sherman-Morrison step and the write direction;
  *   - both norms are guarded as x / max(||x||, eps) (Section 5.3: "eps for
  *     all denominators").
  * No blocking, fusion or reordering: every matrix-vector product is a double
@@ -23,6 +25,8 @@
  *                Section 3.4, Proposition 1's norm identities.
  *   readout      S_t q_t from dumped states; denominator from a direct sum.
  *   state carry  split invariance.
+ *   refresh      u = 0 closed form, step-by-step brute force with matrix inverses,
+ *                split invariance with the carried step offset.
  * Absolute output values on random data are otherwise fixed by nothing the
  * paper prints ("parity unpinned" beyond the pins above): this file is the
  * definition the CUDA path is compared with.
@@ -63,7 +67,8 @@ static double dot(const double* a, const double* b, int n) {
 static void scan_unit(const void* q, const void* k, const void* v, const void* u_in,
                       size_t qk_off, size_t v_off, int dtype, int T, int dk, int dv,
                       unsigned flags, double eps, double* S, double* A, double* zk,
-                      double* out, const vla_oracle_trace_t* tr) {
+                      double* out, const vla_oracle_trace_t* tr,
+                      const vla_oracle_refresh_t* rf) {
   const int identity = (flags & VLA_ORACLE_IDENTITY_MAP) != 0;
   double* kf = (double*)malloc(sizeof(double) * (size_t)dk);
   double* khat = (double*)malloc(sizeof(double) * (size_t)dk);
@@ -98,6 +103,9 @@ static void scan_unit(const void* q, const void* k, const void* v, const void* u
     if (delta < eps) delta = eps; /* Algorithm 1's clamp; inert since delta >= 1 */
     for (int i = 0; i < dk; ++i)
       for (int j = 0; j < dk; ++j) A[(size_t)i * dk + j] -= zsm[i] * zsm[j] / delta;
+    /* periodic identity refresh (Algorithm 1: "if t mod period = 0 then A <- A + eta I") */
+    if (rf && rf->period > 0 && (rf->step_offset + t + 1) % rf->period == 0)
+      for (int i = 0; i < dk; ++i) A[(size_t)i * dk + i] += rf->eta;
 
     /* --- write direction from the POST-update A_t (Eq. "s-update") --- */
     {
@@ -149,6 +157,7 @@ typedef struct {
   const double *S0, *A0, *z0;
   double *out, *S_T, *A_T, *z_T;
   const vla_oracle_trace_t* tr;
+  const vla_oracle_refresh_t* rf;
   long unit_begin, unit_end;
 } job_t;
 
@@ -172,7 +181,7 @@ static void* run_units(void* arg) {
 
     scan_unit(jb->q, jb->k, jb->v, jb->u, (size_t)n * T * dk, (size_t)n * T * dv, jb->dtype,
               jb->T, jb->dk, jb->dv, jb->flags, jb->eps, S, A, zk,
-              jb->out + (size_t)n * T * dv, jb->tr);
+              jb->out + (size_t)n * T * dv, jb->tr, jb->rf);
 
     if (jb->S_T) memcpy(jb->S_T + (size_t)n * dv * dk, S, sizeof(double) * dv * dk);
     if (jb->A_T) memcpy(jb->A_T + (size_t)n * dk * dk, A, sizeof(double) * dk * dk);
@@ -198,7 +207,7 @@ int vla_oracle_forward(const void* q, const void* k, const void* v, const void* 
                        int in_dtype, double lambda, int B, int H, int T, int d_k, int d_v,
                        const double* S0, const double* A0, const double* z0, unsigned flags,
                        double eps, double* out, double* S_T, double* A_T, double* z_T,
-                       int n_threads) {
+                       int n_threads, const vla_oracle_refresh_t* refresh) {
   if (B < 0 || H < 0) return -1;
   const long units = (long)B * (long)H;
   if (check_args(q, k, v, in_dtype, lambda, units, T, d_k, d_v, A0, eps, out)) return -1;
@@ -207,7 +216,7 @@ int vla_oracle_forward(const void* q, const void* k, const void* v, const void* 
   if (n_threads > units) n_threads = (int)units;
 
   job_t base = {q, k, v, u, in_dtype, T, d_k, d_v, lambda, eps, flags,
-                S0, A0, z0, out, S_T, A_T, z_T, NULL, 0, 0};
+                S0, A0, z0, out, S_T, A_T, z_T, NULL, refresh, 0, 0};
   if (n_threads == 1) {
     base.unit_begin = 0;
     base.unit_end = units;
@@ -231,10 +240,11 @@ int vla_oracle_forward_trace(const void* q, const void* k, const void* v, const 
                              int in_dtype, double lambda, int T, int d_k, int d_v,
                              const double* S0, const double* A0, const double* z0,
                              unsigned flags, double eps, double* out, double* S_T,
-                             double* A_T, double* z_T, const vla_oracle_trace_t* trace) {
+                             double* A_T, double* z_T, const vla_oracle_trace_t* trace,
+                             const vla_oracle_refresh_t* refresh) {
   if (check_args(q, k, v, in_dtype, lambda, 1, T, d_k, d_v, A0, eps, out)) return -1;
   job_t jb = {q, k, v, u, in_dtype, T, d_k, d_v, lambda, eps, flags,
-              S0, A0, z0, out, S_T, A_T, z_T, trace, 0, 1};
+              S0, A0, z0, out, S_T, A_T, z_T, trace, refresh, 0, 1};
   run_units(&jb);
   return 0;
 }

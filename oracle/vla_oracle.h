@@ -35,6 +35,16 @@ enum {
   VLA_ORACLE_IDENTITY_MAP = 1u << 0
 };
 
+/* Algorithm 1's periodic identity refresh: after the Sherman-Morrison step of the token whose
+   1-based position in the whole sequence is a multiple of `period`, A += eta * I.  The paper
+   uses period 20, eta 1e-3 (Section 5.3).  `step_offset` = tokens of the sequence processed
+   before this call (for carried state).  NULL or period <= 0: no refresh. */
+typedef struct {
+  int period;
+  double eta;
+  long step_offset;
+} vla_oracle_refresh_t;
+
 /* Optional per-step dump of one unit (any pointer may be NULL). */
 typedef struct {
   double* A;      /* [T, d_k, d_k]  A_t after the Sherman-Morrison step            */
@@ -60,7 +70,7 @@ int vla_oracle_forward(const void* q, const void* k, const void* v, const void* 
                        const double* S0, const double* A0, const double* z0,
                        unsigned flags, double eps,
                        double* out, double* S_T, double* A_T, double* z_T,
-                       int n_threads);
+                       int n_threads, const vla_oracle_refresh_t* refresh);
 
 /* Same recurrence for ONE unit (B = H = 1) with a per-step trace. */
 int vla_oracle_forward_trace(const void* q, const void* k, const void* v, const void* u,
@@ -68,7 +78,8 @@ int vla_oracle_forward_trace(const void* q, const void* k, const void* v, const 
                              const double* S0, const double* A0, const double* z0,
                              unsigned flags, double eps,
                              double* out, double* S_T, double* A_T, double* z_T,
-                             const vla_oracle_trace_t* trace);
+                             const vla_oracle_trace_t* trace,
+                             const vla_oracle_refresh_t* refresh);
 
 #ifdef __cplusplus
 }

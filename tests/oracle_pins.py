@@ -376,9 +376,75 @@ def pin_paper_constants(orc, golden):
     assert np.all(r.S_T == 0) and np.all(r.z_T == 0)
 
 
+# --------------------------------------------------------------------------
+# periodic identity refresh (Algorithm 1; Section 5.3: every 20 steps, + 1e-3 I)
+# --------------------------------------------------------------------------
+def pin_refresh_closed_form_with_zero_u(orc):
+    """u = 0 leaves only the refresh: A_T = A_0 + (number of refresh steps) * eta * I, counted on
+    the 1-based global position (carried step offset), and S still follows the normalised
+    delta rule because A stays a multiple of I."""
+    dk, dv, T, lam, eta, period = 5, 4, 47, 0.1, 1e-3, 20
+    q, k, v, g = _rand(201, T, dk, dv)
+    for off in (0, 7, 19, 33):
+        r = orc.forward_trace(q, k, v, lam, u=np.zeros((T, dk)), flags=IDENT, refresh=(period, eta, off))
+        n_ref = (off + T) // period - off // period
+        assert np.abs(r.A_T - (1 / lam + n_ref * eta) * np.eye(dk)).max() < 1e-12
+        for t in range(T):
+            n_t = (off + t + 1) // period - off // period
+            assert np.abs(r.trace["A"][t] - (1 / lam + n_t * eta) * np.eye(dk)).max() < 1e-12
+        S = np.zeros((dv, dk))
+        for t in range(T):
+            kh = k[t] / np.linalg.norm(k[t])
+            S = S + np.outer(v[t] - S @ kh, kh)
+        assert np.abs(r.S_T - S).max() < 1e-12
+    # a period longer than the sequence, or period 0, changes nothing
+    base = orc.forward_trace(q, k, v, lam, flags=0)
+    for rf in ((T + 1, eta, 0), (0, eta, 0), None):
+        r = orc.forward_trace(q, k, v, lam, flags=0, refresh=rf)
+        assert np.array_equal(r.out, base.out) and np.array_equal(r.A_T, base.A_T)
+
+
+def pin_refresh_step_by_step_brute_force(orc):
+    """A_t = (A_{t-1}^{-1} + u u^T)^{-1}, plus eta*I on refresh steps, with numpy inverses;
+    the write direction uses the refreshed A_t (the refresh sits before it in Algorithm 1)."""
+    dk, T, lam, eta, period = 6, 45, 0.2, 1e-3, 20
+    q, k, v, g = _rand(211, T, dk, dk)
+    for uu in (None, _unit(g.standard_normal((T, dk)))):
+        r = orc.forward_trace(q, k, v, lam, u=uu, flags=0, refresh=(period, eta, 0))
+        kh = _khat(k, 0)
+        used = kh if uu is None else uu
+        A = np.eye(dk) / lam
+        for t in range(T):
+            A = np.linalg.inv(np.linalg.inv(A) + np.outer(used[t], used[t]))
+            if (t + 1) % period == 0:
+                A = A + eta * np.eye(dk)
+            assert np.abs(r.trace["A"][t] - A).max() < 1e-10 * np.abs(A).max(), t
+            a = A @ kh[t]
+            assert np.abs(r.trace["alpha"][t] - a / np.linalg.norm(a)).max() < 1e-10, t
+
+
+def pin_refresh_state_carry(orc):
+    """Split invariance needs the step offset to be carried along with (S, A, z)."""
+    B, H, T, dk, dv, lam = 1, 2, 53, 5, 4, 0.1
+    g = np.random.default_rng(221)
+    q = g.standard_normal((B, H, T, dk)); k = g.standard_normal((B, H, T, dk))
+    v = g.standard_normal((B, H, T, dv))
+    full = orc.forward(q, k, v, lam, in_dtype=2, refresh=(20, 1e-3, 0))
+    for T1 in (13, 20, 40):
+        a = orc.forward(q[:, :, :T1], k[:, :, :T1], v[:, :, :T1], lam, in_dtype=2, refresh=(20, 1e-3, 0))
+        b = orc.forward(q[:, :, T1:], k[:, :, T1:], v[:, :, T1:], lam, in_dtype=2, S0=a.S_T, A0=a.A_T,
+                        z0=a.z_T, refresh=(20, 1e-3, T1))
+        assert np.abs(np.concatenate([a.out, b.out], axis=2) - full.out).max() < 1e-12
+        assert np.abs(b.A_T - full.A_T).max() < 1e-12 and np.abs(b.S_T - full.S_T).max() < 1e-12
+    wrong = orc.forward(q[:, :, 13:], k[:, :, 13:], v[:, :, 13:], lam, in_dtype=2, refresh=(20, 1e-3, 0))
+    assert np.abs(wrong.A_T - full.A_T).max() > 1e-6      # offset matters
+
+
 PINS = [pin_A_is_brute_force_inverse, pin_A_invariants, pin_delta_value,
         pin_alpha_from_post_update_A, pin_first_step_closed_form,
         pin_orthonormal_keys_exact_recall, pin_repeated_key,
         pin_zero_u_is_normalised_delta_rule, pin_associative_composition,
         pin_proposition_1, pin_readout, pin_feature_map_values, pin_eps_guards,
-        pin_state_carry, pin_units_layout_threads_dtypes, pin_jacobian_spectrum]
+        pin_state_carry, pin_units_layout_threads_dtypes, pin_jacobian_spectrum,
+        pin_refresh_closed_form_with_zero_u, pin_refresh_step_by_step_brute_force,
+        pin_refresh_state_carry]

@@ -39,8 +39,12 @@ MUTANTS = [
     ("A0_is_lambda_I", "A[i * dk + i] = 1.0 / jb->lambda;", "A[i * dk + i] = jb->lambda;"),
     ("z0_ignored", "if (jb->z0) memcpy(zk,", "if (0) memcpy(zk,"),
     ("S0_ignored", "if (jb->S0) memcpy(S,", "if (0) memcpy(S,"),
-    ("out_unit_stride", "jb->out + (size_t)n * T * dv, jb->tr);", "jb->out + (size_t)n * T * dk, jb->tr);"),
+    ("out_unit_stride", "jb->out + (size_t)n * T * dv, jb->tr, jb->rf);", "jb->out + (size_t)n * T * dk, jb->tr, jb->rf);"),
     ("bf16_shift", "[idx] << 16;", "[idx] << 15;"),
+    ("refresh_wrong_step", "(rf->step_offset + t + 1) % rf->period == 0", "(rf->step_offset + t) % rf->period == 0"),
+    ("refresh_ignores_offset", "(rf->step_offset + t + 1) % rf->period == 0", "(t + 1) % rf->period == 0"),
+    ("refresh_sign", "A[(size_t)i * dk + i] += rf->eta;", "A[(size_t)i * dk + i] -= rf->eta;"),
+    ("refresh_every_step", "rf->period > 0 && (rf->step_offset + t + 1) % rf->period == 0", "rf->period > 0"),
     ("eps_guard_missing", "double g = nrm > eps ? nrm : eps;\n      for (int j = 0; j < dk; ++j) khat[j]",
      "double g = nrm;\n      for (int j = 0; j < dk; ++j) khat[j]"),
 ]

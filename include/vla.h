@@ -70,6 +70,13 @@ typedef struct {
   int32_t* status;       /* device int32, 0 on entry; set to a negative vla_status_t on a
                             device-side problem.  Read it after synchronising.  NULL allowed    */
   int32_t kernel;        /* vla_kernel_t                                                        */
+  /* Algorithm 1's periodic identity refresh (Section 5.3: every 20 steps, + 1e-3 I): after
+     the Sherman-Morrison step of each token whose 1-based position in the whole sequence
+     (step_offset + t + 1) is a multiple of refresh_period, A += refresh_eta * I.  Off when
+     refresh_period <= 0 (the default: it breaks A_t = M_t^-1).  Runs on the token kernel.   */
+  int32_t refresh_period;
+  float refresh_eta;
+  int64_t step_offset;   /* tokens of this sequence processed by earlier calls (state carry)     */
 } vla_opts_t;
 
 /*

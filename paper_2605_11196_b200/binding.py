@@ -33,7 +33,8 @@ class VlaOpts(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_uint32), ("qkv_dtype", ctypes.c_int32),
                 ("u", ctypes.c_void_p), ("flags", ctypes.c_uint32), ("eps", ctypes.c_float),
                 ("z0", ctypes.c_void_p), ("zT", ctypes.c_void_p), ("status", ctypes.c_void_p),
-                ("kernel", ctypes.c_int32)]
+                ("kernel", ctypes.c_int32), ("refresh_period", ctypes.c_int32),
+                ("refresh_eta", ctypes.c_float), ("step_offset", ctypes.c_int64)]
 
 
 class VlaError(RuntimeError):
@@ -133,7 +134,7 @@ class VlaResult:
     status: Optional[torch.Tensor]  # device int32 scalar; read after synchronising
 
 
-def _make_opts(dt, u, flags, eps, z0, zT, status, kernel):
+def _make_opts(dt, u, flags, eps, z0, zT, status, kernel, refresh=None):
     o = VlaOpts()
     o.struct_size = ctypes.sizeof(VlaOpts)
     o.qkv_dtype = dt
@@ -144,13 +145,15 @@ def _make_opts(dt, u, flags, eps, z0, zT, status, kernel):
     o.zT = None if zT is None else zT.data_ptr()
     o.status = None if status is None else status.data_ptr()
     o.kernel = kernel
+    if refresh is not None:     # (period, eta, step_offset): Algorithm 1's periodic A += eta I
+        o.refresh_period, o.refresh_eta, o.step_offset = int(refresh[0]), float(refresh[1]), int(refresh[2])
     return o
 
 
 def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags: int = 0,
                 eps: float = 1e-4, out=None, S_T=None, A_T=None, z_T=None, status=None,
                 kernel: int = VLA_KERNEL_AUTO, stream: Optional[torch.cuda.Stream] = None,
-                want_status: bool = True) -> VlaResult:
+                want_status: bool = True, refresh=None) -> VlaResult:
     """Enqueue the scan for CUDA tensors ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``.
 
     Output tensors are allocated with torch unless passed in.  Nothing is synchronised.
@@ -180,7 +183,7 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
     if status is None and want_status:
         status = torch.zeros((), dtype=torch.int32, device=dev)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
-    opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel)
+    opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel, refresh)
     with torch.cuda.device(dev):
         rc = lib.vla_forward(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv,
                              _ptr(S0), _ptr(A0), _ptr(out), _ptr(S_T), _ptr(A_T),

@@ -33,6 +33,8 @@ int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
   if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_INVALID_ARG;
   if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN && r->kernel != VLA_KERNEL_CHUNK)
     return VLA_ERR_INVALID_ARG;
+  if (r->refresh_period > 0 && (r->step_offset < 0 || !(r->refresh_eta == r->refresh_eta)))
+    return VLA_ERR_INVALID_ARG;
   return VLA_OK;
 }
 
@@ -55,7 +57,14 @@ int launch_token(const ScanParams& p, cudaStream_t st) {
 }
 
 template <int D>
-int launch_token_d(const ScanParams& p, int dtype, cudaStream_t st) {
+int launch_token_d(const ScanParams& p_in, int dtype, cudaStream_t st) {
+  // The periodic refresh lives in the two-exchange variant (the write direction is no longer
+  // parallel to z on a refresh step); without an explicit u that variant is told to use k_hat.
+  ScanParams p = p_in;
+  if (p.refresh_period > 0 && p.u == nullptr) {
+    p.u = p.k;   // a valid address for the ring's fourth tensor; its contents are not used
+    p.u_is_khat = 1;
+  }
   const bool has_u = p.u != nullptr;
   if (dtype == VLA_F32)
     return has_u ? launch_token<D, float, true>(p, st) : launch_token<D, float, false>(p, st);
@@ -115,7 +124,9 @@ int launch_chunk_d(const ScanParams& p, int dtype, cudaStream_t st) {
 
 // The chunk kernel covers u = k_hat and d in {32, 64, 128}; everything else runs on the
 // token kernel.  Both are CUDA paths; there is no host fallback.
-bool chunk_covers(const ScanParams& p, int d) { return p.u == nullptr && d >= 32; }
+bool chunk_covers(const ScanParams& p, int d) {
+  return p.u == nullptr && d >= 32 && p.refresh_period <= 0;
+}
 
 int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
   bool chunk = chunk_covers(p, d);
@@ -207,6 +218,8 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
   p.status = o.status;
   p.lambda = lambda_; p.eps = o.eps;
   p.T = T; p.units = units; p.flags = o.flags;
+  p.refresh_period = o.refresh_period; p.refresh_eta = o.refresh_eta;
+  p.step_offset = o.step_offset; p.u_is_khat = 0;
   return launch(p, d_k, o.qkv_dtype, o.kernel, static_cast<cudaStream_t>(stream));
 }
 

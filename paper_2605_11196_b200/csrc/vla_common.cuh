@@ -27,6 +27,10 @@ struct ScanParams {
   int T;
   int units;
   uint32_t flags;
+  int refresh_period;        // <= 0: no periodic refresh of A
+  float refresh_eta;
+  long long step_offset;     // tokens processed before this call
+  int u_is_khat;             // token kernel, two-exchange path: use u = k_hat although no u was given
 #ifdef VLA_SECTION_TIMERS
   long long* dbg;      // debug builds only: per-section clock64 totals of unit 0
 #endif

@@ -180,7 +180,9 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
         if (!ident) reinterpret_cast<float4*>(w_kf + ptok * D)[pc4] = kf;
         if (HAS_U) {
           const TIn* ru = raw + (size_t(s) * NIN + 3) * C * D + ptok * D;
-          reinterpret_cast<float4*>(w_u + ptok * D)[pc4] = load4(ru, pc4);
+          reinterpret_cast<float4*>(w_u + ptok * D)[pc4] =
+              p.u_is_khat ? make_float4(kf.x * inv, kf.y * inv, kf.z * inv, kf.w * inv)
+                          : load4(ru, pc4);
         }
       }
       if (!ident) {
@@ -281,8 +283,11 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
             !isfinite(t0 + t1 + t2))
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
       } else {
-        // a = A_t k_hat = A_{t-1} k_hat - z (k_hat.z)/delta
-        const float ai = fmaf(-zi, t1 * inv_d, wi);
+        // a = A_t k_hat = A_{t-1} k_hat - z (k_hat.z)/delta  (+ eta k_hat on a refresh step)
+        float ai = fmaf(-zi, t1 * inv_d, wi);
+        const bool refresh_now = p.refresh_period > 0 &&
+            (p.step_offset + (long long)c * C + t + 1) % p.refresh_period == 0;
+        if (refresh_now) ai = fmaf(p.refresh_eta, khi, ai);
         float a0 = ai * ai, a1 = ai * qi;
 #pragma unroll
         for (int off = 4; off <= 16; off <<= 1) {
@@ -307,6 +312,10 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
       }
       const float* zvec = zbuf + b * D;
+      // Algorithm 1's periodic refresh: A += eta I right after the rank-1 downdate
+      const float diag_add = (HAS_U && p.refresh_period > 0 &&
+                              (p.step_offset + (long long)c * C + t + 1) % p.refresh_period == 0)
+                                 ? p.refresh_eta : 0.0f;
 #pragma unroll
       for (int m = 0; m < NV; ++m) {
         const int c4 = m * 4 + j;
@@ -315,6 +324,12 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
         if (HAS_U) a4 = reinterpret_cast<const float4*>(wvec)[c4];
         A[4 * m + 0] = fmaf(-zs, z4.x, A[4 * m + 0]); A[4 * m + 1] = fmaf(-zs, z4.y, A[4 * m + 1]);
         A[4 * m + 2] = fmaf(-zs, z4.z, A[4 * m + 2]); A[4 * m + 3] = fmaf(-zs, z4.w, A[4 * m + 3]);
+        if (HAS_U) {
+          A[4 * m + 0] += (c4 * 4 + 0 == i) ? diag_add : 0.0f;
+          A[4 * m + 1] += (c4 * 4 + 1 == i) ? diag_add : 0.0f;
+          A[4 * m + 2] += (c4 * 4 + 2 == i) ? diag_add : 0.0f;
+          A[4 * m + 3] += (c4 * 4 + 3 == i) ? diag_add : 0.0f;
+        }
         S[4 * m + 0] = fmaf(es, a4.x, S[4 * m + 0]); S[4 * m + 1] = fmaf(es, a4.y, S[4 * m + 1]);
         S[4 * m + 2] = fmaf(es, a4.z, S[4 * m + 2]); S[4 * m + 3] = fmaf(es, a4.w, S[4 * m + 3]);
       }

@@ -20,14 +20,14 @@ def to_oracle_array(t: torch.Tensor):
     return t.numpy(), oracle.F32
 
 
-def run_oracle(q, k, v, lam, u=None, S0=None, A0=None, z0=None, flags=0, eps=1e-4):
+def run_oracle(q, k, v, lam, u=None, S0=None, A0=None, z0=None, flags=0, eps=1e-4, refresh=None):
     qa, dt = to_oracle_array(q)
     ka, _ = to_oracle_array(k)
     va, _ = to_oracle_array(v)
     ua = None if u is None else to_oracle_array(u)[0]
     f64 = lambda x: None if x is None else x.detach().cpu().double().numpy()
     return oracle.forward(qa, ka, va, lam, u=ua, in_dtype=dt, S0=f64(S0), A0=f64(A0), z0=f64(z0),
-                          flags=flags, eps=eps, n_threads=NTHREADS)
+                          flags=flags, eps=eps, n_threads=NTHREADS, refresh=refresh)
 
 
 def rel_err(x_gpu: torch.Tensor, x_ref: np.ndarray) -> float:
@@ -41,20 +41,20 @@ def rel_err(x_gpu: torch.Tensor, x_ref: np.ndarray) -> float:
     return float(np.abs(x - x_ref).max() / (den if den > 0 else 1.0))
 
 
-def run_gpu(q, k, v, lam, u=None, S0=None, A0=None, z0=None, flags=0, eps=1e-4, kernel=0):
+def run_gpu(q, k, v, lam, u=None, S0=None, A0=None, z0=None, flags=0, eps=1e-4, kernel=0, refresh=None):
     dev = torch.device("cuda:0")
     mv = lambda x: None if x is None else x.to(dev).contiguous()
     r = vla.vla_forward(mv(q), mv(k), mv(v), lam, u=mv(u), S0=mv(S0), A0=mv(A0), z0=mv(z0),
-                        flags=flags, eps=eps, kernel=kernel)
+                        flags=flags, eps=eps, kernel=kernel, refresh=refresh)
     torch.cuda.synchronize()
     assert int(r.status.item()) == 0, vla.status_string(int(r.status.item()))
     return r
 
 
 def check_parity(q, k, v, lam, tol, *, u=None, S0=None, A0=None, z0=None, flags=0, eps=1e-4,
-                 kernel=0, label=""):
-    ref = run_oracle(q, k, v, lam, u, S0, A0, z0, flags, eps)
-    got = run_gpu(q, k, v, lam, u, S0, A0, z0, flags, eps, kernel)
+                 kernel=0, label="", refresh=None):
+    ref = run_oracle(q, k, v, lam, u, S0, A0, z0, flags, eps, refresh)
+    got = run_gpu(q, k, v, lam, u, S0, A0, z0, flags, eps, kernel, refresh)
     errs = {"o": rel_err(got.out, ref.out), "S_T": rel_err(got.S_T, ref.S_T),
             "A_T": rel_err(got.A_T, ref.A_T), "z_T": rel_err(got.z_T, ref.z_T)}
     for name, e in errs.items():

@@ -123,6 +123,34 @@ def test_more_units_than_resident_ctas(d, units, flags):
     assert rel_err(tok.out, ref.out) <= 1e-4
 
 
+@pytest.mark.parametrize("d", [16, 32, 128])
+@pytest.mark.parametrize("flags", [0, IDENT])
+@pytest.mark.parametrize("umode", ["khat", "unit_over_sqrt_d"])
+def test_periodic_refresh_as_in_algorithm_1(d, flags, umode):
+    """Algorithm 1 to the letter: lambda_0 = 0.1, A += 1e-3 I every 20 steps, with and without an
+    explicit u, in one call and split in two with the step offset carried."""
+    w = _small(d, 130, "f32", units=(1, 3), seed=500 + d)
+    q, k, v = W.make_inputs(w)
+    u = None if umode == "khat" else W.make_u(w, d ** -0.5)
+    rf = (20, 1e-3, 0)
+    errs, got, ref = check_parity(q, k, v, 0.1, 1e-4, u=u, flags=flags, refresh=rf, label="refresh d=%d" % d)
+    plain = run_oracle(q, k, v, 0.1, u=u, flags=flags)
+    assert np.abs(plain.A_T - ref.A_T).max() > 1e-4           # the refresh is visible in A_T
+    T1 = 53
+    sl = lambda x, a, b: None if x is None else x[:, :, a:b].contiguous()
+    a = run_gpu(sl(q, 0, T1), sl(k, 0, T1), sl(v, 0, T1), 0.1, u=sl(u, 0, T1), flags=flags, refresh=rf)
+    b = run_gpu(sl(q, T1, 130), sl(k, T1, 130), sl(v, T1, 130), 0.1, u=sl(u, T1, 130), flags=flags,
+                S0=a.S_T, A0=a.A_T, z0=a.z_T, refresh=(20, 1e-3, T1))
+    assert rel_err(torch.cat([a.out, b.out], dim=2), ref.out) <= 1e-4
+    assert rel_err(b.A_T, ref.A_T) <= 1e-4 and rel_err(b.S_T, ref.S_T) <= 1e-4
+    # the chunk kernel does not implement the refresh and says so when forced
+    if d >= 32 and u is None:
+        dev = torch.device("cuda:0")
+        with pytest.raises(vla.VlaError) as ei:
+            vla.vla_forward(q.to(dev), k.to(dev), v.to(dev), 0.1, refresh=rf, kernel=vla.VLA_KERNEL_CHUNK)
+        assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+
+
 def test_in_place_state_and_canaries():
     """S_T/A_T may alias S0/A0; nothing is written outside the output tensors."""
     dev = torch.device("cuda:0")

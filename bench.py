@@ -387,6 +387,33 @@ def main():
                          "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
                          "hbm_frac": alg_bytes_per_token(ww.d, ib) * ww.tokens / (ms * 1e-3) / 1e9 / hbm_peak,
                          "units": ww.units, "unit_limited_frac_bound": min(ww.units, n_sm) / n_sm}
+        # single-step decode (T = 1, carried states): bound by moving S and A through HBM once
+        wd = W.EXTRA["decode"]
+        q2, k2, v2 = [x.to(dev) for x in W.make_inputs(wd)]
+        S0 = torch.zeros((wd.B, wd.H, wd.d, wd.d), device=dev)
+        A0 = torch.eye(wd.d, device=dev).expand(wd.B, wd.H, wd.d, wd.d).contiguous()
+        bufs = dict(out=torch.empty((wd.B, wd.H, 1, wd.d), device=dev), S_T=torch.empty_like(S0),
+                    A_T=torch.empty_like(A0), z_T=torch.empty((wd.B, wd.H, wd.d), device=dev), status=status)
+        dcall = lambda: vla.vla_forward(q2, k2, v2, wd.lam, S0=S0, A0=A0, stream=stream, **bufs)
+        fl = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+        evs = []
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                dcall()
+            for _ in range(10):
+                fl.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); dcall(); b.record(stream)
+                evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+        state_bytes = wd.units * (4 * wd.d * wd.d * 4 + 2 * wd.d * 4)       # S, A read and written; z
+        io_bytes = wd.units * (3 * wd.d * 2 + wd.d * 4)
+        per["decode"] = {"ms": ms, "units": wd.units, "steps_per_s": wd.units / (ms * 1e-3),
+                         "kernel": "vla_scan_token_kernel", "bound": "hbm",
+                         "hbm_gbs": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9,
+                         "hbm_frac": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9 / hbm_peak,
+                         "hbm_peak_source": peak_src}
         line["per_workload"] = per
 
     if not args.no_cpu_baseline:

@@ -128,9 +128,15 @@ bool chunk_covers(const ScanParams& p, int d) {
   return p.u == nullptr && d >= 32 && p.refresh_period <= 0;
 }
 
+// Very short sequences (single-step decode and the like) are bound by reading and writing
+// the states once; there the token kernel is faster than a 16-token chunk that is mostly
+// padding (measured crossover: T ~ 12 at d = 128, T ~ 20 at d = 64).
+bool chunk_pays_off(const ScanParams& p, int d) { return p.T > (d >= 128 ? 8 : 16); }
+
 int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
   bool chunk = chunk_covers(p, d);
   if (kernel == VLA_KERNEL_CHUNK && !chunk) return VLA_ERR_UNSUPPORTED;
+  if (kernel == VLA_KERNEL_AUTO && !chunk_pays_off(p, d)) chunk = false;
   if (kernel == VLA_KERNEL_TOKEN) chunk = false;
   if (chunk) {
     switch (d) {

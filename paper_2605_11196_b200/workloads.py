@@ -63,6 +63,9 @@ WORKLOADS = {
     "throughput": Workload("throughput", 32, 16, 128, 8192, "bf16", 4),
 }
 ORDER = ("tiny", "mid", "recall", "long", "throughput")
+# Not one of the five: a single-step decode shape (state read and written once per unit),
+# reported by bench.py --all-workloads against the HBM roofline.
+EXTRA = {"decode": Workload("decode", 64, 64, 128, 1, "bf16", 5)}
 
 
 def scaled(w: Workload, **kw) -> Workload:

@@ -86,13 +86,17 @@ def test_state_carry_split_invariance():
     u = W.make_u(w)
     for flags in (0, IDENT):
         for uu in (None, u):
-            full = run_gpu(q, k, v, 0.1, u=uu, flags=flags)
+            # one kernel for all three calls (AUTO would pick by length), so that a
+            # chunk-aligned split can be compared bit for bit
+            kern = vla.VLA_KERNEL_CHUNK if uu is None else vla.VLA_KERNEL_TOKEN
+            full = run_gpu(q, k, v, 0.1, u=uu, flags=flags, kernel=kern)
             ref = run_oracle(q, k, v, 0.1, u=uu, flags=flags)
             for T1 in (16, 37, 64):
                 sl = lambda x, a, b: None if x is None else x[:, :, a:b].contiguous()
-                a = run_gpu(sl(q, 0, T1), sl(k, 0, T1), sl(v, 0, T1), 0.1, u=sl(uu, 0, T1), flags=flags)
+                a = run_gpu(sl(q, 0, T1), sl(k, 0, T1), sl(v, 0, T1), 0.1, u=sl(uu, 0, T1), flags=flags,
+                            kernel=kern)
                 b = run_gpu(sl(q, T1, 100), sl(k, T1, 100), sl(v, T1, 100), 0.1, u=sl(uu, T1, 100),
-                            S0=a.S_T, A0=a.A_T, z0=a.z_T, flags=flags)
+                            S0=a.S_T, A0=a.A_T, z0=a.z_T, flags=flags, kernel=kern)
                 cat = torch.cat([a.out, b.out], dim=2)
                 assert rel_err(cat, ref.out) <= 1e-4
                 assert rel_err(b.S_T, ref.S_T) <= 1e-4 and rel_err(b.A_T, ref.A_T) <= 1e-4

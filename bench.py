@@ -387,6 +387,26 @@ def main():
                          "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
                          "hbm_frac": alg_bytes_per_token(ww.d, ib) * ww.tokens / (ms * 1e-3) / 1e9 / hbm_peak,
                          "units": ww.units, "unit_limited_frac_bound": min(ww.units, n_sm) / n_sm}
+        # the headline workload with an explicit penalty direction u = unit / sqrt(d_h)
+        # (the paper's learned-u setting at the scan's input level)
+        uu = W.make_u(w, w.d ** -0.5).to(dev)
+        ucall = lambda: vla.vla_forward(qd, kd, vd, w.lam, u=uu, out=out, S_T=S_T, A_T=A_T, z_T=z_T,
+                                        status=status, stream=stream)
+        evs = []
+        with torch.cuda.stream(stream):
+            for _ in range(2):
+                ucall()
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); ucall(); b.record(stream)
+                evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+        per[w.name + "_explicit_u"] = {
+            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T,
+            "fp32_frac_nominal": alg_flops_per_token(w.d, True) * w.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
+            "units": w.units, "kernel": "vla_scan_chunk_kernel (explicit u)"}
+        del uu
         # single-step decode (T = 1, carried states): bound by moving S and A through HBM once
         wd = W.EXTRA["decode"]
         q2, k2, v2 = [x.to(dev) for x in W.make_inputs(wd)]

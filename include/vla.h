@@ -54,8 +54,8 @@ enum {
 typedef enum {
   VLA_KERNEL_AUTO = 0,
   VLA_KERNEL_TOKEN = 1, /* one CTA per unit, one state pass per token; every shape, explicit u */
-  VLA_KERNEL_CHUNK = 2  /* 16 tokens per state pass (exact Woodbury form); u = k_hat, d >= 32;
-                           VLA_ERR_UNSUPPORTED otherwise */
+  VLA_KERNEL_CHUNK = 2  /* 16 tokens per state pass (exact Woodbury form); d >= 32, no periodic
+                           refresh; VLA_ERR_UNSUPPORTED otherwise */
 } vla_kernel_t;
 
 typedef struct {

@@ -75,11 +75,11 @@ int launch_token_d(const ScanParams& p_in, int dtype, cudaStream_t st) {
 // means "done"; ids never repeat within 2^32 launches, so the flags never need clearing).
 std::atomic<unsigned int> g_launch_epoch{0};
 
-template <int D, typename TIn>
+template <int D, typename TIn, bool HAS_U>
 int launch_chunk(const ScanParams& p, cudaStream_t st) {
-  using Cfg = vla::ChunkCfg<D, TIn>;
-  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false>;     // one CTA per unit
-  auto kern_bal = vla::vla_scan_chunk_kernel<D, TIn, true>;  // persistent grid, units cut at chunks
+  using Cfg = vla::ChunkCfg<D, TIn, HAS_U>;
+  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, HAS_U>;     // one CTA per unit
+  auto kern_bal = vla::vla_scan_chunk_kernel<D, TIn, true, HAS_U>;  // persistent grid, units cut at chunks
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(Cfg::smem_bytes)) != cudaSuccess ||
       cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -119,14 +119,16 @@ int launch_chunk(const ScanParams& p, cudaStream_t st) {
 
 template <int D>
 int launch_chunk_d(const ScanParams& p, int dtype, cudaStream_t st) {
-  return dtype == VLA_F32 ? launch_chunk<D, float>(p, st) : launch_chunk<D, uint16_t>(p, st);
+  if (p.u)
+    return dtype == VLA_F32 ? launch_chunk<D, float, true>(p, st)
+                            : launch_chunk<D, uint16_t, true>(p, st);
+  return dtype == VLA_F32 ? launch_chunk<D, float, false>(p, st)
+                          : launch_chunk<D, uint16_t, false>(p, st);
 }
 
-// The chunk kernel covers u = k_hat and d in {32, 64, 128}; everything else runs on the
-// token kernel.  Both are CUDA paths; there is no host fallback.
-bool chunk_covers(const ScanParams& p, int d) {
-  return p.u == nullptr && d >= 32 && p.refresh_period <= 0;
-}
+// The chunk kernel covers d in {32, 64, 128} without the periodic refresh; everything else
+// runs on the token kernel.  Both are CUDA paths; there is no host fallback.
+bool chunk_covers(const ScanParams& p, int d) { return d >= 32 && p.refresh_period <= 0; }
 
 // Very short sequences (single-step decode and the like) are bound by reading and writing
 // the states once; there the token kernel is faster than a 16-token chunk that is mostly

@@ -1,4 +1,4 @@
-// VLA forward scan, "chunk" kernel (u = k_hat): the recurrence of Section 3.3 evaluated
+// VLA forward scan, "chunk" kernel: the recurrence of Section 3.3 evaluated
 // C = 16 tokens at a time in exact algebra, so that the fp32 FMA pipe works on rank-16
 // updates instead of a chain of rank-1 steps.  One CTA works on one (batch, head) unit at a
 // time (see "work distribution" below), two warp groups of D threads each:
@@ -17,6 +17,12 @@
 //   B  = V^T - S K^T                    e_t = b_t - sum_{s<t} Gu[s,t] e_s,  Gu[s,t] = alpha_s.k_hat_t
 //   e'_t = sc_t e_t                     o_t = (S q_t + sum_{s<=t} e'_s (z_s.q_t)) / den_t
 //   S <- S + E' Z^T
+//
+// The lines above are the u = k_hat case.  With an explicit u (HAS_U): Z0 = A U^T and
+// W = U Z0 give delta, L and Z as above; W0 = A K^T and X = U W0 give, by the same
+// elimination, N[s,t] = z_s.k_hat_t and a_t = A_t k_hat_t = W0_t - sum_{s<=t} z_s N[s,t]/delta_s;
+// alpha_t = a_t / max(||a_t||, eps), Gu[s,t] = alpha_s.k_hat_t, and a takes Z's place in the
+// S update and in the readout.
 //
 // Group A runs ahead of group S.  It owns the input stream: q/k/v arrive through a ring of
 // 1-D bulk-async (TMA) copies, and group A widens them (phi, k_hat, ||phi(k)||) into a
@@ -78,7 +84,7 @@ struct ChunkTile {
   static constexpr int TR = D / TW;              // state rows per thread (= lanes per row block)
 };
 
-template <int D, typename TIn>
+template <int D, typename TIn, bool HAS_U = false>
 struct ChunkCfg {
   static constexpr int C = 16;                   // tokens per chunk
   static constexpr int TW = ChunkTile<D>::TW;
@@ -88,19 +94,22 @@ struct ChunkCfg {
   static constexpr int NG = D;                   // threads per warp group
   static constexpr int NT = 2 * D;               // threads per CTA
   static constexpr int NWG = D / 32;             // warps per group
-  static constexpr int NSTAGE = sizeof(TIn) == 2 ? 4 : 2;  // raw q/k/v chunks in flight
+  static constexpr int NIN = HAS_U ? 4 : 3;      // q, k, v[, u]
+  // raw q/k/v[/u] chunks in flight (fewer with an explicit u: shared memory is the limit)
+  static constexpr int NSTAGE = HAS_U ? (sizeof(TIn) == 2 ? 2 : 1) : (sizeof(TIn) == 2 ? 4 : 2);
   static constexpr int RING = 2;                 // Z / Gu / HT / sc slots (group A -> group S)
   static constexpr int KRING = 3;                // widened k_hat / q_f / v / ||phi(k)|| slots
   static constexpr int CP = C + 4;               // padded row of the small C x C matrices
 
   // shared memory layout (floats unless noted)
-  static constexpr size_t raw_bytes = size_t(NSTAGE) * 3 * C * D * sizeof(TIn);
+  static constexpr size_t raw_bytes = size_t(NSTAGE) * NIN * C * D * sizeof(TIn);
   static constexpr size_t kslot_floats = size_t(3) * C * D + C;             // Kh, Qf, Vf, nrm
   static constexpr size_t slot_floats = size_t(C) * D + 2 * C * CP + 2 * C; // Zs, GuT, HT, sc, inv_den
-  static constexpr size_t a_floats = size_t(2) * C * D + 2 * C * CP + 2 * NWG * C + 2 * C;
-  //   Z0s, ZDs | Ws, Ls | N2p, denp | delta, inv_delta
-  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D;
-  //   VS(B), R0s, Eps | ostage[2]
+  static constexpr size_t a_floats = size_t(HAS_U ? 4 : 1) * C * D + (HAS_U ? 4 : 2) * C * CP +
+                                     2 * NWG * C + 3 * C;
+  //   Z0s [, W0s, Uf[2]] | Ws, Ls [, Xs, PTs] | N2p, denp | delta, 1/delta, -1/delta
+  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + (HAS_U ? 2 * C * CP : 0);
+  //   VS(B), R0s, Eps | ostage[2] [| GuL, HTL]
   static constexpr size_t smem_bytes = raw_bytes +
       (KRING * kslot_floats + RING * slot_floats + a_floats + s_floats) * sizeof(float) +
       (NSTAGE + 2 * RING) * sizeof(uint64_t) + 16 + 128;
@@ -193,19 +202,22 @@ __device__ __forceinline__ void tile_matvec_chunk(const float2 (&st)[TR][TW / 2]
   sink(C - 1, v[1][0]);
 }
 
-// tile += sum_s coef[s][rows of the tile] (x) vec[s][cols of the tile]   (rank-16 update)
-template <int TR, int TW, int LPR, int D, int C, bool NEGATE>
+// tile += sum_s scale[s] * coef[s][rows of the tile] (x) vec[s][cols of the tile]   (rank-16
+// update; scale == nullptr means 1)
+template <int TR, int TW, int LPR, int D, int C>
 __device__ __forceinline__ void tile_rank_update(float2 (&st)[TR][TW / 2], const float* coef,
-                                                 const float* vec, int rb, int cg) {
+                                                 const float* vec, const float* scale, int rb,
+                                                 int cg) {
   constexpr int NV = TW / 4;
 #pragma unroll 2
   for (int s2 = 0; s2 < C; ++s2) {
+    const float sc = scale ? scale[s2] : 1.0f;
     float cf[TR];
 #pragma unroll
     for (int r4 = 0; r4 < TR / 4; ++r4) {
       const float4 x = reinterpret_cast<const float4*>(coef + s2 * D + rb * TR)[r4];
-      cf[4 * r4 + 0] = NEGATE ? -x.x : x.x; cf[4 * r4 + 1] = NEGATE ? -x.y : x.y;
-      cf[4 * r4 + 2] = NEGATE ? -x.z : x.z; cf[4 * r4 + 3] = NEGATE ? -x.w : x.w;
+      cf[4 * r4 + 0] = x.x * sc; cf[4 * r4 + 1] = x.y * sc;
+      cf[4 * r4 + 2] = x.z * sc; cf[4 * r4 + 3] = x.w * sc;
     }
 #pragma unroll
     for (int m = 0; m < NV; ++m) {
@@ -332,10 +344,11 @@ __device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) 
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-template <int D, typename TIn, bool BALANCED>
+template <int D, typename TIn, bool BALANCED, bool HAS_U>
 __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanParams p,
                                                                   const SchedParams sp) {
-  using Cfg = ChunkCfg<D, TIn>;
+  using Cfg = ChunkCfg<D, TIn, HAS_U>;
+  constexpr int NIN = Cfg::NIN;
   constexpr int C = Cfg::C, TW = Cfg::TW, TR = Cfg::TR, LPR = Cfg::LPR, NV = Cfg::NV;
   constexpr int NG = Cfg::NG, NWG = Cfg::NWG, NSTAGE = Cfg::NSTAGE, RING = Cfg::RING;
   constexpr int KRING = Cfg::KRING, CP = Cfg::CP;
@@ -348,19 +361,25 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   float* kring = fbase;                               // [KRING] { Kh, Qf, Vf : [C][D], nrm[C] }
   float* zring = kring + KRING * Cfg::kslot_floats;   // [RING] { Zs[C][D], GuT, HT : [C][CP], sc, inv_den : [C] }
   float* abase = zring + RING * Cfg::slot_floats;
-  float* Z0s = abase;               // [C][D]
-  float* ZDs = Z0s + C * D;         // [C][D]  z_t / delta_t
-  float* Ws = ZDs + C * D;          // [C][CP] K A K^T
-  float* Ls = Ws + C * CP;          // [C][CP] unit lower factor
-  float* N2p = Ls + C * CP;         // [NWG][C]
-  float* denp = N2p + NWG * C;      // [NWG][C]
-  float* dlt = denp + NWG * C;      // [C]
-  float* idl = dlt + C;             // [C]
+  float* Z0s = abase;                              // [C][D]  A U^T, then Z in place (explicit u)
+  float* W0s = Z0s + C * D;                        // [C][D]  A K^T            (explicit u only)
+  float* Ufs = W0s + C * D;                        // [2][C][D] widened u      (explicit u only)
+  float* Ws = abase + (HAS_U ? 4 : 1) * C * D;     // [C][CP] U A U^T (K A K^T when u = k_hat)
+  float* Ls = Ws + C * CP;                         // [C][CP] unit lower factor
+  float* Xs = Ls + C * CP;                         // [C][CP] U A K^T          (explicit u only)
+  float* PTs = Xs + C * CP;                        // [C][CP] PT[t][s] = (z_s.k_t)/delta_s (explicit u only)
+  float* N2p = Ws + (HAS_U ? 4 : 2) * C * CP;      // [NWG][C]
+  float* denp = N2p + NWG * C;                     // [NWG][C]
+  float* dlt = denp + NWG * C;                     // [C]
+  float* idl = dlt + C;                            // [C]  1/delta
+  float* nidl = idl + C;                           // [C] -1/delta
   float* sbase = abase + Cfg::a_floats;
   float* VS = sbase;                // [C][D]  B = V^T - S K^T
   float* R0s = VS + C * D;          // [C][D]
   float* Eps = R0s + C * D;         // [C][D]
   float* ostage = Eps + C * D;      // [2][C][D]
+  float* GuL = ostage + 2 * C * D;  // [C][CP] GuL[t][s] = k_hat_t . a_s   (explicit u only)
+  float* HTL = GuL + C * CP;        // [C][CP] HTL[t][s] = q_t . a_s       (explicit u only)
   uint64_t* bars = reinterpret_cast<uint64_t*>(
       (reinterpret_cast<uintptr_t>(sbase + Cfg::s_floats) + 15) & ~uintptr_t(15));
   uint64_t* full = bars;                    // [NSTAGE] raw stage filled by TMA
@@ -418,11 +437,12 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     const int s = c % NSTAGE;
     const int n = min(C, T - c * C);
     const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
-    TIn* dst = raw + size_t(s) * 3 * C * D;
-    mbar_arrive_expect_tx(&full[s], 3 * bytes);
+    TIn* dst = raw + size_t(s) * NIN * C * D;
+    mbar_arrive_expect_tx(&full[s], NIN * bytes);
     bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &full[s]);
     bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &full[s]);
     bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
+    if (HAS_U) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
   };
 
   // (re)arm the barriers of this piece; a tail piece also waits for its unit's head
@@ -496,9 +516,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       const int s = c % NSTAGE;
       const int n = min(C, T - c * C);
       wait(&full[s], (c / NSTAGE) & 1);
-      const TIn* rq = raw + (size_t(s) * 3 + 0) * C * D;
-      const TIn* rk = raw + (size_t(s) * 3 + 1) * C * D;
-      const TIn* rv = raw + (size_t(s) * 3 + 2) * C * D;
+      const TIn* rq = raw + (size_t(s) * NIN + 0) * C * D;
+      const TIn* rk = raw + (size_t(s) * NIN + 1) * C * D;
+      const TIn* rv = raw + (size_t(s) * NIN + 2) * C * D;
+      const TIn* ru = raw + (size_t(s) * NIN + (HAS_U ? 3 : 0)) * C * D;
+      float* Uf = Ufs + size_t(c & 1) * C * D;   // penalty directions, verbatim
       float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
       float* Qf = Kh + C * D;
       float* Vf = Qf + C * D;
@@ -527,6 +549,9 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           }
           reinterpret_cast<float4*>(Qf + tt * D)[f] = qf;
           reinterpret_cast<float4*>(Vf + tt * D)[f] = vv;
+          if (HAS_U)
+            reinterpret_cast<float4*>(Uf + tt * D)[f] =
+                act ? load4(ru + tt * D, f) : make_float4(0.f, 0.f, 0.f, 0.f);
           ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
           ss = fmaf(kf[i].z, kf[i].z, ss); ss = fmaf(kf[i].w, kf[i].w, ss);
         }
@@ -595,13 +620,17 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         if ((lane & 1) == 0) denp[gw * C + (lane >> 1)] = tot;
       }
 
-      // ---- Z0 = A K^T
-      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) { Z0s[t * D + g] = x; });
+      // ---- Z0 = A U^T (U = K when no u is given); with an explicit u also W0 = A K^T
+      const float* Uf = HAS_U ? (Ufs + size_t(c & 1) * C * D) : Kh;
+      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Uf, cg, [&](int t, float x) { Z0s[t * D + g] = x; });
+      if (HAS_U)
+        tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) { W0s[t * D + g] = x; });
       group_bar(1, NG);
       VLA_MARK(1)
 
-      // ---- W = K Z0 (C x C)
-      gram16<D, NG, CP>(Kh, Z0s, Ws, g);
+      // ---- W = U Z0 (C x C, symmetric); with an explicit u also X[s][t] = u_s . (A k_hat_t)
+      gram16<D, NG, CP>(Uf, Z0s, Ws, g);
+      if (HAS_U) gram16<D, NG, CP>(Uf, W0s, Xs, g);
       group_bar(1, NG);
       VLA_MARK(2)
 
@@ -637,7 +666,29 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
             m[j] = fmaf(-l, msj, m[j]);
           }
           if (h == hs) Ls[r * CP + s2] = l;
-          if (lane == 0) { dlt[s2] = piv; idl[s2] = ipiv; }
+          if (lane == 0) { dlt[s2] = piv; idl[s2] = ipiv; nidl[s2] = -ipiv; }
+        }
+        if (HAS_U) {
+          // N[s][t] = z_s . k_hat_t (s <= t) from X by the same elimination:
+          //   N[s][t] = X[s][t] - sum_{r<s} L[s][r] N[r][t];  PT[t][s] = N[s][t] / delta_s.
+          // Lane t < 16 owns column t (both halves of the warp compute the same thing).
+          __syncwarp();
+          const int t = lane & 15;
+          float nn[16];
+#pragma unroll
+          for (int s2 = 0; s2 < 16; ++s2) {
+            float a0 = Xs[s2 * CP + t], a1 = 0.f;
+#pragma unroll
+            for (int r4 = 0; r4 * 4 < s2; ++r4) {
+              const float4 l4 = reinterpret_cast<const float4*>(Ls + s2 * CP)[r4];
+              if (4 * r4 + 0 < s2) a0 = fmaf(-l4.x, nn[4 * r4 + 0], a0);
+              if (4 * r4 + 1 < s2) a1 = fmaf(-l4.y, nn[4 * r4 + 1], a1);
+              if (4 * r4 + 2 < s2) a0 = fmaf(-l4.z, nn[4 * r4 + 2], a0);
+              if (4 * r4 + 3 < s2) a1 = fmaf(-l4.w, nn[4 * r4 + 3], a1);
+            }
+            nn[s2] = a0 + a1;
+            if (h == 0) PTs[t * CP + s2] = (s2 <= t) ? nn[s2] * idl[s2] : 0.0f;
+          }
         }
         VLA_MARK(8)
         if (NWG == 1 && c + 1 < nchunks) prep_inputs(c + 1, 0, 1);
@@ -667,11 +718,32 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           z[t] = a0 + a1;
         }
         float sq[16];
+        if (!HAS_U) {
+          // A_t k_hat_t = z_t / delta_t: group S gets Z itself (and sc carries the 1/delta)
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          Zs[t * D + g] = z[t];
-          ZDs[t * D + g] = z[t] * idl[t];
-          sq[t] = z[t] * z[t];
+          for (int t = 0; t < 16; ++t) {
+            Zs[t * D + g] = z[t];
+            sq[t] = z[t] * z[t];
+          }
+        } else {
+          // a_t = A_t k_hat_t = A k_hat_t - sum_{s<=t} z_s (z_s.k_hat_t)/delta_s: group S gets a;
+          // Z stays with group A (in place over Z0) for the update of A
+#pragma unroll
+          for (int t = 0; t < 16; ++t) {
+            float a0 = W0s[t * D + g], a1 = 0.f;
+#pragma unroll
+            for (int s4 = 0; s4 * 4 <= t; ++s4) {
+              const float4 p4 = reinterpret_cast<const float4*>(PTs + t * CP)[s4];
+              if (4 * s4 + 0 <= t) a0 = fmaf(-p4.x, z[4 * s4 + 0], a0);
+              if (4 * s4 + 1 <= t) a1 = fmaf(-p4.y, z[4 * s4 + 1], a1);
+              if (4 * s4 + 2 <= t) a0 = fmaf(-p4.z, z[4 * s4 + 2], a0);
+              if (4 * s4 + 3 <= t) a1 = fmaf(-p4.w, z[4 * s4 + 3], a1);
+            }
+            const float at = a0 + a1;
+            Zs[t * D + g] = at;
+            Z0s[t * D + g] = z[t];
+            sq[t] = at * at;
+          }
         }
         const float tot = warp_reduce_scatter16(sq, lane);
         if ((lane & 1) == 0) N2p[gw * C + (lane >> 1)] = tot;
@@ -686,28 +758,36 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 #pragma unroll
         for (int w2 = 0; w2 < NWG; ++w2) n2 += N2p[w2 * C + r];
         const float id_r = idl[r], d_r = dlt[r];
-        // alpha_r = sc_r z_r with sc_r = (1/delta) / max(||z||/delta, eps)
-        const float sc_r = id_r * rcp_nr(fmaxf(sqrt_approx(n2) * id_r, eps));
+        // u = k_hat:   alpha_r = sc_r z_r, sc_r = (1/delta) / max(||z||/delta, eps)
+        // explicit u:  alpha_r = sc_r a_r, sc_r = 1 / max(||a||, eps)
+        const float sc_r = HAS_U ? rcp_nr(fmaxf(sqrt_approx(n2), eps))
+                                 : id_r * rcp_nr(fmaxf(sqrt_approx(n2) * id_r, eps));
         if ((p.flags & VLA_FLAG_CHECK_FINITE) && p.status && !isfinite(n2 + d_r))
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
-        const float scd = sc_r * d_r;   // multiplies column r of L
         if (h == 0) scs[r] = sc_r;
-        // lane (r, h) writes GuT[r][h*8 .. h*8+7]: GuT[r][s] = scd_s L[r][s]
+        if (!HAS_U) {
+          const float scd = sc_r * d_r;   // multiplies column r of L
+          // lane (r, h) writes GuT[r][h*8 .. h*8+7]: GuT[r][s] = scd_s L[r][s]
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int s2 = h * 8 + j;
-          const float scd_s = __shfl_sync(0xffffffffu, scd, s2);
-          GuT[r * CP + s2] = (s2 < r) ? scd_s * Ls[r * CP + s2] : 0.0f;
+          for (int j = 0; j < 8; ++j) {
+            const int s2 = h * 8 + j;
+            const float scd_s = __shfl_sync(0xffffffffu, scd, s2);
+            GuT[r * CP + s2] = (s2 < r) ? scd_s * Ls[r * CP + s2] : 0.0f;
+          }
         }
       }
-      // ---- HT[t][s] = q_t . z_s (C x C), then publish the chunk to group S
-      gram16<D, NG, CP>(Qf, Zs, HT, g);
+      // ---- HT[t][s] = q_t . z_s (C x C), then publish the chunk to group S.  With an
+      //      explicit u group S forms its two small matrices from a itself.
+      if (!HAS_U) gram16<D, NG, CP>(Qf, Zs, HT, g);
       group_bar(1, NG);
       if (g == 0) mbar_arrive(&ring_full[slot]);
       VLA_MARK(6)
 
       // ---- A <- A - Z diag(1/delta) Z^T
-      tile_rank_update<TR, TW, LPR, D, C, true>(st, ZDs, Zs, rb, cg);
+      {
+        const float* Zown = HAS_U ? Z0s : Zs;
+        tile_rank_update<TR, TW, LPR, D, C>(st, Zown, Zown, nidl, rb, cg);
+      }
       VLA_MARK(7)
     }
     if (p.zT) p.zT[size_t(unit) * D + g] = zk;
@@ -746,10 +826,23 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       });
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
       if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
+      // explicit u: the ring's Z slot carries a_t = A_t k_hat_t; the two small matrices
+      // k_hat_t . a_s and q_t . a_s are formed here (for u = k_hat they come from group A)
+      const float* Gm = GuT;
+      const float* Hm = HT;
+      if (HAS_U) {
+        gram16<D, NG, CP>(Kh, Zs, GuL, g);
+        gram16<D, NG, CP>(Qf, Zs, HTL, g);
+        group_bar(2, NG);
+        Gm = GuL;
+        Hm = HTL;
+      }
       VLA_MARK(2)
 
       // ---- row g: e_t = b_t - sum_{s<t} Gu[s][t] e_s; e'_t = sc_t e_t;
       //             o_t = (r0_t + sum_{s<=t} e'_s HT[t][s]) / den_t
+      //      (u = k_hat: Gm holds Gu with sc folded in; explicit u: Gm holds k_hat_t . a_s and
+      //       Gu[s][t] e_s = Gm[t][s] e'_s)
       float o[16];
       {
         float e[16], ep[16];
@@ -758,11 +851,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           float a0 = VS[t * D + g], a1 = 0.f;
 #pragma unroll
           for (int s4 = 0; s4 * 4 < t; ++s4) {
-            const float4 g4 = reinterpret_cast<const float4*>(GuT + t * CP)[s4];
-            if (4 * s4 + 0 < t) a0 = fmaf(-g4.x, e[4 * s4 + 0], a0);
-            if (4 * s4 + 1 < t) a1 = fmaf(-g4.y, e[4 * s4 + 1], a1);
-            if (4 * s4 + 2 < t) a0 = fmaf(-g4.z, e[4 * s4 + 2], a0);
-            if (4 * s4 + 3 < t) a1 = fmaf(-g4.w, e[4 * s4 + 3], a1);
+            const float4 g4 = reinterpret_cast<const float4*>(Gm + t * CP)[s4];
+            if (4 * s4 + 0 < t) a0 = fmaf(-g4.x, HAS_U ? ep[4 * s4 + 0] : e[4 * s4 + 0], a0);
+            if (4 * s4 + 1 < t) a1 = fmaf(-g4.y, HAS_U ? ep[4 * s4 + 1] : e[4 * s4 + 1], a1);
+            if (4 * s4 + 2 < t) a0 = fmaf(-g4.z, HAS_U ? ep[4 * s4 + 2] : e[4 * s4 + 2], a0);
+            if (4 * s4 + 3 < t) a1 = fmaf(-g4.w, HAS_U ? ep[4 * s4 + 3] : e[4 * s4 + 3], a1);
           }
           e[t] = a0 + a1;
           ep[t] = e[t] * scs[t];
@@ -773,7 +866,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           float a0 = R0s[t * D + g], a1 = 0.f;
 #pragma unroll
           for (int s4 = 0; s4 * 4 <= t; ++s4) {
-            const float4 h4 = reinterpret_cast<const float4*>(HT + t * CP)[s4];
+            const float4 h4 = reinterpret_cast<const float4*>(Hm + t * CP)[s4];
             if (4 * s4 + 0 <= t) a0 = fmaf(h4.x, ep[4 * s4 + 0], a0);
             if (4 * s4 + 1 <= t) a1 = fmaf(h4.y, ep[4 * s4 + 1], a1);
             if (4 * s4 + 2 <= t) a0 = fmaf(h4.z, ep[4 * s4 + 2], a0);
@@ -799,7 +892,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       VLA_MARK(3)
 
       // ---- S <- S + E' Z^T
-      tile_rank_update<TR, TW, LPR, D, C, false>(st, Eps, Zs, rb, cg);
+      tile_rank_update<TR, TW, LPR, D, C>(st, Eps, Zs, nullptr, rb, cg);
       group_bar(2, NG);
       if (g == 0) mbar_arrive(&ring_empty[slot]);
       VLA_MARK(4)

@@ -20,7 +20,7 @@ KERNELS = {"token": vla.VLA_KERNEL_TOKEN, "chunk": vla.VLA_KERNEL_CHUNK}
 
 
 def _chunk_covers(d, umode="khat"):
-    return d >= 32 and umode == "khat"
+    return d >= 32
 
 
 @pytest.mark.parametrize("kernel", ["token", "chunk"])
@@ -31,7 +31,7 @@ def _chunk_covers(d, umode="khat"):
 def test_small_shapes(kernel, d, dtype, flags, umode):
     """Several chunks plus a ragged tail (T = 83 = 5*16 + 3), 6 units, both kernels."""
     if kernel == "chunk" and not _chunk_covers(d, umode):
-        pytest.skip("the chunk kernel covers u = k_hat, d >= 32")
+        pytest.skip("the chunk kernel covers d >= 32")
     w = _small(d, 83, dtype, seed=7 * d + len(umode))
     q, k, v = W.make_inputs(w)
     u = None
@@ -51,8 +51,8 @@ def test_forced_chunk_kernel_rejects_what_it_does_not_cover():
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
     w = _small(64, 8, "f32")
     q, k, v = [x.to(dev) for x in W.make_inputs(w)]
-    with pytest.raises(vla.VlaError):
-        vla.vla_forward(q, k, v, 1.0, u=W.make_u(w).to(dev), kernel=vla.VLA_KERNEL_CHUNK)
+    with pytest.raises(vla.VlaError):          # the periodic refresh lives in the token kernel
+        vla.vla_forward(q, k, v, 1.0, refresh=(20, 1e-3, 0), kernel=vla.VLA_KERNEL_CHUNK)
 
 
 @pytest.mark.parametrize("T", [0, 1, 2, 15, 16, 17, 31, 32, 33, 48, 49, 63, 64, 65, 97])
@@ -88,7 +88,7 @@ def test_state_carry_split_invariance():
         for uu in (None, u):
             # one kernel for all three calls (AUTO would pick by length), so that a
             # chunk-aligned split can be compared bit for bit
-            kern = vla.VLA_KERNEL_CHUNK if uu is None else vla.VLA_KERNEL_TOKEN
+            kern = vla.VLA_KERNEL_CHUNK
             full = run_gpu(q, k, v, 0.1, u=uu, flags=flags, kernel=kern)
             ref = run_oracle(q, k, v, 0.1, u=uu, flags=flags)
             for T1 in (16, 37, 64):
@@ -119,6 +119,9 @@ def test_more_units_than_resident_ctas(d, units, flags):
     z0 = torch.rand((B, H, d), generator=g)
     errs, got, ref = check_parity(q, k, v, 1.0, 1e-4, S0=S0, z0=z0, flags=flags,
                                   kernel=vla.VLA_KERNEL_CHUNK, label="balanced d=%d" % d)
+    if flags == 0:   # and with an explicit penalty direction (the paper's u / sqrt(d_h))
+        check_parity(q, k, v, 0.1, 1e-4, u=W.make_u(w, d ** -0.5), S0=S0, z0=z0, flags=flags,
+                     kernel=vla.VLA_KERNEL_CHUNK, label="balanced explicit-u d=%d" % d)
     # the same launch twice is bitwise reproducible (the cut points are fixed by the shape)
     again = run_gpu(q, k, v, 1.0, S0=S0, z0=z0, flags=flags, kernel=vla.VLA_KERNEL_CHUNK)
     assert torch.equal(got.out, again.out) and torch.equal(got.S_T, again.S_T)

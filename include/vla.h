@@ -54,8 +54,8 @@ enum {
 typedef enum {
   VLA_KERNEL_AUTO = 0,
   VLA_KERNEL_TOKEN = 1, /* one CTA per unit, one state pass per token; every shape, explicit u */
-  VLA_KERNEL_CHUNK = 2  /* 16 tokens per state pass (exact Woodbury form); d >= 32, no periodic
-                           refresh; VLA_ERR_UNSUPPORTED otherwise */
+  VLA_KERNEL_CHUNK = 2  /* 16 tokens per state pass (exact Woodbury form); d >= 32, every option;
+                           VLA_ERR_UNSUPPORTED for d = 16 */
 } vla_kernel_t;
 
 typedef struct {
@@ -73,7 +73,7 @@ typedef struct {
   /* Algorithm 1's periodic identity refresh (Section 5.3: every 20 steps, + 1e-3 I): after
      the Sherman-Morrison step of each token whose 1-based position in the whole sequence
      (step_offset + t + 1) is a multiple of refresh_period, A += refresh_eta * I.  Off when
-     refresh_period <= 0 (the default: it breaks A_t = M_t^-1).  Runs on the token kernel.   */
+     refresh_period <= 0 (the default: it breaks A_t = M_t^-1).  Both kernels implement it.   */
   int32_t refresh_period;
   float refresh_eta;
   int64_t step_offset;   /* tokens of this sequence processed by earlier calls (state carry)     */

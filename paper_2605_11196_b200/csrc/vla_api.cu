@@ -75,11 +75,12 @@ int launch_token_d(const ScanParams& p_in, int dtype, cudaStream_t st) {
 // means "done"; ids never repeat within 2^32 launches, so the flags never need clearing).
 std::atomic<unsigned int> g_launch_epoch{0};
 
-template <int D, typename TIn, bool HAS_U>
+template <int D, typename TIn, int UM>
 int launch_chunk(const ScanParams& p, cudaStream_t st) {
-  using Cfg = vla::ChunkCfg<D, TIn, HAS_U>;
-  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, HAS_U>;     // one CTA per unit
-  auto kern_bal = vla::vla_scan_chunk_kernel<D, TIn, true, HAS_U>;  // persistent grid, units cut at chunks
+  using Cfg = vla::ChunkCfg<D, TIn, UM>;
+  static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
+  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, UM>;     // one CTA per unit
+  auto kern_bal = vla::vla_scan_chunk_kernel<D, TIn, true, UM>;  // persistent grid, units cut at chunks
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(Cfg::smem_bytes)) != cudaSuccess ||
       cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -120,15 +121,19 @@ int launch_chunk(const ScanParams& p, cudaStream_t st) {
 template <int D>
 int launch_chunk_d(const ScanParams& p, int dtype, cudaStream_t st) {
   if (p.u)
-    return dtype == VLA_F32 ? launch_chunk<D, float, true>(p, st)
-                            : launch_chunk<D, uint16_t, true>(p, st);
-  return dtype == VLA_F32 ? launch_chunk<D, float, false>(p, st)
-                          : launch_chunk<D, uint16_t, false>(p, st);
+    return dtype == VLA_F32 ? launch_chunk<D, float, vla::kUTensor>(p, st)
+                            : launch_chunk<D, uint16_t, vla::kUTensor>(p, st);
+  // The periodic refresh makes A_t k_hat_t leave the direction of z_t: general path, u = k_hat.
+  if (p.refresh_period > 0)
+    return dtype == VLA_F32 ? launch_chunk<D, float, vla::kUKhatGen>(p, st)
+                            : launch_chunk<D, uint16_t, vla::kUKhatGen>(p, st);
+  return dtype == VLA_F32 ? launch_chunk<D, float, vla::kUKhat>(p, st)
+                          : launch_chunk<D, uint16_t, vla::kUKhat>(p, st);
 }
 
-// The chunk kernel covers d in {32, 64, 128} without the periodic refresh; everything else
-// runs on the token kernel.  Both are CUDA paths; there is no host fallback.
-bool chunk_covers(const ScanParams& p, int d) { return d >= 32 && p.refresh_period <= 0; }
+// The chunk kernel covers d in {32, 64, 128}; d = 16 runs on the token kernel.  Both are CUDA
+// paths; there is no host fallback.
+bool chunk_covers(const ScanParams&, int d) { return d >= 32; }
 
 // Very short sequences (single-step decode and the like) are bound by reading and writing
 // the states once; there the token kernel is faster than a 16-token chunk that is mostly

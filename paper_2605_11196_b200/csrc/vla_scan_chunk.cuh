@@ -18,11 +18,14 @@
 //   e'_t = sc_t e_t                     o_t = (S q_t + sum_{s<=t} e'_s (z_s.q_t)) / den_t
 //   S <- S + E' Z^T
 //
-// The lines above are the u = k_hat case.  With an explicit u (HAS_U): Z0 = A U^T and
+// The lines above are the u = k_hat case.  General path (explicit u, or refresh): Z0 = A U^T and
 // W = U Z0 give delta, L and Z as above; W0 = A K^T and X = U W0 give, by the same
 // elimination, N[s,t] = z_s.k_hat_t and a_t = A_t k_hat_t = W0_t - sum_{s<=t} z_s N[s,t]/delta_s;
 // alpha_t = a_t / max(||a_t||, eps), Gu[s,t] = alpha_s.k_hat_t, and a takes Z's place in the
-// S update and in the readout.
+// S update and in the readout.  Algorithm 1's periodic refresh (A += eta I after every
+// period-th token) runs on the general path: with rho(t) refreshes after tokens < t of the
+// chunk, Z0_t += eta rho(t) u_t, W[s,t] += eta rho(min(s,t)) u_s.u_t, X[s,t] += eta rho(s) u_s.k_t,
+// a_t += eta rho(t+1) k_hat_t, and the chunk ends with A += eta rho(n) I.
 //
 // Group A runs ahead of group S.  It owns the input stream: q/k/v arrive through a ring of
 // 1-D bulk-async (TMA) copies, and group A widens them (phi, k_hat, ||phi(k)||) into a
@@ -84,8 +87,18 @@ struct ChunkTile {
   static constexpr int TR = D / TW;              // state rows per thread (= lanes per row block)
 };
 
-template <int D, typename TIn, bool HAS_U = false>
+// How the penalty direction u_t is obtained and which algebra the chunk uses:
+//   kUKhat    u = k_hat, no refresh: A_t k_hat_t = z_t / delta_t, one product with A per chunk
+//   kUTensor  u read from the caller's tensor: general path (a_t = A_t k_hat_t by a second
+//             elimination), three products with A per chunk
+//   kUKhatGen u = k_hat on the general path: used for Algorithm 1's periodic refresh, after
+//             which A_t k_hat_t is no longer parallel to z_t; one product with A per chunk
+enum : int { kUKhat = 0, kUTensor = 1, kUKhatGen = 2 };
+
+template <int D, typename TIn, int UM = kUKhat>
 struct ChunkCfg {
+  static constexpr bool GEN = UM != kUKhat;      // general path
+  static constexpr bool UT = UM == kUTensor;     // a fourth input tensor
   static constexpr int C = 16;                   // tokens per chunk
   static constexpr int TW = ChunkTile<D>::TW;
   static constexpr int TR = ChunkTile<D>::TR;
@@ -94,9 +107,9 @@ struct ChunkCfg {
   static constexpr int NG = D;                   // threads per warp group
   static constexpr int NT = 2 * D;               // threads per CTA
   static constexpr int NWG = D / 32;             // warps per group
-  static constexpr int NIN = HAS_U ? 4 : 3;      // q, k, v[, u]
-  // raw q/k/v[/u] chunks in flight (fewer with an explicit u: shared memory is the limit)
-  static constexpr int NSTAGE = HAS_U ? (sizeof(TIn) == 2 ? 2 : 1) : (sizeof(TIn) == 2 ? 4 : 2);
+  static constexpr int NIN = UT ? 4 : 3;         // q, k, v[, u]
+  // raw q/k/v[/u] chunks in flight (fewer on the general path: shared memory is the limit)
+  static constexpr int NSTAGE = UT ? (sizeof(TIn) == 2 ? 2 : 1) : (sizeof(TIn) == 2 ? 4 : 2);
   static constexpr int RING = 2;                 // Z / Gu / HT / sc slots (group A -> group S)
   static constexpr int KRING = 3;                // widened k_hat / q_f / v / ||phi(k)|| slots
   static constexpr int CP = C + 4;               // padded row of the small C x C matrices
@@ -105,10 +118,13 @@ struct ChunkCfg {
   static constexpr size_t raw_bytes = size_t(NSTAGE) * NIN * C * D * sizeof(TIn);
   static constexpr size_t kslot_floats = size_t(3) * C * D + C;             // Kh, Qf, Vf, nrm
   static constexpr size_t slot_floats = size_t(C) * D + 2 * C * CP + 2 * C; // Zs, GuT, HT, sc, inv_den
-  static constexpr size_t a_floats = size_t(HAS_U ? 4 : 1) * C * D + (HAS_U ? 4 : 2) * C * CP +
-                                     2 * NWG * C + 3 * C;
-  //   Z0s [, W0s, Uf[2]] | Ws, Ls [, Xs, PTs] | N2p, denp | delta, 1/delta, -1/delta
-  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + (HAS_U ? 2 * C * CP : 0);
+  static constexpr int a_big = UT ? 4 : 1;       // Z0s [, W0s, Uf[2]]
+  static constexpr int a_small = UT ? 6 : (GEN ? 4 : 2);
+  //   Ws, Ls [, PTs, Guu] [, Xs, Guk]
+  static constexpr size_t a_floats = size_t(a_big) * C * D + size_t(a_small) * C * CP +
+                                     2 * NWG * C + 3 * C + 32;
+  //   ... | N2p, denp | delta, 1/delta, -1/delta | eta * refresh counts [C + 1] (padded)
+  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + (GEN ? 2 * C * CP : 0);
   //   VS(B), R0s, Eps | ostage[2] [| GuL, HTL]
   static constexpr size_t smem_bytes = raw_bytes +
       (KRING * kslot_floats + RING * slot_floats + a_floats + s_floats) * sizeof(float) +
@@ -344,10 +360,12 @@ __device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) 
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-template <int D, typename TIn, bool BALANCED, bool HAS_U>
+template <int D, typename TIn, bool BALANCED, int UM>
 __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanParams p,
                                                                   const SchedParams sp) {
-  using Cfg = ChunkCfg<D, TIn, HAS_U>;
+  using Cfg = ChunkCfg<D, TIn, UM>;
+  constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly
+  constexpr bool UT = Cfg::UT;       // u comes from the caller's tensor
   constexpr int NIN = Cfg::NIN;
   constexpr int C = Cfg::C, TW = Cfg::TW, TR = Cfg::TR, LPR = Cfg::LPR, NV = Cfg::NV;
   constexpr int NG = Cfg::NG, NWG = Cfg::NWG, NSTAGE = Cfg::NSTAGE, RING = Cfg::RING;
@@ -361,25 +379,28 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   float* kring = fbase;                               // [KRING] { Kh, Qf, Vf : [C][D], nrm[C] }
   float* zring = kring + KRING * Cfg::kslot_floats;   // [RING] { Zs[C][D], GuT, HT : [C][CP], sc, inv_den : [C] }
   float* abase = zring + RING * Cfg::slot_floats;
-  float* Z0s = abase;                              // [C][D]  A U^T, then Z in place (explicit u)
-  float* W0s = Z0s + C * D;                        // [C][D]  A K^T            (explicit u only)
-  float* Ufs = W0s + C * D;                        // [2][C][D] widened u      (explicit u only)
-  float* Ws = abase + (HAS_U ? 4 : 1) * C * D;     // [C][CP] U A U^T (K A K^T when u = k_hat)
+  float* Z0s = abase;                              // [C][D]  A U^T, then Z in place (general path)
+  float* W0s = UT ? Z0s + C * D : Z0s;             // [C][D]  A K^T (== A U^T unless u is a tensor)
+  float* Ufs = Z0s + 2 * C * D;                    // [2][C][D] widened u      (u tensor only)
+  float* Ws = abase + Cfg::a_big * C * D;          // [C][CP] U A U^T (K A K^T when u = k_hat)
   float* Ls = Ws + C * CP;                         // [C][CP] unit lower factor
-  float* Xs = Ls + C * CP;                         // [C][CP] U A K^T          (explicit u only)
-  float* PTs = Xs + C * CP;                        // [C][CP] PT[t][s] = (z_s.k_t)/delta_s (explicit u only)
-  float* N2p = Ws + (HAS_U ? 4 : 2) * C * CP;      // [NWG][C]
+  float* PTs = Ls + C * CP;                        // [C][CP] PT[t][s] = (z_s.k_t)/delta_s (general path)
+  float* Guu = PTs + C * CP;                       // [C][CP] U U^T, refresh only (general path)
+  float* Xs = UT ? Guu + C * CP : Ws;              // [C][CP] U A K^T (== W unless u is a tensor)
+  float* Guk = UT ? Xs + C * CP : Guu;             // [C][CP] U K^T, refresh only
+  float* N2p = Ws + Cfg::a_small * C * CP;         // [NWG][C]
   float* denp = N2p + NWG * C;                     // [NWG][C]
   float* dlt = denp + NWG * C;                     // [C]
   float* idl = dlt + C;                            // [C]  1/delta
   float* nidl = idl + C;                           // [C] -1/delta
+  float* nrs = nidl + C;                           // [C+1] eta * (refreshes before token t of the chunk)
   float* sbase = abase + Cfg::a_floats;
   float* VS = sbase;                // [C][D]  B = V^T - S K^T
   float* R0s = VS + C * D;          // [C][D]
   float* Eps = R0s + C * D;         // [C][D]
   float* ostage = Eps + C * D;      // [2][C][D]
-  float* GuL = ostage + 2 * C * D;  // [C][CP] GuL[t][s] = k_hat_t . a_s   (explicit u only)
-  float* HTL = GuL + C * CP;        // [C][CP] HTL[t][s] = q_t . a_s       (explicit u only)
+  float* GuL = ostage + 2 * C * D;  // [C][CP] GuL[t][s] = k_hat_t . a_s   (general path)
+  float* HTL = GuL + C * CP;        // [C][CP] HTL[t][s] = q_t . a_s       (general path)
   uint64_t* bars = reinterpret_cast<uint64_t*>(
       (reinterpret_cast<uintptr_t>(sbase + Cfg::s_floats) + 15) & ~uintptr_t(15));
   uint64_t* full = bars;                    // [NSTAGE] raw stage filled by TMA
@@ -442,7 +463,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &full[s]);
     bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &full[s]);
     bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
-    if (HAS_U) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
+    if (UT) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
   };
 
   // (re)arm the barriers of this piece; a tail piece also waits for its unit's head
@@ -519,7 +540,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       const TIn* rq = raw + (size_t(s) * NIN + 0) * C * D;
       const TIn* rk = raw + (size_t(s) * NIN + 1) * C * D;
       const TIn* rv = raw + (size_t(s) * NIN + 2) * C * D;
-      const TIn* ru = raw + (size_t(s) * NIN + (HAS_U ? 3 : 0)) * C * D;
+      const TIn* ru = raw + (size_t(s) * NIN + (UT ? 3 : 0)) * C * D;
       float* Uf = Ufs + size_t(c & 1) * C * D;   // penalty directions, verbatim
       float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
       float* Qf = Kh + C * D;
@@ -549,7 +570,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           }
           reinterpret_cast<float4*>(Qf + tt * D)[f] = qf;
           reinterpret_cast<float4*>(Vf + tt * D)[f] = vv;
-          if (HAS_U)
+          if (UT)
             reinterpret_cast<float4*>(Uf + tt * D)[f] =
                 act ? load4(ru + tt * D, f) : make_float4(0.f, 0.f, 0.f, 0.f);
           ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
@@ -591,6 +612,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       zk = p.z0[size_t(unit) * D + g];
     }
 
+    // Periodic refresh (general path): ph = tokens since the last refresh boundary
+    const bool rf_on = HAS_U && p.refresh_period > 0;
+    const int rfP = rf_on ? p.refresh_period : 1;
+    int ph = rf_on ? int((p.step_offset + t_begin) % rfP) : 0;
+
     if (nchunks > 0) prep_inputs(0, 0, NWG);
     group_bar(1, NG);
     if (g == 0 && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
@@ -605,6 +631,15 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       float* scs = HT + C * CP;
       float* inv_den = scs + C;
       VLA_MARK(0)
+
+      // ---- refresh counts: nrs[t] = eta * (refreshes after tokens < t of this chunk), so that
+      //      token t sees A + nrs[t] I in its Sherman-Morrison step and A + nrs[t+1] I in a_t
+      const int nv = min(C, T - c * C);                 // valid tokens of the chunk
+      const bool rf_chunk = rf_on && (ph + nv) >= rfP;  // at least one refresh inside
+      if (rf_on) {
+        if (g <= C) nrs[g] = p.refresh_eta * float((ph + min(g, nv)) / rfP);
+        ph = (ph + nv) % rfP;
+      }
 
       // ---- running key sum and readout denominators (thread = column g): partial sums
       //      over this warp's columns of q_f,t . zkey_t
@@ -621,16 +656,20 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       }
 
       // ---- Z0 = A U^T (U = K when no u is given); with an explicit u also W0 = A K^T
-      const float* Uf = HAS_U ? (Ufs + size_t(c & 1) * C * D) : Kh;
+      const float* Uf = UT ? (Ufs + size_t(c & 1) * C * D) : Kh;
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Uf, cg, [&](int t, float x) { Z0s[t * D + g] = x; });
-      if (HAS_U)
+      if (UT)
         tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) { W0s[t * D + g] = x; });
       group_bar(1, NG);
       VLA_MARK(1)
 
       // ---- W = U Z0 (C x C, symmetric); with an explicit u also X[s][t] = u_s . (A k_hat_t)
       gram16<D, NG, CP>(Uf, Z0s, Ws, g);
-      if (HAS_U) gram16<D, NG, CP>(Uf, W0s, Xs, g);
+      if (UT) gram16<D, NG, CP>(Uf, W0s, Xs, g);
+      if (rf_chunk) {   // U U^T and U K^T for the refresh terms
+        gram16<D, NG, CP>(Uf, Uf, Guu, g);
+        if (UT) gram16<D, NG, CP>(Uf, Kh, Guk, g);
+      }
       group_bar(1, NG);
       VLA_MARK(2)
 
@@ -652,6 +691,12 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         float m[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) m[j] = Ws[r * CP + h * 8 + j] + ((h * 8 + j == r) ? 1.0f : 0.0f);
+        if (rf_chunk) {
+          // tokens s <= t: u_s . (A + nrs[s] I) u_t, i.e. the count of the earlier token
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            m[j] = fmaf(nrs[min(r, h * 8 + j)], Guu[r * CP + h * 8 + j], m[j]);
+        }
 #pragma unroll
         for (int s2 = 0; s2 < 16; ++s2) {
           const int hs = s2 >> 3, js = s2 & 7;
@@ -678,6 +723,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 #pragma unroll
           for (int s2 = 0; s2 < 16; ++s2) {
             float a0 = Xs[s2 * CP + t], a1 = 0.f;
+            if (rf_chunk) a0 = fmaf(nrs[s2], Guk[s2 * CP + t], a0);
 #pragma unroll
             for (int r4 = 0; r4 * 4 < s2; ++r4) {
               const float4 l4 = reinterpret_cast<const float4*>(Ls + s2 * CP)[r4];
@@ -702,11 +748,13 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       VLA_MARK(4)
 
       // ---- row g of Z by forward substitution: z_t = z0_t - sum_{s<t} L[t][s] z_s
+      const float rf_tot = rf_chunk ? nrs[nv] : 0.0f;   // eta * refreshes in this chunk
       {
         float z[16];
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
           float a0 = Z0s[t * D + g], a1 = 0.f;
+          if (rf_chunk) a0 = fmaf(nrs[t], Uf[t * D + g], a0);
 #pragma unroll
           for (int s4 = 0; s4 * 4 < t; ++s4) {
             const float4 l4 = reinterpret_cast<const float4*>(Ls + t * CP)[s4];
@@ -731,6 +779,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 #pragma unroll
           for (int t = 0; t < 16; ++t) {
             float a0 = W0s[t * D + g], a1 = 0.f;
+            if (rf_chunk) a0 = fmaf(nrs[t + 1], Kh[t * D + g], a0);
 #pragma unroll
             for (int s4 = 0; s4 * 4 <= t; ++s4) {
               const float4 p4 = reinterpret_cast<const float4*>(PTs + t * CP)[s4];
@@ -787,6 +836,18 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       {
         const float* Zown = HAS_U ? Z0s : Zs;
         tile_rank_update<TR, TW, LPR, D, C>(st, Zown, Zown, nidl, rb, cg);
+        if (rf_chunk) {   // + eta I per refresh: the diagonal entries that fall in this tile
+#pragma unroll
+          for (int r = 0; r < TR; ++r)
+#pragma unroll
+            for (int m = 0; m < NV; ++m) {
+              const int dcol = rb * TR + r - (m * LPR + cg) * 4;   // row - first column of the quad
+              if (dcol == 0) st[r][2 * m].x += rf_tot;
+              if (dcol == 1) st[r][2 * m].y += rf_tot;
+              if (dcol == 2) st[r][2 * m + 1].x += rf_tot;
+              if (dcol == 3) st[r][2 * m + 1].y += rf_tot;
+            }
+        }
       }
       VLA_MARK(7)
     }

@@ -49,9 +49,7 @@ def test_forced_chunk_kernel_rejects_what_it_does_not_cover():
     with pytest.raises(vla.VlaError) as ei:
         vla.vla_forward(q, k, v, 1.0, kernel=vla.VLA_KERNEL_CHUNK)
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
-    w = _small(64, 8, "f32")
-    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
-    with pytest.raises(vla.VlaError):          # the periodic refresh lives in the token kernel
+    with pytest.raises(vla.VlaError):          # with the periodic refresh as well
         vla.vla_forward(q, k, v, 1.0, refresh=(20, 1e-3, 0), kernel=vla.VLA_KERNEL_CHUNK)
 
 
@@ -133,29 +131,51 @@ def test_more_units_than_resident_ctas(d, units, flags):
 @pytest.mark.parametrize("d", [16, 32, 128])
 @pytest.mark.parametrize("flags", [0, IDENT])
 @pytest.mark.parametrize("umode", ["khat", "unit_over_sqrt_d"])
-def test_periodic_refresh_as_in_algorithm_1(d, flags, umode):
+@pytest.mark.parametrize("kernel", ["token", "chunk"])
+def test_periodic_refresh_as_in_algorithm_1(d, flags, umode, kernel):
     """Algorithm 1 to the letter: lambda_0 = 0.1, A += 1e-3 I every 20 steps, with and without an
-    explicit u, in one call and split in two with the step offset carried."""
+    explicit u, in one call and split in two with the step offset carried, on both kernels."""
+    if kernel == "chunk" and d < 32:
+        pytest.skip("the chunk kernel starts at d = 32")
+    kern = KERNELS[kernel]
     w = _small(d, 130, "f32", units=(1, 3), seed=500 + d)
     q, k, v = W.make_inputs(w)
     u = None if umode == "khat" else W.make_u(w, d ** -0.5)
     rf = (20, 1e-3, 0)
-    errs, got, ref = check_parity(q, k, v, 0.1, 1e-4, u=u, flags=flags, refresh=rf, label="refresh d=%d" % d)
+    errs, got, ref = check_parity(q, k, v, 0.1, 1e-4, u=u, flags=flags, refresh=rf, kernel=kern,
+                                  label="refresh %s d=%d" % (kernel, d))
     plain = run_oracle(q, k, v, 0.1, u=u, flags=flags)
     assert np.abs(plain.A_T - ref.A_T).max() > 1e-4           # the refresh is visible in A_T
     T1 = 53
     sl = lambda x, a, b: None if x is None else x[:, :, a:b].contiguous()
-    a = run_gpu(sl(q, 0, T1), sl(k, 0, T1), sl(v, 0, T1), 0.1, u=sl(u, 0, T1), flags=flags, refresh=rf)
+    a = run_gpu(sl(q, 0, T1), sl(k, 0, T1), sl(v, 0, T1), 0.1, u=sl(u, 0, T1), flags=flags, refresh=rf,
+                kernel=kern)
     b = run_gpu(sl(q, T1, 130), sl(k, T1, 130), sl(v, T1, 130), 0.1, u=sl(u, T1, 130), flags=flags,
-                S0=a.S_T, A0=a.A_T, z0=a.z_T, refresh=(20, 1e-3, T1))
+                S0=a.S_T, A0=a.A_T, z0=a.z_T, refresh=(20, 1e-3, T1), kernel=kern)
     assert rel_err(torch.cat([a.out, b.out], dim=2), ref.out) <= 1e-4
     assert rel_err(b.A_T, ref.A_T) <= 1e-4 and rel_err(b.S_T, ref.S_T) <= 1e-4
-    # the chunk kernel does not implement the refresh and says so when forced
-    if d >= 32 and u is None:
-        dev = torch.device("cuda:0")
-        with pytest.raises(vla.VlaError) as ei:
-            vla.vla_forward(q.to(dev), k.to(dev), v.to(dev), 0.1, refresh=rf, kernel=vla.VLA_KERNEL_CHUNK)
-        assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("period,eta,offset", [(1, 1e-3, 0), (3, 5e-3, 2), (16, 1e-2, 0), (17, 1e-2, 16),
+                                               (20, 1e-3, 19), (37, 0.05, 1000003), (500, 0.1, 0)])
+@pytest.mark.parametrize("d,dtype", [(32, "f32"), (64, "bf16"), (128, "bf16")])
+def test_refresh_periods_and_offsets_on_the_chunk_kernel(period, eta, offset, d, dtype):
+    """Several refreshes inside one 16-token chunk, none at all, refreshes that fall on chunk
+    boundaries and on the ragged last chunk, and a large carried step offset."""
+    w = _small(d, 83, dtype, units=(1, 2), seed=900 + d + period)
+    q, k, v = W.make_inputs(w)
+    rf = (period, eta, offset)
+    for u in (None, W.make_u(w, d ** -0.5)):
+        check_parity(q, k, v, 0.1, 1e-4, u=u, refresh=rf, kernel=vla.VLA_KERNEL_CHUNK,
+                     label="chunk refresh P=%d d=%d" % (period, d))
+
+
+def test_refresh_on_the_balanced_schedule():
+    """More units than resident CTAs with the refresh: cut units carry the refresh phase."""
+    w = _small(64, 200, "bf16", units=(5, 61), seed=77)
+    q, k, v = W.make_inputs(w)
+    check_parity(q, k, v, 0.1, 1e-4, refresh=(20, 1e-3, 7), kernel=vla.VLA_KERNEL_CHUNK,
+                 label="balanced refresh")
 
 
 def test_in_place_state_and_canaries():

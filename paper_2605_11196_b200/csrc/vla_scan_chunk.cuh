@@ -124,7 +124,9 @@ struct ChunkCfg {
   static constexpr size_t a_floats = size_t(a_big) * C * D + size_t(a_small) * C * CP +
                                      2 * NWG * C + 3 * C + 32;
   //   ... | N2p, denp | delta, 1/delta, -1/delta | eta * refresh counts [C + 1] (padded)
-  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + (GEN ? 2 * C * CP : 0);
+  // group S forms q_t . z_s itself where it is the group with time to spare (d <= 64)
+  static constexpr bool S_HT = !GEN && D <= 64;
+  static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + ((GEN || S_HT) ? 2 * C * CP : 0);
   //   VS(B), R0s, Eps | ostage[2] [| GuL, HTL]
   static constexpr size_t smem_bytes = raw_bytes +
       (KRING * kslot_floats + RING * slot_floats + a_floats + s_floats) * sizeof(float) +
@@ -528,9 +530,10 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 
   if (is_A) {
     // =====================================================================  group A
-    // Input prep of chunk c by the warps [w0, w0 + nw): k_hat, ||phi(k)||, q_f and v as fp32
-    // rows in ring slot c % KRING (zero rows past the end of the sequence).
-    auto prep_inputs = [&](int c, int w0, int nw) {
+    // Input prep of tokens [tok_lo, tok_hi) of chunk c by the warps [w0, w0 + nw): k_hat,
+    // ||phi(k)||, q_f and v as fp32 rows in ring slot c % KRING (zero rows past the end of
+    // the sequence).  tok_lo and tok_hi are multiples of the tokens a warp takes per pass.
+    auto prep_inputs = [&](int c, int w0, int nw, int tok_lo = 0, int tok_hi = Cfg::C) {
       constexpr int LPT = (D >= 128) ? 16 : 8;   // lanes per token
       constexpr int NF = D / (4 * LPT);          // float4 groups per lane and tensor
       constexpr int TPW = 32 / LPT;              // tokens per warp pass
@@ -589,9 +592,9 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         if (pl == 0) nrm[tt] = (tt < n) ? nr : 0.0f;
       };
       // two tokens per lane group and iteration, so that their dependency chains interleave
-      for (int tok0 = (gw - w0) * TPW; tok0 < C; tok0 += 2 * nw * TPW) {
+      for (int tok0 = tok_lo + (gw - w0) * TPW; tok0 < tok_hi; tok0 += 2 * nw * TPW) {
         const int ta = tok0 + sub, tb = tok0 + nw * TPW + sub;
-        const bool two = tok0 + nw * TPW < C;   // warp-uniform
+        const bool two = tok0 + nw * TPW < tok_hi;   // warp-uniform
         float4 ka[NF], kb[NF];
         float sa = token(ta, ka), sb = 0.f;
         if (two) sb = token(tb, kb);
@@ -604,6 +607,10 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         if (two) finish(tb, sb, kb);
       }
     };
+
+    // tokens [0, kPrepSplit) of the next chunk are widened by warps 1.., the rest by warp 0
+    // after the factorisation
+    constexpr int kPrepSplit = (NWG == 1) ? 0 : (NWG == 2) ? 12 : C;
 
     float zk = 0.0f;  // running sum of phi(k), column g
     if (from_handoff) {
@@ -737,9 +744,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           }
         }
         VLA_MARK(8)
-        if (NWG == 1 && c + 1 < nchunks) prep_inputs(c + 1, 0, 1);
+        // the factorising warp takes the tail of the prep where the other warps would
+        // otherwise finish after it (one other warp at d = 64, none at d = 32)
+        if (c + 1 < nchunks && kPrepSplit < C) prep_inputs(c + 1, 0, 1, kPrepSplit, C);
       } else {
-        if (c + 1 < nchunks) prep_inputs(c + 1, 1, NWG - 1);
+        if (c + 1 < nchunks) prep_inputs(c + 1, 1, NWG - 1, 0, kPrepSplit);
         VLA_MARK(8)
       }
       group_bar(1, NG);
@@ -825,9 +834,10 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           }
         }
       }
-      // ---- HT[t][s] = q_t . z_s (C x C), then publish the chunk to group S.  With an
-      //      explicit u group S forms its two small matrices from a itself.
-      if (!HAS_U) gram16<D, NG, CP>(Qf, Zs, HT, g);
+      // ---- HT[t][s] = q_t . z_s (C x C), then publish the chunk to group S.  On the general
+      //      path group S forms its two small matrices from a itself, and at d <= 64 it forms
+      //      HT as well (there group A is the longer chain).
+      if (!HAS_U && !Cfg::S_HT) gram16<D, NG, CP>(Qf, Zs, HT, g);
       group_bar(1, NG);
       if (g == 0) mbar_arrive(&ring_full[slot]);
       VLA_MARK(6)
@@ -896,6 +906,10 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         gram16<D, NG, CP>(Qf, Zs, HTL, g);
         group_bar(2, NG);
         Gm = GuL;
+        Hm = HTL;
+      } else if (Cfg::S_HT) {
+        gram16<D, NG, CP>(Qf, Zs, HTL, g);
+        group_bar(2, NG);
         Hm = HTL;
       }
       VLA_MARK(2)

@@ -387,6 +387,38 @@ def main():
                          "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
                          "hbm_frac": alg_bytes_per_token(ww.d, ib) * ww.tokens / (ms * 1e-3) / 1e9 / hbm_peak,
                          "units": ww.units, "unit_limited_frac_bound": min(ww.units, n_sm) / n_sm}
+            # fewer units than SMs: the sequence-parallel entry point cuts each sequence into
+            # segments that are scanned concurrently (twice the arithmetic, P times the CTAs)
+            P = vla.seqpar_segments(ww.B, ww.H, ww.T, ww.d, q2.dtype)
+            if P > 1:
+                qd2, kd2, vd2 = q2.to(dev), k2.to(dev), v2.to(dev)
+                ws = torch.empty((vla.seqpar_workspace_bytes(ww.B, ww.H, ww.T, ww.d, P),),
+                                 dtype=torch.uint8, device=dev)
+                o2 = torch.empty((ww.B, ww.H, ww.T, ww.d), dtype=torch.float32, device=dev)
+                S2 = torch.empty((ww.B, ww.H, ww.d, ww.d), dtype=torch.float32, device=dev)
+                A2 = torch.empty_like(S2)
+                z2 = torch.empty((ww.B, ww.H, ww.d), dtype=torch.float32, device=dev)
+                st2 = torch.zeros((), dtype=torch.int32, device=dev)
+                call3 = lambda: vla.vla_forward_seqpar(qd2, kd2, vd2, ww.lam, segments=P, workspace=ws,
+                                                       out=o2, S_T=S2, A_T=A2, z_T=z2, status=st2,
+                                                       stream=stream)
+                ms = []
+                with torch.cuda.stream(stream):
+                    for _ in range(3):
+                        call3()
+                    for _ in range(10):
+                        fl.fill_(1)
+                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a.record(stream); call3(); b.record(stream)
+                        ms.append((a, b))
+                torch.cuda.synchronize(dev)
+                ms = float(np.median([a.elapsed_time(b) for a, b in ms]))
+                per[name + "_seqpar"] = {
+                    "ms": ms, "segments": P, "tokens_per_s": ww.tokens / (ms * 1e-3),
+                    "ns_per_scan_step": 1e6 * ms / ww.T,
+                    "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
+                    "status": int(st2.item()), "gpu_launches_per_step": 5}
+                del qd2, kd2, vd2, ws, o2
         # the headline workload with an explicit penalty direction u = unit / sqrt(d_h)
         # (the paper's learned-u setting at the scan's input level)
         uu = W.make_u(w, w.d ** -0.5).to(dev)

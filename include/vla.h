@@ -149,6 +149,40 @@ int vla_forward_host_static(const void* q, const void* k, const void* v, float l
                             float* out, float* S_T, float* A_T,
                             const vla_opts_t* opts, void* stream);
 
+/*
+ * vla_forward_seqpar -- the same forward scan with each unit's sequence cut into `segments`
+ * equal pieces that are scanned at the same time (for long sequences with few (batch, head)
+ * units, where one CTA per unit leaves most of the GPU idle).  It follows the parallel form
+ * of Section 3.4 with the composition written as the recurrence needs it: the memory map
+ * acts on the right, S_t = S_{t-1} (I - k_hat_t alpha_t^T) + v_t alpha_t^T, so a segment
+ * composes to S_end = S_start P + G; and A at a segment start is the inverse of
+ * lambda I + sum of u u^T over the earlier tokens (Eq. "penalty"), formed in fp64.  Results
+ * equal vla_forward's up to rounding.
+ *
+ * Arguments as vla_forward, with these differences: A_0 is always I/lambda (there is no A0);
+ * the periodic refresh and VLA_KERNEL_TOKEN are not available (VLA_ERR_UNSUPPORTED), nor is
+ * d = 16; `segments` must divide T/16 (T a multiple of 16), else VLA_ERR_INVALID_ARG;
+ * segments <= 0 lets the library choose (vla_seqpar_segments), and a choice of 1 runs
+ * vla_forward.  `workspace` is a DEVICE buffer of at least
+ * vla_seqpar_workspace_bytes(B, H, T, d_k, segments) bytes (any alignment; with
+ * segments <= 0 size it for vla_seqpar_segments(...)), owned by the caller and free for
+ * reuse once the work enqueued on `stream` has completed.
+ */
+int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda_,
+                       int B, int H, int T, int d_k, int d_v,
+                       const float* S0,
+                       float* out, float* S_T, float* A_T,
+                       const vla_opts_t* opts, int segments,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* Segments per unit that vla_forward_seqpar picks on the current device for this problem:
+   enough to fill the GPU with 2 * B * H * segments concurrent scans, at least 256 tokens each;
+   1 when cutting does not pay (or the shape is not covered). */
+int vla_seqpar_segments(int B, int H, int T, int d_k, int qkv_dtype);
+
+/* Device bytes vla_forward_seqpar needs for `segments` >= 1 (0 on a bad argument). */
+size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
+
 /* Device bytes vla_forward_host needs for these sizes (0 on invalid sizes). */
 size_t vla_host_workspace_bytes(int B, int H, int T, int d_k, int d_v, int qkv_dtype, int has_u);
 

@@ -9,4 +9,5 @@ from .binding import (VLA_BF16, VLA_ERR_ALIGNMENT, VLA_ERR_CUDA, VLA_ERR_DEVICE_
                       VLA_KERNEL_CHUNK, VLA_KERNEL_TOKEN, VLA_OK, VlaError, VlaOpts, VlaResult, library_path,
                       load_library, status_string, vla_forward, vla_forward_host,
                       vla_forward_host_static, VLA_ERR_TOO_LARGE, VLA_STATIC_SCRATCH_BYTES,
-                      vla_host_workspace_bytes, vla_query_support, vla_version)
+                      vla_host_workspace_bytes, vla_query_support, vla_version,
+                      vla_forward_seqpar, seqpar_segments, seqpar_workspace_bytes)

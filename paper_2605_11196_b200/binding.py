@@ -25,6 +25,7 @@ VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE = 1, 2
 VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK = 0, 1, 2
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",
+           "vla_forward_seqpar", "vla_seqpar_segments", "vla_seqpar_workspace_bytes",
            "vla_query_support", "vla_status_string", "vla_version")
 
 
@@ -72,6 +73,13 @@ def load_library():
             lib.vla_forward_host_static.restype = i
             lib.vla_forward_host_static.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp,
                                                     ctypes.POINTER(VlaOpts), vp]
+            lib.vla_forward_seqpar.restype = i
+            lib.vla_forward_seqpar.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp, i,
+                                               vp, ctypes.c_size_t, vp]
+            lib.vla_seqpar_segments.restype = i
+            lib.vla_seqpar_segments.argtypes = [i, i, i, i, i]
+            lib.vla_seqpar_workspace_bytes.restype = ctypes.c_size_t
+            lib.vla_seqpar_workspace_bytes.argtypes = [i, i, i, i, i]
             lib.vla_host_workspace_bytes.restype = ctypes.c_size_t
             lib.vla_host_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
             lib.vla_query_support.restype = i
@@ -190,6 +198,64 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
                              ctypes.byref(opts), ctypes.c_void_p(st.cuda_stream))
     if rc != VLA_OK:
         raise VlaError(rc, "vla_forward")
+    return VlaResult(out, S_T, A_T, z_T, status)
+
+
+def seqpar_segments(B: int, H: int, T: int, d_k: int, dtype: torch.dtype) -> int:
+    """Segments per unit that ``vla_forward_seqpar`` would choose on the current device."""
+    code = VLA_BF16 if dtype == torch.bfloat16 else VLA_F32
+    return int(load_library().vla_seqpar_segments(B, H, T, d_k, code))
+
+
+def seqpar_workspace_bytes(B: int, H: int, T: int, d_k: int, segments: int) -> int:
+    return int(load_library().vla_seqpar_workspace_bytes(B, H, T, d_k, segments))
+
+
+def vla_forward_seqpar(q, k, v, lam: float, *, segments: int = 0, workspace=None, u=None, S0=None,
+                       z0=None, flags: int = 0, eps: float = 1e-4, out=None, S_T=None, A_T=None,
+                       z_T=None, status=None, stream: Optional[torch.cuda.Stream] = None,
+                       want_status: bool = True) -> VlaResult:
+    """Sequence-parallel scan of CUDA tensors: each unit's sequence is cut into ``segments``
+    pieces that are scanned concurrently (0 = let the library choose).  ``workspace`` is a CUDA
+    uint8 tensor of at least ``seqpar_workspace_bytes`` bytes (allocated with torch if absent)."""
+    lib = load_library()
+    if q.dim() != 4:
+        raise ValueError("q must be [B,H,T,d_k]")
+    B, H, T, dk = q.shape
+    dv = v.shape[-1]
+    dt = _dtype_code(q)
+    dev = q.device
+    _chk(q, (B, H, T, dk), q.dtype, "q"); _chk(k, (B, H, T, dk), q.dtype, "k")
+    _chk(v, (B, H, T, dv), q.dtype, "v"); _chk(u, (B, H, T, dk), q.dtype, "u")
+    f32 = torch.float32
+    _chk(S0, (B, H, dv, dk), f32, "S0"); _chk(z0, (B, H, dk), f32, "z0")
+    if out is None:
+        out = torch.empty((B, H, T, dv), dtype=f32, device=dev)
+    if S_T is None:
+        S_T = torch.empty((B, H, dv, dk), dtype=f32, device=dev)
+    if A_T is None:
+        A_T = torch.empty((B, H, dk, dk), dtype=f32, device=dev)
+    if z_T is None:
+        z_T = torch.empty((B, H, dk), dtype=f32, device=dev)
+    _chk(out, (B, H, T, dv), f32, "out"); _chk(S_T, (B, H, dv, dk), f32, "S_T")
+    _chk(A_T, (B, H, dk, dk), f32, "A_T"); _chk(z_T, (B, H, dk), f32, "z_T")
+    if status is None and want_status:
+        status = torch.zeros((), dtype=torch.int32, device=dev)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        P = segments if segments > 0 else int(lib.vla_seqpar_segments(B, H, T, dk, dt))
+        need = int(lib.vla_seqpar_workspace_bytes(B, H, T, dk, max(P, 1)))
+        if workspace is None:
+            workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
+        if workspace.device != dev or workspace.dtype != torch.uint8 or not workspace.is_contiguous():
+            raise ValueError("workspace must be a contiguous CUDA uint8 tensor on the inputs' device")
+        opts = _make_opts(dt, u, flags, eps, z0, z_T, status, VLA_KERNEL_AUTO, None)
+        rc = lib.vla_forward_seqpar(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv,
+                                    _ptr(S0), _ptr(out), _ptr(S_T), _ptr(A_T), ctypes.byref(opts),
+                                    int(segments), _ptr(workspace), workspace.numel(),
+                                    ctypes.c_void_p(st.cuda_stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_forward_seqpar")
     return VlaResult(out, S_T, A_T, z_T, status)
 
 

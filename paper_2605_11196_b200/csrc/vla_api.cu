@@ -11,6 +11,7 @@
 #include "vla_common.cuh"
 #include "vla_scan_token.cuh"
 #include "vla_scan_chunk.cuh"
+#include "vla_seqpar.cuh"
 
 namespace {
 
@@ -205,6 +206,114 @@ void* static_scratch_for_current_device() {
   return g_scratch_addr[dev];
 }
 
+// ---- sequence-parallel entry point: workspace layout and segment choice
+struct SeqParLayout {
+  size_t Gd, zsum, Astart, zstart, ST2, AT2, zT2, wn, Sstart, total;
+};
+
+SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
+  const size_t N = units * P;
+  SeqParLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t at = off; off += round256(bytes); return at; };
+  L.Gd = take(N * D * D * sizeof(double));
+  L.zsum = take(N * D * sizeof(float));
+  L.Astart = take(N * D * D * sizeof(float));
+  L.zstart = take(N * D * sizeof(float));
+  L.ST2 = take(2 * N * D * D * sizeof(float));
+  L.AT2 = take(2 * N * D * D * sizeof(float));
+  L.zT2 = take(2 * N * D * sizeof(float));
+  L.wn = take(units * T * D * sizeof(float));
+  L.Sstart = take(N * D * D * sizeof(float));
+  L.total = off + 256;
+  return L;
+}
+
+// CTAs of the chunk kernel that one device holds at a time (u = k_hat variant).
+template <int D>
+int chunk_resident_ctas(int dtype) {
+  int dev = 0, sms = 0, per_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) {
+    if (dtype == VLA_F32) {
+      using Cfg = vla::ChunkCfg<D, float, vla::kUKhat>;
+      auto kern = vla::vla_scan_chunk_kernel<D, float, false, vla::kUKhat>;
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes));
+      if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes);
+    } else {
+      using Cfg = vla::ChunkCfg<D, uint16_t, vla::kUKhat>;
+      auto kern = vla::vla_scan_chunk_kernel<D, uint16_t, false, vla::kUKhat>;
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes));
+      if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes);
+    }
+  }
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return sms * per_sm;
+}
+
+// Segments per unit: as many as fill the device with 2 * units * P scans, P a divisor of the
+// number of 16-token chunks, at least 256 tokens per segment.  1 = not worth cutting.
+int seqpar_choose_segments(int units, int T, int d, int dtype) {
+  if (units <= 0 || T <= 0 || T % 16 != 0 || d < 32) return 1;
+  int resident = 0;
+  switch (d) {
+    case 32: resident = chunk_resident_ctas<32>(dtype); break;
+    case 64: resident = chunk_resident_ctas<64>(dtype); break;
+    case 128: resident = chunk_resident_ctas<128>(dtype); break;
+    default: return 1;
+  }
+  const int target = resident / (2 * units);
+  const int nch = T / 16;
+  int best = 1;
+  for (int P = 2; P <= target && P <= nch; ++P)
+    if (nch % P == 0 && T / P >= 256) best = P;
+  return best;
+}
+
+template <int D>
+int launch_seqpar(const vla::SeqParParams& sp, const ScanParams& scan, int dtype, float* A_T,
+                  float* zT, const float* AT2, const float* zT2, cudaStream_t st) {
+  const int N = sp.units * sp.P;
+  const int Ls = sp.T / sp.P;
+  const size_t inv_smem = (size_t(D) * (D + 1) + 2 * D) * sizeof(double);
+  const size_t comb_smem = 2 * size_t(D) * (D + 1) * sizeof(float);
+  const size_t corr_smem = (size_t(D) * (D + 1) + 64 * size_t(D)) * sizeof(float);
+  if (cudaFuncSetAttribute(vla::seqpar_invert_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(inv_smem)) != cudaSuccess ||
+      cudaFuncSetAttribute(vla::seqpar_combine_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(comb_smem)) != cudaSuccess ||
+      cudaFuncSetAttribute(vla::seqpar_correct_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(corr_smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  if (dtype == VLA_F32) vla::seqpar_gram_kernel<D, float><<<N, 256, 0, st>>>(sp);
+  else vla::seqpar_gram_kernel<D, uint16_t><<<N, 256, 0, st>>>(sp);
+  vla::seqpar_invert_kernel<D><<<N, 256, inv_smem, st>>>(sp);
+  if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
+  const int rc = launch_chunk_d<D>(scan, dtype, st);
+  if (rc != VLA_OK) return rc;
+  vla::seqpar_combine_kernel<D><<<sp.units, 256, comb_smem, st>>>(sp);
+  vla::seqpar_correct_kernel<D><<<dim3(N, (Ls + 63) / 64), 256, corr_smem, st>>>(sp);
+  if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
+  // final A and key sum: those of each unit's last segment
+  const size_t P = size_t(sp.P);
+  if (A_T &&
+      cudaMemcpy2DAsync(A_T, size_t(D) * D * 4, AT2 + (P - 1) * D * D, P * D * D * 4, size_t(D) * D * 4,
+                        size_t(sp.units), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return VLA_ERR_CUDA;
+  if (zT && cudaMemcpy2DAsync(zT, size_t(D) * 4, zT2 + (P - 1) * D, P * D * 4, size_t(D) * 4,
+                              size_t(sp.units), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return VLA_ERR_CUDA;
+  return VLA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -233,6 +342,7 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
   p.T = T; p.units = units; p.flags = o.flags;
   p.refresh_period = o.refresh_period; p.refresh_eta = o.refresh_eta;
   p.step_offset = o.step_offset; p.u_is_khat = 0;
+  p.n_main = 0; p.out2 = nullptr;
   return launch(p, d_k, o.qkv_dtype, o.kernel, static_cast<cudaStream_t>(stream));
 }
 
@@ -401,6 +511,80 @@ int vla_forward_host_static(const void* q, const void* k, const void* v, float l
   // nothing left behind by the previous call needs clearing.
   return vla_forward_host(q, k, v, lambda_, B, H, T, d_k, d_v, S0, A0, out, S_T, A_T, opts, scratch,
                           size_t(VLA_STATIC_SCRATCH_BYTES), stream);
+}
+
+int vla_seqpar_segments(int B, int H, int T, int d_k, int qkv_dtype) {
+  if (B <= 0 || H <= 0) return 1;
+  if (qkv_dtype != VLA_F32 && qkv_dtype != VLA_BF16) return 1;
+  const long long units = 1LL * B * H;
+  if (units > 0x7fffffffLL) return 1;
+  return seqpar_choose_segments(int(units), T, d_k, qkv_dtype);
+}
+
+size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments) {
+  if (B < 0 || H < 0 || T < 0 || d_k <= 0 || segments < 1) return 0;
+  return seqpar_layout(size_t(B) * size_t(H), size_t(T), size_t(d_k), size_t(segments)).total;
+}
+
+int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda_, int B, int H,
+                       int T, int d_k, int d_v, const float* S0, float* out, float* S_T, float* A_T,
+                       const vla_opts_t* opts, int segments, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+  vla_opts_t o;
+  int rc = resolve_opts(opts, &o);
+  if (rc != VLA_OK) return rc;
+  rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, nullptr, out);
+  if (rc != VLA_OK) return rc;
+  if (d_k < 32 || o.refresh_period > 0 || o.kernel == VLA_KERNEL_TOKEN) return VLA_ERR_UNSUPPORTED;
+  const void* ptrs[] = {q, k, v, o.u, S0, out, S_T, A_T, o.z0, o.zT};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return VLA_ERR_ALIGNMENT;
+  if (o.status && (reinterpret_cast<uintptr_t>(o.status) & 3u)) return VLA_ERR_ALIGNMENT;
+  const int units = B * H;
+  if (units == 0) return VLA_OK;
+  int P = segments;
+  if (P <= 0) P = seqpar_choose_segments(units, T, d_k, o.qkv_dtype);
+  if (P == 1)   // nothing to cut: the plain scan
+    return vla_forward(q, k, v, lambda_, B, H, T, d_k, d_v, S0, nullptr, out, S_T, A_T, opts, stream);
+  if (T % 16 != 0 || (T / 16) % P != 0) return VLA_ERR_INVALID_ARG;
+  if (2LL * units * P > 0x7fffffffLL) return VLA_ERR_INVALID_ARG;
+  const SeqParLayout L = seqpar_layout(size_t(units), size_t(T), size_t(d_k), size_t(P));
+  if (!workspace || workspace_bytes < L.total) return VLA_ERR_INVALID_ARG;
+  unsigned char* w = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(workspace) + 255) & ~uintptr_t(255));
+  const int N = units * P;
+
+  vla::SeqParParams sp;
+  sp.k = k; sp.u = o.u; sp.S0 = S0; sp.z0 = o.z0; sp.out = out; sp.S_T = S_T;
+  sp.Gd = reinterpret_cast<double*>(w + L.Gd);
+  sp.zsum = reinterpret_cast<float*>(w + L.zsum);
+  sp.Astart = reinterpret_cast<float*>(w + L.Astart);
+  sp.zstart = reinterpret_cast<float*>(w + L.zstart);
+  sp.ST2 = reinterpret_cast<float*>(w + L.ST2);
+  sp.wn = reinterpret_cast<float*>(w + L.wn);
+  sp.Sstart = reinterpret_cast<float*>(w + L.Sstart);
+  sp.lambda = lambda_; sp.eps = o.eps; sp.T = T; sp.P = P; sp.units = units; sp.flags = o.flags;
+  float* AT2 = reinterpret_cast<float*>(w + L.AT2);
+  float* zT2 = reinterpret_cast<float*>(w + L.zT2);
+
+  // every segment and its transfer scan as one launch of 2N units of T / P tokens: a unit's
+  // segments are consecutive blocks of its [T, d] arrays, so the inputs need no copy
+  ScanParams p;
+  p.q = q; p.k = k; p.v = v; p.u = o.u;
+  p.S0 = nullptr; p.A0 = sp.Astart; p.z0 = sp.zstart;
+  p.out = out; p.out2 = reinterpret_cast<float*>(w + L.wn);
+  p.S_T = reinterpret_cast<float*>(w + L.ST2); p.A_T = AT2; p.zT = zT2;
+  p.status = o.status;
+  p.lambda = lambda_; p.eps = o.eps;
+  p.T = T / P; p.units = 2 * N; p.n_main = N; p.flags = o.flags;
+  p.refresh_period = 0; p.refresh_eta = 0.0f; p.step_offset = 0; p.u_is_khat = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  switch (d_k) {
+    case 32: return launch_seqpar<32>(sp, p, o.qkv_dtype, A_T, o.zT, AT2, zT2, st);
+    case 64: return launch_seqpar<64>(sp, p, o.qkv_dtype, A_T, o.zT, AT2, zT2, st);
+    case 128: return launch_seqpar<128>(sp, p, o.qkv_dtype, A_T, o.zT, AT2, zT2, st);
+    default: return VLA_ERR_UNSUPPORTED;
+  }
 }
 
 int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags) {

@@ -31,6 +31,12 @@ struct ScanParams {
   float refresh_eta;
   long long step_offset;     // tokens processed before this call
   int u_is_khat;             // token kernel, two-exchange path: use u = k_hat although no u was given
+  // Sequence-parallel scans (chunk kernel only).  With n_main > 0, units [n_main, units) are
+  // "transfer" scans: unit x reads q, k, u, A0, z0 of unit x - n_main, takes v = 0 and
+  // S0 = I, and writes its readout to out2 instead of out; its S_T is then the product of
+  // the segment's right-acting maps I - k_hat alpha^T.  n_main <= 0: no such units.
+  int n_main;
+  float* out2;               // [units - n_main, T, D]
 #ifdef VLA_SECTION_TIMERS
   long long* dbg;      // debug builds only: per-section clock64 totals of unit 0
 #endif

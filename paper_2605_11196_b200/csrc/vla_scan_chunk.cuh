@@ -445,6 +445,9 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 #pragma unroll 1
   for (int pi = 0; get_piece<BALANCED>(sp, p.units, nch_unit, blockIdx.x, pi, pc); ++pi) {
   const int unit = pc.unit;
+  // transfer scan of a sequence-parallel launch: inputs of unit `uin`, v = 0, S0 = I
+  const bool pscan = p.n_main > 0 && unit >= p.n_main;
+  const int uin = pscan ? unit - p.n_main : unit;
   const int t_begin = pc.cb * C;
   const int T = min(p.T, pc.ce * C) - t_begin;   // tokens of this piece
   const int nchunks = pc.ce - pc.cb;
@@ -456,15 +459,15 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   // global addresses are formed where they are used (two threads of the CTA), so that they
   // do not occupy registers in the FMA loops
   auto issue = [&](int c) {
-    const size_t tok = size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+    const size_t tok = size_t(uin) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
     const int s = c % NSTAGE;
     const int n = min(C, T - c * C);
     const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
     TIn* dst = raw + size_t(s) * NIN * C * D;
-    mbar_arrive_expect_tx(&full[s], NIN * bytes);
+    mbar_arrive_expect_tx(&full[s], (pscan ? NIN - 1 : NIN) * bytes);
     bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &full[s]);
     bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &full[s]);
-    bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
+    if (!pscan) bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
     if (UT) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
   };
 
@@ -505,7 +508,8 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   {
     // a tail piece continues from the state its head left in the caller's output buffers
     // (written by another SM: read past L1)
-    const float* src = from_handoff ? (is_A ? p.A_T : p.S_T) : (is_A ? p.A0 : p.S0);
+    const float* src = from_handoff ? (is_A ? p.A_T : p.S_T) : (is_A ? p.A0 : (pscan ? nullptr : p.S0));
+    const int usrc = from_handoff ? unit : uin;   // a transfer scan reads the A0 of its partner
 #pragma unroll
     for (int r = 0; r < TR; ++r) {
       const int row = rb * TR + r;
@@ -514,9 +518,9 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         const int c4 = m * LPR + cg;
         float4 x;
         if (src) {
-          x = __ldcg(reinterpret_cast<const float4*>(src + (size_t(unit) * D + row) * D) + c4);
+          x = __ldcg(reinterpret_cast<const float4*>(src + (size_t(usrc) * D + row) * D) + c4);
         } else {
-          const float dg = is_A ? 1.0f / p.lambda : 0.0f;
+          const float dg = is_A ? 1.0f / p.lambda : (pscan ? 1.0f : 0.0f);
           x.x = (c4 * 4 + 0 == row) ? dg : 0.0f;
           x.y = (c4 * 4 + 1 == row) ? dg : 0.0f;
           x.z = (c4 * 4 + 2 == row) ? dg : 0.0f;
@@ -563,7 +567,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           if (act) {
             kf[i] = load4(rk + tt * D, f);
             qf = load4(rq + tt * D, f);
-            vv = load4(rv + tt * D, f);
+            if (!pscan) vv = load4(rv + tt * D, f);
             if (!ident) {
               kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
               kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
@@ -616,7 +620,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     if (from_handoff) {
       if (p.zT) zk = __ldcg(p.zT + size_t(unit) * D + g);
     } else if (p.z0) {
-      zk = p.z0[size_t(unit) * D + g];
+      zk = p.z0[size_t(uin) * D + g];
     }
 
     // Periodic refresh (general path): ph = tokens since the last refresh boundary
@@ -959,8 +963,8 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       fence_async_smem();
       group_bar(2, NG);  // Eps and the out stage complete
       if (g == 0) {
-        const size_t tok = size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
-        bulk_store(p.out + tok * D, ostage + size_t(c & 1) * C * D,
+        const size_t tok = size_t(uin) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+        bulk_store((pscan ? p.out2 : p.out) + tok * D, ostage + size_t(c & 1) * C * D,
                    uint32_t(n) * D * sizeof(float));
         bulk_commit();
       }

@@ -1,0 +1,308 @@
+// Sequence-parallel VLA forward: the helper kernels around the chunk kernel.
+//
+// Section 3.4 writes the memory recurrence as a composition of per-token maps.  With the map
+// acting on the right (S_t = S_{t-1} R_t + G_t, R_t = I - k_hat_t alpha_t^T, G_t = v_t alpha_t^T)
+// a segment of tokens composes to S_end = S_start P + G with P = prod R_t and G the state the
+// segment reaches from S = 0.  The penalty side needs no composition at all: A before token t
+// is the inverse of M = lambda I + sum_{s<t} u_s u_s^T (Eq. "penalty"), a prefix SUM, so A at a
+// segment start comes from a Gram matrix and one inversion.  A unit's sequence is therefore cut
+// into P equal segments that are scanned at the same time:
+//
+//   1. gram     G_j = sum_{t in segment j} u_t u_t^T  (fp32 products, fp64 accumulation) and
+//               the segment's sum of phi(k)
+//   2. invert   A_start_j = (lambda I + sum_{i<j} G_i)^-1 in fp64 (Gauss-Jordan, no pivoting:
+//               the matrix is symmetric positive definite), running key sum at the start
+//   3. scan     the chunk kernel over 2 * units * P virtual units: segment j from S = 0
+//               (readout o0_t, final state G_j) and its transfer scan from S = I with v = 0
+//               (readout w_t = P_t q_t / den_t, final state P_j)
+//   4. combine  per unit, in order: S_start_{j+1} = S_start_j P_j + G_j
+//   5. correct  o_t = o0_t + S_start_j w_t
+//
+// All of it is exact algebra; it costs about twice the arithmetic of the plain scan and
+// makes P times as many CTAs, which is what a long sequence with few (batch, head) units needs.
+#pragma once
+
+#include "vla_common.cuh"
+
+namespace vla {
+
+struct SeqParParams {
+  const void* k;        // [units, T, D] raw keys
+  const void* u;        // [units, T, D] explicit penalty directions or nullptr
+  const float* S0;      // [units, D, D] or nullptr
+  const float* z0;      // [units, D] or nullptr
+  float* out;           // [units, T, D] o0 on entry of `correct`, o on exit
+  float* S_T;           // [units, D, D] or nullptr
+  double* Gd;           // [N, D, D]   segment Gram matrices (N = units * P)
+  float* zsum;          // [N, D]      segment sums of phi(k)
+  float* Astart;        // [N, D, D]
+  float* zstart;        // [N, D]
+  const float* ST2;     // [2N, D, D]  G_j, then P_j
+  const float* wn;      // [N, Ls, D]  transfer readouts
+  float* Sstart;        // [N, D, D]
+  float lambda;
+  float eps;
+  int T;                // tokens per unit
+  int P;                // segments per unit
+  int units;
+  uint32_t flags;
+};
+
+__device__ __forceinline__ float seqpar_phi(float x) { return x > 0.0f ? x + 1.0f : __expf(x); }
+
+template <typename TIn>
+__device__ __forceinline__ float load1(const TIn* p, size_t i);
+template <>
+__device__ __forceinline__ float load1<float>(const float* p, size_t i) { return p[i]; }
+template <>
+__device__ __forceinline__ float load1<uint16_t>(const uint16_t* p, size_t i) {
+  return __uint_as_float(uint32_t(p[i]) << 16);
+}
+
+// ---- 1. segment Gram matrix and key sum.  One CTA of 256 threads per (unit, segment); the
+// last segment of a unit needs neither and is skipped.  Thread (ty, tx) of a 16 x 16 grid
+// owns an R x R block of the D x D result, R = D / 16.
+template <int D, typename TIn>
+__global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) {
+  constexpr int R = D / 16;
+  constexpr int TB = 32;          // tokens per shared-memory block (one fp32 partial sum)
+  constexpr int EPL = D / 32;     // elements per lane of a token row
+  __shared__ __align__(16) float U[TB][D + 4];
+  __shared__ float zpart[8][D];
+  const int vu = blockIdx.x, unit = vu / p.P, j = vu % p.P;
+  if (j == p.P - 1) return;
+  const int Ls = p.T / p.P;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ty = tid >> 4, tx = tid & 15;
+  const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
+  const TIn* kk = static_cast<const TIn*>(p.k) + (size_t(unit) * p.T + size_t(j) * Ls) * D;
+  const TIn* uu = p.u ? static_cast<const TIn*>(p.u) + (size_t(unit) * p.T + size_t(j) * Ls) * D : nullptr;
+
+  double accd[R][R];
+#pragma unroll
+  for (int a = 0; a < R; ++a)
+#pragma unroll
+    for (int b = 0; b < R; ++b) accd[a][b] = 0.0;
+  float zs[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) zs[e] = 0.0f;
+
+  for (int t0 = 0; t0 < Ls; t0 += TB) {
+    // rows u_t of this block: k_hat = phi(k)/||phi(k)|| (or k/||k||), or the given u verbatim
+    for (int tt = warp; tt < TB; tt += 8) {
+      const int t = t0 + tt;
+      float x[EPL];
+      float ss = 0.0f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        float kf = 0.0f;
+        if (t < Ls) {
+          kf = load1<TIn>(kk, size_t(t) * D + e * 32 + lane);
+          if (!ident) kf = seqpar_phi(kf);
+        }
+        x[e] = kf;
+        zs[e] += kf;
+        ss = fmaf(kf, kf, ss);
+      }
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+      const float inv = 1.0f / fmaxf(sqrtf(ss), p.eps);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        float v = x[e] * inv;
+        if (uu) v = (t < Ls) ? load1<TIn>(uu, size_t(t) * D + e * 32 + lane) : 0.0f;
+        U[tt][e * 32 + lane] = v;
+      }
+    }
+    __syncthreads();
+    float acc[R][R];
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+      for (int b = 0; b < R; ++b) acc[a][b] = 0.0f;
+#pragma unroll 4
+    for (int tt = 0; tt < TB; ++tt) {
+      float ra[R], cb[R];
+#pragma unroll
+      for (int a = 0; a < R; ++a) { ra[a] = U[tt][ty * R + a]; cb[a] = U[tt][tx * R + a]; }
+#pragma unroll
+      for (int a = 0; a < R; ++a)
+#pragma unroll
+        for (int b = 0; b < R; ++b) acc[a][b] = fmaf(ra[a], cb[b], acc[a][b]);
+    }
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+      for (int b = 0; b < R; ++b) accd[a][b] += double(acc[a][b]);
+    __syncthreads();
+  }
+  double* G = p.Gd + size_t(vu) * D * D;
+#pragma unroll
+  for (int a = 0; a < R; ++a)
+#pragma unroll
+    for (int b = 0; b < R; ++b) G[(ty * R + a) * D + tx * R + b] = accd[a][b];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) zpart[warp][e * 32 + lane] = zs[e];
+  __syncthreads();
+  for (int c = tid; c < D; c += 256) {
+    float s = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += zpart[w][c];
+    p.zsum[size_t(vu) * D + c] = s;
+  }
+}
+
+// ---- 2. A at the start of segment j, and the running key sum there.  One CTA per
+// (unit, segment); dynamic shared memory: D * (D + 1) + 2 * D doubles.
+template <int D>
+__global__ void __launch_bounds__(256) seqpar_invert_kernel(const SeqParParams p) {
+  extern __shared__ __align__(16) unsigned char seqpar_smem[];
+  double* M = reinterpret_cast<double*>(seqpar_smem);   // [D][D + 1]
+  double* colp = M + D * (D + 1);
+  double* rowp = colp + D;
+  constexpr int LD = D + 1;
+  const int vu = blockIdx.x, unit = vu / p.P, j = vu % p.P;
+  const int tid = threadIdx.x;
+  float* A = p.Astart + size_t(vu) * D * D;
+  for (int c = tid; c < D; c += 256) {
+    double s = p.z0 ? double(p.z0[size_t(unit) * D + c]) : 0.0;
+    // the identity-map reading has no readout normaliser: the key sum is carried through
+    if (!(p.flags & VLA_FLAG_IDENTITY_MAP))
+      for (int i = 0; i < j; ++i) s += double(p.zsum[(size_t(unit) * p.P + i) * D + c]);
+    p.zstart[size_t(vu) * D + c] = float(s);
+  }
+  if (j == 0) {
+    const float dg = 1.0f / p.lambda;
+    for (int idx = tid; idx < D * D; idx += 256) A[idx] = (idx / D == idx % D) ? dg : 0.0f;
+    return;
+  }
+  for (int idx = tid; idx < D * D; idx += 256) {
+    const int r = idx / D, c = idx % D;
+    double s = (r == c) ? double(p.lambda) : 0.0;
+    for (int i = 0; i < j; ++i) s += p.Gd[(size_t(unit) * p.P + i) * D * D + idx];
+    M[r * LD + c] = s;
+  }
+  __syncthreads();
+  // in-place Gauss-Jordan inversion
+  for (int pv = 0; pv < D; ++pv) {
+    const double d = 1.0 / M[pv * LD + pv];
+    for (int c = tid; c < D; c += 256) {
+      colp[c] = M[c * LD + pv];
+      rowp[c] = M[pv * LD + c] * d;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < D * D; idx += 256) {
+      const int r = idx / D, c = idx % D;
+      double v;
+      if (r == pv) v = (c == pv) ? d : rowp[c];
+      else if (c == pv) v = -colp[r] * d;
+      else v = M[r * LD + c] - colp[r] * rowp[c];
+      M[r * LD + c] = v;
+    }
+    __syncthreads();
+  }
+  for (int idx = tid; idx < D * D; idx += 256) A[idx] = float(M[(idx / D) * LD + idx % D]);
+}
+
+// ---- 4. states at the segment starts, in order.  One CTA per unit; dynamic shared memory:
+// 2 * D * (D + 1) floats.
+template <int D>
+__global__ void __launch_bounds__(256) seqpar_combine_kernel(const SeqParParams p) {
+  extern __shared__ __align__(16) unsigned char seqpar_smem[];
+  constexpr int LD = D + 1, R = D / 16;
+  float* Sc = reinterpret_cast<float*>(seqpar_smem);   // current S_start
+  float* Pj = Sc + D * LD;
+  const int unit = blockIdx.x, tid = threadIdx.x;
+  const int ty = tid >> 4, tx = tid & 15;
+  const size_t N = size_t(p.units) * p.P;
+  for (int idx = tid; idx < D * D; idx += 256)
+    Sc[(idx / D) * LD + idx % D] = p.S0 ? p.S0[size_t(unit) * D * D + idx] : 0.0f;
+  __syncthreads();
+  for (int j = 0; j < p.P; ++j) {
+    const size_t vu = size_t(unit) * p.P + j;
+    const float* G = p.ST2 + vu * D * D;
+    const float* Pg = p.ST2 + (N + vu) * D * D;
+    float* Ss = p.Sstart + vu * D * D;
+    for (int idx = tid; idx < D * D; idx += 256) {
+      Ss[idx] = Sc[(idx / D) * LD + idx % D];
+      Pj[(idx / D) * LD + idx % D] = Pg[idx];
+    }
+    __syncthreads();
+    float acc[R][R];
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+      for (int b = 0; b < R; ++b) acc[a][b] = G[(ty * R + a) * D + tx * R + b];
+    for (int m = 0; m < D; ++m) {
+      float sa[R], pb[R];
+#pragma unroll
+      for (int a = 0; a < R; ++a) { sa[a] = Sc[(ty * R + a) * LD + m]; pb[a] = Pj[m * LD + tx * R + a]; }
+#pragma unroll
+      for (int a = 0; a < R; ++a)
+#pragma unroll
+        for (int b = 0; b < R; ++b) acc[a][b] = fmaf(sa[a], pb[b], acc[a][b]);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+      for (int b = 0; b < R; ++b) Sc[(ty * R + a) * LD + tx * R + b] = acc[a][b];
+    __syncthreads();
+  }
+  if (p.S_T)
+    for (int idx = tid; idx < D * D; idx += 256)
+      p.S_T[size_t(unit) * D * D + idx] = Sc[(idx / D) * LD + idx % D];
+}
+
+// ---- 5. o_t = o0_t + S_start_j w_t.  Grid (units * P, Ls / 64); dynamic shared memory:
+// D * (D + 1) + 64 * D floats.
+template <int D>
+__global__ void __launch_bounds__(256) seqpar_correct_kernel(const SeqParParams p) {
+  extern __shared__ __align__(16) unsigned char seqpar_smem[];
+  constexpr int LD = D + 1, TBK = 64;
+  constexpr int RW = D >= 64 ? 4 : 2;          // rows per thread
+  constexpr int TRW = D / RW;                  // threads along the rows
+  constexpr int TTK = 256 / TRW;               // threads along the tokens
+  constexpr int TT = TBK / TTK;                // tokens per thread
+  float* Ss = reinterpret_cast<float*>(seqpar_smem);   // [D][LD]
+  float* Wb = Ss + D * LD;                              // [TBK][D]
+  const int vu = blockIdx.x, j = vu % p.P;
+  if (j == 0 && !p.S0) return;                 // S_start = 0: nothing to add
+  const int Ls = p.T / p.P;
+  const int t0 = blockIdx.y * TBK;
+  const int nt = min(TBK, Ls - t0);
+  const int tid = threadIdx.x;
+  const float* Sg = p.Sstart + size_t(vu) * D * D;
+  for (int idx = tid; idx < D * D; idx += 256) Ss[(idx / D) * LD + idx % D] = Sg[idx];
+  const float* wg = p.wn + (size_t(vu) * Ls + t0) * D;
+  for (int idx = tid; idx < TBK * D; idx += 256) Wb[idx] = (idx / D < nt) ? wg[idx] : 0.0f;
+  __syncthreads();
+  const int tr = tid % TRW, tk = tid / TRW;
+  float acc[TT][RW];
+#pragma unroll
+  for (int a = 0; a < TT; ++a)
+#pragma unroll
+    for (int b = 0; b < RW; ++b) acc[a][b] = 0.0f;
+  for (int m = 0; m < D; ++m) {
+    float sv[RW], wv[TT];
+#pragma unroll
+    for (int b = 0; b < RW; ++b) sv[b] = Ss[(tr * RW + b) * LD + m];
+#pragma unroll
+    for (int a = 0; a < TT; ++a) wv[a] = Wb[(tk * TT + a) * D + m];
+#pragma unroll
+    for (int a = 0; a < TT; ++a)
+#pragma unroll
+      for (int b = 0; b < RW; ++b) acc[a][b] = fmaf(wv[a], sv[b], acc[a][b]);
+  }
+  float* og = p.out + (size_t(vu) * Ls + t0) * D;
+#pragma unroll
+  for (int a = 0; a < TT; ++a) {
+    const int t = tk * TT + a;
+    if (t < nt) {
+#pragma unroll
+      for (int b = 0; b < RW; ++b) og[size_t(t) * D + tr * RW + b] += acc[a][b];
+    }
+  }
+}
+
+}  // namespace vla

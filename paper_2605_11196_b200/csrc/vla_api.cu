@@ -216,8 +216,8 @@ SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
   SeqParLayout L;
   size_t off = 0;
   auto take = [&](size_t bytes) { const size_t at = off; off += round256(bytes); return at; };
-  L.Gd = take(N * D * D * sizeof(double));
-  L.zsum = take(N * D * sizeof(float));
+  L.Gd = take(N * vla::kGramSplit * D * D * sizeof(double));
+  L.zsum = take(N * vla::kGramSplit * D * sizeof(float));
   L.Astart = take(N * D * D * sizeof(float));
   L.zstart = take(N * D * sizeof(float));
   L.ST2 = take(2 * N * D * D * sizeof(float));
@@ -283,7 +283,7 @@ int launch_seqpar(const vla::SeqParParams& sp, const ScanParams& scan, int dtype
   const int Ls = sp.T / sp.P;
   const size_t inv_smem = (size_t(D) * (D + 1) + 2 * D) * sizeof(double);
   const size_t comb_smem = 2 * size_t(D) * (D + 1) * sizeof(float);
-  const size_t corr_smem = (size_t(D) * (D + 1) + 64 * size_t(D)) * sizeof(float);
+  const size_t corr_smem = (size_t(D) + 64) * (D + 4) * sizeof(float);
   if (cudaFuncSetAttribute(vla::seqpar_invert_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(inv_smem)) != cudaSuccess ||
       cudaFuncSetAttribute(vla::seqpar_combine_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -293,8 +293,8 @@ int launch_seqpar(const vla::SeqParParams& sp, const ScanParams& scan, int dtype
     cudaGetLastError();
     return VLA_ERR_CUDA;
   }
-  if (dtype == VLA_F32) vla::seqpar_gram_kernel<D, float><<<N, 256, 0, st>>>(sp);
-  else vla::seqpar_gram_kernel<D, uint16_t><<<N, 256, 0, st>>>(sp);
+  if (dtype == VLA_F32) vla::seqpar_gram_kernel<D, float><<<dim3(N, vla::kGramSplit), 256, 0, st>>>(sp);
+  else vla::seqpar_gram_kernel<D, uint16_t><<<dim3(N, vla::kGramSplit), 256, 0, st>>>(sp);
   vla::seqpar_invert_kernel<D><<<N, 256, inv_smem, st>>>(sp);
   if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
   const int rc = launch_chunk_d<D>(scan, dtype, st);

@@ -33,8 +33,8 @@ struct SeqParParams {
   const float* z0;      // [units, D] or nullptr
   float* out;           // [units, T, D] o0 on entry of `correct`, o on exit
   float* S_T;           // [units, D, D] or nullptr
-  double* Gd;           // [N, D, D]   segment Gram matrices (N = units * P)
-  float* zsum;          // [N, D]      segment sums of phi(k)
+  double* Gd;           // [N, kGramSplit, D, D]  partial Gram matrices (N = units * P)
+  float* zsum;          // [N, kGramSplit, D]     partial sums of phi(k)
   float* Astart;        // [N, D, D]
   float* zstart;        // [N, D]
   const float* ST2;     // [2N, D, D]  G_j, then P_j
@@ -59,21 +59,31 @@ __device__ __forceinline__ float load1<uint16_t>(const uint16_t* p, size_t i) {
   return __uint_as_float(uint32_t(p[i]) << 16);
 }
 
-// ---- 1. segment Gram matrix and key sum.  One CTA of 256 threads per (unit, segment); the
-// last segment of a unit needs neither and is skipped.  Thread (ty, tx) of a 16 x 16 grid
-// owns an R x R block of the D x D result, R = D / 16.
+// ---- 1. Gram matrix and key sum of one slice of a segment.  Grid (units * P, kGramSplit): a
+// segment's tokens are divided among kGramSplit CTAs of 256 threads, whose partial results
+// the inversion kernel adds up; the last segment of a unit needs neither and is skipped.
+// Input rows: 8 lanes per token, 32 tokens per block, every load of a block in flight at once.
+// Thread (ty, tx) of a 16 x 16 grid owns an R x R block of the D x D result, R = D / 16.
+constexpr int kGramSplit = 4;
+
 template <int D, typename TIn>
 __global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) {
   constexpr int R = D / 16;
   constexpr int TB = 32;          // tokens per shared-memory block (one fp32 partial sum)
-  constexpr int EPL = D / 32;     // elements per lane of a token row
-  __shared__ __align__(16) float U[TB][D + 4];
-  __shared__ float zpart[8][D];
+  constexpr int EPL = D / 8;      // elements per lane of a token row (8 lanes per token)
+  constexpr int LDU = D + 4;
+  __shared__ __align__(16) float U[TB][LDU];
+  __shared__ float zpart[TB][D];
   const int vu = blockIdx.x, unit = vu / p.P, j = vu % p.P;
   if (j == p.P - 1) return;
   const int Ls = p.T / p.P;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // this CTA's tokens of the segment: [tlo, thi), whole 32-token blocks except at the end
+  const int nblk = (Ls + TB - 1) / TB;
+  const int tlo = int((long long)nblk * blockIdx.y / kGramSplit) * TB;
+  const int thi = min(Ls, int((long long)nblk * (blockIdx.y + 1) / kGramSplit) * TB);
+  const int tid = threadIdx.x;
   const int ty = tid >> 4, tx = tid & 15;
+  const int tok = tid >> 3, pl = tid & 7;      // input stage: token of the block, lane of the token
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
   const TIn* kk = static_cast<const TIn*>(p.k) + (size_t(unit) * p.T + size_t(j) * Ls) * D;
   const TIn* uu = p.u ? static_cast<const TIn*>(p.u) + (size_t(unit) * p.T + size_t(j) * Ls) * D : nullptr;
@@ -87,31 +97,36 @@ __global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) 
 #pragma unroll
   for (int e = 0; e < EPL; ++e) zs[e] = 0.0f;
 
-  for (int t0 = 0; t0 < Ls; t0 += TB) {
+  for (int t0 = tlo; t0 < thi; t0 += TB) {
     // rows u_t of this block: k_hat = phi(k)/||phi(k)|| (or k/||k||), or the given u verbatim
-    for (int tt = warp; tt < TB; tt += 8) {
-      const int t = t0 + tt;
+    {
+      const int t = t0 + tok;
+      const bool act = t < thi;
       float x[EPL];
       float ss = 0.0f;
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        float kf = 0.0f;
-        if (t < Ls) {
-          kf = load1<TIn>(kk, size_t(t) * D + e * 32 + lane);
-          if (!ident) kf = seqpar_phi(kf);
+      for (int f = 0; f < EPL / 4; ++f) {
+        float4 k4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (act) k4 = load4(kk + size_t(t) * D, f * 8 + pl);
+        if (act && !ident) {
+          k4.x = seqpar_phi(k4.x); k4.y = seqpar_phi(k4.y);
+          k4.z = seqpar_phi(k4.z); k4.w = seqpar_phi(k4.w);
         }
-        x[e] = kf;
-        zs[e] += kf;
-        ss = fmaf(kf, kf, ss);
+        x[4 * f + 0] = k4.x; x[4 * f + 1] = k4.y; x[4 * f + 2] = k4.z; x[4 * f + 3] = k4.w;
       }
 #pragma unroll
-      for (int off = 16; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+      for (int e = 0; e < EPL; ++e) {
+        zs[e] += x[e];
+        ss = fmaf(x[e], x[e], ss);
+      }
+#pragma unroll
+      for (int off = 4; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
       const float inv = 1.0f / fmaxf(sqrtf(ss), p.eps);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        float v = x[e] * inv;
-        if (uu) v = (t < Ls) ? load1<TIn>(uu, size_t(t) * D + e * 32 + lane) : 0.0f;
-        U[tt][e * 32 + lane] = v;
+      for (int f = 0; f < EPL / 4; ++f) {
+        float4 v4 = make_float4(x[4 * f] * inv, x[4 * f + 1] * inv, x[4 * f + 2] * inv, x[4 * f + 3] * inv);
+        if (uu) v4 = act ? load4(uu + size_t(t) * D, f * 8 + pl) : make_float4(0.f, 0.f, 0.f, 0.f);
+        *reinterpret_cast<float4*>(&U[tok][(f * 8 + pl) * 4]) = v4;
       }
     }
     __syncthreads();
@@ -136,19 +151,20 @@ __global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) 
       for (int b = 0; b < R; ++b) accd[a][b] += double(acc[a][b]);
     __syncthreads();
   }
-  double* G = p.Gd + size_t(vu) * D * D;
+  double* G = p.Gd + (size_t(vu) * kGramSplit + blockIdx.y) * D * D;
 #pragma unroll
   for (int a = 0; a < R; ++a)
 #pragma unroll
     for (int b = 0; b < R; ++b) G[(ty * R + a) * D + tx * R + b] = accd[a][b];
+  // key sum: this thread's columns are (f * 8 + pl) * 4 + i; add over the 32 token slots
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) zpart[warp][e * 32 + lane] = zs[e];
+  for (int e = 0; e < EPL; ++e) zpart[tok][((e / 4) * 8 + pl) * 4 + (e & 3)] = zs[e];
   __syncthreads();
   for (int c = tid; c < D; c += 256) {
     float s = 0.0f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) s += zpart[w][c];
-    p.zsum[size_t(vu) * D + c] = s;
+    for (int w = 0; w < TB; ++w) s += zpart[w][c];
+    p.zsum[(size_t(vu) * kGramSplit + blockIdx.y) * D + c] = s;
   }
 }
 
@@ -168,7 +184,8 @@ __global__ void __launch_bounds__(256) seqpar_invert_kernel(const SeqParParams p
     double s = p.z0 ? double(p.z0[size_t(unit) * D + c]) : 0.0;
     // the identity-map reading has no readout normaliser: the key sum is carried through
     if (!(p.flags & VLA_FLAG_IDENTITY_MAP))
-      for (int i = 0; i < j; ++i) s += double(p.zsum[(size_t(unit) * p.P + i) * D + c]);
+      for (int i = 0; i < j * kGramSplit; ++i)
+        s += double(p.zsum[(size_t(unit) * p.P * kGramSplit + i) * D + c]);
     p.zstart[size_t(vu) * D + c] = float(s);
   }
   if (j == 0) {
@@ -179,7 +196,8 @@ __global__ void __launch_bounds__(256) seqpar_invert_kernel(const SeqParParams p
   for (int idx = tid; idx < D * D; idx += 256) {
     const int r = idx / D, c = idx % D;
     double s = (r == c) ? double(p.lambda) : 0.0;
-    for (int i = 0; i < j; ++i) s += p.Gd[(size_t(unit) * p.P + i) * D * D + idx];
+    for (int i = 0; i < j * kGramSplit; ++i)
+      s += p.Gd[(size_t(unit) * p.P * kGramSplit + i) * D * D + idx];
     M[r * LD + c] = s;
   }
   __syncthreads();
@@ -255,27 +273,32 @@ __global__ void __launch_bounds__(256) seqpar_combine_kernel(const SeqParParams 
 }
 
 // ---- 5. o_t = o0_t + S_start_j w_t.  Grid (units * P, Ls / 64); dynamic shared memory:
-// D * (D + 1) + 64 * D floats.
+// D * (D + 4) + 64 * (D + 4) floats.
 template <int D>
 __global__ void __launch_bounds__(256) seqpar_correct_kernel(const SeqParParams p) {
   extern __shared__ __align__(16) unsigned char seqpar_smem[];
-  constexpr int LD = D + 1, TBK = 64;
-  constexpr int RW = D >= 64 ? 4 : 2;          // rows per thread
+  constexpr int LD = D + 4, TBK = 64;
+  constexpr int RW = D >= 64 ? 4 : 2;          // rows per thread: tr, tr + TRW, ...
   constexpr int TRW = D / RW;                  // threads along the rows
   constexpr int TTK = 256 / TRW;               // threads along the tokens
   constexpr int TT = TBK / TTK;                // tokens per thread
   float* Ss = reinterpret_cast<float*>(seqpar_smem);   // [D][LD]
-  float* Wb = Ss + D * LD;                              // [TBK][D]
+  float* Wb = Ss + D * LD;                              // [TBK][LD]
   const int vu = blockIdx.x, j = vu % p.P;
   if (j == 0 && !p.S0) return;                 // S_start = 0: nothing to add
   const int Ls = p.T / p.P;
   const int t0 = blockIdx.y * TBK;
   const int nt = min(TBK, Ls - t0);
   const int tid = threadIdx.x;
-  const float* Sg = p.Sstart + size_t(vu) * D * D;
-  for (int idx = tid; idx < D * D; idx += 256) Ss[(idx / D) * LD + idx % D] = Sg[idx];
-  const float* wg = p.wn + (size_t(vu) * Ls + t0) * D;
-  for (int idx = tid; idx < TBK * D; idx += 256) Wb[idx] = (idx / D < nt) ? wg[idx] : 0.0f;
+  const float4* Sg = reinterpret_cast<const float4*>(p.Sstart + size_t(vu) * D * D);
+  for (int idx = tid; idx < D * D / 4; idx += 256)
+    *reinterpret_cast<float4*>(&Ss[(idx / (D / 4)) * LD + (idx % (D / 4)) * 4]) = Sg[idx];
+  const float4* wg = reinterpret_cast<const float4*>(p.wn + (size_t(vu) * Ls + t0) * D);
+  for (int idx = tid; idx < TBK * D / 4; idx += 256) {
+    const int t = idx / (D / 4);
+    *reinterpret_cast<float4*>(&Wb[t * LD + (idx % (D / 4)) * 4]) =
+        t < nt ? wg[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   __syncthreads();
   const int tr = tid % TRW, tk = tid / TRW;
   float acc[TT][RW];
@@ -283,16 +306,22 @@ __global__ void __launch_bounds__(256) seqpar_correct_kernel(const SeqParParams 
   for (int a = 0; a < TT; ++a)
 #pragma unroll
     for (int b = 0; b < RW; ++b) acc[a][b] = 0.0f;
-  for (int m = 0; m < D; ++m) {
-    float sv[RW], wv[TT];
+#pragma unroll 2
+  for (int m = 0; m < D; m += 4) {
+    float4 sv[RW], wv[TT];
 #pragma unroll
-    for (int b = 0; b < RW; ++b) sv[b] = Ss[(tr * RW + b) * LD + m];
+    for (int b = 0; b < RW; ++b) sv[b] = *reinterpret_cast<const float4*>(&Ss[(tr + b * TRW) * LD + m]);
 #pragma unroll
-    for (int a = 0; a < TT; ++a) wv[a] = Wb[(tk * TT + a) * D + m];
+    for (int a = 0; a < TT; ++a) wv[a] = *reinterpret_cast<const float4*>(&Wb[(tk * TT + a) * LD + m]);
 #pragma unroll
     for (int a = 0; a < TT; ++a)
 #pragma unroll
-      for (int b = 0; b < RW; ++b) acc[a][b] = fmaf(wv[a], sv[b], acc[a][b]);
+      for (int b = 0; b < RW; ++b) {
+        acc[a][b] = fmaf(wv[a].x, sv[b].x, acc[a][b]);
+        acc[a][b] = fmaf(wv[a].y, sv[b].y, acc[a][b]);
+        acc[a][b] = fmaf(wv[a].z, sv[b].z, acc[a][b]);
+        acc[a][b] = fmaf(wv[a].w, sv[b].w, acc[a][b]);
+      }
   }
   float* og = p.out + (size_t(vu) * Ls + t0) * D;
 #pragma unroll
@@ -300,7 +329,7 @@ __global__ void __launch_bounds__(256) seqpar_correct_kernel(const SeqParParams 
     const int t = tk * TT + a;
     if (t < nt) {
 #pragma unroll
-      for (int b = 0; b < RW; ++b) og[size_t(t) * D + tr * RW + b] += acc[a][b];
+      for (int b = 0; b < RW; ++b) og[size_t(t) * D + tr + b * TRW] += acc[a][b];
     }
   }
 }

@@ -119,6 +119,35 @@ int launch_chunk(const ScanParams& p, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
+// Three warp groups per CTA (sequence-parallel launches at d <= 64): one CTA per segment runs
+// the segment and its transfer scan on one pass of group A.  p.units CTAs, p.n_main == p.units.
+template <int D, typename TIn, int UM>
+int launch_chunk_tri(const ScanParams& p, cudaStream_t st) {
+  using Cfg = vla::ChunkCfg<D, TIn, UM, true>;
+  static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
+  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, UM, true>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  vla::SchedParams sp;
+  sp.balanced = 0;
+  sp.grid = p.units;
+  sp.epoch = 0;
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D>
+int launch_chunk_tri_d(const ScanParams& p, int dtype, cudaStream_t st) {
+  if (p.u)
+    return dtype == VLA_F32 ? launch_chunk_tri<D, float, vla::kUTensor>(p, st)
+                            : launch_chunk_tri<D, uint16_t, vla::kUTensor>(p, st);
+  return dtype == VLA_F32 ? launch_chunk_tri<D, float, vla::kUKhat>(p, st)
+                          : launch_chunk_tri<D, uint16_t, vla::kUKhat>(p, st);
+}
+
 template <int D>
 int launch_chunk_d(const ScanParams& p, int dtype, cudaStream_t st) {
   if (p.u)
@@ -229,27 +258,19 @@ SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
   return L;
 }
 
-// CTAs of the chunk kernel that one device holds at a time (u = k_hat variant).
-template <int D>
-int chunk_resident_ctas(int dtype) {
+// CTAs of the chunk kernel that one device holds at a time (u = k_hat variant; TRI: the
+// three-group kernel of the sequence-parallel path).
+template <int D, typename TIn, bool TRI>
+int chunk_resident_ctas_t() {
+  using Cfg = vla::ChunkCfg<D, TIn, vla::kUKhat, TRI>;
+  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, vla::kUKhat, TRI>;
   int dev = 0, sms = 0, per_sm = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (e == cudaSuccess) {
-    if (dtype == VLA_F32) {
-      using Cfg = vla::ChunkCfg<D, float, vla::kUKhat>;
-      auto kern = vla::vla_scan_chunk_kernel<D, float, false, vla::kUKhat>;
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes));
-      if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes);
-    } else {
-      using Cfg = vla::ChunkCfg<D, uint16_t, vla::kUKhat>;
-      auto kern = vla::vla_scan_chunk_kernel<D, uint16_t, false, vla::kUKhat>;
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes));
-      if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes);
-    }
-  }
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes));
+  if (e == cudaSuccess)
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return 0;
@@ -257,18 +278,23 @@ int chunk_resident_ctas(int dtype) {
   return sms * per_sm;
 }
 
+// The sequence-parallel path runs a segment and its transfer scan in one three-group CTA at
+// d <= 64, and as two CTAs at d = 128 (where two states fill the register file).
+constexpr bool seqpar_tri(int d) { return d <= 64; }
+
 // Segments per unit: as many as fill the device with 2 * units * P scans, P a divisor of the
 // number of 16-token chunks, at least 256 tokens per segment.  1 = not worth cutting.
 int seqpar_choose_segments(int units, int T, int d, int dtype) {
   if (units <= 0 || T <= 0 || T % 16 != 0 || d < 32) return 1;
   int resident = 0;
+  const bool f32 = dtype == VLA_F32;
   switch (d) {
-    case 32: resident = chunk_resident_ctas<32>(dtype); break;
-    case 64: resident = chunk_resident_ctas<64>(dtype); break;
-    case 128: resident = chunk_resident_ctas<128>(dtype); break;
+    case 32: resident = f32 ? chunk_resident_ctas_t<32, float, true>() : chunk_resident_ctas_t<32, uint16_t, true>(); break;
+    case 64: resident = f32 ? chunk_resident_ctas_t<64, float, true>() : chunk_resident_ctas_t<64, uint16_t, true>(); break;
+    case 128: resident = f32 ? chunk_resident_ctas_t<128, float, false>() : chunk_resident_ctas_t<128, uint16_t, false>(); break;
     default: return 1;
   }
-  const int target = resident / (2 * units);
+  const int target = resident / ((seqpar_tri(d) ? 1 : 2) * units);
   const int nch = T / 16;
   int best = 1;
   for (int P = 2; P <= target && P <= nch; ++P)
@@ -297,7 +323,9 @@ int launch_seqpar(const vla::SeqParParams& sp, const ScanParams& scan, int dtype
   else vla::seqpar_gram_kernel<D, uint16_t><<<dim3(N, vla::kGramSplit), 256, 0, st>>>(sp);
   vla::seqpar_invert_kernel<D><<<N, 256, inv_smem, st>>>(sp);
   if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
-  const int rc = launch_chunk_d<D>(scan, dtype, st);
+  int rc;
+  if constexpr (seqpar_tri(D)) rc = launch_chunk_tri_d<D>(scan, dtype, st);
+  else rc = launch_chunk_d<D>(scan, dtype, st);
   if (rc != VLA_OK) return rc;
   vla::seqpar_combine_kernel<D><<<sp.units, 256, comb_smem, st>>>(sp);
   vla::seqpar_correct_kernel<D><<<dim3(N, (Ls + 63) / 64), 256, corr_smem, st>>>(sp);
@@ -576,7 +604,8 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   p.S_T = reinterpret_cast<float*>(w + L.ST2); p.A_T = AT2; p.zT = zT2;
   p.status = o.status;
   p.lambda = lambda_; p.eps = o.eps;
-  p.T = T / P; p.units = 2 * N; p.n_main = N; p.flags = o.flags;
+  // d <= 64: N CTAs of three warp groups; d = 128: 2N CTAs, the transfer scans second
+  p.T = T / P; p.units = seqpar_tri(d_k) ? N : 2 * N; p.n_main = N; p.flags = o.flags;
   p.refresh_period = 0; p.refresh_eta = 0.0f; p.step_offset = 0; p.u_is_khat = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   switch (d_k) {

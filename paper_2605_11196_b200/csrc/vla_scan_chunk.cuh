@@ -95,7 +95,7 @@ struct ChunkTile {
 //             which A_t k_hat_t is no longer parallel to z_t; one product with A per chunk
 enum : int { kUKhat = 0, kUTensor = 1, kUKhatGen = 2 };
 
-template <int D, typename TIn, int UM = kUKhat>
+template <int D, typename TIn, int UM = kUKhat, bool TRI = false>
 struct ChunkCfg {
   static constexpr bool GEN = UM != kUKhat;      // general path
   static constexpr bool UT = UM == kUTensor;     // a fourth input tensor
@@ -105,7 +105,8 @@ struct ChunkCfg {
   static constexpr int LPR = D / TW;             // lanes that share a row block (== TR)
   static constexpr int NV = TW / 4;              // float4 operand groups per thread
   static constexpr int NG = D;                   // threads per warp group
-  static constexpr int NT = 2 * D;               // threads per CTA
+  static constexpr int NGROUPS = TRI ? 3 : 2;    // A, S [, transfer scan]
+  static constexpr int NT = NGROUPS * D;         // threads per CTA
   static constexpr int NWG = D / 32;             // warps per group
   static constexpr int NIN = UT ? 4 : 3;         // q, k, v[, u]
   // raw q/k/v[/u] chunks in flight (fewer on the general path: shared memory is the limit)
@@ -129,7 +130,7 @@ struct ChunkCfg {
   static constexpr size_t s_floats = size_t(3) * C * D + 2 * C * D + ((GEN || S_HT) ? 2 * C * CP : 0);
   //   VS(B), R0s, Eps | ostage[2] [| GuL, HTL]
   static constexpr size_t smem_bytes = raw_bytes +
-      (KRING * kslot_floats + RING * slot_floats + a_floats + s_floats) * sizeof(float) +
+      (KRING * kslot_floats + RING * slot_floats + a_floats + (NGROUPS - 1) * s_floats) * sizeof(float) +
       (NSTAGE + 2 * RING) * sizeof(uint64_t) + 16 + 128;
 };
 
@@ -362,10 +363,14 @@ __device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) 
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-template <int D, typename TIn, bool BALANCED, int UM>
-__global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanParams p,
-                                                                  const SchedParams sp) {
-  using Cfg = ChunkCfg<D, TIn, UM>;
+// TRI: a third warp group runs the segment's transfer scan (S from I, v = 0; sequence-parallel
+// launches at d <= 64) next to group S, on the same products of group A.  Its readout goes to
+// out2 and its final state to S_T[n_main + unit].
+template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false>
+__global__ void __launch_bounds__((TRI ? 3 : 2) * D, 1) vla_scan_chunk_kernel(const ScanParams p,
+                                                                              const SchedParams sp) {
+  using Cfg = ChunkCfg<D, TIn, UM, TRI>;
+  static_assert(!TRI || (D <= 64 && !BALANCED), "three groups: d <= 64, one CTA per unit");
   constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly
   constexpr bool UT = Cfg::UT;       // u comes from the caller's tensor
   constexpr int NIN = Cfg::NIN;
@@ -396,7 +401,8 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   float* idl = dlt + C;                            // [C]  1/delta
   float* nidl = idl + C;                           // [C] -1/delta
   float* nrs = nidl + C;                           // [C+1] eta * (refreshes before token t of the chunk)
-  float* sbase = abase + Cfg::a_floats;
+  const int grp = threadIdx.x / Cfg::NG;   // 0: A, 1: S, 2: transfer scan (TRI)
+  float* sbase = abase + Cfg::a_floats + (grp == 2 ? Cfg::s_floats : 0);
   float* VS = sbase;                // [C][D]  B = V^T - S K^T
   float* R0s = VS + C * D;          // [C][D]
   float* Eps = R0s + C * D;         // [C][D]
@@ -404,7 +410,8 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   float* GuL = ostage + 2 * C * D;  // [C][CP] GuL[t][s] = k_hat_t . a_s   (general path)
   float* HTL = GuL + C * CP;        // [C][CP] HTL[t][s] = q_t . a_s       (general path)
   uint64_t* bars = reinterpret_cast<uint64_t*>(
-      (reinterpret_cast<uintptr_t>(sbase + Cfg::s_floats) + 15) & ~uintptr_t(15));
+      (reinterpret_cast<uintptr_t>(abase + Cfg::a_floats + (Cfg::NGROUPS - 1) * Cfg::s_floats) + 15) &
+      ~uintptr_t(15));
   uint64_t* full = bars;                    // [NSTAGE] raw stage filled by TMA
   uint64_t* ring_full = full + NSTAGE;      // [RING] group A published chunk c
   uint64_t* ring_empty = ring_full + RING;  // [RING] group S is done with chunk c
@@ -412,7 +419,8 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 
   const int tid = threadIdx.x;
   const bool is_A = tid < NG;
-  const int g = is_A ? tid : tid - NG;   // thread within its group; also the row it owns
+  const int g = tid - grp * NG;          // thread within its group; also the row it owns
+  const int sbar = 1 + grp;              // named barrier of this S-like group
   const int lane = g & 31, gw = g >> 5;
   const int cg = g % LPR;                // column group
   const int rb = g / LPR;                // row block: rows rb*TR .. rb*TR+TR-1
@@ -446,8 +454,11 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
   for (int pi = 0; get_piece<BALANCED>(sp, p.units, nch_unit, blockIdx.x, pi, pc); ++pi) {
   const int unit = pc.unit;
   // transfer scan of a sequence-parallel launch: inputs of unit `uin`, v = 0, S0 = I
-  const bool pscan = p.n_main > 0 && unit >= p.n_main;
-  const int uin = pscan ? unit - p.n_main : unit;
+  // TRI: the third group is the transfer scan of this very unit; otherwise transfer scans are
+  // the CTAs of units >= n_main
+  const bool pscan_cta = !TRI && p.n_main > 0 && unit >= p.n_main;
+  const bool pscan = TRI ? (grp == 2) : pscan_cta;
+  const int uin = pscan_cta ? unit - p.n_main : unit;
   const int t_begin = pc.cb * C;
   const int T = min(p.T, pc.ce * C) - t_begin;   // tokens of this piece
   const int nchunks = pc.ce - pc.cb;
@@ -464,10 +475,10 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     const int n = min(C, T - c * C);
     const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
     TIn* dst = raw + size_t(s) * NIN * C * D;
-    mbar_arrive_expect_tx(&full[s], (pscan ? NIN - 1 : NIN) * bytes);
+    mbar_arrive_expect_tx(&full[s], (pscan_cta ? NIN - 1 : NIN) * bytes);
     bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &full[s]);
     bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &full[s]);
-    if (!pscan) bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
+    if (!pscan_cta) bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
     if (UT) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
   };
 
@@ -484,7 +495,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&ring_empty[r])) : "memory");
       }
       mbar_init(&ring_full[r], 1);
-      mbar_init(&ring_empty[r], 1);
+      mbar_init(&ring_empty[r], Cfg::NGROUPS - 1);
     }
     mbar_init_fence();
     if (from_handoff && !*abort_flag) {
@@ -509,7 +520,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
     // a tail piece continues from the state its head left in the caller's output buffers
     // (written by another SM: read past L1)
     const float* src = from_handoff ? (is_A ? p.A_T : p.S_T) : (is_A ? p.A0 : (pscan ? nullptr : p.S0));
-    const int usrc = from_handoff ? unit : uin;   // a transfer scan reads the A0 of its partner
+    const int usrc = from_handoff ? unit : uin;   // a transfer-scan CTA reads the A0 of its partner
 #pragma unroll
     for (int r = 0; r < TR; ++r) {
       const int row = rb * TR + r;
@@ -567,7 +578,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           if (act) {
             kf[i] = load4(rk + tt * D, f);
             qf = load4(rq + tt * D, f);
-            if (!pscan) vv = load4(rv + tt * D, f);
+            if (!pscan_cta) vv = load4(rv + tt * D, f);
             if (!ident) {
               kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
               kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
@@ -897,7 +908,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 
       // ---- B = V^T - S K^T and R0 = S Q^T, row g of each
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) {
-        VS[t * D + g] = Vf[t * D + g] - x;
+        VS[t * D + g] = (TRI && pscan ? 0.0f : Vf[t * D + g]) - x;
       });
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
       if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
@@ -908,12 +919,12 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
       if (HAS_U) {
         gram16<D, NG, CP>(Kh, Zs, GuL, g);
         gram16<D, NG, CP>(Qf, Zs, HTL, g);
-        group_bar(2, NG);
+        group_bar(sbar, NG);
         Gm = GuL;
         Hm = HTL;
       } else if (Cfg::S_HT) {
         gram16<D, NG, CP>(Qf, Zs, HTL, g);
-        group_bar(2, NG);
+        group_bar(sbar, NG);
         Hm = HTL;
       }
       VLA_MARK(2)
@@ -954,14 +965,14 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
           o[t] = a0 + a1;
         }
       }
-      group_bar(2, NG);  // bulk_wait_read above is ordered before the stage is rewritten
+      group_bar(sbar, NG);  // bulk_wait_read above is ordered before the stage is rewritten
       {
         float* ost = ostage + size_t(c & 1) * C * D;
 #pragma unroll
         for (int t = 0; t < 16; ++t) ost[t * D + g] = o[t] * inv_den[t];
       }
       fence_async_smem();
-      group_bar(2, NG);  // Eps and the out stage complete
+      group_bar(sbar, NG);  // Eps and the out stage complete
       if (g == 0) {
         const size_t tok = size_t(uin) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
         bulk_store((pscan ? p.out2 : p.out) + tok * D, ostage + size_t(c & 1) * C * D,
@@ -972,7 +983,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
 
       // ---- S <- S + E' Z^T
       tile_rank_update<TR, TW, LPR, D, C>(st, Eps, Zs, nullptr, rb, cg);
-      group_bar(2, NG);
+      group_bar(sbar, NG);
       if (g == 0) mbar_arrive(&ring_empty[slot]);
       VLA_MARK(4)
     }
@@ -983,7 +994,7 @@ __global__ void __launch_bounds__(2 * D, 1) vla_scan_chunk_kernel(const ScanPara
         const int row = rb * TR + r;
 #pragma unroll
         for (int m = 0; m < NV; ++m)
-          reinterpret_cast<float4*>(p.S_T + (size_t(unit) * D + row) * D)[m * LPR + cg] =
+          reinterpret_cast<float4*>(p.S_T + (size_t(TRI && pscan ? unit + p.n_main : unit) * D + row) * D)[m * LPR + cg] =
               make_float4(st[r][2 * m].x, st[r][2 * m].y, st[r][2 * m + 1].x, st[r][2 * m + 1].y);
       }
     }

@@ -8,10 +8,7 @@
 #include <mutex>
 
 #include "vla.h"
-#include "vla_common.cuh"
-#include "vla_scan_token.cuh"
-#include "vla_scan_chunk.cuh"
-#include "vla_seqpar.cuh"
+#include "vla_launch.h"
 
 namespace {
 
@@ -43,123 +40,9 @@ bool shape_supported(int d_k, int d_v) {
   return d_k == d_v && (d_k == 16 || d_k == 32 || d_k == 64 || d_k == 128);
 }
 
-template <int D, typename TIn, bool HAS_U>
-int launch_token(const ScanParams& p, cudaStream_t st) {
-  using Cfg = vla::TokenCfg<D, TIn, HAS_U>;
-  auto kern = vla::vla_scan_token_kernel<D, TIn, HAS_U>;
-  // Idempotent; needed once per device and cheap enough to repeat (no global state kept).
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(Cfg::smem_bytes)) != cudaSuccess) {
-    cudaGetLastError();
-    return VLA_ERR_CUDA;
-  }
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
-  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
-}
-
-template <int D>
-int launch_token_d(const ScanParams& p_in, int dtype, cudaStream_t st) {
-  // The periodic refresh lives in the two-exchange variant (the write direction is no longer
-  // parallel to z on a refresh step); without an explicit u that variant is told to use k_hat.
-  ScanParams p = p_in;
-  if (p.refresh_period > 0 && p.u == nullptr) {
-    p.u = p.k;   // a valid address for the ring's fourth tensor; its contents are not used
-    p.u_is_khat = 1;
-  }
-  const bool has_u = p.u != nullptr;
-  if (dtype == VLA_F32)
-    return has_u ? launch_token<D, float, true>(p, st) : launch_token<D, float, false>(p, st);
-  return has_u ? launch_token<D, uint16_t, true>(p, st) : launch_token<D, uint16_t, false>(p, st);
-}
-
 // Launch ids for the balanced schedule's hand-off flags (a flag equal to the launch's id
 // means "done"; ids never repeat within 2^32 launches, so the flags never need clearing).
 std::atomic<unsigned int> g_launch_epoch{0};
-
-template <int D, typename TIn, int UM>
-int launch_chunk(const ScanParams& p, cudaStream_t st) {
-  using Cfg = vla::ChunkCfg<D, TIn, UM>;
-  static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
-  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, UM>;     // one CTA per unit
-  auto kern_bal = vla::vla_scan_chunk_kernel<D, TIn, true, UM>;  // persistent grid, units cut at chunks
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(Cfg::smem_bytes)) != cudaSuccess ||
-      cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(Cfg::smem_bytes)) != cudaSuccess) {
-    cudaGetLastError();
-    return VLA_ERR_CUDA;
-  }
-  vla::SchedParams sp;
-  sp.balanced = 0;
-  sp.grid = p.units;
-  sp.epoch = 0;
-  // Balanced schedule: only when a plain launch would leave SMs idle in its last wave, every
-  // CTA of the persistent grid is resident at once, and the caller's S_T / A_T / zT can carry
-  // a unit's state from the CTA that starts it to the CTA that finishes it.
-  int dev = 0, sms = 0, per_sm = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess &&
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern_bal, Cfg::NT, Cfg::smem_bytes) ==
-          cudaSuccess) {
-    const int resident = sms * per_sm;
-    const bool state_out = p.S_T && p.A_T && (p.zT || (p.flags & VLA_FLAG_IDENTITY_MAP));
-    if (resident > 0 && p.units > resident && p.units % resident != 0 && p.T > 0 && state_out &&
-        p.units <= vla::kSchedMaxUnits) {
-      sp.balanced = 1;
-      sp.grid = resident;
-      unsigned int e = ++g_launch_epoch;
-      if (e == 0) e = ++g_launch_epoch;   // 0 is the flags' initial value
-      sp.epoch = e;
-    }
-  } else {
-    cudaGetLastError();
-  }
-  if (sp.balanced) kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
-  else kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
-  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
-}
-
-// Three warp groups per CTA (sequence-parallel launches at d <= 64): one CTA per segment runs
-// the segment and its transfer scan on one pass of group A.  p.units CTAs, p.n_main == p.units.
-template <int D, typename TIn, int UM>
-int launch_chunk_tri(const ScanParams& p, cudaStream_t st) {
-  using Cfg = vla::ChunkCfg<D, TIn, UM, true>;
-  static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
-  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, UM, true>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(Cfg::smem_bytes)) != cudaSuccess) {
-    cudaGetLastError();
-    return VLA_ERR_CUDA;
-  }
-  vla::SchedParams sp;
-  sp.balanced = 0;
-  sp.grid = p.units;
-  sp.epoch = 0;
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
-  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
-}
-
-template <int D>
-int launch_chunk_tri_d(const ScanParams& p, int dtype, cudaStream_t st) {
-  if (p.u)
-    return dtype == VLA_F32 ? launch_chunk_tri<D, float, vla::kUTensor>(p, st)
-                            : launch_chunk_tri<D, uint16_t, vla::kUTensor>(p, st);
-  return dtype == VLA_F32 ? launch_chunk_tri<D, float, vla::kUKhat>(p, st)
-                          : launch_chunk_tri<D, uint16_t, vla::kUKhat>(p, st);
-}
-
-template <int D>
-int launch_chunk_d(const ScanParams& p, int dtype, cudaStream_t st) {
-  if (p.u)
-    return dtype == VLA_F32 ? launch_chunk<D, float, vla::kUTensor>(p, st)
-                            : launch_chunk<D, uint16_t, vla::kUTensor>(p, st);
-  // The periodic refresh makes A_t k_hat_t leave the direction of z_t: general path, u = k_hat.
-  if (p.refresh_period > 0)
-    return dtype == VLA_F32 ? launch_chunk<D, float, vla::kUKhatGen>(p, st)
-                            : launch_chunk<D, uint16_t, vla::kUKhatGen>(p, st);
-  return dtype == VLA_F32 ? launch_chunk<D, float, vla::kUKhat>(p, st)
-                          : launch_chunk<D, uint16_t, vla::kUKhat>(p, st);
-}
 
 // The chunk kernel covers d in {32, 64, 128}; d = 16 runs on the token kernel.  Both are CUDA
 // paths; there is no host fallback.
@@ -175,21 +58,8 @@ int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
   if (kernel == VLA_KERNEL_CHUNK && !chunk) return VLA_ERR_UNSUPPORTED;
   if (kernel == VLA_KERNEL_AUTO && !chunk_pays_off(p, d)) chunk = false;
   if (kernel == VLA_KERNEL_TOKEN) chunk = false;
-  if (chunk) {
-    switch (d) {
-      case 32: return launch_chunk_d<32>(p, dtype, st);
-      case 64: return launch_chunk_d<64>(p, dtype, st);
-      case 128: return launch_chunk_d<128>(p, dtype, st);
-      default: return VLA_ERR_UNSUPPORTED;
-    }
-  }
-  switch (d) {
-    case 16: return launch_token_d<16>(p, dtype, st);
-    case 32: return launch_token_d<32>(p, dtype, st);
-    case 64: return launch_token_d<64>(p, dtype, st);
-    case 128: return launch_token_d<128>(p, dtype, st);
-    default: return VLA_ERR_UNSUPPORTED;
-  }
+  if (chunk) return vla::launch_chunk(d, dtype, p, st);
+  return vla::launch_token(d, dtype, p, st);
 }
 
 // Argument checks shared by the device- and host-pointer entry points.
@@ -258,26 +128,6 @@ SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
   return L;
 }
 
-// CTAs of the chunk kernel that one device holds at a time (u = k_hat variant; TRI: the
-// three-group kernel of the sequence-parallel path).
-template <int D, typename TIn, bool TRI>
-int chunk_resident_ctas_t() {
-  using Cfg = vla::ChunkCfg<D, TIn, vla::kUKhat, TRI>;
-  auto kern = vla::vla_scan_chunk_kernel<D, TIn, false, vla::kUKhat, TRI>;
-  int dev = 0, sms = 0, per_sm = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes));
-  if (e == cudaSuccess)
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes);
-  if (e != cudaSuccess) {
-    cudaGetLastError();
-    return 0;
-  }
-  return sms * per_sm;
-}
-
 // The sequence-parallel path runs a segment and its transfer scan in one three-group CTA at
 // d <= 64, and as two CTAs at d = 128 (where two states fill the register file).
 constexpr bool seqpar_tri(int d) { return d <= 64; }
@@ -286,14 +136,7 @@ constexpr bool seqpar_tri(int d) { return d <= 64; }
 // number of 16-token chunks, at least 256 tokens per segment.  1 = not worth cutting.
 int seqpar_choose_segments(int units, int T, int d, int dtype) {
   if (units <= 0 || T <= 0 || T % 16 != 0 || d < 32) return 1;
-  int resident = 0;
-  const bool f32 = dtype == VLA_F32;
-  switch (d) {
-    case 32: resident = f32 ? chunk_resident_ctas_t<32, float, true>() : chunk_resident_ctas_t<32, uint16_t, true>(); break;
-    case 64: resident = f32 ? chunk_resident_ctas_t<64, float, true>() : chunk_resident_ctas_t<64, uint16_t, true>(); break;
-    case 128: resident = f32 ? chunk_resident_ctas_t<128, float, false>() : chunk_resident_ctas_t<128, uint16_t, false>(); break;
-    default: return 1;
-  }
+  const int resident = vla::chunk_resident_ctas(d, dtype, seqpar_tri(d));
   const int target = resident / ((seqpar_tri(d) ? 1 : 2) * units);
   const int nch = T / 16;
   int best = 1;
@@ -302,47 +145,15 @@ int seqpar_choose_segments(int units, int T, int d, int dtype) {
   return best;
 }
 
-template <int D>
-int launch_seqpar(const vla::SeqParParams& sp, const ScanParams& scan, int dtype, float* A_T,
-                  float* zT, const float* AT2, const float* zT2, cudaStream_t st) {
-  const int N = sp.units * sp.P;
-  const int Ls = sp.T / sp.P;
-  const size_t inv_smem = (size_t(D) * (D + 1) + 2 * D) * sizeof(double);
-  const size_t comb_smem = 2 * size_t(D) * (D + 1) * sizeof(float);
-  const size_t corr_smem = (size_t(D) + 64) * (D + 4) * sizeof(float);
-  if (cudaFuncSetAttribute(vla::seqpar_invert_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(inv_smem)) != cudaSuccess ||
-      cudaFuncSetAttribute(vla::seqpar_combine_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(comb_smem)) != cudaSuccess ||
-      cudaFuncSetAttribute(vla::seqpar_correct_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(corr_smem)) != cudaSuccess) {
-    cudaGetLastError();
-    return VLA_ERR_CUDA;
-  }
-  if (dtype == VLA_F32) vla::seqpar_gram_kernel<D, float><<<dim3(N, vla::kGramSplit), 256, 0, st>>>(sp);
-  else vla::seqpar_gram_kernel<D, uint16_t><<<dim3(N, vla::kGramSplit), 256, 0, st>>>(sp);
-  vla::seqpar_invert_kernel<D><<<N, 256, inv_smem, st>>>(sp);
-  if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
-  int rc;
-  if constexpr (seqpar_tri(D)) rc = launch_chunk_tri_d<D>(scan, dtype, st);
-  else rc = launch_chunk_d<D>(scan, dtype, st);
-  if (rc != VLA_OK) return rc;
-  vla::seqpar_combine_kernel<D><<<sp.units, 256, comb_smem, st>>>(sp);
-  vla::seqpar_correct_kernel<D><<<dim3(N, (Ls + 63) / 64), 256, corr_smem, st>>>(sp);
-  if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
-  // final A and key sum: those of each unit's last segment
-  const size_t P = size_t(sp.P);
-  if (A_T &&
-      cudaMemcpy2DAsync(A_T, size_t(D) * D * 4, AT2 + (P - 1) * D * D, P * D * D * 4, size_t(D) * D * 4,
-                        size_t(sp.units), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-    return VLA_ERR_CUDA;
-  if (zT && cudaMemcpy2DAsync(zT, size_t(D) * 4, zT2 + (P - 1) * D, P * D * 4, size_t(D) * 4,
-                              size_t(sp.units), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-    return VLA_ERR_CUDA;
-  return VLA_OK;
-}
-
 }  // namespace
+
+namespace vla {
+unsigned int next_launch_epoch() {
+  unsigned int e = ++g_launch_epoch;
+  if (e == 0) e = ++g_launch_epoch;   // 0 is the flags' initial value
+  return e;
+}
+}  // namespace vla
 
 extern "C" {
 
@@ -608,12 +419,12 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   p.T = T / P; p.units = seqpar_tri(d_k) ? N : 2 * N; p.n_main = N; p.flags = o.flags;
   p.refresh_period = 0; p.refresh_eta = 0.0f; p.step_offset = 0; p.u_is_khat = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  switch (d_k) {
-    case 32: return launch_seqpar<32>(sp, p, o.qkv_dtype, A_T, o.zT, AT2, zT2, st);
-    case 64: return launch_seqpar<64>(sp, p, o.qkv_dtype, A_T, o.zT, AT2, zT2, st);
-    case 128: return launch_seqpar<128>(sp, p, o.qkv_dtype, A_T, o.zT, AT2, zT2, st);
-    default: return VLA_ERR_UNSUPPORTED;
-  }
+  rc = vla::seqpar_before_scan(d_k, o.qkv_dtype, sp, st);
+  if (rc != VLA_OK) return rc;
+  rc = seqpar_tri(d_k) ? vla::launch_chunk_tri(d_k, o.qkv_dtype, p, st)
+                       : vla::launch_chunk(d_k, o.qkv_dtype, p, st);
+  if (rc != VLA_OK) return rc;
+  return vla::seqpar_after_scan(d_k, sp, A_T, o.zT, AT2, zT2, st);
 }
 
 int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags) {

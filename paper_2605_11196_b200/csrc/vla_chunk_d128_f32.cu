@@ -1,0 +1,4 @@
+// Chunk kernel, d = 128, fp32 inputs.
+#include "vla_chunk_launch.cuh"
+
+VLA_DEFINE_CHUNK_TU(128, float, d128_f32)

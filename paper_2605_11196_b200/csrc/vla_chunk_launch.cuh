@@ -1,0 +1,127 @@
+// Launchers of the chunk kernel for one (d, input type).  Each vla_chunk_d*_*.cu instantiates
+// them once through VLA_DEFINE_CHUNK_TU.
+#pragma once
+
+#include "vla.h"
+#include "vla_launch.h"
+#include "vla_scan_chunk.cuh"
+
+namespace vla {
+
+template <int D, typename TIn, int UM>
+int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
+  using Cfg = ChunkCfg<D, TIn, UM>;
+  static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM>;     // one CTA per unit
+  auto kern_bal = vla_scan_chunk_kernel<D, TIn, true, UM>;  // persistent grid, units cut at chunks
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess ||
+      cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  SchedParams sp;
+  sp.balanced = 0;
+  sp.grid = p.units;
+  sp.epoch = 0;
+  // Balanced schedule: only when a plain launch would leave SMs idle in its last wave, every
+  // CTA of the persistent grid is resident at once, and the caller's S_T / A_T / zT can carry
+  // a unit's state from the CTA that starts it to the CTA that finishes it.
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern_bal, Cfg::NT, Cfg::smem_bytes) ==
+          cudaSuccess) {
+    const int resident = sms * per_sm;
+    const bool state_out = p.S_T && p.A_T && (p.zT || (p.flags & VLA_FLAG_IDENTITY_MAP));
+    if (resident > 0 && p.units > resident && p.units % resident != 0 && p.T > 0 && state_out &&
+        p.units <= kSchedMaxUnits && p.n_main <= 0) {
+      sp.balanced = 1;
+      sp.grid = resident;
+      sp.epoch = next_launch_epoch();
+    }
+  } else {
+    cudaGetLastError();
+  }
+  if (sp.balanced) kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  else kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D, typename TIn>
+int launch_chunk_t(const ScanParams& p, cudaStream_t st) {
+  if (p.u) return launch_chunk_um<D, TIn, kUTensor>(p, st);
+  // The periodic refresh makes A_t k_hat_t leave the direction of z_t: general path, u = k_hat.
+  if (p.refresh_period > 0) return launch_chunk_um<D, TIn, kUKhatGen>(p, st);
+  return launch_chunk_um<D, TIn, kUKhat>(p, st);
+}
+
+// Three warp groups per CTA (sequence-parallel launches at d <= 64): one CTA per segment runs
+// the segment and its transfer scan on one pass of group A.  p.units CTAs, p.n_main == p.units.
+template <int D, typename TIn, int UM>
+int launch_chunk_tri_um(const ScanParams& p, cudaStream_t st) {
+  using Cfg = ChunkCfg<D, TIn, UM, true>;
+  static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, true>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  SchedParams sp;
+  sp.balanced = 0;
+  sp.grid = p.units;
+  sp.epoch = 0;
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D, typename TIn>
+int launch_chunk_tri_t(const ScanParams& p, cudaStream_t st) {
+  if constexpr (D <= 64) {
+    if (p.refresh_period > 0) return VLA_ERR_UNSUPPORTED;
+    if (p.u) return launch_chunk_tri_um<D, TIn, kUTensor>(p, st);
+    return launch_chunk_tri_um<D, TIn, kUKhat>(p, st);
+  } else {
+    return VLA_ERR_UNSUPPORTED;
+  }
+}
+
+template <int D, typename TIn, bool TRI>
+int chunk_resident_ctas_t() {
+  using Cfg = ChunkCfg<D, TIn, kUKhat, TRI>;
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, kUKhat, TRI>;
+  int dev = 0, sms = 0, per_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes));
+  if (e == cudaSuccess)
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return sms * per_sm;
+}
+
+template <int D, typename TIn>
+int chunk_resident_t(bool tri) {
+  if constexpr (D <= 64) {
+    if (tri) return chunk_resident_ctas_t<D, TIn, true>();
+  }
+  return chunk_resident_ctas_t<D, TIn, false>();
+}
+
+}  // namespace vla
+
+// The three entry points of one (d, input type) translation unit.
+#define VLA_DEFINE_CHUNK_TU(D, TIN, TAG)                                                        \
+  namespace vla {                                                                               \
+  int launch_chunk_##TAG(const ScanParams& p, cudaStream_t st) { return launch_chunk_t<D, TIN>(p, st); } \
+  int launch_chunk_tri_##TAG(const ScanParams& p, cudaStream_t st) {                            \
+    return launch_chunk_tri_t<D, TIN>(p, st);                                                   \
+  }                                                                                             \
+  int chunk_resident_##TAG(bool tri) { return chunk_resident_t<D, TIN>(tri); }                  \
+  }

@@ -1,0 +1,160 @@
+// Dispatch from (d, input type) to the translation unit that holds the kernels, the token
+// kernel's launchers, and the helper launches of the sequence-parallel path.
+#include "vla.h"
+#include "vla_launch.h"
+#include "vla_scan_token.cuh"
+#include "vla_seqpar.cuh"
+
+namespace vla {
+
+#define VLA_DECLARE_CHUNK_TU(TAG)                                   \
+  int launch_chunk_##TAG(const ScanParams& p, cudaStream_t st);     \
+  int launch_chunk_tri_##TAG(const ScanParams& p, cudaStream_t st); \
+  int chunk_resident_##TAG(bool tri);
+VLA_DECLARE_CHUNK_TU(d32_f32)
+VLA_DECLARE_CHUNK_TU(d32_bf16)
+VLA_DECLARE_CHUNK_TU(d64_f32)
+VLA_DECLARE_CHUNK_TU(d64_bf16)
+VLA_DECLARE_CHUNK_TU(d128_f32)
+VLA_DECLARE_CHUNK_TU(d128_bf16)
+#undef VLA_DECLARE_CHUNK_TU
+
+#define VLA_CHUNK_DISPATCH(FN, ...)                                                         \
+  do {                                                                                      \
+    const bool f32 = dtype == VLA_F32;                                                      \
+    switch (d) {                                                                            \
+      case 32: return f32 ? FN##_d32_f32(__VA_ARGS__) : FN##_d32_bf16(__VA_ARGS__);         \
+      case 64: return f32 ? FN##_d64_f32(__VA_ARGS__) : FN##_d64_bf16(__VA_ARGS__);         \
+      case 128: return f32 ? FN##_d128_f32(__VA_ARGS__) : FN##_d128_bf16(__VA_ARGS__);      \
+      default: break;                                                                       \
+    }                                                                                       \
+  } while (0)
+
+int launch_chunk(int d, int dtype, const ScanParams& p, cudaStream_t st) {
+  VLA_CHUNK_DISPATCH(launch_chunk, p, st);
+  return VLA_ERR_UNSUPPORTED;
+}
+
+int launch_chunk_tri(int d, int dtype, const ScanParams& p, cudaStream_t st) {
+  VLA_CHUNK_DISPATCH(launch_chunk_tri, p, st);
+  return VLA_ERR_UNSUPPORTED;
+}
+
+int chunk_resident_ctas(int d, int dtype, bool tri) {
+  VLA_CHUNK_DISPATCH(chunk_resident, tri);
+  return 0;
+}
+
+// ---------------------------------------------------------------- token kernel
+namespace {
+
+template <int D, typename TIn, bool HAS_U>
+int launch_token_t(const ScanParams& p, cudaStream_t st) {
+  using Cfg = TokenCfg<D, TIn, HAS_U>;
+  auto kern = vla_scan_token_kernel<D, TIn, HAS_U>;
+  // Idempotent; needed once per device and cheap enough to repeat (no global state kept).
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D>
+int launch_token_d(const ScanParams& p_in, int dtype, cudaStream_t st) {
+  // The periodic refresh lives in the two-exchange variant (the write direction is no longer
+  // parallel to z on a refresh step); without an explicit u that variant is told to use k_hat.
+  ScanParams p = p_in;
+  if (p.refresh_period > 0 && p.u == nullptr) {
+    p.u = p.k;   // a valid address for the ring's fourth tensor; its contents are not used
+    p.u_is_khat = 1;
+  }
+  const bool has_u = p.u != nullptr;
+  if (dtype == VLA_F32)
+    return has_u ? launch_token_t<D, float, true>(p, st) : launch_token_t<D, float, false>(p, st);
+  return has_u ? launch_token_t<D, uint16_t, true>(p, st) : launch_token_t<D, uint16_t, false>(p, st);
+}
+
+}  // namespace
+
+int launch_token(int d, int dtype, const ScanParams& p, cudaStream_t st) {
+  switch (d) {
+    case 16: return launch_token_d<16>(p, dtype, st);
+    case 32: return launch_token_d<32>(p, dtype, st);
+    case 64: return launch_token_d<64>(p, dtype, st);
+    case 128: return launch_token_d<128>(p, dtype, st);
+    default: return VLA_ERR_UNSUPPORTED;
+  }
+}
+
+// ---------------------------------------------------------------- sequence-parallel helpers
+namespace {
+
+template <int D>
+int seqpar_before_d(int dtype, const SeqParParams& sp, cudaStream_t st) {
+  const int N = sp.units * sp.P;
+  const size_t inv_smem = (size_t(D) * (D + 1) + 2 * D) * sizeof(double);
+  if (cudaFuncSetAttribute(seqpar_invert_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(inv_smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  if (dtype == VLA_F32) seqpar_gram_kernel<D, float><<<dim3(N, kGramSplit), 256, 0, st>>>(sp);
+  else seqpar_gram_kernel<D, uint16_t><<<dim3(N, kGramSplit), 256, 0, st>>>(sp);
+  seqpar_invert_kernel<D><<<N, 256, inv_smem, st>>>(sp);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D>
+int seqpar_after_d(const SeqParParams& sp, float* A_T, float* zT, const float* AT2, const float* zT2,
+                   cudaStream_t st) {
+  const int N = sp.units * sp.P;
+  const int Ls = sp.T / sp.P;
+  const size_t comb_smem = 2 * size_t(D) * (D + 1) * sizeof(float);
+  const size_t corr_smem = (size_t(D) + 64) * (D + 4) * sizeof(float);
+  if (cudaFuncSetAttribute(seqpar_combine_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(comb_smem)) != cudaSuccess ||
+      cudaFuncSetAttribute(seqpar_correct_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(corr_smem)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  seqpar_combine_kernel<D><<<sp.units, 256, comb_smem, st>>>(sp);
+  seqpar_correct_kernel<D><<<dim3(N, (Ls + 63) / 64), 256, corr_smem, st>>>(sp);
+  if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
+  // final A and key sum: those of each unit's last segment
+  const size_t P = size_t(sp.P);
+  if (A_T &&
+      cudaMemcpy2DAsync(A_T, size_t(D) * D * 4, AT2 + (P - 1) * D * D, P * D * D * 4, size_t(D) * D * 4,
+                        size_t(sp.units), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return VLA_ERR_CUDA;
+  if (zT && cudaMemcpy2DAsync(zT, size_t(D) * 4, zT2 + (P - 1) * D, P * D * 4, size_t(D) * 4,
+                              size_t(sp.units), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return VLA_ERR_CUDA;
+  return VLA_OK;
+}
+
+}  // namespace
+
+int seqpar_before_scan(int d, int dtype, const SeqParParams& sp, cudaStream_t st) {
+  switch (d) {
+    case 32: return seqpar_before_d<32>(dtype, sp, st);
+    case 64: return seqpar_before_d<64>(dtype, sp, st);
+    case 128: return seqpar_before_d<128>(dtype, sp, st);
+    default: return VLA_ERR_UNSUPPORTED;
+  }
+}
+
+int seqpar_after_scan(int d, const SeqParParams& sp, float* A_T, float* zT, const float* AT2,
+                      const float* zT2, cudaStream_t st) {
+  switch (d) {
+    case 32: return seqpar_after_d<32>(sp, A_T, zT, AT2, zT2, st);
+    case 64: return seqpar_after_d<64>(sp, A_T, zT, AT2, zT2, st);
+    case 128: return seqpar_after_d<128>(sp, A_T, zT, AT2, zT2, st);
+    default: return VLA_ERR_UNSUPPORTED;
+  }
+}
+
+}  // namespace vla

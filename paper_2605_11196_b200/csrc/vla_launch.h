@@ -1,0 +1,35 @@
+// Host-side interface between the C ABI (vla_api.cu) and the translation units that hold the
+// kernels.  The kernels are spread over several .cu files only so that they compile in
+// parallel; none of this is visible outside the library.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "vla_common.cuh"
+#include "vla_seqpar_params.h"
+
+namespace vla {
+
+// Token kernel, d in {16, 32, 64, 128}.  Returns a vla_status_t.
+int launch_token(int d, int dtype, const ScanParams& p, cudaStream_t st);
+
+// Chunk kernel, d in {32, 64, 128}: plain or balanced grid, chosen from the shape.
+int launch_chunk(int d, int dtype, const ScanParams& p, cudaStream_t st);
+
+// Chunk kernel with three warp groups per CTA (d in {32, 64}; sequence-parallel launches).
+int launch_chunk_tri(int d, int dtype, const ScanParams& p, cudaStream_t st);
+
+// CTAs of the chunk kernel (u = k_hat variant) that the current device holds at a time.
+int chunk_resident_ctas(int d, int dtype, bool tri);
+
+// Sequence-parallel helpers: Gram matrices + inversion before the scan, combination +
+// correction + final-state copies after it.
+int seqpar_before_scan(int d, int dtype, const SeqParParams& sp, cudaStream_t st);
+int seqpar_after_scan(int d, const SeqParParams& sp, float* A_T, float* zT, const float* AT2,
+                      const float* zT2, cudaStream_t st);
+
+// Launch ids for the balanced schedule's hand-off flags (never 0, never repeated within
+// 2^32 launches).
+unsigned int next_launch_epoch();
+
+}  // namespace vla

@@ -23,30 +23,10 @@
 #pragma once
 
 #include "vla_common.cuh"
+#include "vla_seqpar_params.h"
 
 namespace vla {
 
-struct SeqParParams {
-  const void* k;        // [units, T, D] raw keys
-  const void* u;        // [units, T, D] explicit penalty directions or nullptr
-  const float* S0;      // [units, D, D] or nullptr
-  const float* z0;      // [units, D] or nullptr
-  float* out;           // [units, T, D] o0 on entry of `correct`, o on exit
-  float* S_T;           // [units, D, D] or nullptr
-  double* Gd;           // [N, kGramSplit, D, D]  partial Gram matrices (N = units * P)
-  float* zsum;          // [N, kGramSplit, D]     partial sums of phi(k)
-  float* Astart;        // [N, D, D]
-  float* zstart;        // [N, D]
-  const float* ST2;     // [2N, D, D]  G_j, then P_j
-  const float* wn;      // [N, Ls, D]  transfer readouts
-  float* Sstart;        // [N, D, D]
-  float lambda;
-  float eps;
-  int T;                // tokens per unit
-  int P;                // segments per unit
-  int units;
-  uint32_t flags;
-};
 
 __device__ __forceinline__ float seqpar_phi(float x) { return x > 0.0f ? x + 1.0f : __expf(x); }
 
@@ -64,7 +44,6 @@ __device__ __forceinline__ float load1<uint16_t>(const uint16_t* p, size_t i) {
 // the inversion kernel adds up; the last segment of a unit needs neither and is skipped.
 // Input rows: 8 lanes per token, 32 tokens per block, every load of a block in flight at once.
 // Thread (ty, tx) of a 16 x 16 grid owns an R x R block of the D x D result, R = D / 16.
-constexpr int kGramSplit = 4;
 
 template <int D, typename TIn>
 __global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) {

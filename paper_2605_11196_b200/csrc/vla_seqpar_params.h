@@ -1,0 +1,34 @@
+// Arguments of the sequence-parallel helper kernels (see vla_seqpar.cuh).
+#pragma once
+
+#include <cstdint>
+
+namespace vla {
+
+// CTAs that share the Gram matrix of one segment (their partial results are added up by the
+// inversion kernel)
+constexpr int kGramSplit = 4;
+
+struct SeqParParams {
+  const void* k;        // [units, T, D] raw keys
+  const void* u;        // [units, T, D] explicit penalty directions or nullptr
+  const float* S0;      // [units, D, D] or nullptr
+  const float* z0;      // [units, D] or nullptr
+  float* out;           // [units, T, D] o0 on entry of `correct`, o on exit
+  float* S_T;           // [units, D, D] or nullptr
+  double* Gd;           // [N, kGramSplit, D, D]  partial Gram matrices (N = units * P)
+  float* zsum;          // [N, kGramSplit, D]     partial sums of phi(k)
+  float* Astart;        // [N, D, D]
+  float* zstart;        // [N, D]
+  const float* ST2;     // [2N, D, D]  G_j, then P_j
+  const float* wn;      // [N, Ls, D]  transfer readouts
+  float* Sstart;        // [N, D, D]
+  float lambda;
+  float eps;
+  int T;                // tokens per unit
+  int P;                // segments per unit
+  int units;
+  uint32_t flags;
+};
+
+}  // namespace vla

@@ -115,8 +115,8 @@ SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
   SeqParLayout L;
   size_t off = 0;
   auto take = [&](size_t bytes) { const size_t at = off; off += round256(bytes); return at; };
-  L.Gd = take(N * vla::kGramSplit * D * D * sizeof(double));
-  L.zsum = take(N * vla::kGramSplit * D * sizeof(float));
+  L.Gd = take(N * D * D * sizeof(double));
+  L.zsum = take(N * D * sizeof(float));
   L.Astart = take(N * D * D * sizeof(float));
   L.zstart = take(N * D * sizeof(float));
   L.ST2 = take(2 * N * D * D * sizeof(float));

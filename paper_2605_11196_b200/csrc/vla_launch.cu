@@ -95,15 +95,13 @@ namespace {
 template <int D>
 int seqpar_before_d(int dtype, const SeqParParams& sp, cudaStream_t st) {
   const int N = sp.units * sp.P;
-  const size_t inv_smem = (size_t(D) * (D + 1) + 2 * D) * sizeof(double);
-  if (cudaFuncSetAttribute(seqpar_invert_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(inv_smem)) != cudaSuccess) {
-    cudaGetLastError();
+  // the Gram kernel's CTAs add into these
+  if (cudaMemsetAsync(sp.Gd, 0, size_t(N) * D * D * sizeof(double), st) != cudaSuccess ||
+      cudaMemsetAsync(sp.zsum, 0, size_t(N) * D * sizeof(float), st) != cudaSuccess)
     return VLA_ERR_CUDA;
-  }
   if (dtype == VLA_F32) seqpar_gram_kernel<D, float><<<dim3(N, kGramSplit), 256, 0, st>>>(sp);
   else seqpar_gram_kernel<D, uint16_t><<<dim3(N, kGramSplit), 256, 0, st>>>(sp);
-  seqpar_invert_kernel<D><<<N, 256, inv_smem, st>>>(sp);
+  seqpar_invert_kernel<D><<<N, 256, 0, st>>>(sp);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

@@ -40,8 +40,8 @@ __device__ __forceinline__ float load1<uint16_t>(const uint16_t* p, size_t i) {
 }
 
 // ---- 1. Gram matrix and key sum of one slice of a segment.  Grid (units * P, kGramSplit): a
-// segment's tokens are divided among kGramSplit CTAs of 256 threads, whose partial results
-// the inversion kernel adds up; the last segment of a unit needs neither and is skipped.
+// segment's tokens are divided among kGramSplit CTAs of 256 threads, which add their results
+// into the segment's (zeroed) matrix; the last segment of a unit needs neither and is skipped.
 // Input rows: 8 lanes per token, 32 tokens per block, every load of a block in flight at once.
 // Thread (ty, tx) of a 16 x 16 grid owns an R x R block of the D x D result, R = D / 16.
 
@@ -130,11 +130,13 @@ __global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) 
       for (int b = 0; b < R; ++b) accd[a][b] += double(acc[a][b]);
     __syncthreads();
   }
-  double* G = p.Gd + (size_t(vu) * kGramSplit + blockIdx.y) * D * D;
+  // the kGramSplit CTAs of a segment add into one matrix (zeroed by the host before the
+  // launch): fp64 additions are scarce on this part, the inversion kernel should not repeat them
+  double* G = p.Gd + size_t(vu) * D * D;
 #pragma unroll
   for (int a = 0; a < R; ++a)
 #pragma unroll
-    for (int b = 0; b < R; ++b) G[(ty * R + a) * D + tx * R + b] = accd[a][b];
+    for (int b = 0; b < R; ++b) atomicAdd(&G[(ty * R + a) * D + tx * R + b], accd[a][b]);
   // key sum: this thread's columns are (f * 8 + pl) * 4 + i; add over the 32 token slots
 #pragma unroll
   for (int e = 0; e < EPL; ++e) zpart[tok][((e / 4) * 8 + pl) * 4 + (e & 3)] = zs[e];
@@ -143,62 +145,76 @@ __global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) 
     float s = 0.0f;
 #pragma unroll
     for (int w = 0; w < TB; ++w) s += zpart[w][c];
-    p.zsum[(size_t(vu) * kGramSplit + blockIdx.y) * D + c] = s;
+    atomicAdd(&p.zsum[size_t(vu) * D + c], s);
   }
 }
 
-// ---- 2. A at the start of segment j, and the running key sum there.  One CTA per
-// (unit, segment); dynamic shared memory: D * (D + 1) + 2 * D doubles.
+// ---- 2. A at the start of segment j, and the running key sum there.  One CTA of 256
+// threads per (unit, segment).  The matrix stays in registers: thread t owns D*D/256
+// consecutive elements of one row; a pivot step exchanges only the pivot row and column
+// through shared memory.
 template <int D>
 __global__ void __launch_bounds__(256) seqpar_invert_kernel(const SeqParParams p) {
-  extern __shared__ __align__(16) unsigned char seqpar_smem[];
-  double* M = reinterpret_cast<double*>(seqpar_smem);   // [D][D + 1]
-  double* colp = M + D * (D + 1);
-  double* rowp = colp + D;
-  constexpr int LD = D + 1;
+  constexpr int EC = D * D / 256;     // elements per thread
+  constexpr int TPR = D / EC;         // threads per row
+  __shared__ double rowraw[D];        // pivot row before scaling
+  __shared__ double colp[D];          // pivot column
   const int vu = blockIdx.x, unit = vu / p.P, j = vu % p.P;
   const int tid = threadIdx.x;
+  const int r = tid / TPR, c0 = (tid % TPR) * EC;
   float* A = p.Astart + size_t(vu) * D * D;
   for (int c = tid; c < D; c += 256) {
     double s = p.z0 ? double(p.z0[size_t(unit) * D + c]) : 0.0;
     // the identity-map reading has no readout normaliser: the key sum is carried through
     if (!(p.flags & VLA_FLAG_IDENTITY_MAP))
-      for (int i = 0; i < j * kGramSplit; ++i)
-        s += double(p.zsum[(size_t(unit) * p.P * kGramSplit + i) * D + c]);
+      for (int i = 0; i < j; ++i) s += double(p.zsum[(size_t(unit) * p.P + i) * D + c]);
     p.zstart[size_t(vu) * D + c] = float(s);
   }
   if (j == 0) {
     const float dg = 1.0f / p.lambda;
-    for (int idx = tid; idx < D * D; idx += 256) A[idx] = (idx / D == idx % D) ? dg : 0.0f;
+#pragma unroll
+    for (int e = 0; e < EC; ++e) A[r * D + c0 + e] = (c0 + e == r) ? dg : 0.0f;
     return;
   }
-  for (int idx = tid; idx < D * D; idx += 256) {
-    const int r = idx / D, c = idx % D;
-    double s = (r == c) ? double(p.lambda) : 0.0;
-    for (int i = 0; i < j * kGramSplit; ++i)
-      s += p.Gd[(size_t(unit) * p.P * kGramSplit + i) * D * D + idx];
-    M[r * LD + c] = s;
+  // M = lambda I + the Gram matrices of the earlier segments
+  double m[EC];
+#pragma unroll
+  for (int e = 0; e < EC; ++e) m[e] = (c0 + e == r) ? double(p.lambda) : 0.0;
+  for (int i = 0; i < j; ++i) {
+    const double* G = p.Gd + (size_t(unit) * p.P + i) * D * D + r * D + c0;
+#pragma unroll
+    for (int e = 0; e < EC; ++e) m[e] += G[e];
   }
-  __syncthreads();
-  // in-place Gauss-Jordan inversion
+  // in-place Gauss-Jordan inversion (no pivoting: symmetric positive definite)
+#pragma unroll 1
   for (int pv = 0; pv < D; ++pv) {
-    const double d = 1.0 / M[pv * LD + pv];
-    for (int c = tid; c < D; c += 256) {
-      colp[c] = M[c * LD + pv];
-      rowp[c] = M[pv * LD + c] * d;
+    if (r == pv) {
+#pragma unroll
+      for (int e = 0; e < EC; ++e) rowraw[c0 + e] = m[e];
+    }
+    if (pv >= c0 && pv < c0 + EC) {
+      double x = 0.0;
+#pragma unroll
+      for (int e = 0; e < EC; ++e)
+        if (c0 + e == pv) x = m[e];
+      colp[r] = x;
     }
     __syncthreads();
-    for (int idx = tid; idx < D * D; idx += 256) {
-      const int r = idx / D, c = idx % D;
-      double v;
-      if (r == pv) v = (c == pv) ? d : rowp[c];
-      else if (c == pv) v = -colp[r] * d;
-      else v = M[r * LD + c] - colp[r] * rowp[c];
-      M[r * LD + c] = v;
+    // fp64 arithmetic is scarce on this part: one FMA per element, the pivot's reciprocal
+    // folded into the column factor
+    const double d = 1.0 / rowraw[pv];
+    const double ncrd = -colp[r] * d;
+    if (r == pv) {
+#pragma unroll
+      for (int e = 0; e < EC; ++e) m[e] = (c0 + e == pv) ? d : rowraw[c0 + e] * d;
+    } else {
+#pragma unroll
+      for (int e = 0; e < EC; ++e) m[e] = (c0 + e == pv) ? ncrd : fma(ncrd, rowraw[c0 + e], m[e]);
     }
     __syncthreads();
   }
-  for (int idx = tid; idx < D * D; idx += 256) A[idx] = float(M[(idx / D) * LD + idx % D]);
+#pragma unroll
+  for (int e = 0; e < EC; ++e) A[r * D + c0 + e] = float(m[e]);
 }
 
 // ---- 4. states at the segment starts, in order.  One CTA per unit; dynamic shared memory:

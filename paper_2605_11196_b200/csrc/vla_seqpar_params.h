@@ -5,8 +5,7 @@
 
 namespace vla {
 
-// CTAs that share the Gram matrix of one segment (their partial results are added up by the
-// inversion kernel)
+// CTAs that share the Gram matrix of one segment (they add into it atomically)
 constexpr int kGramSplit = 4;
 
 struct SeqParParams {
@@ -16,8 +15,8 @@ struct SeqParParams {
   const float* z0;      // [units, D] or nullptr
   float* out;           // [units, T, D] o0 on entry of `correct`, o on exit
   float* S_T;           // [units, D, D] or nullptr
-  double* Gd;           // [N, kGramSplit, D, D]  partial Gram matrices (N = units * P)
-  float* zsum;          // [N, kGramSplit, D]     partial sums of phi(k)
+  double* Gd;           // [N, D, D]  segment Gram matrices, zero on entry (N = units * P)
+  float* zsum;          // [N, D]     segment sums of phi(k), zero on entry
   float* Astart;        // [N, D, D]
   float* zstart;        // [N, D]
   const float* ST2;     // [2N, D, D]  G_j, then P_j

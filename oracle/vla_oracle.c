@@ -24,7 +24,8 @@
  *                separately, the corrected associative (R, G) composition of
  *                Section 3.4, Proposition 1's norm identities.
  *   readout      S_t q_t from dumped states; denominator from a direct sum.
- *   state carry  split invariance.
+ *   state carry  split invariance; segments stitched through a transfer scan
+ *                (S_end = S_start P + G) with A at the cuts from matrix inverses.
  *   refresh      u = 0 closed form, step-by-step brute force with matrix inverses,
  *                split invariance with the carried step offset.
  * Absolute output values on random data are otherwise fixed by nothing the

@@ -2,8 +2,8 @@
  * vla_oracle.h -- CPU oracle for the Variational Linear Attention forward scan.
  *
  * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, fp64 restatement of the
- * paper's sequential forward pass (Algorithm 1 without the projections and
- * without the periodic refresh; Eqs. "sm", "s-update", "output" of Section 3.3).
+ * paper's sequential forward pass (Algorithm 1 without the projections, its
+ * periodic refresh optional; Eqs. "sm", "s-update", "output" of Section 3.3).
  * It shares no code with the CUDA library and the CUDA library never calls it.
  * Only the tests, the smoke check and the CPU-baseline leg of the benchmark
  * may load it.

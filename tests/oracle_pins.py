@@ -440,6 +440,39 @@ def pin_refresh_state_carry(orc):
     assert np.abs(wrong.A_T - full.A_T).max() > 1e-6      # offset matters
 
 
+def pin_segments_compose_through_a_transfer_scan(orc):
+    """The facts the sequence-parallel GPU path rests on, checked on the oracle alone.  Cut a
+    sequence in segments.  (i) A before a segment is the brute-force inverse of
+    lambda I + sum of u u^T over the earlier tokens (Eq. "penalty").  (ii) With that A and the
+    running key sum carried in, the segment scanned from S = 0 gives G and readouts o0_t; the
+    same segment with v = 0 from S = I gives P and w_t; then S_end = S_start P + G and
+    o_t = o0_t + S_start w_t (Section 3.4's composition with the map acting on the right)."""
+    dk, T, lam = 7, 48, 0.3
+    for flags in (0, IDENT):
+        for with_u in (False, True):
+            q, k, v, g = _rand(131 + flags, T, dk, dk)
+            u = _unit(g.standard_normal((T, dk))) / np.sqrt(dk) if with_u else None
+            S0 = 0.4 * g.standard_normal((dk, dk))
+            z0 = g.uniform(0.0, 1.0, dk)
+            full = orc.forward_trace(q, k, v, lam, u=u, S0=S0, z0=z0, flags=flags)
+            uu = u if with_u else _khat(k, flags)
+            kf = k if flags & IDENT else _phi(k)
+            S_start = S0
+            for a, b in ((0, 16), (16, 32), (32, 48)):
+                A_start = np.linalg.inv(lam * np.eye(dk) + uu[:a].T @ uu[:a])
+                z_start = z0 if flags & IDENT else z0 + kf[:a].sum(axis=0)
+                sl = lambda x: None if x is None else np.ascontiguousarray(x[a:b])
+                seg = orc.forward_trace(sl(q), sl(k), sl(v), lam, u=sl(u), A0=A_start, z0=z_start,
+                                        flags=flags)
+                tr = orc.forward_trace(sl(q), sl(k), np.zeros((b - a, dk)), lam, u=sl(u), S0=np.eye(dk),
+                                       A0=A_start, z0=z_start, flags=flags)
+                o = np.reshape(seg.out, (b - a, dk)) + np.reshape(tr.out, (b - a, dk)) @ S_start.T
+                assert np.abs(o - np.reshape(full.out, (T, dk))[a:b]).max() < 1e-9
+                S_start = S_start @ np.reshape(tr.S_T, (dk, dk)) + np.reshape(seg.S_T, (dk, dk))
+            assert np.abs(S_start - np.reshape(full.S_T, (dk, dk))).max() < 1e-9
+            assert np.abs(np.reshape(seg.A_T, (dk, dk)) - np.reshape(full.A_T, (dk, dk))).max() < 1e-9
+
+
 PINS = [pin_A_is_brute_force_inverse, pin_A_invariants, pin_delta_value,
         pin_alpha_from_post_update_A, pin_first_step_closed_form,
         pin_orthonormal_keys_exact_recall, pin_repeated_key,
@@ -447,4 +480,4 @@ PINS = [pin_A_is_brute_force_inverse, pin_A_invariants, pin_delta_value,
         pin_proposition_1, pin_readout, pin_feature_map_values, pin_eps_guards,
         pin_state_carry, pin_units_layout_threads_dtypes, pin_jacobian_spectrum,
         pin_refresh_closed_form_with_zero_u, pin_refresh_step_by_step_brute_force,
-        pin_refresh_state_carry]
+        pin_refresh_state_carry, pin_segments_compose_through_a_transfer_scan]

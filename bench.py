@@ -446,26 +446,29 @@ def main():
         A0 = torch.eye(wd.d, device=dev).expand(wd.B, wd.H, wd.d, wd.d).contiguous()
         bufs = dict(out=torch.empty((wd.B, wd.H, 1, wd.d), device=dev), S_T=torch.empty_like(S0),
                     A_T=torch.empty_like(A0), z_T=torch.empty((wd.B, wd.H, wd.d), device=dev), status=status)
-        dcall = lambda: vla.vla_forward(q2, k2, v2, wd.lam, S0=S0, A0=A0, stream=stream, **bufs)
         fl = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
-        evs = []
-        with torch.cuda.stream(stream):
-            for _ in range(3):
-                dcall()
-            for _ in range(10):
-                fl.fill_(1)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); dcall(); b.record(stream)
-                evs.append((a, b))
-        torch.cuda.synchronize(dev)
-        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
         state_bytes = wd.units * (4 * wd.d * wd.d * 4 + 2 * wd.d * 4)       # S, A read and written; z
         io_bytes = wd.units * (3 * wd.d * 2 + wd.d * 4)
-        per["decode"] = {"ms": ms, "units": wd.units, "steps_per_s": wd.units / (ms * 1e-3),
-                         "kernel": "vla_scan_token_kernel", "bound": "hbm",
-                         "hbm_gbs": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9,
-                         "hbm_frac": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9 / hbm_peak,
-                         "hbm_peak_source": peak_src}
+        for key, kern, kname in (("decode", vla.VLA_KERNEL_AUTO, "vla_decode_kernel"),
+                                 ("decode_token_kernel", vla.VLA_KERNEL_TOKEN, "vla_scan_token_kernel")):
+            dcall = lambda: vla.vla_forward(q2, k2, v2, wd.lam, S0=S0, A0=A0, stream=stream, kernel=kern,
+                                            **bufs)
+            evs = []
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    dcall()
+                for _ in range(10):
+                    fl.fill_(1)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream); dcall(); b.record(stream)
+                    evs.append((a, b))
+            torch.cuda.synchronize(dev)
+            ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+            per[key] = {"ms": ms, "units": wd.units, "steps_per_s": wd.units / (ms * 1e-3),
+                        "kernel": kname, "bound": "hbm",
+                        "hbm_gbs": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9,
+                        "hbm_frac": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9 / hbm_peak,
+                        "hbm_peak_source": peak_src}
         line["per_workload"] = per
 
     if not args.no_cpu_baseline:

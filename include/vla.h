@@ -54,8 +54,11 @@ enum {
 typedef enum {
   VLA_KERNEL_AUTO = 0,
   VLA_KERNEL_TOKEN = 1, /* one CTA per unit, one state pass per token; every shape, explicit u */
-  VLA_KERNEL_CHUNK = 2  /* 16 tokens per state pass (exact Woodbury form); d >= 32, every option;
+  VLA_KERNEL_CHUNK = 2, /* 16 tokens per state pass (exact Woodbury form); d >= 32, every option;
                            VLA_ERR_UNSUPPORTED for d = 16 */
+  VLA_KERNEL_DECODE = 3 /* one step (T = 1) with S0, A0, S_T, A_T all given, u = k_hat, no refresh,
+                           d >= 32: the states stream through shared memory once (HBM-bound);
+                           VLA_ERR_UNSUPPORTED otherwise.  AUTO picks it when it applies */
 } vla_kernel_t;
 
 typedef struct {

@@ -22,7 +22,7 @@ VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE, VLA_ERR_TOO_LARGE = -4,
 VLA_STATIC_SCRATCH_BYTES = 32 << 20
 VLA_F32, VLA_BF16 = 0, 1
 VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE = 1, 2
-VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK = 0, 1, 2
+VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK, VLA_KERNEL_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",
            "vla_forward_seqpar", "vla_seqpar_segments", "vla_seqpar_workspace_bytes",

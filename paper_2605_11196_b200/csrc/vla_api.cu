@@ -29,7 +29,8 @@ int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
   if (!(r->eps > 0.0f)) r->eps = 1e-4f;
   if (r->qkv_dtype != VLA_F32 && r->qkv_dtype != VLA_BF16) return VLA_ERR_INVALID_ARG;
   if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_INVALID_ARG;
-  if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN && r->kernel != VLA_KERNEL_CHUNK)
+  if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN && r->kernel != VLA_KERNEL_CHUNK &&
+      r->kernel != VLA_KERNEL_DECODE)
     return VLA_ERR_INVALID_ARG;
   if (r->refresh_period > 0 && (r->step_offset < 0 || !(r->refresh_eta == r->refresh_eta)))
     return VLA_ERR_INVALID_ARG;
@@ -53,7 +54,16 @@ bool chunk_covers(const ScanParams&, int d) { return d >= 32; }
 // padding (measured crossover: T ~ 12 at d = 128, T ~ 20 at d = 64).
 bool chunk_pays_off(const ScanParams& p, int d) { return p.T > (d >= 128 ? 8 : 16); }
 
+// The single-step kernel streams the states through shared memory once: T = 1, states carried
+// in and out, u = k_hat, no refresh.
+bool decode_covers(const ScanParams& p, int d) {
+  return p.T == 1 && d >= 32 && p.S0 && p.A0 && p.S_T && p.A_T && !p.u && p.refresh_period <= 0;
+}
+
 int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
+  if (kernel == VLA_KERNEL_DECODE && !decode_covers(p, d)) return VLA_ERR_UNSUPPORTED;
+  if ((kernel == VLA_KERNEL_DECODE || kernel == VLA_KERNEL_AUTO) && decode_covers(p, d))
+    return vla::launch_decode(d, dtype, p, st);
   bool chunk = chunk_covers(p, d);
   if (kernel == VLA_KERNEL_CHUNK && !chunk) return VLA_ERR_UNSUPPORTED;
   if (kernel == VLA_KERNEL_AUTO && !chunk_pays_off(p, d)) chunk = false;

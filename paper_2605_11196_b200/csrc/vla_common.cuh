@@ -131,6 +131,16 @@ __device__ __forceinline__ float bf16_bits_to_f32(uint32_t bits16) {
   return __uint_as_float(bits16 << 16);
 }
 
+// one element of a row of inputs, widened to fp32
+template <typename TIn>
+__device__ __forceinline__ float load1(const TIn* p, size_t i);
+template <>
+__device__ __forceinline__ float load1<float>(const float* p, size_t i) { return p[i]; }
+template <>
+__device__ __forceinline__ float load1<uint16_t>(const uint16_t* p, size_t i) {
+  return __uint_as_float(uint32_t(p[i]) << 16);
+}
+
 // four consecutive elements of a shared-memory row, widened to fp32
 __device__ __forceinline__ float4 load4(const float* row, int c4) {
   return reinterpret_cast<const float4*>(row)[c4];

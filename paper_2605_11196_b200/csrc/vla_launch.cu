@@ -2,6 +2,7 @@
 // kernel's launchers, and the helper launches of the sequence-parallel path.
 #include "vla.h"
 #include "vla_launch.h"
+#include "vla_decode.cuh"
 #include "vla_scan_token.cuh"
 #include "vla_seqpar.cuh"
 
@@ -85,6 +86,42 @@ int launch_token(int d, int dtype, const ScanParams& p, cudaStream_t st) {
     case 32: return launch_token_d<32>(p, dtype, st);
     case 64: return launch_token_d<64>(p, dtype, st);
     case 128: return launch_token_d<128>(p, dtype, st);
+    default: return VLA_ERR_UNSUPPORTED;
+  }
+}
+
+// ---------------------------------------------------------------- decode kernel
+namespace {
+
+template <int D, typename TIn>
+int launch_decode_t(const ScanParams& p, cudaStream_t st) {
+  using Cfg = DecodeCfg<D, TIn>;
+  static_assert(Cfg::smem_bytes <= 227 * 1024, "decode kernel exceeds the shared memory of one CTA");
+  auto kern = vla_decode_kernel<D, TIn>;
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess ||
+      cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, Cfg::NT, Cfg::smem_bytes) !=
+          cudaSuccess ||
+      per_sm < 1) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  const int grid = p.units < sms * per_sm ? p.units : sms * per_sm;   // persistent CTAs
+  kern<<<grid, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_decode(int d, int dtype, const ScanParams& p, cudaStream_t st) {
+  const bool f32 = dtype == VLA_F32;
+  switch (d) {
+    case 32: return f32 ? launch_decode_t<32, float>(p, st) : launch_decode_t<32, uint16_t>(p, st);
+    case 64: return f32 ? launch_decode_t<64, float>(p, st) : launch_decode_t<64, uint16_t>(p, st);
+    case 128: return f32 ? launch_decode_t<128, float>(p, st) : launch_decode_t<128, uint16_t>(p, st);
     default: return VLA_ERR_UNSUPPORTED;
   }
 }

@@ -13,6 +13,9 @@ namespace vla {
 // Token kernel, d in {16, 32, 64, 128}.  Returns a vla_status_t.
 int launch_token(int d, int dtype, const ScanParams& p, cudaStream_t st);
 
+// Single-step kernel (T = 1, carried states in and out, u = k_hat, no refresh), d in {32, 64, 128}.
+int launch_decode(int d, int dtype, const ScanParams& p, cudaStream_t st);
+
 // Chunk kernel, d in {32, 64, 128}: plain or balanced grid, chosen from the shape.
 int launch_chunk(int d, int dtype, const ScanParams& p, cudaStream_t st);
 

@@ -30,15 +30,6 @@ namespace vla {
 
 __device__ __forceinline__ float seqpar_phi(float x) { return x > 0.0f ? x + 1.0f : __expf(x); }
 
-template <typename TIn>
-__device__ __forceinline__ float load1(const TIn* p, size_t i);
-template <>
-__device__ __forceinline__ float load1<float>(const float* p, size_t i) { return p[i]; }
-template <>
-__device__ __forceinline__ float load1<uint16_t>(const uint16_t* p, size_t i) {
-  return __uint_as_float(uint32_t(p[i]) << 16);
-}
-
 // ---- 1. Gram matrix and key sum of one slice of a segment.  Grid (units * P, kGramSplit): a
 // segment's tokens are divided among kGramSplit CTAs of 256 threads, which add their results
 // into the segment's (zeroed) matrix; the last segment of a unit needs neither and is skipped.

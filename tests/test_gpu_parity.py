@@ -307,3 +307,59 @@ def test_workload_throughput_sampled_units(flags):
         for n, (b, h) in enumerate(units):
             e = rel_err(got[b, h], want[0, n])
             assert e <= w.tol, "unit (%d,%d) %s rel err %.3e" % (b, h, name, e)
+
+
+# ---------------------------------------------------------------- single-step kernel
+def _spd(shape, g, d):
+    h = torch.randn(shape + (d, d), generator=g) * 0.05
+    return h @ h.transpose(-1, -2) + 0.5 * torch.eye(d)
+
+
+@pytest.mark.parametrize("d,units", [(32, (3, 5)), (64, (2, 331)), (128, (7, 29)), (128, (1, 1))])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_single_step_kernel(d, units, dtype, flags):
+    """T = 1 with carried states: the kernel that streams S and A through shared memory, with
+    fewer and more units than persistent CTAs, against the oracle and the token kernel."""
+    w = _small(d, 1, dtype, units=units, seed=2000 + d)
+    q, k, v = W.make_inputs(w)
+    B, H = units
+    g = torch.Generator().manual_seed(d + B)
+    S0 = torch.randn((B, H, d, d), generator=g) * 0.3
+    A0 = _spd((B, H), g, d)
+    z0 = torch.rand((B, H, d), generator=g) * 3.0
+    errs, got, ref = check_parity(q, k, v, 1.0, 1e-5, S0=S0, A0=A0, z0=z0, flags=flags,
+                                  kernel=vla.VLA_KERNEL_DECODE, label="decode d=%d" % d)
+    tok = run_gpu(q, k, v, 1.0, S0=S0, A0=A0, z0=z0, flags=flags, kernel=vla.VLA_KERNEL_TOKEN)
+    assert rel_err(tok.out, ref.out) <= 1e-5
+    auto = run_gpu(q, k, v, 1.0, S0=S0, A0=A0, z0=z0, flags=flags)     # AUTO takes the same kernel
+    assert torch.equal(auto.out, got.out) and torch.equal(auto.S_T, got.S_T) and torch.equal(auto.A_T, got.A_T)
+
+
+def test_single_step_kernel_in_a_decode_loop_and_its_limits():
+    """Five steps, one call each, states updated in place; then the shapes it does not take."""
+    dev = torch.device("cuda:0")
+    d, T = 128, 5
+    w = _small(d, T, "bf16", units=(2, 100), seed=77)
+    q, k, v = W.make_inputs(w)
+    g = torch.Generator().manual_seed(1)
+    S0 = torch.randn((2, 100, d, d), generator=g) * 0.1
+    A0 = _spd((2, 100), g, d)
+    z0 = torch.rand((2, 100, d), generator=g)
+    ref = run_oracle(q, k, v, 1.0, S0=S0, A0=A0, z0=z0)
+    S, A, z = S0.to(dev), A0.to(dev), z0.to(dev)
+    outs = []
+    for t in range(T):
+        sl = lambda x: x[:, :, t:t + 1].contiguous().to(dev)
+        r = vla.vla_forward(sl(q), sl(k), sl(v), 1.0, S0=S, A0=A, z0=z, S_T=S, A_T=A, z_T=z,
+                            kernel=vla.VLA_KERNEL_DECODE)
+        outs.append(r.out)
+    torch.cuda.synchronize()
+    assert rel_err(torch.cat(outs, dim=2), ref.out) <= 1e-5
+    assert rel_err(S, ref.S_T) <= 1e-5 and rel_err(A, ref.A_T) <= 1e-5 and rel_err(z, ref.z_T) <= 1e-5
+    sl = lambda x: x[:, :, :1].contiguous().to(dev)
+    with pytest.raises(vla.VlaError) as ei:      # no carried state: nothing to stream
+        vla.vla_forward(sl(q), sl(k), sl(v), 1.0, kernel=vla.VLA_KERNEL_DECODE)
+    assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+    with pytest.raises(vla.VlaError):            # more than one step
+        vla.vla_forward(q.to(dev), k.to(dev), v.to(dev), 1.0, S0=S, A0=A, kernel=vla.VLA_KERNEL_DECODE)

@@ -9,8 +9,11 @@
 //   bulk load (TMA, mbarrier)  ->  compute in place  ->  bulk store (bulk group)
 //
 // While job m is computed, job m+1 is landing and job m-1 is leaving, so loads and stores
-// of different units overlap with each other and with the arithmetic.  The unit's q, k, v
-// rows and key sum travel with its A job.  Every mbarrier wait is bounded.
+// of different units overlap with each other and with the arithmetic.  The copies are driven
+// by one thread of a ninth warp, so that the eight computing warps never wait for a store to
+// drain: it stores a buffer as soon as the job in it is computed, waits until the store has
+// read the buffer, and refills it with the job three ahead.  The unit's q, k, v rows and key
+// sum travel with its A job.  Every mbarrier wait is bounded.
 //
 //   A job:  z = A k_hat;  delta = max(1 + k_hat.z, eps);  A <- A - z z^T / delta;
 //           alpha = (z/delta) / max(||z||/delta, eps)          (u = k_hat: A_t k_hat = z/delta)
@@ -24,20 +27,21 @@ namespace vla {
 
 template <int D, typename TIn>
 struct DecodeCfg {
-  static constexpr int NT = 256;
+  static constexpr int NC = 256;             // computing threads
+  static constexpr int NT = NC + 32;         // + the copy warp
   static constexpr int NBUF = 3;
   static constexpr size_t mat_bytes = size_t(D) * D * sizeof(float);
   static constexpr size_t vec_in_bytes = 3 * size_t(D) * sizeof(TIn) + size_t(D) * sizeof(float);  // q,k,v,z0
   static constexpr size_t vec_stage_bytes = (vec_in_bytes + 127) / 128 * 128;
   static constexpr size_t work_floats = 8 * size_t(D) + 16;   // khat qf vf zsum | z alpha e r | scalars
   static constexpr size_t smem_bytes = NBUF * mat_bytes + 2 * vec_stage_bytes +
-                                       work_floats * sizeof(float) + (NBUF + 1) * sizeof(uint64_t) + 128;
+                                       work_floats * sizeof(float) + (2 * NBUF + 1) * sizeof(uint64_t) + 128;
 };
 
 template <int D, typename TIn>
-__global__ void __launch_bounds__(256, 1) vla_decode_kernel(const ScanParams p) {
+__global__ void __launch_bounds__(288, 1) vla_decode_kernel(const ScanParams p) {
   using Cfg = DecodeCfg<D, TIn>;
-  constexpr int NT = Cfg::NT, NBUF = Cfg::NBUF;
+  constexpr int NT = Cfg::NC, NBUF = Cfg::NBUF;   // NT: computing threads
   constexpr int LPR = D / 4;            // lanes that cover one row as float4
   constexpr int RPP = NT / LPR;         // rows per pass of the whole CTA
   constexpr int NPASS = D / RPP;        // passes over a matrix
@@ -57,7 +61,8 @@ __global__ void __launch_bounds__(256, 1) vla_decode_kernel(const ScanParams p) 
   float* scal = rv + D;          // [0] 1/den
   uint64_t* mfull = reinterpret_cast<uint64_t*>(
       (reinterpret_cast<uintptr_t>(scal + D + 16) + 7) & ~uintptr_t(7));        // [NBUF]
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(mfull + NBUF);
+  uint64_t* mdone = mfull + NBUF;                                                // [NBUF] job computed
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(mdone + NBUF);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int rl = tid / LPR;             // row within a pass
@@ -96,14 +101,34 @@ __global__ void __launch_bounds__(256, 1) vla_decode_kernel(const ScanParams p) 
 
   if (tid == 0) {
     *abort_flag = 0;
-    for (int b = 0; b < NBUF; ++b) mbar_init(&mfull[b], 1);
+    for (int b = 0; b < NBUF; ++b) {
+      mbar_init(&mfull[b], 1);
+      mbar_init(&mdone[b], 1);
+    }
     mbar_init_fence();
   }
   __syncthreads();
-  if (tid == 0) {
-    if (njobs > 0) issue(0);
-    if (njobs > 1) issue(1);
+  if (warp == NT / 32) {
+    // ---- copy warp: one thread owns every bulk load and store of this CTA
+    if (lane != 0) return;
+    for (int m = 0; m < NBUF && m < njobs; ++m) issue(m);
+    for (int m = 0; m < njobs; ++m) {
+      const int unit = int(blockIdx.x) + (m >> 1) * int(gridDim.x);
+      const int b = m % NBUF;
+      wait(&mdone[b], uint32_t(m / NBUF) & 1u);
+      if (*abort_flag) break;
+      bulk_store(((m & 1) == 0 ? p.A_T : p.S_T) + size_t(unit) * D * D, mat + size_t(b) * D * D,
+                 uint32_t(Cfg::mat_bytes));
+      bulk_commit();
+      if (m + NBUF < njobs) {
+        bulk_wait_read<0>();     // the store has read the buffer: refill it
+        issue(m + NBUF);
+      }
+    }
+    bulk_wait_all<0>();
+    return;
   }
+  auto cta_bar = [&]() { asm volatile("bar.sync 1, %0;" ::"n"(Cfg::NC) : "memory"); };
 
   float delta_inv = 1.0f;   // 1/delta of the current unit
 #pragma unroll 1
@@ -147,7 +172,7 @@ __global__ void __launch_bounds__(256, 1) vla_decode_kernel(const ScanParams p) 
         for (int e = 0; e < D / 32; ++e) khat[e * 32 + lane] = kf[e] * inv;
         if (lane == 0) scal[0] = ident ? 1.0f : 1.0f / fmaxf(dn, eps);
       }
-      __syncthreads();
+      cta_bar();
       // ---- z = A k_hat (row dots: LPR lanes per row)
       const float4 k4 = reinterpret_cast<const float4*>(khat)[c4];
 #pragma unroll
@@ -159,7 +184,7 @@ __global__ void __launch_bounds__(256, 1) vla_decode_kernel(const ScanParams p) 
         for (int off = LPR / 2; off >= 1; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
         if (c4 == 0) zv[row] = s;
       }
-      __syncthreads();
+      cta_bar();
       // ---- delta, ||z||, alpha (every warp forms the two sums itself)
       float kz = 0.f, zz = 0.f;
 #pragma unroll
@@ -208,7 +233,7 @@ __global__ void __launch_bounds__(256, 1) vla_decode_kernel(const ScanParams p) 
         }
         if (c4 == 0) { ev[row] = vf[row] - s; rv[row] = r; }
       }
-      __syncthreads();
+      cta_bar();
       // ---- o = (r + e (alpha.q_f)) / den
       float aq = 0.f;
 #pragma unroll
@@ -229,20 +254,13 @@ __global__ void __launch_bounds__(256, 1) vla_decode_kernel(const ScanParams p) 
         *sp = a;
       }
     }
-    // ---- the updated matrix leaves; the buffer of job m-1 is free for job m+2 once its store
-    //      has read it
+    // ---- the updated matrix is ready to leave: hand the buffer to the copy thread
     fence_async_smem();
-    __syncthreads();
+    cta_bar();
     if (tid == 0) {
-      bulk_store((is_A ? p.A_T : p.S_T) + size_t(unit) * D * D, M, uint32_t(Cfg::mat_bytes));
-      bulk_commit();
-      if (m + 2 < njobs) {
-        bulk_wait_read<1>();
-        issue(m + 2);
-      }
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&mdone[b])) : "memory");
     }
   }
-  if (tid == 0) bulk_wait_all<0>();
 }
 
 }  // namespace vla

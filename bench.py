@@ -347,6 +347,15 @@ def main():
             "unit_limited_frac_bound": min(w.units, n_sm) / n_sm}
     if clocks and clocks.get("sm_mhz"):
         roof["frac_at_sampled_clock"] = achieved_tflops / (fp32_peak_nominal * clocks["sm_mhz"] / sm_max_mhz)
+    # the fp32 FMA rate this device sustains right now (register-only loop in the library),
+    # measured after the timed region so that it cannot disturb it
+    try:
+        measured = vla.measure_fp32_fma_tflops(dev)
+        roof["fp32_peak_measured_tflops"] = measured
+        roof["frac_of_measured_fp32"] = achieved_tflops / measured
+    except Exception as exc:   # the roofline above stands on the derived peak
+        roof["fp32_peak_measured_tflops"] = None
+        roof["fp32_peak_measured_error"] = str(exc)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * total_s_max / args.steps,

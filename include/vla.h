@@ -186,6 +186,16 @@ int vla_seqpar_segments(int B, int H, int T, int d_k, int qkv_dtype);
 /* Device bytes vla_forward_seqpar needs for `segments` >= 1 (0 on a bad argument). */
 size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
 
+/*
+ * vla_probe_fp32_fma -- measurement helper (the paper has no counterpart): enqueues a
+ * register-only loop of fp32 FMAs on every SM (2048 threads per SM, 16 independent chains per
+ * thread, `iters` x 128 FMAs per thread) and reports the floating-point operations launched in
+ * *flops (HOST pointer, may be NULL).  Timed with events by the caller it gives the fp32
+ * FMA rate this device sustains at its current clocks -- the "alu" roofline the scan kernels
+ * are measured against.  `sink` is a DEVICE float the kernel never actually writes.
+ */
+int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream);
+
 /* Device bytes vla_forward_host needs for these sizes (0 on invalid sizes). */
 size_t vla_host_workspace_bytes(int B, int H, int T, int d_k, int d_v, int qkv_dtype, int has_u);
 

@@ -26,6 +26,7 @@ VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK, VLA_KERNEL_DECODE = 0, 1, 2
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",
            "vla_forward_seqpar", "vla_seqpar_segments", "vla_seqpar_workspace_bytes",
+           "vla_probe_fp32_fma",
            "vla_query_support", "vla_status_string", "vla_version")
 
 
@@ -80,6 +81,8 @@ def load_library():
             lib.vla_seqpar_segments.argtypes = [i, i, i, i, i]
             lib.vla_seqpar_workspace_bytes.restype = ctypes.c_size_t
             lib.vla_seqpar_workspace_bytes.argtypes = [i, i, i, i, i]
+            lib.vla_probe_fp32_fma.restype = i
+            lib.vla_probe_fp32_fma.argtypes = [i, vp, ctypes.POINTER(ctypes.c_double), vp]
             lib.vla_host_workspace_bytes.restype = ctypes.c_size_t
             lib.vla_host_workspace_bytes.argtypes = [i, i, i, i, i, i, i]
             lib.vla_query_support.restype = i
@@ -199,6 +202,29 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
     if rc != VLA_OK:
         raise VlaError(rc, "vla_forward")
     return VlaResult(out, S_T, A_T, z_T, status)
+
+
+def measure_fp32_fma_tflops(device=None, iters: int = 4096, reps: int = 5) -> float:
+    """fp32 FMA rate of the device at its current clocks (register-only loop, best of ``reps``)."""
+    lib = load_library()
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    sink = torch.zeros((4,), dtype=torch.float32, device=dev)
+    flops = ctypes.c_double(0.0)
+    best = 0.0
+    with torch.cuda.device(dev):
+        st = torch.cuda.current_stream(dev)
+        for r in range(reps + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
+            rc = lib.vla_probe_fp32_fma(int(iters), _ptr(sink), ctypes.byref(flops),
+                                        ctypes.c_void_p(st.cuda_stream))
+            b.record(st)
+            if rc != VLA_OK:
+                raise VlaError(rc, "vla_probe_fp32_fma")
+            b.synchronize()
+            if r > 0:
+                best = max(best, flops.value / (a.elapsed_time(b) * 1e-3) / 1e12)
+    return best
 
 
 def seqpar_segments(B: int, H: int, T: int, d_k: int, dtype: torch.dtype) -> int:

@@ -437,6 +437,11 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   return vla::seqpar_after_scan(d_k, sp, A_T, o.zT, AT2, zT2, st);
 }
 
+int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream) {
+  if (iters <= 0 || !sink) return VLA_ERR_INVALID_ARG;
+  return vla::launch_fp32_probe(iters, sink, flops, static_cast<cudaStream_t>(stream));
+}
+
 int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags) {
   if (qkv_dtype != VLA_F32 && qkv_dtype != VLA_BF16) return VLA_ERR_UNSUPPORTED;
   if (flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_UNSUPPORTED;

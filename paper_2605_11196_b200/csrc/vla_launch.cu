@@ -90,6 +90,45 @@ int launch_token(int d, int dtype, const ScanParams& p, cudaStream_t st) {
   }
 }
 
+// ---------------------------------------------------------------- fp32 FMA rate probe
+namespace {
+
+// Register-only chains of fma.rn.f32: 16 independent accumulators per thread, 2048 threads
+// per SM.  The result is stored only if it equals a value it cannot take, so that the loop
+// is kept but no memory traffic is timed.
+__global__ void __launch_bounds__(1024) fp32_fma_probe_kernel(float* sink, int iters) {
+  float acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc[i] = 1.0f + 1e-3f * float(i) + 1e-6f * float(threadIdx.x);
+  const float m = 0.999f, c = 1e-3f;
+#pragma unroll 1
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+      for (int i = 0; i < 16; ++i) acc[i] = fmaf(acc[i], m, c);
+  }
+  float s = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) s += acc[i];
+  if (s == 123456.789f) sink[0] = s;
+}
+
+}  // namespace
+
+int launch_fp32_probe(int iters, float* sink, double* flops, cudaStream_t st) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  const int grid = 2 * sms, block = 1024;
+  fp32_fma_probe_kernel<<<grid, block, 0, st>>>(sink, iters);
+  if (flops) *flops = 2.0 * 16.0 * 8.0 * double(iters) * double(grid) * double(block);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
 // ---------------------------------------------------------------- decode kernel
 namespace {
 

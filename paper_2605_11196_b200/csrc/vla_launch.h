@@ -31,6 +31,9 @@ int seqpar_before_scan(int d, int dtype, const SeqParParams& sp, cudaStream_t st
 int seqpar_after_scan(int d, const SeqParParams& sp, float* A_T, float* zT, const float* AT2,
                       const float* zT2, cudaStream_t st);
 
+// Register-only fp32 FMA loop over the whole device (measurement helper); *flops = work launched.
+int launch_fp32_probe(int iters, float* sink, double* flops, cudaStream_t st);
+
 // Launch ids for the balanced schedule's hand-off flags (never 0, never repeated within
 // 2^32 launches).
 unsigned int next_launch_epoch();

@@ -162,7 +162,8 @@ int vla_forward_host_static(const void* q, const void* k, const void* v, float l
  * lambda I + sum of u u^T over the earlier tokens (Eq. "penalty"), formed in fp64.  Results
  * equal vla_forward's up to rounding.
  *
- * Arguments as vla_forward, with these differences: A_0 is always I/lambda (there is no A0);
+ * Arguments as vla_forward, with these differences: a carried-in A0 must be symmetric positive
+ * definite (it is inverted in fp64 to recover the penalty matrix the earlier tokens left);
  * the periodic refresh and VLA_KERNEL_TOKEN are not available (VLA_ERR_UNSUPPORTED), nor is
  * d = 16; `segments` must divide T/16 (T a multiple of 16), else VLA_ERR_INVALID_ARG;
  * segments <= 0 lets the library choose (vla_seqpar_segments), and a choice of 1 runs
@@ -173,7 +174,7 @@ int vla_forward_host_static(const void* q, const void* k, const void* v, float l
  */
 int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda_,
                        int B, int H, int T, int d_k, int d_v,
-                       const float* S0,
+                       const float* S0, const float* A0,
                        float* out, float* S_T, float* A_T,
                        const vla_opts_t* opts, int segments,
                        void* workspace, size_t workspace_bytes, void* stream);

@@ -75,7 +75,7 @@ def load_library():
             lib.vla_forward_host_static.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp,
                                                     ctypes.POINTER(VlaOpts), vp]
             lib.vla_forward_seqpar.restype = i
-            lib.vla_forward_seqpar.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp, i,
+            lib.vla_forward_seqpar.argtypes = [vp, vp, vp, f, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i,
                                                vp, ctypes.c_size_t, vp]
             lib.vla_seqpar_segments.restype = i
             lib.vla_seqpar_segments.argtypes = [i, i, i, i, i]
@@ -238,7 +238,7 @@ def seqpar_workspace_bytes(B: int, H: int, T: int, d_k: int, segments: int) -> i
 
 
 def vla_forward_seqpar(q, k, v, lam: float, *, segments: int = 0, workspace=None, u=None, S0=None,
-                       z0=None, flags: int = 0, eps: float = 1e-4, out=None, S_T=None, A_T=None,
+                       A0=None, z0=None, flags: int = 0, eps: float = 1e-4, out=None, S_T=None, A_T=None,
                        z_T=None, status=None, stream: Optional[torch.cuda.Stream] = None,
                        want_status: bool = True) -> VlaResult:
     """Sequence-parallel scan of CUDA tensors: each unit's sequence is cut into ``segments``
@@ -255,6 +255,7 @@ def vla_forward_seqpar(q, k, v, lam: float, *, segments: int = 0, workspace=None
     _chk(v, (B, H, T, dv), q.dtype, "v"); _chk(u, (B, H, T, dk), q.dtype, "u")
     f32 = torch.float32
     _chk(S0, (B, H, dv, dk), f32, "S0"); _chk(z0, (B, H, dk), f32, "z0")
+    _chk(A0, (B, H, dk, dk), f32, "A0")
     if out is None:
         out = torch.empty((B, H, T, dv), dtype=f32, device=dev)
     if S_T is None:
@@ -277,7 +278,7 @@ def vla_forward_seqpar(q, k, v, lam: float, *, segments: int = 0, workspace=None
             raise ValueError("workspace must be a contiguous CUDA uint8 tensor on the inputs' device")
         opts = _make_opts(dt, u, flags, eps, z0, z_T, status, VLA_KERNEL_AUTO, None)
         rc = lib.vla_forward_seqpar(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv,
-                                    _ptr(S0), _ptr(out), _ptr(S_T), _ptr(A_T), ctypes.byref(opts),
+                                    _ptr(S0), _ptr(A0), _ptr(out), _ptr(S_T), _ptr(A_T), ctypes.byref(opts),
                                     int(segments), _ptr(workspace), workspace.numel(),
                                     ctypes.c_void_p(st.cuda_stream))
     if rc != VLA_OK:

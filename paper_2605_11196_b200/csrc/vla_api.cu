@@ -117,7 +117,7 @@ void* static_scratch_for_current_device() {
 
 // ---- sequence-parallel entry point: workspace layout and segment choice
 struct SeqParLayout {
-  size_t Gd, zsum, Astart, zstart, ST2, AT2, zT2, wn, Sstart, total;
+  size_t Gd, zsum, Astart, zstart, ST2, AT2, zT2, wn, Sstart, M0, total;
 };
 
 SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
@@ -134,6 +134,7 @@ SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
   L.zT2 = take(2 * N * D * sizeof(float));
   L.wn = take(units * T * D * sizeof(float));
   L.Sstart = take(N * D * D * sizeof(float));
+  L.M0 = take(units * D * D * sizeof(double));
   L.total = off + 256;
   return L;
 }
@@ -376,16 +377,17 @@ size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments) {
 }
 
 int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda_, int B, int H,
-                       int T, int d_k, int d_v, const float* S0, float* out, float* S_T, float* A_T,
+                       int T, int d_k, int d_v, const float* S0, const float* A0, float* out,
+                       float* S_T, float* A_T,
                        const vla_opts_t* opts, int segments, void* workspace,
                        size_t workspace_bytes, void* stream) {
   vla_opts_t o;
   int rc = resolve_opts(opts, &o);
   if (rc != VLA_OK) return rc;
-  rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, nullptr, out);
+  rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, out);
   if (rc != VLA_OK) return rc;
   if (d_k < 32 || o.refresh_period > 0 || o.kernel == VLA_KERNEL_TOKEN) return VLA_ERR_UNSUPPORTED;
-  const void* ptrs[] = {q, k, v, o.u, S0, out, S_T, A_T, o.z0, o.zT};
+  const void* ptrs[] = {q, k, v, o.u, S0, A0, out, S_T, A_T, o.z0, o.zT};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return VLA_ERR_ALIGNMENT;
   if (o.status && (reinterpret_cast<uintptr_t>(o.status) & 3u)) return VLA_ERR_ALIGNMENT;
@@ -394,7 +396,7 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   int P = segments;
   if (P <= 0) P = seqpar_choose_segments(units, T, d_k, o.qkv_dtype);
   if (P == 1)   // nothing to cut: the plain scan
-    return vla_forward(q, k, v, lambda_, B, H, T, d_k, d_v, S0, nullptr, out, S_T, A_T, opts, stream);
+    return vla_forward(q, k, v, lambda_, B, H, T, d_k, d_v, S0, A0, out, S_T, A_T, opts, stream);
   if (T % 16 != 0 || (T / 16) % P != 0) return VLA_ERR_INVALID_ARG;
   if (2LL * units * P > 0x7fffffffLL) return VLA_ERR_INVALID_ARG;
   const SeqParLayout L = seqpar_layout(size_t(units), size_t(T), size_t(d_k), size_t(P));
@@ -404,7 +406,8 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   const int N = units * P;
 
   vla::SeqParParams sp;
-  sp.k = k; sp.u = o.u; sp.S0 = S0; sp.z0 = o.z0; sp.out = out; sp.S_T = S_T;
+  sp.k = k; sp.u = o.u; sp.S0 = S0; sp.A0 = A0; sp.z0 = o.z0; sp.out = out; sp.S_T = S_T;
+  sp.M0 = reinterpret_cast<double*>(w + L.M0);
   sp.Gd = reinterpret_cast<double*>(w + L.Gd);
   sp.zsum = reinterpret_cast<float*>(w + L.zsum);
   sp.Astart = reinterpret_cast<float*>(w + L.Astart);

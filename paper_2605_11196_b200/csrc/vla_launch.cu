@@ -177,6 +177,7 @@ int seqpar_before_d(int dtype, const SeqParParams& sp, cudaStream_t st) {
     return VLA_ERR_CUDA;
   if (dtype == VLA_F32) seqpar_gram_kernel<D, float><<<dim3(N, kGramSplit), 256, 0, st>>>(sp);
   else seqpar_gram_kernel<D, uint16_t><<<dim3(N, kGramSplit), 256, 0, st>>>(sp);
+  if (sp.A0) seqpar_m0_kernel<D><<<sp.units, 256, 0, st>>>(sp);
   seqpar_invert_kernel<D><<<N, 256, 0, st>>>(sp);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }

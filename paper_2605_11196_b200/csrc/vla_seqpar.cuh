@@ -11,7 +11,8 @@
 //   1. gram     G_j = sum_{t in segment j} u_t u_t^T  (fp32 products, fp64 accumulation) and
 //               the segment's sum of phi(k)
 //   2. invert   A_start_j = (lambda I + sum_{i<j} G_i)^-1 in fp64 (Gauss-Jordan, no pivoting:
-//               the matrix is symmetric positive definite), running key sum at the start
+//               the matrix is symmetric positive definite), running key sum at the start;
+//               with a carried-in A0, lambda I is replaced by A0^-1 (also formed in fp64)
 //   3. scan     the chunk kernel over 2 * units * P virtual units: segment j from S = 0
 //               (readout o0_t, final state G_j) and its transfer scan from S = I with v = 0
 //               (readout w_t = P_t q_t / den_t, final state P_j)
@@ -140,6 +141,57 @@ __global__ void __launch_bounds__(256) seqpar_gram_kernel(const SeqParParams p) 
   }
 }
 
+// In-place Gauss-Jordan inversion of a symmetric positive definite D x D matrix held in
+// registers by 256 threads (thread: row r, columns c0 .. c0 + EC - 1); no pivoting.  fp64
+// arithmetic is scarce on this part: one FMA per element and pivot, the pivot's reciprocal
+// folded into the column factor.
+template <int D, int EC>
+__device__ __forceinline__ void seqpar_gauss_jordan(double (&m)[EC], int r, int c0, double* rowraw,
+                                                    double* colp) {
+#pragma unroll 1
+  for (int pv = 0; pv < D; ++pv) {
+    if (r == pv) {
+#pragma unroll
+      for (int e = 0; e < EC; ++e) rowraw[c0 + e] = m[e];
+    }
+    if (pv >= c0 && pv < c0 + EC) {
+      double x = 0.0;
+#pragma unroll
+      for (int e = 0; e < EC; ++e)
+        if (c0 + e == pv) x = m[e];
+      colp[r] = x;
+    }
+    __syncthreads();
+    const double d = 1.0 / rowraw[pv];
+    const double ncrd = -colp[r] * d;
+    if (r == pv) {
+#pragma unroll
+      for (int e = 0; e < EC; ++e) m[e] = (c0 + e == pv) ? d : rowraw[c0 + e] * d;
+    } else {
+#pragma unroll
+      for (int e = 0; e < EC; ++e) m[e] = (c0 + e == pv) ? ncrd : fma(ncrd, rowraw[c0 + e], m[e]);
+    }
+    __syncthreads();
+  }
+}
+
+// ---- 2a. With a carried-in A0: M0 = A0^-1 per unit in fp64 (the penalty matrix the earlier
+// tokens left behind).  One CTA of 256 threads per unit.
+template <int D>
+__global__ void __launch_bounds__(256) seqpar_m0_kernel(const SeqParParams p) {
+  constexpr int EC = D * D / 256, TPR = D / EC;
+  __shared__ double rowraw[D];
+  __shared__ double colp[D];
+  const int unit = blockIdx.x, tid = threadIdx.x;
+  const int r = tid / TPR, c0 = (tid % TPR) * EC;
+  double m[EC];
+#pragma unroll
+  for (int e = 0; e < EC; ++e) m[e] = double(p.A0[(size_t(unit) * D + r) * D + c0 + e]);
+  seqpar_gauss_jordan<D, EC>(m, r, c0, rowraw, colp);
+#pragma unroll
+  for (int e = 0; e < EC; ++e) p.M0[(size_t(unit) * D + r) * D + c0 + e] = m[e];
+}
+
 // ---- 2. A at the start of segment j, and the running key sum there.  One CTA of 256
 // threads per (unit, segment).  The matrix stays in registers: thread t owns D*D/256
 // consecutive elements of one row; a pivot step exchanges only the pivot row and column
@@ -164,46 +216,21 @@ __global__ void __launch_bounds__(256) seqpar_invert_kernel(const SeqParParams p
   if (j == 0) {
     const float dg = 1.0f / p.lambda;
 #pragma unroll
-    for (int e = 0; e < EC; ++e) A[r * D + c0 + e] = (c0 + e == r) ? dg : 0.0f;
+    for (int e = 0; e < EC; ++e)
+      A[r * D + c0 + e] = p.A0 ? p.A0[(size_t(unit) * D + r) * D + c0 + e] : ((c0 + e == r) ? dg : 0.0f);
     return;
   }
-  // M = lambda I + the Gram matrices of the earlier segments
+  // M = lambda I (or the carried-in A0^-1) + the Gram matrices of the earlier segments
   double m[EC];
 #pragma unroll
-  for (int e = 0; e < EC; ++e) m[e] = (c0 + e == r) ? double(p.lambda) : 0.0;
+  for (int e = 0; e < EC; ++e)
+    m[e] = p.A0 ? p.M0[(size_t(unit) * D + r) * D + c0 + e] : ((c0 + e == r) ? double(p.lambda) : 0.0);
   for (int i = 0; i < j; ++i) {
     const double* G = p.Gd + (size_t(unit) * p.P + i) * D * D + r * D + c0;
 #pragma unroll
     for (int e = 0; e < EC; ++e) m[e] += G[e];
   }
-  // in-place Gauss-Jordan inversion (no pivoting: symmetric positive definite)
-#pragma unroll 1
-  for (int pv = 0; pv < D; ++pv) {
-    if (r == pv) {
-#pragma unroll
-      for (int e = 0; e < EC; ++e) rowraw[c0 + e] = m[e];
-    }
-    if (pv >= c0 && pv < c0 + EC) {
-      double x = 0.0;
-#pragma unroll
-      for (int e = 0; e < EC; ++e)
-        if (c0 + e == pv) x = m[e];
-      colp[r] = x;
-    }
-    __syncthreads();
-    // fp64 arithmetic is scarce on this part: one FMA per element, the pivot's reciprocal
-    // folded into the column factor
-    const double d = 1.0 / rowraw[pv];
-    const double ncrd = -colp[r] * d;
-    if (r == pv) {
-#pragma unroll
-      for (int e = 0; e < EC; ++e) m[e] = (c0 + e == pv) ? d : rowraw[c0 + e] * d;
-    } else {
-#pragma unroll
-      for (int e = 0; e < EC; ++e) m[e] = (c0 + e == pv) ? ncrd : fma(ncrd, rowraw[c0 + e], m[e]);
-    }
-    __syncthreads();
-  }
+  seqpar_gauss_jordan<D, EC>(m, r, c0, rowraw, colp);
 #pragma unroll
   for (int e = 0; e < EC; ++e) A[r * D + c0 + e] = float(m[e]);
 }

@@ -12,6 +12,8 @@ struct SeqParParams {
   const void* k;        // [units, T, D] raw keys
   const void* u;        // [units, T, D] explicit penalty directions or nullptr
   const float* S0;      // [units, D, D] or nullptr
+  const float* A0;      // [units, D, D] symmetric positive definite, or nullptr (I / lambda)
+  double* M0;           // [units, D, D] A0^-1 (only with A0)
   const float* z0;      // [units, D] or nullptr
   float* out;           // [units, T, D] o0 on entry of `correct`, o on exit
   float* S_T;           // [units, D, D] or nullptr

@@ -18,10 +18,10 @@ def _small(d, T, dtype, units=(1, 2), seed=1):
     return W.Workload("t", units[0], units[1], d, T, dtype, seed)
 
 
-def _run_seqpar(q, k, v, lam, segments, u=None, S0=None, z0=None, flags=0):
+def _run_seqpar(q, k, v, lam, segments, u=None, S0=None, A0=None, z0=None, flags=0):
     dev = torch.device("cuda:0")
     mv = lambda x: None if x is None else x.to(dev).contiguous()
-    r = vla.vla_forward_seqpar(mv(q), mv(k), mv(v), lam, segments=segments, u=mv(u), S0=mv(S0), z0=mv(z0),
+    r = vla.vla_forward_seqpar(mv(q), mv(k), mv(v), lam, segments=segments, u=mv(u), S0=mv(S0), A0=mv(A0), z0=mv(z0),
                                flags=flags)
     torch.cuda.synchronize()
     assert int(r.status.item()) == 0, vla.status_string(int(r.status.item()))
@@ -52,18 +52,21 @@ def test_segments_agree_with_the_oracle(d, dtype, flags, segments):
 @pytest.mark.parametrize("d", [32, 128])
 @pytest.mark.parametrize("flags", [0, IDENT])
 def test_carried_state_and_explicit_u(d, flags):
-    """S0 and z0 carried in (A_0 is always I/lambda here), explicit penalty directions, many
+    """S0, z0 and a symmetric positive definite A0 carried in, explicit penalty directions, many
     short segments (one chunk each)."""
     w = _small(d, 192, "f32", units=(1, 3), seed=70 + d)
     q, k, v = W.make_inputs(w)
     g = torch.Generator().manual_seed(d)
     S0 = torch.randn((1, 3, d, d), generator=g) * 0.1
     z0 = torch.rand((1, 3, d), generator=g)
+    h = torch.randn((1, 3, d, d), generator=g) * 0.1
+    A0s = h @ h.transpose(-1, -2) + 0.3 * torch.eye(d)
     for u in (None, W.make_u(w, d ** -0.5)):
-        ref = run_oracle(q, k, v, 0.5, u=u, S0=S0, z0=z0, flags=flags)
-        for segments in (3, 12):
-            r = _run_seqpar(q, k, v, 0.5, segments, u=u, S0=S0, z0=z0, flags=flags)
-            _check(r, ref, 1e-4, "seqpar carried d=%d P=%d" % (d, segments))
+        for A0 in (None, A0s):
+            ref = run_oracle(q, k, v, 0.5, u=u, S0=S0, A0=A0, z0=z0, flags=flags)
+            for segments in (3, 12):
+                r = _run_seqpar(q, k, v, 0.5, segments, u=u, S0=S0, A0=A0, z0=z0, flags=flags)
+                _check(r, ref, 1e-4, "seqpar carried d=%d P=%d" % (d, segments))
 
 
 def test_one_segment_is_the_plain_scan_and_bad_arguments_are_refused():

@@ -110,7 +110,9 @@ struct ChunkCfg {
   static constexpr int NWG = D / 32;             // warps per group
   static constexpr int NIN = UT ? 4 : 3;         // q, k, v[, u]
   // raw q/k/v[/u] chunks in flight (fewer on the general path: shared memory is the limit)
-  static constexpr int NSTAGE = UT ? (sizeof(TIn) == 2 ? 2 : 1) : (sizeof(TIn) == 2 ? 4 : 2);
+  // (the three-group kernel with 16-bit inputs keeps one stage: two of its CTAs then share an SM)
+  static constexpr int NSTAGE = TRI ? (sizeof(TIn) == 2 ? 1 : 2)
+                                    : UT ? (sizeof(TIn) == 2 ? 2 : 1) : (sizeof(TIn) == 2 ? 4 : 2);
   static constexpr int RING = 2;                 // Z / Gu / HT / sc slots (group A -> group S)
   static constexpr int KRING = 3;                // widened k_hat / q_f / v / ||phi(k)|| slots
   static constexpr int CP = C + 4;               // padded row of the small C x C matrices
@@ -367,8 +369,8 @@ __device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) 
 // launches at d <= 64) next to group S, on the same products of group A.  Its readout goes to
 // out2 and its final state to S_T[n_main + unit].
 template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false>
-__global__ void __launch_bounds__((TRI ? 3 : 2) * D, 1) vla_scan_chunk_kernel(const ScanParams p,
-                                                                              const SchedParams sp) {
+__global__ void __launch_bounds__((TRI ? 3 : 2) * D, (TRI && sizeof(TIn) == 2) ? 2 : 1)
+vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
   using Cfg = ChunkCfg<D, TIn, UM, TRI>;
   static_assert(!TRI || (D <= 64 && !BALANCED), "three groups: d <= 64, one CTA per unit");
   constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly

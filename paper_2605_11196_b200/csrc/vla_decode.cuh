@@ -10,7 +10,7 @@
 //
 // While job m is computed, job m+1 is landing and job m-1 is leaving, so loads and stores
 // of different units overlap with each other and with the arithmetic.  The copies are driven
-// by one thread of a ninth warp, so that the eight computing warps never wait for a store to
+// by one thread of an extra warp, so that the sixteen computing warps never wait for a store to
 // drain: it stores a buffer as soon as the job in it is computed, waits until the store has
 // read the buffer, and refills it with the job three ahead.  The unit's q, k, v rows and key
 // sum travel with its A job.  Every mbarrier wait is bounded.
@@ -27,7 +27,7 @@ namespace vla {
 
 template <int D, typename TIn>
 struct DecodeCfg {
-  static constexpr int NC = 256;             // computing threads
+  static constexpr int NC = D >= 64 ? 512 : 256;   // computing threads
   static constexpr int NT = NC + 32;         // + the copy warp
   static constexpr int NBUF = 3;
   static constexpr size_t mat_bytes = size_t(D) * D * sizeof(float);
@@ -39,7 +39,7 @@ struct DecodeCfg {
 };
 
 template <int D, typename TIn>
-__global__ void __launch_bounds__(288, 1) vla_decode_kernel(const ScanParams p) {
+__global__ void __launch_bounds__(DecodeCfg<D, TIn>::NT, 1) vla_decode_kernel(const ScanParams p) {
   using Cfg = DecodeCfg<D, TIn>;
   constexpr int NT = Cfg::NC, NBUF = Cfg::NBUF;   // NT: computing threads
   constexpr int LPR = D / 4;            // lanes that cover one row as float4

@@ -187,7 +187,7 @@ int seqpar_after_d(const SeqParParams& sp, float* A_T, float* zT, const float* A
                    cudaStream_t st) {
   const int N = sp.units * sp.P;
   const int Ls = sp.T / sp.P;
-  const size_t comb_smem = 2 * size_t(D) * (D + 1) * sizeof(float);
+  const size_t comb_smem = (16 + size_t(D)) * (D + 1) * sizeof(float);
   const size_t corr_smem = (size_t(D) + 64) * (D + 4) * sizeof(float);
   if (cudaFuncSetAttribute(seqpar_combine_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(comb_smem)) != cudaSuccess ||
@@ -196,8 +196,9 @@ int seqpar_after_d(const SeqParParams& sp, float* A_T, float* zT, const float* A
     cudaGetLastError();
     return VLA_ERR_CUDA;
   }
-  seqpar_combine_kernel<D><<<sp.units, 256, comb_smem, st>>>(sp);
-  seqpar_correct_kernel<D><<<dim3(N, (Ls + 63) / 64), 256, corr_smem, st>>>(sp);
+  seqpar_combine_kernel<D><<<dim3(sp.units, D / 16), 256, comb_smem, st>>>(sp);
+  const int per_cta = kCorrectTile * kCorrectTiles;
+  seqpar_correct_kernel<D><<<dim3(N, (Ls + per_cta - 1) / per_cta), 256, corr_smem, st>>>(sp);
   if (cudaGetLastError() != cudaSuccess) return VLA_ERR_CUDA;
   // final A and key sum: those of each unit's last segment
   const size_t P = size_t(sp.P);

@@ -235,62 +235,59 @@ __global__ void __launch_bounds__(256) seqpar_invert_kernel(const SeqParParams p
   for (int e = 0; e < EC; ++e) A[r * D + c0 + e] = float(m[e]);
 }
 
-// ---- 4. states at the segment starts, in order.  One CTA per unit; dynamic shared memory:
-// 2 * D * (D + 1) floats.
+// ---- 4. states at the segment starts, in order: S_start_{j+1} = S_start_j P_j + G_j.  The rows
+// of S do not mix, so a unit is spread over D / 16 CTAs of 16 rows each: grid (units, D / 16),
+// 256 threads (thread = one row of the block, D / 16 columns); dynamic shared memory:
+// (16 + D) * (D + 1) floats.
 template <int D>
 __global__ void __launch_bounds__(256) seqpar_combine_kernel(const SeqParParams p) {
   extern __shared__ __align__(16) unsigned char seqpar_smem[];
-  constexpr int LD = D + 1, R = D / 16;
-  float* Sc = reinterpret_cast<float*>(seqpar_smem);   // current S_start
-  float* Pj = Sc + D * LD;
-  const int unit = blockIdx.x, tid = threadIdx.x;
+  constexpr int LD = D + 1, R = D / 16, RB = 16;
+  float* Sc = reinterpret_cast<float*>(seqpar_smem);   // [RB][LD] current rows of S_start
+  float* Pj = Sc + RB * LD;                            // [D][LD]
+  const int unit = blockIdx.x, row0 = blockIdx.y * RB, tid = threadIdx.x;
   const int ty = tid >> 4, tx = tid & 15;
   const size_t N = size_t(p.units) * p.P;
-  for (int idx = tid; idx < D * D; idx += 256)
-    Sc[(idx / D) * LD + idx % D] = p.S0 ? p.S0[size_t(unit) * D * D + idx] : 0.0f;
+  for (int idx = tid; idx < RB * D; idx += 256)
+    Sc[(idx / D) * LD + idx % D] = p.S0 ? p.S0[(size_t(unit) * D + row0) * D + idx] : 0.0f;
   __syncthreads();
   for (int j = 0; j < p.P; ++j) {
     const size_t vu = size_t(unit) * p.P + j;
-    const float* G = p.ST2 + vu * D * D;
+    const float* G = p.ST2 + (vu * D + row0) * D;
     const float* Pg = p.ST2 + (N + vu) * D * D;
-    float* Ss = p.Sstart + vu * D * D;
-    for (int idx = tid; idx < D * D; idx += 256) {
-      Ss[idx] = Sc[(idx / D) * LD + idx % D];
-      Pj[(idx / D) * LD + idx % D] = Pg[idx];
-    }
+    float* Ss = p.Sstart + (vu * D + row0) * D;
+    for (int idx = tid; idx < RB * D; idx += 256) Ss[idx] = Sc[(idx / D) * LD + idx % D];
+    for (int idx = tid; idx < D * D; idx += 256) Pj[(idx / D) * LD + idx % D] = Pg[idx];
     __syncthreads();
-    float acc[R][R];
+    float acc[R];
 #pragma unroll
-    for (int a = 0; a < R; ++a)
-#pragma unroll
-      for (int b = 0; b < R; ++b) acc[a][b] = G[(ty * R + a) * D + tx * R + b];
+    for (int b = 0; b < R; ++b) acc[b] = G[ty * D + tx * R + b];
+#pragma unroll 4
     for (int m = 0; m < D; ++m) {
-      float sa[R], pb[R];
+      const float sa = Sc[ty * LD + m];
 #pragma unroll
-      for (int a = 0; a < R; ++a) { sa[a] = Sc[(ty * R + a) * LD + m]; pb[a] = Pj[m * LD + tx * R + a]; }
-#pragma unroll
-      for (int a = 0; a < R; ++a)
-#pragma unroll
-        for (int b = 0; b < R; ++b) acc[a][b] = fmaf(sa[a], pb[b], acc[a][b]);
+      for (int b = 0; b < R; ++b) acc[b] = fmaf(sa, Pj[m * LD + tx * R + b], acc[b]);
     }
     __syncthreads();
 #pragma unroll
-    for (int a = 0; a < R; ++a)
-#pragma unroll
-      for (int b = 0; b < R; ++b) Sc[(ty * R + a) * LD + tx * R + b] = acc[a][b];
+    for (int b = 0; b < R; ++b) Sc[ty * LD + tx * R + b] = acc[b];
     __syncthreads();
   }
   if (p.S_T)
-    for (int idx = tid; idx < D * D; idx += 256)
-      p.S_T[size_t(unit) * D * D + idx] = Sc[(idx / D) * LD + idx % D];
+    for (int idx = tid; idx < RB * D; idx += 256)
+      p.S_T[(size_t(unit) * D + row0) * D + idx] = Sc[(idx / D) * LD + idx % D];
 }
 
-// ---- 5. o_t = o0_t + S_start_j w_t.  Grid (units * P, Ls / 64); dynamic shared memory:
+// ---- 5. o_t = o0_t + S_start_j w_t.  Grid (units * P, ceil(Ls / 256)): a CTA keeps S_start_j
+// in shared memory and walks four 64-token tiles of its segment; dynamic shared memory:
 // D * (D + 4) + 64 * (D + 4) floats.
+constexpr int kCorrectTile = 64;     // tokens per shared-memory tile
+constexpr int kCorrectTiles = 4;     // tiles per CTA
+
 template <int D>
 __global__ void __launch_bounds__(256) seqpar_correct_kernel(const SeqParParams p) {
   extern __shared__ __align__(16) unsigned char seqpar_smem[];
-  constexpr int LD = D + 4, TBK = 64;
+  constexpr int LD = D + 4, TBK = kCorrectTile;
   constexpr int RW = D >= 64 ? 4 : 2;          // rows per thread: tr, tr + TRW, ...
   constexpr int TRW = D / RW;                  // threads along the rows
   constexpr int TTK = 256 / TRW;               // threads along the tokens
@@ -300,49 +297,53 @@ __global__ void __launch_bounds__(256) seqpar_correct_kernel(const SeqParParams 
   const int vu = blockIdx.x, j = vu % p.P;
   if (j == 0 && !p.S0) return;                 // S_start = 0: nothing to add
   const int Ls = p.T / p.P;
-  const int t0 = blockIdx.y * TBK;
-  const int nt = min(TBK, Ls - t0);
   const int tid = threadIdx.x;
+  const int tr = tid % TRW, tk = tid / TRW;
   const float4* Sg = reinterpret_cast<const float4*>(p.Sstart + size_t(vu) * D * D);
   for (int idx = tid; idx < D * D / 4; idx += 256)
     *reinterpret_cast<float4*>(&Ss[(idx / (D / 4)) * LD + (idx % (D / 4)) * 4]) = Sg[idx];
-  const float4* wg = reinterpret_cast<const float4*>(p.wn + (size_t(vu) * Ls + t0) * D);
-  for (int idx = tid; idx < TBK * D / 4; idx += 256) {
-    const int t = idx / (D / 4);
-    *reinterpret_cast<float4*>(&Wb[t * LD + (idx % (D / 4)) * 4]) =
-        t < nt ? wg[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  __syncthreads();
-  const int tr = tid % TRW, tk = tid / TRW;
-  float acc[TT][RW];
-#pragma unroll
-  for (int a = 0; a < TT; ++a)
-#pragma unroll
-    for (int b = 0; b < RW; ++b) acc[a][b] = 0.0f;
-#pragma unroll 2
-  for (int m = 0; m < D; m += 4) {
-    float4 sv[RW], wv[TT];
-#pragma unroll
-    for (int b = 0; b < RW; ++b) sv[b] = *reinterpret_cast<const float4*>(&Ss[(tr + b * TRW) * LD + m]);
-#pragma unroll
-    for (int a = 0; a < TT; ++a) wv[a] = *reinterpret_cast<const float4*>(&Wb[(tk * TT + a) * LD + m]);
+  for (int tile = 0; tile < kCorrectTiles; ++tile) {
+    const int t0 = (blockIdx.y * kCorrectTiles + tile) * TBK;
+    if (t0 >= Ls) break;                       // uniform over the CTA
+    const int nt = min(TBK, Ls - t0);
+    __syncthreads();                           // the previous tile has been consumed
+    const float4* wg = reinterpret_cast<const float4*>(p.wn + (size_t(vu) * Ls + t0) * D);
+    for (int idx = tid; idx < TBK * D / 4; idx += 256) {
+      const int t = idx / (D / 4);
+      *reinterpret_cast<float4*>(&Wb[t * LD + (idx % (D / 4)) * 4]) =
+          t < nt ? wg[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    __syncthreads();
+    float acc[TT][RW];
 #pragma unroll
     for (int a = 0; a < TT; ++a)
 #pragma unroll
-      for (int b = 0; b < RW; ++b) {
-        acc[a][b] = fmaf(wv[a].x, sv[b].x, acc[a][b]);
-        acc[a][b] = fmaf(wv[a].y, sv[b].y, acc[a][b]);
-        acc[a][b] = fmaf(wv[a].z, sv[b].z, acc[a][b]);
-        acc[a][b] = fmaf(wv[a].w, sv[b].w, acc[a][b]);
+      for (int b = 0; b < RW; ++b) acc[a][b] = 0.0f;
+#pragma unroll 2
+    for (int m = 0; m < D; m += 4) {
+      float4 sv[RW], wv[TT];
+#pragma unroll
+      for (int b = 0; b < RW; ++b) sv[b] = *reinterpret_cast<const float4*>(&Ss[(tr + b * TRW) * LD + m]);
+#pragma unroll
+      for (int a = 0; a < TT; ++a) wv[a] = *reinterpret_cast<const float4*>(&Wb[(tk * TT + a) * LD + m]);
+#pragma unroll
+      for (int a = 0; a < TT; ++a)
+#pragma unroll
+        for (int b = 0; b < RW; ++b) {
+          acc[a][b] = fmaf(wv[a].x, sv[b].x, acc[a][b]);
+          acc[a][b] = fmaf(wv[a].y, sv[b].y, acc[a][b]);
+          acc[a][b] = fmaf(wv[a].z, sv[b].z, acc[a][b]);
+          acc[a][b] = fmaf(wv[a].w, sv[b].w, acc[a][b]);
+        }
+    }
+    float* og = p.out + (size_t(vu) * Ls + t0) * D;
+#pragma unroll
+    for (int a = 0; a < TT; ++a) {
+      const int t = tk * TT + a;
+      if (t < nt) {
+#pragma unroll
+        for (int b = 0; b < RW; ++b) og[size_t(t) * D + tr + b * TRW] += acc[a][b];
       }
-  }
-  float* og = p.out + (size_t(vu) * Ls + t0) * D;
-#pragma unroll
-  for (int a = 0; a < TT; ++a) {
-    const int t = tk * TT + a;
-    if (t < nt) {
-#pragma unroll
-      for (int b = 0; b < RW; ++b) og[size_t(t) * D + tr + b * TRW] += acc[a][b];
     }
   }
 }

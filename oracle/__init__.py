@@ -19,6 +19,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "vla_oracle.c")
 _HDR = os.path.join(_HERE, "vla_oracle.h")
 _LIB = os.path.join(_HERE, "libvla_oracle.so")
+_SRC_BWD = os.path.join(_HERE, "vla_oracle_bwd.c")
+_HDR_BWD = os.path.join(_HERE, "vla_oracle_bwd.h")
+_LIB_BWD = os.path.join(_HERE, "libvla_oracle_bwd.so")
 
 F32, BF16, F64 = 0, 1, 2
 IDENTITY_MAP = 1
@@ -37,6 +40,21 @@ def build(force: bool = False) -> str:
              "-o", tmp, _SRC, "-lm", "-lpthread"])
         os.replace(tmp, _LIB)
     return _LIB
+
+
+def build_bwd(force: bool = False, src: Optional[str] = None, out: Optional[str] = None) -> str:
+    """Compile the backward oracle (a separate shared object; ``src``/``out`` let the mutation
+    tests build a broken copy)."""
+    src = src or _SRC_BWD
+    out = out or _LIB_BWD
+    newest = max(os.path.getmtime(src), os.path.getmtime(_HDR_BWD), os.path.getmtime(_HDR))
+    if force or not os.path.exists(out) or os.path.getmtime(out) < newest:
+        tmp = out + ".tmp.%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-std=c99", "-O2", "-fPIC", "-shared", "-Wall", "-Wextra", "-I", _HERE,
+             "-o", tmp, src, "-lm", "-lpthread"])
+        os.replace(tmp, out)
+    return out
 
 
 class _Trace(ctypes.Structure):
@@ -181,3 +199,68 @@ def forward(*args, **kw) -> OracleResult:
 
 def forward_trace(*args, **kw) -> OracleResult:
     return load().forward_trace(*args, **kw)
+
+
+@dataclass
+class OracleGrads:
+    dq: np.ndarray
+    dk: np.ndarray
+    dv: np.ndarray
+    du: Optional[np.ndarray]
+    dS0: np.ndarray
+    dA0: np.ndarray
+    dz0: np.ndarray
+
+
+class OracleBwdLib:
+    """One loaded build of the backward oracle (``vla_oracle_bwd.c``)."""
+
+    def __init__(self, path: Optional[str] = None):
+        self.path = path or build_bwd()
+        lib = ctypes.CDLL(self.path)
+        vp, i, d, u = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_uint
+        lib.vla_oracle_backward.restype = i
+        lib.vla_oracle_backward.argtypes = [vp, vp, vp, vp, i, d, i, i, i, i, i, vp, vp, vp, u, d,
+                                            vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, vp]
+        self._lib = lib
+
+    def backward(self, q, k, v, lam, d_out, *, u=None, in_dtype=F64, S0=None, A0=None, z0=None,
+                 dS_T=None, dA_T=None, dz_T=None, flags=0, eps=1e-4, n_threads=1,
+                 refresh=None) -> OracleGrads:
+        """Gradients for ``q,k[,u]: [B,H,T,d_k]``, ``v, d_out: [B,H,T,d_v]``."""
+        B, H, T, dk = np.shape(q)
+        dv = np.shape(v)[-1]
+        q = _in(q, in_dtype, (B, H, T, dk))
+        k = _in(k, in_dtype, (B, H, T, dk))
+        v = _in(v, in_dtype, (B, H, T, dv))
+        u = None if u is None else _in(u, in_dtype, (B, H, T, dk))
+        S0 = _opt64(S0, (B, H, dv, dk)); A0 = _opt64(A0, (B, H, dk, dk)); z0 = _opt64(z0, (B, H, dk))
+        d_out = _opt64(d_out, (B, H, T, dv))
+        dS_T = _opt64(dS_T, (B, H, dv, dk)); dA_T = _opt64(dA_T, (B, H, dk, dk))
+        dz_T = _opt64(dz_T, (B, H, dk))
+        dq = np.zeros((B, H, T, dk)); dkk = np.zeros((B, H, T, dk)); dvv = np.zeros((B, H, T, dv))
+        du = None if u is None else np.zeros((B, H, T, dk))
+        dS0 = np.zeros((B, H, dv, dk)); dA0 = np.zeros((B, H, dk, dk)); dz0 = np.zeros((B, H, dk))
+        rc = self._lib.vla_oracle_backward(
+            _ptr(q), _ptr(k), _ptr(v), _ptr(u), in_dtype, float(lam), B, H, T, dk, dv,
+            _ptr(S0), _ptr(A0), _ptr(z0), flags, float(eps), _ptr(d_out), _ptr(dS_T), _ptr(dA_T),
+            _ptr(dz_T), _ptr(dq), _ptr(dkk), _ptr(dvv), _ptr(du), _ptr(dS0), _ptr(dA0), _ptr(dz0),
+            int(n_threads), _refresh_arg(refresh))
+        if rc != 0:
+            raise ValueError("vla_oracle_backward: invalid argument")
+        return OracleGrads(dq, dkk, dvv, du, dS0, dA0, dz0)
+
+
+_default_bwd = None
+
+
+def load_bwd() -> OracleBwdLib:
+    global _default_bwd
+    with _lock:
+        if _default_bwd is None:
+            _default_bwd = OracleBwdLib()
+        return _default_bwd
+
+
+def backward(*args, **kwargs) -> OracleGrads:
+    return load_bwd().backward(*args, **kwargs)

@@ -188,6 +188,32 @@ int vla_seqpar_segments(int B, int H, int T, int d_k, int qkv_dtype);
 size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
 
 /*
+ * vla_backward -- gradients of the forward scan (first correct path: a token kernel).  The
+ * paper gives no backward algorithm; this is reverse-mode differentiation of exactly the
+ * recurrence vla_forward computes (Algorithm 1 without projections; Eqs. "sm", "s-update",
+ * "output"), the gradients its Corollary on gradient flow (Section 4) is about.
+ *
+ * Inputs as vla_forward (q, k, v, lambda_, S0, A0, opts->z0, opts->flags, opts->eps,
+ * opts->qkv_dtype) plus the incoming gradients d_out [B,H,T,d_v] and, optionally, dS_T, dA_T
+ * [B,H,d,d], dz_T [B,H,d_k] (NULL = zero); all gradients are fp32.  Outputs dq, dk [B,H,T,d_k],
+ * dv [B,H,T,d_v] and, when non-NULL, dS0, dA0, dz0.  The forward is recomputed inside; no
+ * state of the forward call is needed.  In identity-map mode z_T = z0, so dz0 = dz_T.
+ *
+ * Covered: u = k_hat (opts->u must be NULL), no periodic refresh, d_k = d_v in {16, 32, 64};
+ * anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a DEVICE buffer of at least
+ * vla_backward_workspace_bytes(B, H, T, d_k) bytes (z_t, e_t and delta_t of every token),
+ * owned by the caller and free for reuse once the work enqueued on `stream` has completed.
+ */
+int vla_backward(const void* q, const void* k, const void* v, float lambda_,
+                 int B, int H, int T, int d_k, int d_v,
+                 const float* S0, const float* A0,
+                 const float* d_out, const float* dS_T, const float* dA_T, const float* dz_T,
+                 float* dq, float* dk, float* dv, float* dS0, float* dA0, float* dz0,
+                 const vla_opts_t* opts, void* workspace, size_t workspace_bytes, void* stream);
+
+size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k);
+
+/*
  * vla_probe_fp32_fma -- measurement helper (the paper has no counterpart): enqueues a
  * register-only loop of fp32 FMAs on every SM (2048 threads per SM, 16 independent chains per
  * thread, `iters` x 128 FMAs per thread) and reports the floating-point operations launched in

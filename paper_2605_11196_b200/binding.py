@@ -10,7 +10,7 @@ import ctypes
 import os
 import threading
 from dataclasses import dataclass
-from typing import Optional
+from typing import NamedTuple, Optional
 
 import torch
 
@@ -26,7 +26,7 @@ VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK, VLA_KERNEL_DECODE = 0, 1, 2
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",
            "vla_forward_seqpar", "vla_seqpar_segments", "vla_seqpar_workspace_bytes",
-           "vla_probe_fp32_fma",
+           "vla_probe_fp32_fma", "vla_backward", "vla_backward_workspace_bytes",
            "vla_query_support", "vla_status_string", "vla_version")
 
 
@@ -81,6 +81,10 @@ def load_library():
             lib.vla_seqpar_segments.argtypes = [i, i, i, i, i]
             lib.vla_seqpar_workspace_bytes.restype = ctypes.c_size_t
             lib.vla_seqpar_workspace_bytes.argtypes = [i, i, i, i, i]
+            lib.vla_backward.restype = i
+            lib.vla_backward.argtypes = [vp, vp, vp, f, i, i, i, i, i] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
+            lib.vla_backward_workspace_bytes.restype = ctypes.c_size_t
+            lib.vla_backward_workspace_bytes.argtypes = [i, i, i, i]
             lib.vla_probe_fp32_fma.restype = i
             lib.vla_probe_fp32_fma.argtypes = [i, vp, ctypes.POINTER(ctypes.c_double), vp]
             lib.vla_host_workspace_bytes.restype = ctypes.c_size_t
@@ -202,6 +206,55 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
     if rc != VLA_OK:
         raise VlaError(rc, "vla_forward")
     return VlaResult(out, S_T, A_T, z_T, status)
+
+
+class VlaGrads(NamedTuple):
+    dq: torch.Tensor
+    dk: torch.Tensor
+    dv: torch.Tensor
+    dS0: torch.Tensor
+    dA0: torch.Tensor
+    dz0: torch.Tensor
+    status: Optional[torch.Tensor]
+
+
+def vla_backward(q, k, v, lam: float, d_out, *, S0=None, A0=None, z0=None, dS_T=None, dA_T=None,
+                 dz_T=None, flags: int = 0, eps: float = 1e-4, workspace=None, status=None,
+                 stream: Optional[torch.cuda.Stream] = None, want_status: bool = True) -> VlaGrads:
+    """Gradients of the forward scan for CUDA tensors (u = k_hat, d in {16, 32, 64}); the
+    forward is recomputed inside.  ``d_out`` is dL/d(out); ``dS_T, dA_T, dz_T`` default to zero."""
+    lib = load_library()
+    B, H, T, dk = q.shape
+    dv_ = v.shape[-1]
+    dt = _dtype_code(q)
+    dev = q.device
+    f32 = torch.float32
+    _chk(q, (B, H, T, dk), q.dtype, "q"); _chk(k, (B, H, T, dk), q.dtype, "k")
+    _chk(v, (B, H, T, dv_), q.dtype, "v"); _chk(d_out, (B, H, T, dv_), f32, "d_out")
+    _chk(S0, (B, H, dv_, dk), f32, "S0"); _chk(A0, (B, H, dk, dk), f32, "A0"); _chk(z0, (B, H, dk), f32, "z0")
+    _chk(dS_T, (B, H, dv_, dk), f32, "dS_T"); _chk(dA_T, (B, H, dk, dk), f32, "dA_T")
+    _chk(dz_T, (B, H, dk), f32, "dz_T")
+    dq = torch.empty((B, H, T, dk), dtype=f32, device=dev)
+    dkk = torch.empty((B, H, T, dk), dtype=f32, device=dev)
+    dvv = torch.empty((B, H, T, dv_), dtype=f32, device=dev)
+    dS0 = torch.empty((B, H, dv_, dk), dtype=f32, device=dev)
+    dA0 = torch.empty((B, H, dk, dk), dtype=f32, device=dev)
+    dz0 = torch.empty((B, H, dk), dtype=f32, device=dev)
+    if status is None and want_status:
+        status = torch.zeros((), dtype=torch.int32, device=dev)
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    need = int(lib.vla_backward_workspace_bytes(B, H, T, dk))
+    if workspace is None:
+        workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
+    opts = _make_opts(dt, None, flags, eps, z0, None, status, VLA_KERNEL_AUTO, None)
+    with torch.cuda.device(dev):
+        rc = lib.vla_backward(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv_, _ptr(S0), _ptr(A0),
+                              _ptr(d_out), _ptr(dS_T), _ptr(dA_T), _ptr(dz_T), _ptr(dq), _ptr(dkk),
+                              _ptr(dvv), _ptr(dS0), _ptr(dA0), _ptr(dz0), ctypes.byref(opts),
+                              _ptr(workspace), workspace.numel(), ctypes.c_void_p(st.cuda_stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_backward")
+    return VlaGrads(dq, dkk, dvv, dS0, dA0, dz0, status)
 
 
 def measure_fp32_fma_tflops(device=None, iters: int = 4096, reps: int = 5) -> float:

@@ -9,6 +9,7 @@
 
 #include "vla.h"
 #include "vla_launch.h"
+#include "vla_backward_params.h"
 
 namespace {
 
@@ -438,6 +439,45 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
                        : vla::launch_chunk(d_k, o.qkv_dtype, p, st);
   if (rc != VLA_OK) return rc;
   return vla::seqpar_after_scan(d_k, sp, A_T, o.zT, AT2, zT2, st);
+}
+
+size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k) {
+  if (B < 0 || H < 0 || T < 0 || d_k <= 0) return 0;
+  const size_t units = size_t(B) * size_t(H);
+  return 2 * round256(units * T * d_k * sizeof(float)) + round256(units * T * sizeof(float)) + 256;
+}
+
+int vla_backward(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,
+                 int d_k, int d_v, const float* S0, const float* A0, const float* d_out,
+                 const float* dS_T, const float* dA_T, const float* dz_T, float* dq, float* dk,
+                 float* dv, float* dS0, float* dA0, float* dz0, const vla_opts_t* opts,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+  vla_opts_t o;
+  int rc = resolve_opts(opts, &o);
+  if (rc != VLA_OK) return rc;
+  rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, d_out);
+  if (rc != VLA_OK) return rc;
+  if (o.u || o.refresh_period > 0 || d_k > 64) return VLA_ERR_UNSUPPORTED;
+  const int units = B * H;
+  if (units > 0 && T > 0 && (!dq || !dk || !dv)) return VLA_ERR_INVALID_ARG;
+  const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0};
+  for (const void* ptr : ptrs)
+    if (!aligned16(ptr)) return VLA_ERR_ALIGNMENT;
+  if (o.status && (reinterpret_cast<uintptr_t>(o.status) & 3u)) return VLA_ERR_ALIGNMENT;
+  if (units == 0) return VLA_OK;
+  if (!workspace || workspace_bytes < vla_backward_workspace_bytes(B, H, T, d_k)) return VLA_ERR_INVALID_ARG;
+  unsigned char* w = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(workspace) + 255) & ~uintptr_t(255));
+  const size_t vec_bytes = round256(size_t(units) * T * d_k * sizeof(float));
+  vla::BackwardParams p;
+  p.q = q; p.k = k; p.v = v; p.S0 = S0; p.A0 = A0; p.z0 = o.z0;
+  p.d_out = d_out; p.dS_T = dS_T; p.dA_T = dA_T; p.dz_T = dz_T;
+  p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;
+  p.zst = reinterpret_cast<float*>(w);
+  p.est = reinterpret_cast<float*>(w + vec_bytes);
+  p.dst = reinterpret_cast<float*>(w + 2 * vec_bytes);
+  p.status = o.status; p.lambda = lambda_; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;
+  return vla::launch_backward(d_k, o.qkv_dtype, p, static_cast<cudaStream_t>(stream));
 }
 
 int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream) {

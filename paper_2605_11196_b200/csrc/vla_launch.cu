@@ -2,6 +2,7 @@
 // kernel's launchers, and the helper launches of the sequence-parallel path.
 #include "vla.h"
 #include "vla_launch.h"
+#include "vla_backward.cuh"
 #include "vla_decode.cuh"
 #include "vla_scan_token.cuh"
 #include "vla_seqpar.cuh"
@@ -126,6 +127,27 @@ int launch_fp32_probe(int iters, float* sink, double* flops, cudaStream_t st) {
   const int grid = 2 * sms, block = 1024;
   fp32_fma_probe_kernel<<<grid, block, 0, st>>>(sink, iters);
   if (flops) *flops = 2.0 * 16.0 * 8.0 * double(iters) * double(grid) * double(block);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------- backward (token kernel)
+int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st) {
+  const bool f32 = dtype == VLA_F32;
+  switch (d) {
+    case 16:
+      if (f32) vla_backward_token_kernel<16, float><<<p.units, 256, 0, st>>>(p);
+      else vla_backward_token_kernel<16, uint16_t><<<p.units, 256, 0, st>>>(p);
+      break;
+    case 32:
+      if (f32) vla_backward_token_kernel<32, float><<<p.units, 256, 0, st>>>(p);
+      else vla_backward_token_kernel<32, uint16_t><<<p.units, 256, 0, st>>>(p);
+      break;
+    case 64:
+      if (f32) vla_backward_token_kernel<64, float><<<p.units, 256, 0, st>>>(p);
+      else vla_backward_token_kernel<64, uint16_t><<<p.units, 256, 0, st>>>(p);
+      break;
+    default: return VLA_ERR_UNSUPPORTED;
+  }
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

@@ -9,6 +9,10 @@
 #include "vla_seqpar_params.h"
 
 namespace vla {
+struct BackwardParams;
+}
+
+namespace vla {
 
 // Token kernel, d in {16, 32, 64, 128}.  Returns a vla_status_t.
 int launch_token(int d, int dtype, const ScanParams& p, cudaStream_t st);
@@ -30,6 +34,9 @@ int chunk_resident_ctas(int d, int dtype, bool tri);
 int seqpar_before_scan(int d, int dtype, const SeqParParams& sp, cudaStream_t st);
 int seqpar_after_scan(int d, const SeqParParams& sp, float* A_T, float* zT, const float* AT2,
                       const float* zT2, cudaStream_t st);
+
+// Backward pass, token kernel, d in {16, 32, 64}, u = k_hat.
+int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st);
 
 // Register-only fp32 FMA loop over the whole device (measurement helper); *flops = work launched.
 int launch_fp32_probe(int iters, float* sink, double* flops, cudaStream_t st);

@@ -1,0 +1,100 @@
+"""Backward kernel (vla_backward) against the fp64 backward oracle, which is itself pinned by
+finite differences of the forward oracle (tests/test_oracle_bwd_pins.py)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_11196_b200 as vla
+from paper_2605_11196_b200 import workloads as W
+from parity_util import NTHREADS, rel_err, to_oracle_array
+
+pytestmark = pytest.mark.gpu
+IDENT = vla.VLA_FLAG_IDENTITY_MAP
+
+
+def _small(d, T, dtype, units=(1, 2), seed=1):
+    return W.Workload("t", units[0], units[1], d, T, dtype, seed)
+
+
+def _run_both(q, k, v, lam, d_out, flags=0, S0=None, A0=None, z0=None, dS_T=None, dA_T=None, dz_T=None):
+    dev = torch.device("cuda:0")
+    mv = lambda x: None if x is None else x.to(dev).contiguous()
+    g = vla.vla_backward(mv(q), mv(k), mv(v), lam, mv(d_out), S0=mv(S0), A0=mv(A0), z0=mv(z0),
+                         dS_T=mv(dS_T), dA_T=mv(dA_T), dz_T=mv(dz_T), flags=flags)
+    torch.cuda.synchronize()
+    assert int(g.status.item()) == 0
+    qa, dt = to_oracle_array(q)
+    ka, _ = to_oracle_array(k)
+    va, _ = to_oracle_array(v)
+    f64 = lambda x: None if x is None else x.detach().cpu().double().numpy()
+    ref = oracle.backward(qa, ka, va, lam, f64(d_out), in_dtype=dt, S0=f64(S0), A0=f64(A0), z0=f64(z0),
+                          dS_T=f64(dS_T), dA_T=f64(dA_T), dz_T=f64(dz_T), flags=flags, n_threads=NTHREADS)
+    return g, ref
+
+
+def _err(x_gpu, x_ref):
+    """max|x - ref| / max|ref|, with a floor on the denominator: a gradient that is exactly
+    zero in exact arithmetic (dq of a single token written into an empty memory) comes out as
+    rounding noise on both sides."""
+    x = x_gpu.detach().cpu().double().numpy()
+    assert x.shape == x_ref.shape and np.all(np.isfinite(x))
+    return float(np.abs(x - x_ref).max() / max(np.abs(x_ref).max(), 1e-3)) if x_ref.size else 0.0
+
+
+def _check(g, ref, tol, label):
+    errs = {"dq": _err(g.dq, ref.dq), "dk": _err(g.dk, ref.dk), "dv": _err(g.dv, ref.dv),
+            "dS0": _err(g.dS0, ref.dS0), "dA0": _err(g.dA0, ref.dA0), "dz0": _err(g.dz0, ref.dz0)}
+    for name, e in errs.items():
+        assert e <= tol, "%s %s: rel err %.3e > %.1e (%s)" % (label, name, e, tol, errs)
+    return errs
+
+
+@pytest.mark.parametrize("d", [16, 32, 64])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+@pytest.mark.parametrize("T", [1, 7, 64, 200])
+def test_gradients_agree_with_the_backward_oracle(d, dtype, flags, T):
+    w = _small(d, T, dtype, units=(2, 3), seed=3000 + d + T)
+    q, k, v = W.make_inputs(w)
+    g = torch.Generator().manual_seed(d * 7 + T)
+    d_out = torch.randn((2, 3, T, d), generator=g)
+    for lam in (1.0, 0.1):
+        got, ref = _run_both(q, k, v, lam, d_out, flags=flags)
+        _check(got, ref, 2e-4, "backward d=%d T=%d lam=%g" % (d, T, lam))
+
+
+@pytest.mark.parametrize("d", [32, 64])
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_carried_states_and_incoming_state_gradients(d, flags):
+    w = _small(d, 96, "f32", units=(1, 4), seed=3100 + d)
+    q, k, v = W.make_inputs(w)
+    g = torch.Generator().manual_seed(d)
+    shape = (1, 4)
+    S0 = torch.randn(shape + (d, d), generator=g) * 0.2
+    h = torch.randn(shape + (d, d), generator=g) * 0.1
+    A0 = h @ h.transpose(-1, -2) + 0.5 * torch.eye(d)
+    z0 = torch.rand(shape + (d,), generator=g) + 0.1
+    d_out = torch.randn(shape + (96, d), generator=g)
+    dS_T = torch.randn(shape + (d, d), generator=g)
+    dA_T = torch.randn(shape + (d, d), generator=g)
+    dz_T = torch.randn(shape + (d,), generator=g)
+    got, ref = _run_both(q, k, v, 0.5, d_out, flags=flags, S0=S0, A0=A0, z0=z0, dS_T=dS_T, dA_T=dA_T, dz_T=dz_T)
+    _check(got, ref, 2e-4, "backward carried d=%d" % d)
+
+
+def test_mid_workload_gradients_and_what_is_not_covered():
+    """The `mid` workload (32 units, d = 64, T = 4096) whole, and the shapes the first backward
+    kernel does not take."""
+    w = W.WORKLOADS["mid"]
+    q, k, v = W.make_inputs(w)
+    g = torch.Generator().manual_seed(11)
+    d_out = torch.randn((w.B, w.H, w.T, w.d), generator=g)
+    got, ref = _run_both(q, k, v, w.lam, d_out)
+    print("mid backward", _check(got, ref, 1e-3, "backward mid"))
+    dev = torch.device("cuda:0")
+    w128 = _small(128, 16, "f32")
+    q, k, v = [x.to(dev) for x in W.make_inputs(w128)]
+    with pytest.raises(vla.VlaError) as ei:
+        vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 16, 128), device=dev))
+    assert ei.value.code == vla.VLA_ERR_UNSUPPORTED

@@ -396,6 +396,25 @@ def main():
                          "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
                          "hbm_frac": alg_bytes_per_token(ww.d, ib) * ww.tokens / (ms * 1e-3) / 1e9 / hbm_peak,
                          "units": ww.units, "unit_limited_frac_bound": min(ww.units, n_sm) / n_sm}
+            # backward pass (first correct path: token kernel, d <= 64): forward recomputed inside
+            if ww.d <= 64 and name in ("mid", "recall"):
+                qd3, kd3, vd3 = q2.to(dev), k2.to(dev), v2.to(dev)
+                go3 = torch.randn((ww.B, ww.H, ww.T, ww.d), device=dev)
+                bcall = lambda: vla.vla_backward(qd3, kd3, vd3, ww.lam, go3, stream=stream)
+                ms = []
+                with torch.cuda.stream(stream):
+                    bcall()
+                    for _ in range(3):
+                        fl.fill_(1)
+                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a.record(stream); bcall(); b.record(stream)
+                        ms.append((a, b))
+                torch.cuda.synchronize(dev)
+                ms = float(np.median([a.elapsed_time(b) for a, b in ms]))
+                per[name + "_backward"] = {"ms": ms, "tokens_per_s": ww.tokens / (ms * 1e-3),
+                                           "ns_per_scan_step": 1e6 * ms / ww.T,
+                                           "kernel": "vla_backward_token_kernel (forward + reverse sweep)"}
+                del qd3, kd3, vd3, go3
             # fewer units than SMs: the sequence-parallel entry point cuts each sequence into
             # segments that are scanned concurrently (twice the arithmetic, P times the CTAs)
             P = vla.seqpar_segments(ww.B, ww.H, ww.T, ww.d, q2.dtype)

@@ -96,6 +96,20 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
   };
 
   // ================================================================ forward sweep
+  // warp 0 reads the rows of token t + 1 from global memory while token t is processed
+  float nxk[EPL], nxv[EPL];
+  auto fetch_kv = [&](int t) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      const int c = e * 32 + lane;
+      nxk[e] = 0.f; nxv[e] = 0.f;
+      if (c < D && t < T) {
+        nxk[e] = load1<TIn>(gk, size_t(t) * D + c);
+        nxv[e] = load1<TIn>(gv, size_t(t) * D + c);
+      }
+    }
+  };
+  if (warp == 0) fetch_kv(0);
   for (int t = 0; t < T; ++t) {
     if (warp == 0) {
       float kx[EPL];
@@ -105,13 +119,14 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
         const int c = e * 32 + lane;
         float x = 0.f;
         if (c < D) {
-          x = load1<TIn>(gk, size_t(t) * D + c);
+          x = nxk[e];
           if (!ident) x = bwd_phi(x);
-          vv[c] = load1<TIn>(gv, size_t(t) * D + c);
+          vv[c] = nxv[e];
         }
         kx[e] = x;
         ss = fmaf(x, x, ss);
       }
+      fetch_kv(t + 1);
       ss = warp_sum(ss);
       const float inv = 1.0f / fmaxf(sqrtf(ss), eps);
 #pragma unroll
@@ -178,8 +193,28 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
   // ================================================================ reverse sweep
   // warp 0's per-token vector work is written as two lambdas: `open` prepares token t,
   // `close` finishes it (and is followed at once by `open` of token t - 1)
-  auto open_token = [&](int t) {
-    const float delta = dst[t];
+  // rows of the token that warp 0 opens next, read from global memory one token ahead
+  float pk[EPL], pq[EPL], pz[EPL], pe[EPL], pg[EPL];
+  float pdelta = 1.0f;
+  auto fetch_token = [&](int t) {
+    if (t < 0) return;
+    pdelta = dst[t];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      const int c = e * 32 + lane;
+      pk[e] = pq[e] = pz[e] = pe[e] = pg[e] = 0.f;
+      if (c < D) {
+        pk[e] = load1<TIn>(gk, size_t(t) * D + c);
+        pq[e] = load1<TIn>(gq, size_t(t) * D + c);
+        pz[e] = zst[size_t(t) * D + c];
+        pe[e] = est[size_t(t) * D + c];
+        pg[e] = gdo[size_t(t) * D + c];
+      }
+    }
+  };
+  float rawk[EPL], rawq[EPL];   // raw k, q of the open token (for phi')
+  auto open_token = [&](int) {
+    const float delta = pdelta;
     float zx[EPL], kx[EPL], qx[EPL];
     float ss = 0.f, zz = 0.f;
 #pragma unroll
@@ -187,12 +222,12 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
       const int c = e * 32 + lane;
       float kk = 0.f, qq = 0.f, z = 0.f;
       if (c < D) {
-        kk = load1<TIn>(gk, size_t(t) * D + c);
-        qq = load1<TIn>(gq, size_t(t) * D + c);
+        rawk[e] = pk[e]; rawq[e] = pq[e];
+        kk = pk[e]; qq = pq[e];
         if (!ident) { kk = bwd_phi(kk); qq = bwd_phi(qq); }
-        z = zst[size_t(t) * D + c];
-        go[c] = gdo[size_t(t) * D + c];
-        et[c] = est[size_t(t) * D + c];
+        z = pz[e];
+        go[c] = pg[e];
+        et[c] = pe[e];
         zt[c] = z;
         kf[c] = kk;
         qf[c] = qq;
@@ -232,10 +267,14 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
     }
   };
 
-  if (warp == 0 && T > 0) open_token(T - 1);
+  if (warp == 0 && T > 0) {
+    fetch_token(T - 1);
+    open_token(T - 1);
+  }
   __syncthreads();
 
   for (int t = T - 1; t >= 0; --t) {
+    if (warp == 0) fetch_token(t - 1);   // in flight while this token is worked on
     // ---- P1: y = S' qf, g1 = GS alpha, gaz = GA z
     {
       float a0[R], a1[R], a2[R];
@@ -435,9 +474,8 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
             gz[c] += dden * qf[c];
             dkf += gz[c];
             zk[c] -= kf[c];
-            const float kraw = load1<TIn>(gk, size_t(t) * D + c), qraw = load1<TIn>(gq, size_t(t) * D + c);
-            dkf *= bwd_dphi(kraw);
-            dq *= bwd_dphi(qraw);
+            dkf *= bwd_dphi(rawk[e]);
+            dq *= bwd_dphi(rawq[e]);
           }
           p.dk[(size_t(unit) * T + t) * D + c] = dkf;
           p.dq[(size_t(unit) * T + t) * D + c] = dq;

@@ -21,8 +21,9 @@
 // Products with a matrix are row dots (reduced over the 16 threads of a row block with
 // shuffles) or column sums (reduced over the 16 row blocks through shared memory); the
 // corrections for updates not yet applied (GS += dy qf^T and so on) are scalar multiples of
-// known vectors, so all four column sums of a token share one reduction.  Vector arithmetic is
-// done by warp 0; six CTA barriers per token.
+// known vectors, so all four column sums of a token share one reduction.  Three tokens are in
+// flight: while warp 0 does the vector arithmetic of token t, warp 1 prepares the inputs of
+// token t - 1 and warp 2 writes dk, dq of token t + 1; four CTA barriers per token.
 #pragma once
 
 #include "vla_backward_params.h"
@@ -45,16 +46,19 @@ template <int D, typename TIn>
 __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardParams p) {
   constexpr int R = D / 16;                      // block edge per thread
   constexpr int EPL = D >= 32 ? D / 32 : 1;      // vector elements per lane of warp 0
-  __shared__ __align__(16) float vec[24][D];     // named rows below
+  __shared__ __align__(16) float vec[14][D];     // named rows below
+  __shared__ float ctx[3][8][D];                 // per-token vectors, ring of three tokens
+  __shared__ float cscl[3][8];                   // per-token scalars
+  __shared__ float res[2][4][D];                 // dk_hat (S part), dqf, A' da, A' dz by token parity
+  __shared__ float rscl[2][4];                   // ddelta, z.dz, dden by token parity
   __shared__ float part[8][4][D];                // column-sum partials per warp
-  __shared__ float scal[16];
-  float* kf = vec[0];   float* kh = vec[1];   float* qf = vec[2];   float* go = vec[3];
-  float* zt = vec[4];   float* et = vec[5];   float* al = vec[6];   float* vv = vec[7];
-  float* yv = vec[8];   float* g1 = vec[9];   float* gaz = vec[10]; float* pv = vec[11];
-  float* cs = vec[12];  // rows 12..15: the four column sums
-  float* dav = vec[16]; float* dzv = vec[17]; float* dqf = vec[18]; float* dkS = vec[19];
-  float* r1 = vec[20];  float* r3 = vec[21];  float* zk = vec[22];  float* gz = vec[23];
-  enum { kDen = 0, kQal, kDelta, kDdelta, kZdz, kNa, kNk, kDenLive, kSc, kDdenVal };
+  float* kh = vec[0];   float* vv = vec[1];   float* zt = vec[2];   float* pv = vec[3];   // forward sweep
+  float* yv = vec[4];   float* g1 = vec[5];   float* gaz = vec[6];
+  float* cs = vec[7];   // rows 7..10: the four column sums
+  float* dav = vec[11]; float* dzv = vec[12];
+  float* zk = vec[13];  // key sum after the forward sweep
+  __shared__ float gzbuf[D];
+  float* gz = gzbuf;    // dL/d(key sum), carried by the closing warp
 
   const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ty = tid >> 4, tx = tid & 15;
@@ -191,9 +195,19 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
   }
 
   // ================================================================ reverse sweep
-  // warp 0's per-token vector work is written as two lambdas: `open` prepares token t,
-  // `close` finishes it (and is followed at once by `open` of token t - 1)
-  // rows of the token that warp 0 opens next, read from global memory one token ahead
+  // Three tokens are alive at a time, each in its own context (ring of three):
+  //   token t     : the matrix work of this iteration (row dots, column sums, warp 0's vectors)
+  //   token t - 1 : being opened by warp 1 (its inputs, alpha, denominator: nothing of this
+  //                 depends on the adjoints)
+  //   token t + 1 : being closed by warp 2 (dk, dq from the finished row dots)
+  // so that only warp 0's vector arithmetic of token t sits between the CTA barriers.
+  auto cvec = [&](int t, int which) { return ctx[((t % 3) + 3) % 3][which]; };
+  auto cscal = [&](int t) { return cscl[((t % 3) + 3) % 3]; };
+  enum { cKf = 0, cKh, cQf, cGo, cZt, cEt, cAl, cZk };
+  enum { sDen = 0, sDenLive, sQal, sDelta, sNa, sNk };
+  enum { rDdelta = 0, rZdz, rDden };
+
+  // rows of the token that warp 1 opens next, read from global memory one iteration ahead
   float pk[EPL], pq[EPL], pz[EPL], pe[EPL], pg[EPL];
   float pdelta = 1.0f;
   auto fetch_token = [&](int t) {
@@ -212,8 +226,14 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
       }
     }
   };
-  float rawk[EPL], rawq[EPL];   // raw k, q of the open token (for phi')
-  auto open_token = [&](int) {
+  // one warp: context of token t from the fetched rows; zk_src = key sum INCLUDING token t
+  // (for t = T - 1 the forward sweep's result, else the context of t + 1 minus its phi(k))
+  auto open_token = [&](int t, bool last) {
+    float* okf = cvec(t, cKf); float* okh = cvec(t, cKh); float* oqf = cvec(t, cQf);
+    float* ogo = cvec(t, cGo); float* ozt = cvec(t, cZt); float* oet = cvec(t, cEt);
+    float* oal = cvec(t, cAl); float* ozk = cvec(t, cZk);
+    const float* nzk = last ? zk : cvec(t + 1, cZk);
+    const float* nkf = cvec(t + 1, cKf);
     const float delta = pdelta;
     float zx[EPL], kx[EPL], qx[EPL];
     float ss = 0.f, zz = 0.f;
@@ -222,15 +242,14 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
       const int c = e * 32 + lane;
       float kk = 0.f, qq = 0.f, z = 0.f;
       if (c < D) {
-        rawk[e] = pk[e]; rawq[e] = pq[e];
         kk = pk[e]; qq = pq[e];
         if (!ident) { kk = bwd_phi(kk); qq = bwd_phi(qq); }
         z = pz[e];
-        go[c] = pg[e];
-        et[c] = pe[e];
-        zt[c] = z;
-        kf[c] = kk;
-        qf[c] = qq;
+        ogo[c] = pg[e];
+        oet[c] = pe[e];
+        ozt[c] = z;
+        okf[c] = kk;
+        oqf[c] = qq;
       }
       kx[e] = kk; qx[e] = qq; zx[e] = z;
       ss = fmaf(kk, kk, ss);
@@ -243,40 +262,122 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
     const float na_raw = sqrtf(zz) * idl;          // ||a||, a = z / delta
     const float sc = idl / fmaxf(na_raw, eps);
     float dn = 0.f, qa = 0.f;
-    __syncwarp();
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
       const int c = e * 32 + lane;
       if (c < D) {
-        kh[c] = kx[e] / nk;
-        al[c] = sc * zx[e];
-        dn = fmaf(zk[c], qx[e], dn);
+        okh[c] = kx[e] / nk;
+        oal[c] = sc * zx[e];
+        const float zkc = last ? nzk[c] : (ident ? nzk[c] : nzk[c] - nkf[c]);
+        ozk[c] = zkc;
+        dn = fmaf(zkc, qx[e], dn);
         qa = fmaf(qx[e], sc * zx[e], qa);
       }
     }
     dn = warp_sum(dn);
     qa = warp_sum(qa);
     if (lane == 0) {
-      scal[kDen] = ident ? 1.0f : fmaxf(dn, eps);
-      scal[kDenLive] = (ident || dn < eps) ? 0.0f : 1.0f;   // 1: the denominator is live
-      scal[kQal] = qa;
-      scal[kDelta] = delta;
-      scal[kNa] = na_raw;
-      scal[kNk] = sqrtf(ss);
-      scal[kSc] = sc;
+      float* os = cscal(t);
+      os[sDen] = ident ? 1.0f : fmaxf(dn, eps);
+      os[sDenLive] = (ident || dn < eps) ? 0.0f : 1.0f;
+      os[sQal] = qa;
+      os[sDelta] = delta;
+      os[sNa] = na_raw;
+      os[sNk] = sqrtf(ss);
+    }
+  };
+  // one warp: dk, dq of token t from its finished products
+  auto close_token = [&](int t) {
+    const int par = t & 1;
+    const float* ckf = cvec(t, cKf); const float* ckh = cvec(t, cKh); const float* cqf = cvec(t, cQf);
+    const float* czt = cvec(t, cZt);
+    const float* cdkS = res[par][0]; const float* cdqf = res[par][1];
+    const float* cr1 = res[par][2]; const float* cr3 = res[par][3];
+    const float ddelta = rscl[par][rDdelta], zdz = rscl[par][rZdz], dden = rscl[par][rDden];
+    const float delta = cscal(t)[sDelta], nkraw = cscal(t)[sNk];
+    const float nk = fmaxf(nkraw, eps);
+    float dkhx[EPL];
+    float kd = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      const int c = e * 32 + lane;
+      dkhx[e] = 0.f;
+      if (c < D) {
+        const float du = ddelta * czt[c] + cr3[c] + czt[c] * (zdz / delta);   // ddelta z + A dz
+        dkhx[e] = cdkS[c] + cr1[c] + du;
+        kd = fmaf(ckh[c], dkhx[e], kd);
+      }
+    }
+    kd = warp_sum(kd);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      const int c = e * 32 + lane;
+      if (c < D) {
+        float dkf = nkraw > eps ? (dkhx[e] - ckh[c] * kd) / nk : dkhx[e] / eps;
+        float dq = cdqf[c];
+        if (!ident) {
+          gz[c] += dden * cqf[c];
+          dkf += gz[c];
+          // phi'(x) from phi(x): 1 where phi > 1 (x > 0), phi itself otherwise (exp(x))
+          dkf *= ckf[c] > 1.0f ? 1.0f : ckf[c];
+          dq *= cqf[c] > 1.0f ? 1.0f : cqf[c];
+        }
+        p.dk[(size_t(unit) * T + t) * D + c] = dkf;
+        p.dq[(size_t(unit) * T + t) * D + c] = dq;
+      }
     }
   };
 
-  if (warp == 0 && T > 0) {
-    fetch_token(T - 1);
-    open_token(T - 1);
+  if (T > 0) {
+    if (warp == 1) {
+      fetch_token(T - 1);
+      open_token(T - 1, true);
+      fetch_token(T - 2);
+    }
+    __syncthreads();
   }
-  __syncthreads();
 
-  for (int t = T - 1; t >= 0; --t) {
-    if (warp == 0) fetch_token(t - 1);   // in flight while this token is worked on
-    // ---- P1: y = S' qf, g1 = GS alpha, gaz = GA z
-    {
+  float dyr[R], der[R];     // dy and de of the token in flight, rows of this thread
+  for (int t = T - 1; t >= -1; --t) {
+    // ---- phase A: finish token t + 1 (row dots A' da, A' dz; the four rank-1 updates), then
+    //      the three row dots of token t
+    if (t + 1 <= T - 1) {
+      const int tp = t + 1, par = tp & 1;
+      const float* kh = cvec(tp, cKh); const float* qf = cvec(tp, cQf); const float* zt = cvec(tp, cZt);
+      const float* et = cvec(tp, cEt); const float* al = cvec(tp, cAl);
+      const float delta = cscal(tp)[sDelta];
+      float b0[R], b1[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        float x0 = 0.f, x1 = 0.f;
+#pragma unroll
+        for (int c = 0; c < R; ++c) {
+          x0 = fmaf(A[r][c], dav[col0 + c], x0);
+          x1 = fmaf(A[r][c], dzv[col0 + c], x1);
+        }
+        b0[r] = reduce16(x0); b1[r] = reduce16(x1);
+      }
+      if (tx == 0) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) { res[par][2][row0 + r] = b0[r]; res[par][3][row0 + r] = b1[r]; }
+      }
+      const float idl = 1.0f / delta;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float er = et[row0 + r], zr = zt[row0 + r], dadz = dav[row0 + r] + dzv[row0 + r];
+#pragma unroll
+        for (int c = 0; c < R; ++c) {
+          const float khc = kh[col0 + c];
+          GS[r][c] = fmaf(dyr[r], qf[col0 + c], GS[r][c]);
+          GS[r][c] = fmaf(-der[r], khc, GS[r][c]);
+          S[r][c] = fmaf(-er, al[col0 + c], S[r][c]);
+          GA[r][c] = fmaf(dadz, khc, GA[r][c]);
+          A[r][c] = fmaf(zr * idl, zt[col0 + c], A[r][c]);
+        }
+      }
+    }
+    if (t >= 0) {
+      const float* qf = cvec(t, cQf); const float* zt = cvec(t, cZt); const float* al = cvec(t, cAl);
       float a0[R], a1[R], a2[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
@@ -295,9 +396,15 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
       }
     }
     __syncthreads();
-    // ---- P2: column sums S'^T dy, GS^T e, S'^T de, GA^T z (partials per warp)
-    const float den = scal[kDen], qal = scal[kQal], delta = scal[kDelta];
-    float dyr[R], der[R];
+    if (t < 0) {   // epilogue: only token 0 is left to close
+      if (warp == 2 && T > 0) close_token(0);
+      break;
+    }
+    const float* kh = cvec(t, cKh); const float* qf = cvec(t, cQf); const float* go = cvec(t, cGo);
+    const float* zt = cvec(t, cZt); const float* et = cvec(t, cEt); const float* al = cvec(t, cAl);
+    const float* zkt = cvec(t, cZk);
+    const float den = cscal(t)[sDen], qal = cscal(t)[sQal], delta = cscal(t)[sDelta];
+    // ---- phase B: column sums S'^T dy, GS^T e, S'^T de, GA^T z (partials per warp)
     {
 #pragma unroll
       for (int r = 0; r < R; ++r) {
@@ -328,6 +435,7 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
       }
     }
     __syncthreads();
+    // ---- phase C: add the eight partials
     for (int j = tid; j < 4 * D; j += 256) {
       const int k2 = j / D, c = j % D;
       float s = 0.f;
@@ -336,10 +444,13 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
       cs[k2 * D + c] = s;
     }
     __syncthreads();
-    // ---- V: warp 0 forms da, dz, dqf, dk_hat (S part)
+    // ---- phase D: warp 0 forms da, dz, dqf, dk_hat (S part) of token t; warp 1 opens token
+    //      t - 1; warp 2 closes token t + 1
     if (warp == 0) {
-      const bool den_live = scal[kDenLive] != 0.0f;
-      const float na = scal[kNa];
+      const int par = t & 1;
+      float* dkS = res[par][0]; float* dqf = res[par][1];
+      const bool den_live = cscal(t)[sDenLive] != 0.0f;
+      const float na = cscal(t)[sNa];
       float odo = 0.f, ede = 0.f, dye = 0.f;
       float dex[EPL];
 #pragma unroll
@@ -363,7 +474,7 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
         const int c = e * 32 + lane;
         dalx[e] = 0.f;
         if (c < D) {
-          dqf[c] = cs[0 * D + c] + dden * zk[c];
+          dqf[c] = cs[0 * D + c] + dden * zkt[c];
           dalx[e] = cs[1 * D + c] + qf[c] * dye;               // (GS + dy qf^T)^T e
           dkS[c] = -(cs[2 * D + c] - al[c] * ede);             // -(S' - e alpha^T)^T de
           adal = fmaf(al[c], dalx[e], adal);
@@ -410,82 +521,18 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
         }
       }
       zdz = warp_sum(zdz);
-      if (lane == 0) { scal[kDdelta] = ddelta; scal[kZdz] = zdz; scal[kDdenVal] = dden; }
-    }
-    __syncthreads();
-    // ---- P5: r1 = A' da, r3 = A' dz, then the four rank-1 updates in registers
-    {
-      float b0[R], b1[R];
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        float x0 = 0.f, x1 = 0.f;
-#pragma unroll
-        for (int c = 0; c < R; ++c) {
-          x0 = fmaf(A[r][c], dav[col0 + c], x0);
-          x1 = fmaf(A[r][c], dzv[col0 + c], x1);
-        }
-        b0[r] = reduce16(x0); b1[r] = reduce16(x1);
+      if (lane == 0) { rscl[par][rDdelta] = ddelta; rscl[par][rZdz] = zdz; rscl[par][rDden] = dden; }
+    } else if (warp == 1) {
+      if (t >= 1) {
+        open_token(t - 1, false);
+        fetch_token(t - 2);
       }
-      if (tx == 0) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) { r1[row0 + r] = b0[r]; r3[row0 + r] = b1[r]; }
-      }
-      const float idl = 1.0f / delta;
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const float er = et[row0 + r], zr = zt[row0 + r], dadz = dav[row0 + r] + dzv[row0 + r];
-#pragma unroll
-        for (int c = 0; c < R; ++c) {
-          const float khc = kh[col0 + c];
-          GS[r][c] = fmaf(dyr[r], qf[col0 + c], GS[r][c]);
-          GS[r][c] = fmaf(-der[r], khc, GS[r][c]);
-          S[r][c] = fmaf(-er, al[col0 + c], S[r][c]);
-          GA[r][c] = fmaf(dadz, khc, GA[r][c]);
-          A[r][c] = fmaf(zr * idl, zt[col0 + c], A[r][c]);
-        }
-      }
-    }
-    __syncthreads();
-    // ---- close token t (warp 0), open token t - 1
-    if (warp == 0) {
-      const float ddelta = scal[kDdelta], zdz = scal[kZdz], dden = scal[kDdenVal];
-      const float nkraw = scal[kNk];
-      const float nk = fmaxf(nkraw, eps);
-      float dkhx[EPL];
-      float kd = 0.f;
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        const int c = e * 32 + lane;
-        dkhx[e] = 0.f;
-        if (c < D) {
-          const float du = ddelta * zt[c] + r3[c] + zt[c] * (zdz / delta);   // ddelta z + A dz
-          dkhx[e] = dkS[c] + r1[c] + du;
-          kd = fmaf(kh[c], dkhx[e], kd);
-        }
-      }
-      kd = warp_sum(kd);
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        const int c = e * 32 + lane;
-        if (c < D) {
-          float dkf = nkraw > eps ? (dkhx[e] - kh[c] * kd) / nk : dkhx[e] / eps;
-          float dq = dqf[c];
-          if (!ident) {
-            gz[c] += dden * qf[c];
-            dkf += gz[c];
-            zk[c] -= kf[c];
-            dkf *= bwd_dphi(rawk[e]);
-            dq *= bwd_dphi(rawq[e]);
-          }
-          p.dk[(size_t(unit) * T + t) * D + c] = dkf;
-          p.dq[(size_t(unit) * T + t) * D + c] = dq;
-        }
-      }
-      __syncwarp();
-      if (t > 0) open_token(t - 1);
+    } else if (warp == 2) {
+      if (t + 1 <= T - 1) close_token(t + 1);
     }
     __syncthreads();
   }
+  __syncthreads();
 
   // ---- gradients of the initial states
 #pragma unroll

@@ -194,6 +194,7 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
   p.refresh_period = o.refresh_period; p.refresh_eta = o.refresh_eta;
   p.step_offset = o.step_offset; p.u_is_khat = 0;
   p.n_main = 0; p.out2 = nullptr;
+  p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr;
   return launch(p, d_k, o.qkv_dtype, o.kernel, static_cast<cudaStream_t>(stream));
 }
 
@@ -432,6 +433,7 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   // d <= 64: N CTAs of three warp groups; d = 128: 2N CTAs, the transfer scans second
   p.T = T / P; p.units = seqpar_tri(d_k) ? N : 2 * N; p.n_main = N; p.flags = o.flags;
   p.refresh_period = 0; p.refresh_eta = 0.0f; p.step_offset = 0; p.u_is_khat = 0;
+  p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = vla::seqpar_before_scan(d_k, o.qkv_dtype, sp, st);
   if (rc != VLA_OK) return rc;

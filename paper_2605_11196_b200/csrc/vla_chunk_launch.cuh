@@ -49,6 +49,25 @@ int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
+// The forward of a backward pass: plain grid, u = k_hat, per-token z, e, delta left in global
+// memory (p.stash_*), readout optional.
+template <int D, typename TIn>
+int launch_chunk_stash_t(const ScanParams& p, cudaStream_t st) {
+  using Cfg = ChunkCfg<D, TIn, kUKhat>;
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, kUKhat, false, true>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  SchedParams sp;
+  sp.balanced = 0;
+  sp.grid = p.units;
+  sp.epoch = 0;
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
 template <int D, typename TIn>
 int launch_chunk_t(const ScanParams& p, cudaStream_t st) {
   if (p.u) return launch_chunk_um<D, TIn, kUTensor>(p, st);
@@ -124,4 +143,7 @@ int chunk_resident_t(bool tri) {
     return launch_chunk_tri_t<D, TIN>(p, st);                                                   \
   }                                                                                             \
   int chunk_resident_##TAG(bool tri) { return chunk_resident_t<D, TIN>(tri); }                  \
+  int launch_chunk_stash_##TAG(const ScanParams& p, cudaStream_t st) {                          \
+    return launch_chunk_stash_t<D, TIN>(p, st);                                                 \
+  }                                                                                             \
   }

@@ -37,6 +37,12 @@ struct ScanParams {
   // the segment's right-acting maps I - k_hat alpha^T.  n_main <= 0: no such units.
   int n_main;
   float* out2;               // [units - n_main, T, D]
+  // Backward pass (chunk kernel, u = k_hat path): per-token z_t, e_t [units, T, D] and delta_t
+  // [units, T] of the forward recurrence are left here; nullptr: not wanted.  With a stash the
+  // readout may be dropped (out == nullptr).
+  float* stash_z;
+  float* stash_e;
+  float* stash_delta;
 #ifdef VLA_SECTION_TIMERS
   long long* dbg;      // debug builds only: per-section clock64 totals of unit 0
 #endif

@@ -12,7 +12,8 @@ namespace vla {
 #define VLA_DECLARE_CHUNK_TU(TAG)                                   \
   int launch_chunk_##TAG(const ScanParams& p, cudaStream_t st);     \
   int launch_chunk_tri_##TAG(const ScanParams& p, cudaStream_t st); \
-  int chunk_resident_##TAG(bool tri);
+  int chunk_resident_##TAG(bool tri);                               \
+  int launch_chunk_stash_##TAG(const ScanParams& p, cudaStream_t st);
 VLA_DECLARE_CHUNK_TU(d32_f32)
 VLA_DECLARE_CHUNK_TU(d32_bf16)
 VLA_DECLARE_CHUNK_TU(d64_f32)
@@ -39,6 +40,11 @@ int launch_chunk(int d, int dtype, const ScanParams& p, cudaStream_t st) {
 
 int launch_chunk_tri(int d, int dtype, const ScanParams& p, cudaStream_t st) {
   VLA_CHUNK_DISPATCH(launch_chunk_tri, p, st);
+  return VLA_ERR_UNSUPPORTED;
+}
+
+int launch_chunk_stash(int d, int dtype, const ScanParams& p, cudaStream_t st) {
+  VLA_CHUNK_DISPATCH(launch_chunk_stash, p, st);
   return VLA_ERR_UNSUPPORTED;
 }
 

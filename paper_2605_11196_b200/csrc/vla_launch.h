@@ -23,6 +23,9 @@ int launch_decode(int d, int dtype, const ScanParams& p, cudaStream_t st);
 // Chunk kernel, d in {32, 64, 128}: plain or balanced grid, chosen from the shape.
 int launch_chunk(int d, int dtype, const ScanParams& p, cudaStream_t st);
 
+// Chunk kernel as the forward of a backward pass: leaves z_t, e_t, delta_t per token (p.stash_*).
+int launch_chunk_stash(int d, int dtype, const ScanParams& p, cudaStream_t st);
+
 // Chunk kernel with three warp groups per CTA (d in {32, 64}; sequence-parallel launches).
 int launch_chunk_tri(int d, int dtype, const ScanParams& p, cudaStream_t st);
 

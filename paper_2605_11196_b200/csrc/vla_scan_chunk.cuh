@@ -368,11 +368,15 @@ __device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) 
 // TRI: a third warp group runs the segment's transfer scan (S from I, v = 0; sequence-parallel
 // launches at d <= 64) next to group S, on the same products of group A.  Its readout goes to
 // out2 and its final state to S_T[n_main + unit].
-template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false>
+// STASH: the launch also leaves z_t, e_t, delta_t of every token in global memory (and may
+// drop the readout) for the backward pass; a separate instantiation so that the plain forward
+// kernel carries none of it.
+template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false, bool STASH = false>
 __global__ void __launch_bounds__((TRI ? 3 : 2) * D, (TRI && sizeof(TIn) == 2) ? 2 : 1)
 vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
   using Cfg = ChunkCfg<D, TIn, UM, TRI>;
   static_assert(!TRI || (D <= 64 && !BALANCED), "three groups: d <= 64, one CTA per unit");
+  static_assert(!STASH || (UM == kUKhat && !TRI && !BALANCED), "the stash belongs to the plain u = k_hat kernel");
   constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly
   constexpr bool UT = Cfg::UT;       // u comes from the caller's tensor
   constexpr int NIN = Cfg::NIN;
@@ -735,7 +739,11 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
             m[j] = fmaf(-l, msj, m[j]);
           }
           if (h == hs) Ls[r * CP + s2] = l;
-          if (lane == 0) { dlt[s2] = piv; idl[s2] = ipiv; nidl[s2] = -ipiv; }
+          if (lane == 0) {
+            dlt[s2] = piv; idl[s2] = ipiv; nidl[s2] = -ipiv;
+            if (STASH && p.stash_delta && s2 < nv)
+              p.stash_delta[size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C + s2] = piv;
+          }
         }
         if (HAS_U) {
           // N[s][t] = z_s . k_hat_t (s <= t) from X by the same elimination:
@@ -798,6 +806,12 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
           for (int t = 0; t < 16; ++t) {
             Zs[t * D + g] = z[t];
             sq[t] = z[t] * z[t];
+          }
+          if (STASH && p.stash_z) {   // the backward pass walks the tokens back with these
+            float* zs = p.stash_z + (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C) * D + g;
+#pragma unroll
+            for (int t = 0; t < 16; ++t)
+              if (t < nv) zs[size_t(t) * D] = z[t];
           }
         } else {
           // a_t = A_t k_hat_t = A k_hat_t - sum_{s<=t} z_s (z_s.k_hat_t)/delta_s: group S gets a;
@@ -953,6 +967,12 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
           ep[t] = e[t] * scs[t];
           Eps[t * D + g] = ep[t];
         }
+        if (STASH && p.stash_e) {
+          float* es = p.stash_e + (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C) * D + g;
+#pragma unroll
+          for (int t = 0; t < 16; ++t)
+            if (t < n) es[size_t(t) * D] = e[t];
+        }
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
           float a0 = R0s[t * D + g], a1 = 0.f;
@@ -977,9 +997,11 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
       group_bar(sbar, NG);  // Eps and the out stage complete
       if (g == 0) {
         const size_t tok = size_t(uin) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
-        bulk_store((pscan ? p.out2 : p.out) + tok * D, ostage + size_t(c & 1) * C * D,
-                   uint32_t(n) * D * sizeof(float));
-        bulk_commit();
+        float* odst = pscan ? p.out2 : p.out;
+        if (!STASH || odst) {   // a backward pass that only wants the stash passes no readout buffer
+          bulk_store(odst + tok * D, ostage + size_t(c & 1) * C * D, uint32_t(n) * D * sizeof(float));
+          bulk_commit();
+        }
       }
       VLA_MARK(3)
 

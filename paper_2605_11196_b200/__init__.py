@@ -11,4 +11,5 @@ from .binding import (VLA_BF16, VLA_ERR_ALIGNMENT, VLA_ERR_CUDA, VLA_ERR_DEVICE_
                       vla_forward_host_static, VLA_ERR_TOO_LARGE, VLA_STATIC_SCRATCH_BYTES,
                       vla_host_workspace_bytes, vla_query_support, vla_version,
                       vla_forward_seqpar, seqpar_segments, seqpar_workspace_bytes,
-                      measure_fp32_fma_tflops, vla_backward, VlaGrads)
+                      measure_fp32_fma_tflops, vla_backward, VlaGrads,
+                      backward_workspace_bytes)

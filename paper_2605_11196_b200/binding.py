@@ -208,6 +208,10 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
     return VlaResult(out, S_T, A_T, z_T, status)
 
 
+def backward_workspace_bytes(B: int, H: int, T: int, d_k: int) -> int:
+    return int(load_library().vla_backward_workspace_bytes(B, H, T, d_k))
+
+
 class VlaGrads(NamedTuple):
     dq: torch.Tensor
     dk: torch.Tensor

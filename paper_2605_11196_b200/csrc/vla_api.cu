@@ -446,7 +446,10 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
 size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k) {
   if (B < 0 || H < 0 || T < 0 || d_k <= 0) return 0;
   const size_t units = size_t(B) * size_t(H);
-  return 2 * round256(units * T * d_k * sizeof(float)) + round256(units * T * sizeof(float)) + 256;
+  const size_t vec = round256(units * T * d_k * sizeof(float));
+  const size_t mat = round256(units * d_k * d_k * sizeof(float));
+  // z, e, dalpha, dk_hat (S part), key-sum gradient per token; delta per token; S_T, A_T, key sum
+  return 5 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + 256;
 }
 
 int vla_backward(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,
@@ -459,7 +462,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   if (rc != VLA_OK) return rc;
   rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, d_out);
   if (rc != VLA_OK) return rc;
-  if (o.u || o.refresh_period > 0 || d_k > 64) return VLA_ERR_UNSUPPORTED;
+  if (o.u || o.refresh_period > 0) return VLA_ERR_UNSUPPORTED;
   const int units = B * H;
   if (units > 0 && T > 0 && (!dq || !dk || !dv)) return VLA_ERR_INVALID_ARG;
   const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0};
@@ -470,16 +473,49 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   if (!workspace || workspace_bytes < vla_backward_workspace_bytes(B, H, T, d_k)) return VLA_ERR_INVALID_ARG;
   unsigned char* w = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(workspace) + 255) & ~uintptr_t(255));
-  const size_t vec_bytes = round256(size_t(units) * T * d_k * sizeof(float));
-  vla::BackwardParams p;
-  p.q = q; p.k = k; p.v = v; p.S0 = S0; p.A0 = A0; p.z0 = o.z0;
-  p.d_out = d_out; p.dS_T = dS_T; p.dA_T = dA_T; p.dz_T = dz_T;
+  const size_t vec = round256(size_t(units) * T * d_k * sizeof(float));
+  const size_t mat = round256(size_t(units) * d_k * d_k * sizeof(float));
+  const size_t sca = round256(size_t(units) * T * sizeof(float));
+  float* zst = reinterpret_cast<float*>(w);
+  float* est = reinterpret_cast<float*>(w + vec);
+  float* dst = reinterpret_cast<float*>(w + 2 * vec);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (d_k == 16) {
+    // d = 16 has no chunk kernel: the single kernel runs its own token-level forward sweep
+    vla::BackwardParams p;
+    p.q = q; p.k = k; p.v = v; p.S0 = S0; p.A0 = A0; p.z0 = o.z0;
+    p.d_out = d_out; p.dS_T = dS_T; p.dA_T = dA_T; p.dz_T = dz_T;
+    p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;
+    p.zst = zst; p.est = est; p.dst = dst;
+    p.status = o.status; p.lambda = lambda_; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;
+    return vla::launch_backward(d_k, o.qkv_dtype, p, st);
+  }
+  // 1. the forward recurrence on the chunk kernel, leaving z_t, e_t, delta_t and the final states
+  float* dalw = reinterpret_cast<float*>(w + 2 * vec + sca);
+  float* dkSw = reinterpret_cast<float*>(w + 3 * vec + sca);
+  float* gztw = reinterpret_cast<float*>(w + 4 * vec + sca);
+  float* STw = reinterpret_cast<float*>(w + 5 * vec + sca);
+  float* ATw = reinterpret_cast<float*>(w + 5 * vec + sca + mat);
+  float* zTw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat);
+  ScanParams f;
+  f.q = q; f.k = k; f.v = v; f.u = nullptr;
+  f.S0 = S0; f.A0 = A0; f.z0 = o.z0;
+  f.out = nullptr; f.S_T = STw; f.A_T = ATw; f.zT = zTw;
+  f.status = o.status; f.lambda = lambda_; f.eps = o.eps;
+  f.T = T; f.units = units; f.flags = o.flags;
+  f.refresh_period = 0; f.refresh_eta = 0.0f; f.step_offset = 0; f.u_is_khat = 0;
+  f.n_main = 0; f.out2 = nullptr;
+  f.stash_z = zst; f.stash_e = est; f.stash_delta = dst;
+  rc = vla::launch_chunk_stash(d_k, o.qkv_dtype, f, st);
+  if (rc != VLA_OK) return rc;
+  // 2. the S-side and A-side reverse scans
+  vla::BackwardSplitParams p;
+  p.q = q; p.k = k; p.z0 = o.z0; p.d_out = d_out; p.dS_T = dS_T; p.dA_T = dA_T; p.dz_T = dz_T;
+  p.ST = STw; p.AT = ATw; p.zT = zTw; p.zst = zst; p.est = est; p.dst = dst;
+  p.dal = dalw; p.dkS = dkSw; p.gzt = gztw;
   p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;
-  p.zst = reinterpret_cast<float*>(w);
-  p.est = reinterpret_cast<float*>(w + vec_bytes);
-  p.dst = reinterpret_cast<float*>(w + 2 * vec_bytes);
-  p.status = o.status; p.lambda = lambda_; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;
-  return vla::launch_backward(d_k, o.qkv_dtype, p, static_cast<cudaStream_t>(stream));
+  p.status = o.status; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;
+  return vla::launch_backward_split(d_k, o.qkv_dtype, p, st);
 }
 
 int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream) {

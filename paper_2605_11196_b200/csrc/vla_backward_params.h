@@ -33,4 +33,35 @@ struct BackwardParams {
   uint32_t flags;
 };
 
+// Arguments of the two reverse scans (see vla_backward_split.cuh).
+struct BackwardSplitParams {
+  const void* q;        // [units, T, D]
+  const void* k;
+  const float* z0;      // unused by the sweeps (the forward consumed it)
+  const float* d_out;   // [units, T, D]
+  const float* dS_T;    // [units, D, D] or nullptr
+  const float* dA_T;
+  const float* dz_T;    // [units, D] or nullptr
+  const float* ST;      // [units, D, D] final states of the forward (workspace)
+  const float* AT;
+  const float* zT;      // [units, D]
+  const float* zst;     // [units, T, D] z_t
+  const float* est;     // [units, T, D] e_t
+  const float* dst;     // [units, T]    delta_t
+  float* dal;           // [units, T, D] S side -> A side: dL/d alpha_t
+  float* dkS;           // [units, T, D] S side -> A side: S-side part of dL/d k_hat_t
+  float* gzt;           // [units, T, D] S side -> A side: dL/d(key sum) seen by token t
+  float* dq;            // [units, T, D]
+  float* dk;
+  float* dv;
+  float* dS0;           // [units, D, D] or nullptr
+  float* dA0;
+  float* dz0;           // [units, D] or nullptr
+  int* status;
+  float eps;
+  int T;
+  int units;
+  uint32_t flags;
+};
+
 }  // namespace vla

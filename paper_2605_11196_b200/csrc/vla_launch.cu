@@ -3,6 +3,7 @@
 #include "vla.h"
 #include "vla_launch.h"
 #include "vla_backward.cuh"
+#include "vla_backward_split.cuh"
 #include "vla_decode.cuh"
 #include "vla_scan_token.cuh"
 #include "vla_seqpar.cuh"
@@ -155,6 +156,26 @@ int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st) 
     default: return VLA_ERR_UNSUPPORTED;
   }
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+// The two reverse scans (after the chunk kernel has left the stash), d in {32, 64, 128}.
+namespace {
+template <int D, typename TIn>
+int launch_backward_split_t(const BackwardSplitParams& p, cudaStream_t st) {
+  vla_backward_s_kernel<D, TIn><<<p.units, 256, 0, st>>>(p);
+  vla_backward_a_kernel<D, TIn><<<p.units, 256, 0, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+}  // namespace
+
+int launch_backward_split(int d, int dtype, const BackwardSplitParams& p, cudaStream_t st) {
+  const bool f32 = dtype == VLA_F32;
+  switch (d) {
+    case 32: return f32 ? launch_backward_split_t<32, float>(p, st) : launch_backward_split_t<32, uint16_t>(p, st);
+    case 64: return f32 ? launch_backward_split_t<64, float>(p, st) : launch_backward_split_t<64, uint16_t>(p, st);
+    case 128: return f32 ? launch_backward_split_t<128, float>(p, st) : launch_backward_split_t<128, uint16_t>(p, st);
+    default: return VLA_ERR_UNSUPPORTED;
+  }
 }
 
 // ---------------------------------------------------------------- decode kernel

@@ -10,6 +10,7 @@
 
 namespace vla {
 struct BackwardParams;
+struct BackwardSplitParams;
 }
 
 namespace vla {
@@ -40,6 +41,9 @@ int seqpar_after_scan(int d, const SeqParParams& sp, float* A_T, float* zT, cons
 
 // Backward pass, token kernel, d in {16, 32, 64}, u = k_hat.
 int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st);
+
+// Backward pass as two reverse scans over the chunk kernel's stash, d in {32, 64, 128}, u = k_hat.
+int launch_backward_split(int d, int dtype, const BackwardSplitParams& p, cudaStream_t st);
 
 // Register-only fp32 FMA loop over the whole device (measurement helper); *flops = work launched.
 int launch_fp32_probe(int iters, float* sink, double* flops, cudaStream_t st);

@@ -50,7 +50,7 @@ def _check(g, ref, tol, label):
     return errs
 
 
-@pytest.mark.parametrize("d", [16, 32, 64])
+@pytest.mark.parametrize("d", [16, 32, 64, 128])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("flags", [0, IDENT])
 @pytest.mark.parametrize("T", [1, 7, 64, 200])
@@ -64,7 +64,7 @@ def test_gradients_agree_with_the_backward_oracle(d, dtype, flags, T):
         _check(got, ref, 2e-4, "backward d=%d T=%d lam=%g" % (d, T, lam))
 
 
-@pytest.mark.parametrize("d", [32, 64])
+@pytest.mark.parametrize("d", [16, 32, 64, 128])
 @pytest.mark.parametrize("flags", [0, IDENT])
 def test_carried_states_and_incoming_state_gradients(d, flags):
     w = _small(d, 96, "f32", units=(1, 4), seed=3100 + d)
@@ -84,8 +84,7 @@ def test_carried_states_and_incoming_state_gradients(d, flags):
 
 
 def test_mid_workload_gradients_and_what_is_not_covered():
-    """The `mid` workload (32 units, d = 64, T = 4096) whole, and the shapes the first backward
-    kernel does not take."""
+    """The `mid` workload (32 units, d = 64, T = 4096) whole, and a shape without kernels."""
     w = W.WORKLOADS["mid"]
     q, k, v = W.make_inputs(w)
     g = torch.Generator().manual_seed(11)
@@ -93,8 +92,8 @@ def test_mid_workload_gradients_and_what_is_not_covered():
     got, ref = _run_both(q, k, v, w.lam, d_out)
     print("mid backward", _check(got, ref, 1e-3, "backward mid"))
     dev = torch.device("cuda:0")
-    w128 = _small(128, 16, "f32")
-    q, k, v = [x.to(dev) for x in W.make_inputs(w128)]
+    w48 = _small(48, 16, "f32")
+    q, k, v = [x.to(dev) for x in W.make_inputs(w48)]
     with pytest.raises(vla.VlaError) as ei:
-        vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 16, 128), device=dev))
+        vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 16, 48), device=dev))
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED

@@ -162,8 +162,17 @@ int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st) 
 namespace {
 template <int D, typename TIn>
 int launch_backward_split_t(const BackwardSplitParams& p, cudaStream_t st) {
-  vla_backward_s_kernel<D, TIn><<<p.units, 256, 0, st>>>(p);
-  vla_backward_a_kernel<D, TIn><<<p.units, 256, 0, st>>>(p);
+  using G = BwdSplitGeom<D>;
+  using M = BackwardSplitSmem<D>;
+  auto ks = vla_backward_s_kernel<D, TIn>;
+  auto ka = vla_backward_a_kernel<D, TIn>;
+  if (cudaFuncSetAttribute(ks, cudaFuncAttributeMaxDynamicSharedMemorySize, int(M::s_bytes)) != cudaSuccess ||
+      cudaFuncSetAttribute(ka, cudaFuncAttributeMaxDynamicSharedMemorySize, int(M::a_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  ks<<<p.units, G::NT, M::s_bytes, st>>>(p);   // TX / 2 matrix warps + 1 helper warp
+  ka<<<p.units, G::NT, M::a_bytes, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 }  // namespace

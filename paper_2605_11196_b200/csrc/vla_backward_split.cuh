@@ -11,28 +11,22 @@
 //
 // each a CTA per unit holding TWO d x d matrices in registers, as R x RC blocks on a grid of
 // 16 x TX threads (R = d / 16 rows, RC = d / TX columns; TX = 16, or 32 at d = 128, where the
-// blocks of a 16-wide grid would not leave registers for a ninth warp).  The forward recurrence is not re-run here: the chunk kernel
-// leaves z_t, e_t, delta_t per token and the final S, A, key sum in the workspace, and both
-// sweeps walk the states back by undoing the rank-1 updates (S_{t-1} = S_t - e alpha^T,
-// A_{t-1} = A_t + z z^T / delta).  Formulas per token: see vla_backward.cuh.
+// blocks of a 16-wide grid would leave no registers for the helper warps).  The blocks are kept
+// as column pairs and every product with them is a packed fma.rn.f32x2.  The forward
+// recurrence is not re-run here: the chunk kernel leaves z_t, e_t, delta_t per token and the
+// final S, A, key sum in the workspace, and both sweeps walk the states back by undoing the
+// rank-1 updates (S_{t-1} = S_t - e alpha^T, A_{t-1} = A_t + z z^T / delta).  Formulas per
+// token: see vla_backward.cuh.
 //
-// Both kernels keep a ring of four per-token contexts in shared memory so that opening a
-// token (loading its rows, alpha, denominators: nothing that depends on the adjoints) and
-// closing one (vector arithmetic on finished products) are done by a ninth warp off the path
-// of the TX / 2 matrix warps; one CTA barrier per token.
+// Both kernels keep a ring of four per-token contexts in shared memory.  Opening a token
+// (loading its rows, alpha, denominators: nothing that depends on the adjoints) and closing one
+// (vector arithmetic on finished products, the stores) are done by two helper warps off the
+// path of the TX / 2 matrix warps; one CTA barrier per token.
 #pragma once
 
 #include "vla_backward.cuh"
 
 namespace vla {
-
-// Dynamic shared memory of the two reverse scans (the kernels assert these against their layouts).
-template <int D>
-struct BackwardSplitSmem {
-  static constexpr int NW = (D >= 128 ? 32 : 16) / 2;
-  static constexpr size_t s_bytes = sizeof(float) * (4 * 7 * D + 4 * 4 + 3 * 2 * D + 2 * NW * 3 * D + D);
-  static constexpr size_t a_bytes = sizeof(float) * (4 * 6 * D + 4 * 4 + 3 * 3 * D + 2 * NW * D + NW * D + 4);
-};
 
 // Thread grid of the two reverse scans.
 template <int D>
@@ -40,12 +34,69 @@ struct BwdSplitGeom {
   static constexpr int TX = D >= 128 ? 32 : 16;   // threads along a matrix row
   static constexpr int R = D / 16;                // rows of a thread's block
   static constexpr int RC = D / TX;               // columns of a thread's block
-  static constexpr int NW = TX / 2;               // matrix warps; warp NW is the helper
-  static constexpr int NT = NW * 32 + 32;
+  static constexpr int NW = TX / 2;               // matrix warps; warp NW closes, warp NW + 1 opens tokens
+  static constexpr int NT = NW * 32 + 64;
+  static constexpr int MINB = D == 64 ? 3 : 1;    // CTAs per SM the register budget is held to
+};
+
+// Dynamic shared memory of the two reverse scans (the kernels assert these against their layouts).
+template <int D>
+struct BackwardSplitSmem {
+  static constexpr int NW = BwdSplitGeom<D>::NW;
+  static constexpr size_t s_bytes = sizeof(float) * (4 * 8 * D + 4 * 4 + 3 * 2 * D + 2 * NW * 3 * D + D);
+  static constexpr size_t a_bytes = sizeof(float) * (4 * 6 * D + 4 * 4 + 3 * 3 * D + 2 * NW * D + NW * D + 4);
 };
 
 // All threads of the CTA, whichever loop they are in.
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;" ::: "memory"); }
+
+__device__ __forceinline__ float2 bwd_ffma2(float2 a, float2 b, float2 c) {
+  uint64_t ra, rb, rc, rd;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rc) : "f"(c.x), "f"(c.y));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+  float2 d;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+  return d;
+}
+
+// N consecutive fp32 values moved as one access (N = 1, 2, 4, 8; 8 as two of 4)
+template <int N>
+struct alignas(N >= 4 ? 16 : 4 * N) BwdVec { float v[N]; };
+template <int N>
+__device__ __forceinline__ void bwd_ld(const float* p, float (&out)[N]) {
+  if constexpr (N > 4) {
+#pragma unroll
+    for (int i = 0; i < N / 4; ++i) {
+      const BwdVec<4> x = reinterpret_cast<const BwdVec<4>*>(p)[i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) out[4 * i + j] = x.v[j];
+    }
+  } else {
+    const BwdVec<N> x = *reinterpret_cast<const BwdVec<N>*>(p);
+#pragma unroll
+    for (int j = 0; j < N; ++j) out[j] = x.v[j];
+  }
+}
+template <int N>
+__device__ __forceinline__ void bwd_st(float* p, const float (&in)[N]) {
+  static_assert(N <= 4, "one access");
+  BwdVec<N> x;
+#pragma unroll
+  for (int j = 0; j < N; ++j) x.v[j] = in[j];
+  *reinterpret_cast<BwdVec<N>*>(p) = x;
+}
+// N consecutive input values (fp32 or bf16 bits) widened to fp32
+template <int N>
+__device__ __forceinline__ void bwd_ld_in(const float* p, float (&out)[N]) { bwd_ld<N>(p, out); }
+template <int N>
+__device__ __forceinline__ void bwd_ld_in(const uint16_t* p, float (&out)[N]) {
+  struct alignas(2 * N) H { uint16_t v[N]; };
+  const H x = *reinterpret_cast<const H*>(p);
+#pragma unroll
+  for (int j = 0; j < N; ++j) out[j] = __uint_as_float(uint32_t(x.v[j]) << 16);
+}
 
 // Sums of N per-thread values over the 2*OFF lanes of a row group, by halving: at each step a
 // lane hands the half of its values that its partner keeps, so N values cost N - 1 shuffles
@@ -69,22 +120,22 @@ __device__ __forceinline__ void rows_reduce(float* v, int lane) {
   }
 }
 
-
 // ------------------------------------------------------------------------------ S side
 template <int D, typename TIn>
-__global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_s_kernel(const BackwardSplitParams p) {
+__global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vla_backward_s_kernel(const BackwardSplitParams p) {
   using G = BwdSplitGeom<D>;
   constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW, NT = G::NT;
-  constexpr int EPL = D / 32;
+  constexpr int RP = RC / 2;          // column pairs of a block
+  constexpr int EPL = D / 32;         // consecutive vector elements per lane of a helper warp
   constexpr int NCTX = 4;
-  enum { cKf = 0, cKh, cQf, cGo, cEt, cAl, cZk, NV };
+  enum { cKf = 0, cKh, cQf, cGo, cDy, cEt, cAl, cZk, NV };
   enum { sDen = 0, sDenLive, sQal };
   struct Smem {
     float ctx[NCTX][NV][D];
     float cscl[NCTX][4];
     float rowv[3][2][D];       // y = S' qf, g1 = GS alpha, ring of three tokens
     float part[2][NW][3][D];   // column-sum partials by token parity and warp
-    float gz[D];               // dL/d(key sum), carried by the helper warp
+    float gz[D];               // dL/d(key sum), carried by the closing warp
   };
   static_assert(sizeof(Smem) == BackwardSplitSmem<D>::s_bytes, "shared memory size of the S side");
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -94,6 +145,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_s_kernel(con
   const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ty = tid / TX, tx = tid % TX;
   const int row0 = ty * R, col0 = tx * RC;
+  const int c0 = lane * EPL;          // first vector element of this lane in a helper warp
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
   const float eps = p.eps;
   const int T = p.T;
@@ -105,154 +157,87 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_s_kernel(con
   const float* est = p.est + ubase;
   const float* dst = p.dst + size_t(unit) * T;
 
-  float S[R][RC], GS[R][RC];
-#pragma unroll
-  for (int r = 0; r < R; ++r)
-#pragma unroll
-    for (int c = 0; c < RC; ++c) {
-      const size_t idx = (size_t(unit) * D + row0 + r) * D + col0 + c;
-      const bool own = warp < NW;   // the helper warp holds no block
-      S[r][c] = own ? p.ST[idx] : 0.0f;
-      GS[r][c] = (own && p.dS_T) ? p.dS_T[idx] : 0.0f;
-    }
   for (int j = tid; j < D; j += NT) gz[j] = p.dz_T ? p.dz_T[size_t(unit) * D + j] : 0.0f;
 
   auto cvec = [&](int t, int which) { return ctx[t & (NCTX - 1)][which]; };
   // after rows_reduce<R, TX / 2> a lane holds the total of row myrow of its group's R rows
   const int myrow = tx / (TX / R);
   const bool row_writer = (tx % (TX / R)) == 0;
-
-  // the helper warp opens tokens two segments ahead; the rows come from global memory one more ahead
-  float pk[EPL], pq[EPL], pz[EPL], pe[EPL], pg[EPL];
-  float pdelta = 1.0f;
-  auto fetch_token = [&](int t) {
-    if (t < 0) return;
-    pdelta = dst[t];
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      pk[e] = load1<TIn>(gk, size_t(t) * D + c);
-      pq[e] = load1<TIn>(gq, size_t(t) * D + c);
-      pz[e] = zst[size_t(t) * D + c];
-      pe[e] = est[size_t(t) * D + c];
-      pg[e] = gdo[size_t(t) * D + c];
-    }
-  };
-  auto open_token = [&](int t, bool last) {
-    float* okf = cvec(t, cKf); float* okh = cvec(t, cKh); float* oqf = cvec(t, cQf);
-    float* ogo = cvec(t, cGo); float* oet = cvec(t, cEt); float* oal = cvec(t, cAl);
-    float* ozk = cvec(t, cZk);
-    const float* nzk = cvec(t + 1, cZk);
-    const float* nkf = cvec(t + 1, cKf);
-    float zx[EPL], kx[EPL], qx[EPL];
-    float ss = 0.f, zz = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      float kk = pk[e], qq = pq[e];
-      if (!ident) { kk = bwd_phi(kk); qq = bwd_phi(qq); }
-      ogo[c] = pg[e];
-      oet[c] = pe[e];
-      okf[c] = kk;
-      oqf[c] = qq;
-      kx[e] = kk; qx[e] = qq; zx[e] = pz[e];
-      ss = fmaf(kk, kk, ss);
-      zz = fmaf(pz[e], pz[e], zz);
-    }
-    ss = warp_sum(ss);
-    zz = warp_sum(zz);
-    const float nk = fmaxf(sqrtf(ss), eps);
-    const float idl = 1.0f / pdelta;
-    const float sc = idl / fmaxf(sqrtf(zz) * idl, eps);
-    float dn = 0.f, qa = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      okh[c] = kx[e] / nk;
-      oal[c] = sc * zx[e];
-      const float zkc = last ? p.zT[size_t(unit) * D + c] : (ident ? nzk[c] : nzk[c] - nkf[c]);
-      ozk[c] = zkc;
-      dn = fmaf(zkc, qx[e], dn);
-      qa = fmaf(qx[e], sc * zx[e], qa);
-    }
-    dn = warp_sum(dn);
-    qa = warp_sum(qa);
-    if (lane == 0) {
-      float* os = cscl[t & (NCTX - 1)];
-      os[sDen] = ident ? 1.0f : fmaxf(dn, eps);
-      os[sDenLive] = (ident || dn < eps) ? 0.0f : 1.0f;
-      os[sQal] = qa;
-    }
-  };
-  // helper warp: the vector results of token t from its finished products
-  auto close_token = [&](int t) {
-    const int par = t & 1;
-    const float* go = cvec(t, cGo); const float* et = cvec(t, cEt); const float* al = cvec(t, cAl);
-    const float* qf = cvec(t, cQf); const float* zkt = cvec(t, cZk);
-    const float* yv = rowv[t % 3][0]; const float* g1 = rowv[t % 3][1];
-    const float den = cscl[t & (NCTX - 1)][sDen], qal = cscl[t & (NCTX - 1)][sQal];
-    const bool den_live = cscl[t & (NCTX - 1)][sDenLive] != 0.0f;
-    float odo = 0.f, ede = 0.f, dye = 0.f;
-    float dex[EPL];
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      const float dy = go[c] / den;
-      dex[e] = g1[c] + dy * qal;
-      odo = fmaf(yv[c], go[c], odo);
-      ede = fmaf(et[c], dex[e], ede);
-      dye = fmaf(dy, et[c], dye);
-    }
-    odo = warp_sum(odo); ede = warp_sum(ede); dye = warp_sum(dye);
-    const float dden = den_live ? -odo / (den * den) : 0.0f;
-    const size_t tb = ubase + size_t(t) * D;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      float c1 = 0.f, c2 = 0.f, c3 = 0.f;
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        c1 += part[par][w][0][c]; c2 += part[par][w][1][c]; c3 += part[par][w][2][c];
-      }
-      float dq = c1 + dden * zkt[c];
-      float gzc = gz[c];
-      if (!ident) {
-        dq *= qf[c] > 1.0f ? 1.0f : qf[c];     // phi'(q) from phi(q)
-        gzc += dden * qf[c];
-        gz[c] = gzc;
-      }
-      p.dq[tb + c] = dq;
-      p.dv[tb + c] = dex[e];
-      p.dal[tb + c] = c2 + qf[c] * dye;               // (GS + dy qf^T)^T e
-      p.dkS[tb + c] = -(c3 - al[c] * ede);            // -(S' - e alpha^T)^T de
-      p.gzt[tb + c] = ident ? 0.0f : gzc;
-    }
-  };
-
-  constexpr int kHelper = NW;   // the last warp opens and closes tokens; the others do the matrix work
-  auto row_dots = [&](int t) {   // y = S' qf, g1 = GS alpha of token t
-    const float* qf = cvec(t, cQf); const float* al = cvec(t, cAl);
-    float a0[R], a1[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      float x0 = 0.f, x1 = 0.f;
-#pragma unroll
-      for (int c = 0; c < RC; ++c) {
-        x0 = fmaf(S[r][c], qf[col0 + c], x0);
-        x1 = fmaf(GS[r][c], al[col0 + c], x1);
-      }
-      a0[r] = x0; a1[r] = x1;
-    }
-    rows_reduce<R, TX / 2>(a0, lane);
-    rows_reduce<R, TX / 2>(a1, lane);
-    if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
-  };
+  constexpr int kCloser = NW, kOpener = NW + 1;
 
   // Segment t (one CTA barrier): the matrix warps take the column sums and the two rank-1
-  // updates of token t, then the row dots of token t - 1; the helper warp closes token t + 1
-  // and opens token t - 2.  The two roles run loops of their own with the same number of
-  // barriers, so that the helper's staging registers and the matrix blocks never share a thread.
-  if (warp == kHelper) {
+  // updates of token t, then the row dots of token t - 1; the closing warp finishes token
+  // t + 1 and the opening warp prepares token t - 2.  The roles run loops of their own with
+  // the same number of barriers, so that staging registers and matrix blocks never share a thread.
+  if (warp == kOpener) {
+    // rows come from global memory one segment before they are opened
+    float pk[EPL], pq[EPL], pz[EPL], pe[EPL], pg[EPL];
+    float pdelta = 1.0f;
+    auto fetch_token = [&](int t) {
+      if (t < 0) return;
+      pdelta = dst[t];
+      const size_t o = size_t(t) * D + c0;
+      bwd_ld_in<EPL>(gk + o, pk);
+      bwd_ld_in<EPL>(gq + o, pq);
+      bwd_ld<EPL>(zst + o, pz);
+      bwd_ld<EPL>(est + o, pe);
+      bwd_ld<EPL>(gdo + o, pg);
+    };
+    auto open_token = [&](int t, bool last) {
+      float kx[EPL], qx[EPL], khx[EPL], alx[EPL], zkx[EPL], dyx[EPL];
+      float ss = 0.f, zz = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        float kk = pk[e], qq = pq[e];
+        if (!ident) { kk = bwd_phi(kk); qq = bwd_phi(qq); }
+        kx[e] = kk; qx[e] = qq;
+        ss = fmaf(kk, kk, ss);
+        zz = fmaf(pz[e], pz[e], zz);
+      }
+      if (last) {
+        bwd_ld<EPL>(p.zT + size_t(unit) * D + c0, zkx);
+      } else {
+        float nz[EPL], nk2[EPL];
+        bwd_ld<EPL>(cvec(t + 1, cZk) + c0, nz);
+        bwd_ld<EPL>(cvec(t + 1, cKf) + c0, nk2);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) zkx[e] = ident ? nz[e] : nz[e] - nk2[e];
+      }
+      ss = warp_sum(ss);
+      zz = warp_sum(zz);
+      const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
+      const float idl = 1.0f / pdelta;
+      const float sc = idl / fmaxf(sqrtf(zz) * idl, eps);
+      float dn = 0.f, qa = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        khx[e] = kx[e] * ink;
+        alx[e] = sc * pz[e];
+        dn = fmaf(zkx[e], qx[e], dn);
+        qa = fmaf(qx[e], alx[e], qa);
+      }
+      dn = warp_sum(dn);
+      qa = warp_sum(qa);
+      const float den = ident ? 1.0f : fmaxf(dn, eps);
+      const float iden = 1.0f / den;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) dyx[e] = pg[e] * iden;
+      bwd_st<EPL>(cvec(t, cKf) + c0, kx);
+      bwd_st<EPL>(cvec(t, cKh) + c0, khx);
+      bwd_st<EPL>(cvec(t, cQf) + c0, qx);
+      bwd_st<EPL>(cvec(t, cGo) + c0, pg);
+      bwd_st<EPL>(cvec(t, cDy) + c0, dyx);
+      bwd_st<EPL>(cvec(t, cEt) + c0, pe);
+      bwd_st<EPL>(cvec(t, cAl) + c0, alx);
+      bwd_st<EPL>(cvec(t, cZk) + c0, zkx);
+      if (lane == 0) {
+        float* os = cscl[t & (NCTX - 1)];
+        os[sDen] = den;
+        os[sDenLive] = (ident || dn < eps) ? 0.0f : 1.0f;
+        os[sQal] = qa;
+      }
+      __syncwarp();   // the next token opened reads this one's key sum and keys
+    };
     if (T > 0) {
       fetch_token(T - 1);
       open_token(T - 1, true);
@@ -263,77 +248,194 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_s_kernel(con
     cta_sync();
     cta_sync();
     for (int t = T - 1; t >= 0; --t) {
-      if (t + 1 <= T - 1) close_token(t + 1);
       if (t - 2 >= 0) {
         open_token(t - 2, false);
         fetch_token(t - 3);
       }
       cta_sync();
     }
+  } else if (warp == kCloser) {
+    // the vector results of token t from its finished products
+    auto close_token = [&](int t) {
+      const int par = t & 1;
+      float go[EPL], dy[EPL], et[EPL], al[EPL], qf[EPL], zkt[EPL], yv[EPL], g1[EPL];
+      bwd_ld<EPL>(cvec(t, cGo) + c0, go);
+      bwd_ld<EPL>(cvec(t, cDy) + c0, dy);
+      bwd_ld<EPL>(cvec(t, cEt) + c0, et);
+      bwd_ld<EPL>(rowv[t % 3][0] + c0, yv);
+      bwd_ld<EPL>(rowv[t % 3][1] + c0, g1);
+      const float den = cscl[t & (NCTX - 1)][sDen], qal = cscl[t & (NCTX - 1)][sQal];
+      const bool den_live = cscl[t & (NCTX - 1)][sDenLive] != 0.0f;
+      float odo = 0.f, ede = 0.f, dye = 0.f;
+      float dex[EPL];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        dex[e] = fmaf(dy[e], qal, g1[e]);
+        odo = fmaf(yv[e], go[e], odo);
+        ede = fmaf(et[e], dex[e], ede);
+        dye = fmaf(dy[e], et[e], dye);
+      }
+      float c1[EPL], c2[EPL], c3[EPL];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) { c1[e] = 0.f; c2[e] = 0.f; c3[e] = 0.f; }
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        float x1[EPL], x2[EPL], x3[EPL];
+        bwd_ld<EPL>(part[par][w][0] + c0, x1);
+        bwd_ld<EPL>(part[par][w][1] + c0, x2);
+        bwd_ld<EPL>(part[par][w][2] + c0, x3);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) { c1[e] += x1[e]; c2[e] += x2[e]; c3[e] += x3[e]; }
+      }
+      bwd_ld<EPL>(cvec(t, cAl) + c0, al);
+      bwd_ld<EPL>(cvec(t, cQf) + c0, qf);
+      bwd_ld<EPL>(cvec(t, cZk) + c0, zkt);
+      odo = warp_sum(odo); ede = warp_sum(ede); dye = warp_sum(dye);
+      const float dden = den_live ? -odo / (den * den) : 0.0f;
+      float gzc[EPL], dq[EPL], dalo[EPL], dko[EPL], gzo[EPL];
+      bwd_ld<EPL>(gz + c0, gzc);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        dq[e] = fmaf(dden, zkt[e], c1[e]);
+        if (!ident) {
+          dq[e] *= qf[e] > 1.0f ? 1.0f : qf[e];     // phi'(q) from phi(q)
+          gzc[e] = fmaf(dden, qf[e], gzc[e]);
+        }
+        dalo[e] = fmaf(qf[e], dye, c2[e]);          // (GS + dy qf^T)^T e
+        dko[e] = -(c3[e] - al[e] * ede);            // -(S' - e alpha^T)^T de
+        gzo[e] = ident ? 0.0f : gzc[e];
+      }
+      if (!ident) bwd_st<EPL>(gz + c0, gzc);
+      const size_t tb = ubase + size_t(t) * D + c0;
+      bwd_st<EPL>(p.dq + tb, dq);
+      bwd_st<EPL>(p.dv + tb, dex);
+      bwd_st<EPL>(p.dal + tb, dalo);
+      bwd_st<EPL>(p.dkS + tb, dko);
+      bwd_st<EPL>(p.gzt + tb, gzo);
+    };
+    cta_sync();
+    cta_sync();
+    for (int t = T - 1; t >= 0; --t) {
+      if (t + 1 <= T - 1) close_token(t + 1);
+      cta_sync();
+    }
     if (T > 0) close_token(0);
   } else {
+    float2 S[R][RP], GS[R][RP];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const size_t idx = (size_t(unit) * D + row0 + r) * D + col0;
+      float sv[RC], gv[RC];
+      bwd_ld<RC>(p.ST + idx, sv);
+      if (p.dS_T) {
+        bwd_ld<RC>(p.dS_T + idx, gv);
+      } else {
+#pragma unroll
+        for (int c = 0; c < RC; ++c) gv[c] = 0.0f;
+      }
+#pragma unroll
+      for (int m = 0; m < RP; ++m) {
+        S[r][m] = make_float2(sv[2 * m], sv[2 * m + 1]);
+        GS[r][m] = make_float2(gv[2 * m], gv[2 * m + 1]);
+      }
+    }
+    auto row_dots = [&](int t) {   // y = S' qf, g1 = GS alpha of token t
+      float qv[RC], av[RC];
+      bwd_ld<RC>(cvec(t, cQf) + col0, qv);
+      bwd_ld<RC>(cvec(t, cAl) + col0, av);
+      float a0[R], a1[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int m = 0; m < RP; ++m) {
+          x0 = bwd_ffma2(S[r][m], make_float2(qv[2 * m], qv[2 * m + 1]), x0);
+          x1 = bwd_ffma2(GS[r][m], make_float2(av[2 * m], av[2 * m + 1]), x1);
+        }
+        a0[r] = x0.x + x0.y; a1[r] = x1.x + x1.y;
+      }
+      rows_reduce<R, TX / 2>(a0, lane);
+      rows_reduce<R, TX / 2>(a1, lane);
+      if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
+    };
     cta_sync();
     if (T > 0) row_dots(T - 1);
     cta_sync();
     for (int t = T - 1; t >= 0; --t) {
-      const float* go = cvec(t, cGo); const float* et = cvec(t, cEt);
-      const float* kh = cvec(t, cKh); const float* qf = cvec(t, cQf); const float* al = cvec(t, cAl);
-      const float* g1 = rowv[t % 3][1];
-      const float den = cscl[t & (NCTX - 1)][sDen], qal = cscl[t & (NCTX - 1)][sQal];
-      float dyr[R], der[R];
+      const float qal = cscl[t & (NCTX - 1)][sQal];
+      float dyr[R], der[R], etr[R];
+      bwd_ld<R>(cvec(t, cDy) + row0, dyr);
+      bwd_ld<R>(rowv[t % 3][1] + row0, der);
+      bwd_ld<R>(cvec(t, cEt) + row0, etr);
+#pragma unroll
+      for (int r = 0; r < R; ++r) der[r] = fmaf(dyr[r], qal, der[r]);      // (GS + dy qf^T) alpha
+      float2 cc[3][RP];
+#pragma unroll
+      for (int m = 0; m < RP; ++m) { cc[0][m] = make_float2(0.f, 0.f); cc[1][m] = cc[0][m]; cc[2][m] = cc[0][m]; }
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        dyr[r] = go[row0 + r] / den;
-        der[r] = g1[row0 + r] + dyr[r] * qal;      // (GS + dy qf^T) alpha
-      }
-      float cc[3][RC];
+        const float2 d2 = make_float2(dyr[r], dyr[r]), e2 = make_float2(etr[r], etr[r]);
+        const float2 r2 = make_float2(der[r], der[r]);
 #pragma unroll
-      for (int c = 0; c < RC; ++c) {
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f;
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          s0 = fmaf(S[r][c], dyr[r], s0);
-          s1 = fmaf(GS[r][c], et[row0 + r], s1);
-          s2 = fmaf(S[r][c], der[r], s2);
+        for (int m = 0; m < RP; ++m) {
+          cc[0][m] = bwd_ffma2(S[r][m], d2, cc[0][m]);
+          cc[1][m] = bwd_ffma2(GS[r][m], e2, cc[1][m]);
+          cc[2][m] = bwd_ffma2(S[r][m], r2, cc[2][m]);
         }
-        cc[0][c] = s0; cc[1][c] = s1; cc[2][c] = s2;
       }
       if constexpr (TX == 16) {
         // two thread rows per warp: each half keeps half of the columns of the pair's sum
         constexpr int HC = RC / 2;
         const bool up = (lane & 16) != 0;
 #pragma unroll
-        for (int k2 = 0; k2 < 3; ++k2)
+        for (int k2 = 0; k2 < 3; ++k2) {
+          float f[RC], o[HC];
+#pragma unroll
+          for (int m = 0; m < RP; ++m) { f[2 * m] = cc[k2][m].x; f[2 * m + 1] = cc[k2][m].y; }
 #pragma unroll
           for (int c = 0; c < HC; ++c) {
-            const float send = up ? cc[k2][c] : cc[k2][c + HC];
-            const float keep = up ? cc[k2][c + HC] : cc[k2][c];
-            part[t & 1][warp][k2][col0 + (up ? HC : 0) + c] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+            const float send = up ? f[c] : f[c + HC];
+            const float keep = up ? f[c + HC] : f[c];
+            o[c] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
           }
+          bwd_st<HC>(part[t & 1][warp][k2] + col0 + (up ? HC : 0), o);
+        }
       } else {
 #pragma unroll
-        for (int k2 = 0; k2 < 3; ++k2)
+        for (int k2 = 0; k2 < 3; ++k2) {
+          float f[RC];
 #pragma unroll
-          for (int c = 0; c < RC; ++c) part[t & 1][warp][k2][col0 + c] = cc[k2][c];
+          for (int m = 0; m < RP; ++m) { f[2 * m] = cc[k2][m].x; f[2 * m + 1] = cc[k2][m].y; }
+          bwd_st<RC>(part[t & 1][warp][k2] + col0, f);
+        }
       }
+      float qv[RC], kv[RC], av[RC];
+      bwd_ld<RC>(cvec(t, cQf) + col0, qv);
+      bwd_ld<RC>(cvec(t, cKh) + col0, kv);
+      bwd_ld<RC>(cvec(t, cAl) + col0, av);
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        const float er = et[row0 + r];
+        const float2 d2 = make_float2(dyr[r], dyr[r]), e2 = make_float2(-etr[r], -etr[r]);
+        const float2 r2 = make_float2(-der[r], -der[r]);
 #pragma unroll
-        for (int c = 0; c < RC; ++c) {
-          GS[r][c] = fmaf(dyr[r], qf[col0 + c], GS[r][c]);
-          GS[r][c] = fmaf(-der[r], kh[col0 + c], GS[r][c]);
-          S[r][c] = fmaf(-er, al[col0 + c], S[r][c]);
+        for (int m = 0; m < RP; ++m) {
+          GS[r][m] = bwd_ffma2(d2, make_float2(qv[2 * m], qv[2 * m + 1]), GS[r][m]);
+          GS[r][m] = bwd_ffma2(r2, make_float2(kv[2 * m], kv[2 * m + 1]), GS[r][m]);
+          S[r][m] = bwd_ffma2(e2, make_float2(av[2 * m], av[2 * m + 1]), S[r][m]);
         }
       }
       if (t >= 1) row_dots(t - 1);
       cta_sync();
     }
+    if (p.dS0) {
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+      for (int r = 0; r < R; ++r) {
+        float gv[RC];
 #pragma unroll
-      for (int c = 0; c < RC; ++c)
-        if (p.dS0) p.dS0[(size_t(unit) * D + row0 + r) * D + col0 + c] = GS[r][c];
+        for (int m = 0; m < RP; ++m) { gv[2 * m] = GS[r][m].x; gv[2 * m + 1] = GS[r][m].y; }
+        bwd_st<RC>(p.dS0 + (size_t(unit) * D + row0 + r) * D + col0, gv);
+      }
+    }
   }
   cta_sync();
   if (p.dz0)
@@ -342,9 +444,10 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_s_kernel(con
 
 // ------------------------------------------------------------------------------ A side
 template <int D, typename TIn>
-__global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_a_kernel(const BackwardSplitParams p) {
+__global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vla_backward_a_kernel(const BackwardSplitParams p) {
   using G = BwdSplitGeom<D>;
-  constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW, NT = G::NT;
+  constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW;
+  constexpr int RP = RC / 2;
   constexpr int EPL = D / 32;
   constexpr int NCTX = 4;
   enum { cKf = 0, cKh, cZt, cDa, cDkS, cGz, NV };
@@ -366,6 +469,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_a_kernel(con
   const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ty = tid / TX, tx = tid % TX;
   const int row0 = ty * R, col0 = tx * RC;
+  const int c0 = lane * EPL;
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
   const float eps = p.eps;
   const int T = p.T;
@@ -374,195 +478,69 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_a_kernel(con
   const float* zst = p.zst + ubase;
   const float* dst = p.dst + size_t(unit) * T;
 
-  float A[R][RC], GA[R][RC];
-#pragma unroll
-  for (int r = 0; r < R; ++r)
-#pragma unroll
-    for (int c = 0; c < RC; ++c) {
-      const size_t idx = (size_t(unit) * D + row0 + r) * D + col0 + c;
-      const bool own = warp < NW;   // the helper warp holds no block
-      A[r][c] = own ? p.AT[idx] : 0.0f;
-      GA[r][c] = (own && p.dA_T) ? p.dA_T[idx] : 0.0f;
-    }
-
   auto cvec = [&](int t, int which) { return ctx[t & (NCTX - 1)][which]; };
-  // after rows_reduce<R, TX / 2> a lane holds the total of row myrow of its group's R rows
   const int myrow = tx / (TX / R);
   const bool row_writer = (tx % (TX / R)) == 0;
+  constexpr int kCloser = NW, kOpener = NW + 1;
 
-  float pk[EPL], pz[EPL], pa[EPL], ps[EPL], pgz[EPL];
-  float pdelta = 1.0f;
-  auto fetch_token = [&](int t) {
-    if (t < 0) return;
-    pdelta = dst[t];
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      pk[e] = load1<TIn>(gk, size_t(t) * D + c);
-      pz[e] = zst[size_t(t) * D + c];
-      pa[e] = p.dal[ubase + size_t(t) * D + c];
-      ps[e] = p.dkS[ubase + size_t(t) * D + c];
-      pgz[e] = p.gzt[ubase + size_t(t) * D + c];
-    }
-  };
-  // one warp: k_hat, alpha, da = (dalpha - alpha (alpha.dalpha)) / ||a|| and the scalars of token t
-  auto open_token = [&](int t) {
-    float* okf = cvec(t, cKf); float* okh = cvec(t, cKh); float* ozt = cvec(t, cZt);
-    float* oda = cvec(t, cDa); float* odk = cvec(t, cDkS); float* ogz = cvec(t, cGz);
-    float kx[EPL];
-    float ss = 0.f, zz = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      float kk = pk[e];
-      if (!ident) kk = bwd_phi(kk);
-      kx[e] = kk;
-      ss = fmaf(kk, kk, ss);
-      zz = fmaf(pz[e], pz[e], zz);
-    }
-    ss = warp_sum(ss);
-    zz = warp_sum(zz);
-    const float nk = fmaxf(sqrtf(ss), eps);
-    const float idl = 1.0f / pdelta;
-    const float na = sqrtf(zz) * idl;              // ||a||, a = z / delta
-    const float sc = idl / fmaxf(na, eps);
-    float adal = 0.f, khz = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      adal = fmaf(sc * pz[e], pa[e], adal);
-      khz = fmaf(kx[e] / nk, pz[e], khz);
-    }
-    adal = warp_sum(adal);
-    khz = warp_sum(khz);
-    float daz = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      const float al = sc * pz[e];
-      const float da = na > eps ? (pa[e] - al * adal) / na : pa[e] / eps;
-      okf[c] = kx[e];
-      okh[c] = kx[e] / nk;
-      ozt[c] = pz[e];
-      oda[c] = da;
-      odk[c] = ps[e];
-      ogz[c] = pgz[e];
-      daz = fmaf(da, pz[e], daz);
-    }
-    daz = warp_sum(daz);
-    if (lane == 0) {
-      float* os = cscl[t & (NCTX - 1)];
-      os[sDelta] = pdelta; os[sKhz] = khz; os[sDaz] = daz; os[sNk] = sqrtf(ss);
-    }
-  };
-  // every matrix warp: dz, ddelta of token t from gaz and the column sums, each warp for itself
-  // (a copy of dz per warp: no CTA barrier between this and the updates that need it)
-  auto mid_token = [&](int t) {
-    const int par = t & 1;
-    const float* kh = cvec(t, cKh); const float* zt = cvec(t, cZt); const float* da = cvec(t, cDa);
-    const float* gaz = rowv[t % 3][0];
-    const float delta = cscl[t & (NCTX - 1)][sDelta], khz = cscl[t & (NCTX - 1)][sKhz];
-    const float daz = cscl[t & (NCTX - 1)][sDaz];
-    float wx[EPL], c4[EPL];
-    float zw = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      float s = 0.f;
-#pragma unroll
-      for (int w = 0; w < NW; ++w) s += part[par][w][c];
-      c4[e] = s;
-      wx[e] = gaz[c] + da[c] * khz;                         // (GA + da k_hat^T) z
-      zw = fmaf(zt[c], wx[e], zw);
-    }
-    zw = warp_sum(zw);
-    const bool delta_live = (1.0f + khz) >= eps;
-    const float ddelta = delta_live ? zw / (delta * delta) : 0.0f;
-    float zdz = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      const float dz = -(wx[e] + c4[e] + kh[c] * daz) / delta + ddelta * kh[c];
-      dzw[warp][c] = dz;
-      zdz = fmaf(zt[c], dz, zdz);
-    }
-    zdz = warp_sum(zdz);
-    if (warp == 0 && lane == 0) { rscl[par][0] = ddelta; rscl[par][1] = zdz; }
-    __syncwarp();
-  };
-  // helper warp: dk of token t
-  auto close_token = [&](int t) {
-    const int par = t & 1;
-    const float* kf = cvec(t, cKf); const float* kh = cvec(t, cKh); const float* zt = cvec(t, cZt);
-    const float* dkS = cvec(t, cDkS); const float* gzv = cvec(t, cGz);
-    const float* r1 = rowv[t % 3][1]; const float* r3 = rowv[t % 3][2];
-    const float ddelta = rscl[par][0], zdz = rscl[par][1];
-    const float delta = cscl[t & (NCTX - 1)][sDelta], nkraw = cscl[t & (NCTX - 1)][sNk];
-    const float nk = fmaxf(nkraw, eps);
-    float dkhx[EPL];
-    float kd = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      const float du = ddelta * zt[c] + r3[c] + zt[c] * (zdz / delta);   // ddelta z + A dz
-      dkhx[e] = dkS[c] + r1[c] + du;
-      kd = fmaf(kh[c], dkhx[e], kd);
-    }
-    kd = warp_sum(kd);
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) {
-      const int c = e * 32 + lane;
-      float dkf = nkraw > eps ? (dkhx[e] - kh[c] * kd) / nk : dkhx[e] / eps;
-      if (!ident) {
-        dkf += gzv[c];
-        dkf *= kf[c] > 1.0f ? 1.0f : kf[c];     // phi'(k) from phi(k)
-      }
-      p.dk[ubase + size_t(t) * D + c] = dkf;
-    }
-  };
-  // gaz = GA z, r1 = A' da and the column partials of GA^T z for token t
-  auto products = [&](int t) {
-    const float* zt = cvec(t, cZt); const float* da = cvec(t, cDa);
-    float a0[R], a1[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      float x0 = 0.f, x1 = 0.f;
-#pragma unroll
-      for (int c = 0; c < RC; ++c) {
-        x0 = fmaf(GA[r][c], zt[col0 + c], x0);
-        x1 = fmaf(A[r][c], da[col0 + c], x1);
-      }
-      a0[r] = x0; a1[r] = x1;
-    }
-    rows_reduce<R, TX / 2>(a0, lane);
-    rows_reduce<R, TX / 2>(a1, lane);
-    if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
-    float cc[RC];
-#pragma unroll
-    for (int c = 0; c < RC; ++c) {
-      float s2 = 0.f;
-#pragma unroll
-      for (int r = 0; r < R; ++r) s2 = fmaf(GA[r][c], zt[row0 + r], s2);
-      cc[c] = s2;
-    }
-    if constexpr (TX == 16) {
-      constexpr int HC = RC / 2;
-      const bool up = (lane & 16) != 0;
-#pragma unroll
-      for (int c = 0; c < HC; ++c) {
-        const float send = up ? cc[c] : cc[c + HC];
-        const float keep = up ? cc[c + HC] : cc[c];
-        part[t & 1][warp][col0 + (up ? HC : 0) + c] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-      }
-    } else {
-#pragma unroll
-      for (int c = 0; c < RC; ++c) part[t & 1][warp][col0 + c] = cc[c];
-    }
-  };
-
-  constexpr int kHelper = NW;
   // Segment t (one CTA barrier): the matrix warps form dz of token t, r3 = A' dz, the two
-  // rank-1 updates, then the products of token t - 1; the helper warp closes token t + 1 and
-  // opens token t - 2.  Two loops with the same number of barriers, as on the S side.
-  if (warp == kHelper) {
+  // rank-1 updates, then the products of token t - 1; the closing warp finishes token t + 1,
+  // the opening warp prepares token t - 2.  Loops of their own, as on the S side.
+  if (warp == kOpener) {
+    float pk[EPL], pz[EPL], pa[EPL], ps[EPL], pgz[EPL];
+    float pdelta = 1.0f;
+    auto fetch_token = [&](int t) {
+      if (t < 0) return;
+      pdelta = dst[t];
+      const size_t o = size_t(t) * D + c0;
+      bwd_ld_in<EPL>(gk + o, pk);
+      bwd_ld<EPL>(zst + o, pz);
+      bwd_ld<EPL>(p.dal + ubase + o, pa);
+      bwd_ld<EPL>(p.dkS + ubase + o, ps);
+      bwd_ld<EPL>(p.gzt + ubase + o, pgz);
+    };
+    // k_hat, alpha, da = (dalpha - alpha (alpha.dalpha)) / ||a|| and the scalars of token t
+    auto open_token = [&](int t) {
+      float kx[EPL], khx[EPL], dax[EPL];
+      float ss = 0.f, zz = 0.f, zpa = 0.f, kz = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        float kk = pk[e];
+        if (!ident) kk = bwd_phi(kk);
+        kx[e] = kk;
+        ss = fmaf(kk, kk, ss);
+        zz = fmaf(pz[e], pz[e], zz);
+        zpa = fmaf(pz[e], pa[e], zpa);
+        kz = fmaf(kk, pz[e], kz);
+      }
+      ss = warp_sum(ss); zz = warp_sum(zz); zpa = warp_sum(zpa); kz = warp_sum(kz);
+      const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
+      const float idl = 1.0f / pdelta;
+      const float na = sqrtf(zz) * idl;              // ||a||, a = z / delta
+      const float sc = idl / fmaxf(na, eps);
+      const float adal = sc * zpa;                   // alpha . dalpha
+      const float khz = kz * ink;
+      const float ina = na > eps ? 1.0f / na : 1.0f / eps;
+      float daz = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        const float al = sc * pz[e];
+        dax[e] = na > eps ? (pa[e] - al * adal) * ina : pa[e] * ina;
+        khx[e] = kx[e] * ink;
+        daz = fmaf(dax[e], pz[e], daz);
+      }
+      daz = warp_sum(daz);
+      bwd_st<EPL>(cvec(t, cKf) + c0, kx);
+      bwd_st<EPL>(cvec(t, cKh) + c0, khx);
+      bwd_st<EPL>(cvec(t, cZt) + c0, pz);
+      bwd_st<EPL>(cvec(t, cDa) + c0, dax);
+      bwd_st<EPL>(cvec(t, cDkS) + c0, ps);
+      bwd_st<EPL>(cvec(t, cGz) + c0, pgz);
+      if (lane == 0) {
+        float* os = cscl[t & (NCTX - 1)];
+        os[sDelta] = pdelta; os[sKhz] = khz; os[sDaz] = daz; os[sNk] = sqrtf(ss);
+      }
+    };
     if (T > 0) {
       fetch_token(T - 1);
       open_token(T - 1);
@@ -573,52 +551,205 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT) vla_backward_a_kernel(con
     cta_sync();
     cta_sync();
     for (int t = T - 1; t >= 0; --t) {
-      if (t + 1 <= T - 1) close_token(t + 1);
       if (t - 2 >= 0) {
         open_token(t - 2);
         fetch_token(t - 3);
       }
       cta_sync();
     }
+  } else if (warp == kCloser) {
+    // dk of token t
+    auto close_token = [&](int t) {
+      const int par = t & 1;
+      float kf[EPL], kh[EPL], zt[EPL], dkS[EPL], gzv[EPL], r1[EPL], r3[EPL];
+      bwd_ld<EPL>(cvec(t, cKf) + c0, kf);
+      bwd_ld<EPL>(cvec(t, cKh) + c0, kh);
+      bwd_ld<EPL>(cvec(t, cZt) + c0, zt);
+      bwd_ld<EPL>(cvec(t, cDkS) + c0, dkS);
+      bwd_ld<EPL>(cvec(t, cGz) + c0, gzv);
+      bwd_ld<EPL>(rowv[t % 3][1] + c0, r1);
+      bwd_ld<EPL>(rowv[t % 3][2] + c0, r3);
+      const float ddelta = rscl[par][0], zdz = rscl[par][1];
+      const float delta = cscl[t & (NCTX - 1)][sDelta], nkraw = cscl[t & (NCTX - 1)][sNk];
+      const float ink = nkraw > eps ? 1.0f / nkraw : 1.0f / eps;
+      const float zs = ddelta + zdz / delta;
+      float dkhx[EPL], out[EPL];
+      float kd = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        dkhx[e] = dkS[e] + r1[e] + fmaf(zt[e], zs, r3[e]);   // + ddelta z + A dz
+        kd = fmaf(kh[e], dkhx[e], kd);
+      }
+      kd = warp_sum(kd);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        float dkf = nkraw > eps ? (dkhx[e] - kh[e] * kd) * ink : dkhx[e] * ink;
+        if (!ident) {
+          dkf += gzv[e];
+          dkf *= kf[e] > 1.0f ? 1.0f : kf[e];     // phi'(k) from phi(k)
+        }
+        out[e] = dkf;
+      }
+      bwd_st<EPL>(p.dk + ubase + size_t(t) * D + c0, out);
+    };
+    cta_sync();
+    cta_sync();
+    for (int t = T - 1; t >= 0; --t) {
+      if (t + 1 <= T - 1) close_token(t + 1);
+      cta_sync();
+    }
     if (T > 0) close_token(0);
   } else {
+    float2 A[R][RP], GA[R][RP];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const size_t idx = (size_t(unit) * D + row0 + r) * D + col0;
+      float sv[RC], gv[RC];
+      bwd_ld<RC>(p.AT + idx, sv);
+      if (p.dA_T) {
+        bwd_ld<RC>(p.dA_T + idx, gv);
+      } else {
+#pragma unroll
+        for (int c = 0; c < RC; ++c) gv[c] = 0.0f;
+      }
+#pragma unroll
+      for (int m = 0; m < RP; ++m) {
+        A[r][m] = make_float2(sv[2 * m], sv[2 * m + 1]);
+        GA[r][m] = make_float2(gv[2 * m], gv[2 * m + 1]);
+      }
+    }
+    // gaz = GA z, r1 = A' da and the column partials of GA^T z for token t
+    auto products = [&](int t) {
+      float zc[RC], dc[RC], zr[R];
+      bwd_ld<RC>(cvec(t, cZt) + col0, zc);
+      bwd_ld<RC>(cvec(t, cDa) + col0, dc);
+      bwd_ld<R>(cvec(t, cZt) + row0, zr);
+      float a0[R], a1[R];
+      float2 cc[RP];
+#pragma unroll
+      for (int m = 0; m < RP; ++m) cc[m] = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+        const float2 z2 = make_float2(zr[r], zr[r]);
+#pragma unroll
+        for (int m = 0; m < RP; ++m) {
+          x0 = bwd_ffma2(GA[r][m], make_float2(zc[2 * m], zc[2 * m + 1]), x0);
+          x1 = bwd_ffma2(A[r][m], make_float2(dc[2 * m], dc[2 * m + 1]), x1);
+          cc[m] = bwd_ffma2(GA[r][m], z2, cc[m]);
+        }
+        a0[r] = x0.x + x0.y; a1[r] = x1.x + x1.y;
+      }
+      rows_reduce<R, TX / 2>(a0, lane);
+      rows_reduce<R, TX / 2>(a1, lane);
+      if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
+      float f[RC];
+#pragma unroll
+      for (int m = 0; m < RP; ++m) { f[2 * m] = cc[m].x; f[2 * m + 1] = cc[m].y; }
+      if constexpr (TX == 16) {
+        constexpr int HC = RC / 2;
+        const bool up = (lane & 16) != 0;
+        float o[HC];
+#pragma unroll
+        for (int c = 0; c < HC; ++c) {
+          const float send = up ? f[c] : f[c + HC];
+          const float keep = up ? f[c + HC] : f[c];
+          o[c] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        }
+        bwd_st<HC>(part[t & 1][warp] + col0 + (up ? HC : 0), o);
+      } else {
+        bwd_st<RC>(part[t & 1][warp] + col0, f);
+      }
+    };
+    // dz, ddelta of token t from gaz and the column sums, each matrix warp for itself (a copy
+    // of dz per warp: no CTA barrier between this and the updates that need it)
+    auto mid_token = [&](int t) {
+      const int par = t & 1;
+      float kh[EPL], zt[EPL], da[EPL], wx[EPL], c4[EPL];
+      bwd_ld<EPL>(cvec(t, cKh) + c0, kh);
+      bwd_ld<EPL>(cvec(t, cZt) + c0, zt);
+      bwd_ld<EPL>(cvec(t, cDa) + c0, da);
+      bwd_ld<EPL>(rowv[t % 3][0] + c0, wx);
+      const float delta = cscl[t & (NCTX - 1)][sDelta], khz = cscl[t & (NCTX - 1)][sKhz];
+      const float daz = cscl[t & (NCTX - 1)][sDaz];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) c4[e] = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        float x[EPL];
+        bwd_ld<EPL>(part[par][w] + c0, x);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) c4[e] += x[e];
+      }
+      float zw = 0.f, zc = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        wx[e] = fmaf(da[e], khz, wx[e]);                    // (GA + da k_hat^T) z
+        zw = fmaf(zt[e], wx[e], zw);
+        zc = fmaf(zt[e], c4[e], zc);
+      }
+      zw = warp_sum(zw);
+      zc = warp_sum(zc);
+      const bool delta_live = (1.0f + khz) >= eps;
+      const float idl = 1.0f / delta;
+      const float ddelta = delta_live ? zw * idl * idl : 0.0f;
+      float dz[EPL];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e)
+        dz[e] = fmaf(ddelta, kh[e], -(wx[e] + c4[e] + kh[e] * daz) * idl);
+      bwd_st<EPL>(dzw[warp] + c0, dz);
+      if (warp == 0 && lane == 0) {
+        rscl[par][0] = ddelta;
+        rscl[par][1] = fmaf(ddelta, khz, -(zw + zc + khz * daz) * idl);   // z . dz
+      }
+      __syncwarp();
+    };
     cta_sync();
     if (T > 0) products(T - 1);
     cta_sync();
     for (int t = T - 1; t >= 0; --t) {
       mid_token(t);
-      const float* kh = cvec(t, cKh); const float* zt = cvec(t, cZt); const float* da = cvec(t, cDa);
-      const float* dz = dzw[warp];
-      const float delta = cscl[t & (NCTX - 1)][sDelta];
+      const float idl = 1.0f / cscl[t & (NCTX - 1)][sDelta];
+      float dzc[RC], dzr[R], zr[R], dar[R], kc[RC], zc[RC];
+      bwd_ld<RC>(dzw[warp] + col0, dzc);
+      bwd_ld<R>(dzw[warp] + row0, dzr);
+      bwd_ld<R>(cvec(t, cZt) + row0, zr);
+      bwd_ld<R>(cvec(t, cDa) + row0, dar);
+      bwd_ld<RC>(cvec(t, cKh) + col0, kc);
+      bwd_ld<RC>(cvec(t, cZt) + col0, zc);
       float b1[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        float x1 = 0.f;
+        float2 x1 = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < RC; ++c) x1 = fmaf(A[r][c], dz[col0 + c], x1);
-        b1[r] = x1;
+        for (int m = 0; m < RP; ++m) x1 = bwd_ffma2(A[r][m], make_float2(dzc[2 * m], dzc[2 * m + 1]), x1);
+        b1[r] = x1.x + x1.y;
       }
       rows_reduce<R, TX / 2>(b1, lane);
       if (row_writer) rowv[t % 3][2][row0 + myrow] = b1[0];
-      const float idl = 1.0f / delta;
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        const float zr = zt[row0 + r], dadz = da[row0 + r] + dz[row0 + r];
+        const float dadz = dar[r] + dzr[r], zs = zr[r] * idl;
+        const float2 g2 = make_float2(dadz, dadz), z2 = make_float2(zs, zs);
 #pragma unroll
-        for (int c = 0; c < RC; ++c) {
-          GA[r][c] = fmaf(dadz, kh[col0 + c], GA[r][c]);
-          A[r][c] = fmaf(zr * idl, zt[col0 + c], A[r][c]);
+        for (int m = 0; m < RP; ++m) {
+          GA[r][m] = bwd_ffma2(g2, make_float2(kc[2 * m], kc[2 * m + 1]), GA[r][m]);
+          A[r][m] = bwd_ffma2(z2, make_float2(zc[2 * m], zc[2 * m + 1]), A[r][m]);
         }
       }
       __syncwarp();   // this warp's dz copy is rewritten in the next segment
       if (t >= 1) products(t - 1);
       cta_sync();
     }
+    if (p.dA0) {
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+      for (int r = 0; r < R; ++r) {
+        float gv[RC];
 #pragma unroll
-      for (int c = 0; c < RC; ++c)
-        if (p.dA0) p.dA0[(size_t(unit) * D + row0 + r) * D + col0 + c] = GA[r][c];
+        for (int m = 0; m < RP; ++m) { gv[2 * m] = GA[r][m].x; gv[2 * m + 1] = GA[r][m].y; }
+        bwd_st<RC>(p.dA0 + (size_t(unit) * D + row0 + r) * D + col0, gv);
+      }
+    }
   }
 }
 

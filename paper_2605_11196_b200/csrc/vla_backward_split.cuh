@@ -7,7 +7,8 @@
 //     vectors for the other side: dalpha_t = dL/d alpha_t, the S-side part of dL/d k_hat_t, and
 //     the running gradient of the key sum.
 //   A side (vla_backward_a_kernel): A and GA = dL/dA in registers.  Per token it turns dalpha_t
-//     into da, forms dz, ddelta and the remaining parts of dL/d k_hat_t, and writes dk.
+//     into da, forms dz, ddelta and the remaining parts of dL/d k_hat_t, and writes dk.  It
+//     carries the symmetric part of GA only; dA0 is formed afterwards (vla_backward_da0_kernel).
 //
 // each a CTA per unit holding TWO d x d matrices in registers, as R x RC blocks on a grid of
 // 16 x TX threads (R = d / 16 rows, RC = d / TX columns; TX = 16, or 32 at d = 128, where the
@@ -20,8 +21,8 @@
 //
 // Both kernels keep a ring of four per-token contexts in shared memory.  Opening a token
 // (loading its rows, alpha, denominators: nothing that depends on the adjoints) and closing one
-// (vector arithmetic on finished products, the stores) are done by two helper warps off the
-// path of the TX / 2 matrix warps; one CTA barrier per token.
+// (vector arithmetic on finished products, the stores) are done by helper warps off the path
+// of the TX / 2 matrix warps; one CTA barrier per token.
 #pragma once
 
 #include "vla_backward.cuh"
@@ -34,8 +35,10 @@ struct BwdSplitGeom {
   static constexpr int TX = D >= 128 ? 32 : 16;   // threads along a matrix row
   static constexpr int R = D / 16;                // rows of a thread's block
   static constexpr int RC = D / TX;               // columns of a thread's block
-  static constexpr int NW = TX / 2;               // matrix warps; warp NW closes, warp NW + 1 opens tokens
-  static constexpr int NT = NW * 32 + 64;
+  static constexpr int NW = TX / 2;               // matrix warps
+  static constexpr int NCLOSE = D >= 128 ? 2 : 1; // warps closing tokens on the S side (the sums over NW partials)
+  static constexpr int NT_S = (NW + NCLOSE + 1) * 32;   // S side: matrix warps, closers, one opener
+  static constexpr int NT_A = (NW + 2) * 32;            // A side: matrix warps, one closer, one opener
   static constexpr int MINB = D == 64 ? 3 : 1;    // CTAs per SM the register budget is held to
 };
 
@@ -44,7 +47,7 @@ template <int D>
 struct BackwardSplitSmem {
   static constexpr int NW = BwdSplitGeom<D>::NW;
   static constexpr size_t s_bytes = sizeof(float) * (4 * 8 * D + 4 * 4 + 3 * 2 * D + 2 * NW * 3 * D + D);
-  static constexpr size_t a_bytes = sizeof(float) * (4 * 6 * D + 4 * 4 + 3 * 3 * D + 2 * NW * D + NW * D + 4);
+  static constexpr size_t a_bytes = sizeof(float) * (4 * 6 * D + 4 * 4 + 3 * 3 * D);
 };
 
 // All threads of the CTA, whichever loop they are in.
@@ -122,9 +125,9 @@ __device__ __forceinline__ void rows_reduce(float* v, int lane) {
 
 // ------------------------------------------------------------------------------ S side
 template <int D, typename TIn>
-__global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vla_backward_s_kernel(const BackwardSplitParams p) {
+__global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) vla_backward_s_kernel(const BackwardSplitParams p) {
   using G = BwdSplitGeom<D>;
-  constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW, NT = G::NT;
+  constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW, NT = G::NT_S, NCLOSE = G::NCLOSE;
   constexpr int RP = RC / 2;          // column pairs of a block
   constexpr int EPL = D / 32;         // consecutive vector elements per lane of a helper warp
   constexpr int NCTX = 4;
@@ -163,7 +166,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
   // after rows_reduce<R, TX / 2> a lane holds the total of row myrow of its group's R rows
   const int myrow = tx / (TX / R);
   const bool row_writer = (tx % (TX / R)) == 0;
-  constexpr int kCloser = NW, kOpener = NW + 1;
+  constexpr int kCloser = NW, kOpener = NW + NCLOSE;   // warps kCloser .. kOpener - 1 close tokens
 
   // Segment t (one CTA barrier): the matrix warps take the column sums and the two rank-1
   // updates of token t, then the row dots of token t - 1; the closing warp finishes token
@@ -254,64 +257,85 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
       }
       cta_sync();
     }
-  } else if (warp == kCloser) {
-    // the vector results of token t from its finished products
+  } else if (warp >= kCloser) {
+    // The vector results of token t from its finished products.  The query part (dq, the
+    // gradient of the key sum) and the key part (dv, dalpha, dk_hat) share nothing but their
+    // inputs: one warp does both, or one warp each.
+    const bool do_q = NCLOSE == 1 || warp == kCloser;
+    const bool do_k = NCLOSE == 1 || warp == kCloser + 1;
     auto close_token = [&](int t) {
       const int par = t & 1;
-      float go[EPL], dy[EPL], et[EPL], al[EPL], qf[EPL], zkt[EPL], yv[EPL], g1[EPL];
-      bwd_ld<EPL>(cvec(t, cGo) + c0, go);
-      bwd_ld<EPL>(cvec(t, cDy) + c0, dy);
-      bwd_ld<EPL>(cvec(t, cEt) + c0, et);
-      bwd_ld<EPL>(rowv[t % 3][0] + c0, yv);
-      bwd_ld<EPL>(rowv[t % 3][1] + c0, g1);
-      const float den = cscl[t & (NCTX - 1)][sDen], qal = cscl[t & (NCTX - 1)][sQal];
-      const bool den_live = cscl[t & (NCTX - 1)][sDenLive] != 0.0f;
-      float odo = 0.f, ede = 0.f, dye = 0.f;
-      float dex[EPL];
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        dex[e] = fmaf(dy[e], qal, g1[e]);
-        odo = fmaf(yv[e], go[e], odo);
-        ede = fmaf(et[e], dex[e], ede);
-        dye = fmaf(dy[e], et[e], dye);
-      }
-      float c1[EPL], c2[EPL], c3[EPL];
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) { c1[e] = 0.f; c2[e] = 0.f; c3[e] = 0.f; }
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        float x1[EPL], x2[EPL], x3[EPL];
-        bwd_ld<EPL>(part[par][w][0] + c0, x1);
-        bwd_ld<EPL>(part[par][w][1] + c0, x2);
-        bwd_ld<EPL>(part[par][w][2] + c0, x3);
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) { c1[e] += x1[e]; c2[e] += x2[e]; c3[e] += x3[e]; }
-      }
-      bwd_ld<EPL>(cvec(t, cAl) + c0, al);
-      bwd_ld<EPL>(cvec(t, cQf) + c0, qf);
-      bwd_ld<EPL>(cvec(t, cZk) + c0, zkt);
-      odo = warp_sum(odo); ede = warp_sum(ede); dye = warp_sum(dye);
-      const float dden = den_live ? -odo / (den * den) : 0.0f;
-      float gzc[EPL], dq[EPL], dalo[EPL], dko[EPL], gzo[EPL];
-      bwd_ld<EPL>(gz + c0, gzc);
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        dq[e] = fmaf(dden, zkt[e], c1[e]);
-        if (!ident) {
-          dq[e] *= qf[e] > 1.0f ? 1.0f : qf[e];     // phi'(q) from phi(q)
-          gzc[e] = fmaf(dden, qf[e], gzc[e]);
-        }
-        dalo[e] = fmaf(qf[e], dye, c2[e]);          // (GS + dy qf^T)^T e
-        dko[e] = -(c3[e] - al[e] * ede);            // -(S' - e alpha^T)^T de
-        gzo[e] = ident ? 0.0f : gzc[e];
-      }
-      if (!ident) bwd_st<EPL>(gz + c0, gzc);
       const size_t tb = ubase + size_t(t) * D + c0;
-      bwd_st<EPL>(p.dq + tb, dq);
-      bwd_st<EPL>(p.dv + tb, dex);
-      bwd_st<EPL>(p.dal + tb, dalo);
-      bwd_st<EPL>(p.dkS + tb, dko);
-      bwd_st<EPL>(p.gzt + tb, gzo);
+      if (do_q) {
+        float go[EPL], qf[EPL], zkt[EPL], yv[EPL], c1[EPL];
+        bwd_ld<EPL>(cvec(t, cGo) + c0, go);
+        bwd_ld<EPL>(rowv[t % 3][0] + c0, yv);
+        const float den = cscl[t & (NCTX - 1)][sDen];
+        const bool den_live = cscl[t & (NCTX - 1)][sDenLive] != 0.0f;
+        float odo = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) { odo = fmaf(yv[e], go[e], odo); c1[e] = 0.f; }
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+          float x1[EPL];
+          bwd_ld<EPL>(part[par][w][0] + c0, x1);
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) c1[e] += x1[e];
+        }
+        bwd_ld<EPL>(cvec(t, cQf) + c0, qf);
+        bwd_ld<EPL>(cvec(t, cZk) + c0, zkt);
+        odo = warp_sum(odo);
+        const float dden = den_live ? -odo / (den * den) : 0.0f;
+        float gzc[EPL], dq[EPL], gzo[EPL];
+        bwd_ld<EPL>(gz + c0, gzc);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          dq[e] = fmaf(dden, zkt[e], c1[e]);
+          if (!ident) {
+            dq[e] *= qf[e] > 1.0f ? 1.0f : qf[e];     // phi'(q) from phi(q)
+            gzc[e] = fmaf(dden, qf[e], gzc[e]);
+          }
+          gzo[e] = ident ? 0.0f : gzc[e];
+        }
+        if (!ident) bwd_st<EPL>(gz + c0, gzc);
+        bwd_st<EPL>(p.dq + tb, dq);
+        bwd_st<EPL>(p.gzt + tb, gzo);
+      }
+      if (do_k) {
+        float dy[EPL], et[EPL], al[EPL], qf[EPL], g1[EPL], dex[EPL], c2[EPL], c3[EPL];
+        bwd_ld<EPL>(cvec(t, cDy) + c0, dy);
+        bwd_ld<EPL>(cvec(t, cEt) + c0, et);
+        bwd_ld<EPL>(rowv[t % 3][1] + c0, g1);
+        const float qal = cscl[t & (NCTX - 1)][sQal];
+        float ede = 0.f, dye = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          dex[e] = fmaf(dy[e], qal, g1[e]);
+          ede = fmaf(et[e], dex[e], ede);
+          dye = fmaf(dy[e], et[e], dye);
+          c2[e] = 0.f; c3[e] = 0.f;
+        }
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+          float x2[EPL], x3[EPL];
+          bwd_ld<EPL>(part[par][w][1] + c0, x2);
+          bwd_ld<EPL>(part[par][w][2] + c0, x3);
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) { c2[e] += x2[e]; c3[e] += x3[e]; }
+        }
+        bwd_ld<EPL>(cvec(t, cAl) + c0, al);
+        bwd_ld<EPL>(cvec(t, cQf) + c0, qf);
+        ede = warp_sum(ede); dye = warp_sum(dye);
+        float dalo[EPL], dko[EPL];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          dalo[e] = fmaf(qf[e], dye, c2[e]);          // (GS + dy qf^T)^T e
+          dko[e] = -(c3[e] - al[e] * ede);            // -(S' - e alpha^T)^T de
+        }
+        bwd_st<EPL>(p.dv + tb, dex);
+        bwd_st<EPL>(p.dal + tb, dalo);
+        bwd_st<EPL>(p.dkS + tb, dko);
+      }
     };
     cta_sync();
     cta_sync();
@@ -443,8 +467,13 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
 }
 
 // ------------------------------------------------------------------------------ A side
+// GA enters the sweep only through (GA + GA^T) z and z^T GA z, so the kernel carries the
+// symmetric part GAs = (GA + GA^T) / 2: both products become row dots of one matrix (no column
+// sums, nothing to combine across warps), and the update GA += w k_hat^T, w = da + dz, becomes
+// GAs += (w k_hat^T + k_hat w^T) / 2.  GA itself is needed for dA0 alone and is linear in the
+// w_t: dA0 = dA_T + sum_t w_t k_hat_t^T, formed from the stored w_t by vla_backward_da0_kernel.
 template <int D, typename TIn>
-__global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vla_backward_a_kernel(const BackwardSplitParams p) {
+__global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) vla_backward_a_kernel(const BackwardSplitParams p) {
   using G = BwdSplitGeom<D>;
   constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW;
   constexpr int RP = RC / 2;
@@ -455,16 +484,12 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
   struct Smem {
     float ctx[NCTX][NV][D];
     float cscl[NCTX][4];
-    float rowv[3][3][D];      // gaz = GA z, r1 = A' da, r3 = A' dz, ring of three tokens
-    float part[2][NW][D];     // column-sum partials GA^T z by token parity and warp
-    float dzw[NW][D];         // dz of the token in hand, one copy per matrix warp
-    float rscl[2][2];         // ddelta, z.dz by token parity
+    float rowv[3][3][D];      // g = GAs z, r1 = A' da, r3 = A' dz, ring of three tokens
   };
   static_assert(sizeof(Smem) == BackwardSplitSmem<D>::a_bytes, "shared memory size of the A side");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
-  auto& ctx = sm.ctx; auto& cscl = sm.cscl; auto& rowv = sm.rowv; auto& part = sm.part;
-  auto& dzw = sm.dzw; auto& rscl = sm.rscl;
+  auto& ctx = sm.ctx; auto& cscl = sm.cscl; auto& rowv = sm.rowv;
 
   const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ty = tid / TX, tx = tid % TX;
@@ -483,9 +508,31 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
   const bool row_writer = (tx % (TX / R)) == 0;
   constexpr int kCloser = NW, kOpener = NW + 1;
 
+  // the scalars of token t that hang on the adjoint: ddelta and the factors of dz
+  //   dz = cK k_hat - idl (2 g + khz da),  cK = ddelta - idl daz,  ddelta = (z.g + daz khz) / delta^2
+  struct MidScalars { float idl, ddelta, cK, khz, zg; };
+  auto mid_scalars = [&](int t) {
+    float zt[EPL], gv[EPL];
+    bwd_ld<EPL>(cvec(t, cZt) + c0, zt);
+    bwd_ld<EPL>(rowv[t % 3][0] + c0, gv);
+    float zg = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) zg = fmaf(zt[e], gv[e], zg);
+    zg = warp_sum(zg);
+    const float* sc = cscl[t & (NCTX - 1)];
+    MidScalars m;
+    m.khz = sc[sKhz];
+    m.idl = 1.0f / sc[sDelta];
+    m.zg = zg;
+    const bool delta_live = (1.0f + m.khz) >= eps;
+    m.ddelta = delta_live ? fmaf(sc[sDaz], m.khz, zg) * m.idl * m.idl : 0.0f;
+    m.cK = fmaf(-m.idl, sc[sDaz], m.ddelta);
+    return m;
+  };
+
   // Segment t (one CTA barrier): the matrix warps form dz of token t, r3 = A' dz, the two
-  // rank-1 updates, then the products of token t - 1; the closing warp finishes token t + 1,
-  // the opening warp prepares token t - 2.  Loops of their own, as on the S side.
+  // updates, then the row dots of token t - 1; the closing warp finishes token t + 1, the
+  // opening warp prepares token t - 2.  Loops of their own, as on the S side.
   if (warp == kOpener) {
     float pk[EPL], pz[EPL], pa[EPL], ps[EPL], pgz[EPL];
     float pdelta = 1.0f;
@@ -558,25 +605,30 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
       cta_sync();
     }
   } else if (warp == kCloser) {
-    // dk of token t
+    // dk of token t; w_t = da + dz goes where dalpha_t was (read two segments ago) for dA0
     auto close_token = [&](int t) {
-      const int par = t & 1;
-      float kf[EPL], kh[EPL], zt[EPL], dkS[EPL], gzv[EPL], r1[EPL], r3[EPL];
+      const MidScalars ms = mid_scalars(t);
+      float kf[EPL], kh[EPL], zt[EPL], da[EPL], dkS[EPL], gzv[EPL], gv[EPL], r1[EPL], r3[EPL];
       bwd_ld<EPL>(cvec(t, cKf) + c0, kf);
       bwd_ld<EPL>(cvec(t, cKh) + c0, kh);
       bwd_ld<EPL>(cvec(t, cZt) + c0, zt);
+      bwd_ld<EPL>(cvec(t, cDa) + c0, da);
       bwd_ld<EPL>(cvec(t, cDkS) + c0, dkS);
       bwd_ld<EPL>(cvec(t, cGz) + c0, gzv);
+      bwd_ld<EPL>(rowv[t % 3][0] + c0, gv);
       bwd_ld<EPL>(rowv[t % 3][1] + c0, r1);
       bwd_ld<EPL>(rowv[t % 3][2] + c0, r3);
-      const float ddelta = rscl[par][0], zdz = rscl[par][1];
-      const float delta = cscl[t & (NCTX - 1)][sDelta], nkraw = cscl[t & (NCTX - 1)][sNk];
+      const float nkraw = cscl[t & (NCTX - 1)][sNk], daz = cscl[t & (NCTX - 1)][sDaz];
       const float ink = nkraw > eps ? 1.0f / nkraw : 1.0f / eps;
-      const float zs = ddelta + zdz / delta;
-      float dkhx[EPL], out[EPL];
+      // z . dz = cK khz - idl (2 z.g + khz daz);  A dz = A' dz + z (z.dz) / delta
+      const float zdz = fmaf(ms.cK, ms.khz, -ms.idl * fmaf(ms.khz, daz, 2.0f * ms.zg));
+      const float zs = fmaf(zdz, ms.idl, ms.ddelta);
+      float dkhx[EPL], out[EPL], wv[EPL];
       float kd = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
+        const float dz = fmaf(ms.cK, kh[e], -ms.idl * fmaf(ms.khz, da[e], 2.0f * gv[e]));
+        wv[e] = da[e] + dz;
         dkhx[e] = dkS[e] + r1[e] + fmaf(zt[e], zs, r3[e]);   // + ddelta z + A dz
         kd = fmaf(kh[e], dkhx[e], kd);
       }
@@ -591,6 +643,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
         out[e] = dkf;
       }
       bwd_st<EPL>(p.dk + ubase + size_t(t) * D + c0, out);
+      if (p.dA0) bwd_st<EPL>(p.dal + ubase + size_t(t) * D + c0, wv);
     };
     cta_sync();
     cta_sync();
@@ -600,157 +653,158 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT, BwdSplitGeom<D>::MINB) vl
     }
     if (T > 0) close_token(0);
   } else {
-    float2 A[R][RP], GA[R][RP];
+    float2 A[R][RP], GA[R][RP];   // GA: the symmetric part
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       const size_t idx = (size_t(unit) * D + row0 + r) * D + col0;
       float sv[RC], gv[RC];
       bwd_ld<RC>(p.AT + idx, sv);
-      if (p.dA_T) {
-        bwd_ld<RC>(p.dA_T + idx, gv);
-      } else {
 #pragma unroll
-        for (int c = 0; c < RC; ++c) gv[c] = 0.0f;
-      }
+      for (int c = 0; c < RC; ++c)
+        gv[c] = p.dA_T ? 0.5f * (p.dA_T[idx + c] + p.dA_T[(size_t(unit) * D + col0 + c) * D + row0 + r]) : 0.0f;
 #pragma unroll
       for (int m = 0; m < RP; ++m) {
         A[r][m] = make_float2(sv[2 * m], sv[2 * m + 1]);
         GA[r][m] = make_float2(gv[2 * m], gv[2 * m + 1]);
       }
     }
-    // gaz = GA z, r1 = A' da and the column partials of GA^T z for token t
+    // g = GAs z and r1 = A' da for token t
     auto products = [&](int t) {
-      float zc[RC], dc[RC], zr[R];
+      float zc[RC], dc[RC];
       bwd_ld<RC>(cvec(t, cZt) + col0, zc);
       bwd_ld<RC>(cvec(t, cDa) + col0, dc);
-      bwd_ld<R>(cvec(t, cZt) + row0, zr);
       float a0[R], a1[R];
-      float2 cc[RP];
-#pragma unroll
-      for (int m = 0; m < RP; ++m) cc[m] = make_float2(0.f, 0.f);
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
-        const float2 z2 = make_float2(zr[r], zr[r]);
 #pragma unroll
         for (int m = 0; m < RP; ++m) {
           x0 = bwd_ffma2(GA[r][m], make_float2(zc[2 * m], zc[2 * m + 1]), x0);
           x1 = bwd_ffma2(A[r][m], make_float2(dc[2 * m], dc[2 * m + 1]), x1);
-          cc[m] = bwd_ffma2(GA[r][m], z2, cc[m]);
         }
         a0[r] = x0.x + x0.y; a1[r] = x1.x + x1.y;
       }
       rows_reduce<R, TX / 2>(a0, lane);
       rows_reduce<R, TX / 2>(a1, lane);
       if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
-      float f[RC];
-#pragma unroll
-      for (int m = 0; m < RP; ++m) { f[2 * m] = cc[m].x; f[2 * m + 1] = cc[m].y; }
-      if constexpr (TX == 16) {
-        constexpr int HC = RC / 2;
-        const bool up = (lane & 16) != 0;
-        float o[HC];
-#pragma unroll
-        for (int c = 0; c < HC; ++c) {
-          const float send = up ? f[c] : f[c + HC];
-          const float keep = up ? f[c + HC] : f[c];
-          o[c] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-        }
-        bwd_st<HC>(part[t & 1][warp] + col0 + (up ? HC : 0), o);
-      } else {
-        bwd_st<RC>(part[t & 1][warp] + col0, f);
-      }
-    };
-    // dz, ddelta of token t from gaz and the column sums, each matrix warp for itself (a copy
-    // of dz per warp: no CTA barrier between this and the updates that need it)
-    auto mid_token = [&](int t) {
-      const int par = t & 1;
-      float kh[EPL], zt[EPL], da[EPL], wx[EPL], c4[EPL];
-      bwd_ld<EPL>(cvec(t, cKh) + c0, kh);
-      bwd_ld<EPL>(cvec(t, cZt) + c0, zt);
-      bwd_ld<EPL>(cvec(t, cDa) + c0, da);
-      bwd_ld<EPL>(rowv[t % 3][0] + c0, wx);
-      const float delta = cscl[t & (NCTX - 1)][sDelta], khz = cscl[t & (NCTX - 1)][sKhz];
-      const float daz = cscl[t & (NCTX - 1)][sDaz];
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) c4[e] = 0.f;
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        float x[EPL];
-        bwd_ld<EPL>(part[par][w] + c0, x);
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) c4[e] += x[e];
-      }
-      float zw = 0.f, zc = 0.f;
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        wx[e] = fmaf(da[e], khz, wx[e]);                    // (GA + da k_hat^T) z
-        zw = fmaf(zt[e], wx[e], zw);
-        zc = fmaf(zt[e], c4[e], zc);
-      }
-      zw = warp_sum(zw);
-      zc = warp_sum(zc);
-      const bool delta_live = (1.0f + khz) >= eps;
-      const float idl = 1.0f / delta;
-      const float ddelta = delta_live ? zw * idl * idl : 0.0f;
-      float dz[EPL];
-#pragma unroll
-      for (int e = 0; e < EPL; ++e)
-        dz[e] = fmaf(ddelta, kh[e], -(wx[e] + c4[e] + kh[e] * daz) * idl);
-      bwd_st<EPL>(dzw[warp] + c0, dz);
-      if (warp == 0 && lane == 0) {
-        rscl[par][0] = ddelta;
-        rscl[par][1] = fmaf(ddelta, khz, -(zw + zc + khz * daz) * idl);   // z . dz
-      }
-      __syncwarp();
     };
     cta_sync();
     if (T > 0) products(T - 1);
     cta_sync();
     for (int t = T - 1; t >= 0; --t) {
-      mid_token(t);
-      const float idl = 1.0f / cscl[t & (NCTX - 1)][sDelta];
-      float dzc[RC], dzr[R], zr[R], dar[R], kc[RC], zc[RC];
-      bwd_ld<RC>(dzw[warp] + col0, dzc);
-      bwd_ld<R>(dzw[warp] + row0, dzr);
-      bwd_ld<R>(cvec(t, cZt) + row0, zr);
-      bwd_ld<R>(cvec(t, cDa) + row0, dar);
+      // dz of token t at this thread's columns; r3 = A' dz (before the update)
+      const MidScalars ms = mid_scalars(t);
+      float kc[RC], zc[RC], wc[RC];
       bwd_ld<RC>(cvec(t, cKh) + col0, kc);
-      bwd_ld<RC>(cvec(t, cZt) + col0, zc);
-      float b1[R];
+      {
+        float dac[RC], gc[RC], dzc[RC];
+        bwd_ld<RC>(cvec(t, cDa) + col0, dac);
+        bwd_ld<RC>(rowv[t % 3][0] + col0, gc);
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        float2 x1 = make_float2(0.f, 0.f);
+        for (int c = 0; c < RC; ++c) {
+          dzc[c] = fmaf(ms.cK, kc[c], -ms.idl * fmaf(ms.khz, dac[c], 2.0f * gc[c]));
+          wc[c] = dac[c] + dzc[c];
+        }
+        float b1[R];
 #pragma unroll
-        for (int m = 0; m < RP; ++m) x1 = bwd_ffma2(A[r][m], make_float2(dzc[2 * m], dzc[2 * m + 1]), x1);
-        b1[r] = x1.x + x1.y;
+        for (int r = 0; r < R; ++r) {
+          float2 x1 = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int m = 0; m < RP; ++m) x1 = bwd_ffma2(A[r][m], make_float2(dzc[2 * m], dzc[2 * m + 1]), x1);
+          b1[r] = x1.x + x1.y;
+        }
+        rows_reduce<R, TX / 2>(b1, lane);
+        if (row_writer) rowv[t % 3][2][row0 + myrow] = b1[0];
       }
-      rows_reduce<R, TX / 2>(b1, lane);
-      if (row_writer) rowv[t % 3][2][row0 + myrow] = b1[0];
+      // GAs += (w k_hat^T + k_hat w^T) / 2,  A += z z^T / delta
+      bwd_ld<RC>(cvec(t, cZt) + col0, zc);
+      constexpr int RG = R >= 4 ? 4 : R;
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const float dadz = dar[r] + dzr[r], zs = zr[r] * idl;
-        const float2 g2 = make_float2(dadz, dadz), z2 = make_float2(zs, zs);
+      for (int rg = 0; rg < R / RG; ++rg) {
+        float kr[RG], zr[RG], dar[RG], gr[RG];
+        bwd_ld<RG>(cvec(t, cKh) + row0 + rg * RG, kr);
+        bwd_ld<RG>(cvec(t, cZt) + row0 + rg * RG, zr);
+        bwd_ld<RG>(cvec(t, cDa) + row0 + rg * RG, dar);
+        bwd_ld<RG>(rowv[t % 3][0] + row0 + rg * RG, gr);
 #pragma unroll
-        for (int m = 0; m < RP; ++m) {
-          GA[r][m] = bwd_ffma2(g2, make_float2(kc[2 * m], kc[2 * m + 1]), GA[r][m]);
-          A[r][m] = bwd_ffma2(z2, make_float2(zc[2 * m], zc[2 * m + 1]), A[r][m]);
+        for (int i = 0; i < RG; ++i) {
+          const int r = rg * RG + i;
+          const float dzr = fmaf(ms.cK, kr[i], -ms.idl * fmaf(ms.khz, dar[i], 2.0f * gr[i]));
+          const float hw = 0.5f * (dar[i] + dzr), hk = 0.5f * kr[i], zs = zr[i] * ms.idl;
+          const float2 w2 = make_float2(hw, hw), k2 = make_float2(hk, hk), z2 = make_float2(zs, zs);
+#pragma unroll
+          for (int m = 0; m < RP; ++m) {
+            GA[r][m] = bwd_ffma2(w2, make_float2(kc[2 * m], kc[2 * m + 1]), GA[r][m]);
+            GA[r][m] = bwd_ffma2(k2, make_float2(wc[2 * m], wc[2 * m + 1]), GA[r][m]);
+            A[r][m] = bwd_ffma2(z2, make_float2(zc[2 * m], zc[2 * m + 1]), A[r][m]);
+          }
         }
       }
-      __syncwarp();   // this warp's dz copy is rewritten in the next segment
       if (t >= 1) products(t - 1);
       cta_sync();
     }
-    if (p.dA0) {
+  }
+}
+
+// dA0 = dA_T + sum_t w_t k_hat_t^T from the w_t the A side left in the workspace (only when
+// the caller asks for dA0).  One CTA of 256 threads per unit; thread (ty, tx) of a 16 x 16 grid
+// accumulates an R x R block over tiles of 16 tokens staged in shared memory.
+template <int D, typename TIn>
+__global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSplitParams p) {
+  constexpr int R = D / 16;
+  constexpr int EPL = D / 32;
+  constexpr int TT = 16;
+  __shared__ float wt[TT][D];
+  __shared__ float kt[TT][D];
+  const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ty = tid >> 4, tx = tid & 15;
+  const int row0 = ty * R, col0 = tx * R;
+  const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
+  const size_t ubase = size_t(unit) * size_t(p.T) * D;
+  const TIn* gk = static_cast<const TIn*>(p.k) + ubase;
+  float acc[R][R];
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        float gv[RC];
+  for (int r = 0; r < R; ++r)
 #pragma unroll
-        for (int m = 0; m < RP; ++m) { gv[2 * m] = GA[r][m].x; gv[2 * m + 1] = GA[r][m].y; }
-        bwd_st<RC>(p.dA0 + (size_t(unit) * D + row0 + r) * D + col0, gv);
+    for (int c = 0; c < R; ++c)
+      acc[r][c] = p.dA_T ? p.dA_T[(size_t(unit) * D + row0 + r) * D + col0 + c] : 0.0f;
+  for (int t0 = 0; t0 < p.T; t0 += TT) {
+    __syncthreads();
+    for (int i = warp; i < TT; i += 8) {
+      const int t = t0 + i;
+      float kx[EPL], wv[EPL];
+      float ss = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        const int c = e * 32 + lane;
+        float kk = t < p.T ? load1<TIn>(gk, size_t(t) * D + c) : 0.0f;
+        if (!ident && t < p.T) kk = bwd_phi(kk);
+        kx[e] = kk;
+        wv[e] = t < p.T ? p.dal[ubase + size_t(t) * D + c] : 0.0f;
+        ss = fmaf(kk, kk, ss);
+      }
+      ss = warp_sum(ss);
+      const float ink = 1.0f / fmaxf(sqrtf(ss), p.eps);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        kt[i][e * 32 + lane] = kx[e] * ink;
+        wt[i][e * 32 + lane] = wv[e];
       }
     }
+    __syncthreads();
+#pragma unroll 4
+    for (int i = 0; i < TT; ++i)
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float w = wt[i][row0 + r];
+#pragma unroll
+        for (int c = 0; c < R; ++c) acc[r][c] = fmaf(w, kt[i][col0 + c], acc[r][c]);
+      }
   }
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int c = 0; c < R; ++c) p.dA0[(size_t(unit) * D + row0 + r) * D + col0 + c] = acc[r][c];
 }
 
 }  // namespace vla

@@ -171,8 +171,9 @@ int launch_backward_split_t(const BackwardSplitParams& p, cudaStream_t st) {
     cudaGetLastError();
     return VLA_ERR_CUDA;
   }
-  ks<<<p.units, G::NT, M::s_bytes, st>>>(p);   // TX / 2 matrix warps + 1 helper warp
-  ka<<<p.units, G::NT, M::a_bytes, st>>>(p);
+  ks<<<p.units, G::NT_S, M::s_bytes, st>>>(p);   // matrix warps + closing and opening helper warps
+  ka<<<p.units, G::NT_A, M::a_bytes, st>>>(p);
+  if (p.dA0) vla_backward_da0_kernel<D, TIn><<<p.units, 256, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 }  // namespace

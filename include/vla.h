@@ -47,7 +47,10 @@ typedef enum { VLA_F32 = 0, VLA_BF16 = 1 } vla_dtype_t;
 
 enum {
   VLA_FLAG_IDENTITY_MAP = 1u << 0, /* Section 3.1: k_hat = k/||k||, o_t = S_t q_t              */
-  VLA_FLAG_CHECK_FINITE = 1u << 1  /* report non-finite delta or ||A_t k_hat|| in opts->status */
+  VLA_FLAG_CHECK_FINITE = 1u << 1, /* report non-finite delta or ||A_t k_hat|| in opts->status */
+  VLA_FLAG_TOKEN_MAJOR = 1u << 2   /* q, k, v, u and out are [B,T,H,d] (the layout projections write)
+                                      instead of [B,H,T,d]; the states stay [B,H,d,d].  vla_forward
+                                      and the host-buffer calls; VLA_ERR_UNSUPPORTED elsewhere */
 };
 
 /* Which scan kernel runs.  AUTO picks by shape; the others force one (tests, benchmarks). */
@@ -212,6 +215,23 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_,
                  const vla_opts_t* opts, void* workspace, size_t workspace_bytes, void* stream);
 
 size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k);
+
+/*
+ * vla_make_u -- the penalty directions of Algorithm 1 from a projection (its step
+ * "u_t = L2norm(W_u k_t) / sqrt(d_h)", Section 3.2 "learned penalty"):
+ *
+ *     y_t = W_u[h] k_t,     u_t = scale * y_t / max(||y_t||_2, eps)
+ *
+ * for every token of every (b, h), in fp32 on the device.  k [B,H,T,d_k] (k_dtype, the raw keys:
+ * no feature map is applied), W_u [H,d_k,d_k] fp32 row-major (one matrix per head; y = W k),
+ * u [B,H,T,d_k] (u_dtype: VLA_F32, or VLA_BF16 rounded to nearest even) -- the buffer a later
+ * vla_forward takes as opts->u (with opts->qkv_dtype == u_dtype).  scale is used as given
+ * (Algorithm 1: 1/sqrt(d_k); Eq. "penalty": 1); eps <= 0 => 1e-4.  All DEVICE pointers, 16-byte
+ * aligned, caller-owned; asynchronous on `stream`; nothing allocated.  d_k in {16,32,64,128},
+ * else VLA_ERR_UNSUPPORTED.  A zero y_t gives u_t = 0 (no penalty for that token).
+ */
+int vla_make_u(const void* k, const float* W_u, int B, int H, int T, int d_k, int k_dtype, int u_dtype,
+               float scale, float eps, void* u, void* stream);
 
 /*
  * vla_probe_fp32_fma -- measurement helper (the paper has no counterpart): enqueues a

@@ -21,12 +21,12 @@ VLA_ERR_INVALID_ARG, VLA_ERR_UNSUPPORTED, VLA_ERR_ALIGNMENT = -1, -2, -3
 VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE, VLA_ERR_TOO_LARGE = -4, -5, -6, -7
 VLA_STATIC_SCRATCH_BYTES = 32 << 20
 VLA_F32, VLA_BF16 = 0, 1
-VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE = 1, 2
+VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE, VLA_FLAG_TOKEN_MAJOR = 1, 2, 4
 VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK, VLA_KERNEL_DECODE = 0, 1, 2, 3
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",
            "vla_forward_seqpar", "vla_seqpar_segments", "vla_seqpar_workspace_bytes",
-           "vla_probe_fp32_fma", "vla_backward", "vla_backward_workspace_bytes",
+           "vla_probe_fp32_fma", "vla_backward", "vla_backward_workspace_bytes", "vla_make_u",
            "vla_query_support", "vla_status_string", "vla_version")
 
 
@@ -85,6 +85,8 @@ def load_library():
             lib.vla_backward.argtypes = [vp, vp, vp, f, i, i, i, i, i] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
             lib.vla_backward_workspace_bytes.restype = ctypes.c_size_t
             lib.vla_backward_workspace_bytes.argtypes = [i, i, i, i]
+            lib.vla_make_u.restype = i
+            lib.vla_make_u.argtypes = [vp, vp, i, i, i, i, i, i, ctypes.c_float, ctypes.c_float, vp, vp]
             lib.vla_probe_fp32_fma.restype = i
             lib.vla_probe_fp32_fma.argtypes = [i, vp, ctypes.POINTER(ctypes.c_double), vp]
             lib.vla_host_workspace_bytes.restype = ctypes.c_size_t
@@ -109,6 +111,29 @@ def vla_version() -> int:
 
 def vla_query_support(d_k: int, d_v: int, qkv_dtype: int = VLA_F32, flags: int = 0) -> int:
     return load_library().vla_query_support(d_k, d_v, qkv_dtype, flags)
+
+
+def vla_make_u(k, W_u, *, scale: Optional[float] = None, eps: float = 1e-4, out=None, out_dtype=None,
+               stream: Optional[torch.cuda.Stream] = None):
+    """``u = scale * L2norm(W_u[h] k)`` for CUDA tensors ``k: [B,H,T,d]``, ``W_u: [H,d,d]`` fp32.
+    ``scale`` defaults to Algorithm 1's ``1/sqrt(d)``; the result has ``out_dtype`` (default: k's)."""
+    lib = load_library()
+    B, H, T, d = k.shape
+    if out_dtype is None:
+        out_dtype = k.dtype if out is None else out.dtype
+    _chk(k, (B, H, T, d), k.dtype, "k"); _chk(W_u, (H, d, d), torch.float32, "W_u")
+    if out is None:
+        out = torch.empty((B, H, T, d), dtype=out_dtype, device=k.device)
+    _chk(out, (B, H, T, d), out_dtype, "out")
+    if scale is None:
+        scale = float(d) ** -0.5
+    st = stream if stream is not None else torch.cuda.current_stream(k.device)
+    with torch.cuda.device(k.device):
+        rc = lib.vla_make_u(_ptr(k), _ptr(W_u), B, H, T, d, _dtype_code(k), _dtype_code(out),
+                            float(scale), float(eps), _ptr(out), ctypes.c_void_p(st.cuda_stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_make_u")
+    return out
 
 
 def vla_host_workspace_bytes(B, H, T, d_k, d_v, qkv_dtype=VLA_F32, has_u=False) -> int:
@@ -169,31 +194,37 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
                 eps: float = 1e-4, out=None, S_T=None, A_T=None, z_T=None, status=None,
                 kernel: int = VLA_KERNEL_AUTO, stream: Optional[torch.cuda.Stream] = None,
                 want_status: bool = True, refresh=None) -> VlaResult:
-    """Enqueue the scan for CUDA tensors ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``.
+    """Enqueue the scan for CUDA tensors ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``
+    (``[B,T,H,d]`` for all of them and ``out`` with ``VLA_FLAG_TOKEN_MAJOR``).
 
     Output tensors are allocated with torch unless passed in.  Nothing is synchronised.
     """
     lib = load_library()
     if q.dim() != 4:
         raise ValueError("q must be [B,H,T,d_k]")
-    B, H, T, dk = q.shape
+    if flags & VLA_FLAG_TOKEN_MAJOR:
+        B, T, H, dk = q.shape
+        tok = lambda d_: (B, T, H, d_)
+    else:
+        B, H, T, dk = q.shape
+        tok = lambda d_: (B, H, T, d_)
     dv = v.shape[-1]
     dt = _dtype_code(q)
     dev = q.device
-    _chk(q, (B, H, T, dk), q.dtype, "q"); _chk(k, (B, H, T, dk), q.dtype, "k")
-    _chk(v, (B, H, T, dv), q.dtype, "v"); _chk(u, (B, H, T, dk), q.dtype, "u")
+    _chk(q, tok(dk), q.dtype, "q"); _chk(k, tok(dk), q.dtype, "k")
+    _chk(v, tok(dv), q.dtype, "v"); _chk(u, tok(dk), q.dtype, "u")
     f32 = torch.float32
     _chk(S0, (B, H, dv, dk), f32, "S0"); _chk(A0, (B, H, dk, dk), f32, "A0")
     _chk(z0, (B, H, dk), f32, "z0")
     if out is None:
-        out = torch.empty((B, H, T, dv), dtype=f32, device=dev)
+        out = torch.empty(tok(dv), dtype=f32, device=dev)
     if S_T is None:
         S_T = torch.empty((B, H, dv, dk), dtype=f32, device=dev)
     if A_T is None:
         A_T = torch.empty((B, H, dk, dk), dtype=f32, device=dev)
     if z_T is None:
         z_T = torch.empty((B, H, dk), dtype=f32, device=dev)
-    _chk(out, (B, H, T, dv), f32, "out"); _chk(S_T, (B, H, dv, dk), f32, "S_T")
+    _chk(out, tok(dv), f32, "out"); _chk(S_T, (B, H, dv, dk), f32, "S_T")
     _chk(A_T, (B, H, dk, dk), f32, "A_T"); _chk(z_T, (B, H, dk), f32, "z_T")
     if status is None and want_status:
         status = torch.zeros((), dtype=torch.int32, device=dev)

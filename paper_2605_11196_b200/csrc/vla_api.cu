@@ -10,6 +10,7 @@
 #include "vla.h"
 #include "vla_launch.h"
 #include "vla_backward_params.h"
+#include "vla_make_u_params.h"
 
 namespace {
 
@@ -29,7 +30,8 @@ int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
   }
   if (!(r->eps > 0.0f)) r->eps = 1e-4f;
   if (r->qkv_dtype != VLA_F32 && r->qkv_dtype != VLA_BF16) return VLA_ERR_INVALID_ARG;
-  if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_INVALID_ARG;
+  if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE | VLA_FLAG_TOKEN_MAJOR))
+    return VLA_ERR_INVALID_ARG;
   if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN && r->kernel != VLA_KERNEL_CHUNK &&
       r->kernel != VLA_KERNEL_DECODE)
     return VLA_ERR_INVALID_ARG;
@@ -195,6 +197,7 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
   p.step_offset = o.step_offset; p.u_is_khat = 0;
   p.n_main = 0; p.out2 = nullptr;
   p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr;
+  p.heads = H;
   return launch(p, d_k, o.qkv_dtype, o.kernel, static_cast<cudaStream_t>(stream));
 }
 
@@ -388,7 +391,8 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   if (rc != VLA_OK) return rc;
   rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, out);
   if (rc != VLA_OK) return rc;
-  if (d_k < 32 || o.refresh_period > 0 || o.kernel == VLA_KERNEL_TOKEN) return VLA_ERR_UNSUPPORTED;
+  if (d_k < 32 || o.refresh_period > 0 || o.kernel == VLA_KERNEL_TOKEN || (o.flags & VLA_FLAG_TOKEN_MAJOR))
+    return VLA_ERR_UNSUPPORTED;
   const void* ptrs[] = {q, k, v, o.u, S0, A0, out, S_T, A_T, o.z0, o.zT};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return VLA_ERR_ALIGNMENT;
@@ -434,6 +438,7 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   p.T = T / P; p.units = seqpar_tri(d_k) ? N : 2 * N; p.n_main = N; p.flags = o.flags;
   p.refresh_period = 0; p.refresh_eta = 0.0f; p.step_offset = 0; p.u_is_khat = 0;
   p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr;
+  p.heads = H;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = vla::seqpar_before_scan(d_k, o.qkv_dtype, sp, st);
   if (rc != VLA_OK) return rc;
@@ -462,7 +467,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   if (rc != VLA_OK) return rc;
   rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, d_out);
   if (rc != VLA_OK) return rc;
-  if (o.u || o.refresh_period > 0) return VLA_ERR_UNSUPPORTED;
+  if (o.u || o.refresh_period > 0 || (o.flags & VLA_FLAG_TOKEN_MAJOR)) return VLA_ERR_UNSUPPORTED;
   const int units = B * H;
   if (units > 0 && T > 0 && (!dq || !dk || !dv)) return VLA_ERR_INVALID_ARG;
   const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0};
@@ -506,6 +511,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   f.refresh_period = 0; f.refresh_eta = 0.0f; f.step_offset = 0; f.u_is_khat = 0;
   f.n_main = 0; f.out2 = nullptr;
   f.stash_z = zst; f.stash_e = est; f.stash_delta = dst;
+  f.heads = H;
   rc = vla::launch_chunk_stash(d_k, o.qkv_dtype, f, st);
   if (rc != VLA_OK) return rc;
   // 2. the S-side and A-side reverse scans
@@ -518,6 +524,24 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   return vla::launch_backward_split(d_k, o.qkv_dtype, p, st);
 }
 
+int vla_make_u(const void* k, const float* W_u, int B, int H, int T, int d_k, int k_dtype, int u_dtype,
+               float scale, float eps, void* u, void* stream) {
+  if (B < 0 || H < 0 || T < 0) return VLA_ERR_INVALID_ARG;
+  if ((k_dtype != VLA_F32 && k_dtype != VLA_BF16) || (u_dtype != VLA_F32 && u_dtype != VLA_BF16))
+    return VLA_ERR_INVALID_ARG;
+  if (!(scale == scale)) return VLA_ERR_INVALID_ARG;
+  if (d_k != 16 && d_k != 32 && d_k != 64 && d_k != 128) return VLA_ERR_UNSUPPORTED;
+  const long long units = (long long)B * H;
+  if (units > 0x7fffffffLL) return VLA_ERR_INVALID_ARG;
+  if (units == 0 || T == 0) return VLA_OK;
+  if (!k || !W_u || !u) return VLA_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(W_u) || !aligned16(u)) return VLA_ERR_ALIGNMENT;
+  vla::MakeUParams p;
+  p.k = k; p.W = W_u; p.u = u; p.scale = scale; p.eps = eps > 0.0f ? eps : 1e-4f;
+  p.T = T; p.units = int(units); p.heads = H;
+  return vla::launch_make_u(d_k, k_dtype, u_dtype, p, static_cast<cudaStream_t>(stream));
+}
+
 int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream) {
   if (iters <= 0 || !sink) return VLA_ERR_INVALID_ARG;
   return vla::launch_fp32_probe(iters, sink, flops, static_cast<cudaStream_t>(stream));
@@ -525,7 +549,8 @@ int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream) {
 
 int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags) {
   if (qkv_dtype != VLA_F32 && qkv_dtype != VLA_BF16) return VLA_ERR_UNSUPPORTED;
-  if (flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE)) return VLA_ERR_UNSUPPORTED;
+  if (flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE | VLA_FLAG_TOKEN_MAJOR))
+    return VLA_ERR_UNSUPPORTED;
   return shape_supported(d_k, d_v) ? VLA_OK : VLA_ERR_UNSUPPORTED;
 }
 

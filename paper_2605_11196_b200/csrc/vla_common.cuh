@@ -43,6 +43,9 @@ struct ScanParams {
   float* stash_z;
   float* stash_e;
   float* stash_delta;
+  // Token-major tensors (VLA_FLAG_TOKEN_MAJOR): q, k, v, u, out are [B, T, heads, D] instead of
+  // [B, heads, T, D]; unit = b * heads + h.  The states keep their [units, D, D] layout.
+  int heads;
 #ifdef VLA_SECTION_TIMERS
   long long* dbg;      // debug builds only: per-section clock64 totals of unit 0
 #endif
@@ -116,6 +119,40 @@ __device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src,
 __device__ __forceinline__ void bulk_commit() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
+// Where the tokens of a unit lie in q, k, v, u, out: element offset of token t and the distance
+// between consecutive tokens, for both tensor layouts.
+__device__ __forceinline__ size_t token_offset(const ScanParams& p, int unit, size_t t, int D) {
+  if (p.flags & VLA_FLAG_TOKEN_MAJOR) {
+    const int b = unit / p.heads, h = unit - b * p.heads;
+    return ((size_t(b) * size_t(p.T) + t) * size_t(p.heads) + size_t(h)) * D;
+  }
+  return (size_t(unit) * size_t(p.T) + t) * D;
+}
+__device__ __forceinline__ size_t token_stride(const ScanParams& p, int D) {
+  return (p.flags & VLA_FLAG_TOKEN_MAJOR) ? size_t(p.heads) * D : size_t(D);
+}
+// n rows of row_bytes each, `stride` elements apart in global memory, to (from) dense rows in
+// shared memory: one bulk copy when the rows are adjacent, else one per row
+template <typename TEl>
+__device__ __forceinline__ void bulk_load_rows(TEl* smem_dst, const TEl* gmem_src, size_t stride, int n,
+                                               int D, uint64_t* bar) {
+  if (stride == size_t(D)) {
+    bulk_load(smem_dst, gmem_src, uint32_t(n) * D * sizeof(TEl), bar);
+  } else {
+    for (int i = 0; i < n; ++i)
+      bulk_load(smem_dst + size_t(i) * D, gmem_src + size_t(i) * stride, uint32_t(D * sizeof(TEl)), bar);
+  }
+}
+template <typename TEl>
+__device__ __forceinline__ void bulk_store_rows(TEl* gmem_dst, const TEl* smem_src, size_t stride, int n, int D) {
+  if (stride == size_t(D)) {
+    bulk_store(gmem_dst, smem_src, uint32_t(n) * D * sizeof(TEl));
+  } else {
+    for (int i = 0; i < n; ++i)
+      bulk_store(gmem_dst + size_t(i) * stride, smem_src + size_t(i) * D, uint32_t(D * sizeof(TEl)));
+  }
+}
+
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() {  // <= N groups still reading shared memory
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");

@@ -11,6 +11,7 @@
 namespace vla {
 struct BackwardParams;
 struct BackwardSplitParams;
+struct MakeUParams;
 }
 
 namespace vla {
@@ -44,6 +45,8 @@ int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st);
 
 // Backward pass as two reverse scans over the chunk kernel's stash, d in {32, 64, 128}, u = k_hat.
 int launch_backward_split(int d, int dtype, const BackwardSplitParams& p, cudaStream_t st);
+// u = scale * L2norm(W_u k): in_dtype of k, out_dtype of u
+int launch_make_u(int d, int in_dtype, int out_dtype, const MakeUParams& p, cudaStream_t st);
 
 // Register-only fp32 FMA loop over the whole device (measurement helper); *flops = work launched.
 int launch_fp32_probe(int iters, float* sink, double* flops, cudaStream_t st);

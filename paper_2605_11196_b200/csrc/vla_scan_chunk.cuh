@@ -476,16 +476,17 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
   // global addresses are formed where they are used (two threads of the CTA), so that they
   // do not occupy registers in the FMA loops
   auto issue = [&](int c) {
-    const size_t tok = size_t(uin) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+    const size_t off = token_offset(p, uin, size_t(t_begin) + size_t(c) * C, D);
+    const size_t step = token_stride(p, D);
     const int s = c % NSTAGE;
     const int n = min(C, T - c * C);
     const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
     TIn* dst = raw + size_t(s) * NIN * C * D;
     mbar_arrive_expect_tx(&full[s], (pscan_cta ? NIN - 1 : NIN) * bytes);
-    bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &full[s]);
-    bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &full[s]);
-    if (!pscan_cta) bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
-    if (UT) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
+    bulk_load_rows(dst + 0 * C * D, static_cast<const TIn*>(p.q) + off, step, n, D, &full[s]);
+    bulk_load_rows(dst + 1 * C * D, static_cast<const TIn*>(p.k) + off, step, n, D, &full[s]);
+    if (!pscan_cta) bulk_load_rows(dst + 2 * C * D, static_cast<const TIn*>(p.v) + off, step, n, D, &full[s]);
+    if (UT) bulk_load_rows(dst + 3 * C * D, static_cast<const TIn*>(p.u) + off, step, n, D, &full[s]);
   };
 
   // (re)arm the barriers of this piece; a tail piece also waits for its unit's head
@@ -996,10 +997,16 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
       fence_async_smem();
       group_bar(sbar, NG);  // Eps and the out stage complete
       if (g == 0) {
-        const size_t tok = size_t(uin) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+        // the readout of a transfer scan is workspace, always [units, T, D]
+        const size_t tq = size_t(t_begin) + size_t(c) * C;
         float* odst = pscan ? p.out2 : p.out;
         if (!STASH || odst) {   // a backward pass that only wants the stash passes no readout buffer
-          bulk_store(odst + tok * D, ostage + size_t(c & 1) * C * D, uint32_t(n) * D * sizeof(float));
+          if (pscan)
+            bulk_store(odst + (size_t(uin) * size_t(p.T) + tq) * D, ostage + size_t(c & 1) * C * D,
+                       uint32_t(n) * D * sizeof(float));
+          else
+            bulk_store_rows(odst + token_offset(p, uin, tq, D), ostage + size_t(c & 1) * C * D,
+                            token_stride(p, D), n, D);
           bulk_commit();
         }
       }

@@ -79,12 +79,13 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
   const float eps = p.eps;
   const int nchunks = (T + C - 1) / C;
 
-  const size_t tok_base = size_t(unit) * size_t(T);
-  const TIn* gq = static_cast<const TIn*>(p.q) + tok_base * D;
-  const TIn* gk = static_cast<const TIn*>(p.k) + tok_base * D;
-  const TIn* gv = static_cast<const TIn*>(p.v) + tok_base * D;
-  const TIn* gu = HAS_U ? static_cast<const TIn*>(p.u) + tok_base * D : nullptr;
-  float* gout = p.out + tok_base * D;
+  const size_t tok_base = token_offset(p, unit, 0, D);   // element offset of this unit's token 0
+  const size_t tok_step = token_stride(p, D);            // elements between its tokens
+  const TIn* gq = static_cast<const TIn*>(p.q) + tok_base;
+  const TIn* gk = static_cast<const TIn*>(p.k) + tok_base;
+  const TIn* gv = static_cast<const TIn*>(p.v) + tok_base;
+  const TIn* gu = HAS_U ? static_cast<const TIn*>(p.u) + tok_base : nullptr;
+  float* gout = p.out + tok_base;
 
   // ---- ring set-up and the first loads (one elected thread)
   auto issue = [&](int c) {
@@ -92,12 +93,12 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
     const int n = min(C, T - c * C);
     const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
     TIn* dst = raw + size_t(s) * NIN * C * D;
-    const size_t off = size_t(c) * C * D;
+    const size_t off = size_t(c) * C * tok_step;
     mbar_arrive_expect_tx(&full[s], NIN * bytes);
-    bulk_load(dst + 0 * C * D, gq + off, bytes, &full[s]);
-    bulk_load(dst + 1 * C * D, gk + off, bytes, &full[s]);
-    bulk_load(dst + 2 * C * D, gv + off, bytes, &full[s]);
-    if (HAS_U) bulk_load(dst + 3 * C * D, gu + off, bytes, &full[s]);
+    bulk_load_rows(dst + 0 * C * D, gq + off, tok_step, n, D, &full[s]);
+    bulk_load_rows(dst + 1 * C * D, gk + off, tok_step, n, D, &full[s]);
+    bulk_load_rows(dst + 2 * C * D, gv + off, tok_step, n, D, &full[s]);
+    if (HAS_U) bulk_load_rows(dst + 3 * C * D, gu + off, tok_step, n, D, &full[s]);
   };
   if (tid == 0) {
     for (int s = 0; s < NSTAGE; ++s) mbar_init(&full[s], 1);
@@ -340,7 +341,7 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
     fence_async_smem();
     __syncthreads();
     if (tid == 0) {
-      bulk_store(gout + size_t(c) * C * D, ost, uint32_t(n) * D * sizeof(float));
+      bulk_store_rows(gout + size_t(c) * C * tok_step, ost, tok_step, n, D);
       bulk_commit();
     }
   }

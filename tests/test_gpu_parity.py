@@ -363,3 +363,62 @@ def test_single_step_kernel_in_a_decode_loop_and_its_limits():
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
     with pytest.raises(vla.VlaError):            # more than one step
         vla.vla_forward(q.to(dev), k.to(dev), v.to(dev), 1.0, S0=S, A0=A, kernel=vla.VLA_KERNEL_DECODE)
+
+
+# ---- token-major tensors: q, k, v, u, out as [B, T, H, d] (the layout a projection writes)
+TOKEN_MAJOR = vla.VLA_FLAG_TOKEN_MAJOR
+
+
+@pytest.mark.parametrize("kernel", ["token", "chunk"])
+@pytest.mark.parametrize("d", [16, 32, 64, 128])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+@pytest.mark.parametrize("umode", ["khat", "unit_over_sqrt_d"])
+def test_token_major_layout(kernel, d, dtype, flags, umode):
+    """The same scan with the sequence tensors transposed to [B, T, H, d]: bit-identical to the
+    head-major call (the layout changes addresses, not arithmetic) and within tolerance of the
+    oracle, which is given the head-major arrays."""
+    if kernel == "chunk" and not _chunk_covers(d, umode):
+        pytest.skip("no chunk kernel for this shape")
+    kcode = vla.VLA_KERNEL_TOKEN if kernel == "token" else vla.VLA_KERNEL_CHUNK
+    w = _small(d, 83, dtype, units=(2, 3), seed=300 + d)
+    q, k, v = W.make_inputs(w)
+    u = None if umode == "khat" else W.make_u(w, d ** -0.5)
+    dev = torch.device("cuda:0")
+    tm = lambda x: None if x is None else x.permute(0, 2, 1, 3).contiguous().to(dev)
+    g = torch.Generator().manual_seed(d)
+    S0 = torch.randn((2, 3, d, d), generator=g) * 0.1
+    z0 = torch.rand((2, 3, d), generator=g)
+    plain = run_gpu(q, k, v, w.lam, u=u, S0=S0, z0=z0, flags=flags, kernel=kcode)
+    r = vla.vla_forward(tm(q), tm(k), tm(v), w.lam, u=tm(u), S0=S0.to(dev), z0=z0.to(dev),
+                        flags=flags | TOKEN_MAJOR, kernel=kcode)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    assert r.out.shape == (2, 83, 3, d)
+    assert torch.equal(r.out.permute(0, 2, 1, 3), plain.out)
+    assert torch.equal(r.S_T, plain.S_T) and torch.equal(r.A_T, plain.A_T) and torch.equal(r.z_T, plain.z_T)
+    ref = run_oracle(q, k, v, w.lam, u=u, S0=S0, z0=z0, flags=flags)
+    assert rel_err(r.out.permute(0, 2, 1, 3), ref.out) <= 1e-4
+    assert rel_err(r.S_T, ref.S_T) <= 1e-4 and rel_err(r.A_T, ref.A_T) <= 1e-4
+
+
+def test_token_major_on_the_balanced_schedule_and_where_it_is_refused():
+    """Few long units (the schedule that cuts units into pieces) read and write [B, T, H, d] too;
+    the calls that do not take the layout say so."""
+    dev = torch.device("cuda:0")
+    w = W.Workload("t", 1, 5, 64, 4096 + 37, "bf16", 77)
+    q, k, v = W.make_inputs(w)
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(dev)
+    plain = run_gpu(q, k, v, w.lam)
+    r = vla.vla_forward(tm(q), tm(k), tm(v), w.lam, flags=TOKEN_MAJOR)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    assert torch.equal(r.out.permute(0, 2, 1, 3), plain.out) and torch.equal(r.S_T, plain.S_T)
+    ref = run_oracle(q, k, v, w.lam)
+    assert rel_err(r.out.permute(0, 2, 1, 3), ref.out) <= 1e-4
+    assert vla.vla_query_support(64, 64, vla.VLA_BF16, TOKEN_MAJOR) == vla.VLA_OK
+    w2 = W.Workload("t", 1, 2, 64, 64, "f32", 78)
+    q, k, v = [x.to(dev) for x in W.make_inputs(w2)]
+    with pytest.raises(vla.VlaError) as ei:
+        vla.vla_forward_seqpar(q, k, v, 1.0, segments=2, flags=TOKEN_MAJOR)
+    assert ei.value.code == vla.VLA_ERR_UNSUPPORTED

@@ -486,7 +486,43 @@ def main():
             "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T,
             "fp32_frac_nominal": alg_flops_per_token(w.d, True) * w.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
             "units": w.units, "kernel": "vla_scan_chunk_kernel (explicit u)"}
-        del uu
+        # the same with u formed on the device from a projection (Algorithm 1: u = L2norm(W_u k) / sqrt(d_h))
+        Wu = (torch.randn((w.H, w.d, w.d), generator=torch.Generator().manual_seed(11)) / w.d ** 0.5).to(dev)
+        def wcall():
+            vla.vla_make_u(kd, Wu, out=uu, stream=stream)
+            vla.vla_forward(qd, kd, vd, w.lam, u=uu, out=out, S_T=S_T, A_T=A_T, z_T=z_T, status=status, stream=stream)
+        evs = []
+        with torch.cuda.stream(stream):
+            wcall()
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); wcall(); b.record(stream)
+                evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+        per[w.name + "_projected_u"] = {
+            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
+            "kernel": "vla_make_u_kernel + vla_scan_chunk_kernel (explicit u)", "gpu_launches_per_step": 2}
+        del uu, Wu
+        # the headline workload with q, k, v, out as [B, T, H, d]
+        qt, kt, vt = [x.view(w.B, w.H, w.T, w.d).permute(0, 2, 1, 3).contiguous() for x in (qd, kd, vd)]
+        out_t = torch.empty((w.B, w.T, w.H, w.d), dtype=torch.float32, device=dev)
+        tcall = lambda: vla.vla_forward(qt, kt, vt, w.lam, out=out_t, S_T=S_T, A_T=A_T, z_T=z_T, status=status,
+                                        stream=stream, flags=vla.VLA_FLAG_TOKEN_MAJOR)
+        evs = []
+        with torch.cuda.stream(stream):
+            tcall()
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); tcall(); b.record(stream)
+                evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+        per[w.name + "_token_major"] = {
+            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
+            "fp32_frac_nominal": alg_flops_per_token(w.d, False) * w.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
+            "kernel": "vla_scan_chunk_kernel, [B,T,H,d] tensors"}
+        del qt, kt, vt, out_t
         # single-step decode (T = 1, carried states): bound by moving S and A through HBM once
         wd = W.EXTRA["decode"]
         q2, k2, v2 = [x.to(dev) for x in W.make_inputs(wd)]

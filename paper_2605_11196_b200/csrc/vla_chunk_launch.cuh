@@ -8,12 +8,14 @@
 
 namespace vla {
 
-template <int D, typename TIn, int UM>
-int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
+// TM: q, k, v, u, out are [B, T, H, d] (an instantiation of its own: one bulk copy per token row).
+template <int D, typename TIn, int UM, bool TM>
+int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
   using Cfg = ChunkCfg<D, TIn, UM>;
   static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
-  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM>;     // one CTA per unit
-  auto kern_bal = vla_scan_chunk_kernel<D, TIn, true, UM>;  // persistent grid, units cut at chunks
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, false, false, TM>;     // one CTA per unit
+  auto kern_bal = vla_scan_chunk_kernel<D, TIn, true, UM, false, false, TM>;  // persistent grid, units cut at chunks
+  if (TM && p.n_main > 0) return VLA_ERR_UNSUPPORTED;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(Cfg::smem_bytes)) != cudaSuccess ||
       cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -47,6 +49,12 @@ int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
   if (sp.balanced) kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
   else kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D, typename TIn, int UM>
+int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
+  if (p.flags & VLA_FLAG_TOKEN_MAJOR) return launch_chunk_um_tm<D, TIn, UM, true>(p, st);
+  return launch_chunk_um_tm<D, TIn, UM, false>(p, st);
 }
 
 // The forward of a backward pass: plain grid, u = k_hat, per-token z, e, delta left in global

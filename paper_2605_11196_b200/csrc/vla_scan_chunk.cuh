@@ -371,7 +371,7 @@ __device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) 
 // STASH: the launch also leaves z_t, e_t, delta_t of every token in global memory (and may
 // drop the readout) for the backward pass; a separate instantiation so that the plain forward
 // kernel carries none of it.
-template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false, bool STASH = false>
+template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false, bool STASH = false, bool TM = false>
 __global__ void __launch_bounds__((TRI ? 3 : 2) * D, (TRI && sizeof(TIn) == 2) ? 2 : 1)
 vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
   using Cfg = ChunkCfg<D, TIn, UM, TRI>;
@@ -476,17 +476,32 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
   // global addresses are formed where they are used (two threads of the CTA), so that they
   // do not occupy registers in the FMA loops
   auto issue = [&](int c) {
-    const size_t off = token_offset(p, uin, size_t(t_begin) + size_t(c) * C, D);
-    const size_t step = token_stride(p, D);
     const int s = c % NSTAGE;
     const int n = min(C, T - c * C);
     const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
     TIn* dst = raw + size_t(s) * NIN * C * D;
-    mbar_arrive_expect_tx(&full[s], (pscan_cta ? NIN - 1 : NIN) * bytes);
-    bulk_load_rows(dst + 0 * C * D, static_cast<const TIn*>(p.q) + off, step, n, D, &full[s]);
-    bulk_load_rows(dst + 1 * C * D, static_cast<const TIn*>(p.k) + off, step, n, D, &full[s]);
-    if (!pscan_cta) bulk_load_rows(dst + 2 * C * D, static_cast<const TIn*>(p.v) + off, step, n, D, &full[s]);
-    if (UT) bulk_load_rows(dst + 3 * C * D, static_cast<const TIn*>(p.u) + off, step, n, D, &full[s]);
+    if constexpr (!TM) {
+      mbar_arrive_expect_tx(&full[s], (pscan_cta ? NIN - 1 : NIN) * bytes);
+      const size_t tok = size_t(uin) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+      bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &full[s]);
+      bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &full[s]);
+      if (!pscan_cta) bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
+      if (UT) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
+    } else {
+      // [B, T, H, d] tensors: one bulk copy per token row, lane r of the group's first warp
+      // (all of which calls this) taking row r
+      const int r = tid & 31;
+      if (r == 0) mbar_arrive_expect_tx(&full[s], NIN * bytes);
+      __syncwarp();
+      if (r < n) {
+        const size_t off = token_offset(p, uin, size_t(t_begin) + size_t(c) * C + r, D);
+        const uint32_t rb = uint32_t(D * sizeof(TIn));
+        bulk_load(dst + 0 * C * D + r * D, static_cast<const TIn*>(p.q) + off, rb, &full[s]);
+        bulk_load(dst + 1 * C * D + r * D, static_cast<const TIn*>(p.k) + off, rb, &full[s]);
+        bulk_load(dst + 2 * C * D + r * D, static_cast<const TIn*>(p.v) + off, rb, &full[s]);
+        if (UT) bulk_load(dst + 3 * C * D + r * D, static_cast<const TIn*>(p.u) + off, rb, &full[s]);
+      }
+    }
   };
 
   // (re)arm the barriers of this piece; a tail piece also waits for its unit's head
@@ -518,7 +533,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
     }
   }
   __syncthreads();
-  if (tid == 0) {  // thread 0 of group A is the TMA producer
+  if (TM ? tid < 32 : tid == 0) {  // thread 0 (token-major tensors: warp 0) of group A is the TMA producer
     for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue(c);
   }
 
@@ -648,7 +663,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
 
     if (nchunks > 0) prep_inputs(0, 0, NWG);
     group_bar(1, NG);
-    if (g == 0 && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
+    if ((TM ? g < 32 : g == 0) && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
 
     for (int c = 0; c < nchunks; ++c) {
       const int slot = c % RING;
@@ -779,7 +794,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
       }
       group_bar(1, NG);
       // the raw stage of chunk c + 1 has been consumed: refill it
-      if (g == 0 && c + 1 + NSTAGE < nchunks) issue(c + 1 + NSTAGE);
+      if ((TM ? g < 32 : g == 0) && c + 1 + NSTAGE < nchunks) issue(c + 1 + NSTAGE);
       VLA_MARK(4)
 
       // ---- row g of Z by forward substitution: z_t = z0_t - sum_{s<t} L[t][s] z_s
@@ -928,7 +943,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
         VS[t * D + g] = (TRI && pscan ? 0.0f : Vf[t * D + g]) - x;
       });
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
-      if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
+      if (TM ? g < C : g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
       // explicit u: the ring's Z slot carries a_t = A_t k_hat_t; the two small matrices
       // k_hat_t . a_s and q_t . a_s are formed here (for u = k_hat they come from group A)
       const float* Gm = GuT;
@@ -996,17 +1011,18 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
       }
       fence_async_smem();
       group_bar(sbar, NG);  // Eps and the out stage complete
-      if (g == 0) {
-        // the readout of a transfer scan is workspace, always [units, T, D]
+      if (TM ? g < C : g == 0) {   // token-major tensors: thread r stores row r, in bulk groups of its own
         const size_t tq = size_t(t_begin) + size_t(c) * C;
         float* odst = pscan ? p.out2 : p.out;
         if (!STASH || odst) {   // a backward pass that only wants the stash passes no readout buffer
-          if (pscan)
+          if constexpr (!TM) {
             bulk_store(odst + (size_t(uin) * size_t(p.T) + tq) * D, ostage + size_t(c & 1) * C * D,
                        uint32_t(n) * D * sizeof(float));
-          else
-            bulk_store_rows(odst + token_offset(p, uin, tq, D), ostage + size_t(c & 1) * C * D,
-                            token_stride(p, D), n, D);
+          } else {
+            if (g < n)
+              bulk_store(odst + token_offset(p, uin, tq + g, D), ostage + size_t(c & 1) * C * D + g * D,
+                         uint32_t(D * sizeof(float)));
+          }
           bulk_commit();
         }
       }
@@ -1029,7 +1045,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
               make_float4(st[r][2 * m].x, st[r][2 * m].y, st[r][2 * m + 1].x, st[r][2 * m + 1].y);
       }
     }
-    if (g == 0) bulk_wait_all<0>();
+    if (TM ? g < C : g == 0) bulk_wait_all<0>();
   }
   if (to_handoff) {   // every thread's state stores precede the flag
     __syncthreads();

@@ -402,9 +402,9 @@ def test_token_major_layout(kernel, d, dtype, flags, umode):
     assert rel_err(r.S_T, ref.S_T) <= 1e-4 and rel_err(r.A_T, ref.A_T) <= 1e-4
 
 
-def test_token_major_on_the_balanced_schedule_and_where_it_is_refused():
-    """Few long units (the schedule that cuts units into pieces) read and write [B, T, H, d] too;
-    the calls that do not take the layout say so."""
+def test_token_major_long_units_and_where_it_is_refused():
+    """Long units with a ragged tail in [B, T, H, d], on the plain grid and on the schedule that
+    cuts units into pieces; the calls that do not take the layout say so."""
     dev = torch.device("cuda:0")
     w = W.Workload("t", 1, 5, 64, 4096 + 37, "bf16", 77)
     q, k, v = W.make_inputs(w)
@@ -416,6 +416,13 @@ def test_token_major_on_the_balanced_schedule_and_where_it_is_refused():
     assert torch.equal(r.out.permute(0, 2, 1, 3), plain.out) and torch.equal(r.S_T, plain.S_T)
     ref = run_oracle(q, k, v, w.lam)
     assert rel_err(r.out.permute(0, 2, 1, 3), ref.out) <= 1e-4
+    wb = W.Workload("t", 1, 151, 128, 256 + 5, "bf16", 79)      # more units than resident CTAs
+    q, k, v = W.make_inputs(wb)
+    plain = run_gpu(q, k, v, wb.lam)
+    r = vla.vla_forward(tm(q), tm(k), tm(v), wb.lam, flags=TOKEN_MAJOR)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    assert torch.equal(r.out.permute(0, 2, 1, 3), plain.out) and torch.equal(r.A_T, plain.A_T)
     assert vla.vla_query_support(64, 64, vla.VLA_BF16, TOKEN_MAJOR) == vla.VLA_OK
     w2 = W.Workload("t", 1, 2, 64, 64, "f32", 78)
     q, k, v = [x.to(dev) for x in W.make_inputs(w2)]

@@ -202,10 +202,11 @@ size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
  * dv [B,H,T,d_v] and, when non-NULL, dS0, dA0, dz0.  The forward is recomputed inside; no
  * state of the forward call is needed.  In identity-map mode z_T = z0, so dz0 = dz_T.
  *
- * Covered: u = k_hat (opts->u must be NULL), no periodic refresh, d_k = d_v in {16, 32, 64};
- * anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a DEVICE buffer of at least
- * vla_backward_workspace_bytes(B, H, T, d_k) bytes (z_t, e_t and delta_t of every token),
- * owned by the caller and free for reuse once the work enqueued on `stream` has completed.
+ * Covered: u = k_hat (opts->u must be NULL), no periodic refresh, head-major tensors,
+ * d_k = d_v in {16, 32, 64, 128}; anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a
+ * DEVICE buffer of at least vla_backward_workspace_bytes(B, H, T, d_k) bytes (per token: z_t,
+ * e_t, delta_t of the forward and three vectors the two reverse scans exchange; the final
+ * states), owned by the caller and free for reuse once the work enqueued on `stream` has completed.
  */
 int vla_backward(const void* q, const void* k, const void* v, float lambda_,
                  int B, int H, int T, int d_k, int d_v,

@@ -256,7 +256,7 @@ class VlaGrads(NamedTuple):
 def vla_backward(q, k, v, lam: float, d_out, *, S0=None, A0=None, z0=None, dS_T=None, dA_T=None,
                  dz_T=None, flags: int = 0, eps: float = 1e-4, workspace=None, status=None,
                  stream: Optional[torch.cuda.Stream] = None, want_status: bool = True) -> VlaGrads:
-    """Gradients of the forward scan for CUDA tensors (u = k_hat, d in {16, 32, 64}); the
+    """Gradients of the forward scan for CUDA tensors (u = k_hat, d in {16, 32, 64, 128}); the
     forward is recomputed inside.  ``d_out`` is dL/d(out); ``dS_T, dA_T, dz_T`` default to zero."""
     lib = load_library()
     B, H, T, dk = q.shape

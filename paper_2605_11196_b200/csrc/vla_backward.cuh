@@ -138,7 +138,12 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
         const int c = e * 32 + lane;
         if (c < D) {
           kh[c] = kx[e] * inv;
-          if (!ident) zk[c] += kx[e];
+          if (!ident) {
+            zk[c] += kx[e];
+            // the reverse sweep restarts its walk back of the key sum from these (a walk from
+            // the final sum alone would cancel catastrophically at the early tokens)
+            if ((t & 15) == 15) p.zkc[(size_t(unit) * ((T + 15) / 16) + size_t(t >> 4)) * D + c] = zk[c];
+          }
         }
       }
     }
@@ -268,7 +273,9 @@ __global__ void __launch_bounds__(256) vla_backward_token_kernel(const BackwardP
       if (c < D) {
         okh[c] = kx[e] / nk;
         oal[c] = sc * zx[e];
-        const float zkc = last ? nzk[c] : (ident ? nzk[c] : nzk[c] - nkf[c]);
+        float zkc = last ? nzk[c] : (ident ? nzk[c] : nzk[c] - nkf[c]);
+        if (!ident && !last && (t & 15) == 15)
+          zkc = __ldcg(p.zkc + (size_t(unit) * ((T + 15) / 16) + size_t(t >> 4)) * D + c);
         ozk[c] = zkc;
         dn = fmaf(zkc, qx[e], dn);
         qa = fmaf(qx[e], sc * zx[e], qa);

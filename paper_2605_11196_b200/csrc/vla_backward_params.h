@@ -25,6 +25,7 @@ struct BackwardParams {
   float* zst;           // workspace [units, T, D]  z_t
   float* est;           // workspace [units, T, D]  e_t
   float* dst;           // workspace [units, T]     delta_t
+  float* zkc;           // workspace [units, ceil(T / 16), D]  key sum after each 16 tokens
   int* status;
   float lambda;
   float eps;
@@ -48,6 +49,7 @@ struct BackwardSplitParams {
   const float* zst;     // [units, T, D] z_t
   const float* est;     // [units, T, D] e_t
   const float* dst;     // [units, T]    delta_t
+  const float* zkc;     // [units, ceil(T / 16), D] key sum after each 16 tokens (paper mode)
   float* dal;           // [units, T, D] S side -> A side: dL/d alpha_t
   float* dkS;           // [units, T, D] S side -> A side: S-side part of dL/d k_hat_t
   float* gzt;           // [units, T, D] S side -> A side: dL/d(key sum) seen by token t

@@ -186,7 +186,11 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
       bwd_ld<EPL>(est + o, pe);
       bwd_ld<EPL>(gdo + o, pg);
     };
-    auto open_token = [&](int t, bool last) {
+    // the key sum seen by token t: from the forward's checkpoint at the last token of each group
+    // of 16, else walked back one token from t + 1 (at most 15 subtractions from a checkpoint)
+    const int nck = (T + 15) / 16;
+    auto open_token = [&](int t) {
+      const bool last = t == T - 1 || (t & 15) == 15;
       float kx[EPL], qx[EPL], khx[EPL], alx[EPL], zkx[EPL], dyx[EPL];
       float ss = 0.f, zz = 0.f;
 #pragma unroll
@@ -197,14 +201,17 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
         ss = fmaf(kk, kk, ss);
         zz = fmaf(pz[e], pz[e], zz);
       }
-      if (last) {
-        bwd_ld<EPL>(p.zT + size_t(unit) * D + c0, zkx);
+      if (ident) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) zkx[e] = 0.0f;   // not used: o = S q has no denominator
+      } else if (last) {
+        bwd_ld<EPL>(p.zkc + (size_t(unit) * nck + size_t(t >> 4)) * D + c0, zkx);
       } else {
         float nz[EPL], nk2[EPL];
         bwd_ld<EPL>(cvec(t + 1, cZk) + c0, nz);
         bwd_ld<EPL>(cvec(t + 1, cKf) + c0, nk2);
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) zkx[e] = ident ? nz[e] : nz[e] - nk2[e];
+        for (int e = 0; e < EPL; ++e) zkx[e] = nz[e] - nk2[e];
       }
       ss = warp_sum(ss);
       zz = warp_sum(zz);
@@ -243,16 +250,16 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
     };
     if (T > 0) {
       fetch_token(T - 1);
-      open_token(T - 1, true);
+      open_token(T - 1);
       fetch_token(T - 2);
-      if (T >= 2) open_token(T - 2, false);
+      if (T >= 2) open_token(T - 2);
       fetch_token(T - 3);
     }
     cta_sync();
     cta_sync();
     for (int t = T - 1; t >= 0; --t) {
       if (t - 2 >= 0) {
-        open_token(t - 2, false);
+        open_token(t - 2);
         fetch_token(t - 3);
       }
       cta_sync();
@@ -387,24 +394,28 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
     cta_sync();
     for (int t = T - 1; t >= 0; --t) {
       const float qal = cscl[t & (NCTX - 1)][sQal];
-      float dyr[R], der[R], etr[R];
-      bwd_ld<R>(cvec(t, cDy) + row0, dyr);
-      bwd_ld<R>(rowv[t % 3][1] + row0, der);
-      bwd_ld<R>(cvec(t, cEt) + row0, etr);
-#pragma unroll
-      for (int r = 0; r < R; ++r) der[r] = fmaf(dyr[r], qal, der[r]);      // (GS + dy qf^T) alpha
+      constexpr int RG = R >= 4 ? 4 : R;   // rows in hand at a time: their scalars are reloaded, not kept
       float2 cc[3][RP];
 #pragma unroll
       for (int m = 0; m < RP; ++m) { cc[0][m] = make_float2(0.f, 0.f); cc[1][m] = cc[0][m]; cc[2][m] = cc[0][m]; }
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const float2 d2 = make_float2(dyr[r], dyr[r]), e2 = make_float2(etr[r], etr[r]);
-        const float2 r2 = make_float2(der[r], der[r]);
+      for (int rg = 0; rg < R / RG; ++rg) {
+        float dyr[RG], der[RG], etr[RG];
+        bwd_ld<RG>(cvec(t, cDy) + row0 + rg * RG, dyr);
+        bwd_ld<RG>(rowv[t % 3][1] + row0 + rg * RG, der);
+        bwd_ld<RG>(cvec(t, cEt) + row0 + rg * RG, etr);
 #pragma unroll
-        for (int m = 0; m < RP; ++m) {
-          cc[0][m] = bwd_ffma2(S[r][m], d2, cc[0][m]);
-          cc[1][m] = bwd_ffma2(GS[r][m], e2, cc[1][m]);
-          cc[2][m] = bwd_ffma2(S[r][m], r2, cc[2][m]);
+        for (int i = 0; i < RG; ++i) {
+          const int r = rg * RG + i;
+          const float de = fmaf(dyr[i], qal, der[i]);      // (GS + dy qf^T) alpha
+          const float2 d2 = make_float2(dyr[i], dyr[i]), e2 = make_float2(etr[i], etr[i]);
+          const float2 r2 = make_float2(de, de);
+#pragma unroll
+          for (int m = 0; m < RP; ++m) {
+            cc[0][m] = bwd_ffma2(S[r][m], d2, cc[0][m]);
+            cc[1][m] = bwd_ffma2(GS[r][m], e2, cc[1][m]);
+            cc[2][m] = bwd_ffma2(S[r][m], r2, cc[2][m]);
+          }
         }
       }
       if constexpr (TX == 16) {
@@ -438,14 +449,23 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
       bwd_ld<RC>(cvec(t, cKh) + col0, kv);
       bwd_ld<RC>(cvec(t, cAl) + col0, av);
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const float2 d2 = make_float2(dyr[r], dyr[r]), e2 = make_float2(-etr[r], -etr[r]);
-        const float2 r2 = make_float2(-der[r], -der[r]);
+      for (int rg = 0; rg < R / RG; ++rg) {
+        float dyr[RG], der[RG], etr[RG];
+        bwd_ld<RG>(cvec(t, cDy) + row0 + rg * RG, dyr);
+        bwd_ld<RG>(rowv[t % 3][1] + row0 + rg * RG, der);
+        bwd_ld<RG>(cvec(t, cEt) + row0 + rg * RG, etr);
 #pragma unroll
-        for (int m = 0; m < RP; ++m) {
-          GS[r][m] = bwd_ffma2(d2, make_float2(qv[2 * m], qv[2 * m + 1]), GS[r][m]);
-          GS[r][m] = bwd_ffma2(r2, make_float2(kv[2 * m], kv[2 * m + 1]), GS[r][m]);
-          S[r][m] = bwd_ffma2(e2, make_float2(av[2 * m], av[2 * m + 1]), S[r][m]);
+        for (int i = 0; i < RG; ++i) {
+          const int r = rg * RG + i;
+          const float de = fmaf(dyr[i], qal, der[i]);
+          const float2 d2 = make_float2(dyr[i], dyr[i]), e2 = make_float2(-etr[i], -etr[i]);
+          const float2 r2 = make_float2(-de, -de);
+#pragma unroll
+          for (int m = 0; m < RP; ++m) {
+            GS[r][m] = bwd_ffma2(d2, make_float2(qv[2 * m], qv[2 * m + 1]), GS[r][m]);
+            GS[r][m] = bwd_ffma2(r2, make_float2(kv[2 * m], kv[2 * m + 1]), GS[r][m]);
+            S[r][m] = bwd_ffma2(e2, make_float2(av[2 * m], av[2 * m + 1]), S[r][m]);
+          }
         }
       }
       if (t >= 1) row_dots(t - 1);

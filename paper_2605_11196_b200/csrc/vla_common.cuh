@@ -43,6 +43,7 @@ struct ScanParams {
   float* stash_z;
   float* stash_e;
   float* stash_delta;
+  float* stash_zk;           // [units, ceil(T / 16), D]: the key sum after each chunk of 16 tokens
   // Token-major tensors (VLA_FLAG_TOKEN_MAJOR): q, k, v, u, out are [B, T, heads, D] instead of
   // [B, heads, T, D]; unit = b * heads + h.  The states keep their [units, D, D] layout.
   int heads;

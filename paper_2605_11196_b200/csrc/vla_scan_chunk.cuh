@@ -697,6 +697,9 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
         }
         const float tot = warp_reduce_scatter16(pr, lane);
         if ((lane & 1) == 0) denp[gw * C + (lane >> 1)] = tot;
+        // the backward pass restarts its walk back of the key sum from these (a walk from the
+        // final sum alone would cancel catastrophically at the early tokens)
+        if (STASH && p.stash_zk) p.stash_zk[(size_t(unit) * size_t(nch_unit) + size_t(pc.cb + c)) * D + g] = zk;
       }
 
       // ---- Z0 = A U^T (U = K when no u is given); with an explicit u also W0 = A K^T

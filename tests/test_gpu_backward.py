@@ -97,3 +97,31 @@ def test_mid_workload_gradients_and_what_is_not_covered():
     with pytest.raises(vla.VlaError) as ei:
         vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 16, 48), device=dev))
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_throughput_shape_sampled_units(flags):
+    """Units of the headline shape (d = 128, T = 8192, bf16), whole sequences: the longest walk
+    back through undone updates the workloads ask for.  Three units (the oracle's fp64 reverse
+    pass takes seconds per unit); the kernels are launched one CTA per unit as at full size."""
+    w = W.Workload("t", 1, 3, 128, 8192, "bf16", 4)
+    q, k, v = W.make_inputs(w)
+    d_out = torch.randn((1, 3, 8192, 128), generator=torch.Generator().manual_seed(5))
+    got, ref = _run_both(q, k, v, w.lam, d_out, flags=flags)
+    errs = _check(got, ref, 1e-3, "backward throughput-shaped")
+    print(flags, errs)
+
+
+@pytest.mark.parametrize("d,T", [(16, 4096), (32, 4099)])
+def test_long_walk_back_keeps_the_early_tokens(d, T):
+    """Paper mode over thousands of tokens: the readout denominators of the early tokens are
+    small against the final key sum, so they must come from the forward's checkpoints, not
+    from subtracting every key from the final sum."""
+    w = W.Workload("t", 1, 2, d, T, "f32", 9)
+    q, k, v = W.make_inputs(w)
+    d_out = torch.randn((1, 2, T, d), generator=torch.Generator().manual_seed(6))
+    got, ref = _run_both(q, k, v, w.lam, d_out)
+    _check(got, ref, 1e-3, "backward long d=%d" % d)
+    early = slice(0, 64)
+    e = np.abs(got.dq.cpu().double().numpy()[:, :, early] - ref.dq[:, :, early]).max() / np.abs(ref.dq[:, :, early]).max()
+    assert e <= 1e-3, e

@@ -429,3 +429,17 @@ def test_token_major_long_units_and_where_it_is_refused():
     with pytest.raises(vla.VlaError) as ei:
         vla.vla_forward_seqpar(q, k, v, 1.0, segments=2, flags=TOKEN_MAJOR)
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("option", ["explicit_u", "refresh", "explicit_u_refresh"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_throughput_shape_with_algorithm_1_options(option, flags):
+    """Whole sequences of the headline shape (d = 128, T = 8192, bf16) on the general path of
+    the chunk kernel: explicit u = unit / sqrt(d), the periodic refresh every 20 steps, both."""
+    w = W.Workload("t", 1, 4, 128, 8192, "bf16", 4)
+    q, k, v = W.make_inputs(w)
+    u = W.make_u(w, 128 ** -0.5) if "explicit_u" in option else None
+    refresh = (20, 1e-3, 0) if "refresh" in option else None
+    errs, _, _ = check_parity(q, k, v, w.lam, 1e-3, u=u, flags=flags, refresh=refresh,
+                              kernel=vla.VLA_KERNEL_CHUNK, label=option)
+    print(option, flags, errs)

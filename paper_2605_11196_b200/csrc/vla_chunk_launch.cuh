@@ -8,6 +8,10 @@
 
 namespace vla {
 
+// Tensor maps of q, k, v[, u], out as 4-d tensors (d, H, T, B) with a box of one chunk
+// (d x 1 x 16 x 1).  Defined in vla_launch.cu.
+int encode_token_major_maps(const ScanParams& p, int d, int dtype, bool has_u, TokenMajorMaps* maps);
+
 // TM: q, k, v, u, out are [B, T, H, d] (an instantiation of its own: one bulk copy per token row).
 template <int D, typename TIn, int UM, bool TM>
 int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
@@ -46,14 +50,22 @@ int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
   } else {
     cudaGetLastError();
   }
-  if (sp.balanced) kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
-  else kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  typename ChunkMapsArg<TM>::type maps;
+  if constexpr (TM) {
+    const int rc = encode_token_major_maps(p, D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, UM == kUTensor, &maps);
+    if (rc != VLA_OK) return rc;
+  } else {
+    maps.unused = 0;
+  }
+  if (sp.balanced) kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
+  else kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
 template <int D, typename TIn, int UM>
 int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
-  if (p.flags & VLA_FLAG_TOKEN_MAJOR) return launch_chunk_um_tm<D, TIn, UM, true>(p, st);
+  // no tokens: nothing is read or written in either layout
+  if ((p.flags & VLA_FLAG_TOKEN_MAJOR) && p.T > 0) return launch_chunk_um_tm<D, TIn, UM, true>(p, st);
   return launch_chunk_um_tm<D, TIn, UM, false>(p, st);
 }
 
@@ -72,7 +84,7 @@ int launch_chunk_stash_t(const ScanParams& p, cudaStream_t st) {
   sp.balanced = 0;
   sp.grid = p.units;
   sp.epoch = 0;
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, EmptyMaps{0});
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
@@ -100,7 +112,7 @@ int launch_chunk_tri_um(const ScanParams& p, cudaStream_t st) {
   sp.balanced = 0;
   sp.grid = p.units;
   sp.epoch = 0;
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, EmptyMaps{0});
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

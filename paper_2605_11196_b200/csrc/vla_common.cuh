@@ -2,6 +2,7 @@
 // bounded mbarrier waits, 1-D bulk-async (TMA) copies, small math helpers.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -152,6 +153,29 @@ __device__ __forceinline__ void bulk_store_rows(TEl* gmem_dst, const TEl* smem_s
     for (int i = 0; i < n; ++i)
       bulk_store(gmem_dst + size_t(i) * stride, smem_src + size_t(i) * D, uint32_t(D * sizeof(TEl)));
   }
+}
+
+// ---- tiled TMA through a tensor map (token-major tensors).  The innermost coordinate is always
+// 0 here (16-byte rule), loads may run past the tensor's end (zero fill), stores are clipped.
+struct EmptyMaps { char unused; };
+struct alignas(64) TokenMajorMaps { CUtensorMap q, k, v, u, out; };
+template <bool TM> struct ChunkMapsArg { using type = EmptyMaps; };
+template <> struct ChunkMapsArg<true> { using type = TokenMajorMaps; };
+
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                            int c3, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::
+          "r"(smem_u32(smem_dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                             const void* smem_src) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(smem_src))
+               : "memory");
 }
 
 template <int N>

@@ -189,6 +189,53 @@ int launch_backward_split(int d, int dtype, const BackwardSplitParams& p, cudaSt
   }
 }
 
+// ---------------------------------------------------------------- tensor maps (token-major tensors)
+namespace {
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  // resolved through the runtime, so the library needs no link against the driver
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      f = nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+int encode_one(CUtensorMap* m, const void* base, int d, int heads, int T, int B, bool f32) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return VLA_ERR_CUDA;
+  const cuuint64_t es = f32 ? 4 : 2;
+  const cuuint64_t dims[4] = {cuuint64_t(d), cuuint64_t(heads), cuuint64_t(T), cuuint64_t(B)};
+  const cuuint64_t strides[3] = {cuuint64_t(d) * es, cuuint64_t(heads) * d * es, cuuint64_t(T) * heads * d * es};
+  const cuuint32_t box[4] = {cuuint32_t(d), 1u, 16u, 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUresult r = enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+                         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? VLA_OK : VLA_ERR_CUDA;
+}
+}  // namespace
+
+int encode_token_major_maps(const ScanParams& p, int d, int dtype, bool has_u, TokenMajorMaps* maps) {
+  if (p.heads <= 0 || p.units % p.heads != 0 || p.T <= 0) return VLA_ERR_INVALID_ARG;
+  const int B = p.units / p.heads;
+  const bool f32 = dtype == VLA_F32;
+  int rc = encode_one(&maps->q, p.q, d, p.heads, p.T, B, f32);
+  if (rc == VLA_OK) rc = encode_one(&maps->k, p.k, d, p.heads, p.T, B, f32);
+  if (rc == VLA_OK) rc = encode_one(&maps->v, p.v, d, p.heads, p.T, B, f32);
+  if (rc == VLA_OK) rc = encode_one(&maps->u, has_u ? p.u : p.k, d, p.heads, p.T, B, f32);
+  if (rc == VLA_OK) rc = encode_one(&maps->out, p.out, d, p.heads, p.T, B, true);
+  return rc;
+}
+
 // ---------------------------------------------------------------- penalty directions from W_u
 namespace {
 template <int D, typename TIn, typename TOut>

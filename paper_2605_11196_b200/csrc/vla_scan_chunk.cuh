@@ -371,10 +371,18 @@ __device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) 
 // STASH: the launch also leaves z_t, e_t, delta_t of every token in global memory (and may
 // drop the readout) for the backward pass; a separate instantiation so that the plain forward
 // kernel carries none of it.
+// TM: q, k, v, u, out are [B, T, H, d]: the 16 rows of a chunk are H * d apart, so they move as
+// one tiled TMA request per array (box d x 1 x 16 x 1 of the 4-d tensor) through the tensor maps
+// in `maps`; the head-major instantiations take an empty struct there.
 template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false, bool STASH = false, bool TM = false>
 __global__ void __launch_bounds__((TRI ? 3 : 2) * D, (TRI && sizeof(TIn) == 2) ? 2 : 1)
-vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
+vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
+                      const __grid_constant__ typename ChunkMapsArg<TM>::type maps) {
   using Cfg = ChunkCfg<D, TIn, UM, TRI>;
+  static_assert(!TM || (!TRI && !STASH), "token-major tensors: the plain forward kernels");
+  static_assert(!TM || (Cfg::raw_bytes + sizeof(float) * (Cfg::KRING * Cfg::kslot_floats + Cfg::RING * Cfg::slot_floats +
+                                                          Cfg::a_floats + 3 * Cfg::C * D)) % 128 == 0,
+                "the out stage must be 128-byte aligned for a tiled TMA store");
   static_assert(!TRI || (D <= 64 && !BALANCED), "three groups: d <= 64, one CTA per unit");
   static_assert(!STASH || (UM == kUKhat && !TRI && !BALANCED), "the stash belongs to the plain u = k_hat kernel");
   constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly
@@ -488,19 +496,15 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
       if (!pscan_cta) bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &full[s]);
       if (UT) bulk_load(dst + 3 * C * D, static_cast<const TIn*>(p.u) + tok * D, bytes, &full[s]);
     } else {
-      // [B, T, H, d] tensors: one bulk copy per token row, lane r of the group's first warp
-      // (all of which calls this) taking row r
-      const int r = tid & 31;
-      if (r == 0) mbar_arrive_expect_tx(&full[s], NIN * bytes);
-      __syncwarp();
-      if (r < n) {
-        const size_t off = token_offset(p, uin, size_t(t_begin) + size_t(c) * C + r, D);
-        const uint32_t rb = uint32_t(D * sizeof(TIn));
-        bulk_load(dst + 0 * C * D + r * D, static_cast<const TIn*>(p.q) + off, rb, &full[s]);
-        bulk_load(dst + 1 * C * D + r * D, static_cast<const TIn*>(p.k) + off, rb, &full[s]);
-        bulk_load(dst + 2 * C * D + r * D, static_cast<const TIn*>(p.v) + off, rb, &full[s]);
-        if (UT) bulk_load(dst + 3 * C * D + r * D, static_cast<const TIn*>(p.u) + off, rb, &full[s]);
-      }
+      // [B, T, H, d] tensors: one tiled request per array; rows past T arrive as zeros and
+      // count towards the bytes like any other
+      const int b = uin / p.heads, h = uin - b * p.heads, t0 = t_begin + c * C;
+      mbar_arrive_expect_tx(&full[s], NIN * uint32_t(C * D * sizeof(TIn)));
+      tma_load_4d(dst + 0 * C * D, &maps.q, 0, h, t0, b, &full[s]);
+      tma_load_4d(dst + 1 * C * D, &maps.k, 0, h, t0, b, &full[s]);
+      tma_load_4d(dst + 2 * C * D, &maps.v, 0, h, t0, b, &full[s]);
+      if (UT) tma_load_4d(dst + 3 * C * D, &maps.u, 0, h, t0, b, &full[s]);
+      (void)bytes;
     }
   };
 
@@ -533,7 +537,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
     }
   }
   __syncthreads();
-  if (TM ? tid < 32 : tid == 0) {  // thread 0 (token-major tensors: warp 0) of group A is the TMA producer
+  if (tid == 0) {  // thread 0 of group A is the TMA producer
     for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue(c);
   }
 
@@ -663,7 +667,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
 
     if (nchunks > 0) prep_inputs(0, 0, NWG);
     group_bar(1, NG);
-    if ((TM ? g < 32 : g == 0) && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
+    if (g == 0 && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
 
     for (int c = 0; c < nchunks; ++c) {
       const int slot = c % RING;
@@ -797,7 +801,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
       }
       group_bar(1, NG);
       // the raw stage of chunk c + 1 has been consumed: refill it
-      if ((TM ? g < 32 : g == 0) && c + 1 + NSTAGE < nchunks) issue(c + 1 + NSTAGE);
+      if (g == 0 && c + 1 + NSTAGE < nchunks) issue(c + 1 + NSTAGE);
       VLA_MARK(4)
 
       // ---- row g of Z by forward substitution: z_t = z0_t - sum_{s<t} L[t][s] z_s
@@ -946,7 +950,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
         VS[t * D + g] = (TRI && pscan ? 0.0f : Vf[t * D + g]) - x;
       });
       tile_matvec_chunk<TR, TW, LPR, D, C>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
-      if (TM ? g < C : g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
+      if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
       // explicit u: the ring's Z slot carries a_t = A_t k_hat_t; the two small matrices
       // k_hat_t . a_s and q_t . a_s are formed here (for u = k_hat they come from group A)
       const float* Gm = GuT;
@@ -1014,17 +1018,16 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
       }
       fence_async_smem();
       group_bar(sbar, NG);  // Eps and the out stage complete
-      if (TM ? g < C : g == 0) {   // token-major tensors: thread r stores row r, in bulk groups of its own
+      if (g == 0) {
         const size_t tq = size_t(t_begin) + size_t(c) * C;
         float* odst = pscan ? p.out2 : p.out;
         if (!STASH || odst) {   // a backward pass that only wants the stash passes no readout buffer
           if constexpr (!TM) {
             bulk_store(odst + (size_t(uin) * size_t(p.T) + tq) * D, ostage + size_t(c & 1) * C * D,
                        uint32_t(n) * D * sizeof(float));
-          } else {
-            if (g < n)
-              bulk_store(odst + token_offset(p, uin, tq + g, D), ostage + size_t(c & 1) * C * D + g * D,
-                         uint32_t(D * sizeof(float)));
+          } else {   // rows past T are clipped by the tensor map
+            const int b = uin / p.heads, h = uin - b * p.heads;
+            tma_store_4d(&maps.out, 0, h, int(tq), b, ostage + size_t(c & 1) * C * D);
           }
           bulk_commit();
         }
@@ -1048,7 +1051,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp) {
               make_float4(st[r][2 * m].x, st[r][2 * m].y, st[r][2 * m + 1].x, st[r][2 * m + 1].y);
       }
     }
-    if (TM ? g < C : g == 0) bulk_wait_all<0>();
+    if (g == 0) bulk_wait_all<0>();
   }
   if (to_handoff) {   // every thread's state stores precede the flag
     __syncthreads();

@@ -83,6 +83,8 @@ typedef struct {
   int32_t refresh_period;
   float refresh_eta;
   int64_t step_offset;   /* tokens of this sequence processed by earlier calls (state carry)     */
+  float* du;             /* vla_backward with explicit u: [B,H,T,d_k] fp32 gradient of u (required
+                            when u is given there; ignored by the forward calls)                 */
 } vla_opts_t;
 
 /*
@@ -202,8 +204,10 @@ size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
  * dv [B,H,T,d_v] and, when non-NULL, dS0, dA0, dz0.  The forward is recomputed inside; no
  * state of the forward call is needed.  In identity-map mode z_T = z0, so dz0 = dz_T.
  *
- * Covered: u = k_hat (opts->u must be NULL), no periodic refresh, head-major tensors,
- * d_k = d_v in {16, 32, 64, 128}; anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a
+ * Covered: u = k_hat (opts->u NULL; d_k = d_v in {16, 32, 64, 128}) or explicit penalty
+ * directions (opts->u given, used verbatim as in vla_forward; their gradient goes to opts->du,
+ * which must then be non-NULL; d in {32, 64, 128}); no periodic refresh, head-major tensors;
+ * anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a
  * DEVICE buffer of at least vla_backward_workspace_bytes(B, H, T, d_k) bytes (per token: z_t,
  * e_t, delta_t of the forward and three vectors the two reverse scans exchange; the final
  * states), owned by the caller and free for reuse once the work enqueued on `stream` has completed.

@@ -36,7 +36,7 @@ class VlaOpts(ctypes.Structure):
                 ("u", ctypes.c_void_p), ("flags", ctypes.c_uint32), ("eps", ctypes.c_float),
                 ("z0", ctypes.c_void_p), ("zT", ctypes.c_void_p), ("status", ctypes.c_void_p),
                 ("kernel", ctypes.c_int32), ("refresh_period", ctypes.c_int32),
-                ("refresh_eta", ctypes.c_float), ("step_offset", ctypes.c_int64)]
+                ("refresh_eta", ctypes.c_float), ("step_offset", ctypes.c_int64), ("du", ctypes.c_void_p)]
 
 
 class VlaError(RuntimeError):
@@ -251,13 +251,15 @@ class VlaGrads(NamedTuple):
     dA0: torch.Tensor
     dz0: torch.Tensor
     status: Optional[torch.Tensor]
+    du: Optional[torch.Tensor] = None
 
 
-def vla_backward(q, k, v, lam: float, d_out, *, S0=None, A0=None, z0=None, dS_T=None, dA_T=None,
+def vla_backward(q, k, v, lam: float, d_out, *, u=None, S0=None, A0=None, z0=None, dS_T=None, dA_T=None,
                  dz_T=None, flags: int = 0, eps: float = 1e-4, workspace=None, status=None,
                  stream: Optional[torch.cuda.Stream] = None, want_status: bool = True) -> VlaGrads:
-    """Gradients of the forward scan for CUDA tensors (u = k_hat, d in {16, 32, 64, 128}); the
-    forward is recomputed inside.  ``d_out`` is dL/d(out); ``dS_T, dA_T, dz_T`` default to zero."""
+    """Gradients of the forward scan for CUDA tensors (u = k_hat: d in {16, 32, 64, 128}; explicit
+    ``u``: d in {32, 64, 128}, its gradient is returned as ``du``); the forward is recomputed
+    inside.  ``d_out`` is dL/d(out); ``dS_T, dA_T, dz_T`` default to zero."""
     lib = load_library()
     B, H, T, dk = q.shape
     dv_ = v.shape[-1]
@@ -266,6 +268,7 @@ def vla_backward(q, k, v, lam: float, d_out, *, S0=None, A0=None, z0=None, dS_T=
     f32 = torch.float32
     _chk(q, (B, H, T, dk), q.dtype, "q"); _chk(k, (B, H, T, dk), q.dtype, "k")
     _chk(v, (B, H, T, dv_), q.dtype, "v"); _chk(d_out, (B, H, T, dv_), f32, "d_out")
+    _chk(u, (B, H, T, dk), q.dtype, "u")
     _chk(S0, (B, H, dv_, dk), f32, "S0"); _chk(A0, (B, H, dk, dk), f32, "A0"); _chk(z0, (B, H, dk), f32, "z0")
     _chk(dS_T, (B, H, dv_, dk), f32, "dS_T"); _chk(dA_T, (B, H, dk, dk), f32, "dA_T")
     _chk(dz_T, (B, H, dk), f32, "dz_T")
@@ -281,7 +284,9 @@ def vla_backward(q, k, v, lam: float, d_out, *, S0=None, A0=None, z0=None, dS_T=
     need = int(lib.vla_backward_workspace_bytes(B, H, T, dk))
     if workspace is None:
         workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
-    opts = _make_opts(dt, None, flags, eps, z0, None, status, VLA_KERNEL_AUTO, None)
+    du = None if u is None else torch.empty((B, H, T, dk), dtype=f32, device=dev)
+    opts = _make_opts(dt, u, flags, eps, z0, None, status, VLA_KERNEL_AUTO, None)
+    opts.du = None if du is None else du.data_ptr()
     with torch.cuda.device(dev):
         rc = lib.vla_backward(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv_, _ptr(S0), _ptr(A0),
                               _ptr(d_out), _ptr(dS_T), _ptr(dA_T), _ptr(dz_T), _ptr(dq), _ptr(dkk),
@@ -289,7 +294,7 @@ def vla_backward(q, k, v, lam: float, d_out, *, S0=None, A0=None, z0=None, dS_T=
                               _ptr(workspace), workspace.numel(), ctypes.c_void_p(st.cuda_stream))
     if rc != VLA_OK:
         raise VlaError(rc, "vla_backward")
-    return VlaGrads(dq, dkk, dvv, dS0, dA0, dz0, status)
+    return VlaGrads(dq, dkk, dvv, dS0, dA0, dz0, status, du)
 
 
 def measure_fp32_fma_tflops(device=None, iters: int = 4096, reps: int = 5) -> float:

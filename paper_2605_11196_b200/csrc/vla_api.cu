@@ -196,7 +196,7 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
   p.refresh_period = o.refresh_period; p.refresh_eta = o.refresh_eta;
   p.step_offset = o.step_offset; p.u_is_khat = 0;
   p.n_main = 0; p.out2 = nullptr;
-  p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr; p.stash_zk = nullptr;
+  p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr; p.stash_zk = nullptr; p.stash_a = nullptr;
   p.heads = H;
   return launch(p, d_k, o.qkv_dtype, o.kernel, static_cast<cudaStream_t>(stream));
 }
@@ -437,7 +437,7 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   // d <= 64: N CTAs of three warp groups; d = 128: 2N CTAs, the transfer scans second
   p.T = T / P; p.units = seqpar_tri(d_k) ? N : 2 * N; p.n_main = N; p.flags = o.flags;
   p.refresh_period = 0; p.refresh_eta = 0.0f; p.step_offset = 0; p.u_is_khat = 0;
-  p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr; p.stash_zk = nullptr;
+  p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr; p.stash_zk = nullptr; p.stash_a = nullptr;
   p.heads = H;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = vla::seqpar_before_scan(d_k, o.qkv_dtype, sp, st);
@@ -454,9 +454,9 @@ size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k) {
   const size_t vec = round256(units * T * d_k * sizeof(float));
   const size_t mat = round256(units * d_k * d_k * sizeof(float));
   // z, e, dalpha, dk_hat (S part), key-sum gradient per token; delta per token; S_T, A_T, key sum;
-  // the key sum after every 16 tokens
+  // the key sum after every 16 tokens; a_t per token (explicit u)
   const size_t ck = round256(units * ((size_t(T) + 15) / 16) * d_k * sizeof(float));
-  return 5 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + ck + 256;
+  return 6 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + ck + 256;
 }
 
 int vla_backward(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,
@@ -469,10 +469,11 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   if (rc != VLA_OK) return rc;
   rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, d_out);
   if (rc != VLA_OK) return rc;
-  if (o.u || o.refresh_period > 0 || (o.flags & VLA_FLAG_TOKEN_MAJOR)) return VLA_ERR_UNSUPPORTED;
+  if (o.refresh_period > 0 || (o.flags & VLA_FLAG_TOKEN_MAJOR)) return VLA_ERR_UNSUPPORTED;
+  if (o.u && d_k < 32) return VLA_ERR_UNSUPPORTED;   // explicit u: the two reverse scans only
   const int units = B * H;
-  if (units > 0 && T > 0 && (!dq || !dk || !dv)) return VLA_ERR_INVALID_ARG;
-  const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0};
+  if (units > 0 && T > 0 && (!dq || !dk || !dv || (o.u && !o.du))) return VLA_ERR_INVALID_ARG;
+  const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0, o.u, o.du};
   for (const void* ptr : ptrs)
     if (!aligned16(ptr)) return VLA_ERR_ALIGNMENT;
   if (o.status && (reinterpret_cast<uintptr_t>(o.status) & 3u)) return VLA_ERR_ALIGNMENT;
@@ -486,7 +487,9 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   float* zst = reinterpret_cast<float*>(w);
   float* est = reinterpret_cast<float*>(w + vec);
   float* dst = reinterpret_cast<float*>(w + 2 * vec);
+  const size_t ckb = round256(size_t(units) * ((size_t(T) + 15) / 16) * d_k * sizeof(float));
   float* zkcw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)));
+  float* astw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)) + ckb);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (d_k == 16) {
     // d = 16 has no chunk kernel: the single kernel runs its own token-level forward sweep
@@ -506,20 +509,20 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   float* ATw = reinterpret_cast<float*>(w + 5 * vec + sca + mat);
   float* zTw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat);
   ScanParams f;
-  f.q = q; f.k = k; f.v = v; f.u = nullptr;
+  f.q = q; f.k = k; f.v = v; f.u = o.u;
   f.S0 = S0; f.A0 = A0; f.z0 = o.z0;
   f.out = nullptr; f.S_T = STw; f.A_T = ATw; f.zT = zTw;
   f.status = o.status; f.lambda = lambda_; f.eps = o.eps;
   f.T = T; f.units = units; f.flags = o.flags;
   f.refresh_period = 0; f.refresh_eta = 0.0f; f.step_offset = 0; f.u_is_khat = 0;
   f.n_main = 0; f.out2 = nullptr;
-  f.stash_z = zst; f.stash_e = est; f.stash_delta = dst; f.stash_zk = zkcw;
+  f.stash_z = zst; f.stash_e = est; f.stash_delta = dst; f.stash_zk = zkcw; f.stash_a = o.u ? astw : nullptr;
   f.heads = H;
   rc = vla::launch_chunk_stash(d_k, o.qkv_dtype, f, st);
   if (rc != VLA_OK) return rc;
   // 2. the S-side and A-side reverse scans
   vla::BackwardSplitParams p;
-  p.q = q; p.k = k; p.z0 = o.z0; p.d_out = d_out; p.dS_T = dS_T; p.dA_T = dA_T; p.dz_T = dz_T;
+  p.q = q; p.k = k; p.u = o.u; p.ast = astw; p.du = o.du; p.z0 = o.z0; p.d_out = d_out; p.dS_T = dS_T; p.dA_T = dA_T; p.dz_T = dz_T;
   p.ST = STw; p.AT = ATw; p.zT = zTw; p.zst = zst; p.est = est; p.dst = dst; p.zkc = zkcw;
   p.dal = dalw; p.dkS = dkSw; p.gzt = gztw;
   p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;

@@ -38,6 +38,9 @@ struct BackwardParams {
 struct BackwardSplitParams {
   const void* q;        // [units, T, D]
   const void* k;
+  const void* u;        // [units, T, D] explicit penalty directions, or nullptr (u = k_hat)
+  const float* ast;     // [units, T, D] a_t = A_t k_hat_t of the forward (explicit u only)
+  float* du;            // [units, T, D] gradient of u (explicit u only)
   const float* z0;      // unused by the sweeps (the forward consumed it)
   const float* d_out;   // [units, T, D]
   const float* dS_T;    // [units, D, D] or nullptr

@@ -1,4 +1,5 @@
-// VLA backward pass as two reverse scans (u = k_hat, d in {32, 64, 128}).
+// VLA backward pass as two reverse scans (u = k_hat, or explicit penalty directions u with the
+// template flag UX; d in {32, 64, 128}).
 //
 // The adjoint of the memory state, GS = dL/dS, obeys a recurrence of its own that never looks at
 // the penalty side: GS_{t-1} = GS_t + dy qf^T - de k_hat^T.  So the reverse sweep splits into
@@ -47,7 +48,7 @@ template <int D>
 struct BackwardSplitSmem {
   static constexpr int NW = BwdSplitGeom<D>::NW;
   static constexpr size_t s_bytes = sizeof(float) * (4 * 8 * D + 4 * 4 + 3 * 2 * D + 2 * NW * 3 * D + D);
-  static constexpr size_t a_bytes = sizeof(float) * (4 * 6 * D + 4 * 4 + 3 * 3 * D);
+  static constexpr size_t a_bytes = sizeof(float) * (4 * 7 * D + 4 * 8 + 3 * 3 * D);
 };
 
 // All threads of the CTA, whichever loop they are in.
@@ -124,7 +125,9 @@ __device__ __forceinline__ void rows_reduce(float* v, int lane) {
 }
 
 // ------------------------------------------------------------------------------ S side
-template <int D, typename TIn>
+// UX: explicit penalty directions.  The S side only sees them through alpha_t, which then comes
+// from the stashed a_t = A_t k_hat_t instead of z_t / delta_t.
+template <int D, typename TIn, bool UX>
 __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) vla_backward_s_kernel(const BackwardSplitParams p) {
   using G = BwdSplitGeom<D>;
   constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW, NT = G::NT_S, NCLOSE = G::NCLOSE;
@@ -156,7 +159,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
   const TIn* gq = static_cast<const TIn*>(p.q) + ubase;
   const TIn* gk = static_cast<const TIn*>(p.k) + ubase;
   const float* gdo = p.d_out + ubase;
-  const float* zst = p.zst + ubase;
+  const float* zst = (UX ? p.ast : p.zst) + ubase;   // the vector alpha_t is parallel to
   const float* est = p.est + ubase;
   const float* dst = p.dst + size_t(unit) * T;
 
@@ -217,7 +220,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
       zz = warp_sum(zz);
       const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
       const float idl = 1.0f / pdelta;
-      const float sc = idl / fmaxf(sqrtf(zz) * idl, eps);
+      const float sc = UX ? 1.0f / fmaxf(sqrtf(zz), eps) : idl / fmaxf(sqrtf(zz) * idl, eps);
       float dn = 0.f, qa = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
@@ -492,18 +495,23 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
 // sums, nothing to combine across warps), and the update GA += w k_hat^T, w = da + dz, becomes
 // GAs += (w k_hat^T + k_hat w^T) / 2.  GA itself is needed for dA0 alone and is linear in the
 // w_t: dA0 = dA_T + sum_t w_t k_hat_t^T, formed from the stored w_t by vla_backward_da0_kernel.
-template <int D, typename TIn>
+//
+// UX (explicit u): z = A_{t-1} u, delta = 1 + u.z, a = A_t k_hat.  The adjoint of z then flows to
+// u instead of k_hat: dz = ddelta u - (daz k_hat + 2 g + khz da) / delta, du = ddelta z + A_{t-1} dz,
+// dk_hat = (S part) + A_t da, and the update is GAs += sym(da k_hat^T) + sym(dz u^T);
+// dA0 = dA_T + sum_t (da_t k_hat_t^T + dz_t u_t^T).
+template <int D, typename TIn, bool UX>
 __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) vla_backward_a_kernel(const BackwardSplitParams p) {
   using G = BwdSplitGeom<D>;
   constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW;
   constexpr int RP = RC / 2;
   constexpr int EPL = D / 32;
   constexpr int NCTX = 4;
-  enum { cKf = 0, cKh, cZt, cDa, cDkS, cGz, NV };
-  enum { sDelta = 0, sKhz, sDaz, sNk };
+  enum { cKf = 0, cKh, cZt, cDa, cDkS, cGz, cU, NV };
+  enum { sDelta = 0, sKhz, sDaz, sNk, sUz };
   struct Smem {
     float ctx[NCTX][NV][D];
-    float cscl[NCTX][4];
+    float cscl[NCTX][8];
     float rowv[3][3][D];      // g = GAs z, r1 = A' da, r3 = A' dz, ring of three tokens
   };
   static_assert(sizeof(Smem) == BackwardSplitSmem<D>::a_bytes, "shared memory size of the A side");
@@ -520,17 +528,20 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
   const int T = p.T;
   const size_t ubase = size_t(unit) * size_t(T) * D;
   const TIn* gk = static_cast<const TIn*>(p.k) + ubase;
+  const TIn* gu = UX ? static_cast<const TIn*>(p.u) + ubase : nullptr;
   const float* zst = p.zst + ubase;
   const float* dst = p.dst + size_t(unit) * T;
 
   auto cvec = [&](int t, int which) { return ctx[t & (NCTX - 1)][which]; };
+  auto uvec = [&](int t) { return ctx[t & (NCTX - 1)][UX ? cU : cKh]; };   // the direction delta is taken along
   const int myrow = tx / (TX / R);
   const bool row_writer = (tx % (TX / R)) == 0;
   constexpr int kCloser = NW, kOpener = NW + 1;
 
   // the scalars of token t that hang on the adjoint: ddelta and the factors of dz
-  //   dz = cK k_hat - idl (2 g + khz da),  cK = ddelta - idl daz,  ddelta = (z.g + daz khz) / delta^2
-  struct MidScalars { float idl, ddelta, cK, khz, zg; };
+  //   dz = ddelta u + cK k_hat - idl (2 g + khz da),  cK = -idl daz,  ddelta = (z.g + daz khz) / delta^2
+  //   (u = k_hat: one coefficient cK = ddelta - idl daz on k_hat, cU = 0)
+  struct MidScalars { float idl, ddelta, cK, cU, khz, zg; };
   auto mid_scalars = [&](int t) {
     float zt[EPL], gv[EPL];
     bwd_ld<EPL>(cvec(t, cZt) + c0, zt);
@@ -544,9 +555,10 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
     m.khz = sc[sKhz];
     m.idl = 1.0f / sc[sDelta];
     m.zg = zg;
-    const bool delta_live = (1.0f + m.khz) >= eps;
+    const bool delta_live = (1.0f + sc[sUz]) >= eps;
     m.ddelta = delta_live ? fmaf(sc[sDaz], m.khz, zg) * m.idl * m.idl : 0.0f;
-    m.cK = fmaf(-m.idl, sc[sDaz], m.ddelta);
+    m.cK = UX ? -m.idl * sc[sDaz] : fmaf(-m.idl, sc[sDaz], m.ddelta);
+    m.cU = UX ? m.ddelta : 0.0f;
     return m;
   };
 
@@ -554,7 +566,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
   // updates, then the row dots of token t - 1; the closing warp finishes token t + 1, the
   // opening warp prepares token t - 2.  Loops of their own, as on the S side.
   if (warp == kOpener) {
-    float pk[EPL], pz[EPL], pa[EPL], ps[EPL], pgz[EPL];
+    float pk[EPL], pz[EPL], pa[EPL], ps[EPL], pgz[EPL], pu[EPL], pat[EPL];
     float pdelta = 1.0f;
     auto fetch_token = [&](int t) {
       if (t < 0) return;
@@ -565,33 +577,40 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       bwd_ld<EPL>(p.dal + ubase + o, pa);
       bwd_ld<EPL>(p.dkS + ubase + o, ps);
       bwd_ld<EPL>(p.gzt + ubase + o, pgz);
+      if constexpr (UX) {
+        bwd_ld_in<EPL>(gu + o, pu);
+        bwd_ld<EPL>(p.ast + ubase + o, pat);
+      }
     };
     // k_hat, alpha, da = (dalpha - alpha (alpha.dalpha)) / ||a|| and the scalars of token t
     auto open_token = [&](int t) {
       float kx[EPL], khx[EPL], dax[EPL];
-      float ss = 0.f, zz = 0.f, zpa = 0.f, kz = 0.f;
+      float ss = 0.f, zz = 0.f, zpa = 0.f, kz = 0.f, uz = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
         float kk = pk[e];
         if (!ident) kk = bwd_phi(kk);
         kx[e] = kk;
+        const float av = UX ? pat[e] : pz[e];        // a_t up to the factor 1 / delta when u = k_hat
         ss = fmaf(kk, kk, ss);
-        zz = fmaf(pz[e], pz[e], zz);
-        zpa = fmaf(pz[e], pa[e], zpa);
+        zz = fmaf(av, av, zz);
+        zpa = fmaf(av, pa[e], zpa);
         kz = fmaf(kk, pz[e], kz);
+        if (UX) uz = fmaf(pu[e], pz[e], uz);
       }
       ss = warp_sum(ss); zz = warp_sum(zz); zpa = warp_sum(zpa); kz = warp_sum(kz);
+      if (UX) uz = warp_sum(uz);
       const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
       const float idl = 1.0f / pdelta;
-      const float na = sqrtf(zz) * idl;              // ||a||, a = z / delta
-      const float sc = idl / fmaxf(na, eps);
+      const float na = UX ? sqrtf(zz) : sqrtf(zz) * idl;   // ||a||  (a = z / delta when u = k_hat)
+      const float sc = (UX ? 1.0f : idl) / fmaxf(na, eps);
       const float adal = sc * zpa;                   // alpha . dalpha
       const float khz = kz * ink;
       const float ina = na > eps ? 1.0f / na : 1.0f / eps;
       float daz = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
-        const float al = sc * pz[e];
+        const float al = sc * (UX ? pat[e] : pz[e]);
         dax[e] = na > eps ? (pa[e] - al * adal) * ina : pa[e] * ina;
         khx[e] = kx[e] * ink;
         daz = fmaf(dax[e], pz[e], daz);
@@ -603,9 +622,11 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       bwd_st<EPL>(cvec(t, cDa) + c0, dax);
       bwd_st<EPL>(cvec(t, cDkS) + c0, ps);
       bwd_st<EPL>(cvec(t, cGz) + c0, pgz);
+      if constexpr (UX) bwd_st<EPL>(cvec(t, cU) + c0, pu);
       if (lane == 0) {
         float* os = cscl[t & (NCTX - 1)];
         os[sDelta] = pdelta; os[sKhz] = khz; os[sDaz] = daz; os[sNk] = sqrtf(ss);
+        os[sUz] = UX ? uz : khz;
       }
     };
     if (T > 0) {
@@ -628,7 +649,8 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
     // dk of token t; w_t = da + dz goes where dalpha_t was (read two segments ago) for dA0
     auto close_token = [&](int t) {
       const MidScalars ms = mid_scalars(t);
-      float kf[EPL], kh[EPL], zt[EPL], da[EPL], dkS[EPL], gzv[EPL], gv[EPL], r1[EPL], r3[EPL];
+      float kf[EPL], kh[EPL], zt[EPL], da[EPL], dkS[EPL], gzv[EPL], gv[EPL], r1[EPL], r3[EPL], uv[EPL];
+      bwd_ld<EPL>(uvec(t) + c0, uv);
       bwd_ld<EPL>(cvec(t, cKf) + c0, kf);
       bwd_ld<EPL>(cvec(t, cKh) + c0, kh);
       bwd_ld<EPL>(cvec(t, cZt) + c0, zt);
@@ -639,17 +661,20 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       bwd_ld<EPL>(rowv[t % 3][1] + c0, r1);
       bwd_ld<EPL>(rowv[t % 3][2] + c0, r3);
       const float nkraw = cscl[t & (NCTX - 1)][sNk], daz = cscl[t & (NCTX - 1)][sDaz];
+      const float uz = cscl[t & (NCTX - 1)][sUz];
       const float ink = nkraw > eps ? 1.0f / nkraw : 1.0f / eps;
-      // z . dz = cK khz - idl (2 z.g + khz daz);  A dz = A' dz + z (z.dz) / delta
-      const float zdz = fmaf(ms.cK, ms.khz, -ms.idl * fmaf(ms.khz, daz, 2.0f * ms.zg));
+      // z . dz = cU u.z + cK khz - idl (2 z.g + khz daz);  A dz = A' dz + z (z.dz) / delta
+      const float zdz = fmaf(ms.cU, uz, fmaf(ms.cK, ms.khz, -ms.idl * fmaf(ms.khz, daz, 2.0f * ms.zg)));
       const float zs = fmaf(zdz, ms.idl, ms.ddelta);
-      float dkhx[EPL], out[EPL], wv[EPL];
+      float dkhx[EPL], out[EPL], wv[EPL], dzv[EPL], duv[EPL];
       float kd = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
-        const float dz = fmaf(ms.cK, kh[e], -ms.idl * fmaf(ms.khz, da[e], 2.0f * gv[e]));
-        wv[e] = da[e] + dz;
-        dkhx[e] = dkS[e] + r1[e] + fmaf(zt[e], zs, r3[e]);   // + ddelta z + A dz
+        const float dz = fmaf(ms.cU, uv[e], fmaf(ms.cK, kh[e], -ms.idl * fmaf(ms.khz, da[e], 2.0f * gv[e])));
+        dzv[e] = dz;
+        wv[e] = UX ? da[e] : da[e] + dz;
+        duv[e] = fmaf(zt[e], zs, r3[e]);                     // ddelta z + A dz: the gradient of u
+        dkhx[e] = dkS[e] + r1[e] + (UX ? 0.0f : duv[e]);     // u = k_hat: it lands on k_hat
         kd = fmaf(kh[e], dkhx[e], kd);
       }
       kd = warp_sum(kd);
@@ -663,7 +688,11 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
         out[e] = dkf;
       }
       bwd_st<EPL>(p.dk + ubase + size_t(t) * D + c0, out);
-      if (p.dA0) bwd_st<EPL>(p.dal + ubase + size_t(t) * D + c0, wv);
+      if constexpr (UX) bwd_st<EPL>(p.du + ubase + size_t(t) * D + c0, duv);
+      if (p.dA0) {   // for dA0: w_t (u = k_hat), or da_t and dz_t, over vectors this token no longer needs
+        bwd_st<EPL>(p.dal + ubase + size_t(t) * D + c0, wv);
+        if constexpr (UX) bwd_st<EPL>(p.dkS + ubase + size_t(t) * D + c0, dzv);
+      }
     };
     cta_sync();
     cta_sync();
@@ -714,8 +743,9 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
     for (int t = T - 1; t >= 0; --t) {
       // dz of token t at this thread's columns; r3 = A' dz (before the update)
       const MidScalars ms = mid_scalars(t);
-      float kc[RC], zc[RC], wc[RC];
+      float kc[RC], zc[RC], wc[RC], uc[RC], dzk[RC];   // UX: wc = da, dzk = dz at the columns
       bwd_ld<RC>(cvec(t, cKh) + col0, kc);
+      if constexpr (UX) bwd_ld<RC>(cvec(t, cU) + col0, uc);
       {
         float dac[RC], gc[RC], dzc[RC];
         bwd_ld<RC>(cvec(t, cDa) + col0, dac);
@@ -723,7 +753,9 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
 #pragma unroll
         for (int c = 0; c < RC; ++c) {
           dzc[c] = fmaf(ms.cK, kc[c], -ms.idl * fmaf(ms.khz, dac[c], 2.0f * gc[c]));
-          wc[c] = dac[c] + dzc[c];
+          if (UX) dzc[c] = fmaf(ms.cU, uc[c], dzc[c]);
+          wc[c] = UX ? dac[c] : dac[c] + dzc[c];
+          dzk[c] = dzc[c];
         }
         float b1[R];
 #pragma unroll
@@ -741,22 +773,33 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       constexpr int RG = R >= 4 ? 4 : R;
 #pragma unroll
       for (int rg = 0; rg < R / RG; ++rg) {
-        float kr[RG], zr[RG], dar[RG], gr[RG];
+        float kr[RG], zr[RG], dar[RG], gr[RG], ur[RG];
         bwd_ld<RG>(cvec(t, cKh) + row0 + rg * RG, kr);
         bwd_ld<RG>(cvec(t, cZt) + row0 + rg * RG, zr);
         bwd_ld<RG>(cvec(t, cDa) + row0 + rg * RG, dar);
         bwd_ld<RG>(rowv[t % 3][0] + row0 + rg * RG, gr);
+        if constexpr (UX) bwd_ld<RG>(cvec(t, cU) + row0 + rg * RG, ur);
 #pragma unroll
         for (int i = 0; i < RG; ++i) {
           const int r = rg * RG + i;
-          const float dzr = fmaf(ms.cK, kr[i], -ms.idl * fmaf(ms.khz, dar[i], 2.0f * gr[i]));
-          const float hw = 0.5f * (dar[i] + dzr), hk = 0.5f * kr[i], zs = zr[i] * ms.idl;
+          float dzr = fmaf(ms.cK, kr[i], -ms.idl * fmaf(ms.khz, dar[i], 2.0f * gr[i]));
+          if (UX) dzr = fmaf(ms.cU, ur[i], dzr);
+          const float hw = 0.5f * (UX ? dar[i] : dar[i] + dzr), hk = 0.5f * kr[i], zs = zr[i] * ms.idl;
           const float2 w2 = make_float2(hw, hw), k2 = make_float2(hk, hk), z2 = make_float2(zs, zs);
 #pragma unroll
           for (int m = 0; m < RP; ++m) {
             GA[r][m] = bwd_ffma2(w2, make_float2(kc[2 * m], kc[2 * m + 1]), GA[r][m]);
             GA[r][m] = bwd_ffma2(k2, make_float2(wc[2 * m], wc[2 * m + 1]), GA[r][m]);
             A[r][m] = bwd_ffma2(z2, make_float2(zc[2 * m], zc[2 * m + 1]), A[r][m]);
+          }
+          if constexpr (UX) {   // + sym(dz u^T)
+            const float hz = 0.5f * dzr, hu = 0.5f * ur[i];
+            const float2 dz2 = make_float2(hz, hz), u2 = make_float2(hu, hu);
+#pragma unroll
+            for (int m = 0; m < RP; ++m) {
+              GA[r][m] = bwd_ffma2(dz2, make_float2(uc[2 * m], uc[2 * m + 1]), GA[r][m]);
+              GA[r][m] = bwd_ffma2(u2, make_float2(dzk[2 * m], dzk[2 * m + 1]), GA[r][m]);
+            }
           }
         }
       }
@@ -767,15 +810,17 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
 }
 
 // dA0 = dA_T + sum_t w_t k_hat_t^T from the w_t the A side left in the workspace (only when
-// the caller asks for dA0).  One CTA of 256 threads per unit; thread (ty, tx) of a 16 x 16 grid
+// the caller asks for dA0); with explicit u: + sum_t dz_t u_t^T, w_t = da_t.  One CTA of 256 threads per unit; thread (ty, tx) of a 16 x 16 grid
 // accumulates an R x R block over tiles of 16 tokens staged in shared memory.
-template <int D, typename TIn>
+template <int D, typename TIn, bool UX>
 __global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSplitParams p) {
   constexpr int R = D / 16;
   constexpr int EPL = D / 32;
   constexpr int TT = 16;
   __shared__ float wt[TT][D];
   __shared__ float kt[TT][D];
+  __shared__ float zt2[UX ? TT : 1][D];   // dz_t and u_t (explicit u)
+  __shared__ float ut2[UX ? TT : 1][D];
   const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ty = tid >> 4, tx = tid & 15;
   const int row0 = ty * R, col0 = tx * R;
@@ -809,6 +854,11 @@ __global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSpl
       for (int e = 0; e < EPL; ++e) {
         kt[i][e * 32 + lane] = kx[e] * ink;
         wt[i][e * 32 + lane] = wv[e];
+        if constexpr (UX) {
+          const int c = e * 32 + lane;
+          zt2[i][c] = t < p.T ? p.dkS[ubase + size_t(t) * D + c] : 0.0f;
+          ut2[i][c] = t < p.T ? load1<TIn>(static_cast<const TIn*>(p.u) + ubase, size_t(t) * D + c) : 0.0f;
+        }
       }
     }
     __syncthreads();
@@ -819,6 +869,11 @@ __global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSpl
         const float w = wt[i][row0 + r];
 #pragma unroll
         for (int c = 0; c < R; ++c) acc[r][c] = fmaf(w, kt[i][col0 + c], acc[r][c]);
+        if constexpr (UX) {
+          const float z = zt2[i][row0 + r];
+#pragma unroll
+          for (int c = 0; c < R; ++c) acc[r][c] = fmaf(z, ut2[i][col0 + c], acc[r][c]);
+        }
       }
   }
 #pragma unroll

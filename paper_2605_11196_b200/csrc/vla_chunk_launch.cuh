@@ -71,10 +71,10 @@ int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
 
 // The forward of a backward pass: plain grid, u = k_hat, per-token z, e, delta left in global
 // memory (p.stash_*), readout optional.
-template <int D, typename TIn>
-int launch_chunk_stash_t(const ScanParams& p, cudaStream_t st) {
-  using Cfg = ChunkCfg<D, TIn, kUKhat>;
-  auto kern = vla_scan_chunk_kernel<D, TIn, false, kUKhat, false, true>;
+template <int D, typename TIn, int UM>
+int launch_chunk_stash_um(const ScanParams& p, cudaStream_t st) {
+  using Cfg = ChunkCfg<D, TIn, UM>;
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, false, true>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(Cfg::smem_bytes)) != cudaSuccess) {
     cudaGetLastError();
@@ -86,6 +86,12 @@ int launch_chunk_stash_t(const ScanParams& p, cudaStream_t st) {
   sp.epoch = 0;
   kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, EmptyMaps{0});
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D, typename TIn>
+int launch_chunk_stash_t(const ScanParams& p, cudaStream_t st) {
+  if (p.u) return launch_chunk_stash_um<D, TIn, kUTensor>(p, st);
+  return launch_chunk_stash_um<D, TIn, kUKhat>(p, st);
 }
 
 template <int D, typename TIn>

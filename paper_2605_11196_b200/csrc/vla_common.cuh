@@ -45,6 +45,7 @@ struct ScanParams {
   float* stash_e;
   float* stash_delta;
   float* stash_zk;           // [units, ceil(T / 16), D]: the key sum after each chunk of 16 tokens
+  float* stash_a;            // [units, T, D]: a_t = A_t k_hat_t (explicit u only; with u = k_hat it is z_t / delta_t)
   // Token-major tensors (VLA_FLAG_TOKEN_MAJOR): q, k, v, u, out are [B, T, heads, D] instead of
   // [B, heads, T, D]; unit = b * heads + h.  The states keep their [units, D, D] layout.
   int heads;

@@ -161,12 +161,12 @@ int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st) 
 
 // The two reverse scans (after the chunk kernel has left the stash), d in {32, 64, 128}.
 namespace {
-template <int D, typename TIn>
-int launch_backward_split_t(const BackwardSplitParams& p, cudaStream_t st) {
+template <int D, typename TIn, bool UX>
+int launch_backward_split_ux(const BackwardSplitParams& p, cudaStream_t st) {
   using G = BwdSplitGeom<D>;
   using M = BackwardSplitSmem<D>;
-  auto ks = vla_backward_s_kernel<D, TIn>;
-  auto ka = vla_backward_a_kernel<D, TIn>;
+  auto ks = vla_backward_s_kernel<D, TIn, UX>;
+  auto ka = vla_backward_a_kernel<D, TIn, UX>;
   if (cudaFuncSetAttribute(ks, cudaFuncAttributeMaxDynamicSharedMemorySize, int(M::s_bytes)) != cudaSuccess ||
       cudaFuncSetAttribute(ka, cudaFuncAttributeMaxDynamicSharedMemorySize, int(M::a_bytes)) != cudaSuccess) {
     cudaGetLastError();
@@ -174,8 +174,13 @@ int launch_backward_split_t(const BackwardSplitParams& p, cudaStream_t st) {
   }
   ks<<<p.units, G::NT_S, M::s_bytes, st>>>(p);   // matrix warps + closing and opening helper warps
   ka<<<p.units, G::NT_A, M::a_bytes, st>>>(p);
-  if (p.dA0) vla_backward_da0_kernel<D, TIn><<<p.units, 256, 0, st>>>(p);
+  if (p.dA0) vla_backward_da0_kernel<D, TIn, UX><<<p.units, 256, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+template <int D, typename TIn>
+int launch_backward_split_t(const BackwardSplitParams& p, cudaStream_t st) {
+  if (p.u) return launch_backward_split_ux<D, TIn, true>(p, st);
+  return launch_backward_split_ux<D, TIn, false>(p, st);
 }
 }  // namespace
 

@@ -384,7 +384,8 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
                                                           Cfg::a_floats + 3 * Cfg::C * D)) % 128 == 0,
                 "the out stage must be 128-byte aligned for a tiled TMA store");
   static_assert(!TRI || (D <= 64 && !BALANCED), "three groups: d <= 64, one CTA per unit");
-  static_assert(!STASH || (UM == kUKhat && !TRI && !BALANCED), "the stash belongs to the plain u = k_hat kernel");
+  static_assert(!STASH || ((UM == kUKhat || UM == kUTensor) && !TRI && !BALANCED),
+                "the stash belongs to the plain-grid kernels without refresh");
   constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly
   constexpr bool UT = Cfg::UT;       // u comes from the caller's tensor
   constexpr int NIN = Cfg::NIN;
@@ -855,6 +856,11 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
             Zs[t * D + g] = at;
             Z0s[t * D + g] = z[t];
             sq[t] = at * at;
+            if (STASH && p.stash_z && t < nv) {   // backward pass with explicit u: z_t and a_t = A_t k_hat_t
+              const size_t o = (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C + t) * D + g;
+              p.stash_z[o] = z[t];
+              p.stash_a[o] = at;
+            }
           }
         }
         const float tot = warp_reduce_scatter16(sq, lane);

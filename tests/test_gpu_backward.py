@@ -17,10 +17,10 @@ def _small(d, T, dtype, units=(1, 2), seed=1):
     return W.Workload("t", units[0], units[1], d, T, dtype, seed)
 
 
-def _run_both(q, k, v, lam, d_out, flags=0, S0=None, A0=None, z0=None, dS_T=None, dA_T=None, dz_T=None):
+def _run_both(q, k, v, lam, d_out, flags=0, S0=None, A0=None, z0=None, dS_T=None, dA_T=None, dz_T=None, u=None):
     dev = torch.device("cuda:0")
     mv = lambda x: None if x is None else x.to(dev).contiguous()
-    g = vla.vla_backward(mv(q), mv(k), mv(v), lam, mv(d_out), S0=mv(S0), A0=mv(A0), z0=mv(z0),
+    g = vla.vla_backward(mv(q), mv(k), mv(v), lam, mv(d_out), u=mv(u), S0=mv(S0), A0=mv(A0), z0=mv(z0),
                          dS_T=mv(dS_T), dA_T=mv(dA_T), dz_T=mv(dz_T), flags=flags)
     torch.cuda.synchronize()
     assert int(g.status.item()) == 0
@@ -28,7 +28,8 @@ def _run_both(q, k, v, lam, d_out, flags=0, S0=None, A0=None, z0=None, dS_T=None
     ka, _ = to_oracle_array(k)
     va, _ = to_oracle_array(v)
     f64 = lambda x: None if x is None else x.detach().cpu().double().numpy()
-    ref = oracle.backward(qa, ka, va, lam, f64(d_out), in_dtype=dt, S0=f64(S0), A0=f64(A0), z0=f64(z0),
+    ua = None if u is None else to_oracle_array(u)[0]
+    ref = oracle.backward(qa, ka, va, lam, f64(d_out), u=ua, in_dtype=dt, S0=f64(S0), A0=f64(A0), z0=f64(z0),
                           dS_T=f64(dS_T), dA_T=f64(dA_T), dz_T=f64(dz_T), flags=flags, n_threads=NTHREADS)
     return g, ref
 
@@ -45,6 +46,8 @@ def _err(x_gpu, x_ref):
 def _check(g, ref, tol, label):
     errs = {"dq": _err(g.dq, ref.dq), "dk": _err(g.dk, ref.dk), "dv": _err(g.dv, ref.dv),
             "dS0": _err(g.dS0, ref.dS0), "dA0": _err(g.dA0, ref.dA0), "dz0": _err(g.dz0, ref.dz0)}
+    if ref.du is not None:
+        errs["du"] = _err(g.du, ref.du)
     for name, e in errs.items():
         assert e <= tol, "%s %s: rel err %.3e > %.1e (%s)" % (label, name, e, tol, errs)
     return errs
@@ -125,3 +128,56 @@ def test_long_walk_back_keeps_the_early_tokens(d, T):
     early = slice(0, 64)
     e = np.abs(got.dq.cpu().double().numpy()[:, :, early] - ref.dq[:, :, early]).max() / np.abs(ref.dq[:, :, early]).max()
     assert e <= 1e-3, e
+
+
+# ---- explicit penalty directions (the paper's learned-u setting): gradients of q, k, v and u
+@pytest.mark.parametrize("d", [32, 64, 128])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+@pytest.mark.parametrize("T", [1, 7, 64, 200])
+def test_gradients_with_explicit_u(d, dtype, flags, T):
+    w = _small(d, T, dtype, units=(2, 3), seed=3300 + d + T)
+    q, k, v = W.make_inputs(w)
+    d_out = torch.randn((2, 3, T, d), generator=torch.Generator().manual_seed(d * 5 + T))
+    for scale, lam in ((d ** -0.5, 0.1), (1.0, 1.0)):
+        u = W.make_u(w, scale)
+        got, ref = _run_both(q, k, v, lam, d_out, flags=flags, u=u)
+        _check(got, ref, 2e-4, "backward explicit u d=%d T=%d" % (d, T))
+
+
+@pytest.mark.parametrize("d", [32, 128])
+def test_explicit_u_with_carried_states_and_state_gradients(d):
+    w = _small(d, 96, "f32", units=(1, 4), seed=3400 + d)
+    q, k, v = W.make_inputs(w)
+    u = W.make_u(w, d ** -0.5)
+    g = torch.Generator().manual_seed(d)
+    shape = (1, 4)
+    S0 = torch.randn(shape + (d, d), generator=g) * 0.2
+    h = torch.randn(shape + (d, d), generator=g) * 0.1
+    A0 = h @ h.transpose(-1, -2) + 0.5 * torch.eye(d)
+    z0 = torch.rand(shape + (d,), generator=g) + 0.1
+    d_out = torch.randn(shape + (96, d), generator=g)
+    dS_T = torch.randn(shape + (d, d), generator=g)
+    dA_T = torch.randn(shape + (d, d), generator=g)
+    dz_T = torch.randn(shape + (d,), generator=g)
+    got, ref = _run_both(q, k, v, 0.5, d_out, S0=S0, A0=A0, z0=z0, dS_T=dS_T, dA_T=dA_T, dz_T=dz_T, u=u)
+    _check(got, ref, 2e-4, "backward explicit u carried d=%d" % d)
+
+
+def test_explicit_u_equal_to_k_hat_splits_the_key_gradient():
+    """u given as the normalised keys themselves: q, v gradients as in the u = k_hat call."""
+    w = _small(64, 50, "f32", units=(1, 2), seed=3500)
+    q, k, v = W.make_inputs(w)
+    u = k / k.norm(dim=-1, keepdim=True)
+    d_out = torch.randn((1, 2, 50, 64), generator=torch.Generator().manual_seed(1))
+    dev = torch.device("cuda:0")
+    a = vla.vla_backward(q.to(dev), k.to(dev), v.to(dev), 1.0, d_out.to(dev), flags=IDENT)
+    b = vla.vla_backward(q.to(dev), k.to(dev), v.to(dev), 1.0, d_out.to(dev), flags=IDENT, u=u.to(dev))
+    torch.cuda.synchronize()
+    assert torch.allclose(a.dq, b.dq, rtol=1e-3, atol=1e-5) and torch.allclose(a.dv, b.dv, rtol=1e-3, atol=1e-5)
+    assert b.du is not None and torch.isfinite(b.du).all()
+    w16 = _small(16, 8, "f32")
+    q, k, v = [x.to(dev) for x in W.make_inputs(w16)]
+    with pytest.raises(vla.VlaError) as ei:
+        vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 8, 16), device=dev), u=k)
+    assert ei.value.code == vla.VLA_ERR_UNSUPPORTED

@@ -466,7 +466,23 @@ def main():
                                      "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
                                      "kernel": "chunk forward with stash + vla_backward_s_kernel + vla_backward_a_kernel",
                                      "gpu_launches_per_step": 3}
-        del go_h, wsb
+        # the same with explicit penalty directions (gradients of q, k, v and u)
+        uu_b = W.make_u(w, w.d ** -0.5).to(dev)
+        bucall = lambda: vla.vla_backward(qd, kd, vd, w.lam, go_h, u=uu_b, workspace=wsb, stream=stream)
+        evs = []
+        with torch.cuda.stream(stream):
+            bucall()
+            for _ in range(2):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); bucall(); b.record(stream)
+                evs.append((a, b))
+        torch.cuda.synchronize(dev)
+        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+        per[w.name + "_backward_explicit_u"] = {
+            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
+            "kernel": "chunk forward (general path) with stash + vla_backward_s_kernel + vla_backward_a_kernel + dA0",
+            "gpu_launches_per_step": 4}
+        del go_h, wsb, uu_b
         # the headline workload with an explicit penalty direction u = unit / sqrt(d_h)
         # (the paper's learned-u setting at the scan's input level)
         uu = W.make_u(w, w.d ** -0.5).to(dev)

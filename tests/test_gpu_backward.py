@@ -181,3 +181,18 @@ def test_explicit_u_equal_to_k_hat_splits_the_key_gradient():
     with pytest.raises(vla.VlaError) as ei:
         vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 8, 16), device=dev), u=k)
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("umode", ["khat", "unit_over_sqrt_d"])
+def test_long_walk_back_with_a_weak_prior(umode):
+    """lambda = 0.1 (the paper's value): A starts at 10 I and shrinks by two orders of magnitude
+    over the sequence; the reverse sweep rebuilds it by adding the downdates back."""
+    d, T = 64, 4096
+    w = W.Workload("t", 1, 2, d, T, "f32", 12)
+    q, k, v = W.make_inputs(w)
+    u = None if umode == "khat" else W.make_u(w, d ** -0.5)
+    d_out = torch.randn((1, 2, T, d), generator=torch.Generator().manual_seed(8))
+    for flags in (0, IDENT):
+        got, ref = _run_both(q, k, v, 0.1, d_out, flags=flags, u=u)
+        errs = _check(got, ref, 1e-3, "backward lambda=0.1 %s" % umode)
+        print(umode, flags, errs)

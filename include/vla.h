@@ -206,8 +206,8 @@ size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
  *
  * Covered: u = k_hat (opts->u NULL; d_k = d_v in {16, 32, 64, 128}) or explicit penalty
  * directions (opts->u given, used verbatim as in vla_forward; their gradient goes to opts->du,
- * which must then be non-NULL; d in {32, 64, 128}); no periodic refresh, head-major tensors;
- * anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a
+ * which must then be non-NULL; d in {32, 64, 128}); the periodic refresh of opts (d in
+ * {32, 64, 128}); head-major tensors; anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a
  * DEVICE buffer of at least vla_backward_workspace_bytes(B, H, T, d_k) bytes (per token: z_t,
  * e_t, delta_t of the forward and three vectors the two reverse scans exchange; the final
  * states), owned by the caller and free for reuse once the work enqueued on `stream` has completed.

@@ -256,10 +256,11 @@ class VlaGrads(NamedTuple):
 
 def vla_backward(q, k, v, lam: float, d_out, *, u=None, S0=None, A0=None, z0=None, dS_T=None, dA_T=None,
                  dz_T=None, flags: int = 0, eps: float = 1e-4, workspace=None, status=None,
-                 stream: Optional[torch.cuda.Stream] = None, want_status: bool = True) -> VlaGrads:
+                 stream: Optional[torch.cuda.Stream] = None, want_status: bool = True,
+                 refresh=None) -> VlaGrads:
     """Gradients of the forward scan for CUDA tensors (u = k_hat: d in {16, 32, 64, 128}; explicit
-    ``u``: d in {32, 64, 128}, its gradient is returned as ``du``); the forward is recomputed
-    inside.  ``d_out`` is dL/d(out); ``dS_T, dA_T, dz_T`` default to zero."""
+    ``u`` (its gradient is returned as ``du``) and / or the periodic ``refresh`` = (period, eta,
+    step_offset): d in {32, 64, 128}); the forward is recomputed inside.  ``d_out`` is dL/d(out); ``dS_T, dA_T, dz_T`` default to zero."""
     lib = load_library()
     B, H, T, dk = q.shape
     dv_ = v.shape[-1]
@@ -285,7 +286,7 @@ def vla_backward(q, k, v, lam: float, d_out, *, u=None, S0=None, A0=None, z0=Non
     if workspace is None:
         workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
     du = None if u is None else torch.empty((B, H, T, dk), dtype=f32, device=dev)
-    opts = _make_opts(dt, u, flags, eps, z0, None, status, VLA_KERNEL_AUTO, None)
+    opts = _make_opts(dt, u, flags, eps, z0, None, status, VLA_KERNEL_AUTO, refresh)
     opts.du = None if du is None else du.data_ptr()
     with torch.cuda.device(dev):
         rc = lib.vla_backward(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv_, _ptr(S0), _ptr(A0),

@@ -469,8 +469,9 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   if (rc != VLA_OK) return rc;
   rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, d_out);
   if (rc != VLA_OK) return rc;
-  if (o.refresh_period > 0 || (o.flags & VLA_FLAG_TOKEN_MAJOR)) return VLA_ERR_UNSUPPORTED;
-  if (o.u && d_k < 32) return VLA_ERR_UNSUPPORTED;   // explicit u: the two reverse scans only
+  if (o.flags & VLA_FLAG_TOKEN_MAJOR) return VLA_ERR_UNSUPPORTED;
+  const bool general = o.u || o.refresh_period > 0;   // explicit u, the refresh: the two reverse scans only
+  if (general && d_k < 32) return VLA_ERR_UNSUPPORTED;
   const int units = B * H;
   if (units > 0 && T > 0 && (!dq || !dk || !dv || (o.u && !o.du))) return VLA_ERR_INVALID_ARG;
   const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0, o.u, o.du};
@@ -514,9 +515,10 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   f.out = nullptr; f.S_T = STw; f.A_T = ATw; f.zT = zTw;
   f.status = o.status; f.lambda = lambda_; f.eps = o.eps;
   f.T = T; f.units = units; f.flags = o.flags;
-  f.refresh_period = 0; f.refresh_eta = 0.0f; f.step_offset = 0; f.u_is_khat = 0;
+  f.refresh_period = o.refresh_period; f.refresh_eta = o.refresh_eta; f.step_offset = o.step_offset;
+  f.u_is_khat = 0;
   f.n_main = 0; f.out2 = nullptr;
-  f.stash_z = zst; f.stash_e = est; f.stash_delta = dst; f.stash_zk = zkcw; f.stash_a = o.u ? astw : nullptr;
+  f.stash_z = zst; f.stash_e = est; f.stash_delta = dst; f.stash_zk = zkcw; f.stash_a = general ? astw : nullptr;
   f.heads = H;
   rc = vla::launch_chunk_stash(d_k, o.qkv_dtype, f, st);
   if (rc != VLA_OK) return rc;
@@ -527,6 +529,8 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   p.dal = dalw; p.dkS = dkSw; p.gzt = gztw;
   p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;
   p.status = o.status; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;
+  p.general = general ? 1 : 0;
+  p.refresh_period = o.refresh_period; p.refresh_eta = o.refresh_eta; p.step_offset = o.step_offset;
   return vla::launch_backward_split(d_k, o.qkv_dtype, p, st);
 }
 

@@ -67,6 +67,10 @@ struct BackwardSplitParams {
   int T;
   int units;
   uint32_t flags;
+  int general;               // the general path: explicit u and / or the periodic refresh
+  int refresh_period;        // <= 0: none
+  float refresh_eta;
+  long long step_offset;
 };
 
 }  // namespace vla

@@ -528,7 +528,12 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
   const int T = p.T;
   const size_t ubase = size_t(unit) * size_t(T) * D;
   const TIn* gk = static_cast<const TIn*>(p.k) + ubase;
-  const TIn* gu = UX ? static_cast<const TIn*>(p.u) + ubase : nullptr;
+  // general path without a u tensor (the periodic refresh alone): u = k_hat, formed here
+  const TIn* gu = (UX && p.u) ? static_cast<const TIn*>(p.u) + ubase : nullptr;
+  // Algorithm 1's refresh: A_t = (Sherman-Morrison step) + eta I at every refresh_period-th token
+  auto refreshed = [&](int t) {
+    return UX && p.refresh_period > 0 && (p.step_offset + t + 1) % p.refresh_period == 0;
+  };
   const float* zst = p.zst + ubase;
   const float* dst = p.dst + size_t(unit) * T;
 
@@ -578,7 +583,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       bwd_ld<EPL>(p.dkS + ubase + o, ps);
       bwd_ld<EPL>(p.gzt + ubase + o, pgz);
       if constexpr (UX) {
-        bwd_ld_in<EPL>(gu + o, pu);
+        if (gu) bwd_ld_in<EPL>(gu + o, pu);
         bwd_ld<EPL>(p.ast + ubase + o, pat);
       }
     };
@@ -596,11 +601,16 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
         zz = fmaf(av, av, zz);
         zpa = fmaf(av, pa[e], zpa);
         kz = fmaf(kk, pz[e], kz);
-        if (UX) uz = fmaf(pu[e], pz[e], uz);
+        if (UX && gu) uz = fmaf(pu[e], pz[e], uz);
       }
       ss = warp_sum(ss); zz = warp_sum(zz); zpa = warp_sum(zpa); kz = warp_sum(kz);
-      if (UX) uz = warp_sum(uz);
+      if (UX && gu) uz = warp_sum(uz);
       const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
+      if (UX && !gu) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) pu[e] = kx[e] * ink;
+        uz = kz * ink;
+      }
       const float idl = 1.0f / pdelta;
       const float na = UX ? sqrtf(zz) : sqrtf(zz) * idl;   // ||a||  (a = z / delta when u = k_hat)
       const float sc = (UX ? 1.0f : idl) / fmaxf(na, eps);
@@ -666,6 +676,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       // z . dz = cU u.z + cK khz - idl (2 z.g + khz daz);  A dz = A' dz + z (z.dz) / delta
       const float zdz = fmaf(ms.cU, uz, fmaf(ms.cK, ms.khz, -ms.idl * fmaf(ms.khz, daz, 2.0f * ms.zg)));
       const float zs = fmaf(zdz, ms.idl, ms.ddelta);
+      const bool rf = refreshed(t);
       float dkhx[EPL], out[EPL], wv[EPL], dzv[EPL], duv[EPL];
       float kd = 0.f;
 #pragma unroll
@@ -673,8 +684,10 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
         const float dz = fmaf(ms.cU, uv[e], fmaf(ms.cK, kh[e], -ms.idl * fmaf(ms.khz, da[e], 2.0f * gv[e])));
         dzv[e] = dz;
         wv[e] = UX ? da[e] : da[e] + dz;
-        duv[e] = fmaf(zt[e], zs, r3[e]);                     // ddelta z + A dz: the gradient of u
-        dkhx[e] = dkS[e] + r1[e] + (UX ? 0.0f : duv[e]);     // u = k_hat: it lands on k_hat
+        // ddelta z + A_{t-1} dz: the gradient of u.  r3 is A_t dz; a refreshed A_t carries eta I
+        // that A_{t-1} + (the step) does not
+        duv[e] = fmaf(zt[e], zs, r3[e] - (rf ? p.refresh_eta * dz : 0.0f));
+        dkhx[e] = dkS[e] + r1[e] + ((UX && gu) ? 0.0f : duv[e]);   // u = k_hat: it lands on k_hat
         kd = fmaf(kh[e], dkhx[e], kd);
       }
       kd = warp_sum(kd);
@@ -688,7 +701,9 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
         out[e] = dkf;
       }
       bwd_st<EPL>(p.dk + ubase + size_t(t) * D + c0, out);
-      if constexpr (UX) bwd_st<EPL>(p.du + ubase + size_t(t) * D + c0, duv);
+      if constexpr (UX) {
+        if (gu) bwd_st<EPL>(p.du + ubase + size_t(t) * D + c0, duv);
+      }
       if (p.dA0) {   // for dA0: w_t (u = k_hat), or da_t and dz_t, over vectors this token no longer needs
         bwd_st<EPL>(p.dal + ubase + size_t(t) * D + c0, wv);
         if constexpr (UX) bwd_st<EPL>(p.dkS + ubase + size_t(t) * D + c0, dzv);
@@ -800,6 +815,13 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
               GA[r][m] = bwd_ffma2(dz2, make_float2(uc[2 * m], uc[2 * m + 1]), GA[r][m]);
               GA[r][m] = bwd_ffma2(u2, make_float2(dzk[2 * m], dzk[2 * m + 1]), GA[r][m]);
             }
+            if (refreshed(t)) {   // A_t = (the step) + eta I: take the refresh off the diagonal
+#pragma unroll
+              for (int m = 0; m < RP; ++m) {
+                if (row0 + r == col0 + 2 * m) A[r][m].x -= p.refresh_eta;
+                if (row0 + r == col0 + 2 * m + 1) A[r][m].y -= p.refresh_eta;
+              }
+            }
           }
         }
       }
@@ -857,7 +879,8 @@ __global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSpl
         if constexpr (UX) {
           const int c = e * 32 + lane;
           zt2[i][c] = t < p.T ? p.dkS[ubase + size_t(t) * D + c] : 0.0f;
-          ut2[i][c] = t < p.T ? load1<TIn>(static_cast<const TIn*>(p.u) + ubase, size_t(t) * D + c) : 0.0f;
+          ut2[i][c] = !p.u ? kx[e] * ink
+                           : (t < p.T ? load1<TIn>(static_cast<const TIn*>(p.u) + ubase, size_t(t) * D + c) : 0.0f);
         }
       }
     }

@@ -91,6 +91,7 @@ int launch_chunk_stash_um(const ScanParams& p, cudaStream_t st) {
 template <int D, typename TIn>
 int launch_chunk_stash_t(const ScanParams& p, cudaStream_t st) {
   if (p.u) return launch_chunk_stash_um<D, TIn, kUTensor>(p, st);
+  if (p.refresh_period > 0) return launch_chunk_stash_um<D, TIn, kUKhatGen>(p, st);
   return launch_chunk_stash_um<D, TIn, kUKhat>(p, st);
 }
 

@@ -179,7 +179,7 @@ int launch_backward_split_ux(const BackwardSplitParams& p, cudaStream_t st) {
 }
 template <int D, typename TIn>
 int launch_backward_split_t(const BackwardSplitParams& p, cudaStream_t st) {
-  if (p.u) return launch_backward_split_ux<D, TIn, true>(p, st);
+  if (p.general) return launch_backward_split_ux<D, TIn, true>(p, st);
   return launch_backward_split_ux<D, TIn, false>(p, st);
 }
 }  // namespace

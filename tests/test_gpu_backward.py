@@ -17,11 +17,12 @@ def _small(d, T, dtype, units=(1, 2), seed=1):
     return W.Workload("t", units[0], units[1], d, T, dtype, seed)
 
 
-def _run_both(q, k, v, lam, d_out, flags=0, S0=None, A0=None, z0=None, dS_T=None, dA_T=None, dz_T=None, u=None):
+def _run_both(q, k, v, lam, d_out, flags=0, S0=None, A0=None, z0=None, dS_T=None, dA_T=None, dz_T=None, u=None,
+              refresh=None):
     dev = torch.device("cuda:0")
     mv = lambda x: None if x is None else x.to(dev).contiguous()
     g = vla.vla_backward(mv(q), mv(k), mv(v), lam, mv(d_out), u=mv(u), S0=mv(S0), A0=mv(A0), z0=mv(z0),
-                         dS_T=mv(dS_T), dA_T=mv(dA_T), dz_T=mv(dz_T), flags=flags)
+                         dS_T=mv(dS_T), dA_T=mv(dA_T), dz_T=mv(dz_T), flags=flags, refresh=refresh)
     torch.cuda.synchronize()
     assert int(g.status.item()) == 0
     qa, dt = to_oracle_array(q)
@@ -30,7 +31,8 @@ def _run_both(q, k, v, lam, d_out, flags=0, S0=None, A0=None, z0=None, dS_T=None
     f64 = lambda x: None if x is None else x.detach().cpu().double().numpy()
     ua = None if u is None else to_oracle_array(u)[0]
     ref = oracle.backward(qa, ka, va, lam, f64(d_out), u=ua, in_dtype=dt, S0=f64(S0), A0=f64(A0), z0=f64(z0),
-                          dS_T=f64(dS_T), dA_T=f64(dA_T), dz_T=f64(dz_T), flags=flags, n_threads=NTHREADS)
+                          dS_T=f64(dS_T), dA_T=f64(dA_T), dz_T=f64(dz_T), flags=flags, n_threads=NTHREADS,
+                          refresh=refresh)
     return g, ref
 
 
@@ -196,3 +198,29 @@ def test_long_walk_back_with_a_weak_prior(umode):
         got, ref = _run_both(q, k, v, 0.1, d_out, flags=flags, u=u)
         errs = _check(got, ref, 1e-3, "backward lambda=0.1 %s" % umode)
         print(umode, flags, errs)
+
+
+# ---- Algorithm 1's periodic refresh A += eta I in the backward pass
+@pytest.mark.parametrize("d", [32, 64, 128])
+@pytest.mark.parametrize("umode", ["khat", "unit_over_sqrt_d"])
+@pytest.mark.parametrize("flags", [0, IDENT])
+@pytest.mark.parametrize("refresh", [(20, 1e-3, 0), (3, 5e-2, 2), (1, 1e-2, 0), (16, 1e-2, 7)])
+def test_gradients_with_the_periodic_refresh(d, umode, flags, refresh):
+    T = 75
+    w = _small(d, T, "f32", units=(1, 3), seed=3600 + d)
+    q, k, v = W.make_inputs(w)
+    u = None if umode == "khat" else W.make_u(w, d ** -0.5)
+    g = torch.Generator().manual_seed(d + refresh[0])
+    d_out = torch.randn((1, 3, T, d), generator=g)
+    dA_T = torch.randn((1, 3, d, d), generator=g)
+    got, ref = _run_both(q, k, v, 0.1, d_out, flags=flags, u=u, refresh=refresh, dA_T=dA_T)
+    _check(got, ref, 2e-4, "backward refresh %s d=%d %s" % (refresh, d, umode))
+
+
+def test_refresh_is_refused_where_there_is_no_general_path():
+    dev = torch.device("cuda:0")
+    w16 = _small(16, 8, "f32")
+    q, k, v = [x.to(dev) for x in W.make_inputs(w16)]
+    with pytest.raises(vla.VlaError) as ei:
+        vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 8, 16), device=dev), refresh=(4, 1e-3, 0))
+    assert ei.value.code == vla.VLA_ERR_UNSUPPORTED

@@ -413,7 +413,7 @@ def main():
                 ms = float(np.median([a.elapsed_time(b) for a, b in ms]))
                 per[name + "_backward"] = {"ms": ms, "tokens_per_s": ww.tokens / (ms * 1e-3),
                                            "ns_per_scan_step": 1e6 * ms / ww.T,
-                                           "kernel": "chunk forward with stash + vla_backward_s_kernel + vla_backward_a_kernel",
+                                           "kernel": "chunk forward with stash + vla_backward_sa_kernel (both reverse scans) + vla_backward_da0_kernel",
                                            "gpu_launches_per_step": 3}
                 del qd3, kd3, vd3, go3
             # fewer units than SMs: the sequence-parallel entry point cuts each sequence into
@@ -448,8 +448,8 @@ def main():
                     "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
                     "status": int(st2.item()), "gpu_launches_per_step": 5}
                 del qd2, kd2, vd2, ws, o2
-        # backward pass of the headline workload (three launches: chunk forward leaving the per-token
-        # stash, S-side reverse scan, A-side reverse scan)
+        # backward pass of the headline workload (chunk forward leaving the per-token stash, both
+        # reverse scans as one launch, the dA0 kernel)
         go_h = torch.randn((w.B, w.H, w.T, w.d), device=dev)
         wsb = torch.empty((vla.backward_workspace_bytes(w.B, w.H, w.T, w.d),), dtype=torch.uint8, device=dev)
         bcall = lambda: vla.vla_backward(qd, kd, vd, w.lam, go_h, workspace=wsb, stream=stream)
@@ -464,7 +464,7 @@ def main():
         ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
         per[w.name + "_backward"] = {"ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3),
                                      "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
-                                     "kernel": "chunk forward with stash + vla_backward_s_kernel + vla_backward_a_kernel",
+                                     "kernel": "chunk forward with stash + vla_backward_sa_kernel (both reverse scans) + vla_backward_da0_kernel",
                                      "gpu_launches_per_step": 3}
         # the same with explicit penalty directions (gradients of q, k, v and u)
         uu_b = W.make_u(w, w.d ** -0.5).to(dev)
@@ -480,8 +480,8 @@ def main():
         ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
         per[w.name + "_backward_explicit_u"] = {
             "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
-            "kernel": "chunk forward (general path) with stash + vla_backward_s_kernel + vla_backward_a_kernel + dA0",
-            "gpu_launches_per_step": 4}
+            "kernel": "chunk forward (general path) with stash + vla_backward_sa_kernel + vla_backward_da0_kernel",
+            "gpu_launches_per_step": 3}
         del go_h, wsb, uu_b
         # the headline workload with an explicit penalty direction u = unit / sqrt(d_h)
         # (the paper's learned-u setting at the scan's input level)

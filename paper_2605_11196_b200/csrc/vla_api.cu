@@ -456,7 +456,8 @@ size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k) {
   // z, e, dalpha, dk_hat (S part), key-sum gradient per token; delta per token; S_T, A_T, key sum;
   // the key sum after every 16 tokens; a_t per token (explicit u)
   const size_t ck = round256(units * ((size_t(T) + 15) / 16) * d_k * sizeof(float));
-  return 6 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + ck + 256;
+  return 6 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + ck +
+         round256(units * sizeof(int)) + 256;
 }
 
 int vla_backward(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,
@@ -491,6 +492,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   const size_t ckb = round256(size_t(units) * ((size_t(T) + 15) / 16) * d_k * sizeof(float));
   float* zkcw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)));
   float* astw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)) + ckb);
+  int* progw = reinterpret_cast<int*>(w + 6 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)) + ckb);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (d_k == 16) {
     // d = 16 has no chunk kernel: the single kernel runs its own token-level forward sweep
@@ -530,6 +532,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;
   p.status = o.status; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;
   p.general = general ? 1 : 0;
+  p.progress = progw;
   p.refresh_period = o.refresh_period; p.refresh_eta = o.refresh_eta; p.step_offset = o.step_offset;
   return vla::launch_backward_split(d_k, o.qkv_dtype, p, st);
 }

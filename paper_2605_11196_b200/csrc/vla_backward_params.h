@@ -62,6 +62,7 @@ struct BackwardSplitParams {
   float* dS0;           // [units, D, D] or nullptr
   float* dA0;
   float* dz0;           // [units, D] or nullptr
+  int* progress;             // [units], zero on entry: tokens (from the end) whose S-side vectors are out
   int* status;
   float eps;
   int T;

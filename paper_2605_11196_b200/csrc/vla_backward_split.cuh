@@ -51,8 +51,18 @@ struct BackwardSplitSmem {
   static constexpr size_t a_bytes = sizeof(float) * (4 * 7 * D + 4 * 8 + 3 * 3 * D);
 };
 
-// All threads of the CTA, whichever loop they are in.
-__device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 0;" ::: "memory"); }
+// The n threads that take part in this CTA's role, whichever loop they are in.
+__device__ __forceinline__ void cta_sync(int n) { asm volatile("bar.sync 0, %0;" ::"r"(n) : "memory"); }
+
+// progress of a unit's S side, read by its A side (another CTA of the same launch)
+__device__ __forceinline__ void bwd_publish(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int bwd_observe(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 
 __device__ __forceinline__ float2 bwd_ffma2(float2 a, float2 b, float2 c) {
   uint64_t ra, rb, rc, rd;
@@ -128,7 +138,8 @@ __device__ __forceinline__ void rows_reduce(float* v, int lane) {
 // UX: explicit penalty directions.  The S side only sees them through alpha_t, which then comes
 // from the stashed a_t = A_t k_hat_t instead of z_t / delta_t.
 template <int D, typename TIn, bool UX>
-__global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) vla_backward_s_kernel(const BackwardSplitParams p) {
+__device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p, const int unit,
+                                                    unsigned char* smem_raw) {
   using G = BwdSplitGeom<D>;
   constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW, NT = G::NT_S, NCLOSE = G::NCLOSE;
   constexpr int RP = RC / 2;          // column pairs of a block
@@ -144,11 +155,10 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
     float gz[D];               // dL/d(key sum), carried by the closing warp
   };
   static_assert(sizeof(Smem) == BackwardSplitSmem<D>::s_bytes, "shared memory size of the S side");
-  extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   auto& ctx = sm.ctx; auto& cscl = sm.cscl; auto& rowv = sm.rowv; auto& part = sm.part; auto& gz = sm.gz;
 
-  const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int ty = tid / TX, tx = tid % TX;
   const int row0 = ty * R, col0 = tx * RC;
   const int c0 = lane * EPL;          // first vector element of this lane in a helper warp
@@ -258,14 +268,14 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
       if (T >= 2) open_token(T - 2);
       fetch_token(T - 3);
     }
-    cta_sync();
-    cta_sync();
+    cta_sync(NT);
+    cta_sync(NT);
     for (int t = T - 1; t >= 0; --t) {
       if (t - 2 >= 0) {
         open_token(t - 2);
         fetch_token(t - 3);
       }
-      cta_sync();
+      cta_sync(NT);
     }
   } else if (warp >= kCloser) {
     // The vector results of token t from its finished products.  The query part (dq, the
@@ -347,11 +357,15 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
         bwd_st<EPL>(p.dkS + tb, dko);
       }
     };
-    cta_sync();
-    cta_sync();
+    cta_sync(NT);
+    cta_sync(NT);
     for (int t = T - 1; t >= 0; --t) {
+      // tokens >= t + 2 were closed (by both closing warps) before the last barrier: tell the
+      // unit's A side every eighth token
+      const int done = T - (t + 2);
+      if (warp == kCloser && lane == 0 && done > 0 && (done & 7) == 0) bwd_publish(p.progress + unit, done);
       if (t + 1 <= T - 1) close_token(t + 1);
-      cta_sync();
+      cta_sync(NT);
     }
     if (T > 0) close_token(0);
   } else {
@@ -392,9 +406,9 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
       rows_reduce<R, TX / 2>(a1, lane);
       if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
     };
-    cta_sync();
+    cta_sync(NT);
     if (T > 0) row_dots(T - 1);
-    cta_sync();
+    cta_sync(NT);
     for (int t = T - 1; t >= 0; --t) {
       const float qal = cscl[t & (NCTX - 1)][sQal];
       constexpr int RG = R >= 4 ? 4 : R;   // rows in hand at a time: their scalars are reloaded, not kept
@@ -472,7 +486,7 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
         }
       }
       if (t >= 1) row_dots(t - 1);
-      cta_sync();
+      cta_sync(NT);
     }
     if (p.dS0) {
 #pragma unroll
@@ -484,7 +498,8 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
       }
     }
   }
-  cta_sync();
+  cta_sync(NT);
+  if (tid == 0) bwd_publish(p.progress + unit, T);   // every token's vectors are out
   if (p.dz0)
     for (int j = tid; j < D; j += NT) p.dz0[size_t(unit) * D + j] = gz[j];
 }
@@ -501,7 +516,8 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB) 
 // dk_hat = (S part) + A_t da, and the update is GAs += sym(da k_hat^T) + sym(dz u^T);
 // dA0 = dA_T + sum_t (da_t k_hat_t^T + dz_t u_t^T).
 template <int D, typename TIn, bool UX>
-__global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) vla_backward_a_kernel(const BackwardSplitParams p) {
+__device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p, const int unit,
+                                                    unsigned char* smem_raw) {
   using G = BwdSplitGeom<D>;
   constexpr int R = G::R, RC = G::RC, TX = G::TX, NW = G::NW;
   constexpr int RP = RC / 2;
@@ -515,11 +531,12 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
     float rowv[3][3][D];      // g = GAs z, r1 = A' da, r3 = A' dz, ring of three tokens
   };
   static_assert(sizeof(Smem) == BackwardSplitSmem<D>::a_bytes, "shared memory size of the A side");
-  extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   auto& ctx = sm.ctx; auto& cscl = sm.cscl; auto& rowv = sm.rowv;
 
-  const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NT = G::NT_A;
+  if (tid >= NT) return;   // the launch is sized for the S side, which has one more warp at d = 128
   const int ty = tid / TX, tx = tid % TX;
   const int row0 = ty * R, col0 = tx * RC;
   const int c0 = lane * EPL;
@@ -573,8 +590,20 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
   if (warp == kOpener) {
     float pk[EPL], pz[EPL], pa[EPL], ps[EPL], pgz[EPL], pu[EPL], pat[EPL];
     float pdelta = 1.0f;
+    // The unit's S side (another CTA of this launch, dispatched earlier) publishes how many
+    // tokens, counted from the end, have their vectors out.  Bounded wait; on a time-out the
+    // status is set and the sweep goes on with whatever is there.
+    int seen = 0;
     auto fetch_token = [&](int t) {
       if (t < 0) return;
+      if (seen < T - t) {
+        for (int it = 0; it < (1 << 22); ++it) {
+          seen = bwd_observe(p.progress + unit);
+          if (seen >= T - t) break;
+          __nanosleep(256);
+        }
+        if (seen < T - t && lane == 0 && p.status) atomicCAS(p.status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
+      }
       pdelta = dst[t];
       const size_t o = size_t(t) * D + c0;
       bwd_ld_in<EPL>(gk + o, pk);
@@ -646,14 +675,14 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       if (T >= 2) open_token(T - 2);
       fetch_token(T - 3);
     }
-    cta_sync();
-    cta_sync();
+    cta_sync(NT);
+    cta_sync(NT);
     for (int t = T - 1; t >= 0; --t) {
       if (t - 2 >= 0) {
         open_token(t - 2);
         fetch_token(t - 3);
       }
-      cta_sync();
+      cta_sync(NT);
     }
   } else if (warp == kCloser) {
     // dk of token t; w_t = da + dz goes where dalpha_t was (read two segments ago) for dA0
@@ -709,11 +738,11 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
         if constexpr (UX) bwd_st<EPL>(p.dkS + ubase + size_t(t) * D + c0, dzv);
       }
     };
-    cta_sync();
-    cta_sync();
+    cta_sync(NT);
+    cta_sync(NT);
     for (int t = T - 1; t >= 0; --t) {
       if (t + 1 <= T - 1) close_token(t + 1);
-      cta_sync();
+      cta_sync(NT);
     }
     if (T > 0) close_token(0);
   } else {
@@ -752,9 +781,9 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
       rows_reduce<R, TX / 2>(a1, lane);
       if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
     };
-    cta_sync();
+    cta_sync(NT);
     if (T > 0) products(T - 1);
-    cta_sync();
+    cta_sync(NT);
     for (int t = T - 1; t >= 0; --t) {
       // dz of token t at this thread's columns; r3 = A' dz (before the update)
       const MidScalars ms = mid_scalars(t);
@@ -826,9 +855,23 @@ __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_A, BwdSplitGeom<D>::MINB) 
         }
       }
       if (t >= 1) products(t - 1);
-      cta_sync();
+      cta_sync(NT);
     }
   }
+}
+
+// Both reverse scans as ONE launch of 2 * units CTAs: CTA x < units is the S side of unit x, CTA
+// units + x its A side.  CTAs are dispatched in index order, so a unit's S side is running or
+// finished whenever its A side starts; the A side follows it token by token through a progress
+// word in global memory (released every eighth token).  With fewer units than SMs the two sides
+// of a unit run side by side on two SMs; with many units the A-side CTAs fill the SMs the last
+// wave of S-side CTAs leaves idle.
+template <int D, typename TIn, bool UX>
+__global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB)
+vla_backward_sa_kernel(const BackwardSplitParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  if (int(blockIdx.x) < p.units) vla_backward_s_body<D, TIn, UX>(p, int(blockIdx.x), smem_raw);
+  else vla_backward_a_body<D, TIn, UX>(p, int(blockIdx.x) - p.units, smem_raw);
 }
 
 // dA0 = dA_T + sum_t w_t k_hat_t^T from the w_t the A side left in the workspace (only when

@@ -165,15 +165,16 @@ template <int D, typename TIn, bool UX>
 int launch_backward_split_ux(const BackwardSplitParams& p, cudaStream_t st) {
   using G = BwdSplitGeom<D>;
   using M = BackwardSplitSmem<D>;
-  auto ks = vla_backward_s_kernel<D, TIn, UX>;
-  auto ka = vla_backward_a_kernel<D, TIn, UX>;
-  if (cudaFuncSetAttribute(ks, cudaFuncAttributeMaxDynamicSharedMemorySize, int(M::s_bytes)) != cudaSuccess ||
-      cudaFuncSetAttribute(ka, cudaFuncAttributeMaxDynamicSharedMemorySize, int(M::a_bytes)) != cudaSuccess) {
+  auto ksa = vla_backward_sa_kernel<D, TIn, UX>;
+  constexpr size_t smem = M::s_bytes > M::a_bytes ? M::s_bytes : M::a_bytes;
+  if (cudaFuncSetAttribute(ksa, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess ||
+      cudaMemsetAsync(p.progress, 0, size_t(p.units) * sizeof(int), st) != cudaSuccess) {
     cudaGetLastError();
     return VLA_ERR_CUDA;
   }
-  ks<<<p.units, G::NT_S, M::s_bytes, st>>>(p);   // matrix warps + closing and opening helper warps
-  ka<<<p.units, G::NT_A, M::a_bytes, st>>>(p);
+  if (p.units > 0x3fffffff) return VLA_ERR_INVALID_ARG;
+  // one launch: CTAs [0, units) are the S sides, [units, 2 units) the A sides that follow them
+  ksa<<<2 * p.units, G::NT_S, smem, st>>>(p);
   if (p.dA0) vla_backward_da0_kernel<D, TIn, UX><<<p.units, 256, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }

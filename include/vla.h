@@ -49,8 +49,10 @@ enum {
   VLA_FLAG_IDENTITY_MAP = 1u << 0, /* Section 3.1: k_hat = k/||k||, o_t = S_t q_t              */
   VLA_FLAG_CHECK_FINITE = 1u << 1, /* report non-finite delta or ||A_t k_hat|| in opts->status */
   VLA_FLAG_TOKEN_MAJOR = 1u << 2   /* q, k, v, u and out are [B,T,H,d] (the layout projections write)
-                                      instead of [B,H,T,d]; the states stay [B,H,d,d].  vla_forward
-                                      and the host-buffer calls; VLA_ERR_UNSUPPORTED elsewhere */
+                                      instead of [B,H,T,d] (in vla_backward also d_out and the
+                                      gradients of q, k, v, u); the states stay [B,H,d,d].
+                                      vla_forward, the host-buffer calls, vla_backward (d >= 32);
+                                      VLA_ERR_UNSUPPORTED elsewhere */
 };
 
 /* Which scan kernel runs.  AUTO picks by shape; the others force one (tests, benchmarks). */
@@ -207,7 +209,8 @@ size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
  * Covered: u = k_hat (opts->u NULL; d_k = d_v in {16, 32, 64, 128}) or explicit penalty
  * directions (opts->u given, used verbatim as in vla_forward; their gradient goes to opts->du,
  * which must then be non-NULL; d in {32, 64, 128}); the periodic refresh of opts (d in
- * {32, 64, 128}); head-major tensors; anything else returns VLA_ERR_UNSUPPORTED.  `workspace` is a
+ * {32, 64, 128}); VLA_FLAG_TOKEN_MAJOR (d in {32, 64, 128}); anything else returns
+ * VLA_ERR_UNSUPPORTED.  `workspace` is a
  * DEVICE buffer of at least vla_backward_workspace_bytes(B, H, T, d_k) bytes (per token: z_t,
  * e_t, delta_t of the forward and three vectors the two reverse scans exchange; the final
  * states), owned by the caller and free for reuse once the work enqueued on `stream` has completed.

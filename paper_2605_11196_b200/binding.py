@@ -262,20 +262,25 @@ def vla_backward(q, k, v, lam: float, d_out, *, u=None, S0=None, A0=None, z0=Non
     ``u`` (its gradient is returned as ``du``) and / or the periodic ``refresh`` = (period, eta,
     step_offset): d in {32, 64, 128}); the forward is recomputed inside.  ``d_out`` is dL/d(out); ``dS_T, dA_T, dz_T`` default to zero."""
     lib = load_library()
-    B, H, T, dk = q.shape
+    if flags & VLA_FLAG_TOKEN_MAJOR:      # sequence tensors and their gradients as [B, T, H, d]
+        B, T, H, dk = q.shape
+        tok = lambda d_: (B, T, H, d_)
+    else:
+        B, H, T, dk = q.shape
+        tok = lambda d_: (B, H, T, d_)
     dv_ = v.shape[-1]
     dt = _dtype_code(q)
     dev = q.device
     f32 = torch.float32
-    _chk(q, (B, H, T, dk), q.dtype, "q"); _chk(k, (B, H, T, dk), q.dtype, "k")
-    _chk(v, (B, H, T, dv_), q.dtype, "v"); _chk(d_out, (B, H, T, dv_), f32, "d_out")
-    _chk(u, (B, H, T, dk), q.dtype, "u")
+    _chk(q, tok(dk), q.dtype, "q"); _chk(k, tok(dk), q.dtype, "k")
+    _chk(v, tok(dv_), q.dtype, "v"); _chk(d_out, tok(dv_), f32, "d_out")
+    _chk(u, tok(dk), q.dtype, "u")
     _chk(S0, (B, H, dv_, dk), f32, "S0"); _chk(A0, (B, H, dk, dk), f32, "A0"); _chk(z0, (B, H, dk), f32, "z0")
     _chk(dS_T, (B, H, dv_, dk), f32, "dS_T"); _chk(dA_T, (B, H, dk, dk), f32, "dA_T")
     _chk(dz_T, (B, H, dk), f32, "dz_T")
-    dq = torch.empty((B, H, T, dk), dtype=f32, device=dev)
-    dkk = torch.empty((B, H, T, dk), dtype=f32, device=dev)
-    dvv = torch.empty((B, H, T, dv_), dtype=f32, device=dev)
+    dq = torch.empty(tok(dk), dtype=f32, device=dev)
+    dkk = torch.empty(tok(dk), dtype=f32, device=dev)
+    dvv = torch.empty(tok(dv_), dtype=f32, device=dev)
     dS0 = torch.empty((B, H, dv_, dk), dtype=f32, device=dev)
     dA0 = torch.empty((B, H, dk, dk), dtype=f32, device=dev)
     dz0 = torch.empty((B, H, dk), dtype=f32, device=dev)
@@ -285,7 +290,7 @@ def vla_backward(q, k, v, lam: float, d_out, *, u=None, S0=None, A0=None, z0=Non
     need = int(lib.vla_backward_workspace_bytes(B, H, T, dk))
     if workspace is None:
         workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
-    du = None if u is None else torch.empty((B, H, T, dk), dtype=f32, device=dev)
+    du = None if u is None else torch.empty(tok(dk), dtype=f32, device=dev)
     opts = _make_opts(dt, u, flags, eps, z0, None, status, VLA_KERNEL_AUTO, refresh)
     opts.du = None if du is None else du.data_ptr()
     with torch.cuda.device(dev):

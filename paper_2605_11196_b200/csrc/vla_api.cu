@@ -470,9 +470,9 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   if (rc != VLA_OK) return rc;
   rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, d_out);
   if (rc != VLA_OK) return rc;
-  if (o.flags & VLA_FLAG_TOKEN_MAJOR) return VLA_ERR_UNSUPPORTED;
-  const bool general = o.u || o.refresh_period > 0;   // explicit u, the refresh: the two reverse scans only
-  if (general && d_k < 32) return VLA_ERR_UNSUPPORTED;
+  // explicit u, the refresh, token-major tensors: the two reverse scans only
+  const bool general = o.u || o.refresh_period > 0;
+  if ((general || (o.flags & VLA_FLAG_TOKEN_MAJOR)) && d_k < 32) return VLA_ERR_UNSUPPORTED;
   const int units = B * H;
   if (units > 0 && T > 0 && (!dq || !dk || !dv || (o.u && !o.du))) return VLA_ERR_INVALID_ARG;
   const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0, o.u, o.du};
@@ -532,6 +532,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;
   p.status = o.status; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;
   p.general = general ? 1 : 0;
+  p.heads = H;
   p.progress = progw;
   p.refresh_period = o.refresh_period; p.refresh_eta = o.refresh_eta; p.step_offset = o.step_offset;
   return vla::launch_backward_split(d_k, o.qkv_dtype, p, st);

@@ -68,6 +68,7 @@ struct BackwardSplitParams {
   int T;
   int units;
   uint32_t flags;
+  int heads;                 // H, for [B, T, H, d] tensors (VLA_FLAG_TOKEN_MAJOR): unit = b * H + h
   int general;               // the general path: explicit u and / or the periodic refresh
   int refresh_period;        // <= 0: none
   float refresh_eta;

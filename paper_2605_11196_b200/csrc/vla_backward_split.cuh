@@ -112,6 +112,17 @@ __device__ __forceinline__ void bwd_ld_in(const uint16_t* p, float (&out)[N]) {
   for (int j = 0; j < N; ++j) out[j] = __uint_as_float(uint32_t(x.v[j]) << 16);
 }
 
+// Element offset of token t of a unit in the caller's sequence tensors (q, k, u, d_out and the
+// gradients of q, k, v, u): [B, H, T, d], or [B, T, H, d] with VLA_FLAG_TOKEN_MAJOR.  The
+// workspace vectors are always [units, T, d].
+__device__ __forceinline__ size_t bwd_user_row(const BackwardSplitParams& p, int unit, int t, int D) {
+  if (p.flags & VLA_FLAG_TOKEN_MAJOR) {
+    const int b = unit / p.heads, h = unit - b * p.heads;
+    return ((size_t(b) * size_t(p.T) + size_t(t)) * size_t(p.heads) + size_t(h)) * D;
+  }
+  return (size_t(unit) * size_t(p.T) + size_t(t)) * D;
+}
+
 // Sums of N per-thread values over the 2*OFF lanes of a row group, by halving: at each step a
 // lane hands the half of its values that its partner keeps, so N values cost N - 1 shuffles
 // (plus log2(lanes / N) for the last one) instead of N log2(lanes).  Afterwards v[0] of lane l
@@ -166,9 +177,9 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
   const float eps = p.eps;
   const int T = p.T;
   const size_t ubase = size_t(unit) * size_t(T) * D;
-  const TIn* gq = static_cast<const TIn*>(p.q) + ubase;
-  const TIn* gk = static_cast<const TIn*>(p.k) + ubase;
-  const float* gdo = p.d_out + ubase;
+  const TIn* gq = static_cast<const TIn*>(p.q);      // caller's tensors: rows through bwd_user_row
+  const TIn* gk = static_cast<const TIn*>(p.k);
+  const float* gdo = p.d_out;
   const float* zst = (UX ? p.ast : p.zst) + ubase;   // the vector alpha_t is parallel to
   const float* est = p.est + ubase;
   const float* dst = p.dst + size_t(unit) * T;
@@ -193,11 +204,12 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
       if (t < 0) return;
       pdelta = dst[t];
       const size_t o = size_t(t) * D + c0;
-      bwd_ld_in<EPL>(gk + o, pk);
-      bwd_ld_in<EPL>(gq + o, pq);
+      const size_t uo = bwd_user_row(p, unit, t, D) + c0;
+      bwd_ld_in<EPL>(gk + uo, pk);
+      bwd_ld_in<EPL>(gq + uo, pq);
       bwd_ld<EPL>(zst + o, pz);
       bwd_ld<EPL>(est + o, pe);
-      bwd_ld<EPL>(gdo + o, pg);
+      bwd_ld<EPL>(gdo + uo, pg);
     };
     // the key sum seen by token t: from the forward's checkpoint at the last token of each group
     // of 16, else walked back one token from t + 1 (at most 15 subtractions from a checkpoint)
@@ -285,7 +297,8 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
     const bool do_k = NCLOSE == 1 || warp == kCloser + 1;
     auto close_token = [&](int t) {
       const int par = t & 1;
-      const size_t tb = ubase + size_t(t) * D + c0;
+      const size_t tb = ubase + size_t(t) * D + c0;          // workspace vectors
+      const size_t ub = bwd_user_row(p, unit, t, D) + c0;    // the caller's gradients
       if (do_q) {
         float go[EPL], qf[EPL], zkt[EPL], yv[EPL], c1[EPL];
         bwd_ld<EPL>(cvec(t, cGo) + c0, go);
@@ -318,7 +331,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
           gzo[e] = ident ? 0.0f : gzc[e];
         }
         if (!ident) bwd_st<EPL>(gz + c0, gzc);
-        bwd_st<EPL>(p.dq + tb, dq);
+        bwd_st<EPL>(p.dq + ub, dq);
         bwd_st<EPL>(p.gzt + tb, gzo);
       }
       if (do_k) {
@@ -352,7 +365,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
           dalo[e] = fmaf(qf[e], dye, c2[e]);          // (GS + dy qf^T)^T e
           dko[e] = -(c3[e] - al[e] * ede);            // -(S' - e alpha^T)^T de
         }
-        bwd_st<EPL>(p.dv + tb, dex);
+        bwd_st<EPL>(p.dv + ub, dex);
         bwd_st<EPL>(p.dal + tb, dalo);
         bwd_st<EPL>(p.dkS + tb, dko);
       }
@@ -544,9 +557,9 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
   const float eps = p.eps;
   const int T = p.T;
   const size_t ubase = size_t(unit) * size_t(T) * D;
-  const TIn* gk = static_cast<const TIn*>(p.k) + ubase;
+  const TIn* gk = static_cast<const TIn*>(p.k);      // caller's tensors: rows through bwd_user_row
   // general path without a u tensor (the periodic refresh alone): u = k_hat, formed here
-  const TIn* gu = (UX && p.u) ? static_cast<const TIn*>(p.u) + ubase : nullptr;
+  const TIn* gu = (UX && p.u) ? static_cast<const TIn*>(p.u) : nullptr;
   // Algorithm 1's refresh: A_t = (Sherman-Morrison step) + eta I at every refresh_period-th token
   auto refreshed = [&](int t) {
     return UX && p.refresh_period > 0 && (p.step_offset + t + 1) % p.refresh_period == 0;
@@ -606,13 +619,14 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
       }
       pdelta = dst[t];
       const size_t o = size_t(t) * D + c0;
-      bwd_ld_in<EPL>(gk + o, pk);
+      const size_t uo = bwd_user_row(p, unit, t, D) + c0;
+      bwd_ld_in<EPL>(gk + uo, pk);
       bwd_ld<EPL>(zst + o, pz);
       bwd_ld<EPL>(p.dal + ubase + o, pa);
       bwd_ld<EPL>(p.dkS + ubase + o, ps);
       bwd_ld<EPL>(p.gzt + ubase + o, pgz);
       if constexpr (UX) {
-        if (gu) bwd_ld_in<EPL>(gu + o, pu);
+        if (gu) bwd_ld_in<EPL>(gu + uo, pu);
         bwd_ld<EPL>(p.ast + ubase + o, pat);
       }
     };
@@ -729,9 +743,9 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
         }
         out[e] = dkf;
       }
-      bwd_st<EPL>(p.dk + ubase + size_t(t) * D + c0, out);
+      bwd_st<EPL>(p.dk + bwd_user_row(p, unit, t, D) + c0, out);
       if constexpr (UX) {
-        if (gu) bwd_st<EPL>(p.du + ubase + size_t(t) * D + c0, duv);
+        if (gu) bwd_st<EPL>(p.du + bwd_user_row(p, unit, t, D) + c0, duv);
       }
       if (p.dA0) {   // for dA0: w_t (u = k_hat), or da_t and dz_t, over vectors this token no longer needs
         bwd_st<EPL>(p.dal + ubase + size_t(t) * D + c0, wv);
@@ -891,7 +905,7 @@ __global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSpl
   const int row0 = ty * R, col0 = tx * R;
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
   const size_t ubase = size_t(unit) * size_t(p.T) * D;
-  const TIn* gk = static_cast<const TIn*>(p.k) + ubase;
+  const TIn* gk = static_cast<const TIn*>(p.k);
   float acc[R][R];
 #pragma unroll
   for (int r = 0; r < R; ++r)
@@ -907,7 +921,7 @@ __global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSpl
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
         const int c = e * 32 + lane;
-        float kk = t < p.T ? load1<TIn>(gk, size_t(t) * D + c) : 0.0f;
+        float kk = t < p.T ? load1<TIn>(gk, bwd_user_row(p, unit, t, D) + c) : 0.0f;
         if (!ident && t < p.T) kk = bwd_phi(kk);
         kx[e] = kk;
         wv[e] = t < p.T ? p.dal[ubase + size_t(t) * D + c] : 0.0f;
@@ -923,7 +937,7 @@ __global__ void __launch_bounds__(256) vla_backward_da0_kernel(const BackwardSpl
           const int c = e * 32 + lane;
           zt2[i][c] = t < p.T ? p.dkS[ubase + size_t(t) * D + c] : 0.0f;
           ut2[i][c] = !p.u ? kx[e] * ink
-                           : (t < p.T ? load1<TIn>(static_cast<const TIn*>(p.u) + ubase, size_t(t) * D + c) : 0.0f);
+                           : (t < p.T ? load1<TIn>(static_cast<const TIn*>(p.u), bwd_user_row(p, unit, t, D) + c) : 0.0f);
         }
       }
     }

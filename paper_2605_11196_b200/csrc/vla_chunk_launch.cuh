@@ -71,10 +71,10 @@ int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
 
 // The forward of a backward pass: plain grid, u = k_hat, per-token z, e, delta left in global
 // memory (p.stash_*), readout optional.
-template <int D, typename TIn, int UM>
-int launch_chunk_stash_um(const ScanParams& p, cudaStream_t st) {
+template <int D, typename TIn, int UM, bool TM>
+int launch_chunk_stash_um_tm(const ScanParams& p, cudaStream_t st) {
   using Cfg = ChunkCfg<D, TIn, UM>;
-  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, false, true>;
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, false, true, TM>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(Cfg::smem_bytes)) != cudaSuccess) {
     cudaGetLastError();
@@ -84,8 +84,21 @@ int launch_chunk_stash_um(const ScanParams& p, cudaStream_t st) {
   sp.balanced = 0;
   sp.grid = p.units;
   sp.epoch = 0;
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, EmptyMaps{0});
+  typename ChunkMapsArg<TM>::type maps;
+  if constexpr (TM) {
+    const int rc = encode_token_major_maps(p, D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, UM == kUTensor, &maps);
+    if (rc != VLA_OK) return rc;
+  } else {
+    maps.unused = 0;
+  }
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+template <int D, typename TIn, int UM>
+int launch_chunk_stash_um(const ScanParams& p, cudaStream_t st) {
+  if ((p.flags & VLA_FLAG_TOKEN_MAJOR) && p.T > 0) return launch_chunk_stash_um_tm<D, TIn, UM, true>(p, st);
+  return launch_chunk_stash_um_tm<D, TIn, UM, false>(p, st);
 }
 
 template <int D, typename TIn>

@@ -238,7 +238,9 @@ int encode_token_major_maps(const ScanParams& p, int d, int dtype, bool has_u, T
   if (rc == VLA_OK) rc = encode_one(&maps->k, p.k, d, p.heads, p.T, B, f32);
   if (rc == VLA_OK) rc = encode_one(&maps->v, p.v, d, p.heads, p.T, B, f32);
   if (rc == VLA_OK) rc = encode_one(&maps->u, has_u ? p.u : p.k, d, p.heads, p.T, B, f32);
-  if (rc == VLA_OK) rc = encode_one(&maps->out, p.out, d, p.heads, p.T, B, true);
+  // a forward that only leaves the backward pass's stash has no readout buffer
+  if (rc == VLA_OK && p.out) rc = encode_one(&maps->out, p.out, d, p.heads, p.T, B, true);
+  else if (rc == VLA_OK) maps->out = maps->q;
   return rc;
 }
 

@@ -379,7 +379,7 @@ __global__ void __launch_bounds__((TRI ? 3 : 2) * D, (TRI && sizeof(TIn) == 2) ?
 vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
                       const __grid_constant__ typename ChunkMapsArg<TM>::type maps) {
   using Cfg = ChunkCfg<D, TIn, UM, TRI>;
-  static_assert(!TM || (!TRI && !STASH), "token-major tensors: the plain forward kernels");
+  static_assert(!TM || !TRI, "token-major tensors: not with the three-group kernel");
   static_assert(!TM || (Cfg::raw_bytes + sizeof(float) * (Cfg::KRING * Cfg::kslot_floats + Cfg::RING * Cfg::slot_floats +
                                                           Cfg::a_floats + 3 * Cfg::C * D)) % 128 == 0,
                 "the out stage must be 128-byte aligned for a tiled TMA store");

@@ -101,7 +101,7 @@ def test_newer_entry_points_validate_on_the_host():
                                 None, None, None, vp(dq), vp(0x7000), vp(0x8000), None, None, None, opts,
                                 vp(0x10000), 1 << 30, None)
     o = VlaOpts(); o.struct_size = ctypes.sizeof(VlaOpts); o.flags = vla.VLA_FLAG_TOKEN_MAJOR
-    assert bwd(ctypes.byref(o)) == vla.VLA_ERR_UNSUPPORTED          # token-major tensors: forward only
+    assert bwd(ctypes.byref(o), d=16) == vla.VLA_ERR_UNSUPPORTED    # token-major tensors: d >= 32
     o = VlaOpts(); o.struct_size = ctypes.sizeof(VlaOpts); o.u = 0x9000
     assert bwd(ctypes.byref(o)) == vla.VLA_ERR_INVALID_ARG          # explicit u needs opts->du
     o.du = 0xa000

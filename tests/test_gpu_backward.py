@@ -224,3 +224,41 @@ def test_refresh_is_refused_where_there_is_no_general_path():
     with pytest.raises(vla.VlaError) as ei:
         vla.vla_backward(q, k, v, 1.0, torch.zeros((1, 2, 8, 16), device=dev), refresh=(4, 1e-3, 0))
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+
+
+# ---- token-major tensors ([B, T, H, d]) in the backward pass
+@pytest.mark.parametrize("d", [32, 64, 128])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("option", ["plain", "explicit_u", "refresh"])
+def test_token_major_gradients(d, dtype, option):
+    """The same backward call with the sequence tensors and their gradients transposed to
+    [B, T, H, d]: bit-identical to the head-major call, and within tolerance of the oracle."""
+    T = 83
+    w = _small(d, T, dtype, units=(2, 3), seed=3700 + d)
+    q, k, v = W.make_inputs(w)
+    u = W.make_u(w, d ** -0.5) if option == "explicit_u" else None
+    refresh = (20, 1e-3, 3) if option == "refresh" else None
+    g = torch.Generator().manual_seed(d)
+    d_out = torch.randn((2, 3, T, d), generator=g)
+    dS_T = torch.randn((2, 3, d, d), generator=g)
+    got, ref = _run_both(q, k, v, 0.5, d_out, u=u, refresh=refresh, dS_T=dS_T)
+    _check(got, ref, 2e-4, "backward head-major")
+    dev = torch.device("cuda:0")
+    tm = lambda x: None if x is None else x.permute(0, 2, 1, 3).contiguous().to(dev)
+    r = vla.vla_backward(tm(q), tm(k), tm(v), 0.5, tm(d_out), u=tm(u), dS_T=dS_T.to(dev), refresh=refresh,
+                         flags=vla.VLA_FLAG_TOKEN_MAJOR)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    back = lambda x: x.permute(0, 2, 1, 3)
+    assert torch.equal(back(r.dq), got.dq) and torch.equal(back(r.dk), got.dk) and torch.equal(back(r.dv), got.dv)
+    assert torch.equal(r.dS0, got.dS0) and torch.equal(r.dA0, got.dA0) and torch.equal(r.dz0, got.dz0)
+    if u is not None:
+        assert torch.equal(back(r.du), got.du)
+
+
+def test_token_major_is_refused_without_the_reverse_scans():
+    dev = torch.device("cuda:0")
+    x = torch.zeros((1, 8, 2, 16), device=dev)
+    with pytest.raises(vla.VlaError) as ei:
+        vla.vla_backward(x, x, x, 1.0, x, flags=vla.VLA_FLAG_TOKEN_MAJOR)
+    assert ei.value.code == vla.VLA_ERR_UNSUPPORTED

@@ -1,7 +1,9 @@
 // VLA backward pass, token kernel (first correct path): reverse-mode differentiation of the
 // forward recurrence (Algorithm 1 without projections; Eqs. "sm", "s-update", "output") for
-// u = k_hat, d in {16, 32, 64}.  The paper gives no backward algorithm; its Corollary on
-// gradient flow (Section 4) is about these gradients.
+// u = k_hat.  Written for d in {16, 32, 64}; instantiated for d = 16, which has no chunk kernel
+// to leave the stash the two reverse scans of vla_backward_split.cuh start from (they serve
+// d >= 32).  The paper gives no backward algorithm; its Corollary on gradient flow (Section 4)
+// is about these gradients.
 //
 // One CTA of 256 threads per (batch, head) unit.  Thread (ty, tx) of a 16 x 16 grid keeps the
 // R x R blocks (R = d / 16) of FOUR matrices in registers: S, A and the adjoints GS = dL/dS,

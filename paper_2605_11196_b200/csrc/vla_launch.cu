@@ -146,15 +146,7 @@ int launch_backward(int d, int dtype, const BackwardParams& p, cudaStream_t st) 
       if (f32) vla_backward_token_kernel<16, float><<<p.units, 256, 0, st>>>(p);
       else vla_backward_token_kernel<16, uint16_t><<<p.units, 256, 0, st>>>(p);
       break;
-    case 32:
-      if (f32) vla_backward_token_kernel<32, float><<<p.units, 256, 0, st>>>(p);
-      else vla_backward_token_kernel<32, uint16_t><<<p.units, 256, 0, st>>>(p);
-      break;
-    case 64:
-      if (f32) vla_backward_token_kernel<64, float><<<p.units, 256, 0, st>>>(p);
-      else vla_backward_token_kernel<64, uint16_t><<<p.units, 256, 0, st>>>(p);
-      break;
-    default: return VLA_ERR_UNSUPPORTED;
+    default: return VLA_ERR_UNSUPPORTED;   // d >= 32: the two reverse scans (launch_backward_split)
   }
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }

@@ -457,7 +457,7 @@ size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k) {
   // the key sum after every 16 tokens; a_t per token (explicit u)
   const size_t ck = round256(units * ((size_t(T) + 15) / 16) * d_k * sizeof(float));
   return 6 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + ck +
-         round256(units * sizeof(int)) + 256;
+         round256((units + 1) * sizeof(int)) + 256;
 }
 
 int vla_backward(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,

@@ -62,7 +62,8 @@ struct BackwardSplitParams {
   float* dS0;           // [units, D, D] or nullptr
   float* dA0;
   float* dz0;           // [units, D] or nullptr
-  int* progress;             // [units], zero on entry: tokens (from the end) whose S-side vectors are out
+  int* progress;             // [units + 1], zero on entry: per unit the tokens (from the end) whose S-side
+                             // vectors are out; the last word hands out the CTAs' tickets
   int* status;
   float eps;
   int T;

@@ -49,6 +49,8 @@ struct BackwardSplitSmem {
   static constexpr int NW = BwdSplitGeom<D>::NW;
   static constexpr size_t s_bytes = sizeof(float) * (4 * 8 * D + 4 * 4 + 3 * 2 * D + 2 * NW * 3 * D + D);
   static constexpr size_t a_bytes = sizeof(float) * (4 * 7 * D + 4 * 8 + 3 * 3 * D);
+  // one launch for both sides: the larger layout plus the word the CTA's ticket travels through
+  static constexpr size_t sa_bytes = (s_bytes > a_bytes ? s_bytes : a_bytes) + 16;
 };
 
 // The n threads that take part in this CTA's role, whichever loop they are in.
@@ -874,18 +876,23 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
   }
 }
 
-// Both reverse scans as ONE launch of 2 * units CTAs: CTA x < units is the S side of unit x, CTA
-// units + x its A side.  CTAs are dispatched in index order, so a unit's S side is running or
-// finished whenever its A side starts; the A side follows it token by token through a progress
-// word in global memory (released every eighth token).  With fewer units than SMs the two sides
-// of a unit run side by side on two SMs; with many units the A-side CTAs fill the SMs the last
-// wave of S-side CTAs leaves idle.
+// Both reverse scans as ONE launch of 2 * units CTAs.  Each CTA draws a ticket when it starts:
+// ticket x < units is the S side of unit x, ticket units + x its A side, so a unit's S side is
+// running or finished whenever its A side starts, whatever order the CTAs are dispatched in;
+// the A side follows it token by token through a progress word in global memory (released every
+// eighth token).  With fewer units than SMs the two sides of a unit run side by side on two SMs;
+// with many units the A-side CTAs fill the SMs the last wave of S-side CTAs leaves idle.
 template <int D, typename TIn, bool UX>
 __global__ void __launch_bounds__(BwdSplitGeom<D>::NT_S, BwdSplitGeom<D>::MINB)
 vla_backward_sa_kernel(const BackwardSplitParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  if (int(blockIdx.x) < p.units) vla_backward_s_body<D, TIn, UX>(p, int(blockIdx.x), smem_raw);
-  else vla_backward_a_body<D, TIn, UX>(p, int(blockIdx.x) - p.units, smem_raw);
+  // the ticket travels through the last word of the dynamic shared memory (behind both sides' layouts)
+  int* ticket_s = reinterpret_cast<int*>(smem_raw + BackwardSplitSmem<D>::sa_bytes - sizeof(int));
+  if (threadIdx.x == 0) *ticket_s = atomicAdd(p.progress + p.units, 1);   // the word after the units' own
+  __syncthreads();
+  const int ticket = *ticket_s;
+  if (ticket < p.units) vla_backward_s_body<D, TIn, UX>(p, ticket, smem_raw);
+  else vla_backward_a_body<D, TIn, UX>(p, ticket - p.units, smem_raw);
 }
 
 // dA0 = dA_T + sum_t w_t k_hat_t^T from the w_t the A side left in the workspace (only when

@@ -158,14 +158,14 @@ int launch_backward_split_ux(const BackwardSplitParams& p, cudaStream_t st) {
   using G = BwdSplitGeom<D>;
   using M = BackwardSplitSmem<D>;
   auto ksa = vla_backward_sa_kernel<D, TIn, UX>;
-  constexpr size_t smem = M::s_bytes > M::a_bytes ? M::s_bytes : M::a_bytes;
+  constexpr size_t smem = M::sa_bytes;
   if (cudaFuncSetAttribute(ksa, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess ||
-      cudaMemsetAsync(p.progress, 0, size_t(p.units) * sizeof(int), st) != cudaSuccess) {
+      cudaMemsetAsync(p.progress, 0, (size_t(p.units) + 1) * sizeof(int), st) != cudaSuccess) {
     cudaGetLastError();
     return VLA_ERR_CUDA;
   }
   if (p.units > 0x3fffffff) return VLA_ERR_INVALID_ARG;
-  // one launch: CTAs [0, units) are the S sides, [units, 2 units) the A sides that follow them
+  // one launch: the first `units` CTAs to start are the S sides, the others the A sides that follow them
   ksa<<<2 * p.units, G::NT_S, smem, st>>>(p);
   if (p.dA0) vla_backward_da0_kernel<D, TIn, UX><<<p.units, 256, 0, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;

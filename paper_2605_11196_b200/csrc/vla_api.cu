@@ -454,9 +454,9 @@ size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k) {
   const size_t vec = round256(units * T * d_k * sizeof(float));
   const size_t mat = round256(units * d_k * d_k * sizeof(float));
   // z, e, dalpha, dk_hat (S part), key-sum gradient per token; delta per token; S_T, A_T, key sum;
-  // the key sum after every 16 tokens; a_t per token (explicit u)
+  // the key sum after every 16 tokens; a_t per token (explicit u); the forward's readout; progress words
   const size_t ck = round256(units * ((size_t(T) + 15) / 16) * d_k * sizeof(float));
-  return 6 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + ck +
+  return 7 * vec + round256(units * T * sizeof(float)) + 2 * mat + round256(units * d_k * sizeof(float)) + ck +
          round256((units + 1) * sizeof(int)) + 256;
 }
 
@@ -493,6 +493,8 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   float* zkcw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)));
   float* astw = reinterpret_cast<float*>(w + 5 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)) + ckb);
   int* progw = reinterpret_cast<int*>(w + 6 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)) + ckb);
+  float* outw = reinterpret_cast<float*>(w + 6 * vec + sca + 2 * mat + round256(size_t(units) * d_k * sizeof(float)) + ckb +
+                                         round256((size_t(units) + 1) * sizeof(int)));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (d_k == 16) {
     // d = 16 has no chunk kernel: the single kernel runs its own token-level forward sweep
@@ -514,7 +516,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   ScanParams f;
   f.q = q; f.k = k; f.v = v; f.u = o.u;
   f.S0 = S0; f.A0 = A0; f.z0 = o.z0;
-  f.out = nullptr; f.S_T = STw; f.A_T = ATw; f.zT = zTw;
+  f.out = outw; f.S_T = STw; f.A_T = ATw; f.zT = zTw;
   f.status = o.status; f.lambda = lambda_; f.eps = o.eps;
   f.T = T; f.units = units; f.flags = o.flags;
   f.refresh_period = o.refresh_period; f.refresh_eta = o.refresh_eta; f.step_offset = o.step_offset;
@@ -527,7 +529,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   // 2. the S-side and A-side reverse scans
   vla::BackwardSplitParams p;
   p.q = q; p.k = k; p.u = o.u; p.ast = astw; p.du = o.du; p.z0 = o.z0; p.d_out = d_out; p.dS_T = dS_T; p.dA_T = dA_T; p.dz_T = dz_T;
-  p.ST = STw; p.AT = ATw; p.zT = zTw; p.zst = zst; p.est = est; p.dst = dst; p.zkc = zkcw;
+  p.ST = STw; p.AT = ATw; p.zT = zTw; p.zst = zst; p.est = est; p.dst = dst; p.zkc = zkcw; p.ost = outw;
   p.dal = dalw; p.dkS = dkSw; p.gzt = gztw;
   p.dq = dq; p.dk = dk; p.dv = dv; p.dS0 = dS0; p.dA0 = dA0; p.dz0 = dz0;
   p.status = o.status; p.eps = o.eps; p.T = T; p.units = units; p.flags = o.flags;

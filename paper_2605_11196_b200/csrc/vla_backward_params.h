@@ -53,6 +53,7 @@ struct BackwardSplitParams {
   const float* est;     // [units, T, D] e_t
   const float* dst;     // [units, T]    delta_t
   const float* zkc;     // [units, ceil(T / 16), D] key sum after each 16 tokens (paper mode)
+  const float* ost;     // the forward's readout o_t, laid out like q (so that S_t qf_t = den_t o_t needs no product)
   float* dal;           // [units, T, D] S side -> A side: dL/d alpha_t
   float* dkS;           // [units, T, D] S side -> A side: S-side part of dL/d k_hat_t
   float* gzt;           // [units, T, D] S side -> A side: dL/d(key sum) seen by token t

@@ -4,7 +4,7 @@
 // The adjoint of the memory state, GS = dL/dS, obeys a recurrence of its own that never looks at
 // the penalty side: GS_{t-1} = GS_t + dy qf^T - de k_hat^T.  So the reverse sweep splits into
 //
-//   S side (vla_backward_s_kernel): S and GS in registers.  Per token: dq, dv, and three
+//   S side (vla_backward_s_body): S and GS in registers.  Per token: dq, dv, and three
 //     vectors for the other side: dalpha_t = dL/d alpha_t, the S-side part of dL/d k_hat_t, and
 //     the running gradient of the key sum.
 //   A side (vla_backward_a_kernel): A and GA = dL/dA in registers.  Per token it turns dalpha_t
@@ -40,14 +40,14 @@ struct BwdSplitGeom {
   static constexpr int NCLOSE = D >= 128 ? 2 : 1; // warps closing tokens on the S side (the sums over NW partials)
   static constexpr int NT_S = (NW + NCLOSE + 1) * 32;   // S side: matrix warps, closers, one opener
   static constexpr int NT_A = (NW + 2) * 32;            // A side: matrix warps, one closer, one opener
-  static constexpr int MINB = D == 64 ? 3 : 1;    // CTAs per SM the register budget is held to
+  static constexpr int MINB = D == 64 ? 3 : D == 32 ? 4 : 1;   // CTAs per SM the register budget is held to
 };
 
 // Dynamic shared memory of the two reverse scans (the kernels assert these against their layouts).
 template <int D>
 struct BackwardSplitSmem {
   static constexpr int NW = BwdSplitGeom<D>::NW;
-  static constexpr size_t s_bytes = sizeof(float) * (4 * 8 * D + 4 * 4 + 3 * 2 * D + 2 * NW * 3 * D + D);
+  static constexpr size_t s_bytes = sizeof(float) * (4 * 8 * D + 4 * 4 + 3 * 1 * D + 2 * NW * 3 * D + D);
   static constexpr size_t a_bytes = sizeof(float) * (4 * 7 * D + 4 * 8 + 3 * 3 * D);
   // one launch for both sides: the larger layout plus the word the CTA's ticket travels through
   static constexpr size_t sa_bytes = (s_bytes > a_bytes ? s_bytes : a_bytes) + 16;
@@ -159,11 +159,11 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
   constexpr int EPL = D / 32;         // consecutive vector elements per lane of a helper warp
   constexpr int NCTX = 4;
   enum { cKf = 0, cKh, cQf, cGo, cDy, cEt, cAl, cZk, NV };
-  enum { sDen = 0, sDenLive, sQal };
+  enum { sDen = 0, sDenLive, sQal, sOdo };
   struct Smem {
     float ctx[NCTX][NV][D];
     float cscl[NCTX][4];
-    float rowv[3][2][D];       // y = S' qf, g1 = GS alpha, ring of three tokens
+    float rowv[3][1][D];       // g1 = GS alpha, ring of three tokens
     float part[2][NW][3][D];   // column-sum partials by token parity and warp
     float gz[D];               // dL/d(key sum), carried by the closing warp
   };
@@ -200,7 +200,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
   // the same number of barriers, so that staging registers and matrix blocks never share a thread.
   if (warp == kOpener) {
     // rows come from global memory one segment before they are opened
-    float pk[EPL], pq[EPL], pz[EPL], pe[EPL], pg[EPL];
+    float pk[EPL], pq[EPL], pz[EPL], pe[EPL], pg[EPL], po[EPL];
     float pdelta = 1.0f;
     auto fetch_token = [&](int t) {
       if (t < 0) return;
@@ -212,6 +212,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
       bwd_ld<EPL>(zst + o, pz);
       bwd_ld<EPL>(est + o, pe);
       bwd_ld<EPL>(gdo + uo, pg);
+      bwd_ld<EPL>(p.ost + uo, po);   // the forward's readout o_t (laid out like the caller's tensors)
     };
     // the key sum seen by token t: from the forward's checkpoint at the last token of each group
     // of 16, else walked back one token from t + 1 (at most 15 subtractions from a checkpoint)
@@ -219,7 +220,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
     auto open_token = [&](int t) {
       const bool last = t == T - 1 || (t & 15) == 15;
       float kx[EPL], qx[EPL], khx[EPL], alx[EPL], zkx[EPL], dyx[EPL];
-      float ss = 0.f, zz = 0.f;
+      float ss = 0.f, zz = 0.f, og = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
         float kk = pk[e], qq = pq[e];
@@ -227,6 +228,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
         kx[e] = kk; qx[e] = qq;
         ss = fmaf(kk, kk, ss);
         zz = fmaf(pz[e], pz[e], zz);
+        og = fmaf(po[e], pg[e], og);
       }
       if (ident) {
 #pragma unroll
@@ -242,6 +244,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
       }
       ss = warp_sum(ss);
       zz = warp_sum(zz);
+      og = warp_sum(og);
       const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
       const float idl = 1.0f / pdelta;
       const float sc = UX ? 1.0f / fmaxf(sqrtf(zz), eps) : idl / fmaxf(sqrtf(zz) * idl, eps);
@@ -272,6 +275,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
         os[sDen] = den;
         os[sDenLive] = (ident || dn < eps) ? 0.0f : 1.0f;
         os[sQal] = qa;
+        os[sOdo] = og;   // o_t . dO_t: with S_t qf_t = den_t o_t it gives dden without the product S_t qf_t
       }
       __syncwarp();   // the next token opened reads this one's key sum and keys
     };
@@ -302,14 +306,12 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
       const size_t tb = ubase + size_t(t) * D + c0;          // workspace vectors
       const size_t ub = bwd_user_row(p, unit, t, D) + c0;    // the caller's gradients
       if (do_q) {
-        float go[EPL], qf[EPL], zkt[EPL], yv[EPL], c1[EPL];
-        bwd_ld<EPL>(cvec(t, cGo) + c0, go);
-        bwd_ld<EPL>(rowv[t % 3][0] + c0, yv);
+        float qf[EPL], zkt[EPL], c1[EPL];
         const float den = cscl[t & (NCTX - 1)][sDen];
         const bool den_live = cscl[t & (NCTX - 1)][sDenLive] != 0.0f;
-        float odo = 0.f;
+        const float og = cscl[t & (NCTX - 1)][sOdo];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) { odo = fmaf(yv[e], go[e], odo); c1[e] = 0.f; }
+        for (int e = 0; e < EPL; ++e) c1[e] = 0.f;
 #pragma unroll
         for (int w = 0; w < NW; ++w) {
           float x1[EPL];
@@ -319,8 +321,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
         }
         bwd_ld<EPL>(cvec(t, cQf) + c0, qf);
         bwd_ld<EPL>(cvec(t, cZk) + c0, zkt);
-        odo = warp_sum(odo);
-        const float dden = den_live ? -odo / (den * den) : 0.0f;
+        const float dden = den_live ? -og / den : 0.0f;   // -(S_t qf . dO) / den^2 with S_t qf = den o_t
         float gzc[EPL], dq[EPL], gzo[EPL];
         bwd_ld<EPL>(gz + c0, gzc);
 #pragma unroll
@@ -340,7 +341,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
         float dy[EPL], et[EPL], al[EPL], qf[EPL], g1[EPL], dex[EPL], c2[EPL], c3[EPL];
         bwd_ld<EPL>(cvec(t, cDy) + c0, dy);
         bwd_ld<EPL>(cvec(t, cEt) + c0, et);
-        bwd_ld<EPL>(rowv[t % 3][1] + c0, g1);
+        bwd_ld<EPL>(rowv[t % 3][0] + c0, g1);
         const float qal = cscl[t & (NCTX - 1)][sQal];
         float ede = 0.f, dye = 0.f;
 #pragma unroll
@@ -402,24 +403,19 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
         GS[r][m] = make_float2(gv[2 * m], gv[2 * m + 1]);
       }
     }
-    auto row_dots = [&](int t) {   // y = S' qf, g1 = GS alpha of token t
-      float qv[RC], av[RC];
-      bwd_ld<RC>(cvec(t, cQf) + col0, qv);
+    auto row_dots = [&](int t) {   // g1 = GS alpha of token t
+      float av[RC];
       bwd_ld<RC>(cvec(t, cAl) + col0, av);
-      float a0[R], a1[R];
+      float a1[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        float2 x0 = make_float2(0.f, 0.f), x1 = make_float2(0.f, 0.f);
+        float2 x1 = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int m = 0; m < RP; ++m) {
-          x0 = bwd_ffma2(S[r][m], make_float2(qv[2 * m], qv[2 * m + 1]), x0);
-          x1 = bwd_ffma2(GS[r][m], make_float2(av[2 * m], av[2 * m + 1]), x1);
-        }
-        a0[r] = x0.x + x0.y; a1[r] = x1.x + x1.y;
+        for (int m = 0; m < RP; ++m) x1 = bwd_ffma2(GS[r][m], make_float2(av[2 * m], av[2 * m + 1]), x1);
+        a1[r] = x1.x + x1.y;
       }
-      rows_reduce<R, TX / 2>(a0, lane);
       rows_reduce<R, TX / 2>(a1, lane);
-      if (row_writer) { rowv[t % 3][0][row0 + myrow] = a0[0]; rowv[t % 3][1][row0 + myrow] = a1[0]; }
+      if (row_writer) rowv[t % 3][0][row0 + myrow] = a1[0];
     };
     cta_sync(NT);
     if (T > 0) row_dots(T - 1);
@@ -434,7 +430,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
       for (int rg = 0; rg < R / RG; ++rg) {
         float dyr[RG], der[RG], etr[RG];
         bwd_ld<RG>(cvec(t, cDy) + row0 + rg * RG, dyr);
-        bwd_ld<RG>(rowv[t % 3][1] + row0 + rg * RG, der);
+        bwd_ld<RG>(rowv[t % 3][0] + row0 + rg * RG, der);
         bwd_ld<RG>(cvec(t, cEt) + row0 + rg * RG, etr);
 #pragma unroll
         for (int i = 0; i < RG; ++i) {
@@ -484,7 +480,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
       for (int rg = 0; rg < R / RG; ++rg) {
         float dyr[RG], der[RG], etr[RG];
         bwd_ld<RG>(cvec(t, cDy) + row0 + rg * RG, dyr);
-        bwd_ld<RG>(rowv[t % 3][1] + row0 + rg * RG, der);
+        bwd_ld<RG>(rowv[t % 3][0] + row0 + rg * RG, der);
         bwd_ld<RG>(cvec(t, cEt) + row0 + rg * RG, etr);
 #pragma unroll
         for (int i = 0; i < RG; ++i) {

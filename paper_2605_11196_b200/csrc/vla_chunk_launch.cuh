@@ -13,12 +13,15 @@ namespace vla {
 int encode_token_major_maps(const ScanParams& p, int d, int dtype, bool has_u, TokenMajorMaps* maps);
 
 // TM: q, k, v, u, out are [B, T, H, d] (an instantiation of its own: one bulk copy per token row).
-template <int D, typename TIn, int UM, bool TM>
+// STASH: the forward of a backward pass (per-token z, e, delta, ... left in p.stash_*); its
+// token-major instantiation exists on the plain grid only.
+template <int D, typename TIn, int UM, bool TM, bool STASH = false>
 int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
   using Cfg = ChunkCfg<D, TIn, UM>;
   static_assert(Cfg::smem_bytes <= 227 * 1024, "chunk kernel exceeds the shared memory of one CTA");
-  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, false, false, TM>;     // one CTA per unit
-  auto kern_bal = vla_scan_chunk_kernel<D, TIn, true, UM, false, false, TM>;  // persistent grid, units cut at chunks
+  constexpr bool BAL = !(STASH && TM);
+  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, false, STASH, TM>;     // one CTA per unit
+  auto kern_bal = vla_scan_chunk_kernel<D, TIn, BAL, UM, false, STASH, TM>;   // persistent grid, units cut at chunks
   if (TM && p.n_main > 0) return VLA_ERR_UNSUPPORTED;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            int(Cfg::smem_bytes)) != cudaSuccess ||
@@ -41,7 +44,7 @@ int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
           cudaSuccess) {
     const int resident = sms * per_sm;
     const bool state_out = p.S_T && p.A_T && (p.zT || (p.flags & VLA_FLAG_IDENTITY_MAP));
-    if (resident > 0 && p.units > resident && p.units % resident != 0 && p.T > 0 && state_out &&
+    if (BAL && resident > 0 && p.units > resident && p.units % resident != 0 && p.T > 0 && state_out &&
         p.units <= kSchedMaxUnits && p.n_main <= 0) {
       sp.balanced = 1;
       sp.grid = resident;
@@ -69,36 +72,10 @@ int launch_chunk_um(const ScanParams& p, cudaStream_t st) {
   return launch_chunk_um_tm<D, TIn, UM, false>(p, st);
 }
 
-// The forward of a backward pass: plain grid, u = k_hat, per-token z, e, delta left in global
-// memory (p.stash_*), readout optional.
-template <int D, typename TIn, int UM, bool TM>
-int launch_chunk_stash_um_tm(const ScanParams& p, cudaStream_t st) {
-  using Cfg = ChunkCfg<D, TIn, UM>;
-  auto kern = vla_scan_chunk_kernel<D, TIn, false, UM, false, true, TM>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           int(Cfg::smem_bytes)) != cudaSuccess) {
-    cudaGetLastError();
-    return VLA_ERR_CUDA;
-  }
-  SchedParams sp;
-  sp.balanced = 0;
-  sp.grid = p.units;
-  sp.epoch = 0;
-  typename ChunkMapsArg<TM>::type maps;
-  if constexpr (TM) {
-    const int rc = encode_token_major_maps(p, D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, UM == kUTensor, &maps);
-    if (rc != VLA_OK) return rc;
-  } else {
-    maps.unused = 0;
-  }
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
-  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
-}
-
 template <int D, typename TIn, int UM>
 int launch_chunk_stash_um(const ScanParams& p, cudaStream_t st) {
-  if ((p.flags & VLA_FLAG_TOKEN_MAJOR) && p.T > 0) return launch_chunk_stash_um_tm<D, TIn, UM, true>(p, st);
-  return launch_chunk_stash_um_tm<D, TIn, UM, false>(p, st);
+  if ((p.flags & VLA_FLAG_TOKEN_MAJOR) && p.T > 0) return launch_chunk_um_tm<D, TIn, UM, true, true>(p, st);
+  return launch_chunk_um_tm<D, TIn, UM, false, true>(p, st);
 }
 
 template <int D, typename TIn>
@@ -175,7 +152,8 @@ int chunk_resident_t(bool tri) {
 
 }  // namespace vla
 
-// The three entry points of one (d, input type) translation unit.
+// The entry points of one (d, input type): the forward kernels in one translation unit, the
+// forward-with-stash kernels of the backward pass in another (they compile in parallel).
 #define VLA_DEFINE_CHUNK_TU(D, TIN, TAG)                                                        \
   namespace vla {                                                                               \
   int launch_chunk_##TAG(const ScanParams& p, cudaStream_t st) { return launch_chunk_t<D, TIN>(p, st); } \
@@ -183,6 +161,9 @@ int chunk_resident_t(bool tri) {
     return launch_chunk_tri_t<D, TIN>(p, st);                                                   \
   }                                                                                             \
   int chunk_resident_##TAG(bool tri) { return chunk_resident_t<D, TIN>(tri); }                  \
+  }
+#define VLA_DEFINE_CHUNK_STASH_TU(D, TIN, TAG)                                                  \
+  namespace vla {                                                                               \
   int launch_chunk_stash_##TAG(const ScanParams& p, cudaStream_t st) {                          \
     return launch_chunk_stash_t<D, TIN>(p, st);                                                 \
   }                                                                                             \

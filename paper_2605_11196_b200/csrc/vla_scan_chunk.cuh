@@ -384,7 +384,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
                                                           Cfg::a_floats + 3 * Cfg::C * D)) % 128 == 0,
                 "the out stage must be 128-byte aligned for a tiled TMA store");
   static_assert(!TRI || (D <= 64 && !BALANCED), "three groups: d <= 64, one CTA per unit");
-  static_assert(!STASH || (!TRI && !BALANCED), "the stash belongs to the plain-grid kernels");
+  static_assert(!STASH || !TRI, "the stash: not with the three-group kernel");
   constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly
   constexpr bool UT = Cfg::UT;       // u comes from the caller's tensor
   constexpr int NIN = Cfg::NIN;

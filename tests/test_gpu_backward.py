@@ -262,3 +262,17 @@ def test_token_major_is_refused_without_the_reverse_scans():
     with pytest.raises(vla.VlaError) as ei:
         vla.vla_backward(x, x, x, 1.0, x, flags=vla.VLA_FLAG_TOKEN_MAJOR)
     assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("umode", ["khat", "unit_over_sqrt_d"])
+def test_more_units_than_resident_ctas(umode):
+    """More units than the SMs hold at once, not a multiple of them: the forward that leaves the
+    stash runs on the schedule that cuts units at chunk boundaries, and the reverse scans' second
+    halves (the A sides) start as CTAs of the first wave retire."""
+    d, T = 128, 80
+    w = W.Workload("t", 1, 151, d, T, "bf16", 21)
+    q, k, v = W.make_inputs(w)
+    u = None if umode == "khat" else W.make_u(w, d ** -0.5)
+    d_out = torch.randn((1, 151, T, d), generator=torch.Generator().manual_seed(3))
+    got, ref = _run_both(q, k, v, w.lam, d_out, u=u)
+    _check(got, ref, 2e-4, "backward 151 units")

@@ -13,3 +13,4 @@ from .binding import (VLA_BF16, VLA_ERR_ALIGNMENT, VLA_ERR_CUDA, VLA_ERR_DEVICE_
                       vla_forward_seqpar, seqpar_segments, seqpar_workspace_bytes,
                       measure_fp32_fma_tflops, vla_backward, VlaGrads,
                       backward_workspace_bytes, vla_make_u)
+from .autograd import vla_scan  # noqa: F401,E402

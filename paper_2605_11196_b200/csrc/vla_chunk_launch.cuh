@@ -37,8 +37,15 @@ int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
   // Balanced schedule: only when a plain launch would leave SMs idle in its last wave, every
   // CTA of the persistent grid is resident at once, and the caller's S_T / A_T / zT can carry
   // a unit's state from the CTA that starts it to the CTA that finishes it.
+  // Not while the stream is being captured into a CUDA graph: the hand-over flags are keyed by a
+  // launch number drawn here, on the host, and every replay of the graph would carry the same one.
+  cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &capture) != cudaSuccess) {
+    cudaGetLastError();
+    capture = cudaStreamCaptureStatusActive;
+  }
   int dev = 0, sms = 0, per_sm = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess &&
+  if (capture == cudaStreamCaptureStatusNone && cudaGetDevice(&dev) == cudaSuccess &&
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern_bal, Cfg::NT, Cfg::smem_bytes) ==
           cudaSuccess) {

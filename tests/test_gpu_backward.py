@@ -276,3 +276,34 @@ def test_more_units_than_resident_ctas(umode):
     d_out = torch.randn((1, 151, T, d), generator=torch.Generator().manual_seed(3))
     got, ref = _run_both(q, k, v, w.lam, d_out, u=u)
     _check(got, ref, 2e-4, "backward 151 units")
+
+
+def test_backward_replays_from_a_cuda_graph():
+    """Captured once, replayed on new inputs: the launch that runs both reverse scans zeroes its
+    progress words and ticket counter with a memset node of the same graph."""
+    dev = torch.device("cuda:0")
+    w = W.Workload("t", 1, 151, 64, 48, "f32", 41)
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    d_out = torch.randn((1, 151, 48, 64), generator=torch.Generator().manual_seed(1)).to(dev)
+    ws = torch.empty((vla.backward_workspace_bytes(1, 151, 48, 64),), dtype=torch.uint8, device=dev)
+    status = torch.zeros((), dtype=torch.int32, device=dev)
+    call = lambda: vla.vla_backward(q, k, v, w.lam, d_out, workspace=ws, status=status)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        call()
+    torch.cuda.current_stream().wait_stream(s)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        g = call()
+    for seed in (42, 43):
+        q2, k2, v2 = W.make_inputs(W.Workload("t", 1, 151, 64, 48, "f32", seed))
+        q.copy_(q2); k.copy_(k2); v.copy_(v2)
+        graph.replay()
+        torch.cuda.synchronize()
+        got = [x.clone() for x in (g.dq, g.dk, g.dv, g.dA0)]
+        fresh = vla.vla_backward(q, k, v, w.lam, d_out)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for a, b in zip(got, (fresh.dq, fresh.dk, fresh.dv, fresh.dA0)):
+            assert torch.equal(a, b)

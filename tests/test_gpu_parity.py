@@ -443,3 +443,36 @@ def test_throughput_shape_with_algorithm_1_options(option, flags):
     errs, _, _ = check_parity(q, k, v, w.lam, 1e-3, u=u, flags=flags, refresh=refresh,
                               kernel=vla.VLA_KERNEL_CHUNK, label=option)
     print(option, flags, errs)
+
+
+def test_forward_and_backward_replay_from_a_cuda_graph():
+    """The calls allocate nothing and never synchronise, so they can be captured; a replayed
+    graph must give what a fresh call gives on the buffers' current contents (more units than
+    resident CTAs: the shape on which a plain call would cut units across CTAs)."""
+    dev = torch.device("cuda:0")
+    w = W.Workload("t", 1, 151, 128, 64, "bf16", 31)
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    out = torch.empty((1, 151, 64, 128), device=dev)
+    S_T = torch.empty((1, 151, 128, 128), device=dev)
+    A_T = torch.empty_like(S_T)
+    z_T = torch.empty((1, 151, 128), device=dev)
+    status = torch.zeros((), dtype=torch.int32, device=dev)
+    call = lambda: vla.vla_forward(q, k, v, w.lam, out=out, S_T=S_T, A_T=A_T, z_T=z_T, status=status)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        call()                                  # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(s)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call()
+    for seed in (32, 33, 34):
+        q2, k2, v2 = W.make_inputs(W.Workload("t", 1, 151, 128, 64, "bf16", seed))
+        q.copy_(q2); k.copy_(k2); v.copy_(v2)
+        graph.replay()
+        torch.cuda.synchronize()
+        got = (out.clone(), S_T.clone(), A_T.clone())
+        fresh = vla.vla_forward(q, k, v, w.lam)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(got[0], fresh.out) and torch.equal(got[1], fresh.S_T) and torch.equal(got[2], fresh.A_T)

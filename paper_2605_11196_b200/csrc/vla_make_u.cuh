@@ -24,6 +24,17 @@ struct MakeUCfg {
   static constexpr size_t smem_bytes = sizeof(float) * (size_t(D) * WS + size_t(kMakeUTile) * WS);
 };
 
+__device__ __forceinline__ float2 make_u_ffma2(float2 a, float2 b, float2 c) {
+  uint64_t ra, rb, rc, rd;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(rc) : "f"(c.x), "f"(c.y));
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+  float2 d;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+  return d;
+}
+
 __device__ __forceinline__ void store_u(float* p, float x) { *p = x; }
 __device__ __forceinline__ void store_u(uint16_t* p, float x) {   // bf16, round to nearest even
   uint32_t b = __float_as_uint(x);
@@ -61,27 +72,73 @@ __global__ void __launch_bounds__(256) vla_make_u_kernel(const MakeUParams p) {
     }
     __syncthreads();
     float acc[4][CPT];
+    if constexpr (CPT % 2 == 0) {
+      // column pairs: packed fp32 FMAs (half the issue slots of the scalar form)
+      float2 acc2[4][CPT / 2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
-      for (int c = 0; c < CPT; ++c) acc[i][c] = 0.0f;
+        for (int c = 0; c < CPT / 2; ++c) acc2[i][c] = make_float2(0.0f, 0.0f);
 #pragma unroll 2
-    for (int j = 0; j < D; j += 4) {
-      float a[4][4];
+      for (int j = 0; j < D; j += 4) {
+        float a[4][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float4 x = *reinterpret_cast<const float4*>(Ks + (ty * 4 + i) * WS + j);
-        a[i][0] = x.x; a[i][1] = x.y; a[i][2] = x.z; a[i][3] = x.w;
+        for (int i = 0; i < 4; ++i) {
+          const float4 x = *reinterpret_cast<const float4*>(Ks + (ty * 4 + i) * WS + j);
+          a[i][0] = x.x; a[i][1] = x.y; a[i][2] = x.z; a[i][3] = x.w;
+        }
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          float2 b[CPT / 2];
+          if constexpr (CPT >= 4) {
+            // this thread's columns come in groups of four, 64 apart: a warp's 16-byte reads of
+            // one group are adjacent (no bank conflicts)
+#pragma unroll
+            for (int g4 = 0; g4 < CPT / 4; ++g4) {
+              const float4 x = *reinterpret_cast<const float4*>(Wt + (j + jj) * WS + g4 * 64 + tx * 4);
+              b[2 * g4] = make_float2(x.x, x.y);
+              b[2 * g4 + 1] = make_float2(x.z, x.w);
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < CPT / 2; ++c)
+              b[c] = *reinterpret_cast<const float2*>(Wt + (j + jj) * WS + tx * CPT + 2 * c);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float2 aa = make_float2(a[i][jj], a[i][jj]);
+#pragma unroll
+            for (int c = 0; c < CPT / 2; ++c) acc2[i][c] = make_u_ffma2(aa, b[c], acc2[i][c]);
+          }
+        }
       }
 #pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        float b[CPT];
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int c = 0; c < CPT; ++c) b[c] = Wt[(j + jj) * WS + tx * CPT + c];
+        for (int c = 0; c < CPT / 2; ++c) { acc[i][2 * c] = acc2[i][c].x; acc[i][2 * c + 1] = acc2[i][c].y; }
+    } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int c = 0; c < CPT; ++c) acc[i][c] = fmaf(a[i][jj], b[c], acc[i][c]);
+        for (int c = 0; c < CPT; ++c) acc[i][c] = 0.0f;
+#pragma unroll 2
+      for (int j = 0; j < D; j += 4) {
+        float a[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 x = *reinterpret_cast<const float4*>(Ks + (ty * 4 + i) * WS + j);
+          a[i][0] = x.x; a[i][1] = x.y; a[i][2] = x.z; a[i][3] = x.w;
+        }
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          float b[CPT];
+#pragma unroll
+          for (int c = 0; c < CPT; ++c) b[c] = Wt[(j + jj) * WS + tx * CPT + c];
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int c = 0; c < CPT; ++c) acc[i][c] = fmaf(a[i][jj], b[c], acc[i][c]);
+        }
       }
     }
 #pragma unroll
@@ -95,7 +152,10 @@ __global__ void __launch_bounds__(256) vla_make_u_kernel(const MakeUParams p) {
       const int tk = ty * 4 + i;
       if (tk < n) {
 #pragma unroll
-        for (int c = 0; c < CPT; ++c) store_u(gu + size_t(t0 + tk) * D + tx * CPT + c, acc[i][c] * f);
+        for (int c = 0; c < CPT; ++c) {
+          const int col = CPT >= 4 ? (c / 4) * 64 + tx * 4 + (c % 4) : tx * CPT + c;
+          store_u(gu + size_t(t0 + tk) * D + col, acc[i][c] * f);
+        }
       }
     }
   }

@@ -1,5 +1,5 @@
-// VLA backward pass as two reverse scans (u = k_hat, or explicit penalty directions u with the
-// template flag UX; d in {32, 64, 128}).
+// VLA backward pass as two reverse scans, run as one launch (u = k_hat; with the template flag UX
+// the general path: explicit penalty directions u and / or the periodic refresh; d in {32, 64, 128}).
 //
 // The adjoint of the memory state, GS = dL/dS, obeys a recurrence of its own that never looks at
 // the penalty side: GS_{t-1} = GS_t + dy qf^T - de k_hat^T.  So the reverse sweep splits into
@@ -7,7 +7,7 @@
 //   S side (vla_backward_s_body): S and GS in registers.  Per token: dq, dv, and three
 //     vectors for the other side: dalpha_t = dL/d alpha_t, the S-side part of dL/d k_hat_t, and
 //     the running gradient of the key sum.
-//   A side (vla_backward_a_kernel): A and GA = dL/dA in registers.  Per token it turns dalpha_t
+//   A side (vla_backward_a_body): A and GA = dL/dA in registers.  Per token it turns dalpha_t
 //     into da, forms dz, ddelta and the remaining parts of dL/d k_hat_t, and writes dk.  It
 //     carries the symmetric part of GA only; dA0 is formed afterwards (vla_backward_da0_kernel).
 //
@@ -15,12 +15,14 @@
 // 16 x TX threads (R = d / 16 rows, RC = d / TX columns; TX = 16, or 32 at d = 128, where the
 // blocks of a 16-wide grid would leave no registers for the helper warps).  The blocks are kept
 // as column pairs and every product with them is a packed fma.rn.f32x2.  The forward
-// recurrence is not re-run here: the chunk kernel leaves z_t, e_t, delta_t per token and the
-// final S, A, key sum in the workspace, and both sweeps walk the states back by undoing the
-// rank-1 updates (S_{t-1} = S_t - e alpha^T, A_{t-1} = A_t + z z^T / delta).  Formulas per
-// token: see vla_backward.cuh.
+// recurrence is not re-run here: the chunk kernel leaves z_t, e_t, delta_t (a_t on the general
+// path), its readout o_t, the key sum after every 16 tokens and the final S, A, key sum in the
+// workspace, and both sweeps walk the states back by undoing the rank-1 updates
+// (S_{t-1} = S_t - e alpha^T, A_{t-1} = A_t + z z^T / delta).  Formulas per token: see
+// vla_backward.cuh.  vla_backward_sa_kernel (end of this file) runs the S side and the A side
+// of every unit as CTAs of one launch, the A side following the S side through a progress word.
 //
-// Both kernels keep a ring of four per-token contexts in shared memory.  Opening a token
+// Both sides keep a ring of four per-token contexts in shared memory.  Opening a token
 // (loading its rows, alpha, denominators: nothing that depends on the adjoints) and closing one
 // (vector arithmetic on finished products, the stores) are done by helper warps off the path
 // of the TX / 2 matrix warps; one CTA barrier per token.

@@ -87,6 +87,12 @@ typedef struct {
   int64_t step_offset;   /* tokens of this sequence processed by earlier calls (state carry)     */
   float* du;             /* vla_backward with explicit u: [B,H,T,d_k] fp32 gradient of u (required
                             when u is given there; ignored by the forward calls)                 */
+  void* workspace;       /* vla_forward, kernel AUTO: optional DEVICE scratch.  When the problem has
+                            too few units to fill the device and the library would cut its sequences
+                            (vla_seqpar_segments(...) > 1) and this holds at least
+                            vla_seqpar_workspace_bytes(B, H, T, d_k, that many) bytes, the call runs as
+                            vla_forward_seqpar; otherwise it is not touched.  NULL: never            */
+  size_t workspace_bytes;
 } vla_opts_t;
 
 /*

@@ -36,7 +36,8 @@ class VlaOpts(ctypes.Structure):
                 ("u", ctypes.c_void_p), ("flags", ctypes.c_uint32), ("eps", ctypes.c_float),
                 ("z0", ctypes.c_void_p), ("zT", ctypes.c_void_p), ("status", ctypes.c_void_p),
                 ("kernel", ctypes.c_int32), ("refresh_period", ctypes.c_int32),
-                ("refresh_eta", ctypes.c_float), ("step_offset", ctypes.c_int64), ("du", ctypes.c_void_p)]
+                ("refresh_eta", ctypes.c_float), ("step_offset", ctypes.c_int64), ("du", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
 
 class VlaError(RuntimeError):
@@ -193,11 +194,14 @@ def _make_opts(dt, u, flags, eps, z0, zT, status, kernel, refresh=None):
 def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags: int = 0,
                 eps: float = 1e-4, out=None, S_T=None, A_T=None, z_T=None, status=None,
                 kernel: int = VLA_KERNEL_AUTO, stream: Optional[torch.cuda.Stream] = None,
-                want_status: bool = True, refresh=None) -> VlaResult:
+                want_status: bool = True, refresh=None, workspace=None) -> VlaResult:
     """Enqueue the scan for CUDA tensors ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``
     (``[B,T,H,d]`` for all of them and ``out`` with ``VLA_FLAG_TOKEN_MAJOR``).
 
     Output tensors are allocated with torch unless passed in.  Nothing is synchronised.
+    ``workspace``: device scratch the library may use to cut the sequences of a problem with few
+    units into concurrently scanned segments (``opts->workspace``); ``True`` allocates what the
+    library asks for with torch, ``None`` / ``False`` passes none.
     """
     lib = load_library()
     if q.dim() != 4:
@@ -230,6 +234,12 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
         status = torch.zeros((), dtype=torch.int32, device=dev)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
     opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel, refresh)
+    if workspace is True:
+        P = int(lib.vla_seqpar_segments(B, H, T, dk, dt)) if kernel == VLA_KERNEL_AUTO else 1
+        workspace = None if P <= 1 else torch.empty((int(lib.vla_seqpar_workspace_bytes(B, H, T, dk, P)),),
+                                                    dtype=torch.uint8, device=dev)
+    if workspace is not None and workspace is not False:
+        opts.workspace, opts.workspace_bytes = workspace.data_ptr(), workspace.numel()
     with torch.cuda.device(dev):
         rc = lib.vla_forward(_ptr(q), _ptr(k), _ptr(v), float(lam), B, H, T, dk, dv,
                              _ptr(S0), _ptr(A0), _ptr(out), _ptr(S_T), _ptr(A_T),

@@ -186,6 +186,15 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
   const int units = B * H;
   if (units == 0) return VLA_OK;
 
+  // Few units and scratch memory at hand: cut the sequences into concurrently scanned segments
+  if (o.kernel == VLA_KERNEL_AUTO && o.workspace && d_k >= 32 && o.refresh_period <= 0 &&
+      !(o.flags & VLA_FLAG_TOKEN_MAJOR) && T > 0 && T % 16 == 0) {
+    const int P = seqpar_choose_segments(units, T, d_k, o.qkv_dtype);
+    if (P > 1 && o.workspace_bytes >= seqpar_layout(size_t(units), size_t(T), size_t(d_k), size_t(P)).total)
+      return vla_forward_seqpar(q, k, v, lambda_, B, H, T, d_k, d_v, S0, A0, out, S_T, A_T, &o, P, o.workspace,
+                                o.workspace_bytes, stream);
+  }
+
   ScanParams p;
   p.q = q; p.k = k; p.v = v; p.u = o.u;
   p.S0 = S0; p.A0 = A0; p.z0 = o.z0;

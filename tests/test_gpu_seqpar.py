@@ -113,3 +113,36 @@ def test_few_unit_workloads_full_size(name, flags):
     plain = run_gpu(q, k, v, w.lam, flags=flags)
     print(name, flags, errs, "plain o err", rel_err(plain.out, ref.out))
     assert np.isfinite(r.out.cpu().numpy()).all()
+
+
+def test_vla_forward_takes_the_segmented_route_when_given_scratch():
+    """kernel AUTO + opts->workspace: a problem with few long units runs as vla_forward_seqpar
+    (the scratch is used, the result is that call's up to the order of its atomic sums), one
+    that fills the device, or too little scratch, leaves it to the plain scan."""
+    dev = torch.device("cuda:0")
+    w = W.Workload("t", 1, 6, 64, 2048, "bf16", 91)
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    P = vla.seqpar_segments(1, 6, 2048, 64, torch.bfloat16)
+    assert P > 1
+    ws = torch.full((vla.seqpar_workspace_bytes(1, 6, 2048, 64, P),), 0x5A, dtype=torch.uint8, device=dev)
+    a = vla.vla_forward(q, k, v, w.lam, workspace=ws)
+    b = vla.vla_forward_seqpar(q, k, v, w.lam, segments=P)
+    c = vla.vla_forward(q, k, v, w.lam)
+    a2 = vla.vla_forward(q, k, v, w.lam, workspace=True)        # scratch allocated by the binding
+    torch.cuda.synchronize()
+    assert bool((ws != 0x5A).any())                              # the segmented route ran
+    f64 = lambda x: x.cpu().double().numpy()
+    assert rel_err(a.out, f64(b.out)) <= 1e-6 and rel_err(a.S_T, f64(b.S_T)) <= 1e-6
+    assert rel_err(a2.out, f64(b.out)) <= 1e-6
+    assert rel_err(a.out, f64(c.out)) <= 1e-4                    # the same scan in another order
+    small = torch.full((1024,), 0x5A, dtype=torch.uint8, device=dev)   # too little scratch: the plain scan
+    d2 = vla.vla_forward(q, k, v, w.lam, workspace=small)
+    torch.cuda.synchronize()
+    assert torch.equal(d2.out, c.out) and bool((small == 0x5A).all())
+    wf = W.Workload("t", 4, 80, 32, 64, "f32", 92)               # the device is full: nothing to cut
+    q, k, v = [x.to(dev) for x in W.make_inputs(wf)]
+    big = torch.full((1 << 20,), 0x5A, dtype=torch.uint8, device=dev)
+    e = vla.vla_forward(q, k, v, wf.lam, workspace=big)
+    f = vla.vla_forward(q, k, v, wf.lam)
+    torch.cuda.synchronize()
+    assert torch.equal(e.out, f.out) and bool((big == 0x5A).all())

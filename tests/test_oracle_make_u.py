@@ -6,14 +6,18 @@ import math
 import numpy as np
 import pytest
 
-from oracle import make_u as O
+import importlib.util
+import os
+import types
+
+from oracle import make_u as ORACLE
 
 
 def _rand(shape, seed):
     return np.random.default_rng(seed).standard_normal(shape)
 
 
-def test_identity_projection_is_the_normalised_key():
+def pin_identity_projection_is_the_normalised_key(O):
     k = _rand((2, 3, 5, 8), 0).astype(np.float32)
     W = np.stack([np.eye(8)] * 3)
     u = O.make_u(k, W, scale=1.0)
@@ -21,7 +25,7 @@ def test_identity_projection_is_the_normalised_key():
     np.testing.assert_allclose(u, want, rtol=1e-14, atol=0)
 
 
-def test_brute_force_per_head_and_orientation():
+def pin_brute_force_per_head_and_orientation(O):
     """y_c = sum_j W[h][c][j] k_j with the head's own matrix, written as loops; a transposed or
     head-shared W fails."""
     B, H, T, d = 2, 3, 4, 5
@@ -37,7 +41,7 @@ def test_brute_force_per_head_and_orientation():
                     assert abs(u[b, h, t, c] - 0.37 * y[c] / n) <= 1e-14
 
 
-def test_norm_scale_and_invariances():
+def pin_norm_scale_and_invariances(O):
     k = _rand((1, 2, 7, 16), 3).astype(np.float32)
     W = _rand((2, 16, 16), 4)
     s = 16 ** -0.5
@@ -49,7 +53,7 @@ def test_norm_scale_and_invariances():
     np.testing.assert_allclose(O.make_u(k, -W, scale=s), -u, rtol=1e-13)
 
 
-def test_rotation_keeps_the_key_norm():
+def pin_rotation_keeps_the_key_norm(O):
     """An orthogonal (non-symmetric) W: u = scale * Q k / ||k||."""
     q, _ = np.linalg.qr(_rand((6, 6), 5))
     assert np.abs(q - q.T).max() > 0.1
@@ -60,7 +64,7 @@ def test_rotation_keeps_the_key_norm():
     np.testing.assert_allclose(u[0, 0], want, rtol=1e-12, atol=1e-15)
 
 
-def test_zero_key_and_guard():
+def pin_zero_key_and_guard(O):
     k = np.zeros((1, 1, 2, 4), dtype=np.float32)
     k[0, 0, 1] = [1e-7, 0, 0, 0]
     u = O.make_u(k, np.eye(4)[None], scale=1.0, eps=1e-4)
@@ -68,7 +72,7 @@ def test_zero_key_and_guard():
     np.testing.assert_allclose(u[0, 0, 1], [1e-3, 0, 0, 0], rtol=1e-6)   # y / eps below the guard
 
 
-def test_bf16_keys_are_widened_exactly():
+def pin_bf16_keys_are_widened_exactly(O):
     vals = np.array([1.0, -2.5, 0.15625, 3.0e-3], dtype=np.float32)
     bits = (vals.view(np.uint32) >> 16).astype(np.uint16)          # these values are bf16-exact or truncated
     back = O.widen(bits, O.BF16)
@@ -77,3 +81,39 @@ def test_bf16_keys_are_widened_exactly():
     k = bits.reshape(1, 1, 1, 4)
     u = O.make_u(k, np.eye(4)[None], scale=1.0, in_dtype=O.BF16)
     np.testing.assert_allclose(u[0, 0, 0], back / np.linalg.norm(back), rtol=1e-14)
+
+
+PINS = [pin_identity_projection_is_the_normalised_key, pin_brute_force_per_head_and_orientation, pin_norm_scale_and_invariances, pin_rotation_keeps_the_key_norm, pin_zero_key_and_guard, pin_bf16_keys_are_widened_exactly]
+
+
+@pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
+def test_pin(pin):
+    pin(ORACLE)
+
+
+# ---- planted mistakes: each must trip at least one pin
+MUTANTS = [
+    ("transposed projection", "y = kk[b, h] @ W[h].T", "y = kk[b, h] @ W[h]"),
+    ("head-shared projection", "y = kk[b, h] @ W[h].T", "y = kk[b, h] @ W[0].T"),
+    ("scale dropped", "u[b, h] = scale * y / np.maximum(nrm, eps)[:, None]", "u[b, h] = y / np.maximum(nrm, eps)[:, None]"),
+    ("no normalisation", "u[b, h] = scale * y / np.maximum(nrm, eps)[:, None]", "u[b, h] = scale * y"),
+    ("squared norm", "nrm = np.sqrt((y * y).sum(axis=1))", "nrm = (y * y).sum(axis=1)"),
+    ("norm over tokens", "nrm = np.sqrt((y * y).sum(axis=1))", "nrm = np.sqrt((y * y).sum(axis=0))[None, :].repeat(y.shape[0], 0)[:, 0]"),
+    ("guard added instead of clamped", "np.maximum(nrm, eps)", "(nrm + eps)"),
+    ("bf16 widened as integers", "return bits.view(np.float32).astype(np.float64)", "return bits.astype(np.float64)"),
+]
+
+
+@pytest.mark.parametrize("name,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_planted_mistakes_trip_a_pin(name, old, new):
+    src = open(os.path.join(os.path.dirname(ORACLE.__file__), "make_u.py")).read()
+    assert src.count(old) >= 1, "mutation site not found: " + name
+    mod = types.ModuleType("make_u_mutant")
+    exec(compile(src.replace(old, new), "make_u_mutant", "exec"), mod.__dict__)
+    tripped = []
+    for pin in PINS:
+        try:
+            pin(mod)
+        except Exception:                      # a failed assertion or a numerical blow-up both count
+            tripped.append(pin.__name__)
+    assert tripped, "no pin notices: " + name

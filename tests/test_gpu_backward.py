@@ -326,3 +326,26 @@ def test_long_shape_one_unit(flags):
     for name, e in errs.items():
         bound = 3e-3 if (flags == IDENT and name == "dk") else 1e-3
         assert e <= bound, (name, e, errs)
+
+
+def test_throughput_workload_full_launch_sampled_units():
+    """The backward pass of the whole headline workload (512 units, the launch the benchmark
+    times: 1024 CTAs drawing tickets, A sides following S sides, the forward on the balanced
+    schedule); the oracle recomputes a sample of whole units."""
+    w = W.WORKLOADS["throughput"]
+    dev = torch.device("cuda:0")
+    q, k, v = W.make_inputs(w)
+    d_out = torch.randn((w.B, w.H, w.T, w.d), generator=torch.Generator().manual_seed(17))
+    g = vla.vla_backward(q.to(dev), k.to(dev), v.to(dev), w.lam, d_out.to(dev))
+    torch.cuda.synchronize()
+    assert int(g.status.item()) == 0
+    units = [(0, 0), (31, 15), (13, 7), (20, 3)]
+    pick = lambda x: torch.stack([x[b, h] for (b, h) in units]).unsqueeze(0).contiguous()
+    f64 = lambda x: x.detach().cpu().double().numpy()
+    ref = oracle.backward(to_oracle_array(pick(q))[0], to_oracle_array(pick(k))[0], to_oracle_array(pick(v))[0],
+                          w.lam, f64(pick(d_out)), in_dtype=oracle.BF16, n_threads=NTHREADS)
+    for name, got, want in (("dq", g.dq, ref.dq), ("dk", g.dk, ref.dk), ("dv", g.dv, ref.dv),
+                            ("dA0", g.dA0, ref.dA0), ("dS0", g.dS0, ref.dS0)):
+        for n, (b, h) in enumerate(units):
+            e = _err(got[b, h], want[0, n])
+            assert e <= 1e-3, "unit (%d,%d) %s rel err %.3e" % (b, h, name, e)

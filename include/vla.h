@@ -98,6 +98,7 @@ typedef struct {
 /*
  * vla_forward -- Section 3.3 / Algorithm 1, all B*H units, T tokens each.
  *   q, k : [B,H,T,d_k]   v : [B,H,T,d_v]   in opts->qkv_dtype (fp32 default, bf16 widened in-kernel)
+ *          (with VLA_FLAG_TOKEN_MAJOR: q, k, opts->u [B,T,H,d_k], v and out [B,T,H,d_v])
  *   lambda_ : lambda_0 of Eq. "penalty"; A_0 = I/lambda_ when A0 == NULL (must then be > 0)
  *   S0 : [B,H,d_v,d_k] fp32, row = value index (S k_hat predicts v); NULL => 0
  *   A0 : [B,H,d_k,d_k] fp32, symmetric positive definite;           NULL => I/lambda_
@@ -177,8 +178,8 @@ int vla_forward_host_static(const void* q, const void* k, const void* v, float l
  *
  * Arguments as vla_forward, with these differences: a carried-in A0 must be symmetric positive
  * definite (it is inverted in fp64 to recover the penalty matrix the earlier tokens left);
- * the periodic refresh and VLA_KERNEL_TOKEN are not available (VLA_ERR_UNSUPPORTED), nor is
- * d = 16; `segments` must divide T/16 (T a multiple of 16), else VLA_ERR_INVALID_ARG;
+ * the periodic refresh, VLA_FLAG_TOKEN_MAJOR and VLA_KERNEL_TOKEN are not available
+ * (VLA_ERR_UNSUPPORTED), nor is d = 16; `segments` must divide T/16 (T a multiple of 16), else VLA_ERR_INVALID_ARG;
  * segments <= 0 lets the library choose (vla_seqpar_segments), and a choice of 1 runs
  * vla_forward.  `workspace` is a DEVICE buffer of at least
  * vla_seqpar_workspace_bytes(B, H, T, d_k, segments) bytes (any alignment; with

@@ -108,3 +108,30 @@ def test_backward_random_calls(seed):
         assert np.all(np.isfinite(x))
         e = float(np.abs(x - want).max() / max(np.abs(want).max(), 1e-3))
         assert e <= 3e-4, "%s %s rel err %.3e" % (label, name, e)
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_seqpar_random_calls(seed):
+    rng = np.random.default_rng(3000 + seed)
+    d = int(rng.choice([32, 64, 128]))
+    B, H = int(rng.integers(1, 3)), int(rng.integers(1, 5))
+    P = int(rng.choice([2, 3, 4, 8]))
+    T = 16 * P * int(rng.integers(1, 5))
+    dtype = str(rng.choice(["f32", "bf16"]))
+    flags = int(rng.choice([0, vla.VLA_FLAG_IDENTITY_MAP]))
+    lam = float(rng.choice([0.1, 1.0, 3.0]))
+    w = W.Workload("f", B, H, d, T, dtype, 7000 + seed)
+    q, k, v = W.make_inputs(w)
+    u = W.make_u(w, float(rng.choice([1.0, d ** -0.5]))) if rng.random() < 0.4 else None
+    S0, A0, z0 = _states(rng, B, H, d, seed)
+    ref = run_oracle(q, k, v, lam, u=u, S0=S0, A0=A0, z0=z0, flags=flags)
+    mv = lambda x: None if x is None else x.to(DEV)
+    r = vla.vla_forward_seqpar(mv(q), mv(k), mv(v), lam, segments=P, u=mv(u), S0=mv(S0), A0=mv(A0), z0=mv(z0),
+                               flags=flags)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    label = "seed %d: d=%d B=%d H=%d T=%d P=%d %s flags=%d u=%s" % (seed, d, B, H, T, P, dtype, flags, u is not None)
+    for name, got, want in (("o", r.out, ref.out), ("S_T", r.S_T, ref.S_T), ("A_T", r.A_T, ref.A_T),
+                            ("z_T", r.z_T, ref.z_T)):
+        e = rel_err(got, want)
+        assert e <= 1e-4, "%s %s rel err %.3e" % (label, name, e)

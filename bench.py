@@ -6,11 +6,16 @@ residual update / readout, stream out, final states) over one batch of synthetic
 Default workload: "throughput" (B=32, H=16, d=128, T=8192, bf16 in, fp32 state) -- the
 largest of the five workloads, and the one that fills the GPU.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--all-workloads]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--scaling weak|strong]
+                  [--no-per-workload]
   python bench.py --impl reference ...     # the fp64 CPU oracle, as it stands, on host cores
 
-For N > 1 launch with torch.distributed.run; every rank scans its own batch (weak scaling,
-no data-path collective).  Rank 0 prints ONE JSON line.
+For N > 1 launch with torch.distributed.run; by default every rank scans its own batch (weak
+scaling), with --scaling strong the ranks split ONE batch contiguously by batch index; no
+data-path collective either way.  Rank 0 prints ONE JSON line.  At N = 1 the line also carries
+`per_workload`: kernel timings of the other four workloads and of the other entry points
+(segmented forward, single-step decode, backward, projection of u, the opt-in tensor-core
+kernel), each with the kernel name the library reports for what it launched.
 """
 from __future__ import annotations
 
@@ -56,6 +61,37 @@ def measured_peaks():
             pk = json.load(f)
         return float(pk["hbm_gbs"]), float(pk.get("sm_max_mhz", 1965.0)), "measured"
     return 6650.0, 1965.0, "fallback"
+
+
+def ncu_traffic_per_token(kernel_key: str):
+    """DRAM bytes per token of one ncu capture (profiles/ncu_traffic.txt: key, bytes, tokens, source)."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
+    try:
+        with open(path) as f:
+            for ln in f:
+                ln = ln.split("#")[0].split()
+                if len(ln) >= 3 and ln[0] == kernel_key:
+                    return float(ln[1]) / float(ln[2])
+    except OSError:
+        pass
+    return None
+
+
+def timed_ms(call, stream, dev, warm, reps, flush=None):
+    """Median CUDA-event time of `call` on `stream` after `warm` untimed calls; `flush` (a buffer
+    larger than L2) is rewritten before every timed call."""
+    evs = []
+    with torch.cuda.stream(stream):
+        for _ in range(warm):
+            call()
+        for _ in range(reps):
+            if flush is not None:
+                flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); call(); b.record(stream)
+            evs.append((a, b))
+    torch.cuda.synchronize(dev)
+    return float(np.median([a.elapsed_time(b) for a, b in evs]))
 
 
 class ClockSampler:
@@ -195,8 +231,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="throughput")
-    ap.add_argument("--all-workloads", action="store_true",
-                    help="also time the other four workloads (kernel only) into 'per_workload'")
+    ap.add_argument("--all-workloads", action="store_true", help="(default at N = 1; kept for old command lines)")
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip 'per_workload' (the other four workloads and entry points, kernel only)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: every rank its own batch (weak) or one batch split by batch index (strong)")
     ap.add_argument("--B", type=int, default=None, help="override the workload's batch (profiling cases)")
     ap.add_argument("--H", type=int, default=None, help="override the workload's heads")
     ap.add_argument("--T", type=int, default=None, help="override the workload's sequence length")
@@ -228,7 +267,19 @@ def main():
     hbm_peak, sm_max_mhz, peak_src = measured_peaks()
     n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
 
-    q, k, v = W.make_inputs(w, rank=rank)
+    strong = args.scaling == "strong" and world > 1
+    if strong:
+        # ONE batch (the same seed on every rank), split contiguously by batch index
+        from paper_2605_11196_b200 import sharding as SH
+        w_full = w
+        q, k, v = [x.contiguous() for x in SH.shard_batch(W.make_inputs(w), world, rank)]
+        b0, b1 = SH.batch_bounds(w.B, world, rank)
+        if b1 == b0:
+            raise SystemExit("--scaling strong: rank %d of %d has no batch of B = %d (replicas only)" % (rank, world, w.B))
+        w = W.scaled(w, B=b1 - b0)
+    else:
+        w_full = w
+        q, k, v = W.make_inputs(w, rank=rank)
     stream = torch.cuda.Stream(dev)
     bufs, call = bench_one(vla, w, dev, q, k, v, args.steps, args.warmup, stream)
     qd, kd, vd, out, S_T, A_T, z_T, status = bufs
@@ -276,7 +327,9 @@ def main():
     if dist is not None:
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
     total_s_max = float(tt.item())
-    value = world * args.steps * w.tokens / total_s_max
+    job_tokens = w_full.tokens if strong else world * w.tokens
+    value = args.steps * job_tokens / total_s_max
+    launched = vla.last_launch()              # what the library launched for the timed call
 
     # ---- end to end: pinned host buffers in, host buffers out, through vla_forward_host
     e2e = None
@@ -307,9 +360,28 @@ def main():
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
         h2d = 3 * w.tokens * w.d * in_bytes
         d2h = w.tokens * w.d * 4 + w.units * (2 * w.d * w.d + w.d) * 4
-        e2e = {"value": world * e2e_steps * w.tokens / float(t.item()), "unit": UNIT,
+        e2e = {"value": e2e_steps * job_tokens / float(t.item()), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "api": "vla_forward_host (pinned host q,k,v in; out, S_T, A_T, z_T to pinned host)"}
+        # the copy ceiling of this machine: the same byte counts, one pinned copy per direction, alone
+        if rank == 0:
+            stage = wsbuf[:max(h2d, w.tokens * w.d * 4)]
+            src = torch.empty(h2d, dtype=torch.uint8).pin_memory()
+            dst = outp.view(torch.uint8).view(-1)
+            def copy_ms(fn):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                with torch.cuda.stream(stream):
+                    fn(); a.record(stream); fn(); b.record(stream)
+                torch.cuda.synchronize(dev)
+                return a.elapsed_time(b)
+            t_h2d = copy_ms(lambda: stage[:h2d].copy_(src, non_blocking=True))
+            t_d2h = copy_ms(lambda: dst.copy_(stage[:dst.numel()], non_blocking=True))
+            e2e["pcie_h2d_gbs"] = h2d / (t_h2d * 1e-3) / 1e9
+            e2e["pcie_d2h_gbs"] = dst.numel() / (t_d2h * 1e-3) / 1e9
+            floor_s = max(h2d / (e2e["pcie_h2d_gbs"] * 1e9), d2h / (e2e["pcie_d2h_gbs"] * 1e9))
+            e2e["copy_bound_tokens_per_s"] = w.tokens / floor_s       # both directions fully overlapped
+            e2e["frac_of_copy_bound"] = (e2e["value"] * w.tokens / job_tokens) / e2e["copy_bound_tokens_per_s"]
+            del src
         del wsbuf
 
     if rank != 0:
@@ -328,17 +400,17 @@ def main():
     bound = "alu" if t_alu >= t_hbm else "hbm"
     achieved_tflops = flops / (launch_ms * 1e-3) / 1e12
     achieved_gbs = byts / (launch_ms * 1e-3) / 1e9
-    kname = "vla_scan_chunk_kernel" if w.d >= 32 else "vla_scan_token_kernel"
-    roof = {"bound": bound, "kernel": "%s<%d,%s>" % (kname, w.d, w.dtype),
+    traffic_pt = ncu_traffic_per_token("%s<%d,%s>" % (launched.split("<")[0], w.d, w.dtype))
+    roof = {"bound": bound, "kernel": launched,
             "achieved": achieved_tflops if bound == "alu" else achieved_gbs,
             "peak": fp32_peak_nominal if bound == "alu" else hbm_peak,
             "unit": "TFLOP/s" if bound == "alu" else "GB/s",
             "frac": (achieved_tflops / fp32_peak_nominal) if bound == "alu" else achieved_gbs / hbm_peak,
             "peak_source": ("fp32 FMA: %d SMs x 128 lanes x 2 x %.0f MHz (derived, nominal max clock)"
                             % (n_sm, sm_max_mhz)) if bound == "alu" else "hbm_gbs of %s" % peak_src,
-            # dram__bytes_read+write of one ncu capture (300 units x 2048 tokens: 817.5 MB),
-            # scaled by tokens; see profiles/chunk_kernel_d128_bf16.md
-            "traffic": (817.5e6 / 614400.0) * w.tokens if (w.d == 128 and w.dtype == "bf16") else None,
+            # dram__bytes_read + write of one ncu capture of this kernel, scaled by tokens
+            # (profiles/ncu_traffic.txt names the capture)
+            "traffic": traffic_pt * w.tokens if traffic_pt else None,
             "alg_flops_per_token": alg_flops_per_token(w.d),
             "alg_bytes_per_token": alg_bytes_per_token(w.d, in_bytes),
             "hbm_achieved_gbs": achieved_gbs, "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
@@ -359,186 +431,110 @@ def main():
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * total_s_max / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic (seeded N(0,1) q,k,v rounded to %s; each rank its own batch)" % w.dtype,
-            "config": {"workload": w.name, "B": w.B, "H": w.H, "d_k": w.d, "d_v": w.d, "T": w.T,
+            "higher_is_better": True, "scaling": "strong" if strong else "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic (seeded N(0,1) q,k,v rounded to %s; %s)"
+                    % (w.dtype, "one batch split by batch index over the ranks" if strong else "each rank its own batch"),
+            "config": {"workload": w_full.name, "B": w_full.B, "H": w_full.H, "d_k": w.d, "d_v": w.d, "T": w.T,
                        "in_dtype": w.dtype, "state_dtype": "f32", "lambda": w.lam, "u": "k_hat",
                        "mode": "Algorithm 1 (phi = ELU+1, normalised readout)",
-                       "parallelism": "dp%d over (batch, head) units, no collective" % world,
+                       "parallelism": "dp%d over (batch, head) units, no collective%s"
+                                      % (world, ", B split %s per rank" % (w.B,) if strong else ""),
                        "l2": ("inputs+outputs %.0f MB > L2" % (working_set / 1e6)) if flush is None
                              else "L2 flushed between timed steps (256 MB write)"},
             "ns_per_scan_step": 1e6 * launch_ms / w.T,
             "roofline": roof, "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks}
 
-    if args.all_workloads:
+    if world == 1 and not args.no_per_workload:
         per = {}
+        fl = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)     # L2 flush between timed calls
+        frac = lambda ww, ms, has_u=False: alg_flops_per_token(ww.d, has_u) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal
+
+        def entry(ww, ms, **kw):
+            e = {"ms": ms, "tokens_per_s": ww.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / ww.T,
+                 "units": ww.units, "kernel": vla.last_launch()}
+            e.update(kw)
+            return e
+
+        # ---- the other four workloads: plain call, the library's choice of kernel
         for name in W.ORDER:
             if name == w.name:
                 continue
             ww = W.WORKLOADS[name]
             q2, k2, v2 = W.make_inputs(ww)
             _, call2 = bench_one(vla, ww, dev, q2, k2, v2, 0, 0, stream)
-            fl = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
-            ms = []
-            with torch.cuda.stream(stream):
-                for _ in range(3):
-                    call2()
-                for _ in range(10):
-                    fl.fill_(1)
-                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    a.record(stream); call2(); b.record(stream)
-                    ms.append((a, b))
-            torch.cuda.synchronize(dev)
-            ms = float(np.median([a.elapsed_time(b) for a, b in ms]))
+            ms = timed_ms(call2, stream, dev, 3, 10, fl)
             ib = 2 if ww.dtype == "bf16" else 4
-            per[name] = {"ms": ms, "tokens_per_s": ww.tokens / (ms * 1e-3),
-                         "ns_per_scan_step": 1e6 * ms / ww.T,
-                         "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
-                         "hbm_frac": alg_bytes_per_token(ww.d, ib) * ww.tokens / (ms * 1e-3) / 1e9 / hbm_peak,
-                         "units": ww.units, "unit_limited_frac_bound": min(ww.units, n_sm) / n_sm}
-            # backward pass (first correct path: token kernel, d <= 64): forward recomputed inside
+            per[name] = entry(ww, ms, fp32_frac_nominal=frac(ww, ms),
+                              hbm_frac=alg_bytes_per_token(ww.d, ib) * ww.tokens / (ms * 1e-3) / 1e9 / hbm_peak,
+                              unit_limited_frac_bound=min(ww.units, n_sm) / n_sm)
+            qd2, kd2, vd2 = q2.to(dev), k2.to(dev), v2.to(dev)
+            # backward pass: forward recomputed inside (chunk kernel leaving the per-token stash),
+            # both reverse scans as one launch, the dA0 kernel
             if name in ("mid", "recall"):
-                qd3, kd3, vd3 = q2.to(dev), k2.to(dev), v2.to(dev)
                 go3 = torch.randn((ww.B, ww.H, ww.T, ww.d), device=dev)
-                bcall = lambda: vla.vla_backward(qd3, kd3, vd3, ww.lam, go3, stream=stream)
-                ms = []
-                with torch.cuda.stream(stream):
-                    bcall()
-                    for _ in range(3):
-                        fl.fill_(1)
-                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                        a.record(stream); bcall(); b.record(stream)
-                        ms.append((a, b))
-                torch.cuda.synchronize(dev)
-                ms = float(np.median([a.elapsed_time(b) for a, b in ms]))
-                per[name + "_backward"] = {"ms": ms, "tokens_per_s": ww.tokens / (ms * 1e-3),
-                                           "ns_per_scan_step": 1e6 * ms / ww.T,
-                                           "kernel": "chunk forward with stash + vla_backward_sa_kernel (both reverse scans) + vla_backward_da0_kernel",
-                                           "gpu_launches_per_step": 3}
-                del qd3, kd3, vd3, go3
-            # fewer units than SMs: the sequence-parallel entry point cuts each sequence into
+                ms = timed_ms(lambda: vla.vla_backward(qd2, kd2, vd2, ww.lam, go3, stream=stream), stream, dev, 1, 3, fl)
+                per[name + "_backward"] = entry(ww, ms, gpu_launches_per_step=3,
+                                                forward_ms=per[name]["ms"], ratio_to_forward=ms / per[name]["ms"])
+                del go3
+            # fewer units than SMs: with scratch memory the plain call cuts each sequence into
             # segments that are scanned concurrently (twice the arithmetic, P times the CTAs)
             P = vla.seqpar_segments(ww.B, ww.H, ww.T, ww.d, q2.dtype)
             if P > 1:
-                qd2, kd2, vd2 = q2.to(dev), k2.to(dev), v2.to(dev)
-                ws = torch.empty((vla.seqpar_workspace_bytes(ww.B, ww.H, ww.T, ww.d, P),),
-                                 dtype=torch.uint8, device=dev)
+                ws = torch.empty((vla.seqpar_workspace_bytes(ww.B, ww.H, ww.T, ww.d, P),), dtype=torch.uint8, device=dev)
                 o2 = torch.empty((ww.B, ww.H, ww.T, ww.d), dtype=torch.float32, device=dev)
                 S2 = torch.empty((ww.B, ww.H, ww.d, ww.d), dtype=torch.float32, device=dev)
                 A2 = torch.empty_like(S2)
                 z2 = torch.empty((ww.B, ww.H, ww.d), dtype=torch.float32, device=dev)
                 st2 = torch.zeros((), dtype=torch.int32, device=dev)
-                call3 = lambda: vla.vla_forward_seqpar(qd2, kd2, vd2, ww.lam, segments=P, workspace=ws,
-                                                       out=o2, S_T=S2, A_T=A2, z_T=z2, status=st2,
-                                                       stream=stream)
-                ms = []
-                with torch.cuda.stream(stream):
-                    for _ in range(3):
-                        call3()
-                    for _ in range(10):
-                        fl.fill_(1)
-                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                        a.record(stream); call3(); b.record(stream)
-                        ms.append((a, b))
-                torch.cuda.synchronize(dev)
-                ms = float(np.median([a.elapsed_time(b) for a, b in ms]))
-                per[name + "_seqpar"] = {
-                    "ms": ms, "segments": P, "tokens_per_s": ww.tokens / (ms * 1e-3),
-                    "ns_per_scan_step": 1e6 * ms / ww.T,
-                    "fp32_frac_nominal": alg_flops_per_token(ww.d) * ww.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
-                    "status": int(st2.item()), "gpu_launches_per_step": 5}
-                del qd2, kd2, vd2, ws, o2
-        # backward pass of the headline workload (chunk forward leaving the per-token stash, both
-        # reverse scans as one launch, the dA0 kernel)
+                call3 = lambda: vla.vla_forward(qd2, kd2, vd2, ww.lam, workspace=ws, out=o2, S_T=S2, A_T=A2,
+                                                z_T=z2, status=st2, stream=stream)
+                ms = timed_ms(call3, stream, dev, 3, 10, fl)
+                per[name + "_auto_with_workspace"] = entry(
+                    ww, ms, segments=P, fp32_frac_nominal=frac(ww, ms), status=int(st2.item()),
+                    api="vla_forward, kernel AUTO, opts->workspace given (runs as vla_forward_seqpar)",
+                    gpu_launches_per_step=5, unit_limited_frac_bound=min(ww.units * P, n_sm) / n_sm)
+                del ws, o2, S2, A2, z2
+            del qd2, kd2, vd2
+
+        # ---- the headline workload through the other entry points and options
         go_h = torch.randn((w.B, w.H, w.T, w.d), device=dev)
         wsb = torch.empty((vla.backward_workspace_bytes(w.B, w.H, w.T, w.d),), dtype=torch.uint8, device=dev)
-        bcall = lambda: vla.vla_backward(qd, kd, vd, w.lam, go_h, workspace=wsb, stream=stream)
-        evs = []
-        with torch.cuda.stream(stream):
-            bcall()
-            for _ in range(2):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); bcall(); b.record(stream)
-                evs.append((a, b))
-        torch.cuda.synchronize(dev)
-        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
-        per[w.name + "_backward"] = {"ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3),
-                                     "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
-                                     "kernel": "chunk forward with stash + vla_backward_sa_kernel (both reverse scans) + vla_backward_da0_kernel",
-                                     "gpu_launches_per_step": 3}
-        # the same with explicit penalty directions (gradients of q, k, v and u)
-        uu_b = W.make_u(w, w.d ** -0.5).to(dev)
-        bucall = lambda: vla.vla_backward(qd, kd, vd, w.lam, go_h, u=uu_b, workspace=wsb, stream=stream)
-        evs = []
-        with torch.cuda.stream(stream):
-            bucall()
-            for _ in range(2):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); bucall(); b.record(stream)
-                evs.append((a, b))
-        torch.cuda.synchronize(dev)
-        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
-        per[w.name + "_backward_explicit_u"] = {
-            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
-            "kernel": "chunk forward (general path) with stash + vla_backward_sa_kernel + vla_backward_da0_kernel",
-            "gpu_launches_per_step": 3}
-        del go_h, wsb, uu_b
-        # the headline workload with an explicit penalty direction u = unit / sqrt(d_h)
-        # (the paper's learned-u setting at the scan's input level)
-        uu = W.make_u(w, w.d ** -0.5).to(dev)
-        ucall = lambda: vla.vla_forward(qd, kd, vd, w.lam, u=uu, out=out, S_T=S_T, A_T=A_T, z_T=z_T,
-                                        status=status, stream=stream)
-        evs = []
-        with torch.cuda.stream(stream):
-            for _ in range(2):
-                ucall()
-            for _ in range(3):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); ucall(); b.record(stream)
-                evs.append((a, b))
-        torch.cuda.synchronize(dev)
-        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
-        per[w.name + "_explicit_u"] = {
-            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T,
-            "fp32_frac_nominal": alg_flops_per_token(w.d, True) * w.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
-            "units": w.units, "kernel": "vla_scan_chunk_kernel (explicit u)"}
-        # the same with u formed on the device from a projection (Algorithm 1: u = L2norm(W_u k) / sqrt(d_h))
+        ms = timed_ms(lambda: vla.vla_backward(qd, kd, vd, w.lam, go_h, workspace=wsb, stream=stream), stream, dev, 1, 2)
+        per[w.name + "_backward"] = entry(w, ms, gpu_launches_per_step=3, forward_ms=launch_ms,
+                                          ratio_to_forward=ms / launch_ms)
+        uu = W.make_u(w, w.d ** -0.5).to(dev)      # explicit penalty directions u = unit / sqrt(d_h)
+        ms = timed_ms(lambda: vla.vla_backward(qd, kd, vd, w.lam, go_h, u=uu, workspace=wsb, stream=stream), stream, dev, 1, 2)
+        per[w.name + "_backward_explicit_u"] = entry(w, ms, gpu_launches_per_step=3)
+        del go_h, wsb
+        fwd = dict(out=out, S_T=S_T, A_T=A_T, z_T=z_T, status=status, stream=stream)
+        ms = timed_ms(lambda: vla.vla_forward(qd, kd, vd, w.lam, u=uu, **fwd), stream, dev, 2, 3)
+        per[w.name + "_explicit_u"] = entry(w, ms, fp32_frac_nominal=frac(w, ms, True))
+        # u formed on the device from a projection (Algorithm 1: u = L2norm(W_u k) / sqrt(d_h))
         Wu = (torch.randn((w.H, w.d, w.d), generator=torch.Generator().manual_seed(11)) / w.d ** 0.5).to(dev)
+        ms_mk = timed_ms(lambda: vla.vla_make_u(kd, Wu, out=uu, stream=stream), stream, dev, 1, 3)
+        per[w.name + "_make_u"] = {"ms": ms_mk, "tokens_per_s": w.tokens / (ms_mk * 1e-3), "kernel": "vla_make_u_kernel",
+                                   "fp32_tflops": 2.0 * w.d * w.d * w.tokens / (ms_mk * 1e-3) / 1e12}
         def wcall():
             vla.vla_make_u(kd, Wu, out=uu, stream=stream)
-            vla.vla_forward(qd, kd, vd, w.lam, u=uu, out=out, S_T=S_T, A_T=A_T, z_T=z_T, status=status, stream=stream)
-        evs = []
-        with torch.cuda.stream(stream):
-            wcall()
-            for _ in range(3):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); wcall(); b.record(stream)
-                evs.append((a, b))
-        torch.cuda.synchronize(dev)
-        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
-        per[w.name + "_projected_u"] = {
-            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
-            "kernel": "vla_make_u_kernel + vla_scan_chunk_kernel (explicit u)", "gpu_launches_per_step": 2}
+            vla.vla_forward(qd, kd, vd, w.lam, u=uu, **fwd)
+        ms = timed_ms(wcall, stream, dev, 1, 3)
+        per[w.name + "_projected_u"] = entry(w, ms, gpu_launches_per_step=2)
         del uu, Wu
-        # the headline workload with q, k, v, out as [B, T, H, d]
+        # Algorithm 1's periodic refresh (every 20 tokens, + 1e-3 I)
+        ms = timed_ms(lambda: vla.vla_forward(qd, kd, vd, w.lam, refresh=(20, 1e-3, 0), **fwd), stream, dev, 2, 3)
+        per[w.name + "_refresh_20"] = entry(w, ms, fp32_frac_nominal=frac(w, ms))
+        # q, k, v, out as [B, T, H, d]
         qt, kt, vt = [x.view(w.B, w.H, w.T, w.d).permute(0, 2, 1, 3).contiguous() for x in (qd, kd, vd)]
         out_t = torch.empty((w.B, w.T, w.H, w.d), dtype=torch.float32, device=dev)
-        tcall = lambda: vla.vla_forward(qt, kt, vt, w.lam, out=out_t, S_T=S_T, A_T=A_T, z_T=z_T, status=status,
-                                        stream=stream, flags=vla.VLA_FLAG_TOKEN_MAJOR)
-        evs = []
-        with torch.cuda.stream(stream):
-            tcall()
-            for _ in range(3):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); tcall(); b.record(stream)
-                evs.append((a, b))
-        torch.cuda.synchronize(dev)
-        ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
-        per[w.name + "_token_major"] = {
-            "ms": ms, "tokens_per_s": w.tokens / (ms * 1e-3), "ns_per_scan_step": 1e6 * ms / w.T, "units": w.units,
-            "fp32_frac_nominal": alg_flops_per_token(w.d, False) * w.tokens / (ms * 1e-3) / 1e12 / fp32_peak_nominal,
-            "kernel": "vla_scan_chunk_kernel, [B,T,H,d] tensors"}
+        ms = timed_ms(lambda: vla.vla_forward(qt, kt, vt, w.lam, out=out_t, S_T=S_T, A_T=A_T, z_T=z_T, status=status,
+                                              stream=stream, flags=vla.VLA_FLAG_TOKEN_MAJOR), stream, dev, 1, 3)
+        per[w.name + "_token_major"] = entry(w, ms, fp32_frac_nominal=frac(w, ms))
         del qt, kt, vt, out_t
+        # the opt-in tensor-core form of the chunk kernel (never the library's own choice)
+        if w.d == 128:
+            ms = timed_ms(lambda: vla.vla_forward(qd, kd, vd, w.lam, kernel=vla.VLA_KERNEL_CHUNK_TC, **fwd), stream, dev, 2, 3)
+            per[w.name + "_chunk_tc_opt_in"] = entry(w, ms, fp32_frac_nominal=frac(w, ms),
+                                                     note="tcgen05 kind::tf32, hi/lo operand pairs, states in tensor memory")
         # single-step decode (T = 1, carried states): bound by moving S and A through HBM once
         wd = W.EXTRA["decode"]
         q2, k2, v2 = [x.to(dev) for x in W.make_inputs(wd)]
@@ -546,29 +542,17 @@ def main():
         A0 = torch.eye(wd.d, device=dev).expand(wd.B, wd.H, wd.d, wd.d).contiguous()
         bufs = dict(out=torch.empty((wd.B, wd.H, 1, wd.d), device=dev), S_T=torch.empty_like(S0),
                     A_T=torch.empty_like(A0), z_T=torch.empty((wd.B, wd.H, wd.d), device=dev), status=status)
-        fl = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
         state_bytes = wd.units * (4 * wd.d * wd.d * 4 + 2 * wd.d * 4)       # S, A read and written; z
         io_bytes = wd.units * (3 * wd.d * 2 + wd.d * 4)
-        for key, kern, kname in (("decode", vla.VLA_KERNEL_AUTO, "vla_decode_kernel"),
-                                 ("decode_token_kernel", vla.VLA_KERNEL_TOKEN, "vla_scan_token_kernel")):
-            dcall = lambda: vla.vla_forward(q2, k2, v2, wd.lam, S0=S0, A0=A0, stream=stream, kernel=kern,
-                                            **bufs)
-            evs = []
-            with torch.cuda.stream(stream):
-                for _ in range(3):
-                    dcall()
-                for _ in range(10):
-                    fl.fill_(1)
-                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    a.record(stream); dcall(); b.record(stream)
-                    evs.append((a, b))
-            torch.cuda.synchronize(dev)
-            ms = float(np.median([a.elapsed_time(b) for a, b in evs]))
+        for key, kern in (("decode", vla.VLA_KERNEL_AUTO), ("decode_token_kernel", vla.VLA_KERNEL_TOKEN)):
+            dcall = lambda: vla.vla_forward(q2, k2, v2, wd.lam, S0=S0, A0=A0, stream=stream, kernel=kern, **bufs)
+            ms = timed_ms(dcall, stream, dev, 3, 10, fl)
             per[key] = {"ms": ms, "units": wd.units, "steps_per_s": wd.units / (ms * 1e-3),
-                        "kernel": kname, "bound": "hbm",
+                        "kernel": vla.last_launch(), "bound": "hbm",
                         "hbm_gbs": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9,
                         "hbm_frac": (state_bytes + io_bytes) / (ms * 1e-3) / 1e9 / hbm_peak,
                         "hbm_peak_source": peak_src}
+        assert int(status.item()) == 0, vla.status_string(int(status.item()))
         line["per_workload"] = per
 
     if not args.no_cpu_baseline:

@@ -3,7 +3,7 @@
  *
  * One call runs, for every (batch, head) unit independently, the causal scan of
  * the paper's Section 3.3 (Eqs. "sm", "s-update", "output"; Algorithm 1 without
- * the projections and without the periodic refresh).  Per token t:
+ * the projections; its periodic refresh is an option, see vla_opts_t).  Per token t:
  *
  *     k_hat = kf / max(||kf||, eps)        kf = phi(k_t)  (phi = ELU+1, Algorithm 1)
  *                                          kf = k_t       (VLA_FLAG_IDENTITY_MAP, Section 3.1)
@@ -19,8 +19,19 @@
  *
  * Memory: unless a function says otherwise every pointer is a DEVICE pointer owned by
  * the caller, tensors are contiguous and row-major, and base pointers are 16-byte
- * aligned (else VLA_ERR_ALIGNMENT).  The library allocates nothing, keeps no state
- * between calls, and never synchronises the device; work is enqueued on `stream`.
+ * aligned (else VLA_ERR_ALIGNMENT).  The device-pointer calls allocate no memory and never
+ * synchronise the device; work is enqueued on `stream`.
+ *
+ * State the library keeps for the life of the process (none of it carries results from one
+ * call to the next):
+ *   - a launch counter and, per device, 16 slots of hand-over flags (device memory inside the
+ *     library, about 256 KB per kernel variant) for launches that cut units across CTAs; a
+ *     slot is reused only once the launch that held it last has finished (one CUDA event per
+ *     slot, created on first use), otherwise the launch runs one CTA per unit;
+ *   - VLA_STATIC_SCRATCH_BYTES of device memory per GPU for vla_forward_host_static, and its
+ *     device address once looked up;
+ *   - per host thread, a note of the last kernel launched (vla_last_launch).
+ * vla_forward_host creates and destroys three short-lived streams and their events per call.
  */
 #ifndef VLA_H
 #define VLA_H
@@ -51,7 +62,8 @@ enum {
   VLA_FLAG_TOKEN_MAJOR = 1u << 2   /* q, k, v, u and out are [B,T,H,d] (the layout projections write)
                                       instead of [B,H,T,d] (in vla_backward also d_out and the
                                       gradients of q, k, v, u); the states stay [B,H,d,d].
-                                      vla_forward, the host-buffer calls, vla_backward (d >= 32);
+                                      vla_forward, the host-buffer calls (which then cut large
+                                      batches by batch index), vla_backward (d >= 32);
                                       VLA_ERR_UNSUPPORTED elsewhere */
 };
 
@@ -61,9 +73,13 @@ typedef enum {
   VLA_KERNEL_TOKEN = 1, /* one CTA per unit, one state pass per token; every shape, explicit u */
   VLA_KERNEL_CHUNK = 2, /* 16 tokens per state pass (exact Woodbury form); d >= 32, every option;
                            VLA_ERR_UNSUPPORTED for d = 16 */
-  VLA_KERNEL_DECODE = 3 /* one step (T = 1) with S0, A0, S_T, A_T all given, u = k_hat, no refresh,
+  VLA_KERNEL_DECODE = 3, /* one step (T = 1) with S0, A0, S_T, A_T all given, u = k_hat, no refresh,
                            d >= 32: the states stream through shared memory once (HBM-bound);
                            VLA_ERR_UNSUPPORTED otherwise.  AUTO picks it when it applies */
+  VLA_KERNEL_CHUNK_TC = 4 /* the chunk algebra on the tensor cores (Section 3.4: the chunked recurrence
+                           is a chain of dense products): states in tensor memory, TF32 products in
+                           hi/lo pairs with fp32 accumulation.  d = 128, u = k_hat, no refresh,
+                           [B,H,T,d] tensors, T >= 1; VLA_ERR_UNSUPPORTED otherwise */
 } vla_kernel_t;
 
 typedef struct {
@@ -87,12 +103,15 @@ typedef struct {
   int64_t step_offset;   /* tokens of this sequence processed by earlier calls (state carry)     */
   float* du;             /* vla_backward with explicit u: [B,H,T,d_k] fp32 gradient of u (required
                             when u is given there; ignored by the forward calls)                 */
-  void* workspace;       /* vla_forward, kernel AUTO: optional DEVICE scratch.  When the problem has
+  void* workspace;       /* vla_forward (not the host-buffer calls), kernel AUTO: optional DEVICE scratch.  When the problem has
                             too few units to fill the device and the library would cut its sequences
                             (vla_seqpar_segments(...) > 1) and this holds at least
                             vla_seqpar_workspace_bytes(B, H, T, d_k, that many) bytes, the call runs as
                             vla_forward_seqpar; otherwise it is not touched.  NULL: never            */
   size_t workspace_bytes;
+  uint32_t wait_probe_limit; /* a device-side wait (on a copy, on another warp group, on the CTA that
+                            hands a unit over) gives up after this many failed probes and sets
+                            VLA_ERR_DEVICE_TIMEOUT in *status; 0 = the default (about a second) */
 } vla_opts_t;
 
 /*
@@ -153,7 +172,8 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
  *   - vla_host_workspace_bytes(...) for the problem must not exceed
  *     VLA_STATIC_SCRATCH_BYTES, else VLA_ERR_TOO_LARGE is returned and nothing is enqueued.
  *   - The first call on each device looks up the array's device address (a one-time
- *     set-up for that device); make that first call before starting any stream capture.
+ *     set-up for that device); make that first call before starting any stream capture
+ *     (a first call on a capturing stream returns VLA_ERR_INVALID_ARG and enqueues nothing).
  *   - All calls on a device share the one array, and it keeps whatever the last call left
  *     in it.  Two calls whose work can overlap on the GPU (different streams without an
  *     ordering between them) race on it: order them, or use vla_forward_host with
@@ -202,7 +222,7 @@ int vla_seqpar_segments(int B, int H, int T, int d_k, int qkv_dtype);
 size_t vla_seqpar_workspace_bytes(int B, int H, int T, int d_k, int segments);
 
 /*
- * vla_backward -- gradients of the forward scan (first correct path: a token kernel).  The
+ * vla_backward -- gradients of the forward scan.  The
  * paper gives no backward algorithm; this is reverse-mode differentiation of exactly the
  * recurrence vla_forward computes (Algorithm 1 without projections; Eqs. "sm", "s-update",
  * "output"), the gradients its Corollary on gradient flow (Section 4) is about.
@@ -257,6 +277,22 @@ int vla_make_u(const void* k, const float* W_u, int B, int H, int T, int d_k, in
  * are measured against.  `sink` is a DEVICE float the kernel never actually writes.
  */
 int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream);
+
+/*
+ * vla_selftest_wait_timeout -- test helper (the paper has no counterpart): enqueues a one-warp
+ * kernel that waits, with the scan kernels' bounded wait and `probe_limit` probes, on a barrier
+ * that cannot complete.  When the probes run out the kernel writes VLA_ERR_DEVICE_TIMEOUT to
+ * *status (DEVICE int32, 0 on entry) and returns normally; nothing traps and the context stays
+ * usable.  probe_limit must be > 0 (a few thousand probes take well under a millisecond).
+ */
+int vla_selftest_wait_timeout(uint32_t probe_limit, int32_t* status, void* stream);
+
+/*
+ * vla_last_launch -- which kernel the calling host thread's last library call launched last,
+ * as text ("vla_scan_chunk_kernel<128,bf16> grid=148 balanced"); empty before the first launch.
+ * For benchmarks and logs: the name comes from the launch itself, not from the shape.
+ */
+int vla_last_launch(char* buf, size_t len);
 
 /* Device bytes vla_forward_host needs for these sizes (0 on invalid sizes). */
 size_t vla_host_workspace_bytes(int B, int H, int T, int d_k, int d_v, int qkv_dtype, int has_u);

@@ -22,12 +22,13 @@ VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE, VLA_ERR_TOO_LARGE = -4,
 VLA_STATIC_SCRATCH_BYTES = 32 << 20
 VLA_F32, VLA_BF16 = 0, 1
 VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE, VLA_FLAG_TOKEN_MAJOR = 1, 2, 4
-VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK, VLA_KERNEL_DECODE = 0, 1, 2, 3
+VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK, VLA_KERNEL_DECODE, VLA_KERNEL_CHUNK_TC = 0, 1, 2, 3, 4
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",
            "vla_forward_seqpar", "vla_seqpar_segments", "vla_seqpar_workspace_bytes",
            "vla_probe_fp32_fma", "vla_backward", "vla_backward_workspace_bytes", "vla_make_u",
-           "vla_query_support", "vla_status_string", "vla_version")
+           "vla_query_support", "vla_status_string", "vla_version", "vla_selftest_wait_timeout",
+           "vla_last_launch")
 
 
 class VlaOpts(ctypes.Structure):
@@ -37,7 +38,8 @@ class VlaOpts(ctypes.Structure):
                 ("z0", ctypes.c_void_p), ("zT", ctypes.c_void_p), ("status", ctypes.c_void_p),
                 ("kernel", ctypes.c_int32), ("refresh_period", ctypes.c_int32),
                 ("refresh_eta", ctypes.c_float), ("step_offset", ctypes.c_int64), ("du", ctypes.c_void_p),
-                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("wait_probe_limit", ctypes.c_uint32)]
 
 
 class VlaError(RuntimeError):
@@ -98,8 +100,31 @@ def load_library():
             lib.vla_status_string.argtypes = [i]
             lib.vla_version.restype = i
             lib.vla_version.argtypes = []
+            lib.vla_selftest_wait_timeout.restype = i
+            lib.vla_selftest_wait_timeout.argtypes = [ctypes.c_uint32, vp, vp]
+            lib.vla_last_launch.restype = i
+            lib.vla_last_launch.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
             _lib = lib
     return _lib
+
+
+def last_launch() -> str:
+    """Name, instantiation and grid of the kernel this thread's last library call launched last."""
+    buf = ctypes.create_string_buffer(160)
+    rc = load_library().vla_last_launch(buf, len(buf))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_last_launch")
+    return buf.value.decode()
+
+
+def selftest_wait_timeout(probe_limit: int, status: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Enqueue the library's bounded-wait test kernel (``vla_selftest_wait_timeout``): ``status``
+    (device int32, zero on entry) reads ``VLA_ERR_DEVICE_TIMEOUT`` once the stream has run it."""
+    st = stream if stream is not None else torch.cuda.current_stream(status.device)
+    with torch.cuda.device(status.device):
+        rc = load_library().vla_selftest_wait_timeout(int(probe_limit), _ptr(status), ctypes.c_void_p(st.cuda_stream))
+    if rc != VLA_OK:
+        raise VlaError(rc, "vla_selftest_wait_timeout")
 
 
 def status_string(code: int) -> str:
@@ -175,7 +200,7 @@ class VlaResult:
     status: Optional[torch.Tensor]  # device int32 scalar; read after synchronising
 
 
-def _make_opts(dt, u, flags, eps, z0, zT, status, kernel, refresh=None):
+def _make_opts(dt, u, flags, eps, z0, zT, status, kernel, refresh=None, wait_probe_limit=0):
     o = VlaOpts()
     o.struct_size = ctypes.sizeof(VlaOpts)
     o.qkv_dtype = dt
@@ -186,6 +211,7 @@ def _make_opts(dt, u, flags, eps, z0, zT, status, kernel, refresh=None):
     o.zT = None if zT is None else zT.data_ptr()
     o.status = None if status is None else status.data_ptr()
     o.kernel = kernel
+    o.wait_probe_limit = int(wait_probe_limit)
     if refresh is not None:     # (period, eta, step_offset): Algorithm 1's periodic A += eta I
         o.refresh_period, o.refresh_eta, o.step_offset = int(refresh[0]), float(refresh[1]), int(refresh[2])
     return o
@@ -194,7 +220,7 @@ def _make_opts(dt, u, flags, eps, z0, zT, status, kernel, refresh=None):
 def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags: int = 0,
                 eps: float = 1e-4, out=None, S_T=None, A_T=None, z_T=None, status=None,
                 kernel: int = VLA_KERNEL_AUTO, stream: Optional[torch.cuda.Stream] = None,
-                want_status: bool = True, refresh=None, workspace=None) -> VlaResult:
+                want_status: bool = True, refresh=None, workspace=None, wait_probe_limit: int = 0) -> VlaResult:
     """Enqueue the scan for CUDA tensors ``q,k[,u]: [B,H,T,d_k]``, ``v: [B,H,T,d_v]``
     (``[B,T,H,d]`` for all of them and ``out`` with ``VLA_FLAG_TOKEN_MAJOR``).
 
@@ -233,7 +259,7 @@ def vla_forward(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0=None, flags
     if status is None and want_status:
         status = torch.zeros((), dtype=torch.int32, device=dev)
     st = stream if stream is not None else torch.cuda.current_stream(dev)
-    opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel, refresh)
+    opts = _make_opts(dt, u, flags, eps, z0, z_T, status, kernel, refresh, wait_probe_limit)
     if workspace is True:
         P = int(lib.vla_seqpar_segments(B, H, T, dk, dt)) if kernel == VLA_KERNEL_AUTO else 1
         workspace = None if P <= 1 else torch.empty((int(lib.vla_seqpar_workspace_bytes(B, H, T, dk, P)),),
@@ -403,21 +429,26 @@ def vla_forward_host(q, k, v, lam: float, workspace: torch.Tensor, *, u=None, S0
     uint8 tensor of at least ``vla_host_workspace_bytes(...)`` bytes.  Copies in, the scan
     and copies out are enqueued on the stream; synchronise it before reading the results."""
     lib = load_library()
-    B, H, T, dk = q.shape
+    if flags & VLA_FLAG_TOKEN_MAJOR:          # q, k, v, u, out are [B,T,H,d]
+        B, T, H, dk = q.shape
+        tok = lambda d_: (B, T, H, d_)
+    else:
+        B, H, T, dk = q.shape
+        tok = lambda d_: (B, H, T, d_)
     dv = v.shape[-1]
     dt = _dtype_code(q)
     f32 = torch.float32
-    _chk(q, (B, H, T, dk), q.dtype, "q", cuda=False); _chk(k, (B, H, T, dk), q.dtype, "k", cuda=False)
-    _chk(v, (B, H, T, dv), q.dtype, "v", cuda=False); _chk(u, (B, H, T, dk), q.dtype, "u", cuda=False)
+    _chk(q, tok(dk), q.dtype, "q", cuda=False); _chk(k, tok(dk), q.dtype, "k", cuda=False)
+    _chk(v, tok(dv), q.dtype, "v", cuda=False); _chk(u, tok(dk), q.dtype, "u", cuda=False)
     _chk(S0, (B, H, dv, dk), f32, "S0", cuda=False); _chk(A0, (B, H, dk, dk), f32, "A0", cuda=False)
     _chk(z0, (B, H, dk), f32, "z0", cuda=False)
     pin = torch.cuda.is_available()
     mk = lambda shape: torch.empty(shape, dtype=f32, pin_memory=pin)
-    out = mk((B, H, T, dv)) if out is None else out
+    out = mk(tok(dv)) if out is None else out
     S_T = mk((B, H, dv, dk)) if S_T is None else S_T
     A_T = mk((B, H, dk, dk)) if A_T is None else A_T
     z_T = mk((B, H, dk)) if z_T is None else z_T
-    _chk(out, (B, H, T, dv), f32, "out", cuda=False); _chk(S_T, (B, H, dv, dk), f32, "S_T", cuda=False)
+    _chk(out, tok(dv), f32, "out", cuda=False); _chk(S_T, (B, H, dv, dk), f32, "S_T", cuda=False)
     _chk(A_T, (B, H, dk, dk), f32, "A_T", cuda=False); _chk(z_T, (B, H, dk), f32, "z_T", cuda=False)
     if not workspace.is_cuda or workspace.dtype != torch.uint8 or not workspace.is_contiguous():
         raise ValueError("workspace must be a contiguous CUDA uint8 tensor")
@@ -445,21 +476,26 @@ def vla_forward_host_static(q, k, v, lam: float, *, u=None, S0=None, A0=None, z0
     allocate).  Problems whose staging need exceeds the array raise ``VLA_ERR_TOO_LARGE``.
     Calls on one device share the array: do not let two of them overlap on the GPU."""
     lib = load_library()
-    B, H, T, dk = q.shape
+    if flags & VLA_FLAG_TOKEN_MAJOR:          # q, k, v, u, out are [B,T,H,d]
+        B, T, H, dk = q.shape
+        tok = lambda d_: (B, T, H, d_)
+    else:
+        B, H, T, dk = q.shape
+        tok = lambda d_: (B, H, T, d_)
     dv = v.shape[-1]
     dt = _dtype_code(q)
     f32 = torch.float32
-    _chk(q, (B, H, T, dk), q.dtype, "q", cuda=False); _chk(k, (B, H, T, dk), q.dtype, "k", cuda=False)
-    _chk(v, (B, H, T, dv), q.dtype, "v", cuda=False); _chk(u, (B, H, T, dk), q.dtype, "u", cuda=False)
+    _chk(q, tok(dk), q.dtype, "q", cuda=False); _chk(k, tok(dk), q.dtype, "k", cuda=False)
+    _chk(v, tok(dv), q.dtype, "v", cuda=False); _chk(u, tok(dk), q.dtype, "u", cuda=False)
     _chk(S0, (B, H, dv, dk), f32, "S0", cuda=False); _chk(A0, (B, H, dk, dk), f32, "A0", cuda=False)
     _chk(z0, (B, H, dk), f32, "z0", cuda=False)
     pin = torch.cuda.is_available()
     mk = lambda shape: torch.empty(shape, dtype=f32, pin_memory=pin)
-    out = mk((B, H, T, dv)) if out is None else out
+    out = mk(tok(dv)) if out is None else out
     S_T = mk((B, H, dv, dk)) if S_T is None else S_T
     A_T = mk((B, H, dk, dk)) if A_T is None else A_T
     z_T = mk((B, H, dk)) if z_T is None else z_T
-    _chk(out, (B, H, T, dv), f32, "out", cuda=False); _chk(S_T, (B, H, dv, dk), f32, "S_T", cuda=False)
+    _chk(out, tok(dv), f32, "out", cuda=False); _chk(S_T, (B, H, dv, dk), f32, "S_T", cuda=False)
     _chk(A_T, (B, H, dk, dk), f32, "A_T", cuda=False); _chk(z_T, (B, H, dk), f32, "z_T", cuda=False)
     dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
     st = stream if stream is not None else torch.cuda.current_stream(dev)

@@ -1,6 +1,12 @@
 // C ABI of the VLA forward scan (declared in include/vla.h): host-side validation,
-// kernel selection and launch.  No allocation, no synchronisation, no global state.
+// kernel selection and launch.  No allocation and no synchronisation on the device-pointer
+// calls.  Process-wide state kept here: the launch counter and the per-slot events of the
+// balanced schedule's hand-off flags, the device address of the built-in staging buffer of
+// vla_forward_host_static, and a per-thread note of the last launch (vla_last_launch).
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
+
+#include <cstdio>
 
 #include <atomic>
 #include <cstdint>
@@ -15,6 +21,14 @@
 namespace {
 
 using vla::ScanParams;
+
+// NVTX range around the host side of an entry point (a profiler shows the launches inside it).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
+
+constexpr int kMaxDevices = 64;
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -33,7 +47,7 @@ int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
   if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE | VLA_FLAG_TOKEN_MAJOR))
     return VLA_ERR_INVALID_ARG;
   if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN && r->kernel != VLA_KERNEL_CHUNK &&
-      r->kernel != VLA_KERNEL_DECODE)
+      r->kernel != VLA_KERNEL_DECODE && r->kernel != VLA_KERNEL_CHUNK_TC)
     return VLA_ERR_INVALID_ARG;
   if (r->refresh_period > 0 && (r->step_offset < 0 || !(r->refresh_eta == r->refresh_eta)))
     return VLA_ERR_INVALID_ARG;
@@ -63,7 +77,14 @@ bool decode_covers(const ScanParams& p, int d) {
   return p.T == 1 && d >= 32 && p.S0 && p.A0 && p.S_T && p.A_T && !p.u && p.refresh_period <= 0;
 }
 
+// The tensor-core form of the chunk kernel: d = 128, u = k_hat, no refresh, head-major tensors.
+bool chunk_tc_covers(const ScanParams& p, int d) {
+  return d == 128 && !p.u && p.refresh_period <= 0 && !(p.flags & VLA_FLAG_TOKEN_MAJOR) && p.T > 0;
+}
+
 int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
+  if (kernel == VLA_KERNEL_CHUNK_TC)
+    return chunk_tc_covers(p, d) ? vla::launch_chunk_tc(d, dtype, p, st) : VLA_ERR_UNSUPPORTED;
   if (kernel == VLA_KERNEL_DECODE && !decode_covers(p, d)) return VLA_ERR_UNSUPPORTED;
   if ((kernel == VLA_KERNEL_DECODE || kernel == VLA_KERNEL_AUTO) && decode_covers(p, d))
     return vla::launch_decode(d, dtype, p, st);
@@ -95,27 +116,35 @@ inline size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 // cudaGetSymbolAddress, once per device, with that device current.
 static __device__ __align__(256) unsigned char g_static_scratch[VLA_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_scratch_mutex;
 void* g_scratch_addr[kMaxDevices] = {};   // per device, filled on the first call there
 
-// Device address of the built-in buffer on the current device (nullptr on failure).
-void* static_scratch_for_current_device() {
+// Device address of the built-in buffer on the current device.  VLA_OK and *out set, or
+// VLA_ERR_INVALID_ARG when the address is not known yet and `st` is being captured into a graph
+// (the one-time look-up must not happen inside a capture), or VLA_ERR_CUDA.
+int static_scratch_for_current_device(cudaStream_t st, void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
     cudaGetLastError();
-    return nullptr;
+    return VLA_ERR_CUDA;
   }
   std::lock_guard<std::mutex> lock(g_scratch_mutex);
   if (!g_scratch_addr[dev]) {
+    cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &capture) != cudaSuccess) {
+      cudaGetLastError();
+      return VLA_ERR_CUDA;
+    }
+    if (capture != cudaStreamCaptureStatusNone) return VLA_ERR_INVALID_ARG;
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
       cudaGetLastError();
-      return nullptr;
+      return VLA_ERR_CUDA;
     }
     g_scratch_addr[dev] = ptr;
   }
-  return g_scratch_addr[dev];
+  *out = g_scratch_addr[dev];
+  return VLA_OK;
 }
 
 // ---- sequence-parallel entry point: workspace layout and segment choice
@@ -159,6 +188,15 @@ int seqpar_choose_segments(int units, int T, int d, int dtype) {
   return best;
 }
 
+// One event per (device, flag slot) of the balanced schedule, recorded behind the launch that
+// used the slot last.  Created on first use; they live until the process exits.
+constexpr int kSlotCount = 16;   // == kSchedSlots of the chunk kernel
+std::mutex g_slot_mutex;
+cudaEvent_t g_slot_event[kMaxDevices][kSlotCount] = {};
+
+struct LaunchNote { char kernel[48]; int d, dtype, grid, balanced; };
+thread_local LaunchNote g_last_launch = {"", 0, 0, 0, 0};
+
 }  // namespace
 
 namespace vla {
@@ -167,6 +205,44 @@ unsigned int next_launch_epoch() {
   if (e == 0) e = ++g_launch_epoch;   // 0 is the flags' initial value
   return e;
 }
+
+bool sched_slot_free(unsigned int epoch) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return false;
+  }
+  std::lock_guard<std::mutex> lock(g_slot_mutex);
+  cudaEvent_t& ev = g_slot_event[dev][epoch % kSlotCount];
+  if (!ev) {
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      ev = nullptr;
+      return false;
+    }
+    return true;   // never used
+  }
+  const cudaError_t q = cudaEventQuery(ev);
+  if (q == cudaSuccess) return true;
+  cudaGetLastError();   // cudaErrorNotReady (or a failure): treat the slot as busy
+  return false;
+}
+
+void sched_slot_mark(unsigned int epoch, cudaStream_t st) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    cudaGetLastError();
+    return;
+  }
+  std::lock_guard<std::mutex> lock(g_slot_mutex);
+  cudaEvent_t ev = g_slot_event[dev][epoch % kSlotCount];
+  if (ev && cudaEventRecord(ev, st) != cudaSuccess) cudaGetLastError();
+}
+
+void note_launch(const char* kernel, int d, int dtype, int grid, int balanced) {
+  std::snprintf(g_last_launch.kernel, sizeof(g_last_launch.kernel), "%s", kernel);
+  g_last_launch.d = d; g_last_launch.dtype = dtype; g_last_launch.grid = grid; g_last_launch.balanced = balanced;
+}
 }  // namespace vla
 
 extern "C" {
@@ -174,6 +250,7 @@ extern "C" {
 int vla_forward(const void* q, const void* k, const void* v, float lambda_, int B, int H, int T,
                 int d_k, int d_v, const float* S0, const float* A0, float* out, float* S_T,
                 float* A_T, const vla_opts_t* opts, void* stream) {
+  NvtxRange nvtx_range("vla_forward");
   vla_opts_t o;
   int rc = resolve_opts(opts, &o);
   if (rc != VLA_OK) return rc;
@@ -207,6 +284,7 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
   p.n_main = 0; p.out2 = nullptr;
   p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr; p.stash_zk = nullptr; p.stash_a = nullptr;
   p.heads = H;
+  p.wait_limit = o.wait_probe_limit;
   return launch(p, d_k, o.qkv_dtype, o.kernel, static_cast<cudaStream_t>(stream));
 }
 
@@ -226,6 +304,7 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
                      int T, int d_k, int d_v, const float* S0, const float* A0, float* out,
                      float* S_T, float* A_T, const vla_opts_t* opts, void* workspace,
                      size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("vla_forward_host");
   vla_opts_t o;
   int rc = resolve_opts(opts, &o);
   if (rc != VLA_OK) return rc;
@@ -295,10 +374,16 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
     }
   }
 
+  // [B,T,H,d] tensors: a slice is a range of batch indices (contiguous in that layout, and its
+  // units b*H .. are contiguous in the [B,H,...] states), scanned as a batch of its own
+  const bool token_major = (o.flags & VLA_FLAG_TOKEN_MAJOR) != 0;
+  if (token_major && nslices > B) nslices = B;
   bool bad = false;
   int rc_scan = VLA_OK;
   for (int sl = 0; sl < nslices; ++sl) {
-    const size_t u0 = units * sl / nslices, u1 = units * (sl + 1) / nslices, nu = u1 - u0;
+    const size_t u0 = token_major ? size_t(size_t(B) * sl / nslices) * H : units * sl / nslices;
+    const size_t u1 = token_major ? size_t(size_t(B) * (sl + 1) / nslices) * H : units * (sl + 1) / nslices;
+    const size_t nu = u1 - u0;
     cudaStream_t ls = lanes[sl % kLanes];
     auto h2d = [&](void* d, const void* h, size_t per_unit) {
       const size_t off = u0 * per_unit, bytes = nu * per_unit;
@@ -325,11 +410,14 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
     if (bad) break;
 
     vla_opts_t od = o;
+    od.workspace = nullptr;        // the slices run concurrently: they must not share scratch
+    od.workspace_bytes = 0;
     od.u = at(du, qk_u);
     od.z0 = o.z0 ? static_cast<const float*>(at(dz0, z_u)) : nullptr;
     od.zT = static_cast<float*>(at(dzT, z_u));   // device copies of the final states are always
                                                  // kept: they let the scan cut units across CTAs
-    rc_scan = vla_forward(at(dq, qk_u), at(dk, qk_u), at(dv, v_u), lambda_, 1, int(nu), T, d_k, d_v,
+    rc_scan = vla_forward(at(dq, qk_u), at(dk, qk_u), at(dv, v_u), lambda_,
+                          token_major ? int(nu / size_t(H)) : 1, token_major ? H : int(nu), T, d_k, d_v,
                           S0 ? static_cast<const float*>(at(dS0, S_u)) : nullptr,
                           A0 ? static_cast<const float*>(at(dA0, A_u)) : nullptr,
                           static_cast<float*>(at(dout, o_u)), static_cast<float*>(at(dST, S_u)),
@@ -361,6 +449,7 @@ int vla_forward_host_static(const void* q, const void* k, const void* v, float l
                             int H, int T, int d_k, int d_v, const float* S0, const float* A0,
                             float* out, float* S_T, float* A_T, const vla_opts_t* opts,
                             void* stream) {
+  NvtxRange nvtx_range("vla_forward_host_static");
   // Size check first: it needs no CUDA call and gives the clearest answer.
   vla_opts_t o;
   int rc = resolve_opts(opts, &o);
@@ -369,8 +458,9 @@ int vla_forward_host_static(const void* q, const void* k, const void* v, float l
   if (rc != VLA_OK) return rc;
   const size_t need = vla_host_workspace_bytes(B, H, T, d_k, d_v, o.qkv_dtype, o.u != nullptr);
   if (need > size_t(VLA_STATIC_SCRATCH_BYTES)) return VLA_ERR_TOO_LARGE;
-  void* scratch = static_scratch_for_current_device();
-  if (!scratch) return VLA_ERR_CUDA;
+  void* scratch = nullptr;
+  rc = static_scratch_for_current_device(static_cast<cudaStream_t>(stream), &scratch);
+  if (rc != VLA_OK) return rc;
   // Every staging region is written (by a copy or by the scan) before it is read, so
   // nothing left behind by the previous call needs clearing.
   return vla_forward_host(q, k, v, lambda_, B, H, T, d_k, d_v, S0, A0, out, S_T, A_T, opts, scratch,
@@ -395,6 +485,7 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
                        float* S_T, float* A_T,
                        const vla_opts_t* opts, int segments, void* workspace,
                        size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("vla_forward_seqpar");
   vla_opts_t o;
   int rc = resolve_opts(opts, &o);
   if (rc != VLA_OK) return rc;
@@ -448,6 +539,7 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   p.refresh_period = 0; p.refresh_eta = 0.0f; p.step_offset = 0; p.u_is_khat = 0;
   p.stash_z = nullptr; p.stash_e = nullptr; p.stash_delta = nullptr; p.stash_zk = nullptr; p.stash_a = nullptr;
   p.heads = H;
+  p.wait_limit = o.wait_probe_limit;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = vla::seqpar_before_scan(d_k, o.qkv_dtype, sp, st);
   if (rc != VLA_OK) return rc;
@@ -474,6 +566,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
                  const float* dS_T, const float* dA_T, const float* dz_T, float* dq, float* dk,
                  float* dv, float* dS0, float* dA0, float* dz0, const vla_opts_t* opts,
                  void* workspace, size_t workspace_bytes, void* stream) {
+  NvtxRange nvtx_range("vla_backward");
   vla_opts_t o;
   int rc = resolve_opts(opts, &o);
   if (rc != VLA_OK) return rc;
@@ -533,6 +626,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   f.n_main = 0; f.out2 = nullptr;
   f.stash_z = zst; f.stash_e = est; f.stash_delta = dst; f.stash_zk = zkcw; f.stash_a = general ? astw : nullptr;
   f.heads = H;
+  f.wait_limit = o.wait_probe_limit;
   rc = vla::launch_chunk_stash(d_k, o.qkv_dtype, f, st);
   if (rc != VLA_OK) return rc;
   // 2. the S-side and A-side reverse scans
@@ -551,6 +645,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
 
 int vla_make_u(const void* k, const float* W_u, int B, int H, int T, int d_k, int k_dtype, int u_dtype,
                float scale, float eps, void* u, void* stream) {
+  NvtxRange nvtx_range("vla_make_u");
   if (B < 0 || H < 0 || T < 0) return VLA_ERR_INVALID_ARG;
   if ((k_dtype != VLA_F32 && k_dtype != VLA_BF16) || (u_dtype != VLA_F32 && u_dtype != VLA_BF16))
     return VLA_ERR_INVALID_ARG;
@@ -595,6 +690,24 @@ const char* vla_status_string(int status) {
   }
 }
 
-int vla_version(void) { return 100; }
+int vla_selftest_wait_timeout(uint32_t probe_limit, int32_t* status, void* stream) {
+  if (!status || probe_limit == 0) return VLA_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(status) & 3u) return VLA_ERR_ALIGNMENT;
+  return vla::launch_wait_selftest(probe_limit, status, static_cast<cudaStream_t>(stream));
+}
+
+int vla_last_launch(char* buf, size_t len) {
+  if (!buf || len == 0) return VLA_ERR_INVALID_ARG;
+  const LaunchNote& n = g_last_launch;
+  if (!n.kernel[0]) {
+    buf[0] = 0;
+    return VLA_OK;
+  }
+  std::snprintf(buf, len, "%s<%d,%s> grid=%d%s", n.kernel, n.d, n.dtype == VLA_BF16 ? "bf16" : "f32", n.grid,
+                n.balanced ? " balanced" : "");
+  return VLA_OK;
+}
+
+int vla_version(void) { return 200; }
 
 }  // extern "C"

@@ -53,9 +53,14 @@ int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
     const bool state_out = p.S_T && p.A_T && (p.zT || (p.flags & VLA_FLAG_IDENTITY_MAP));
     if (BAL && resident > 0 && p.units > resident && p.units % resident != 0 && p.T > 0 && state_out &&
         p.units <= kSchedMaxUnits && p.n_main <= 0) {
-      sp.balanced = 1;
-      sp.grid = resident;
-      sp.epoch = next_launch_epoch();
+      // the flag slot of this launch id must not still be in use by an earlier launch that may
+      // overlap this one on the device (another stream): then the plain grid runs instead
+      const unsigned int epoch = next_launch_epoch();
+      if (sched_slot_free(epoch)) {
+        sp.balanced = 1;
+        sp.grid = resident;
+        sp.epoch = epoch;
+      }
     }
   } else {
     cudaGetLastError();
@@ -67,8 +72,14 @@ int launch_chunk_um_tm(const ScanParams& p, cudaStream_t st) {
   } else {
     maps.unused = 0;
   }
-  if (sp.balanced) kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
-  else kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
+  if (sp.balanced) {
+    kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
+    sched_slot_mark(sp.epoch, st);
+  } else {
+    kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
+  }
+  note_launch(STASH ? "vla_scan_chunk_kernel(stash)" : "vla_scan_chunk_kernel", D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32,
+              sp.grid, sp.balanced);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
@@ -117,6 +128,7 @@ int launch_chunk_tri_um(const ScanParams& p, cudaStream_t st) {
   sp.grid = p.units;
   sp.epoch = 0;
   kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, EmptyMaps{0});
+  note_launch("vla_scan_chunk_kernel(three groups)", D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, p.units, 0);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

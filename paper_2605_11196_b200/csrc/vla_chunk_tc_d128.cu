@@ -1,0 +1,13 @@
+// Tensor-core chunk kernel, d = 128, fp32 and bf16 inputs.
+#include "vla.h"
+#include "vla_launch.h"
+#include "vla_scan_tc.cuh"
+
+namespace vla {
+
+int launch_chunk_tc(int d, int dtype, const ScanParams& p, cudaStream_t st) {
+  if (d != 128) return VLA_ERR_UNSUPPORTED;
+  return dtype == VLA_F32 ? launch_chunk_tc_t<float>(p, st) : launch_chunk_tc_t<uint16_t>(p, st);
+}
+
+}  // namespace vla

@@ -49,6 +49,9 @@ struct ScanParams {
   // Token-major tensors (VLA_FLAG_TOKEN_MAJOR): q, k, v, u, out are [B, T, heads, D] instead of
   // [B, heads, T, D]; unit = b * heads + h.  The states keep their [units, D, D] layout.
   int heads;
+  // Failed probes after which a device-side wait gives up and reports VLA_ERR_DEVICE_TIMEOUT
+  // (0: the library's default, kWaitProbeLimit).
+  uint32_t wait_limit = 0;
 #ifdef VLA_SECTION_TIMERS
   long long* dbg;      // debug builds only: per-section clock64 totals of unit 0
 #endif
@@ -95,8 +98,9 @@ constexpr uint32_t kWaitProbeLimit = 1u << 22;
 
 // Returns false when the limit ran out (the caller reports VLA_ERR_DEVICE_TIMEOUT and
 // leaves through the common exit so that no thread is left at a CTA barrier).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kWaitProbeLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
+                                                  uint32_t limit = kWaitProbeLimit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
   }
   return false;
@@ -222,6 +226,66 @@ __device__ __forceinline__ float4 load4(const uint16_t* row, int c4) {
   f.z = bf16_bits_to_f32(r.y & 0xffffu);
   f.w = bf16_bits_to_f32(r.y >> 16);
   return f;
+}
+
+// ---------------------------------------------------------------- helpers of the chunk kernels
+// ---- packed fp32x2 arithmetic (one instruction, two FMAs on the fp32 pipe)
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+  unsigned long long ra, rb, rc, rd;
+  ra = *reinterpret_cast<unsigned long long*>(&a);
+  rb = *reinterpret_cast<unsigned long long*>(&b);
+  rc = *reinterpret_cast<unsigned long long*>(&c);
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+  return *reinterpret_cast<float2*>(&rd);
+}
+
+__device__ __forceinline__ void group_bar(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Fast elementwise helpers of the prep pass (relative error ~1e-6, far inside the parity bound).
+// Branch-free: both sides are evaluated and selected, so a warp never diverges here.
+__device__ __forceinline__ float phi_fast(float x) {
+  const float xm = x > 0.0f ? 0.0f : x;   // keeps a NaN (fminf would drop it)
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(xm * 1.4426950408889634f));
+  return x > 0.0f ? x + 1.0f : e;
+}
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float r;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float r;
+  asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+// 1/x to within an ulp or so: hardware estimate plus one Newton step
+__device__ __forceinline__ float rcp_nr(float x) {
+  const float r = rcp_approx(x);
+  return fmaf(r, fmaf(-x, r, 1.0f), r);
+}
+
+// Reduce-scatter of 16 values over a full warp: lanes 2t and 2t+1 end with the sum of v[t].
+__device__ __forceinline__ float warp_reduce_scatter16(float (&v)[16], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 2; off >>= 1) {
+    const int n = off / 2;  // values kept after this step
+    const bool up = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < n; ++i) {
+      const float send = up ? v[i] : v[i + n];
+      const float keep = up ? v[i + n] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+  v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
+  return v[0];  // token index = lane >> 1
 }
 
 }  // namespace vla

@@ -69,6 +69,7 @@ int launch_token_t(const ScanParams& p, cudaStream_t st) {
     return VLA_ERR_CUDA;
   }
   kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  note_launch("vla_scan_token_kernel", D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, p.units, 0);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
@@ -292,6 +293,7 @@ int launch_decode_t(const ScanParams& p, cudaStream_t st) {
   }
   const int grid = p.units < sms * per_sm ? p.units : sms * per_sm;   // persistent CTAs
   kern<<<grid, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  note_launch("vla_decode_kernel", D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, grid, 0);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
@@ -373,6 +375,32 @@ int seqpar_after_scan(int d, const SeqParParams& sp, float* A_T, float* zT, cons
     case 128: return seqpar_after_d<128>(sp, A_T, zT, AT2, zT2, st);
     default: return VLA_ERR_UNSUPPORTED;
   }
+}
+
+// ---------------------------------------------------------------- the bounded wait, tested
+// One warp waits, with the kernels' own mbar_wait_bounded, on a barrier that expects two
+// arrivals and gets one: the wait can only end by running out of probes.  The kernel then does
+// what the scan kernels do: it records VLA_ERR_DEVICE_TIMEOUT in the caller's status word and
+// returns normally (no trap, the context stays usable).
+namespace {
+__global__ void wait_selftest_kernel(unsigned int probe_limit, int* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 2);
+    mbar_init_fence();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_arrive(&bar);      // one of the two arrivals; the other never comes
+  __syncthreads();
+  if (!mbar_wait_bounded(&bar, 0, probe_limit) && threadIdx.x == 0)
+    atomicCAS(status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
+}
+}  // namespace
+
+int launch_wait_selftest(unsigned int probe_limit, int* status, cudaStream_t st) {
+  wait_selftest_kernel<<<1, 32, 0, st>>>(probe_limit, status);
+  note_launch("wait_selftest_kernel", 0, VLA_F32, 1, 0);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 
 }  // namespace vla

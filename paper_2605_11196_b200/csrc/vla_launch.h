@@ -25,6 +25,9 @@ int launch_decode(int d, int dtype, const ScanParams& p, cudaStream_t st);
 // Chunk kernel, d in {32, 64, 128}: plain or balanced grid, chosen from the shape.
 int launch_chunk(int d, int dtype, const ScanParams& p, cudaStream_t st);
 
+// Tensor-core form of the chunk kernel: d = 128, u = k_hat, no refresh, [B,H,T,d] tensors.
+int launch_chunk_tc(int d, int dtype, const ScanParams& p, cudaStream_t st);
+
 // Chunk kernel as the forward of a backward pass: leaves z_t, e_t, delta_t per token (p.stash_*).
 int launch_chunk_stash(int d, int dtype, const ScanParams& p, cudaStream_t st);
 
@@ -54,5 +57,18 @@ int launch_fp32_probe(int iters, float* sink, double* flops, cudaStream_t st);
 // Launch ids for the balanced schedule's hand-off flags (never 0, never repeated within
 // 2^32 launches).
 unsigned int next_launch_epoch();
+
+// The hand-off flags of a balanced launch live in one of kSchedSlots slots (launch id modulo the
+// slot count).  A slot may be taken again only once the launch that used it last has finished:
+// sched_slot_free() asks the event recorded behind that launch, sched_slot_mark() records it.
+// A launch that finds its slot busy runs on the plain grid instead (no flags needed).
+bool sched_slot_free(unsigned int epoch);
+void sched_slot_mark(unsigned int epoch, cudaStream_t st);
+
+// What the calling thread launched last (read back by vla_last_launch).
+void note_launch(const char* kernel, int d, int dtype, int grid, int balanced);
+
+// Test kernel of the bounded wait: a barrier that never completes.
+int launch_wait_selftest(unsigned int probe_limit, int* status, cudaStream_t st);
 
 }  // namespace vla

@@ -39,48 +39,6 @@
 
 namespace vla {
 
-// ---- packed fp32x2 arithmetic (one instruction, two FMAs on the fp32 pipe)
-__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
-  unsigned long long ra, rb, rc, rd;
-  ra = *reinterpret_cast<unsigned long long*>(&a);
-  rb = *reinterpret_cast<unsigned long long*>(&b);
-  rc = *reinterpret_cast<unsigned long long*>(&c);
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
-  return *reinterpret_cast<float2*>(&rd);
-}
-
-__device__ __forceinline__ void group_bar(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// Fast elementwise helpers of the prep pass (relative error ~1e-6, far inside the parity bound).
-// Branch-free: both sides are evaluated and selected, so a warp never diverges here.
-__device__ __forceinline__ float phi_fast(float x) {
-  const float xm = x > 0.0f ? 0.0f : x;   // keeps a NaN (fminf would drop it)
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(xm * 1.4426950408889634f));
-  return x > 0.0f ? x + 1.0f : e;
-}
-__device__ __forceinline__ float sqrt_approx(float x) {
-  float r;
-  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
-}
-__device__ __forceinline__ float rcp_approx(float x) {
-  float r;
-  asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
-}
-// 1/x to within an ulp or so: hardware estimate plus one Newton step
-__device__ __forceinline__ float rcp_nr(float x) {
-  const float r = rcp_approx(x);
-  return fmaf(r, fmaf(-x, r, 1.0f), r);
-}
-
 template <int D>
 struct ChunkTile {
   static constexpr int TW = (D >= 64) ? 16 : 8;  // state columns per thread
@@ -152,23 +110,6 @@ __device__ __forceinline__ void reduce_scatter(float (&v)[NTOK][LPR], int cg) {
         v[k][i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
       }
   }
-}
-
-// Reduce-scatter of 16 values over a full warp: lanes 2t and 2t+1 end with the sum of v[t].
-__device__ __forceinline__ float warp_reduce_scatter16(float (&v)[16], int lane) {
-#pragma unroll
-  for (int off = 16; off >= 2; off >>= 1) {
-    const int n = off / 2;  // values kept after this step
-    const bool up = (lane & off) != 0;
-#pragma unroll
-    for (int i = 0; i < n; ++i) {
-      const float send = up ? v[i] : v[i + n];
-      const float keep = up ? v[i + n] : v[i];
-      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-    }
-  }
-  v[0] += __shfl_xor_sync(0xffffffffu, v[0], 1);
-  return v[0];  // token index = lane >> 1
 }
 
 // For every token t of the chunk: sink(t, row g of (state tile) . op[t]).  Two tokens per
@@ -444,9 +385,10 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   unsigned int* sched_flags = g_sched_flags + size_t(sp.epoch % kSchedSlots) * kSchedMaxUnits;
 
   // Bounded wait shared by every mbarrier in this kernel.
+  const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitProbeLimit;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (*abort_flag) return;
-    if (!mbar_wait_bounded(bar, parity)) {
+    if (!mbar_wait_bounded(bar, parity, wait_limit)) {
       *abort_flag = 1;
       if (p.status) atomicCAS(p.status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
     }
@@ -526,7 +468,8 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
     mbar_init_fence();
     if (from_handoff && !*abort_flag) {
       bool seen = false;
-      for (uint32_t it = 0; it < (1u << 24) && !seen; ++it) {
+      // four times the probes of a barrier wait: a probe here is one acquire load and a short sleep
+      for (uint64_t it = 0; it < 4ull * wait_limit && !seen; ++it) {
         seen = ld_acquire_gpu(&sched_flags[unit]) == sp.epoch;
         if (!seen) __nanosleep(64);
       }

@@ -1,0 +1,810 @@
+// VLA forward scan, tensor-core form of the chunk kernel (d = 128, u = k_hat, no refresh).
+//
+// The 16-token chunk algebra of vla_scan_chunk.cuh (Section 3.3's recurrence in its exact
+// Woodbury / LDL^T form; Section 3.4's observation that the chunked recurrence is a chain of
+// dense products) with the d x d work on the 5th-generation tensor cores:
+//
+//   * both states live in tensor memory as fp32 accumulators (A: columns 0..127, S: 128..255,
+//     lane = row), so a rank-16 update  A -= Z diag(1/delta) Z^T,  S += E' Z^T  is a handful
+//     of tcgen05.mma instructions that accumulate straight into the state;
+//   * the chunk products  Z0 = A K^T,  P = S K^T,  R0 = S Q^T  take the state as the
+//     tensor-memory operand of the MMA;
+//   * fp32 accuracy out of TF32 products: every operand x is used as hi(x) + lo(x), hi = the
+//     upper 19 bits (what the tensor core reads of a 32-bit word), lo = x - hi (exact), and a
+//     product is hi*hi + hi*lo + lo*hi (the dropped lo*lo term is ~2^-22 relative).  For the
+//     state the lo part is recomputed once per chunk from tensor memory into a scratch region
+//     of 128 columns that the two states take turns in;
+//   * the 16 x 16 factorisation, the two row substitutions, the Gram matrices and the input
+//     prep stay on the fp32 pipe, as in the FMA kernel.
+//
+// One CTA per unit, 12 warps: group A (warps 0-3) owns the A chain, group S (warps 4-7) the
+// S chain and the readout, group P (warps 8-9) the TMA ring and the input prep; lane 0 of
+// warps 10 and 11 issues the MMAs of group A and of group S.  Thread g of
+// groups A and S owns row g of its state (tensor-memory lane g).  Every mbarrier wait is
+// bounded; on expiry the CTA records VLA_ERR_DEVICE_TIMEOUT, stops waiting, frees its tensor
+// memory and runs to its end.
+//
+// Operand layouts in shared memory (K-major, no swizzle, 8 x 16-byte core matrices): an
+// operand with R rows and K columns is the float4 array [K/4][R], i.e. element (r, k) at
+// float4 index (k/4) * R + r, component k%4.  Descriptor: stride (8-row groups) 128 B,
+// leading (next 4 k) 16*R B; one MMA (K = 8) advances the start address by 32*R B.
+#pragma once
+
+#include "vla_common.cuh"
+#include "vla_launch.h"
+
+namespace vla {
+
+// ---------------------------------------------------------------- tcgen05 wrappers
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lead_bytes, uint32_t stride_bytes) {
+  return uint64_t((saddr & 0x3FFFFu) >> 4) | (uint64_t(lead_bytes >> 4) << 16) |
+         (uint64_t(stride_bytes >> 4) << 32) | (1ull << 46);
+}
+// kind::tf32, fp32 accumulate, both operands K-major, M x N
+__host__ __device__ constexpr uint32_t umma_idesc_tf32(int M, int N) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] B[smem]^T
+__device__ __forceinline__ void umma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n" ::"r"(d),
+      "l"(a), "l"(b), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] B[smem]^T
+__device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d),
+      "r"(a), "l"(b), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// the barrier receives one arrival once every MMA this thread has issued so far is complete
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 consecutive columns of this thread's lane (no wait)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Splitting an fp32 value for TF32 products.  The tensor core reads the upper 19 bits of a
+// 32-bit word (it truncates).  Operands written by threads are split around the NEAREST TF32
+// value, x = hi + lo with hi = rn_tf32(x) and lo = rn_tf32(x - hi), so that lo has either sign
+// and the dropped lo*lo products do not add up; the state, which the tensor core reads in
+// place, is split as it reads it: hi = the truncated word, lo = rn_tf32(x - hi).
+__device__ __forceinline__ float tf32_trunc(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+__device__ __forceinline__ float tf32_rn(float x) { return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u); }
+__device__ __forceinline__ float tf32_state_lo(float x) { return tf32_rn(x - tf32_trunc(x)); }
+__device__ __forceinline__ void tf32_split4(float4 x, float4& hi, float4& lo) {
+  hi = make_float4(tf32_rn(x.x), tf32_rn(x.y), tf32_rn(x.z), tf32_rn(x.w));
+  lo = make_float4(tf32_rn(x.x - hi.x), tf32_rn(x.y - hi.y), tf32_rn(x.z - hi.z), tf32_rn(x.w - hi.w));
+}
+__device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
+// ---------------------------------------------------------------- configuration
+template <typename TIn>
+struct TcCfg {
+  static constexpr int D = 128;
+  static constexpr int C = 16;                  // tokens per chunk
+  static constexpr int NG = 128;                // threads of group A and of group S
+  static constexpr int NP = 64;                 // threads of the prep group
+  static constexpr int NI = 64;                 // two warps whose lane 0 issues the MMAs of group A / group S
+  static constexpr int NT = 2 * NG + NP + NI;
+  static constexpr int NSTAGE = sizeof(TIn) == 2 ? 2 : 1;   // raw q/k/v chunks in flight
+  static constexpr int KRING = 2;               // widened chunks (prep -> A, S)
+  static constexpr int RING = 1;                // Z / Gu / HT / sc slots (A -> S)
+  static constexpr int CP = C + 4;              // padded row of the small C x C matrices
+  static constexpr int VP = D + 4;              // padded row of the widened k_hat, q_f, v chunks
+  // tensor-memory columns
+  static constexpr uint32_t COL_A = 0, COL_S = 128, COL_LO = 256, COL_Z0 = 384, COL_PR = 432;   // 48, 64
+  static constexpr uint32_t TMEM_COLS = 512;
+  // shared memory (bytes)
+  static constexpr size_t raw_bytes = size_t(NSTAGE) * 3 * C * D * sizeof(TIn);
+  static constexpr int KQR = 64;                // operand rows of a chunk: hi(k_hat) | hi(q_f) | lo(k_hat) | lo(q_f)
+  static constexpr size_t kq_bytes = size_t(KQR) * D * 4;           // [32][64] float4
+  static constexpr size_t kp_bytes = size_t(2) * C * VP * 4;        // k_hat, q_f as plain fp32 rows [C][VP]
+  static constexpr size_t kslot_bytes = kq_bytes + kp_bytes + size_t(C) * VP * 4 + 2 * C * 4;   // + v, nrm, 1/den
+  static constexpr size_t op16_bytes = size_t(D) * C * 4;           // [4][128] float4: a 128 x 16 operand
+  static constexpr size_t zslot_bytes = 2 * op16_bytes + (2 * C * CP + C) * 4;      // Z, lo(Z), GuT, HT, sc
+  static constexpr size_t a_bytes = 2 * op16_bytes + size_t(C) * D * 4 + (2 * C * CP + 4 * C + 3 * C) * 4;
+  //   -Z/delta, lo | Z0 / Z rows [C][D] | W, L | N2p[4][C] | delta, 1/delta, -1/delta
+  static constexpr size_t s_bytes = 2 * op16_bytes + 2 * size_t(C) * D * 4;         // E', lo(E') | out stage [2]
+  static constexpr size_t p_bytes = 2 * C * 4;                                      // denp[2][C]
+  static constexpr int NBAR = NSTAGE + 2 * KRING + 2 * RING + 9;
+  static constexpr size_t smem_bytes = raw_bytes + KRING * kslot_bytes + RING * zslot_bytes + a_bytes + s_bytes +
+                                       p_bytes + NBAR * 8 + 16 + 128;
+};
+
+// G[i][j] = X[i] . Y[j] for two sets of 16 plain rows of length 128 (row stride XS and 128); result
+// rows have stride CP.  4x4 output tiles, 8 threads per tile splitting the 128 index.
+template <int CP, int XS>
+__device__ __forceinline__ void gram16_tc(const float* X, const float* Y, float* G, int g) {
+  constexpr int P = 8;
+  const int tile = g / P, part = g % P;
+  const int i0 = (tile >> 2) * 4, j0 = (tile & 3) * 4;
+  float2 w2[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) w2[i] = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int step = 0; step < 4; ++step) {
+    const int f = step * P + part;
+    float4 a[4], b[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      a[i] = reinterpret_cast<const float4*>(X + (i0 + i) * XS)[f];
+      b[i] = reinterpret_cast<const float4*>(Y + (j0 + i) * 128)[f];
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        w2[4 * i + j] = ffma2(make_float2(a[i].x, a[i].y), make_float2(b[j].x, b[j].y), w2[4 * i + j]);
+        w2[4 * i + j] = ffma2(make_float2(a[i].z, a[i].w), make_float2(b[j].z, b[j].w), w2[4 * i + j]);
+      }
+  }
+  float w[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) w[i] = w2[i].x + w2[i].y;
+#pragma unroll
+  for (int off = P / 2; off >= 1; off >>= 1)
+#pragma unroll
+    for (int i = 0; i < 16; ++i) w[i] += __shfl_xor_sync(0xffffffffu, w[i], off);
+  if (part == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      *reinterpret_cast<float4*>(G + (i0 + i) * CP + j0) =
+          make_float4(w[4 * i + 0], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+  }
+}
+
+template <typename TIn>
+__global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const ScanParams p) {
+  using Cfg = TcCfg<TIn>;
+  constexpr int D = Cfg::D, C = Cfg::C, NG = Cfg::NG, NP = Cfg::NP, CP = Cfg::CP, VP = Cfg::VP;
+  constexpr int NSTAGE = Cfg::NSTAGE, KRING = Cfg::KRING, RING = Cfg::RING;
+
+  extern __shared__ __align__(128) unsigned char smem[];
+  TIn* raw = reinterpret_cast<TIn*>(smem);
+  unsigned char* kslots = smem + Cfg::raw_bytes;
+  unsigned char* zslots = kslots + KRING * Cfg::kslot_bytes;
+  unsigned char* abase = zslots + RING * Cfg::zslot_bytes;
+  unsigned char* sbase = abase + Cfg::a_bytes;
+  unsigned char* pbase = sbase + Cfg::s_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(pbase + Cfg::p_bytes) + 15) & ~uintptr_t(15));
+  uint64_t* raw_full = bars;                      // [NSTAGE] TMA filled a raw stage
+  uint64_t* k_full = raw_full + NSTAGE;           // [KRING] prep published a widened chunk
+  uint64_t* k_empty = k_full + KRING;             // [KRING] groups A and S are done with it
+  uint64_t* z_full = k_empty + KRING;             // [RING] group A published Z, Gu, HT, sc
+  uint64_t* z_empty = z_full + RING;              // [RING] both rank-16 updates have read Z
+  uint64_t* b_z0 = z_empty + RING;                // Z0 products complete
+  uint64_t* b_aupd = b_z0 + 1;                    // update of A complete
+  uint64_t* b_pr = b_aupd + 1;                    // P / R0 products complete
+  uint64_t* b_supd = b_pr + 1;                    // update of S complete
+  uint64_t* b_lo_s = b_supd + 1;                  // group A's products have read the lo scratch: S may fill it
+  uint64_t* b_lo_a = b_lo_s + 1;                  // group S's products have read the lo scratch: A may fill it
+  uint64_t* b_lo_rdy_a = b_lo_a + 1;              // group A has written the lo scratch
+  uint64_t* b_lo_rdy_s = b_lo_rdy_a + 1;          // group S has written the lo scratch
+  uint64_t* b_ep_rdy = b_lo_rdy_s + 1;            // group S has written E' and its lo part
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b_ep_rdy + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x;
+  const int grp = tid < NG ? 0 : (tid < 2 * NG ? 1 : (tid < 2 * NG + NP ? 2 : 3));   // A, S, prep, MMA issue
+  const int g = tid - (grp == 3 ? 2 * NG + NP : grp * NG);   // thread within its group
+  const int lane = tid & 31, gw = g >> 5;
+  const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
+  const float eps = p.eps;
+  const int unit = blockIdx.x;
+  const int T = p.T;
+  const int nchunks = (T + C - 1) / C;
+
+  const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitProbeLimit;
+  auto wait = [&](uint64_t* bar, uint32_t parity) {
+    if (*abort_flag) return;
+    if (!mbar_wait_bounded(bar, parity, wait_limit)) {
+      *abort_flag = 1;
+      if (p.status) atomicCAS(p.status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
+    }
+  };
+
+#ifdef VLA_SECTION_TIMERS
+  long long tsec[12];
+  for (int i = 0; i < 12; ++i) tsec[i] = 0;
+  long long tlast = clock64();
+#define VLA_MARK(i) { long long now_ = clock64(); tsec[i] += now_ - tlast; tlast = now_; }
+#else
+#define VLA_MARK(i)
+#endif
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < NSTAGE; ++s) mbar_init(&raw_full[s], 1);
+    for (int s = 0; s < KRING; ++s) { mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 2); }
+    for (int s = 0; s < RING; ++s) { mbar_init(&z_full[s], 1); mbar_init(&z_empty[s], 2); }
+    mbar_init(b_z0, 1); mbar_init(b_aupd, 1); mbar_init(b_pr, 1); mbar_init(b_supd, 1);
+    mbar_init(b_lo_s, 1); mbar_init(b_lo_a, 1);
+    mbar_init(b_lo_rdy_a, 1); mbar_init(b_lo_rdy_s, 1); mbar_init(b_ep_rdy, 1);
+    mbar_init_fence();
+  }
+  if (tid < 32) {   // warp 0 allocates the CTA's tensor memory (all 512 columns: one CTA per SM)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(Cfg::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tbase = *tmem_slot;
+  const uint32_t trow = tbase + (uint32_t((tid >> 5) & 3) << 21);   // this warp's 32 lanes: lane field = bits 16..
+
+  // one state row: global (or the initial value) -> tensor memory
+  auto state_in = [&](const float* src, float diag, uint32_t col) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      uint32_t r[32];
+      if (src) {
+        const float4* s4 = reinterpret_cast<const float4*>(src + (size_t(unit) * D + g) * D + c0);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float4 x = __ldg(s4 + i);
+          r[4 * i + 0] = __float_as_uint(x.x); r[4 * i + 1] = __float_as_uint(x.y);
+          r[4 * i + 2] = __float_as_uint(x.z); r[4 * i + 3] = __float_as_uint(x.w);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint((c0 + i == g) ? diag : 0.0f);
+      }
+      tmem_st32(trow + col + c0, r);
+    }
+    tmem_wait_st();
+  };
+  auto state_out = [&](float* dst, uint32_t col) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld32(trow + col + c0, r);
+      tmem_wait_ld();
+      float4* d4 = reinterpret_cast<float4*>(dst + (size_t(unit) * D + g) * D + c0);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        d4[i] = make_float4(__uint_as_float(r[4 * i + 0]), __uint_as_float(r[4 * i + 1]),
+                            __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+    }
+  };
+  // lo scratch <- state - hi(state), this thread's row
+  auto split_state = [&](uint32_t col) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld32(trow + col + c0, r);
+      tmem_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(tf32_state_lo(__uint_as_float(r[i])));
+      tmem_st32(trow + Cfg::COL_LO + c0, r);
+    }
+    tmem_wait_st();
+  };
+
+  if (grp == 0) {
+    // =====================================================================  group A
+    float* Zsf = reinterpret_cast<float*>(abase);            // [4][128] float4: -z_t / delta_t
+    float* Zsl = Zsf + D * C;                                // its lo part
+    float* Zp = Zsl + D * C;                                 // [C][D] rows: Z0, then Z
+    float* Ws = Zp + C * D;                                  // [C][CP] K A K^T
+    float* Ls = Ws + C * CP;                                 // [C][CP] unit lower factor
+    float* N2p = Ls + C * CP;                                // [4][C]
+    float* dlt = N2p + 4 * C;                                // [C]
+    float* idl = dlt + C;                                    // [C]  1/delta
+    float* nidl = idl + C;                                   // [C] -1/delta
+    state_in(p.A0, 1.0f / p.lambda, Cfg::COL_A);
+
+#pragma unroll 1
+    for (int c = 0; c < nchunks; ++c) {
+      const int ks = c % KRING, zs = c % RING;
+      unsigned char* kslot = kslots + size_t(ks) * Cfg::kslot_bytes;
+      const float* Kp = reinterpret_cast<const float*>(kslot + Cfg::kq_bytes);   // [C][VP] k_hat
+      const float* Qp = Kp + C * VP;                                             // [C][VP] q_f
+      unsigned char* zslot = zslots + size_t(zs) * Cfg::zslot_bytes;
+      float* Zf = reinterpret_cast<float*>(zslot);           // [4][128] float4: z_t
+      float* Zl = Zf + D * C;
+      float* GuT = Zl + D * C;                               // [C][CP]
+      float* HT = GuT + C * CP;                              // [C][CP]
+      float* scs = HT + C * CP;                              // [C]
+
+      VLA_MARK(8)
+      // A is final once the update of the previous chunk has completed
+      if (c > 0) wait(b_aupd, (c - 1) & 1);
+      VLA_MARK(0)
+      wait(&k_full[ks], (c / KRING) & 1);
+      // the lo scratch is free once group S's products of the previous chunk have read it
+      if (c > 0) wait(b_lo_a, (c - 1) & 1);
+      tc_fence_after();
+      VLA_MARK(9)
+      split_state(Cfg::COL_A);
+      tc_fence_before();
+      group_bar(1, NG);
+      if (g == 0) mbar_arrive(b_lo_rdy_a);
+      VLA_MARK(1)
+      wait(b_z0, c & 1);
+      tc_fence_after();
+      VLA_MARK(2)
+      float z[16];
+      {
+        uint32_t r0[16], r1[16];
+        tmem_ld16(trow + Cfg::COL_Z0, r0);
+        tmem_ld16(trow + Cfg::COL_Z0 + 32, r1);
+        tmem_wait_ld();
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          z[t] = __uint_as_float(r0[t]) + __uint_as_float(r1[t]);   // row g of Z0 = A K^T
+          Zp[t * D + g] = z[t];
+        }
+      }
+      tc_fence_before();
+      group_bar(1, NG);
+      VLA_MARK(3)
+
+      // ---- W = K Z0 (C x C, symmetric)
+      gram16_tc<CP, VP>(Kp, Zp, Ws, g);
+      group_bar(1, NG);
+      VLA_MARK(4)
+
+      // ---- warp 0: I + W = L diag(delta) L^T
+      if (gw == 0) {
+        const int r = lane & 15, h = lane >> 4;
+        float m[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m[j] = Ws[r * CP + h * 8 + j] + ((h * 8 + j == r) ? 1.0f : 0.0f);
+#pragma unroll
+        for (int s2 = 0; s2 < 16; ++s2) {
+          const int hs = s2 >> 3, js = s2 & 7;
+          const float piv = fmaxf(__shfl_sync(0xffffffffu, m[js], s2 + 16 * hs), eps);
+          const float mrs = __shfl_sync(0xffffffffu, m[js], r + 16 * hs);
+          const float ipiv = rcp_nr(piv);
+          const float l = (r > s2) ? mrs * ipiv : 0.0f;  // L[r][s2]
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float msj = __shfl_sync(0xffffffffu, m[j], s2 + 16 * h);
+            m[j] = fmaf(-l, msj, m[j]);
+          }
+          if (h == hs) Ls[r * CP + s2] = l;
+          if (lane == 0) { dlt[s2] = piv; idl[s2] = ipiv; nidl[s2] = -ipiv; }
+        }
+      }
+      group_bar(1, NG);
+      VLA_MARK(5)
+
+      // ---- row g of Z by forward substitution: z_t = z0_t - sum_{s<t} L[t][s] z_s
+#pragma unroll
+      for (int t = 1; t < 16; ++t) {
+        float a0 = z[t], a1 = 0.f;
+#pragma unroll
+        for (int s4 = 0; s4 * 4 < t; ++s4) {
+          const float4 l4 = reinterpret_cast<const float4*>(Ls + t * CP)[s4];
+          if (4 * s4 + 0 < t) a0 = fmaf(-l4.x, z[4 * s4 + 0], a0);
+          if (4 * s4 + 1 < t) a1 = fmaf(-l4.y, z[4 * s4 + 1], a1);
+          if (4 * s4 + 2 < t) a0 = fmaf(-l4.z, z[4 * s4 + 2], a0);
+          if (4 * s4 + 3 < t) a1 = fmaf(-l4.w, z[4 * s4 + 3], a1);
+        }
+        z[t] = a0 + a1;
+      }
+      // both rank-16 updates of chunk c - RING have read the Z slot
+      if (c >= RING) wait(&z_empty[zs], ((c / RING) + 1) & 1);
+      {
+        float sq[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          Zp[t * D + g] = z[t];
+          sq[t] = z[t] * z[t];
+        }
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) {
+          const float4 zz = make_float4(z[4 * k4], z[4 * k4 + 1], z[4 * k4 + 2], z[4 * k4 + 3]);
+          const float4 ni = *reinterpret_cast<const float4*>(nidl + 4 * k4);
+          const float4 zsc = make_float4(zz.x * ni.x, zz.y * ni.y, zz.z * ni.z, zz.w * ni.w);
+          float4 hi, lo;
+          tf32_split4(zz, hi, lo);
+          reinterpret_cast<float4*>(Zf)[k4 * 128 + g] = hi;
+          reinterpret_cast<float4*>(Zl)[k4 * 128 + g] = lo;
+          tf32_split4(zsc, hi, lo);
+          reinterpret_cast<float4*>(Zsf)[k4 * 128 + g] = hi;
+          reinterpret_cast<float4*>(Zsl)[k4 * 128 + g] = lo;
+        }
+        const float tot = warp_reduce_scatter16(sq, lane);
+        if ((lane & 1) == 0) N2p[gw * C + (lane >> 1)] = tot;
+      }
+      group_bar(1, NG);
+      VLA_MARK(6)
+
+      // ---- warp 0: sc_t and GuT[t][s] = Gu[s][t] = sc_s delta_s L[t][s]
+      if (gw == 0) {
+        const int r = lane & 15, h = lane >> 4;
+        const float n2 = N2p[r] + N2p[C + r] + N2p[2 * C + r] + N2p[3 * C + r];
+        const float id_r = idl[r], d_r = dlt[r];
+        // alpha_r = sc_r z_r, sc_r = (1/delta) / max(||z||/delta, eps)      (A_t k_hat_t = z_t / delta_t)
+        const float sc_r = id_r * rcp_nr(fmaxf(sqrt_approx(n2) * id_r, eps));
+        if ((p.flags & VLA_FLAG_CHECK_FINITE) && p.status && !isfinite(n2 + d_r))
+          atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
+        if (h == 0) scs[r] = sc_r;
+        const float scd = sc_r * d_r;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int s2 = h * 8 + j;
+          const float scd_s = __shfl_sync(0xffffffffu, scd, s2);
+          GuT[r * CP + s2] = (s2 < r) ? scd_s * Ls[r * CP + s2] : 0.0f;
+        }
+      }
+      // ---- HT[t][s] = q_t . z_s
+      gram16_tc<CP, VP>(Qp, Zp, HT, g);
+      fence_async_smem();     // Z, lo(Z), -Z/delta: written here, read by the tensor core
+      group_bar(1, NG);
+      if (g == 0) {
+        mbar_arrive(&z_full[zs]);    // group S and the issuing warp of the update of A
+        mbar_arrive(&k_empty[ks]);
+      }
+      VLA_MARK(7)
+    }
+    if (nchunks > 0) wait(b_aupd, (nchunks - 1) & 1);
+    tc_fence_after();
+    if (p.A_T) state_out(p.A_T, Cfg::COL_A);
+  } else if (grp == 1) {
+    // =====================================================================  group S
+    float* Epf = reinterpret_cast<float*>(sbase);            // [4][128] float4: e'_t
+    float* Epl = Epf + D * C;
+    float* ostage = Epl + D * C;                             // [2][C][D]
+    state_in(p.S0, 0.0f, Cfg::COL_S);
+
+#pragma unroll 1
+    for (int c = 0; c < nchunks; ++c) {
+      const int n = min(C, T - c * C);
+      const int ks = c % KRING, zs = c % RING;
+      unsigned char* kslot = kslots + size_t(ks) * Cfg::kslot_bytes;
+      const float* Vf = reinterpret_cast<const float*>(kslot + Cfg::kq_bytes + Cfg::kp_bytes);   // [C][VP]
+      const float* inv_den = Vf + C * VP + C;
+      unsigned char* zslot = zslots + size_t(zs) * Cfg::zslot_bytes;
+      const float* GuT = reinterpret_cast<const float*>(zslot) + 2 * D * C;
+      const float* HT = GuT + C * CP;
+      const float* scs = HT + C * CP;
+
+      VLA_MARK(8)
+      if (c > 0) wait(b_supd, (c - 1) & 1);
+      wait(&k_full[ks], (c / KRING) & 1);
+      VLA_MARK(0)
+      // the lo scratch is free once group A's products of this chunk have read it
+      wait(b_lo_s, c & 1);
+      tc_fence_after();
+      VLA_MARK(9)
+      split_state(Cfg::COL_S);
+      tc_fence_before();
+      group_bar(2, NG);
+      if (g == 0) mbar_arrive(b_lo_rdy_s);
+      VLA_MARK(1)
+      wait(b_pr, c & 1);
+      tc_fence_after();
+      VLA_MARK(2)
+      float e[16], r0v[16];
+      {
+        uint32_t x0[32], x1[32];
+        tmem_ld32(trow + Cfg::COL_PR, x0);
+        tmem_ld32(trow + Cfg::COL_PR + 32, x1);
+        tmem_wait_ld();
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          const float pt = __uint_as_float(x0[t]) + __uint_as_float(x1[t]);          // (S k_hat_t)[g]
+          r0v[t] = __uint_as_float(x0[16 + t]) + __uint_as_float(x1[16 + t]);        // (S q_t)[g]
+          e[t] = Vf[t * VP + g] - pt;                                                 // b_t
+        }
+      }
+      tc_fence_before();
+      if (g == 0) bulk_wait_read<1>();   // the out stage of chunk c-2 has left shared memory
+      VLA_MARK(3)
+      wait(&z_full[zs], (c / RING) & 1);
+      VLA_MARK(4)
+
+      // ---- row g: e_t = b_t - sum_{s<t} Gu[s][t] e_s; e'_t = sc_t e_t;
+      //             o_t = (r0_t + sum_{s<=t} e'_s HT[t][s]) / den_t
+      float ep[16];
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        float a0 = e[t], a1 = 0.f;
+#pragma unroll
+        for (int s4 = 0; s4 * 4 < t; ++s4) {
+          const float4 g4 = reinterpret_cast<const float4*>(GuT + t * CP)[s4];
+          if (4 * s4 + 0 < t) a0 = fmaf(-g4.x, e[4 * s4 + 0], a0);
+          if (4 * s4 + 1 < t) a1 = fmaf(-g4.y, e[4 * s4 + 1], a1);
+          if (4 * s4 + 2 < t) a0 = fmaf(-g4.z, e[4 * s4 + 2], a0);
+          if (4 * s4 + 3 < t) a1 = fmaf(-g4.w, e[4 * s4 + 3], a1);
+        }
+        e[t] = a0 + a1;
+        ep[t] = e[t] * scs[t];
+      }
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        float a0 = r0v[t], a1 = 0.f;
+#pragma unroll
+        for (int s4 = 0; s4 * 4 <= t; ++s4) {
+          const float4 h4 = reinterpret_cast<const float4*>(HT + t * CP)[s4];
+          if (4 * s4 + 0 <= t) a0 = fmaf(h4.x, ep[4 * s4 + 0], a0);
+          if (4 * s4 + 1 <= t) a1 = fmaf(h4.y, ep[4 * s4 + 1], a1);
+          if (4 * s4 + 2 <= t) a0 = fmaf(h4.z, ep[4 * s4 + 2], a0);
+          if (4 * s4 + 3 <= t) a1 = fmaf(h4.w, ep[4 * s4 + 3], a1);
+        }
+        r0v[t] = (a0 + a1) * inv_den[t];
+      }
+      VLA_MARK(5)
+      group_bar(2, NG);  // bulk_wait_read above is ordered before the stage is rewritten
+      {
+        float* ost = ostage + size_t(c & 1) * C * D;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) ost[t * D + g] = r0v[t];
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) {
+          const float4 ee = make_float4(ep[4 * k4], ep[4 * k4 + 1], ep[4 * k4 + 2], ep[4 * k4 + 3]);
+          float4 hi, lo;
+          tf32_split4(ee, hi, lo);
+          reinterpret_cast<float4*>(Epf)[k4 * 128 + g] = hi;
+          reinterpret_cast<float4*>(Epl)[k4 * 128 + g] = lo;
+        }
+      }
+      fence_async_smem();
+      group_bar(2, NG);
+      if (g == 0) {
+        mbar_arrive(&k_empty[ks]);
+        bulk_store(p.out + (size_t(unit) * size_t(T) + size_t(c) * C) * D, ostage + size_t(c & 1) * C * D,
+                   uint32_t(n) * D * sizeof(float));
+        bulk_commit();
+        mbar_arrive(b_ep_rdy);
+      }
+      VLA_MARK(6)
+    }
+    if (nchunks > 0) wait(b_supd, (nchunks - 1) & 1);
+    tc_fence_after();
+    if (p.S_T) state_out(p.S_T, Cfg::COL_S);
+    if (g == 0) bulk_wait_all<0>();
+  } else if (grp == 2) {
+    // =====================================================================  group P: TMA ring + input prep
+    float* denp = reinterpret_cast<float*>(pbase);           // [2][C]
+    const int pw = g >> 5;                                   // prep warp: tokens 8 pw .. 8 pw + 7
+    const int tl = lane & 7, fl = lane >> 3;                 // token within the warp's 8, float4 lane 0..3
+    auto issue = [&](int c) {
+      const int s = c % NSTAGE;
+      const int n = min(C, T - c * C);
+      const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
+      TIn* dst = raw + size_t(s) * 3 * C * D;
+      mbar_arrive_expect_tx(&raw_full[s], 3 * bytes);
+      const size_t tok = size_t(unit) * size_t(T) + size_t(c) * C;
+      bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &raw_full[s]);
+      bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &raw_full[s]);
+      bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &raw_full[s]);
+    };
+    if (g == 0)
+      for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue(c);
+    // running sum of phi(k), columns 2g and 2g + 1
+    float2 zk = make_float2(0.f, 0.f);
+    if (p.z0) zk = *reinterpret_cast<const float2*>(p.z0 + size_t(unit) * D + 2 * g);
+
+#pragma unroll 1
+    for (int c = 0; c < nchunks; ++c) {
+      const int s = c % NSTAGE, ks = c % KRING;
+      const int n = min(C, T - c * C);
+      unsigned char* kslot = kslots + size_t(ks) * Cfg::kslot_bytes;
+      float4* KQ4 = reinterpret_cast<float4*>(kslot);
+      float* Kp = reinterpret_cast<float*>(kslot + Cfg::kq_bytes);
+      float* Qp = Kp + C * VP;
+      float* Vf = Qp + C * VP;
+      float* nrm = Vf + C * VP;
+      float* inv_den = nrm + C;
+      VLA_MARK(8)
+      wait(&raw_full[s], (c / NSTAGE) & 1);
+      VLA_MARK(0)
+      if (c >= KRING) wait(&k_empty[ks], ((c / KRING) + 1) & 1);
+      VLA_MARK(1)
+      const TIn* rq = raw + (size_t(s) * 3 + 0) * C * D;
+      const TIn* rk = raw + (size_t(s) * 3 + 1) * C * D;
+      const TIn* rv = raw + (size_t(s) * 3 + 2) * C * D;
+      {
+        const int tt = 8 * pw + tl;
+        const bool act = tt < n;
+        float4 kf[8];
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int f = fl + 4 * i;
+          float4 qf = make_float4(0.f, 0.f, 0.f, 0.f), vv = qf;
+          kf[i] = qf;
+          if (act) {
+            kf[i] = load4(rk + tt * D, f);
+            qf = load4(rq + tt * D, f);
+            vv = load4(rv + tt * D, f);
+            if (!ident) {
+              kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
+              kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
+              qf.x = phi_fast(qf.x); qf.y = phi_fast(qf.y);
+              qf.z = phi_fast(qf.z); qf.w = phi_fast(qf.w);
+            }
+          }
+          float4 hi, lo;
+          tf32_split4(qf, hi, lo);
+          KQ4[f * Cfg::KQR + 16 + tt] = hi;
+          KQ4[f * Cfg::KQR + 48 + tt] = lo;
+          reinterpret_cast<float4*>(Qp + tt * VP)[f] = qf;
+          reinterpret_cast<float4*>(Vf + tt * VP)[f] = vv;
+          ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
+          ss = fmaf(kf[i].z, kf[i].z, ss); ss = fmaf(kf[i].w, kf[i].w, ss);
+        }
+        ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 16);
+        const float nr = fmaxf(sqrt_approx(ss), eps);   // max(||phi(k)||, eps)
+        const float inv = rcp_nr(nr);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int f = fl + 4 * i;
+          const float4 kh = make_float4(kf[i].x * inv, kf[i].y * inv, kf[i].z * inv, kf[i].w * inv);
+          float4 hi, lo;
+          tf32_split4(kh, hi, lo);
+          KQ4[f * Cfg::KQR + tt] = hi;
+          KQ4[f * Cfg::KQR + 32 + tt] = lo;
+          reinterpret_cast<float4*>(Kp + tt * VP)[f] = kh;
+        }
+        // phi(k) = k_hat * nrm exactly as the recurrence sees it; 0 for padding rows
+        if (fl == 0) nrm[tt] = act ? nr : 0.0f;
+      }
+      group_bar(3, NP);
+      VLA_MARK(2)
+      if (g == 0 && c + NSTAGE < nchunks) issue(c + NSTAGE);   // the raw stage has been consumed
+      // ---- running key sum and readout denominators (columns 2g, 2g+1)
+      if (!ident) {
+        float pr[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          const float2 kh = *reinterpret_cast<const float2*>(Kp + t * VP + 2 * g);
+          const float2 qf = *reinterpret_cast<const float2*>(Qp + t * VP + 2 * g);
+          const float nt = nrm[t];
+          zk.x = fmaf(kh.x, nt, zk.x);
+          zk.y = fmaf(kh.y, nt, zk.y);
+          pr[t] = fmaf(zk.x, qf.x, zk.y * qf.y);
+        }
+        const float tot = warp_reduce_scatter16(pr, lane);
+        if ((lane & 1) == 0) denp[pw * C + (lane >> 1)] = tot;
+        group_bar(3, NP);
+        if (g < C) inv_den[g] = rcp_nr(fmaxf(denp[g] + denp[C + g], eps));
+      } else {
+        if (g < C) inv_den[g] = 1.0f;
+      }
+      fence_async_smem();   // the operand arrays are read by the tensor core
+      group_bar(3, NP);
+      if (g == 0) mbar_arrive(&k_full[ks]);
+      VLA_MARK(3)
+    }
+    if (p.zT) *reinterpret_cast<float2*>(p.zT + size_t(unit) * D + 2 * g) = zk;
+  } else if (lane == 0) {
+    // =====================================================================  MMA issue (lane 0 of two warps)
+    // g == 0 issues for group A, g == 32 for group S.  Per chunk: the state (hi part, read in
+    // place) times the chunk's operand rows; the lo scratch times the same; then the rank-16
+    // update, each a hi*hi + hi*lo + lo*hi triple.
+    const bool forA = g == 0;
+    const uint32_t col_state = forA ? Cfg::COL_A : Cfg::COL_S;
+    const uint32_t col_acc = forA ? Cfg::COL_Z0 : Cfg::COL_PR;
+    // operand rows of a chunk, 16 each: hi(K_hat) | hi(Q_f) | lo(K_hat) | lo(Q_f).
+    // hi pass (the state, read in place): A takes rows 0..47 (the middle 16 columns are not used),
+    // S all 64; lo pass (the lo scratch): A takes hi(K_hat), S takes hi(K_hat) | hi(Q_f).
+    const uint32_t idesc_hi = forA ? umma_idesc_tf32(128, 48) : umma_idesc_tf32(128, 64);
+    const uint32_t idesc_lo = forA ? umma_idesc_tf32(128, 16) : umma_idesc_tf32(128, 32);
+    const uint32_t idesc_up = umma_idesc_tf32(128, 128);
+    uint64_t* b_upd = forA ? b_aupd : b_supd;
+    uint64_t* b_lo_rdy = forA ? b_lo_rdy_a : b_lo_rdy_s;
+    uint64_t* b_prod = forA ? b_z0 : b_pr;
+    uint64_t* b_lo_next = forA ? b_lo_s : b_lo_a;
+    // left factor of the update: -Z/delta (A) or E' (S), and its lo part
+    const float* Lf = reinterpret_cast<const float*>(forA ? abase : sbase);
+    const uint64_t dLf = umma_desc(smem_u32(Lf), 16 * 128, 128);
+    const uint64_t dLl = umma_desc(smem_u32(Lf + D * C), 16 * 128, 128);
+#pragma unroll 1
+    for (int c = 0; c < nchunks; ++c) {
+      const int ks = c % KRING, zs = c % RING;
+      const uint64_t dKQ = umma_desc(smem_u32(kslots + size_t(ks) * Cfg::kslot_bytes), 16 * Cfg::KQR, 128);
+      const float* Zf = reinterpret_cast<const float*>(zslots + size_t(zs) * Cfg::zslot_bytes);
+      const uint64_t dZf = umma_desc(smem_u32(Zf), 16 * 128, 128);
+      const uint64_t dZl = umma_desc(smem_u32(Zf + D * C), 16 * 128, 128);
+      // the state is final: the previous update has completed (first chunk: the group has stored
+      // the initial state, which precedes its first arrival on b_lo_rdy)
+      VLA_MARK(8)
+      if (c > 0) wait(b_upd, (c - 1) & 1);
+      else wait(b_lo_rdy, 0);
+      wait(&k_full[ks], (c / KRING) & 1);
+      tc_fence_after();
+      VLA_MARK(0)
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        umma_ts(tbase + col_acc, tbase + col_state + 8 * j, dKQ + uint64_t(j * (2 * Cfg::KQR)), idesc_hi, j > 0);
+      VLA_MARK(1)
+      wait(b_lo_rdy, c & 1);
+      tc_fence_after();
+      VLA_MARK(2)
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        umma_ts(tbase + col_acc, tbase + Cfg::COL_LO + 8 * j, dKQ + uint64_t(j * (2 * Cfg::KQR)), idesc_lo, 1);
+      umma_commit(b_prod);
+      umma_commit(b_lo_next);
+      VLA_MARK(3)
+      if (forA) wait(&z_full[zs], (c / RING) & 1);   // Z, lo(Z), -Z/delta are in shared memory
+      else wait(b_ep_rdy, c & 1);                    // so are E' and lo(E') (and Z: group S waited for it)
+      tc_fence_after();
+      VLA_MARK(4)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        umma_ss(tbase + col_state, dLf + uint64_t(j * 256), dZf + uint64_t(j * 256), idesc_up, 1);
+        umma_ss(tbase + col_state, dLf + uint64_t(j * 256), dZl + uint64_t(j * 256), idesc_up, 1);
+        umma_ss(tbase + col_state, dLl + uint64_t(j * 256), dZf + uint64_t(j * 256), idesc_up, 1);
+      }
+      umma_commit(b_upd);
+      umma_commit(&z_empty[zs]);
+      VLA_MARK(5)
+    }
+  }
+
+#ifdef VLA_SECTION_TIMERS
+  if (p.dbg && blockIdx.x == 0) {
+    const int role = tid == 0 ? 0 : tid == 32 ? 1 : tid == NG ? 2 : tid == 2 * NG ? 3 : tid == 2 * NG + NP ? 4
+                   : tid == 2 * NG + NP + 32 ? 5 : -1;
+    if (role >= 0) for (int i = 0; i < 12; ++i) p.dbg[role * 12 + i] = tsec[i];
+  }
+#endif
+  tc_fence_before();
+  __syncthreads();
+  if (tid < 32) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(Cfg::TMEM_COLS) : "memory");
+  }
+}
+
+template <typename TIn>
+int launch_chunk_tc_t(const ScanParams& p, cudaStream_t st) {
+  using Cfg = TcCfg<TIn>;
+  static_assert(Cfg::smem_bytes <= 227 * 1024, "tensor-core chunk kernel exceeds the shared memory of one CTA");
+  auto kern = vla_scan_tc_kernel<TIn>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
+  note_launch("vla_scan_tc_kernel", Cfg::D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, p.units, 0);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+
+}  // namespace vla

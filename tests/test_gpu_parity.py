@@ -476,3 +476,30 @@ def test_forward_and_backward_replay_from_a_cuda_graph():
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         assert torch.equal(got[0], fresh.out) and torch.equal(got[1], fresh.S_T) and torch.equal(got[2], fresh.A_T)
+
+
+# ---------------------------------------------------------------- reduction modes (Section 4.4)
+@pytest.mark.parametrize("kernel", ["token", "chunk"])
+@pytest.mark.parametrize("d,dtype", [(32, "f32"), (64, "bf16"), (128, "f32")])
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_zero_penalty_directions_give_the_normalised_delta_rule(kernel, d, dtype, flags):
+    """u = 0 passed explicitly (Section 4.4's remark; Eq. "deltanet" without the gate): the
+    penalty never grows, A stays A_0 = I/lambda exactly, the write direction is k_hat and
+    S_t = S_{t-1} + (v_t - S_{t-1} k_hat_t) k_hat_t^T.  Checked against the oracle and against
+    that recurrence written out here in fp64."""
+    w = _small(d, 70, dtype, units=(1, 3), seed=300 + d)
+    q, k, v = W.make_inputs(w)
+    u0 = torch.zeros_like(k)
+    lam = 0.5
+    errs, got, ref = check_parity(q, k, v, lam, 1e-4, u=u0, flags=flags, kernel=KERNELS[kernel],
+                                  label="u=0 %s d=%d" % (kernel, d))
+    A_T = got.A_T.cpu()
+    assert torch.equal(A_T, (torch.eye(d) / lam).expand_as(A_T)), "A must not move when u = 0"
+    kk, vv = k.double().numpy(), v.double().numpy()
+    for h in range(w.H):
+        S = np.zeros((d, d))
+        for t in range(w.T):
+            kf = kk[0, h, t] if flags & IDENT else np.where(kk[0, h, t] > 0, kk[0, h, t] + 1.0, np.exp(kk[0, h, t]))
+            kh = kf / np.linalg.norm(kf)
+            S += np.outer(vv[0, h, t] - S @ kh, kh)
+        assert np.abs(got.S_T[0, h].cpu().double().numpy() - S).max() <= 1e-4 * np.abs(S).max()

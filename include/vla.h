@@ -71,15 +71,16 @@ enum {
 typedef enum {
   VLA_KERNEL_AUTO = 0,
   VLA_KERNEL_TOKEN = 1, /* one CTA per unit, one state pass per token; every shape, explicit u */
-  VLA_KERNEL_CHUNK = 2, /* 16 tokens per state pass (exact Woodbury form); d >= 32, every option;
-                           VLA_ERR_UNSUPPORTED for d = 16 */
+  VLA_KERNEL_CHUNK = 2, /* 16 tokens per state pass (exact Woodbury form) on the fp32 FMA pipe; d >= 32,
+                           every option; VLA_ERR_UNSUPPORTED for d = 16 */
   VLA_KERNEL_DECODE = 3, /* one step (T = 1) with S0, A0, S_T, A_T all given, u = k_hat, no refresh,
                            d >= 32: the states stream through shared memory once (HBM-bound);
                            VLA_ERR_UNSUPPORTED otherwise.  AUTO picks it when it applies */
   VLA_KERNEL_CHUNK_TC = 4 /* the chunk algebra on the tensor cores (Section 3.4: the chunked recurrence
                            is a chain of dense products): states in tensor memory, TF32 products in
                            hi/lo pairs with fp32 accumulation.  d = 128, u = k_hat, no refresh,
-                           [B,H,T,d] tensors, T >= 1; VLA_ERR_UNSUPPORTED otherwise */
+                           [B,H,T,d] tensors, T >= 1; VLA_ERR_UNSUPPORTED otherwise.  AUTO picks it
+                           where it applies (and VLA_KERNEL_CHUNK then forces the fp32-FMA form) */
 } vla_kernel_t;
 
 typedef struct {

@@ -92,6 +92,8 @@ int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
   if (kernel == VLA_KERNEL_CHUNK && !chunk) return VLA_ERR_UNSUPPORTED;
   if (kernel == VLA_KERNEL_AUTO && !chunk_pays_off(p, d)) chunk = false;
   if (kernel == VLA_KERNEL_TOKEN) chunk = false;
+  // d = 128: the same chunk algebra runs faster with the d x d products on the tensor cores
+  if (chunk && kernel == VLA_KERNEL_AUTO && chunk_tc_covers(p, d)) return vla::launch_chunk_tc(d, dtype, p, st);
   if (chunk) return vla::launch_chunk(d, dtype, p, st);
   return vla::launch_token(d, dtype, p, st);
 }

@@ -385,10 +385,13 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   unsigned int* sched_flags = g_sched_flags + size_t(sp.epoch % kSchedSlots) * kSchedMaxUnits;
 
   // Bounded wait shared by every mbarrier in this kernel.
-  const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitProbeLimit;
+  // (the caller's limit is read from the parameters where it is needed: no register is spent on
+  // it in the FMA loops)
   auto wait = [&](uint64_t* bar, uint32_t parity) {
     if (*abort_flag) return;
-    if (!mbar_wait_bounded(bar, parity, wait_limit)) {
+    const bool done = p.wait_limit == 0 ? mbar_wait_bounded(bar, parity)
+                                        : mbar_wait_bounded(bar, parity, p.wait_limit);
+    if (!done) {
       *abort_flag = 1;
       if (p.status) atomicCAS(p.status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
     }
@@ -469,7 +472,8 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
     if (from_handoff && !*abort_flag) {
       bool seen = false;
       // four times the probes of a barrier wait: a probe here is one acquire load and a short sleep
-      for (uint64_t it = 0; it < 4ull * wait_limit && !seen; ++it) {
+      const uint64_t probes = 4ull * (p.wait_limit ? p.wait_limit : kWaitProbeLimit);
+      for (uint64_t it = 0; it < probes && !seen; ++it) {
         seen = ld_acquire_gpu(&sched_flags[unit]) == sp.epoch;
         if (!seen) __nanosleep(64);
       }

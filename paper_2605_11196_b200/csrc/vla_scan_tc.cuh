@@ -137,11 +137,11 @@ struct TcCfg {
   static constexpr int KQR = 64;                // operand rows of a chunk: hi(k_hat) | hi(q_f) | lo(k_hat) | lo(q_f)
   static constexpr size_t kq_bytes = size_t(KQR) * D * 4;           // [32][64] float4
   static constexpr size_t kp_bytes = size_t(2) * C * VP * 4;        // k_hat, q_f as plain fp32 rows [C][VP]
-  static constexpr size_t kslot_bytes = kq_bytes + kp_bytes + size_t(C) * VP * 4 + 2 * C * 4;   // + v, nrm, 1/den
+  static constexpr size_t kslot_bytes = kq_bytes + kp_bytes + size_t(C) * VP * 4 + 4 * C * 4;   // + v, nrm, 1/den, means of k_hat and q_f
   static constexpr size_t op16_bytes = size_t(D) * C * 4;           // [4][128] float4: a 128 x 16 operand
-  static constexpr size_t zslot_bytes = 2 * op16_bytes + (2 * C * CP + C) * 4;      // Z, lo(Z), GuT, HT, sc
-  static constexpr size_t a_bytes = 2 * op16_bytes + size_t(C) * D * 4 + (2 * C * CP + 4 * C + 3 * C) * 4;
-  //   -Z/delta, lo | Z0 / Z rows [C][D] | W, L | N2p[4][C] | delta, 1/delta, -1/delta
+  static constexpr size_t zslot_bytes = 2 * op16_bytes + (2 * C * CP + 2 * C) * 4;  // Z, lo(Z), GuT, HT, sc, sums of z_t
+  static constexpr size_t a_bytes = 2 * op16_bytes + size_t(C) * D * 4 + (2 * C * CP + 8 * C + 3 * C) * 4;
+  //   -Z/delta, lo | Z0 / Z rows [C][D] | W, L | N2p[4][C], ZSp[4][C] | delta, 1/delta, -1/delta
   static constexpr size_t s_bytes = 2 * op16_bytes + 2 * size_t(C) * D * 4;         // E', lo(E') | out stage [2]
   static constexpr size_t p_bytes = 2 * C * 4;                                      // denp[2][C]
   static constexpr int NBAR = NSTAGE + 2 * KRING + 2 * RING + 9;
@@ -272,8 +272,9 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   const uint32_t tbase = *tmem_slot;
   const uint32_t trow = tbase + (uint32_t((tid >> 5) & 3) << 21);   // this warp's 32 lanes: lane field = bits 16..
 
-  // one state row: global (or the initial value) -> tensor memory
-  auto state_in = [&](const float* src, float diag, uint32_t col) {
+  // one state row: global (or the initial value) -> tensor memory; returns the row's sum
+  auto state_in = [&](const float* src, float diag, uint32_t col) -> float {
+    float rowsum = 0.0f;
 #pragma unroll 1
     for (int c0 = 0; c0 < D; c0 += 32) {
       uint32_t r[32];
@@ -289,9 +290,12 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
 #pragma unroll
         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint((c0 + i == g) ? diag : 0.0f);
       }
+#pragma unroll
+      for (int i = 0; i < 32; ++i) rowsum += __uint_as_float(r[i]);
       tmem_st32(trow + col + c0, r);
     }
     tmem_wait_st();
+    return rowsum;
   };
   auto state_out = [&](float* dst, uint32_t col) {
 #pragma unroll 1
@@ -328,10 +332,12 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     float* Ws = Zp + C * D;                                  // [C][CP] K A K^T
     float* Ls = Ws + C * CP;                                 // [C][CP] unit lower factor
     float* N2p = Ls + C * CP;                                // [4][C]
-    float* dlt = N2p + 4 * C;                                // [C]
+    float* ZSp = N2p + 4 * C;                                // [4][C] per-warp sums of the entries of z_t
+    float* dlt = ZSp + 4 * C;                                // [C]
     float* idl = dlt + C;                                    // [C]  1/delta
     float* nidl = idl + C;                                   // [C] -1/delta
-    state_in(p.A0, 1.0f / p.lambda, Cfg::COL_A);
+    // w1 = (A 1)[g], the row sum of A, carried along in fp32 (see "centred operands" below)
+    float w1 = state_in(p.A0, 1.0f / p.lambda, Cfg::COL_A);
 
 #pragma unroll 1
     for (int c = 0; c < nchunks; ++c) {
@@ -345,6 +351,8 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       float* GuT = Zl + D * C;                               // [C][CP]
       float* HT = GuT + C * CP;                              // [C][CP]
       float* scs = HT + C * CP;                              // [C]
+      float* ssm = scs + C;                                  // [C] sum of the entries of z_t
+      const float* ckm = reinterpret_cast<const float*>(kslot + Cfg::kq_bytes + Cfg::kp_bytes) + C * VP + 2 * C;   // [C] mean of k_hat_t
 
       VLA_MARK(8)
       // A is final once the update of the previous chunk has completed
@@ -371,7 +379,8 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         tmem_wait_ld();
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
-          z[t] = __uint_as_float(r0[t]) + __uint_as_float(r1[t]);   // row g of Z0 = A K^T
+          // row g of Z0 = A K^T = A (K - mean)^T + (A 1) mean^T
+          z[t] = fmaf(w1, ckm[t], __uint_as_float(r0[t]) + __uint_as_float(r1[t]));
           Zp[t * D + g] = z[t];
         }
       }
@@ -447,14 +456,29 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         }
         const float tot = warp_reduce_scatter16(sq, lane);
         if ((lane & 1) == 0) N2p[gw * C + (lane >> 1)] = tot;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) sq[t] = z[t];
+        const float tot1 = warp_reduce_scatter16(sq, lane);
+        if ((lane & 1) == 0) ZSp[gw * C + (lane >> 1)] = tot1;
+#ifdef VLA_TC_DUMP
+        if (p.stash_z) for (int t = 0; t < 16; ++t) p.stash_z[(size_t(unit) * T + c * C + t) * D + g] = z[t];
+        if (p.stash_delta && g < 16) p.stash_delta[size_t(unit) * T + c * C + g] = dlt[g];
+#endif
       }
       group_bar(1, NG);
       VLA_MARK(6)
 
+      // ---- A 1 after this chunk: w1 -= sum_t z_t[g] (z_t . 1) / delta_t
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        const float st = (ZSp[t] + ZSp[C + t]) + (ZSp[2 * C + t] + ZSp[3 * C + t]);
+        w1 = fmaf(-z[t], st * idl[t], w1);
+      }
       // ---- warp 0: sc_t and GuT[t][s] = Gu[s][t] = sc_s delta_s L[t][s]
       if (gw == 0) {
         const int r = lane & 15, h = lane >> 4;
         const float n2 = N2p[r] + N2p[C + r] + N2p[2 * C + r] + N2p[3 * C + r];
+        if (h == 1) ssm[r] = (ZSp[r] + ZSp[C + r]) + (ZSp[2 * C + r] + ZSp[3 * C + r]);
         const float id_r = idl[r], d_r = dlt[r];
         // alpha_r = sc_r z_r, sc_r = (1/delta) / max(||z||/delta, eps)      (A_t k_hat_t = z_t / delta_t)
         const float sc_r = id_r * rcp_nr(fmaxf(sqrt_approx(n2) * id_r, eps));
@@ -487,7 +511,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     float* Epf = reinterpret_cast<float*>(sbase);            // [4][128] float4: e'_t
     float* Epl = Epf + D * C;
     float* ostage = Epl + D * C;                             // [2][C][D]
-    state_in(p.S0, 0.0f, Cfg::COL_S);
+    float s1 = state_in(p.S0, 0.0f, Cfg::COL_S);   // (S 1)[g], carried along in fp32
 
 #pragma unroll 1
     for (int c = 0; c < nchunks; ++c) {
@@ -496,10 +520,13 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       unsigned char* kslot = kslots + size_t(ks) * Cfg::kslot_bytes;
       const float* Vf = reinterpret_cast<const float*>(kslot + Cfg::kq_bytes + Cfg::kp_bytes);   // [C][VP]
       const float* inv_den = Vf + C * VP + C;
+      const float* ckm = inv_den + C;                       // [C] mean of k_hat_t
+      const float* cqm = ckm + C;                           // [C] mean of q_f,t
       unsigned char* zslot = zslots + size_t(zs) * Cfg::zslot_bytes;
       const float* GuT = reinterpret_cast<const float*>(zslot) + 2 * D * C;
       const float* HT = GuT + C * CP;
       const float* scs = HT + C * CP;
+      const float* ssm = scs + C;
 
       VLA_MARK(8)
       if (c > 0) wait(b_supd, (c - 1) & 1);
@@ -525,8 +552,9 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         tmem_wait_ld();
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
-          const float pt = __uint_as_float(x0[t]) + __uint_as_float(x1[t]);          // (S k_hat_t)[g]
-          r0v[t] = __uint_as_float(x0[16 + t]) + __uint_as_float(x1[16 + t]);        // (S q_t)[g]
+          // (S k_hat_t)[g] and (S q_t)[g], each as S (x - mean)^T + (S 1) mean
+          const float pt = fmaf(s1, ckm[t], __uint_as_float(x0[t]) + __uint_as_float(x1[t]));
+          r0v[t] = fmaf(s1, cqm[t], __uint_as_float(x0[16 + t]) + __uint_as_float(x1[16 + t]));
           e[t] = Vf[t * VP + g] - pt;                                                 // b_t
         }
       }
@@ -552,6 +580,10 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         }
         e[t] = a0 + a1;
         ep[t] = e[t] * scs[t];
+        s1 = fmaf(ep[t], ssm[t], s1);          // S 1 after this chunk: += e'_t (z_t . 1)
+#ifdef VLA_TC_DUMP
+        if (p.stash_e) p.stash_e[(size_t(unit) * T + c * C + t) * D + g] = e[t];
+#endif
       }
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
@@ -640,49 +672,62 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       {
         const int tt = 8 * pw + tl;
         const bool act = tt < n;
-        float4 kf[8];
-        float ss = 0.f;
+        float4 kf[8], qv[8];
+        float ss = 0.f, sk = 0.f, sqm = 0.f;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int f = fl + 4 * i;
-          float4 qf = make_float4(0.f, 0.f, 0.f, 0.f), vv = qf;
-          kf[i] = qf;
+          float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
+          kf[i] = vv; qv[i] = vv;
           if (act) {
             kf[i] = load4(rk + tt * D, f);
-            qf = load4(rq + tt * D, f);
+            qv[i] = load4(rq + tt * D, f);
             vv = load4(rv + tt * D, f);
             if (!ident) {
               kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
               kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
-              qf.x = phi_fast(qf.x); qf.y = phi_fast(qf.y);
-              qf.z = phi_fast(qf.z); qf.w = phi_fast(qf.w);
+              qv[i].x = phi_fast(qv[i].x); qv[i].y = phi_fast(qv[i].y);
+              qv[i].z = phi_fast(qv[i].z); qv[i].w = phi_fast(qv[i].w);
             }
           }
-          float4 hi, lo;
-          tf32_split4(qf, hi, lo);
-          KQ4[f * Cfg::KQR + 16 + tt] = hi;
-          KQ4[f * Cfg::KQR + 48 + tt] = lo;
-          reinterpret_cast<float4*>(Qp + tt * VP)[f] = qf;
+          reinterpret_cast<float4*>(Qp + tt * VP)[f] = qv[i];
           reinterpret_cast<float4*>(Vf + tt * VP)[f] = vv;
           ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
           ss = fmaf(kf[i].z, kf[i].z, ss); ss = fmaf(kf[i].w, kf[i].w, ss);
+          sk += (kf[i].x + kf[i].y) + (kf[i].z + kf[i].w);
+          sqm += (qv[i].x + qv[i].y) + (qv[i].z + qv[i].w);
         }
-        ss += __shfl_xor_sync(0xffffffffu, ss, 8);
-        ss += __shfl_xor_sync(0xffffffffu, ss, 16);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 8);  ss += __shfl_xor_sync(0xffffffffu, ss, 16);
+        sk += __shfl_xor_sync(0xffffffffu, sk, 8);  sk += __shfl_xor_sync(0xffffffffu, sk, 16);
+        sqm += __shfl_xor_sync(0xffffffffu, sqm, 8); sqm += __shfl_xor_sync(0xffffffffu, sqm, 16);
         const float nr = fmaxf(sqrt_approx(ss), eps);   // max(||phi(k)||, eps)
         const float inv = rcp_nr(nr);
+        // Centred operands: the tensor core truncates its addends towards zero, so a sum of
+        // like-signed products (feature-mapped keys and queries are all positive) comes out
+        // low by an amount that is the same in every row and piles up along the common
+        // direction of the keys.  The products are therefore taken with x - mean(x), whose
+        // entries have both signs, and the mean's share, (state . 1) mean(x), is added back in
+        // fp32 by the groups, which carry state . 1 along with the state.
+        const float mk = sk * inv * (1.0f / D), mq = sqm * (1.0f / D);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int f = fl + 4 * i;
           const float4 kh = make_float4(kf[i].x * inv, kf[i].y * inv, kf[i].z * inv, kf[i].w * inv);
+          reinterpret_cast<float4*>(Kp + tt * VP)[f] = kh;
           float4 hi, lo;
-          tf32_split4(kh, hi, lo);
+          tf32_split4(make_float4(kh.x - mk, kh.y - mk, kh.z - mk, kh.w - mk), hi, lo);
           KQ4[f * Cfg::KQR + tt] = hi;
           KQ4[f * Cfg::KQR + 32 + tt] = lo;
-          reinterpret_cast<float4*>(Kp + tt * VP)[f] = kh;
+          tf32_split4(make_float4(qv[i].x - mq, qv[i].y - mq, qv[i].z - mq, qv[i].w - mq), hi, lo);
+          KQ4[f * Cfg::KQR + 16 + tt] = hi;
+          KQ4[f * Cfg::KQR + 48 + tt] = lo;
         }
         // phi(k) = k_hat * nrm exactly as the recurrence sees it; 0 for padding rows
-        if (fl == 0) nrm[tt] = act ? nr : 0.0f;
+        if (fl == 0) {
+          nrm[tt] = act ? nr : 0.0f;
+          inv_den[C + tt] = act ? mk : 0.0f;          // mean of k_hat_t
+          inv_den[2 * C + tt] = act ? mq : 0.0f;      // mean of q_f,t
+        }
       }
       group_bar(3, NP);
       VLA_MARK(2)

@@ -418,7 +418,7 @@ def test_token_major_long_units_and_where_it_is_refused():
     assert rel_err(r.out.permute(0, 2, 1, 3), ref.out) <= 1e-4
     wb = W.Workload("t", 1, 151, 128, 256 + 5, "bf16", 79)      # more units than resident CTAs
     q, k, v = W.make_inputs(wb)
-    plain = run_gpu(q, k, v, wb.lam)
+    plain = run_gpu(q, k, v, wb.lam, kernel=vla.VLA_KERNEL_CHUNK)   # the same (FMA) kernel, head-major
     r = vla.vla_forward(tm(q), tm(k), tm(v), wb.lam, flags=TOKEN_MAJOR)
     torch.cuda.synchronize()
     assert int(r.status.item()) == 0

@@ -1,14 +1,12 @@
 """Tensor-core form of the chunk kernel (VLA_KERNEL_CHUNK_TC, d = 128) vs the fp64 CPU oracle,
 element by element, through the C ABI (-m gpu).
 
-The kernel is opt-in: the library's own kernel choice never takes it.  It computes the same
-chunk algebra as the FMA kernel with the d x d products on the tensor cores (TF32 operands in
-hi/lo pairs, fp32 accumulation).  The tensor core truncates when it aligns and accumulates
-its addends, so sums of many like-signed products come out slightly low; with Section 3.1's
-normalised keys (mixed signs) it holds the bounds of the specification at every length, with
-Algorithm 1's feature map (all-positive keys, which share a dominant direction) the final S
-drifts beyond 1e-4 of its maximum on long sequences.  The tests assert the specification's
-bounds wherever the kernel meets them and pin the measured drift where it does not.
+It computes the same chunk algebra as the FMA kernel with the d x d products on the tensor
+cores (TF32 operands in hi/lo pairs, fp32 accumulation, states in tensor memory).  The tensor
+core truncates when it aligns and accumulates its addends; the kernel keeps that from piling
+up along the common direction of feature-mapped (all-positive) keys by centring the operands
+and carrying (state . 1) in fp32.  The tests hold it to the specification's bounds in both
+readings of the feature map, at the lengths of the workloads.
 """
 import numpy as np
 import pytest
@@ -57,8 +55,12 @@ def test_tc_carried_states_and_split_invariance(dtype, flags):
     T1 = 112   # a multiple of the chunk: the second call starts on the same chunk boundaries
     a = run_gpu(q[:, :, :T1], k[:, :, :T1], v[:, :, :T1], 1.0, S0=S0, A0=A0, z0=z0, flags=flags, kernel=TC)
     b = run_gpu(q[:, :, T1:], k[:, :, T1:], v[:, :, T1:], 1.0, S0=a.S_T, A0=a.A_T, z0=a.z_T, flags=flags, kernel=TC)
-    assert torch.equal(torch.cat([a.out, b.out], dim=2), got.out)
-    assert torch.equal(b.S_T, got.S_T) and torch.equal(b.A_T, got.A_T) and torch.equal(b.z_T, got.z_T)
+    # (state . 1) is re-formed from the carried state at the start of a call, so the two runs
+    # agree to rounding, not bit for bit
+    f64 = lambda x: x.cpu().double().numpy()
+    assert rel_err(torch.cat([a.out, b.out], dim=2), f64(got.out)) <= 1e-5
+    assert rel_err(b.S_T, f64(got.S_T)) <= 1e-5 and rel_err(b.A_T, f64(got.A_T)) <= 1e-5
+    assert torch.equal(b.z_T, got.z_T)
 
 
 def test_tc_is_deterministic_and_leaves_canaries_alone():
@@ -102,36 +104,46 @@ def test_tc_many_units_more_than_one_wave():
 
 @pytest.mark.parametrize("dtype,T,tol", [("f32", 4096, 1e-4), ("bf16", 8192, 1e-3)])
 def test_tc_long_sequences_normalised_keys(dtype, T, tol):
-    """Section 3.1's keys: the specification's bounds hold at full length."""
+    """Section 3.1's keys at full length."""
     w = W.Workload("tc", 1, 2, 128, T, dtype, 44)
     q, k, v = W.make_inputs(w)
     errs, _, _ = check_parity(q, k, v, 1.0, tol, flags=IDENT, kernel=TC, label="tc long, normalised keys")
     assert max(errs.values()) <= 2e-5, errs     # measured <= 6e-6
 
 
-def test_tc_long_sequence_feature_map_drift_is_as_measured():
-    """Algorithm 1's feature map at T = 4096: the readout, A_T and z_T hold 1e-4; the final S does
-    not (measured 2.5e-4 of its maximum, against 3e-6 on the FMA kernel), which is why the
-    library never chooses this kernel by itself.  The bound asserted for S_T is the measured
-    drift with margin, not the specification's."""
-    w = W.Workload("tc", 1, 1, 128, 4096, "bf16", 5)
+@pytest.mark.parametrize("T,tol", [(4096, 1e-4), (8192, 1e-3)])
+def test_tc_long_sequences_feature_map(T, tol):
+    """Algorithm 1's feature map: all-positive keys share a dominant direction, which is where a
+    bias of the products would pile up.  The specification's bounds hold (measured: S_T 6e-6 at
+    T = 4096, 1.2e-5 at 8192; the FMA kernel 3e-6)."""
+    w = W.Workload("tc", 1, 1, 128, T, "bf16", 5)
     q, k, v = W.make_inputs(w)
-    ref = run_oracle(q, k, v, 1.0)
-    got = run_gpu(q, k, v, 1.0, kernel=TC)
-    assert rel_err(got.out, ref.out) <= 1e-4
-    assert rel_err(got.A_T, ref.A_T) <= 1e-4
-    assert rel_err(got.z_T, ref.z_T) <= 1e-4
-    assert rel_err(got.S_T, ref.S_T) <= 1e-3
-    fma = run_gpu(q, k, v, 1.0, kernel=vla.VLA_KERNEL_CHUNK)
-    assert rel_err(fma.S_T, ref.S_T) <= 1e-4      # the default kernel holds the bound on the same input
+    errs, _, _ = check_parity(q, k, v, 1.0, tol, kernel=TC, label="tc long, feature map")
+    assert max(errs.values()) <= 1e-4, errs
 
 
-def test_auto_never_picks_the_tc_kernel():
-    """The library's own choice at d = 128 is bit-identical to the FMA chunk kernel."""
+def test_tc_very_long_sequence():
+    """T = 65536 at d = 128, one unit, both readings: within the 1e-3 of long sequences (measured
+    A_T 1.6e-4: the rank-16 updates accumulate into the state with truncation)."""
+    w = W.Workload("tc", 1, 1, 128, 65536, "bf16", 6)
+    q, k, v = W.make_inputs(w)
+    for flags in (0, IDENT):
+        check_parity(q, k, v, 1.0, 1e-3, flags=flags, kernel=TC, label="tc T=65536")
+
+
+def test_auto_picks_the_tc_kernel_where_it_applies():
+    """The library's own choice at d = 128 (u = k_hat, no refresh, [B,H,T,d]) is the tensor-core
+    kernel; an explicit u, the refresh or token-major tensors go to the FMA chunk kernel."""
     dev = torch.device("cuda:0")
     w = W.Workload("tc", 1, 3, 128, 96, "bf16", 8)
     q, k, v = [x.to(dev) for x in W.make_inputs(w)]
     a = vla.vla_forward(q, k, v, 1.0)
-    b = vla.vla_forward(q, k, v, 1.0, kernel=vla.VLA_KERNEL_CHUNK)
+    assert vla.last_launch().startswith("vla_scan_tc_kernel<128,bf16>")
+    b = vla.vla_forward(q, k, v, 1.0, kernel=TC)
     torch.cuda.synchronize()
     assert torch.equal(a.out, b.out) and torch.equal(a.S_T, b.S_T) and torch.equal(a.A_T, b.A_T)
+    vla.vla_forward(q, k, v, 1.0, refresh=(20, 1e-3, 0))
+    assert vla.last_launch().startswith("vla_scan_chunk_kernel<128,bf16>")
+    vla.vla_forward(q, k, v, 1.0, u=W.make_u(w).to(dev))
+    assert vla.last_launch().startswith("vla_scan_chunk_kernel<128,bf16>")
+    torch.cuda.synchronize()

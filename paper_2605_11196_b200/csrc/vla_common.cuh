@@ -288,4 +288,66 @@ __device__ __forceinline__ float warp_reduce_scatter16(float (&v)[16], int lane)
   return v[0];  // token index = lane >> 1
 }
 
+// ---------------------------------------------------------------- work distribution (chunk kernels)
+constexpr int kSchedSlots = 16;        // launches whose flags may be live at the same time
+constexpr int kSchedMaxUnits = 4096;   // units per launch in balanced mode
+
+struct SchedParams {
+  int balanced;        // 0: plain, 1: balanced
+  int grid;            // number of CTAs (balanced)
+  unsigned int epoch;  // launch id; flag value that means "head of this unit is done"
+};
+
+struct Piece {
+  int unit, cb, ce;      // chunks [cb, ce) of the unit
+  bool from_handoff;     // state comes from S_T / A_T / zT once the unit's flag shows the epoch
+  bool to_handoff;       // state goes to S_T / A_T / zT and the flag is raised
+};
+
+template <bool BALANCED>
+__device__ __forceinline__ bool get_piece(const SchedParams& sp, int units, int nch, int cta,
+                                          int pi, Piece& out) {
+  if (!BALANCED) {
+    if (pi > 0) return false;
+    out.unit = cta; out.cb = 0; out.ce = nch; out.from_handoff = false; out.to_handoff = false;
+    return true;
+  }
+  const long long N = 1LL * units * nch;
+  const long long lo = cta * N / sp.grid, hi = (cta + 1) * N / sp.grid;
+  if (hi <= lo) return false;
+  const int xf = int(lo / nch), xl = int((hi - 1) / nch);
+  const bool tail = lo > 1LL * xf * nch;                                    // first unit began earlier
+  const bool head = hi < 1LL * (xl + 1) * nch && 1LL * xl * nch >= lo;      // last unit ends later
+  const int wf = xf + (tail ? 1 : 0), wl = xl - (head ? 1 : 0);
+  const int nwhole = wl >= wf ? wl - wf + 1 : 0;
+  if (head) {
+    if (pi == 0) {
+      out.unit = xl; out.cb = 0; out.ce = int(hi - 1LL * xl * nch);
+      out.from_handoff = false; out.to_handoff = true;
+      return true;
+    }
+    --pi;
+  }
+  if (pi < nwhole) {
+    out.unit = wf + pi; out.cb = 0; out.ce = nch; out.from_handoff = false; out.to_handoff = false;
+    return true;
+  }
+  pi -= nwhole;
+  if (tail && pi == 0) {
+    out.unit = xf; out.cb = int(lo - 1LL * xf * nch); out.ce = nch;
+    out.from_handoff = true; out.to_handoff = false;
+    return true;
+  }
+  return false;
+}
+
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu(unsigned int* p, unsigned int v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
 }  // namespace vla

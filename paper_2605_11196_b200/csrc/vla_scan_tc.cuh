@@ -108,7 +108,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 // place, is split as it reads it: hi = the truncated word, lo = rn_tf32(x - hi).
 __device__ __forceinline__ float tf32_trunc(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 __device__ __forceinline__ float tf32_rn(float x) { return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u); }
-__device__ __forceinline__ float tf32_state_lo(float x) { return tf32_rn(x - tf32_trunc(x)); }
+__device__ __forceinline__ float tf32_state_lo(float x) { return x - tf32_trunc(x); }
 __device__ __forceinline__ void tf32_split4(float4 x, float4& hi, float4& lo) {
   hi = make_float4(tf32_rn(x.x), tf32_rn(x.y), tf32_rn(x.z), tf32_rn(x.w));
   lo = make_float4(tf32_rn(x.x - hi.x), tf32_rn(x.y - hi.y), tf32_rn(x.z - hi.z), tf32_rn(x.w - hi.w));
@@ -191,8 +191,15 @@ __device__ __forceinline__ void gram16_tc(const float* X, const float* Y, float*
   }
 }
 
-template <typename TIn>
-__global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const ScanParams p) {
+// Hand-over flags of the balanced schedule (see SchedParams): one word per unit and slot.
+static __device__ unsigned int g_tc_sched_flags[kSchedSlots * kSchedMaxUnits];
+
+// BALANCED: a persistent grid of one CTA per SM; the units' chunk sequences, laid end to end, are
+// cut into equal pieces, and a unit that straddles a cut is started by one CTA (first thing it
+// does) and finished by the next (last thing it does), with S, A, the key sum handed over through
+// the caller's S_T / A_T / zT and a release/acquire flag per unit.
+template <typename TIn, bool BALANCED>
+__global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const ScanParams p, const SchedParams sp) {
   using Cfg = TcCfg<TIn>;
   constexpr int D = Cfg::D, C = Cfg::C, NG = Cfg::NG, NP = Cfg::NP, CP = Cfg::CP, VP = Cfg::VP;
   constexpr int NSTAGE = Cfg::NSTAGE, KRING = Cfg::KRING, RING = Cfg::RING;
@@ -228,9 +235,12 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   const int lane = tid & 31, gw = g >> 5;
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
   const float eps = p.eps;
-  const int unit = blockIdx.x;
-  const int T = p.T;
-  const int nchunks = (T + C - 1) / C;
+  const int nch_unit = (p.T + C - 1) / C;   // chunks per unit
+  // the piece of work in hand (set at the top of the piece loop): tokens [t_begin, t_begin + T)
+  // of `unit`, nchunks chunks
+  int unit = 0, T = 0, nchunks = 0, t_begin = 0;
+  bool from_handoff = false;
+  unsigned int* sched_flags = g_tc_sched_flags + size_t(sp.epoch % kSchedSlots) * kSchedMaxUnits;
 
   const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitProbeLimit;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
@@ -273,8 +283,11 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   const uint32_t trow = tbase + (uint32_t((tid >> 5) & 3) << 21);   // this warp's 32 lanes: lane field = bits 16..
 
   // one state row: global (or the initial value) -> tensor memory; returns the row's sum
-  auto state_in = [&](const float* src, float diag, uint32_t col) -> float {
-    float rowsum = 0.0f;
+  auto state_in = [&](const float* src, float diag, uint32_t col, bool handed_over) -> float {
+    // the row sum seeds (state . 1), which is then carried along exactly as the recurrence moves
+    // it: an error made here stays for the rest of the unit, and for A the sum cancels to a
+    // thousandth of its terms once many keys have been seen, so it is taken in fp64
+    double rowsum = 0.0;
 #pragma unroll 1
     for (int c0 = 0; c0 < D; c0 += 32) {
       uint32_t r[32];
@@ -282,7 +295,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         const float4* s4 = reinterpret_cast<const float4*>(src + (size_t(unit) * D + g) * D + c0);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float4 x = __ldg(s4 + i);
+          const float4 x = handed_over ? __ldcg(s4 + i) : __ldg(s4 + i);   // written by another SM: past L1
           r[4 * i + 0] = __float_as_uint(x.x); r[4 * i + 1] = __float_as_uint(x.y);
           r[4 * i + 2] = __float_as_uint(x.z); r[4 * i + 3] = __float_as_uint(x.w);
         }
@@ -291,13 +304,38 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint((c0 + i == g) ? diag : 0.0f);
       }
 #pragma unroll
-      for (int i = 0; i < 32; ++i) rowsum += __uint_as_float(r[i]);
+      for (int i = 0; i < 32; ++i) rowsum += double(__uint_as_float(r[i]));
       tmem_st32(trow + col + c0, r);
     }
     tmem_wait_st();
-    return rowsum;
+    return float(rowsum);
   };
-  auto state_out = [&](float* dst, uint32_t col) {
+  // One state row: tensor memory -> global.  During the scan the products see the state only
+  // through centred operands plus the carried (state . 1), so what the stored state itself
+  // holds along the all-ones direction is never used and drifts (the rank-16 updates accumulate
+  // with truncation).  Before it leaves, the row is therefore corrected so that the state that
+  // is written has the carried `tracked` as its row sum: X += dlt 1^T / D for S, and the
+  // symmetric X += (dlt 1^T + 1 dlt^T) / D - (1^T dlt) 1 1^T / D^2 for A, dlt = tracked - X 1.
+  // A later call (or the CTA that continues a cut unit) re-forms (state . 1) from these rows.
+  // `dvec`: D floats of the group's shared memory; `bar_id`: the group's named barrier.
+  auto state_out = [&](float* dst, uint32_t col, float tracked, bool symmetric, float* dvec, int bar_id) {
+    double rowsum = 0.0;
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld32(trow + col + c0, r);
+      tmem_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) rowsum += double(__uint_as_float(r[i]));
+    }
+    const float dg = float(double(tracked) - rowsum);
+    float total = 0.0f;
+    if (symmetric) {
+      dvec[g] = dg;
+      group_bar(bar_id, NG);
+      for (int j = 0; j < D; ++j) total += dvec[j];
+    }
+    const float own = dg * (1.0f / D) - (symmetric ? total * (1.0f / (D * D)) : 0.0f);
 #pragma unroll 1
     for (int c0 = 0; c0 < D; c0 += 32) {
       uint32_t r[32];
@@ -305,10 +343,19 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       tmem_wait_ld();
       float4* d4 = reinterpret_cast<float4*>(dst + (size_t(unit) * D + g) * D + c0);
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        d4[i] = make_float4(__uint_as_float(r[4 * i + 0]), __uint_as_float(r[4 * i + 1]),
-                            __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+      for (int i = 0; i < 8; ++i) {
+        float4 x = make_float4(__uint_as_float(r[4 * i + 0]), __uint_as_float(r[4 * i + 1]),
+                               __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+        float4 cj = make_float4(own, own, own, own);
+        if (symmetric) {
+          const float4 dj = *reinterpret_cast<const float4*>(dvec + c0 + 4 * i);
+          cj = make_float4(fmaf(dj.x, 1.0f / D, own), fmaf(dj.y, 1.0f / D, own), fmaf(dj.z, 1.0f / D, own),
+                           fmaf(dj.w, 1.0f / D, own));
+        }
+        d4[i] = make_float4(x.x + cj.x, x.y + cj.y, x.z + cj.z, x.w + cj.w);
+      }
     }
+    if (symmetric) group_bar(bar_id, NG);   // dvec is free again
   };
   // lo scratch <- state - hi(state), this thread's row
   auto split_state = [&](uint32_t col) {
@@ -324,6 +371,45 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     tmem_wait_st();
   };
 
+  Piece pc;
+#pragma unroll 1
+  for (int pi = 0; get_piece<BALANCED>(sp, p.units, nch_unit, blockIdx.x, pi, pc); ++pi) {
+  unit = pc.unit;
+  t_begin = pc.cb * C;
+  T = min(p.T, pc.ce * C) - t_begin;
+  nchunks = pc.ce - pc.cb;
+  from_handoff = t_begin > 0;                      // continues a unit another CTA started
+  const bool to_handoff = t_begin + T < p.T;       // hands the unit over to the CTA that finishes it
+  if (pi > 0) {
+    // every role has finished the previous piece (CTA barrier at its end): all barrier phases
+    // start over, so the per-piece chunk counters keep giving the parities
+    if (tid == 0) {
+      for (int i = 0; i < Cfg::NBAR; ++i)
+        asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&bars[i])) : "memory");
+      for (int s2 = 0; s2 < NSTAGE; ++s2) mbar_init(&raw_full[s2], 1);
+      for (int s2 = 0; s2 < KRING; ++s2) { mbar_init(&k_full[s2], 1); mbar_init(&k_empty[s2], 2); }
+      for (int s2 = 0; s2 < RING; ++s2) { mbar_init(&z_full[s2], 1); mbar_init(&z_empty[s2], 2); }
+      mbar_init(b_z0, 1); mbar_init(b_aupd, 1); mbar_init(b_pr, 1); mbar_init(b_supd, 1);
+      mbar_init(b_lo_s, 1); mbar_init(b_lo_a, 1);
+      mbar_init(b_lo_rdy_a, 1); mbar_init(b_lo_rdy_s, 1); mbar_init(b_ep_rdy, 1);
+      mbar_init_fence();
+    }
+  }
+  if (tid == 0 && from_handoff && !*abort_flag) {
+    // the head of this unit is done once its flag shows this launch's id (bounded wait)
+    bool seen = false;
+    const uint64_t probes = 4ull * wait_limit;
+    for (uint64_t it = 0; it < probes && !seen; ++it) {
+      seen = ld_acquire_gpu(&sched_flags[unit]) == sp.epoch;
+      if (!seen) __nanosleep(64);
+    }
+    if (!seen) {
+      *abort_flag = 1;
+      if (p.status) atomicCAS(p.status, 0, int(VLA_ERR_DEVICE_TIMEOUT));
+    }
+  }
+  __syncthreads();
+
   if (grp == 0) {
     // =====================================================================  group A
     float* Zsf = reinterpret_cast<float*>(abase);            // [4][128] float4: -z_t / delta_t
@@ -337,7 +423,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     float* idl = dlt + C;                                    // [C]  1/delta
     float* nidl = idl + C;                                   // [C] -1/delta
     // w1 = (A 1)[g], the row sum of A, carried along in fp32 (see "centred operands" below)
-    float w1 = state_in(p.A0, 1.0f / p.lambda, Cfg::COL_A);
+    float w1 = state_in(from_handoff ? p.A_T : p.A0, 1.0f / p.lambda, Cfg::COL_A, from_handoff);
 
 #pragma unroll 1
     for (int c = 0; c < nchunks; ++c) {
@@ -461,8 +547,8 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         const float tot1 = warp_reduce_scatter16(sq, lane);
         if ((lane & 1) == 0) ZSp[gw * C + (lane >> 1)] = tot1;
 #ifdef VLA_TC_DUMP
-        if (p.stash_z) for (int t = 0; t < 16; ++t) p.stash_z[(size_t(unit) * T + c * C + t) * D + g] = z[t];
-        if (p.stash_delta && g < 16) p.stash_delta[size_t(unit) * T + c * C + g] = dlt[g];
+        if (p.stash_z) for (int t = 0; t < 16; ++t) p.stash_z[(size_t(unit) * p.T + t_begin + c * C + t) * D + g] = z[t];
+        if (p.stash_delta && g < 16) p.stash_delta[size_t(unit) * p.T + t_begin + c * C + g] = dlt[g];
 #endif
       }
       group_bar(1, NG);
@@ -505,13 +591,13 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     }
     if (nchunks > 0) wait(b_aupd, (nchunks - 1) & 1);
     tc_fence_after();
-    if (p.A_T) state_out(p.A_T, Cfg::COL_A);
+    if (p.A_T) state_out(p.A_T, Cfg::COL_A, w1, true, Zp, 1);
   } else if (grp == 1) {
     // =====================================================================  group S
     float* Epf = reinterpret_cast<float*>(sbase);            // [4][128] float4: e'_t
     float* Epl = Epf + D * C;
     float* ostage = Epl + D * C;                             // [2][C][D]
-    float s1 = state_in(p.S0, 0.0f, Cfg::COL_S);   // (S 1)[g], carried along in fp32
+    float s1 = state_in(from_handoff ? p.S_T : p.S0, 0.0f, Cfg::COL_S, from_handoff);   // (S 1)[g], carried along in fp32
 
 #pragma unroll 1
     for (int c = 0; c < nchunks; ++c) {
@@ -582,7 +668,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         ep[t] = e[t] * scs[t];
         s1 = fmaf(ep[t], ssm[t], s1);          // S 1 after this chunk: += e'_t (z_t . 1)
 #ifdef VLA_TC_DUMP
-        if (p.stash_e) p.stash_e[(size_t(unit) * T + c * C + t) * D + g] = e[t];
+        if (p.stash_e) p.stash_e[(size_t(unit) * p.T + t_begin + c * C + t) * D + g] = e[t];
 #endif
       }
 #pragma unroll
@@ -617,7 +703,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       group_bar(2, NG);
       if (g == 0) {
         mbar_arrive(&k_empty[ks]);
-        bulk_store(p.out + (size_t(unit) * size_t(T) + size_t(c) * C) * D, ostage + size_t(c & 1) * C * D,
+        bulk_store(p.out + (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C) * D, ostage + size_t(c & 1) * C * D,
                    uint32_t(n) * D * sizeof(float));
         bulk_commit();
         mbar_arrive(b_ep_rdy);
@@ -626,7 +712,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     }
     if (nchunks > 0) wait(b_supd, (nchunks - 1) & 1);
     tc_fence_after();
-    if (p.S_T) state_out(p.S_T, Cfg::COL_S);
+    if (p.S_T) state_out(p.S_T, Cfg::COL_S, s1, false, nullptr, 2);
     if (g == 0) bulk_wait_all<0>();
   } else if (grp == 2) {
     // =====================================================================  group P: TMA ring + input prep
@@ -639,7 +725,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
       TIn* dst = raw + size_t(s) * 3 * C * D;
       mbar_arrive_expect_tx(&raw_full[s], 3 * bytes);
-      const size_t tok = size_t(unit) * size_t(T) + size_t(c) * C;
+      const size_t tok = size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
       bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &raw_full[s]);
       bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &raw_full[s]);
       bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &raw_full[s]);
@@ -648,7 +734,11 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue(c);
     // running sum of phi(k), columns 2g and 2g + 1
     float2 zk = make_float2(0.f, 0.f);
-    if (p.z0) zk = *reinterpret_cast<const float2*>(p.z0 + size_t(unit) * D + 2 * g);
+    if (from_handoff) {
+      if (p.zT) zk = __ldcg(reinterpret_cast<const float2*>(p.zT + size_t(unit) * D + 2 * g));
+    } else if (p.z0) {
+      zk = *reinterpret_cast<const float2*>(p.z0 + size_t(unit) * D + 2 * g);
+    }
 
 #pragma unroll 1
     for (int c = 0; c < nchunks; ++c) {
@@ -821,7 +911,24 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       umma_commit(&z_empty[zs]);
       VLA_MARK(5)
     }
+    // the last arrivals this thread asked for have landed (the barriers are re-armed between pieces)
+    if (nchunks > 0) {
+      wait(b_lo_next, (nchunks - 1) & 1);
+      wait(&z_empty[(nchunks - 1) % RING], ((nchunks - 1) / RING) & 1);
+    }
   }
+
+  // end of the piece: every role is done with it (states and key sum stored, MMAs and copies
+  // that touch shared memory complete), so the barriers may be re-armed and, for a unit that is
+  // handed over, the flag may be raised
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (to_handoff && tid == 0) {
+    __threadfence();
+    st_release_gpu(&sched_flags[unit], sp.epoch);
+  }
+  }  // pieces
 
 #ifdef VLA_SECTION_TIMERS
   if (p.dbg && blockIdx.x == 0) {
@@ -842,13 +949,48 @@ template <typename TIn>
 int launch_chunk_tc_t(const ScanParams& p, cudaStream_t st) {
   using Cfg = TcCfg<TIn>;
   static_assert(Cfg::smem_bytes <= 227 * 1024, "tensor-core chunk kernel exceeds the shared memory of one CTA");
-  auto kern = vla_scan_tc_kernel<TIn>;
-  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess) {
+  auto kern = vla_scan_tc_kernel<TIn, false>;       // one CTA per unit
+  auto kern_bal = vla_scan_tc_kernel<TIn, true>;    // persistent grid, units cut at chunks
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess ||
+      cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess) {
     cudaGetLastError();
     return VLA_ERR_CUDA;
   }
-  kern<<<p.units, Cfg::NT, Cfg::smem_bytes, st>>>(p);
-  note_launch("vla_scan_tc_kernel", Cfg::D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, p.units, 0);
+  SchedParams sp;
+  sp.balanced = 0;
+  sp.grid = p.units;
+  sp.epoch = 0;
+  // Balanced schedule, under the conditions of the FMA chunk kernel's: a last partial wave to
+  // fill, all CTAs resident at once (one per SM: a CTA takes the SM's whole tensor memory),
+  // S_T / A_T / zT there to carry the state across a cut, no stream capture (the launch id is
+  // drawn on the host), a free flag slot.
+  cudaStreamCaptureStatus capture = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(st, &capture) != cudaSuccess) {
+    cudaGetLastError();
+    capture = cudaStreamCaptureStatusActive;
+  }
+  int dev = 0, sms = 0;
+  if (capture == cudaStreamCaptureStatusNone && cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) {
+    const bool state_out = p.S_T && p.A_T && (p.zT || (p.flags & VLA_FLAG_IDENTITY_MAP));
+    if (sms > 0 && p.units > sms && p.units % sms != 0 && p.T > 0 && state_out && p.units <= kSchedMaxUnits) {
+      const unsigned int epoch = next_launch_epoch();
+      if (sched_slot_free(epoch)) {
+        sp.balanced = 1;
+        sp.grid = sms;
+        sp.epoch = epoch;
+      }
+    }
+  } else {
+    cudaGetLastError();
+  }
+  if (sp.balanced) {
+    kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+    sched_slot_mark(sp.epoch, st);
+  } else {
+    kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+  }
+  note_launch("vla_scan_tc_kernel", Cfg::D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, sp.grid, sp.balanced);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

@@ -122,6 +122,42 @@ def test_tc_long_sequences_feature_map(T, tol):
     assert max(errs.values()) <= 1e-4, errs
 
 
+@pytest.mark.parametrize("flags", [0, IDENT])
+def test_tc_long_sequence_in_two_calls(flags):
+    """T = 8192 run as 4096 + 4096 with the states carried through S_T / A_T / z_T.  The kernel
+    carries (state . 1) beside the state and re-forms it from the rows of a state it is given,
+    so the states it writes must hold it accurately (the part of A along the all-ones direction
+    is a thousandth of A's entries by then): the continued run stays as close to the oracle as
+    the single call."""
+    w = W.Workload("tc", 1, 2, 128, 8192, "bf16", 45)
+    q, k, v = W.make_inputs(w)
+    ref = run_oracle(q, k, v, 1.0, flags=flags)
+    h = 4096
+    a = run_gpu(q[:, :, :h], k[:, :, :h], v[:, :, :h], 1.0, flags=flags, kernel=TC)
+    b = run_gpu(q[:, :, h:], k[:, :, h:], v[:, :, h:], 1.0, S0=a.S_T, A0=a.A_T, z0=a.z_T, flags=flags, kernel=TC)
+    assert rel_err(torch.cat([a.out, b.out], dim=2), ref.out) <= 1e-4
+    assert rel_err(b.S_T, ref.S_T) <= 1e-4 and rel_err(b.A_T, ref.A_T) <= 1e-4 and rel_err(b.z_T, ref.z_T) <= 1e-4
+
+
+def test_tc_units_cut_across_ctas_match_the_oracle():
+    """More units than SMs with long sequences: the persistent grid cuts most units in two and
+    hands S, A and the key sum over through S_T / A_T / z_T.  A sample of units (cut and whole)
+    against the oracle."""
+    dev = torch.device("cuda:0")
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    w = W.Workload("tc", 1, sms + 37, 128, 2048, "bf16", 46)
+    q, k, v = W.make_inputs(w)
+    r = vla.vla_forward(q.to(dev), k.to(dev), v.to(dev), 1.0, kernel=TC)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0 and "balanced" in vla.last_launch()
+    sel = [0, 1, 2, 3, 50, 51, 100, sms - 1, sms, sms + 36]
+    ref = run_oracle(q[:, sel].contiguous(), k[:, sel].contiguous(), v[:, sel].contiguous(), 1.0)
+    for i, u in enumerate(sel):
+        for name in ("out", "S_T", "A_T", "z_T"):
+            e = rel_err(getattr(r, name)[0, u], getattr(ref, name)[0, i])
+            assert e <= 1e-4, "unit %d %s: %.3e" % (u, name, e)
+
+
 def test_tc_very_long_sequence():
     """T = 65536 at d = 128, one unit, both readings: within the 1e-3 of long sequences (measured
     A_T 1.6e-4: the rank-16 updates accumulate into the state with truncation)."""

@@ -59,8 +59,8 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             pk = json.load(f)
-        return float(pk["hbm_gbs"]), float(pk.get("sm_max_mhz", 1965.0)), "measured"
-    return 6650.0, 1965.0, "fallback"
+        return float(pk["hbm_gbs"]), float(pk.get("sm_max_mhz", 1965.0)), "measured", float(pk.get("bf16_tflops", 1590.0))
+    return 6650.0, 1965.0, "fallback", 1590.0
 
 
 def ncu_traffic_per_token(kernel_key: str):
@@ -264,7 +264,7 @@ def main():
     over = {n: getattr(args, n) for n in ("B", "H", "T") if getattr(args, n) is not None}
     if over:
         w = W.scaled(w, name=w.name + "-resized", **over)
-    hbm_peak, sm_max_mhz, peak_src = measured_peaks()
+    hbm_peak, sm_max_mhz, peak_src, bf16_peak = measured_peaks()
     n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
 
     strong = args.scaling == "strong" and world > 1
@@ -401,13 +401,28 @@ def main():
     achieved_tflops = flops / (launch_ms * 1e-3) / 1e12
     achieved_gbs = byts / (launch_ms * 1e-3) / 1e9
     traffic_pt = ncu_traffic_per_token("%s<%d,%s>" % (launched.split("<")[0], w.d, w.dtype))
-    roof = {"bound": bound, "kernel": launched,
-            "achieved": achieved_tflops if bound == "alu" else achieved_gbs,
-            "peak": fp32_peak_nominal if bound == "alu" else hbm_peak,
-            "unit": "TFLOP/s" if bound == "alu" else "GB/s",
-            "frac": (achieved_tflops / fp32_peak_nominal) if bound == "alu" else achieved_gbs / hbm_peak,
-            "peak_source": ("fp32 FMA: %d SMs x 128 lanes x 2 x %.0f MHz (derived, nominal max clock)"
-                            % (n_sm, sm_max_mhz)) if bound == "alu" else "hbm_gbs of %s" % peak_src,
+    fp32_src = "fp32 FMA: %d SMs x 128 lanes x 2 x %.0f MHz (derived, nominal max clock)" % (n_sm, sm_max_mhz)
+    on_tensor_cores = launched.startswith("vla_scan_tc_kernel")
+    if on_tensor_cores and bound == "alu":
+        # The d x d products of the chunk algebra run as tcgen05.mma kind::tf32, each as three TF32
+        # products (hi*hi, hi*lo, lo*hi) for fp32 accuracy: the peak for the algorithmic flops is
+        # the dense TF32 rate / 3.  TF32 rate = the measured bf16 GEMM rate x the nominal
+        # TF32 : bf16 ratio (1.1 : 2.25 PFLOP/s).
+        tf32_peak = bf16_peak * (1.1 / 2.25)
+        roof = {"bound": "tensor", "kernel": launched, "achieved": achieved_tflops, "peak": tf32_peak / 3.0,
+                "unit": "TFLOP/s", "frac": achieved_tflops / (tf32_peak / 3.0),
+                "peak_source": ("dense TF32 / 3 passes (hi/lo operand pairs): bf16_tflops of %s (%.0f) x 1.1/2.25 / 3"
+                                % (peak_src, bf16_peak)),
+                "fp32_alu_peak": fp32_peak_nominal, "fp32_alu_frac": achieved_tflops / fp32_peak_nominal,
+                "fp32_alu_peak_source": fp32_src}
+    else:
+        roof = {"bound": bound, "kernel": launched,
+                "achieved": achieved_tflops if bound == "alu" else achieved_gbs,
+                "peak": fp32_peak_nominal if bound == "alu" else hbm_peak,
+                "unit": "TFLOP/s" if bound == "alu" else "GB/s",
+                "frac": (achieved_tflops / fp32_peak_nominal) if bound == "alu" else achieved_gbs / hbm_peak,
+                "peak_source": fp32_src if bound == "alu" else "hbm_gbs of %s" % peak_src}
+    roof.update({
             # dram__bytes_read + write of one ncu capture of this kernel, scaled by tokens
             # (profiles/ncu_traffic.txt names the capture)
             "traffic": traffic_pt * w.tokens if traffic_pt else None,
@@ -416,7 +431,7 @@ def main():
             "hbm_achieved_gbs": achieved_gbs, "hbm_peak_gbs": hbm_peak, "hbm_peak_source": peak_src,
             "hbm_frac": achieved_gbs / hbm_peak,
             "launch_ms": launch_ms,
-            "unit_limited_frac_bound": min(w.units, n_sm) / n_sm}
+            "unit_limited_frac_bound": min(w.units, n_sm) / n_sm})
     if clocks and clocks.get("sm_mhz"):
         roof["frac_at_sampled_clock"] = achieved_tflops / (fp32_peak_nominal * clocks["sm_mhz"] / sm_max_mhz)
     # the fp32 FMA rate this device sustains right now (register-only loop in the library),
@@ -530,11 +545,13 @@ def main():
                                               stream=stream, flags=vla.VLA_FLAG_TOKEN_MAJOR), stream, dev, 1, 3)
         per[w.name + "_token_major"] = entry(w, ms, fp32_frac_nominal=frac(w, ms))
         del qt, kt, vt, out_t
-        # the opt-in tensor-core form of the chunk kernel (never the library's own choice)
+        # the fp32-FMA form of the chunk kernel on the same workload (the library's choice at
+        # d = 128 is the tensor-core form)
         if w.d == 128:
-            ms = timed_ms(lambda: vla.vla_forward(qd, kd, vd, w.lam, kernel=vla.VLA_KERNEL_CHUNK_TC, **fwd), stream, dev, 2, 3)
-            per[w.name + "_chunk_tc_opt_in"] = entry(w, ms, fp32_frac_nominal=frac(w, ms),
-                                                     note="tcgen05 kind::tf32, hi/lo operand pairs, states in tensor memory")
+            ms = timed_ms(lambda: vla.vla_forward(qd, kd, vd, w.lam, kernel=vla.VLA_KERNEL_CHUNK, **fwd), stream, dev, 2, 3)
+            per[w.name + "_chunk_fma"] = entry(w, ms, fp32_frac_nominal=frac(w, ms))
+            ms = timed_ms(lambda: vla.vla_forward(qd, kd, vd, w.lam, flags=vla.VLA_FLAG_IDENTITY_MAP, **fwd), stream, dev, 2, 3)
+            per[w.name + "_identity_map"] = entry(w, ms, fp32_frac_nominal=frac(w, ms))
         # single-step decode (T = 1, carried states): bound by moving S and A through HBM once
         wd = W.EXTRA["decode"]
         q2, k2, v2 = [x.to(dev) for x in W.make_inputs(wd)]

@@ -59,12 +59,20 @@ typedef enum { VLA_F32 = 0, VLA_BF16 = 1 } vla_dtype_t;
 enum {
   VLA_FLAG_IDENTITY_MAP = 1u << 0, /* Section 3.1: k_hat = k/||k||, o_t = S_t q_t              */
   VLA_FLAG_CHECK_FINITE = 1u << 1, /* report non-finite delta or ||A_t k_hat|| in opts->status */
-  VLA_FLAG_TOKEN_MAJOR = 1u << 2   /* q, k, v, u and out are [B,T,H,d] (the layout projections write)
+  VLA_FLAG_TOKEN_MAJOR = 1u << 2,  /* q, k, v, u and out are [B,T,H,d] (the layout projections write)
                                       instead of [B,H,T,d] (in vla_backward also d_out and the
                                       gradients of q, k, v, u); the states stay [B,H,d,d].
                                       vla_forward, the host-buffer calls (which then cut large
                                       batches by batch index), vla_backward (d >= 32);
                                       VLA_ERR_UNSUPPORTED elsewhere */
+  VLA_FLAG_LINEAR_ATTENTION = 1u << 3 /* comparison mode, Section 2, Eq. "linear-attn": the additive
+                                      write S_t = S_{t-1} + v_t phi(k_t)^T of linear attention (no
+                                      penalty matrix, no residual), readout as Eq. "output"; with
+                                      VLA_FLAG_IDENTITY_MAP phi is the identity and o_t = S_t q_t.
+                                      A0 is passed through to A_T.  vla_forward and the host-buffer
+                                      calls, every d, on the token kernel; not with opts->u, the
+                                      refresh, or a forced chunk / decode kernel
+                                      (VLA_ERR_UNSUPPORTED) */
 };
 
 /* Which scan kernel runs.  AUTO picks by shape; the others force one (tests, benchmarks). */

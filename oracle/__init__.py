@@ -25,6 +25,7 @@ _LIB_BWD = os.path.join(_HERE, "libvla_oracle_bwd.so")
 
 F32, BF16, F64 = 0, 1, 2
 IDENTITY_MAP = 1
+LINEAR_ATTENTION = 2
 
 _lock = threading.Lock()
 _default = None
@@ -199,6 +200,16 @@ def forward(*args, **kw) -> OracleResult:
 
 def forward_trace(*args, **kw) -> OracleResult:
     return load().forward_trace(*args, **kw)
+
+
+def state_norms(q, k, v, lam, **kw):
+    """Per-step Frobenius norms (||S_t||_F, ||A_t||_F) of one unit, the quantities of the
+    paper's stability experiment (Section 6.2), from the traced oracle.  A diagnostic: the
+    paper's printed trajectory does not reproduce under any stated u (only ||A_0||_F does)."""
+    r = load().forward_trace(q, k, v, lam, **kw)
+    T = r.trace["S"].shape[0]
+    return (np.linalg.norm(r.trace["S"].reshape(T, -1), axis=1),
+            np.linalg.norm(r.trace["A"].reshape(T, -1), axis=1))
 
 
 @dataclass

@@ -2,8 +2,9 @@
  * vla_oracle.c -- CPU oracle for the Variational Linear Attention forward scan.
  *
  * TEST INFRASTRUCTURE ONLY (see vla_oracle.h).  Plain C, fp64, one token at a
- * time, in the order and notation of the paper's Algorithm 1 ("VLAv3
- * sequential forward pass"), with three stated departures:
+ * time: the recurrence of Section 3.3 (Eqs. "sm", "s-update", "output") taken in the
+ * order Algorithm 1 takes its steps, one helper per equation, with three stated
+ * departures from Algorithm 1:
  *   - the projections W_k, W_q, W_v, W_u are not applied: q, k, v (and u when
  *     given) arrive already projected;
  *   - the periodic identity refresh (A += eta*I every 20 steps) is off unless the
@@ -28,6 +29,7 @@
  *                (S_end = S_start P + G) with A at the cuts from matrix inverses.
  *   refresh      u = 0 closed form, step-by-step brute force with matrix inverses,
  *                split invariance with the carried step offset.
+ *   additive     (linear attention, Eq. "linear-attn") direct double sums over s <= t.
  * Absolute output values on random data are otherwise fixed by nothing the
  * paper prints ("parity unpinned" beyond the pins above): this file is the
  * definition the CUDA path is compared with.
@@ -60,94 +62,135 @@ static double dot(const double* a, const double* b, int n) {
   return s;
 }
 
+/* ---- the steps of one token, one helper per equation of Section 3.3 ---- */
+
+/* Feature map and unit key: key_map = phi(k_t) (Algorithm 1) or k_t itself (Section 3.1),
+   key_unit = key_map / max(||key_map||, eps). */
+static void make_unit_key(const void* k, size_t row, int dtype, int identity, double eps, int dk,
+                          double* key_map, double* key_unit) {
+  for (int j = 0; j < dk; ++j) {
+    double raw = load_elem(k, row + j, dtype);
+    key_map[j] = identity ? raw : phi(raw);
+  }
+  double len = sqrt(dot(key_map, key_map, dk));
+  double guard = len > eps ? len : eps;
+  for (int j = 0; j < dk; ++j) key_unit[j] = key_map[j] / guard;
+}
+
+/* Eq. "sm": rank-1 downdate of the inverse penalty by the direction pen.  gain receives
+   A_{t-1} pen; returns delta (clamped at eps as Algorithm 1 does; it is >= 1 for A > 0). */
+static double inverse_penalty_step(double* A, const double* pen, double* gain, int dk, double eps) {
+  for (int i = 0; i < dk; ++i) gain[i] = dot(A + (size_t)i * dk, pen, dk);
+  double delta = 1.0 + dot(pen, gain, dk);
+  if (delta < eps) delta = eps;
+  for (int i = 0; i < dk; ++i)
+    for (int j = 0; j < dk; ++j) A[(size_t)i * dk + j] -= gain[i] * gain[j] / delta;
+  return delta;
+}
+
+/* Eq. "s-update", first half: unit write direction from the POST-update A_t. */
+static void unit_write_direction(const double* A, const double* key_unit, double* write_dir, int dk,
+                                 double eps) {
+  for (int i = 0; i < dk; ++i) write_dir[i] = dot(A + (size_t)i * dk, key_unit, dk);
+  double len = sqrt(dot(write_dir, write_dir, dk));
+  double guard = len > eps ? len : eps;
+  for (int i = 0; i < dk; ++i) write_dir[i] /= guard;
+}
+
+/* Eq. "s-update", second half: resid = v_t - S_{t-1} key_unit, then S += resid write_dir^T. */
+static void residual_write(double* S, const void* v, size_t row_v, int dtype, const double* key_unit,
+                           const double* write_dir, double* resid, int dk, int dv) {
+  for (int i = 0; i < dv; ++i)
+    resid[i] = load_elem(v, row_v + i, dtype) - dot(S + (size_t)i * dk, key_unit, dk);
+  for (int i = 0; i < dv; ++i)
+    for (int j = 0; j < dk; ++j) S[(size_t)i * dk + j] += resid[i] * write_dir[j];
+}
+
+/* Eq. "linear-attn" (Section 2): the additive write S += v_t phi(k_t)^T of linear attention, the
+   comparison mode (no penalty, no residual; the state stores value (x) key, as S does here). */
+static void additive_write(double* S, const void* v, size_t row_v, int dtype, const double* key_map,
+                           double* resid, int dk, int dv) {
+  for (int i = 0; i < dv; ++i) {
+    resid[i] = load_elem(v, row_v + i, dtype);
+    for (int j = 0; j < dk; ++j) S[(size_t)i * dk + j] += resid[i] * key_map[j];
+  }
+}
+
+/* Eq. "output": o_t = S_t phi(q_t) / max(phi(q_t) . z_t, eps) with z_t the key sum INCLUDING token
+   t; with the identity map o_t = S_t q_t.  Returns the denominator used. */
+static double read_out(const double* S, const void* q, size_t row_q, int dtype, int identity, double eps,
+                       const double* key_map, double* key_sum, double* qry_map, double* o, int dk, int dv) {
+  double den = 1.0;
+  for (int j = 0; j < dk; ++j) {
+    double raw = load_elem(q, row_q + j, dtype);
+    qry_map[j] = identity ? raw : phi(raw);
+  }
+  if (!identity) {
+    for (int j = 0; j < dk; ++j) key_sum[j] += key_map[j];
+    den = dot(key_sum, qry_map, dk);
+    if (den < eps) den = eps;
+  }
+  for (int i = 0; i < dv; ++i) o[i] = dot(S + (size_t)i * dk, qry_map, dk) / den;
+  return den;
+}
+
 /*
  * One (b, h) unit.  q,k,u point at this unit's [T, d_k] block, v at [T, d_v].
- * S [d_v*d_k], A [d_k*d_k], zk [d_k] hold the incoming state and are updated
+ * S [d_v*d_k], A [d_k*d_k], key_sum [d_k] hold the incoming state and are updated
  * in place; out is [T, d_v].
  */
 static void scan_unit(const void* q, const void* k, const void* v, const void* u_in,
                       size_t qk_off, size_t v_off, int dtype, int T, int dk, int dv,
-                      unsigned flags, double eps, double* S, double* A, double* zk,
+                      unsigned flags, double eps, double* S, double* A, double* key_sum,
                       double* out, const vla_oracle_trace_t* tr,
                       const vla_oracle_refresh_t* rf) {
   const int identity = (flags & VLA_ORACLE_IDENTITY_MAP) != 0;
-  double* kf = (double*)malloc(sizeof(double) * (size_t)dk);
-  double* khat = (double*)malloc(sizeof(double) * (size_t)dk);
-  double* u = (double*)malloc(sizeof(double) * (size_t)dk);
-  double* zsm = (double*)malloc(sizeof(double) * (size_t)dk);
-  double* alpha = (double*)malloc(sizeof(double) * (size_t)dk);
-  double* qf = (double*)malloc(sizeof(double) * (size_t)dk);
-  double* e = (double*)malloc(sizeof(double) * (size_t)dv);
+  const int additive = (flags & VLA_ORACLE_LINEAR_ATTENTION) != 0;
+  double* key_map = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* key_unit = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* pen = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* gain = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* write_dir = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* qry_map = (double*)malloc(sizeof(double) * (size_t)dk);
+  double* resid = (double*)malloc(sizeof(double) * (size_t)dv);
 
   for (int t = 0; t < T; ++t) {
     const size_t row_k = qk_off + (size_t)t * (size_t)dk;
     const size_t row_v = v_off + (size_t)t * (size_t)dv;
+    double delta = 1.0;
 
-    /* k_feat = ELU(k_raw) + 1 (Algorithm 1) or k_raw itself (Section 3.1) */
-    for (int j = 0; j < dk; ++j) {
-      double kr = load_elem(k, row_k + j, dtype);
-      kf[j] = identity ? kr : phi(kr);
+    make_unit_key(k, row_k, dtype, identity, eps, dk, key_map, key_unit);
+    if (additive) {
+      /* comparison mode: A is not touched, nothing is normalised */
+      for (int j = 0; j < dk; ++j) { pen[j] = 0.0; write_dir[j] = key_map[j]; }
+      additive_write(S, v, row_v, dtype, key_map, resid, dk, dv);
+    } else {
+      /* penalty direction: supplied verbatim, else the unit key (Section 7.1) */
+      for (int j = 0; j < dk; ++j)
+        pen[j] = u_in ? load_elem(u_in, row_k + j, dtype) : key_unit[j];
+      delta = inverse_penalty_step(A, pen, gain, dk, eps);
+      /* periodic refresh of Section 5.3, placed as Algorithm 1 places it: after the downdate of
+         every period-th token of the whole sequence, before the write direction */
+      if (rf && rf->period > 0 && (rf->step_offset + t + 1) % rf->period == 0)
+        for (int i = 0; i < dk; ++i) A[(size_t)i * dk + i] += rf->eta;
+      unit_write_direction(A, key_unit, write_dir, dk, eps);
+      residual_write(S, v, row_v, dtype, key_unit, write_dir, resid, dk, dv);
     }
-    /* k_hat = k_feat / ||k_feat|| */
-    {
-      double nrm = sqrt(dot(kf, kf, dk));
-      double g = nrm > eps ? nrm : eps;
-      for (int j = 0; j < dk; ++j) khat[j] = kf[j] / g;
-    }
-    /* penalty direction: supplied verbatim, else u_t = k_hat_t */
-    for (int j = 0; j < dk; ++j)
-      u[j] = u_in ? load_elem(u_in, row_k + j, dtype) : khat[j];
-
-    /* --- Sherman-Morrison (Eq. "sm") --- */
-    for (int i = 0; i < dk; ++i) zsm[i] = dot(A + (size_t)i * dk, u, dk); /* z = A_{t-1} u */
-    double delta = 1.0 + dot(u, zsm, dk);
-    if (delta < eps) delta = eps; /* Algorithm 1's clamp; inert since delta >= 1 */
-    for (int i = 0; i < dk; ++i)
-      for (int j = 0; j < dk; ++j) A[(size_t)i * dk + j] -= zsm[i] * zsm[j] / delta;
-    /* periodic identity refresh (Algorithm 1: "if t mod period = 0 then A <- A + eta I") */
-    if (rf && rf->period > 0 && (rf->step_offset + t + 1) % rf->period == 0)
-      for (int i = 0; i < dk; ++i) A[(size_t)i * dk + i] += rf->eta;
-
-    /* --- write direction from the POST-update A_t (Eq. "s-update") --- */
-    {
-      for (int i = 0; i < dk; ++i) alpha[i] = dot(A + (size_t)i * dk, khat, dk);
-      double nrm = sqrt(dot(alpha, alpha, dk));
-      double g = nrm > eps ? nrm : eps;
-      for (int i = 0; i < dk; ++i) alpha[i] /= g;
-    }
-
-    /* --- residual state update: e = v - S_{t-1} k_hat ; S += e alpha^T --- */
-    for (int i = 0; i < dv; ++i)
-      e[i] = load_elem(v, row_v + i, dtype) - dot(S + (size_t)i * dk, khat, dk);
-    for (int i = 0; i < dv; ++i)
-      for (int j = 0; j < dk; ++j) S[(size_t)i * dk + j] += e[i] * alpha[j];
-
-    /* --- readout (Eq. "output") --- */
-    double den = 1.0;
-    for (int j = 0; j < dk; ++j) {
-      double qr = load_elem(q, row_k + j, dtype);
-      qf[j] = identity ? qr : phi(qr);
-    }
-    if (!identity) {
-      for (int j = 0; j < dk; ++j) zk[j] += kf[j]; /* z^key includes token t */
-      den = dot(zk, qf, dk);
-      if (den < eps) den = eps;
-    }
-    for (int i = 0; i < dv; ++i)
-      out[(size_t)t * dv + i] = dot(S + (size_t)i * dk, qf, dk) / den;
+    double den = read_out(S, q, row_k, dtype, identity, eps, key_map, key_sum, qry_map,
+                          out + (size_t)t * dv, dk, dv);
 
     if (tr) {
       if (tr->A) memcpy(tr->A + (size_t)t * dk * dk, A, sizeof(double) * (size_t)dk * dk);
       if (tr->S) memcpy(tr->S + (size_t)t * dv * dk, S, sizeof(double) * (size_t)dv * dk);
-      if (tr->khat) memcpy(tr->khat + (size_t)t * dk, khat, sizeof(double) * (size_t)dk);
-      if (tr->u) memcpy(tr->u + (size_t)t * dk, u, sizeof(double) * (size_t)dk);
-      if (tr->alpha) memcpy(tr->alpha + (size_t)t * dk, alpha, sizeof(double) * (size_t)dk);
-      if (tr->e) memcpy(tr->e + (size_t)t * dv, e, sizeof(double) * (size_t)dv);
+      if (tr->khat) memcpy(tr->khat + (size_t)t * dk, key_unit, sizeof(double) * (size_t)dk);
+      if (tr->u) memcpy(tr->u + (size_t)t * dk, pen, sizeof(double) * (size_t)dk);
+      if (tr->alpha) memcpy(tr->alpha + (size_t)t * dk, write_dir, sizeof(double) * (size_t)dk);
+      if (tr->e) memcpy(tr->e + (size_t)t * dv, resid, sizeof(double) * (size_t)dv);
       if (tr->delta) tr->delta[t] = delta;
       if (tr->den) tr->den[t] = den;
     }
   }
-  free(kf); free(khat); free(u); free(zsm); free(alpha); free(qf); free(e);
+  free(key_map); free(key_unit); free(pen); free(gain); free(write_dir); free(qry_map); free(resid);
 }
 
 typedef struct {

@@ -32,7 +32,11 @@ enum { VLA_ORACLE_F32 = 0, VLA_ORACLE_BF16 = 1, VLA_ORACLE_F64 = 2 };
 enum {
   /* Section 3.1 reading: k_hat = k/||k||, o_t = S_t q_t (no feature map, no
      normaliser).  Without it: Algorithm 1 (phi = ELU+1 on k and q, Eq. "output"). */
-  VLA_ORACLE_IDENTITY_MAP = 1u << 0
+  VLA_ORACLE_IDENTITY_MAP = 1u << 0,
+  /* Comparison mode, Section 2, Eq. "linear-attn": S_t = S_{t-1} + v_t phi(k_t)^T (additive write,
+     no penalty matrix, no residual); readout as Eq. "output".  A is passed through untouched;
+     u and the refresh are ignored. */
+  VLA_ORACLE_LINEAR_ATTENTION = 1u << 1
 };
 
 /* Algorithm 1's periodic identity refresh: after the Sherman-Morrison step of the token whose

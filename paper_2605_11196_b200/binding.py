@@ -21,7 +21,7 @@ VLA_ERR_INVALID_ARG, VLA_ERR_UNSUPPORTED, VLA_ERR_ALIGNMENT = -1, -2, -3
 VLA_ERR_CUDA, VLA_ERR_DEVICE_TIMEOUT, VLA_ERR_NONFINITE, VLA_ERR_TOO_LARGE = -4, -5, -6, -7
 VLA_STATIC_SCRATCH_BYTES = 32 << 20
 VLA_F32, VLA_BF16 = 0, 1
-VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE, VLA_FLAG_TOKEN_MAJOR = 1, 2, 4
+VLA_FLAG_IDENTITY_MAP, VLA_FLAG_CHECK_FINITE, VLA_FLAG_TOKEN_MAJOR, VLA_FLAG_LINEAR_ATTENTION = 1, 2, 4, 8
 VLA_KERNEL_AUTO, VLA_KERNEL_TOKEN, VLA_KERNEL_CHUNK, VLA_KERNEL_DECODE, VLA_KERNEL_CHUNK_TC = 0, 1, 2, 3, 4
 
 EXPORTS = ("vla_forward", "vla_forward_host", "vla_forward_host_static", "vla_host_workspace_bytes",

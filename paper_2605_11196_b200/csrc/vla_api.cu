@@ -44,7 +44,8 @@ int resolve_opts(const vla_opts_t* opts, vla_opts_t* r) {
   }
   if (!(r->eps > 0.0f)) r->eps = 1e-4f;
   if (r->qkv_dtype != VLA_F32 && r->qkv_dtype != VLA_BF16) return VLA_ERR_INVALID_ARG;
-  if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE | VLA_FLAG_TOKEN_MAJOR))
+  if (r->flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE | VLA_FLAG_TOKEN_MAJOR |
+                           VLA_FLAG_LINEAR_ATTENTION))
     return VLA_ERR_INVALID_ARG;
   if (r->kernel != VLA_KERNEL_AUTO && r->kernel != VLA_KERNEL_TOKEN && r->kernel != VLA_KERNEL_CHUNK &&
       r->kernel != VLA_KERNEL_DECODE && r->kernel != VLA_KERNEL_CHUNK_TC)
@@ -83,6 +84,12 @@ bool chunk_tc_covers(const ScanParams& p, int d) {
 }
 
 int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {
+  // the linear-attention comparison mode lives in the token kernel (u = k_hat instantiation)
+  if (p.flags & VLA_FLAG_LINEAR_ATTENTION) {
+    if (p.u || p.refresh_period > 0 || (kernel != VLA_KERNEL_AUTO && kernel != VLA_KERNEL_TOKEN))
+      return VLA_ERR_UNSUPPORTED;
+    return vla::launch_token(d, dtype, p, st);
+  }
   if (kernel == VLA_KERNEL_CHUNK_TC)
     return chunk_tc_covers(p, d) ? vla::launch_chunk_tc(d, dtype, p, st) : VLA_ERR_UNSUPPORTED;
   if (kernel == VLA_KERNEL_DECODE && !decode_covers(p, d)) return VLA_ERR_UNSUPPORTED;
@@ -267,7 +274,7 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_, int 
 
   // Few units and scratch memory at hand: cut the sequences into concurrently scanned segments
   if (o.kernel == VLA_KERNEL_AUTO && o.workspace && d_k >= 32 && o.refresh_period <= 0 &&
-      !(o.flags & VLA_FLAG_TOKEN_MAJOR) && T > 0 && T % 16 == 0) {
+      !(o.flags & (VLA_FLAG_TOKEN_MAJOR | VLA_FLAG_LINEAR_ATTENTION)) && T > 0 && T % 16 == 0) {
     const int P = seqpar_choose_segments(units, T, d_k, o.qkv_dtype);
     if (P > 1 && o.workspace_bytes >= seqpar_layout(size_t(units), size_t(T), size_t(d_k), size_t(P)).total)
       return vla_forward_seqpar(q, k, v, lambda_, B, H, T, d_k, d_v, S0, A0, out, S_T, A_T, &o, P, o.workspace,
@@ -493,7 +500,8 @@ int vla_forward_seqpar(const void* q, const void* k, const void* v, float lambda
   if (rc != VLA_OK) return rc;
   rc = check_common(q, k, v, lambda_, B, H, T, d_k, d_v, A0, out);
   if (rc != VLA_OK) return rc;
-  if (d_k < 32 || o.refresh_period > 0 || o.kernel == VLA_KERNEL_TOKEN || (o.flags & VLA_FLAG_TOKEN_MAJOR))
+  if (d_k < 32 || o.refresh_period > 0 || o.kernel == VLA_KERNEL_TOKEN ||
+      (o.flags & (VLA_FLAG_TOKEN_MAJOR | VLA_FLAG_LINEAR_ATTENTION)))
     return VLA_ERR_UNSUPPORTED;
   const void* ptrs[] = {q, k, v, o.u, S0, A0, out, S_T, A_T, o.z0, o.zT};
   for (const void* ptr : ptrs)
@@ -577,6 +585,7 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   // explicit u, the refresh, token-major tensors: the two reverse scans only
   const bool general = o.u || o.refresh_period > 0;
   if ((general || (o.flags & VLA_FLAG_TOKEN_MAJOR)) && d_k < 32) return VLA_ERR_UNSUPPORTED;
+  if (o.flags & VLA_FLAG_LINEAR_ATTENTION) return VLA_ERR_UNSUPPORTED;   // a forward-only comparison mode
   const int units = B * H;
   if (units > 0 && T > 0 && (!dq || !dk || !dv || (o.u && !o.du))) return VLA_ERR_INVALID_ARG;
   const void* ptrs[] = {q, k, v, S0, A0, d_out, dS_T, dA_T, dz_T, dq, dk, dv, dS0, dA0, dz0, o.z0, o.u, o.du};
@@ -671,7 +680,8 @@ int vla_probe_fp32_fma(int iters, float* sink, double* flops, void* stream) {
 
 int vla_query_support(int d_k, int d_v, int qkv_dtype, uint32_t flags) {
   if (qkv_dtype != VLA_F32 && qkv_dtype != VLA_BF16) return VLA_ERR_UNSUPPORTED;
-  if (flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE | VLA_FLAG_TOKEN_MAJOR))
+  if (flags & ~uint32_t(VLA_FLAG_IDENTITY_MAP | VLA_FLAG_CHECK_FINITE | VLA_FLAG_TOKEN_MAJOR |
+                        VLA_FLAG_LINEAR_ATTENTION))
     return VLA_ERR_UNSUPPORTED;
   return shape_supported(d_k, d_v) ? VLA_OK : VLA_ERR_UNSUPPORTED;
 }

@@ -76,6 +76,7 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
   const int unit = blockIdx.x;
   const int T = p.T;
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
+  const bool lin = !HAS_U && (p.flags & VLA_FLAG_LINEAR_ATTENTION) != 0;
   const float eps = p.eps;
   const int nchunks = (T + C - 1) / C;
 
@@ -172,7 +173,8 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
       float ss = kf.x * kf.x + kf.y * kf.y + kf.z * kf.z + kf.w * kf.w;
 #pragma unroll
       for (int off = TOK_LANES / 2; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-      const float inv = 1.0f / fmaxf(sqrtf(ss), eps);
+      // linear-attention mode writes along phi(k) itself: no normalisation
+      const float inv = lin ? 1.0f : 1.0f / fmaxf(sqrtf(ss), eps);
       if (act) {
         reinterpret_cast<float4*>(w_khat + ptok * D)[pc4] =
             make_float4(kf.x * inv, kf.y * inv, kf.z * inv, kf.w * inv);
@@ -245,6 +247,9 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
 
       const float khi = kh[i], qi = qv[i], vi = w_v[t * D + i];
       const float ui = HAS_U ? uv[i] : khi;
+      // Linear attention (Eq. "linear-attn"): the write direction is phi(k_t) itself, which takes
+      // z's place in the exchange below (so that t2 = phi(k).phi(q) and the update adds v phi(k)^T)
+      if (!HAS_U && lin) zi = khi;
 
       // warp partials over its 8 rows (each row's value sits on 4 lanes: offsets 4, 8, 16)
       float s0 = ui * zi;                     // u.z
@@ -268,14 +273,14 @@ __global__ void __launch_bounds__(4 * D) vla_scan_token_kernel(const ScanParams 
       }
       const float delta = fmaxf(1.0f + t0, eps);  // Algorithm 1's clamp; delta >= 1 for A > 0
       const float inv_d = 1.0f / delta;
-      const float ei = vi - pi;                   // e = v - S_{t-1} k_hat
-      const float zs = zi * inv_d;
+      const float ei = lin ? vi : vi - pi;        // e = v - S_{t-1} k_hat (linear attention: no residual)
+      const float zs = lin ? 0.0f : zi * inv_d;   // (linear attention: A is not touched)
       float es, oi;
       const float* wvec;                          // direction alpha is proportional to
       if (!HAS_U) {
         // A_t k_hat = z/delta; alpha = (z/delta) / max(||z||/delta, eps)
         const float nz = sqrtf(t1);
-        const float sc = inv_d / fmaxf(nz * inv_d, eps);
+        const float sc = lin ? 1.0f : inv_d / fmaxf(nz * inv_d, eps);
         es = ei * sc;
         oi = (ri + ei * (t2 * sc)) * inv_den[t];
         wvec = zbuf + b * D;

@@ -473,6 +473,56 @@ def pin_segments_compose_through_a_transfer_scan(orc):
             assert np.abs(np.reshape(seg.A_T, (dk, dk)) - np.reshape(full.A_T, (dk, dk))).max() < 1e-9
 
 
+# --------------------------------------------------------------------------
+# Comparison mode: additive linear attention (Section 2, Eq. "linear-attn")
+# --------------------------------------------------------------------------
+LINATT = 2  # oracle.LINEAR_ATTENTION
+
+
+def pin_linear_attention_is_a_direct_sum(orc):
+    """o_t = sum_{s<=t} v_s (phi(k_s).phi(q_t)) / sum_{s<=t} phi(k_s).phi(q_t), S_T = sum v_s phi(k_s)^T,
+    z_T = sum phi(k_s): written as plain double sums; A is passed through; carried states add on."""
+    for dk, dv, T, seed in [(3, 2, 7, 1), (8, 8, 40, 2), (16, 5, 33, 3)]:
+        q, k, v, g = _rand(seed, T, dk, dv)
+        fk, fq = _phi(k), _phi(q)
+        A0 = np.eye(dk) * 3.0 + 0.1
+        r = orc.forward_trace(q, k, v, 0.7, flags=LINATT, A0=A0)
+        for t in range(T):
+            num = sum(v[s] * (fk[s] @ fq[t]) for s in range(t + 1))
+            den = sum(fk[s] @ fq[t] for s in range(t + 1))
+            assert np.abs(r.out[t] - num / den).max() < 1e-10 * max(1.0, np.abs(num / den).max()), (dk, t)
+        assert np.abs(r.S_T - sum(np.outer(v[s], fk[s]) for s in range(T))).max() < 1e-10
+        assert np.abs(r.z_T - fk.sum(axis=0)).max() < 1e-10
+        assert np.array_equal(r.A_T, A0)                      # no penalty matrix in this mode
+        # carried S0, z0 simply add to the sums; u is ignored
+        S0, z0 = g.standard_normal((dv, dk)), np.abs(g.standard_normal(dk))
+        r2 = orc.forward_trace(q, k, v, 0.7, flags=LINATT, S0=S0, z0=z0, u=g.standard_normal((T, dk)))
+        t = T - 1
+        num = S0 @ fq[t] + sum(v[s] * (fk[s] @ fq[t]) for s in range(T))
+        den = z0 @ fq[t] + sum(fk[s] @ fq[t] for s in range(T))
+        assert np.abs(r2.out[t] - num / den).max() < 1e-10 * max(1.0, np.abs(num / den).max())
+        # with the identity map: S_T = sum v_s k_s^T and o_t = S_t q_t (no normaliser)
+        r3 = orc.forward_trace(q, k, v, 0.7, flags=LINATT | IDENT)
+        assert np.abs(r3.S_T - v.T @ k).max() < 1e-10
+        assert np.abs(r3.out[T - 1] - (v.T @ k) @ q[T - 1]).max() < 1e-9
+
+
+def pin_linear_attention_state_grows_where_vla_stays_bounded(orc):
+    """Section 2's point about the additive update against Proposition 1: on the same random
+    inputs ||S_t||_F of linear attention keeps growing (like sqrt(t) for zero-mean values; O(t) is
+    the paper's bound), while the residual update's levels off far below it."""
+    dk = dv = 16
+    T = 600
+    q, k, v, _ = _rand(11, T, dk, dv)
+    la = orc.forward_trace(q, k, v, 0.1, flags=LINATT)
+    vl = orc.forward_trace(q, k, v, 0.1)
+    nla = np.linalg.norm(la.trace["S"].reshape(T, -1), axis=1)
+    nvl = np.linalg.norm(vl.trace["S"].reshape(T, -1), axis=1)
+    assert nla[-1] > 1.3 * nla[T // 2 - 1] > 1.3 * 1.3 * nla[T // 4 - 1]    # still growing
+    assert nvl[T // 2:].max() < 1.5 * nvl[T // 4:T // 2].max()                # levelled off
+    assert nla[-1] > 10 * nvl[-1]
+
+
 PINS = [pin_A_is_brute_force_inverse, pin_A_invariants, pin_delta_value,
         pin_alpha_from_post_update_A, pin_first_step_closed_form,
         pin_orthonormal_keys_exact_recall, pin_repeated_key,
@@ -480,4 +530,5 @@ PINS = [pin_A_is_brute_force_inverse, pin_A_invariants, pin_delta_value,
         pin_proposition_1, pin_readout, pin_feature_map_values, pin_eps_guards,
         pin_state_carry, pin_units_layout_threads_dtypes, pin_jacobian_spectrum,
         pin_refresh_closed_form_with_zero_u, pin_refresh_step_by_step_brute_force,
-        pin_refresh_state_carry, pin_segments_compose_through_a_transfer_scan]
+        pin_refresh_state_carry, pin_segments_compose_through_a_transfer_scan,
+        pin_linear_attention_is_a_direct_sum, pin_linear_attention_state_grows_where_vla_stays_bounded]

@@ -26,6 +26,9 @@ def run_oracle(q, k, v, lam, u=None, S0=None, A0=None, z0=None, flags=0, eps=1e-
     va, _ = to_oracle_array(v)
     ua = None if u is None else to_oracle_array(u)[0]
     f64 = lambda x: None if x is None else x.detach().cpu().double().numpy()
+    # the library's flag bits -> the oracle's (it knows the two that change the arithmetic)
+    flags = (oracle.IDENTITY_MAP if flags & vla.VLA_FLAG_IDENTITY_MAP else 0) | \
+            (oracle.LINEAR_ATTENTION if flags & vla.VLA_FLAG_LINEAR_ATTENTION else 0)
     return oracle.forward(qa, ka, va, lam, u=ua, in_dtype=dt, S0=f64(S0), A0=f64(A0), z0=f64(z0),
                           flags=flags, eps=eps, n_threads=NTHREADS, refresh=refresh)
 

@@ -511,3 +511,42 @@ def test_zero_penalty_directions_give_the_normalised_delta_rule(kernel, d, dtype
             kh = kf / np.linalg.norm(kf)
             S += np.outer(vv[0, h, t] - S @ kh, kh)
         assert np.abs(got.S_T[0, h].cpu().double().numpy() - S).max() <= 1e-4 * np.abs(S).max()
+
+
+LINATT = vla.VLA_FLAG_LINEAR_ATTENTION
+
+
+@pytest.mark.parametrize("d", [16, 32, 64, 128])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [LINATT, LINATT | IDENT])
+def test_linear_attention_mode(d, dtype, flags):
+    """Section 2, Eq. "linear-attn" as a mode of the same scan: additive write S += v phi(k)^T, the
+    readout of Eq. "output"; A passes through.  Against the oracle (whose additive mode is pinned
+    by direct double sums) with carried S0, z0, and the layouts."""
+    w = _small(d, 83, dtype, units=(2, 3), seed=500 + d)
+    q, k, v = W.make_inputs(w)
+    g = torch.Generator().manual_seed(d)
+    S0 = torch.randn((2, 3, d, d), generator=g) * 0.1
+    z0 = torch.rand((2, 3, d), generator=g)
+    A0 = _spd((2, 3), g, d)
+    errs, got, ref = check_parity(q, k, v, 1.0, 1e-4, S0=S0, A0=A0, z0=z0, flags=flags, label="linear attention d=%d" % d)
+    assert torch.equal(got.A_T.cpu(), A0)                       # no penalty matrix in this mode
+    assert vla.last_launch().startswith("vla_scan_token_kernel")
+    dev = torch.device("cuda:0")
+    tm = lambda x: x.permute(0, 2, 1, 3).contiguous().to(dev)
+    r = vla.vla_forward(tm(q), tm(k), tm(v), 1.0, S0=S0.to(dev), A0=A0.to(dev), z0=z0.to(dev),
+                        flags=flags | TOKEN_MAJOR)
+    torch.cuda.synchronize()
+    assert torch.equal(r.out.permute(0, 2, 1, 3), got.out) and torch.equal(r.S_T, got.S_T)
+
+
+def test_linear_attention_mode_is_refused_where_it_has_no_meaning():
+    dev = torch.device("cuda:0")
+    w = _small(64, 32, "f32")
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    for kw in (dict(u=W.make_u(w).to(dev)), dict(refresh=(20, 1e-3, 0)), dict(kernel=vla.VLA_KERNEL_CHUNK)):
+        with pytest.raises(vla.VlaError) as ei:
+            vla.vla_forward(q, k, v, 1.0, flags=LINATT, **kw)
+        assert ei.value.code == vla.VLA_ERR_UNSUPPORTED
+    with pytest.raises(vla.VlaError):
+        vla.vla_backward(q, k, v, 1.0, torch.zeros_like(q), flags=LINATT)

@@ -378,6 +378,20 @@ def main():
             t_d2h = copy_ms(lambda: dst.copy_(stage[:dst.numel()], non_blocking=True))
             e2e["pcie_h2d_gbs"] = h2d / (t_h2d * 1e-3) / 1e9
             e2e["pcie_d2h_gbs"] = dst.numel() / (t_d2h * 1e-3) / 1e9
+            # both directions at once (what a fully overlapped pipeline sees): the same two copies
+            # on two streams, timed together
+            s2 = torch.cuda.Stream(dev)
+            stage2 = torch.empty(dst.numel(), dtype=torch.uint8, device=dev)
+            def both():
+                s2.wait_stream(stream)
+                with torch.cuda.stream(s2):
+                    dst.copy_(stage2, non_blocking=True)
+                stage[:h2d].copy_(src, non_blocking=True)
+                stream.wait_stream(s2)
+            t_both = copy_ms(both)
+            e2e["pcie_both_directions_ms"] = t_both
+            e2e["frac_of_concurrent_copy_time"] = (t_both * 1e-3) / (job_tokens / e2e["value"])   # copies alone / a whole step
+            del stage2
             floor_s = max(h2d / (e2e["pcie_h2d_gbs"] * 1e9), d2h / (e2e["pcie_d2h_gbs"] * 1e9))
             e2e["copy_bound_tokens_per_s"] = w.tokens / floor_s       # both directions fully overlapped
             e2e["frac_of_copy_bound"] = (e2e["value"] * w.tokens / job_tokens) / e2e["copy_bound_tokens_per_s"]

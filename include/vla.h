@@ -31,7 +31,7 @@
  *   - VLA_STATIC_SCRATCH_BYTES of device memory per GPU for vla_forward_host_static, and its
  *     device address once looked up;
  *   - per host thread, a note of the last kernel launched (vla_last_launch).
- * vla_forward_host creates and destroys three short-lived streams and their events per call.
+ * vla_forward_host creates and destroys its short-lived streams and events per call.
  */
 #ifndef VLA_H
 #define VLA_H
@@ -152,8 +152,9 @@ int vla_forward(const void* q, const void* k, const void* v, float lambda_,
  * enqueues host->device copies, the scan and device->host copies and returns without
  * synchronising; everything is ordered after the work already in `stream`, and `stream`
  * completes only after all of it, so outputs are valid once `stream` has been synchronised.
- * Batches of at least one unit per SM and 64 MB are pipelined in slices of whole units over
- * three short-lived internal streams (copy-in, scan and copy-out of different slices overlap).
+ * Batches that move at least 64 MB are pipelined in up to 32 slices of whole units over
+ * short-lived internal streams (one for every copy-in, one for every copy-out, four for the
+ * scans), so that what stays exposed is the first copy-in and the last scan and copy-out.
  * opts->status, when given, stays a DEVICE pointer.
  */
 int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,

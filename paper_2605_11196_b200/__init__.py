@@ -14,4 +14,4 @@ from .binding import (VLA_BF16, VLA_ERR_ALIGNMENT, VLA_ERR_CUDA, VLA_ERR_DEVICE_
                       measure_fp32_fma_tflops, vla_backward, VlaGrads,
                       backward_workspace_bytes, vla_make_u, last_launch,
                       selftest_wait_timeout)
-from .autograd import vla_scan  # noqa: F401,E402
+from .autograd import vla_scan, check_status  # noqa: F401,E402

@@ -339,72 +339,82 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
   float* dA0 = static_cast<float*>(take(A_b)); float* dAT = static_cast<float*>(take(A_b));
   float* dz0 = static_cast<float*>(take(z_b)); float* dzT = static_cast<float*>(take(z_b));
 
-  // Large batches are cut into slices of whole units that rotate over three internal
-  // streams, so that the copy-in of one slice, the scan of another and the copy-out of a
-  // third overlap (separate copy engines per direction).  Slices keep at least half a unit
-  // per SM; smaller problems run on the caller's stream alone.
+  // Large batches are cut into slices of whole units and pipelined over short-lived internal
+  // streams by role: one stream carries every copy-in back to back (the host->device engine never
+  // waits for anything: each slice has its own part of the workspace), a few streams carry the
+  // scans (a slice has few units, so consecutive slices share the GPU), one stream carries every
+  // copy-out.  Events order a slice's scan after its copy-in and its copy-out after its scan.
+  // What stays exposed is the first copy-in and the last scan and copy-out.  Smaller problems
+  // run on the caller's stream alone.
+  constexpr int kMaxSlices = 32, kScanLanes = 4;
+  const bool token_major = (o.flags & VLA_FLAG_TOKEN_MAJOR) != 0;
   int nslices = 1;
   {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
-      const size_t moved = 2 * qk_b + v_b + o_b;
-      if (moved >= (size_t(64) << 20)) nslices = int(2 * units / size_t(sms));
-      if (nslices < 1) nslices = 1;
-      if (nslices > 8) nslices = 8;
-    } else {
-      cudaGetLastError();
-    }
+    const size_t moved = 2 * qk_b + v_b + o_b;
+    if (moved >= (size_t(64) << 20)) nslices = int(units / 8 < size_t(kMaxSlices) ? units / 8 : size_t(kMaxSlices));
+    if (nslices < 1) nslices = 1;
+    // [B,T,H,d] tensors: a slice is a range of batch indices (contiguous in that layout, and its
+    // units b*H .. are contiguous in the [B,H,...] states), scanned as a batch of its own
+    if (token_major && nslices > B) nslices = B;
   }
-  constexpr int kLanes = 3;
-  cudaStream_t lanes[kLanes] = {st, st, st};
-  cudaEvent_t ev_begin = nullptr, ev_end[kLanes] = {nullptr, nullptr, nullptr};
+  cudaStream_t s_in = st, s_out = st, s_scan[kScanLanes] = {st, st, st, st};
+  cudaEvent_t ev_begin = nullptr, ev_in[kMaxSlices] = {}, ev_scan[kMaxSlices] = {}, ev_done[kScanLanes + 2] = {};
   bool own_streams = false;
-  if (nslices > 1) {
-    own_streams = cudaEventCreateWithFlags(&ev_begin, cudaEventDisableTiming) == cudaSuccess &&
-                  cudaEventRecord(ev_begin, st) == cudaSuccess;
-    for (int i = 0; i < kLanes && own_streams; ++i) {
-      lanes[i] = nullptr;
-      own_streams = cudaStreamCreateWithFlags(&lanes[i], cudaStreamNonBlocking) == cudaSuccess &&
-                    cudaEventCreateWithFlags(&ev_end[i], cudaEventDisableTiming) == cudaSuccess &&
-                    cudaStreamWaitEvent(lanes[i], ev_begin, 0) == cudaSuccess;
+  auto destroy_all = [&]() {
+    if (s_in != st && s_in) cudaStreamDestroy(s_in);
+    if (s_out != st && s_out) cudaStreamDestroy(s_out);
+    for (int i = 0; i < kScanLanes; ++i)
+      if (s_scan[i] != st && s_scan[i]) cudaStreamDestroy(s_scan[i]);
+    if (ev_begin) cudaEventDestroy(ev_begin);
+    for (int i = 0; i < kMaxSlices; ++i) {
+      if (ev_in[i]) cudaEventDestroy(ev_in[i]);
+      if (ev_scan[i]) cudaEventDestroy(ev_scan[i]);
     }
-    if (!own_streams) {   // could not set the lanes up: run everything on the caller's stream
+    for (int i = 0; i < kScanLanes + 2; ++i)
+      if (ev_done[i]) cudaEventDestroy(ev_done[i]);
+  };
+  if (nslices > 1) {
+    auto mk_stream = [&](cudaStream_t* out) {
+      *out = nullptr;
+      return cudaStreamCreateWithFlags(out, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaStreamWaitEvent(*out, ev_begin, 0) == cudaSuccess;
+    };
+    auto mk_event = [&](cudaEvent_t* e) { return cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+    own_streams = mk_event(&ev_begin) && cudaEventRecord(ev_begin, st) == cudaSuccess && mk_stream(&s_in) &&
+                  mk_stream(&s_out);
+    for (int i = 0; i < kScanLanes && own_streams; ++i) own_streams = mk_stream(&s_scan[i]);
+    for (int i = 0; i < nslices && own_streams; ++i) own_streams = mk_event(&ev_in[i]) && mk_event(&ev_scan[i]);
+    for (int i = 0; i < kScanLanes + 2 && own_streams; ++i) own_streams = mk_event(&ev_done[i]);
+    if (!own_streams) {   // could not set the pipeline up: run everything on the caller's stream
       cudaGetLastError();
-      for (int i = 0; i < kLanes; ++i) {
-        if (lanes[i] && lanes[i] != st) cudaStreamDestroy(lanes[i]);
-        if (ev_end[i]) cudaEventDestroy(ev_end[i]);
-        lanes[i] = st;
-        ev_end[i] = nullptr;
-      }
-      if (ev_begin) cudaEventDestroy(ev_begin);
+      destroy_all();
+      s_in = s_out = st;
+      for (int i = 0; i < kScanLanes; ++i) s_scan[i] = st;
       ev_begin = nullptr;
+      for (int i = 0; i < kMaxSlices; ++i) ev_in[i] = ev_scan[i] = nullptr;
+      for (int i = 0; i < kScanLanes + 2; ++i) ev_done[i] = nullptr;
       nslices = 1;
     }
   }
 
-  // [B,T,H,d] tensors: a slice is a range of batch indices (contiguous in that layout, and its
-  // units b*H .. are contiguous in the [B,H,...] states), scanned as a batch of its own
-  const bool token_major = (o.flags & VLA_FLAG_TOKEN_MAJOR) != 0;
-  if (token_major && nslices > B) nslices = B;
   bool bad = false;
   int rc_scan = VLA_OK;
   for (int sl = 0; sl < nslices; ++sl) {
     const size_t u0 = token_major ? size_t(size_t(B) * sl / nslices) * H : units * sl / nslices;
     const size_t u1 = token_major ? size_t(size_t(B) * (sl + 1) / nslices) * H : units * (sl + 1) / nslices;
     const size_t nu = u1 - u0;
-    cudaStream_t ls = lanes[sl % kLanes];
+    cudaStream_t ls = s_scan[sl % kScanLanes];
     auto h2d = [&](void* d, const void* h, size_t per_unit) {
       const size_t off = u0 * per_unit, bytes = nu * per_unit;
       if (bytes && cudaMemcpyAsync(static_cast<unsigned char*>(d) + off,
                                    static_cast<const unsigned char*>(h) + off, bytes,
-                                   cudaMemcpyHostToDevice, ls) != cudaSuccess) bad = true;
+                                   cudaMemcpyHostToDevice, s_in) != cudaSuccess) bad = true;
     };
     auto d2h = [&](void* h, const void* d, size_t per_unit) {
       const size_t off = u0 * per_unit, bytes = nu * per_unit;
       if (bytes && cudaMemcpyAsync(static_cast<unsigned char*>(h) + off,
                                    static_cast<const unsigned char*>(d) + off, bytes,
-                                   cudaMemcpyDeviceToHost, ls) != cudaSuccess) bad = true;
+                                   cudaMemcpyDeviceToHost, s_out) != cudaSuccess) bad = true;
     };
     auto at = [&](void* base, size_t per_unit) {
       return base ? static_cast<void*>(static_cast<unsigned char*>(base) + u0 * per_unit) : nullptr;
@@ -417,6 +427,8 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
     if (A0) h2d(dA0, A0, A_u);
     if (o.z0) h2d(dz0, o.z0, z_u);
     if (bad) break;
+    if (own_streams && (cudaEventRecord(ev_in[sl], s_in) != cudaSuccess ||
+                        cudaStreamWaitEvent(ls, ev_in[sl], 0) != cudaSuccess)) { bad = true; break; }
 
     vla_opts_t od = o;
     od.workspace = nullptr;        // the slices run concurrently: they must not share scratch
@@ -432,6 +444,8 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
                           static_cast<float*>(at(dout, o_u)), static_cast<float*>(at(dST, S_u)),
                           static_cast<float*>(at(dAT, A_u)), &od, ls);
     if (rc_scan != VLA_OK) break;
+    if (own_streams && (cudaEventRecord(ev_scan[sl], ls) != cudaSuccess ||
+                        cudaStreamWaitEvent(s_out, ev_scan[sl], 0) != cudaSuccess)) { bad = true; break; }
     d2h(out, dout, o_u);
     if (S_T) d2h(S_T, dST, S_u);
     if (A_T) d2h(A_T, dAT, A_u);
@@ -439,15 +453,13 @@ int vla_forward_host(const void* q, const void* k, const void* v, float lambda_,
     if (bad) break;
   }
   if (own_streams) {
-    // the caller's stream continues only after every lane has drained; destroying a
+    // the caller's stream continues only after every internal stream has drained; destroying a
     // stream or event with work pending is deferred by the runtime until that work is done
-    for (int i = 0; i < kLanes; ++i) {
-      if (cudaEventRecord(ev_end[i], lanes[i]) != cudaSuccess ||
-          cudaStreamWaitEvent(st, ev_end[i], 0) != cudaSuccess) bad = true;
-      cudaEventDestroy(ev_end[i]);
-      cudaStreamDestroy(lanes[i]);
-    }
-    cudaEventDestroy(ev_begin);
+    cudaStream_t all[kScanLanes + 2] = {s_in, s_out, s_scan[0], s_scan[1], s_scan[2], s_scan[3]};
+    for (int i = 0; i < kScanLanes + 2; ++i)
+      if (cudaEventRecord(ev_done[i], all[i]) != cudaSuccess || cudaStreamWaitEvent(st, ev_done[i], 0) != cudaSuccess)
+        bad = true;
+    destroy_all();
   }
   if (rc_scan != VLA_OK) return rc_scan;
   if (bad) { cudaGetLastError(); return VLA_ERR_CUDA; }

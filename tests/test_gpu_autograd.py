@@ -67,3 +67,21 @@ def test_learned_penalty_directions_train_through_it():
         want = float((ref.du * fd).sum())
         got = float((f64(Wu.grad) * dW).sum())
         assert abs(got - want) <= 2e-3 * max(abs(want), 1e-3), (got, want)
+
+
+def test_device_side_problems_of_vla_scan_are_reported_by_check_status():
+    """vla_scan never synchronises; what a kernel reports on the device (here: a non-finite value
+    under VLA_FLAG_CHECK_FINITE) is read back by check_status(), which clears it."""
+    dev = torch.device("cuda:0")
+    vla.check_status(dev)                               # clean to begin with
+    w = W.Workload("ag", 1, 2, 64, 40, "f32", 9)
+    q, k, v = [x.to(dev) for x in W.make_inputs(w)]
+    vla.vla_scan(q, k, v, 1.0, flags=vla.VLA_FLAG_CHECK_FINITE)
+    vla.check_status(dev)                               # a finite run leaves the word at 0
+    k_bad = k.clone()
+    k_bad[0, 1, 7, 3] = float("nan")
+    vla.vla_scan(q, k_bad, v, 1.0, flags=vla.VLA_FLAG_CHECK_FINITE)
+    with pytest.raises(vla.VlaError) as ei:
+        vla.check_status(dev)
+    assert ei.value.code == vla.VLA_ERR_NONFINITE
+    vla.check_status(dev)                               # cleared

@@ -761,6 +761,19 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
     if (T > 0) close_token(0);
   } else {
     float2 A[R][RP], GA[R][RP];   // GA: the symmetric part
+    // The adjoint sums one update per token; over tens of thousands of tokens the rounding of a
+    // single fp32 accumulator (a random walk of one half-ulp of the SUM per token) reaches 1e-3 of
+    // the early tokens' gradients, whose own scale is far below the sum's.  Two levels: updates go
+    // to a small accumulator that is folded into the large one every kFold tokens, so the large one
+    // is rounded T / kFold times instead of T (d <= 64; at d = 128 the registers are spoken for
+    // and no workload is that long).
+    constexpr bool TWO_LEVEL = D <= 64;
+    constexpr int kFold = 1024;
+    float2 GAs[TWO_LEVEL ? R : 1][TWO_LEVEL ? RP : 1];
+#pragma unroll
+    for (int r = 0; r < (TWO_LEVEL ? R : 1); ++r)
+#pragma unroll
+      for (int m = 0; m < (TWO_LEVEL ? RP : 1); ++m) GAs[r][m] = make_float2(0.f, 0.f);
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       const size_t idx = (size_t(unit) * D + row0 + r) * D + col0;
@@ -788,6 +801,12 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
         for (int m = 0; m < RP; ++m) {
           x0 = bwd_ffma2(GA[r][m], make_float2(zc[2 * m], zc[2 * m + 1]), x0);
           x1 = bwd_ffma2(A[r][m], make_float2(dc[2 * m], dc[2 * m + 1]), x1);
+        }
+        if constexpr (TWO_LEVEL) {
+          float2 xs = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int m = 0; m < RP; ++m) xs = bwd_ffma2(GAs[r][m], make_float2(zc[2 * m], zc[2 * m + 1]), xs);
+          x0.x += xs.x; x0.y += xs.y;
         }
         a0[r] = x0.x + x0.y; a1[r] = x1.x + x1.y;
       }
@@ -846,8 +865,9 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
           const float2 w2 = make_float2(hw, hw), k2 = make_float2(hk, hk), z2 = make_float2(zs, zs);
 #pragma unroll
           for (int m = 0; m < RP; ++m) {
-            GA[r][m] = bwd_ffma2(w2, make_float2(kc[2 * m], kc[2 * m + 1]), GA[r][m]);
-            GA[r][m] = bwd_ffma2(k2, make_float2(wc[2 * m], wc[2 * m + 1]), GA[r][m]);
+            float2& acc = TWO_LEVEL ? GAs[r][m] : GA[r][m];
+            acc = bwd_ffma2(w2, make_float2(kc[2 * m], kc[2 * m + 1]), acc);
+            acc = bwd_ffma2(k2, make_float2(wc[2 * m], wc[2 * m + 1]), acc);
             A[r][m] = bwd_ffma2(z2, make_float2(zc[2 * m], zc[2 * m + 1]), A[r][m]);
           }
           if constexpr (UX) {   // + sym(dz u^T)
@@ -855,8 +875,9 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
             const float2 dz2 = make_float2(hz, hz), u2 = make_float2(hu, hu);
 #pragma unroll
             for (int m = 0; m < RP; ++m) {
-              GA[r][m] = bwd_ffma2(dz2, make_float2(uc[2 * m], uc[2 * m + 1]), GA[r][m]);
-              GA[r][m] = bwd_ffma2(u2, make_float2(dzk[2 * m], dzk[2 * m + 1]), GA[r][m]);
+              float2& acc = TWO_LEVEL ? GAs[r][m] : GA[r][m];
+              acc = bwd_ffma2(dz2, make_float2(uc[2 * m], uc[2 * m + 1]), acc);
+              acc = bwd_ffma2(u2, make_float2(dzk[2 * m], dzk[2 * m + 1]), acc);
             }
             if (refreshed(t)) {   // A_t = (the step) + eta I: take the refresh off the diagonal
 #pragma unroll
@@ -866,6 +887,17 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
               }
             }
           }
+        }
+      }
+      if constexpr (TWO_LEVEL) {
+        if ((t % kFold) == 0) {
+#pragma unroll
+          for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int m = 0; m < RP; ++m) {
+              GA[r][m].x += GAs[r][m].x; GA[r][m].y += GAs[r][m].y;
+              GAs[r][m] = make_float2(0.f, 0.f);
+            }
         }
       }
       if (t >= 1) products(t - 1);

@@ -185,7 +185,8 @@ SeqParLayout seqpar_layout(size_t units, size_t T, size_t D, size_t P) {
 constexpr bool seqpar_tri(int d) { return d <= 64; }
 
 // Segments per unit: as many as fill the device with 2 * units * P scans, P a divisor of the
-// number of 16-token chunks, at least 256 tokens per segment.  1 = not worth cutting.
+// number of 16-token chunks, at least kSeqparMinTokens tokens per segment.  1 = not worth cutting.
+constexpr int kSeqparMinTokens = 64;   // shortest segment worth its Gram matrix, inversion and correction
 int seqpar_choose_segments(int units, int T, int d, int dtype) {
   if (units <= 0 || T <= 0 || T % 16 != 0 || d < 32) return 1;
   const int resident = vla::chunk_resident_ctas(d, dtype, seqpar_tri(d));
@@ -193,7 +194,7 @@ int seqpar_choose_segments(int units, int T, int d, int dtype) {
   const int nch = T / 16;
   int best = 1;
   for (int P = 2; P <= target && P <= nch; ++P)
-    if (nch % P == 0 && T / P >= 256) best = P;
+    if (nch % P == 0 && T / P >= kSeqparMinTokens) best = P;
   return best;
 }
 

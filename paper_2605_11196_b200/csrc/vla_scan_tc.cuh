@@ -65,6 +65,12 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -115,6 +121,9 @@ __device__ __forceinline__ void tf32_split4(float4 x, float4& hi, float4& lo) {
 }
 __device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
 
+#ifndef VLA_TC_LOOP_UNROLL
+#define VLA_TC_LOOP_UNROLL 1
+#endif
 // ---------------------------------------------------------------- configuration
 template <typename TIn>
 struct TcCfg {
@@ -159,7 +168,7 @@ __device__ __forceinline__ void gram16_tc(const float* X, const float* Y, float*
   float2 w2[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) w2[i] = make_float2(0.f, 0.f);
-#pragma unroll
+#pragma unroll 1   // rolled: the chunk loop of all roles together has to stay in the instruction cache
   for (int step = 0; step < 4; ++step) {
     const int f = step * P + part;
     float4 a[4], b[4];
@@ -203,6 +212,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   using Cfg = TcCfg<TIn>;
   constexpr int D = Cfg::D, C = Cfg::C, NG = Cfg::NG, NP = Cfg::NP, CP = Cfg::CP, VP = Cfg::VP;
   constexpr int NSTAGE = Cfg::NSTAGE, KRING = Cfg::KRING, RING = Cfg::RING;
+  constexpr int kLoopUnroll = VLA_TC_LOOP_UNROLL;
 
   extern __shared__ __align__(128) unsigned char smem[];
   TIn* raw = reinterpret_cast<TIn*>(smem);
@@ -230,9 +240,16 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x;
-  const int grp = tid < NG ? 0 : (tid < 2 * NG ? 1 : (tid < 2 * NG + NP ? 2 : 3));   // A, S, prep, MMA issue
-  const int g = tid - (grp == 3 ? 2 * NG + NP : grp * NG);   // thread within its group
-  const int lane = tid & 31, gw = g >> 5;
+  // The warp index is read from lane 0 so that the compiler sees it as uniform over the warp:
+  // the role branches below are then uniform branches, and the warp shuffles inside them are
+  // compiled as plain shuffles (as code the compiler takes for divergent they are several
+  // times longer, and the chunk loop then no longer fits the instruction cache).
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+  constexpr int WA = NG / 32, WP = NP / 32;
+  const int grp = warp < WA ? 0 : (warp < 2 * WA ? 1 : (warp < 2 * WA + WP ? 2 : 3));   // A, S, prep, MMA issue
+  const int gw = warp - (grp == 3 ? 2 * WA + WP : grp * WA);   // warp within its group
+  const int lane = tid & 31;
+  const int g = gw * 32 + lane;                                // thread within its group
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;
   const float eps = p.eps;
   const int nch_unit = (p.T + C - 1) / C;   // chunks per unit
@@ -255,6 +272,9 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   long long tsec[12];
   for (int i = 0; i < 12; ++i) tsec[i] = 0;
   long long tlast = clock64();
+  const long long tk0_ = tlast;
+  unsigned long long tg0_;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tg0_));
 #define VLA_MARK(i) { long long now_ = clock64(); tsec[i] += now_ - tlast; tlast = now_; }
 #else
 #define VLA_MARK(i)
@@ -415,7 +435,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     float* Zsf = reinterpret_cast<float*>(abase);            // [4][128] float4: -z_t / delta_t
     float* Zsl = Zsf + D * C;                                // its lo part
     float* Zp = Zsl + D * C;                                 // [C][D] rows: Z0, then Z
-    float* Ws = Zp + C * D;                                  // [C][CP] K A K^T
+    float* Ws = Zp + C * D;                                  // [C][CP] K A K^T, then its factors
     float* Ls = Ws + C * CP;                                 // [C][CP] unit lower factor
     float* N2p = Ls + C * CP;                                // [4][C]
     float* ZSp = N2p + 4 * C;                                // [4][C] per-warp sums of the entries of z_t
@@ -425,7 +445,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     // w1 = (A 1)[g], the row sum of A, carried along in fp32 (see "centred operands" below)
     float w1 = state_in(from_handoff ? p.A_T : p.A0, 1.0f / p.lambda, Cfg::COL_A, from_handoff);
 
-#pragma unroll 1
+#pragma unroll kLoopUnroll
     for (int c = 0; c < nchunks; ++c) {
       const int ks = c % KRING, zs = c % RING;
       unsigned char* kslot = kslots + size_t(ks) * Cfg::kslot_bytes;
@@ -479,7 +499,10 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       group_bar(1, NG);
       VLA_MARK(4)
 
-      // ---- warp 0: I + W = L diag(delta) L^T
+      // ---- warp 0: I + W = L diag(delta) L^T by elimination, in place: once column s is
+      // eliminated its slots below the diagonal are free, and the row operations applied to the
+      // identity fill them with L^-1.  At the end the row holds L^-1 (left of the diagonal),
+      // delta (on it) and delta_s L[t][s] (right of it).
       if (gw == 0) {
         const int r = lane & 15, h = lane >> 4;
         float m[8];
@@ -497,26 +520,34 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
             const float msj = __shfl_sync(0xffffffffu, m[j], s2 + 16 * h);
             m[j] = fmaf(-l, msj, m[j]);
           }
-          if (h == hs) Ls[r * CP + s2] = l;
+          if (h == hs && r > s2) m[js] = -l;             // (row r of the identity) -= l (row s2 of it)
           if (lane == 0) { dlt[s2] = piv; idl[s2] = ipiv; nidl[s2] = -ipiv; }
         }
+        __syncwarp();
+        *reinterpret_cast<float4*>(Ws + r * CP + h * 8) = make_float4(m[0], m[1], m[2], m[3]);
+        *reinterpret_cast<float4*>(Ws + r * CP + h * 8 + 4) = make_float4(m[4], m[5], m[6], m[7]);
       }
       group_bar(1, NG);
       VLA_MARK(5)
 
-      // ---- row g of Z by forward substitution: z_t = z0_t - sum_{s<t} L[t][s] z_s
+      // ---- row g of Z = Z0 L^-T: z_t = z0_t + sum_{s<t} (L^-1)[t][s] z0_s, sixteen independent sums
+      {
+        float zn[16];
 #pragma unroll
-      for (int t = 1; t < 16; ++t) {
-        float a0 = z[t], a1 = 0.f;
+        for (int t = 0; t < 16; ++t) {
+          float a0 = z[t], a1 = 0.f;
 #pragma unroll
-        for (int s4 = 0; s4 * 4 < t; ++s4) {
-          const float4 l4 = reinterpret_cast<const float4*>(Ls + t * CP)[s4];
-          if (4 * s4 + 0 < t) a0 = fmaf(-l4.x, z[4 * s4 + 0], a0);
-          if (4 * s4 + 1 < t) a1 = fmaf(-l4.y, z[4 * s4 + 1], a1);
-          if (4 * s4 + 2 < t) a0 = fmaf(-l4.z, z[4 * s4 + 2], a0);
-          if (4 * s4 + 3 < t) a1 = fmaf(-l4.w, z[4 * s4 + 3], a1);
+          for (int s4 = 0; s4 * 4 < t; ++s4) {
+            const float4 x4 = reinterpret_cast<const float4*>(Ws + t * CP)[s4];
+            if (4 * s4 + 0 < t) a0 = fmaf(x4.x, z[4 * s4 + 0], a0);
+            if (4 * s4 + 1 < t) a1 = fmaf(x4.y, z[4 * s4 + 1], a1);
+            if (4 * s4 + 2 < t) a0 = fmaf(x4.z, z[4 * s4 + 2], a0);
+            if (4 * s4 + 3 < t) a1 = fmaf(x4.w, z[4 * s4 + 3], a1);
+          }
+          zn[t] = a0 + a1;
         }
-        z[t] = a0 + a1;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) z[t] = zn[t];
       }
       // both rank-16 updates of chunk c - RING have read the Z slot
       if (c >= RING) wait(&z_empty[zs], ((c / RING) + 1) & 1);
@@ -571,12 +602,11 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         if ((p.flags & VLA_FLAG_CHECK_FINITE) && p.status && !isfinite(n2 + d_r))
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
         if (h == 0) scs[r] = sc_r;
-        const float scd = sc_r * d_r;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int s2 = h * 8 + j;
-          const float scd_s = __shfl_sync(0xffffffffu, scd, s2);
-          GuT[r * CP + s2] = (s2 < r) ? scd_s * Ls[r * CP + s2] : 0.0f;
+          const float sc_s = __shfl_sync(0xffffffffu, sc_r, s2);
+          GuT[r * CP + s2] = (s2 < r) ? sc_s * Ws[s2 * CP + r] : 0.0f;   // Ws[s][t] = delta_s L[t][s]
         }
       }
       // ---- HT[t][s] = q_t . z_s
@@ -599,7 +629,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     float* ostage = Epl + D * C;                             // [2][C][D]
     float s1 = state_in(from_handoff ? p.S_T : p.S0, 0.0f, Cfg::COL_S, from_handoff);   // (S 1)[g], carried along in fp32
 
-#pragma unroll 1
+#pragma unroll kLoopUnroll
     for (int c = 0; c < nchunks; ++c) {
       const int n = min(C, T - c * C);
       const int ks = c % KRING, zs = c % RING;
@@ -740,7 +770,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       zk = *reinterpret_cast<const float2*>(p.z0 + size_t(unit) * D + 2 * g);
     }
 
-#pragma unroll 1
+#pragma unroll kLoopUnroll
     for (int c = 0; c < nchunks; ++c) {
       const int s = c % NSTAGE, ks = c % KRING;
       const int n = min(C, T - c * C);
@@ -762,30 +792,31 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       {
         const int tt = 8 * pw + tl;
         const bool act = tt < n;
-        float4 kf[8], qv[8];
+        // pass 1 (rolled; this group has time to spare and the chunk loop of all roles together
+        // has to stay in the instruction cache): widen, feature map, plain rows; phi(k) is
+        // parked in the row of k_hat until its norm is known
         float ss = 0.f, sk = 0.f, sqm = 0.f;
-#pragma unroll
+#pragma unroll 2
         for (int i = 0; i < 8; ++i) {
           const int f = fl + 4 * i;
           float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
-          kf[i] = vv; qv[i] = vv;
+          float4 kf = vv, qv = vv;
           if (act) {
-            kf[i] = load4(rk + tt * D, f);
-            qv[i] = load4(rq + tt * D, f);
+            kf = load4(rk + tt * D, f);
+            qv = load4(rq + tt * D, f);
             vv = load4(rv + tt * D, f);
             if (!ident) {
-              kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
-              kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
-              qv[i].x = phi_fast(qv[i].x); qv[i].y = phi_fast(qv[i].y);
-              qv[i].z = phi_fast(qv[i].z); qv[i].w = phi_fast(qv[i].w);
+              kf.x = phi_fast(kf.x); kf.y = phi_fast(kf.y); kf.z = phi_fast(kf.z); kf.w = phi_fast(kf.w);
+              qv.x = phi_fast(qv.x); qv.y = phi_fast(qv.y); qv.z = phi_fast(qv.z); qv.w = phi_fast(qv.w);
             }
           }
-          reinterpret_cast<float4*>(Qp + tt * VP)[f] = qv[i];
+          reinterpret_cast<float4*>(Kp + tt * VP)[f] = kf;
+          reinterpret_cast<float4*>(Qp + tt * VP)[f] = qv;
           reinterpret_cast<float4*>(Vf + tt * VP)[f] = vv;
-          ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
-          ss = fmaf(kf[i].z, kf[i].z, ss); ss = fmaf(kf[i].w, kf[i].w, ss);
-          sk += (kf[i].x + kf[i].y) + (kf[i].z + kf[i].w);
-          sqm += (qv[i].x + qv[i].y) + (qv[i].z + qv[i].w);
+          ss = fmaf(kf.x, kf.x, ss); ss = fmaf(kf.y, kf.y, ss);
+          ss = fmaf(kf.z, kf.z, ss); ss = fmaf(kf.w, kf.w, ss);
+          sk += (kf.x + kf.y) + (kf.z + kf.w);
+          sqm += (qv.x + qv.y) + (qv.z + qv.w);
         }
         ss += __shfl_xor_sync(0xffffffffu, ss, 8);  ss += __shfl_xor_sync(0xffffffffu, ss, 16);
         sk += __shfl_xor_sync(0xffffffffu, sk, 8);  sk += __shfl_xor_sync(0xffffffffu, sk, 16);
@@ -799,16 +830,19 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         // entries have both signs, and the mean's share, (state . 1) mean(x), is added back in
         // fp32 by the groups, which carry state . 1 along with the state.
         const float mk = sk * inv * (1.0f / D), mq = sqm * (1.0f / D);
-#pragma unroll
+        // pass 2: k_hat, and the centred operand rows in hi/lo pairs (each thread re-reads what it wrote)
+#pragma unroll 2
         for (int i = 0; i < 8; ++i) {
           const int f = fl + 4 * i;
-          const float4 kh = make_float4(kf[i].x * inv, kf[i].y * inv, kf[i].z * inv, kf[i].w * inv);
+          const float4 kf = reinterpret_cast<const float4*>(Kp + tt * VP)[f];
+          const float4 qv = reinterpret_cast<const float4*>(Qp + tt * VP)[f];
+          const float4 kh = make_float4(kf.x * inv, kf.y * inv, kf.z * inv, kf.w * inv);
           reinterpret_cast<float4*>(Kp + tt * VP)[f] = kh;
           float4 hi, lo;
           tf32_split4(make_float4(kh.x - mk, kh.y - mk, kh.z - mk, kh.w - mk), hi, lo);
           KQ4[f * Cfg::KQR + tt] = hi;
           KQ4[f * Cfg::KQR + 32 + tt] = lo;
-          tf32_split4(make_float4(qv[i].x - mq, qv[i].y - mq, qv[i].z - mq, qv[i].w - mq), hi, lo);
+          tf32_split4(make_float4(qv.x - mq, qv.y - mq, qv.z - mq, qv.w - mq), hi, lo);
           KQ4[f * Cfg::KQR + 16 + tt] = hi;
           KQ4[f * Cfg::KQR + 48 + tt] = lo;
         }
@@ -847,12 +881,14 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       VLA_MARK(3)
     }
     if (p.zT) *reinterpret_cast<float2*>(p.zT + size_t(unit) * D + 2 * g) = zk;
-  } else if (lane == 0) {
-    // =====================================================================  MMA issue (lane 0 of two warps)
-    // g == 0 issues for group A, g == 32 for group S.  Per chunk: the state (hi part, read in
-    // place) times the chunk's operand rows; the lo scratch times the same; then the rank-16
-    // update, each a hi*hi + hi*lo + lo*hi triple.
-    const bool forA = g == 0;
+  } else {
+    // =====================================================================  MMA issue (two warps)
+    // Warp 0 of the group issues for group A, warp 1 for group S; the whole warp follows the
+    // barriers and one elected lane issues.  Per chunk: the state (hi part, read in place)
+    // times the chunk's operand rows; the lo scratch times the same; then the rank-16 update,
+    // each a hi*hi + hi*lo + lo*hi triple.
+    const bool forA = gw == 0;
+    const bool leader = elect_one();
     const uint32_t col_state = forA ? Cfg::COL_A : Cfg::COL_S;
     const uint32_t col_acc = forA ? Cfg::COL_Z0 : Cfg::COL_PR;
     // operand rows of a chunk, 16 each: hi(K_hat) | hi(Q_f) | lo(K_hat) | lo(Q_f).
@@ -869,7 +905,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
     const float* Lf = reinterpret_cast<const float*>(forA ? abase : sbase);
     const uint64_t dLf = umma_desc(smem_u32(Lf), 16 * 128, 128);
     const uint64_t dLl = umma_desc(smem_u32(Lf + D * C), 16 * 128, 128);
-#pragma unroll 1
+#pragma unroll kLoopUnroll
     for (int c = 0; c < nchunks; ++c) {
       const int ks = c % KRING, zs = c % RING;
       const uint64_t dKQ = umma_desc(smem_u32(kslots + size_t(ks) * Cfg::kslot_bytes), 16 * Cfg::KQR, 128);
@@ -884,31 +920,38 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       wait(&k_full[ks], (c / KRING) & 1);
       tc_fence_after();
       VLA_MARK(0)
-#pragma unroll
-      for (int j = 0; j < 16; ++j)
-        umma_ts(tbase + col_acc, tbase + col_state + 8 * j, dKQ + uint64_t(j * (2 * Cfg::KQR)), idesc_hi, j > 0);
+      if (leader) {
+#pragma unroll 2
+        for (int j = 0; j < 16; ++j)
+          umma_ts(tbase + col_acc, tbase + col_state + 8 * j, dKQ + uint64_t(j * (2 * Cfg::KQR)), idesc_hi, j > 0);
+      }
       VLA_MARK(1)
       wait(b_lo_rdy, c & 1);
       tc_fence_after();
       VLA_MARK(2)
-#pragma unroll
-      for (int j = 0; j < 16; ++j)
-        umma_ts(tbase + col_acc, tbase + Cfg::COL_LO + 8 * j, dKQ + uint64_t(j * (2 * Cfg::KQR)), idesc_lo, 1);
-      umma_commit(b_prod);
-      umma_commit(b_lo_next);
+      if (leader) {
+#pragma unroll 2
+        for (int j = 0; j < 16; ++j)
+          umma_ts(tbase + col_acc, tbase + Cfg::COL_LO + 8 * j, dKQ + uint64_t(j * (2 * Cfg::KQR)), idesc_lo, 1);
+        umma_commit(b_prod);
+        umma_commit(b_lo_next);
+      }
       VLA_MARK(3)
       if (forA) wait(&z_full[zs], (c / RING) & 1);   // Z, lo(Z), -Z/delta are in shared memory
       else wait(b_ep_rdy, c & 1);                    // so are E' and lo(E') (and Z: group S waited for it)
       tc_fence_after();
       VLA_MARK(4)
+      if (leader) {
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        umma_ss(tbase + col_state, dLf + uint64_t(j * 256), dZf + uint64_t(j * 256), idesc_up, 1);
-        umma_ss(tbase + col_state, dLf + uint64_t(j * 256), dZl + uint64_t(j * 256), idesc_up, 1);
-        umma_ss(tbase + col_state, dLl + uint64_t(j * 256), dZf + uint64_t(j * 256), idesc_up, 1);
+        for (int j = 0; j < 2; ++j) {
+          umma_ss(tbase + col_state, dLf + uint64_t(j * 256), dZf + uint64_t(j * 256), idesc_up, 1);
+          umma_ss(tbase + col_state, dLf + uint64_t(j * 256), dZl + uint64_t(j * 256), idesc_up, 1);
+          umma_ss(tbase + col_state, dLl + uint64_t(j * 256), dZf + uint64_t(j * 256), idesc_up, 1);
+        }
+        umma_commit(b_upd);
+        umma_commit(&z_empty[zs]);
       }
-      umma_commit(b_upd);
-      umma_commit(&z_empty[zs]);
+      __syncwarp();
       VLA_MARK(5)
     }
     // the last arrivals this thread asked for have landed (the barriers are re-armed between pieces)
@@ -931,9 +974,19 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   }  // pieces
 
 #ifdef VLA_SECTION_TIMERS
+  if (p.dbg && tid == 0) {
+    unsigned smid_;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_));
+    p.dbg[96 + 2 * blockIdx.x] = clock64() - tk0_;
+    p.dbg[96 + 2 * blockIdx.x + 1] = smid_;
+  }
   if (p.dbg && blockIdx.x == 0) {
     const int role = tid == 0 ? 0 : tid == 32 ? 1 : tid == NG ? 2 : tid == 2 * NG ? 3 : tid == 2 * NG + NP ? 4
                    : tid == 2 * NG + NP + 32 ? 5 : -1;
+    unsigned long long tg1_;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tg1_));
+    tsec[10] = clock64() - tk0_;
+    tsec[11] = (long long)(tg1_ - tg0_);
     if (role >= 0) for (int i = 0; i < 12; ++i) p.dbg[role * 12 + i] = tsec[i];
   }
 #endif

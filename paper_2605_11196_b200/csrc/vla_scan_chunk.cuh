@@ -296,7 +296,12 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   float* idl = dlt + C;                            // [C]  1/delta
   float* nidl = idl + C;                           // [C] -1/delta
   float* nrs = nidl + C;                           // [C+1] eta * (refreshes before token t of the chunk)
-  const int grp = threadIdx.x / Cfg::NG;   // 0: A, 1: S, 2: transfer scan (TRI)
+  // The warp index is read from lane 0 so that the compiler sees it (and the group derived from
+  // it) as uniform over the warp: the role branches are then uniform branches and the warp
+  // shuffles inside them compile to plain shuffles.  Taken as divergent code they are several
+  // times longer, and the chunk loop then overflows the instruction cache.
+  const int warp_u = __shfl_sync(0xffffffffu, int(threadIdx.x >> 5), 0);
+  const int grp = warp_u / (Cfg::NG / 32);   // 0: A, 1: S, 2: transfer scan (TRI)
   float* sbase = abase + Cfg::a_floats + (grp == 2 ? Cfg::s_floats : 0);
   float* VS = sbase;                // [C][D]  B = V^T - S K^T
   float* R0s = VS + C * D;          // [C][D]
@@ -313,10 +318,11 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ring_empty + RING);
 
   const int tid = threadIdx.x;
-  const bool is_A = tid < NG;
-  const int g = tid - grp * NG;          // thread within its group; also the row it owns
+  const bool is_A = grp == 0;
+  const int gw = warp_u - grp * (NG / 32);   // warp within its group
+  const int lane = tid & 31;
+  const int g = gw * 32 + lane;          // thread within its group; also the row it owns
   const int sbar = 1 + grp;              // named barrier of this S-like group
-  const int lane = g & 31, gw = g >> 5;
   const int cg = g % LPR;                // column group
   const int rb = g / LPR;                // row block: rows rb*TR .. rb*TR+TR-1
   const bool ident = (p.flags & VLA_FLAG_IDENTITY_MAP) != 0;

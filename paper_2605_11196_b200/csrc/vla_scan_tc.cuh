@@ -121,6 +121,12 @@ __device__ __forceinline__ void tf32_split4(float4 x, float4& hi, float4& lo) {
 }
 __device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
 
+#ifndef VLA_TC_GRAM_UNROLL
+#define VLA_TC_GRAM_UNROLL 4
+#endif
+#ifndef VLA_TC_PREP_UNROLL
+#define VLA_TC_PREP_UNROLL 2
+#endif
 #ifndef VLA_TC_LOOP_UNROLL
 #define VLA_TC_LOOP_UNROLL 1
 #endif
@@ -163,12 +169,13 @@ struct TcCfg {
 template <int CP, int XS>
 __device__ __forceinline__ void gram16_tc(const float* X, const float* Y, float* G, int g) {
   constexpr int P = 8;
+  constexpr int kGramUnroll = VLA_TC_GRAM_UNROLL;
   const int tile = g / P, part = g % P;
   const int i0 = (tile >> 2) * 4, j0 = (tile & 3) * 4;
   float2 w2[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) w2[i] = make_float2(0.f, 0.f);
-#pragma unroll 1   // rolled: the chunk loop of all roles together has to stay in the instruction cache
+#pragma unroll kGramUnroll   // rolled: the chunk loop of all roles together has to stay in the instruction cache
   for (int step = 0; step < 4; ++step) {
     const int f = step * P + part;
     float4 a[4], b[4];
@@ -213,6 +220,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   constexpr int D = Cfg::D, C = Cfg::C, NG = Cfg::NG, NP = Cfg::NP, CP = Cfg::CP, VP = Cfg::VP;
   constexpr int NSTAGE = Cfg::NSTAGE, KRING = Cfg::KRING, RING = Cfg::RING;
   constexpr int kLoopUnroll = VLA_TC_LOOP_UNROLL;
+  constexpr int kPrepUnroll = VLA_TC_PREP_UNROLL;
 
   extern __shared__ __align__(128) unsigned char smem[];
   TIn* raw = reinterpret_cast<TIn*>(smem);
@@ -269,8 +277,8 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   };
 
 #ifdef VLA_SECTION_TIMERS
-  long long tsec[12];
-  for (int i = 0; i < 12; ++i) tsec[i] = 0;
+  long long tsec[20];
+  for (int i = 0; i < 20; ++i) tsec[i] = 0;
   long long tlast = clock64();
   const long long tk0_ = tlast;
   unsigned long long tg0_;
@@ -483,13 +491,21 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         tmem_ld16(trow + Cfg::COL_Z0, r0);
         tmem_ld16(trow + Cfg::COL_Z0 + 32, r1);
         tmem_wait_ld();
+        VLA_MARK(10)
+        // (all shared-memory loads before the first store: the compiler cannot tell the arrays
+        // apart and would otherwise wait for each load behind the store before it)
+        float cm[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) cm[t] = ckm[t];
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
           // row g of Z0 = A K^T = A (K - mean)^T + (A 1) mean^T
-          z[t] = fmaf(w1, ckm[t], __uint_as_float(r0[t]) + __uint_as_float(r1[t]));
-          Zp[t * D + g] = z[t];
+          z[t] = fmaf(w1, cm[t], __uint_as_float(r0[t]) + __uint_as_float(r1[t]));
         }
+#pragma unroll
+        for (int t = 0; t < 16; ++t) Zp[t * D + g] = z[t];
       }
+      VLA_MARK(11)
       tc_fence_before();
       group_bar(1, NG);
       VLA_MARK(3)
@@ -549,10 +565,15 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
 #pragma unroll
         for (int t = 0; t < 16; ++t) z[t] = zn[t];
       }
+      VLA_MARK(12)
       // both rank-16 updates of chunk c - RING have read the Z slot
       if (c >= RING) wait(&z_empty[zs], ((c / RING) + 1) & 1);
+      VLA_MARK(13)
       {
         float sq[16];
+        float4 nid[4];
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) nid[k4] = *reinterpret_cast<const float4*>(nidl + 4 * k4);
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
           Zp[t * D + g] = z[t];
@@ -561,7 +582,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
 #pragma unroll
         for (int k4 = 0; k4 < 4; ++k4) {
           const float4 zz = make_float4(z[4 * k4], z[4 * k4 + 1], z[4 * k4 + 2], z[4 * k4 + 3]);
-          const float4 ni = *reinterpret_cast<const float4*>(nidl + 4 * k4);
+          const float4 ni = nid[k4];
           const float4 zsc = make_float4(zz.x * ni.x, zz.y * ni.y, zz.z * ni.z, zz.w * ni.w);
           float4 hi, lo;
           tf32_split4(zz, hi, lo);
@@ -602,13 +623,17 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         if ((p.flags & VLA_FLAG_CHECK_FINITE) && p.status && !isfinite(n2 + d_r))
           atomicCAS(p.status, 0, int(VLA_ERR_NONFINITE));
         if (h == 0) scs[r] = sc_r;
+        float us[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) us[j] = Ws[(h * 8 + j) * CP + r];    // Ws[s][t] = delta_s L[t][s]
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int s2 = h * 8 + j;
           const float sc_s = __shfl_sync(0xffffffffu, sc_r, s2);
-          GuT[r * CP + s2] = (s2 < r) ? sc_s * Ws[s2 * CP + r] : 0.0f;   // Ws[s][t] = delta_s L[t][s]
+          GuT[r * CP + s2] = (s2 < r) ? sc_s * us[j] : 0.0f;
         }
       }
+      VLA_MARK(14)
       // ---- HT[t][s] = q_t . z_s
       gram16_tc<CP, VP>(Qp, Zp, HT, g);
       fence_async_smem();     // Z, lo(Z), -Z/delta: written here, read by the tensor core
@@ -796,7 +821,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         // has to stay in the instruction cache): widen, feature map, plain rows; phi(k) is
         // parked in the row of k_hat until its norm is known
         float ss = 0.f, sk = 0.f, sqm = 0.f;
-#pragma unroll 2
+#pragma unroll kPrepUnroll
         for (int i = 0; i < 8; ++i) {
           const int f = fl + 4 * i;
           float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -831,7 +856,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
         // fp32 by the groups, which carry state . 1 along with the state.
         const float mk = sk * inv * (1.0f / D), mq = sqm * (1.0f / D);
         // pass 2: k_hat, and the centred operand rows in hi/lo pairs (each thread re-reads what it wrote)
-#pragma unroll 2
+#pragma unroll kPrepUnroll
         for (int i = 0; i < 8; ++i) {
           const int f = fl + 4 * i;
           const float4 kf = reinterpret_cast<const float4*>(Kp + tt * VP)[f];
@@ -977,17 +1002,17 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   if (p.dbg && tid == 0) {
     unsigned smid_;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_));
-    p.dbg[96 + 2 * blockIdx.x] = clock64() - tk0_;
-    p.dbg[96 + 2 * blockIdx.x + 1] = smid_;
+    p.dbg[120 + 2 * blockIdx.x] = clock64() - tk0_;
+    p.dbg[120 + 2 * blockIdx.x + 1] = smid_;
   }
   if (p.dbg && blockIdx.x == 0) {
     const int role = tid == 0 ? 0 : tid == 32 ? 1 : tid == NG ? 2 : tid == 2 * NG ? 3 : tid == 2 * NG + NP ? 4
                    : tid == 2 * NG + NP + 32 ? 5 : -1;
     unsigned long long tg1_;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(tg1_));
-    tsec[10] = clock64() - tk0_;
-    tsec[11] = (long long)(tg1_ - tg0_);
-    if (role >= 0) for (int i = 0; i < 12; ++i) p.dbg[role * 12 + i] = tsec[i];
+    tsec[18] = clock64() - tk0_;
+    tsec[19] = (long long)(tg1_ - tg0_);
+    if (role >= 0) for (int i = 0; i < 20; ++i) p.dbg[role * 20 + i] = tsec[i];
   }
 #endif
   tc_fence_before();

@@ -64,7 +64,10 @@ struct ChunkCfg {
   static constexpr int NV = TW / 4;              // float4 operand groups per thread
   static constexpr int NG = D;                   // threads per warp group
   static constexpr int NGROUPS = TRI ? 3 : 2;    // A, S [, transfer scan]
-  static constexpr int NT = NGROUPS * D;         // threads per CTA
+  // d = 32: group A is a single warp, and widening the next chunk's inputs after the
+  // factorisation was a fifth of its chain; there a warp of its own does it
+  static constexpr bool PREPW = D == 32;
+  static constexpr int NT = NGROUPS * D + (PREPW ? 32 : 0);   // threads per CTA
   static constexpr int NWG = D / 32;             // warps per group
   static constexpr int NIN = UT ? 4 : 3;         // q, k, v[, u]
   // raw q/k/v[/u] chunks in flight (fewer on the general path: shared memory is the limit)
@@ -91,7 +94,7 @@ struct ChunkCfg {
   //   VS(B), R0s, Eps | ostage[2] [| GuL, HTL]
   static constexpr size_t smem_bytes = raw_bytes +
       (KRING * kslot_floats + RING * slot_floats + a_floats + (NGROUPS - 1) * s_floats) * sizeof(float) +
-      (NSTAGE + 2 * RING) * sizeof(uint64_t) + 16 + 128;
+      (NSTAGE + 2 * RING + (PREPW ? KRING + 1 : 0)) * sizeof(uint64_t) + 16 + 128;
 };
 
 // Reduce-scatter of NTOK x LPR values over LPR consecutive lanes: on return v[k][0] is the
@@ -256,7 +259,7 @@ static __device__ unsigned int g_sched_flags[kSchedSlots * kSchedMaxUnits];
 // one tiled TMA request per array (box d x 1 x 16 x 1 of the 4-d tensor) through the tensor maps
 // in `maps`; the head-major instantiations take an empty struct there.
 template <int D, typename TIn, bool BALANCED, int UM, bool TRI = false, bool STASH = false, bool TM = false>
-__global__ void __launch_bounds__((TRI ? 3 : 2) * D, (TRI && sizeof(TIn) == 2) ? 2 : 1)
+__global__ void __launch_bounds__((ChunkCfg<D, TIn, UM, TRI>::NT), (TRI && sizeof(TIn) == 2) ? 2 : 1)
 vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
                       const __grid_constant__ typename ChunkMapsArg<TM>::type maps) {
   using Cfg = ChunkCfg<D, TIn, UM, TRI>;
@@ -315,10 +318,13 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   uint64_t* full = bars;                    // [NSTAGE] raw stage filled by TMA
   uint64_t* ring_full = full + NSTAGE;      // [RING] group A published chunk c
   uint64_t* ring_empty = ring_full + RING;  // [RING] group S is done with chunk c
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ring_empty + RING);
+  uint64_t* kfull = ring_empty + RING;      // [KRING] the prep warp has widened chunk c      (PREPW)
+  uint64_t* kgo = kfull + KRING;            // group A: the slot of chunk c + 1 may be written (PREPW)
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ring_empty + RING + (Cfg::PREPW ? KRING + 1 : 0));
 
   const int tid = threadIdx.x;
   const bool is_A = grp == 0;
+  const bool is_P = Cfg::PREPW && grp == Cfg::NGROUPS;   // the prep warp
   const int gw = warp_u - grp * (NG / 32);   // warp within its group
   const int lane = tid & 31;
   const int g = gw * 32 + lane;          // thread within its group; also the row it owns
@@ -414,6 +420,12 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
       mbar_init(&ring_full[r], 1);
       mbar_init(&ring_empty[r], Cfg::NGROUPS - 1);
     }
+    if constexpr (Cfg::PREPW) {
+      for (int r = 0; r <= KRING; ++r) {   // kfull[KRING], kgo
+        if (pi > 0) asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&kfull[r])) : "memory");
+        mbar_init(&kfull[r], 1);
+      }
+    }
     mbar_init_fence();
     if (from_handoff && !*abort_flag) {
       bool seen = false;
@@ -435,7 +447,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   }
 
   // ---- a0: load the state tile
-  {
+  if (!is_P) {
     // a tail piece continues from the state its head left in the caller's output buffers
     // (written by another SM: read past L1)
     const float* src = from_handoff ? (is_A ? p.A_T : p.S_T) : (is_A ? p.A0 : (pscan ? nullptr : p.S0));
@@ -462,90 +474,90 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
     }
   }
 
+  // Input prep of tokens [tok_lo, tok_hi) of chunk c by the warps [w0, w0 + nw): k_hat,
+  // ||phi(k)||, q_f and v as fp32 rows in ring slot c % KRING (zero rows past the end of
+  // the sequence).  tok_lo and tok_hi are multiples of the tokens a warp takes per pass.
+  auto prep_inputs = [&](int c, int w0, int nw, int tok_lo = 0, int tok_hi = Cfg::C) {
+    constexpr int LPT = (D >= 128) ? 16 : 8;   // lanes per token
+    constexpr int NF = D / (4 * LPT);          // float4 groups per lane and tensor
+    constexpr int TPW = 32 / LPT;              // tokens per warp pass
+    const int s = c % NSTAGE;
+    const int n = min(C, T - c * C);
+    wait(&full[s], (c / NSTAGE) & 1);
+    const TIn* rq = raw + (size_t(s) * NIN + 0) * C * D;
+    const TIn* rk = raw + (size_t(s) * NIN + 1) * C * D;
+    const TIn* rv = raw + (size_t(s) * NIN + 2) * C * D;
+    const TIn* ru = raw + (size_t(s) * NIN + (UT ? 3 : 0)) * C * D;
+    float* Uf = Ufs + size_t(c & 1) * C * D;   // penalty directions, verbatim
+    float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
+    float* Qf = Kh + C * D;
+    float* Vf = Qf + C * D;
+    float* nrm = Vf + C * D;
+    const int sub = lane / LPT, pl = lane % LPT;
+    // one token per 8 lanes; `token` does the elementwise work and returns the partial
+    // sum of squares, `finish` normalises once the 8 lanes have been summed
+    auto token = [&](int tt, float4 (&kf)[NF]) -> float {
+      const bool act = tt < n;
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < NF; ++i) {
+        const int f = i * LPT + pl;
+        float4 qf = make_float4(0.f, 0.f, 0.f, 0.f), vv = qf;
+        kf[i] = qf;
+        if (act) {
+          kf[i] = load4(rk + tt * D, f);
+          qf = load4(rq + tt * D, f);
+          if (!pscan_cta) vv = load4(rv + tt * D, f);
+          if (!ident) {
+            kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
+            kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
+            qf.x = phi_fast(qf.x); qf.y = phi_fast(qf.y);
+            qf.z = phi_fast(qf.z); qf.w = phi_fast(qf.w);
+          }
+        }
+        reinterpret_cast<float4*>(Qf + tt * D)[f] = qf;
+        reinterpret_cast<float4*>(Vf + tt * D)[f] = vv;
+        if (UT)
+          reinterpret_cast<float4*>(Uf + tt * D)[f] =
+              act ? load4(ru + tt * D, f) : make_float4(0.f, 0.f, 0.f, 0.f);
+        ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
+        ss = fmaf(kf[i].z, kf[i].z, ss); ss = fmaf(kf[i].w, kf[i].w, ss);
+      }
+      return ss;
+    };
+    auto finish = [&](int tt, float ss, const float4 (&kf)[NF]) {
+      const float nr = fmaxf(sqrt_approx(ss), eps);   // max(||phi(k)||, eps)
+      const float inv = rcp_nr(nr);
+#pragma unroll
+      for (int i = 0; i < NF; ++i)
+        reinterpret_cast<float4*>(Kh + tt * D)[i * LPT + pl] =
+            make_float4(kf[i].x * inv, kf[i].y * inv, kf[i].z * inv, kf[i].w * inv);
+      // phi(k) = k_hat * nrm exactly as the recurrence sees it; 0 for padding rows
+      if (pl == 0) nrm[tt] = (tt < n) ? nr : 0.0f;
+    };
+    // two tokens per lane group and iteration, so that their dependency chains interleave
+    for (int tok0 = tok_lo + (gw - w0) * TPW; tok0 < tok_hi; tok0 += 2 * nw * TPW) {
+      const int ta = tok0 + sub, tb = tok0 + nw * TPW + sub;
+      const bool two = tok0 + nw * TPW < tok_hi;   // warp-uniform
+      float4 ka[NF], kb[NF];
+      float sa = token(ta, ka), sb = 0.f;
+      if (two) sb = token(tb, kb);
+#pragma unroll
+      for (int off = LPT / 2; off >= 1; off >>= 1) {
+        sa += __shfl_xor_sync(0xffffffffu, sa, off);
+        sb += __shfl_xor_sync(0xffffffffu, sb, off);
+      }
+      finish(ta, sa, ka);
+      if (two) finish(tb, sb, kb);
+    }
+  };
+
+  // tokens [0, kPrepSplit) of the next chunk are widened by warps 1.., the rest by warp 0
+  // after the factorisation
+  constexpr int kPrepSplit = (NWG == 1) ? 0 : (NWG == 2) ? 12 : C;
+
   if (is_A) {
     // =====================================================================  group A
-    // Input prep of tokens [tok_lo, tok_hi) of chunk c by the warps [w0, w0 + nw): k_hat,
-    // ||phi(k)||, q_f and v as fp32 rows in ring slot c % KRING (zero rows past the end of
-    // the sequence).  tok_lo and tok_hi are multiples of the tokens a warp takes per pass.
-    auto prep_inputs = [&](int c, int w0, int nw, int tok_lo = 0, int tok_hi = Cfg::C) {
-      constexpr int LPT = (D >= 128) ? 16 : 8;   // lanes per token
-      constexpr int NF = D / (4 * LPT);          // float4 groups per lane and tensor
-      constexpr int TPW = 32 / LPT;              // tokens per warp pass
-      const int s = c % NSTAGE;
-      const int n = min(C, T - c * C);
-      wait(&full[s], (c / NSTAGE) & 1);
-      const TIn* rq = raw + (size_t(s) * NIN + 0) * C * D;
-      const TIn* rk = raw + (size_t(s) * NIN + 1) * C * D;
-      const TIn* rv = raw + (size_t(s) * NIN + 2) * C * D;
-      const TIn* ru = raw + (size_t(s) * NIN + (UT ? 3 : 0)) * C * D;
-      float* Uf = Ufs + size_t(c & 1) * C * D;   // penalty directions, verbatim
-      float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
-      float* Qf = Kh + C * D;
-      float* Vf = Qf + C * D;
-      float* nrm = Vf + C * D;
-      const int sub = lane / LPT, pl = lane % LPT;
-      // one token per 8 lanes; `token` does the elementwise work and returns the partial
-      // sum of squares, `finish` normalises once the 8 lanes have been summed
-      auto token = [&](int tt, float4 (&kf)[NF]) -> float {
-        const bool act = tt < n;
-        float ss = 0.f;
-#pragma unroll
-        for (int i = 0; i < NF; ++i) {
-          const int f = i * LPT + pl;
-          float4 qf = make_float4(0.f, 0.f, 0.f, 0.f), vv = qf;
-          kf[i] = qf;
-          if (act) {
-            kf[i] = load4(rk + tt * D, f);
-            qf = load4(rq + tt * D, f);
-            if (!pscan_cta) vv = load4(rv + tt * D, f);
-            if (!ident) {
-              kf[i].x = phi_fast(kf[i].x); kf[i].y = phi_fast(kf[i].y);
-              kf[i].z = phi_fast(kf[i].z); kf[i].w = phi_fast(kf[i].w);
-              qf.x = phi_fast(qf.x); qf.y = phi_fast(qf.y);
-              qf.z = phi_fast(qf.z); qf.w = phi_fast(qf.w);
-            }
-          }
-          reinterpret_cast<float4*>(Qf + tt * D)[f] = qf;
-          reinterpret_cast<float4*>(Vf + tt * D)[f] = vv;
-          if (UT)
-            reinterpret_cast<float4*>(Uf + tt * D)[f] =
-                act ? load4(ru + tt * D, f) : make_float4(0.f, 0.f, 0.f, 0.f);
-          ss = fmaf(kf[i].x, kf[i].x, ss); ss = fmaf(kf[i].y, kf[i].y, ss);
-          ss = fmaf(kf[i].z, kf[i].z, ss); ss = fmaf(kf[i].w, kf[i].w, ss);
-        }
-        return ss;
-      };
-      auto finish = [&](int tt, float ss, const float4 (&kf)[NF]) {
-        const float nr = fmaxf(sqrt_approx(ss), eps);   // max(||phi(k)||, eps)
-        const float inv = rcp_nr(nr);
-#pragma unroll
-        for (int i = 0; i < NF; ++i)
-          reinterpret_cast<float4*>(Kh + tt * D)[i * LPT + pl] =
-              make_float4(kf[i].x * inv, kf[i].y * inv, kf[i].z * inv, kf[i].w * inv);
-        // phi(k) = k_hat * nrm exactly as the recurrence sees it; 0 for padding rows
-        if (pl == 0) nrm[tt] = (tt < n) ? nr : 0.0f;
-      };
-      // two tokens per lane group and iteration, so that their dependency chains interleave
-      for (int tok0 = tok_lo + (gw - w0) * TPW; tok0 < tok_hi; tok0 += 2 * nw * TPW) {
-        const int ta = tok0 + sub, tb = tok0 + nw * TPW + sub;
-        const bool two = tok0 + nw * TPW < tok_hi;   // warp-uniform
-        float4 ka[NF], kb[NF];
-        float sa = token(ta, ka), sb = 0.f;
-        if (two) sb = token(tb, kb);
-#pragma unroll
-        for (int off = LPT / 2; off >= 1; off >>= 1) {
-          sa += __shfl_xor_sync(0xffffffffu, sa, off);
-          sb += __shfl_xor_sync(0xffffffffu, sb, off);
-        }
-        finish(ta, sa, ka);
-        if (two) finish(tb, sb, kb);
-      }
-    };
-
-    // tokens [0, kPrepSplit) of the next chunk are widened by warps 1.., the rest by warp 0
-    // after the factorisation
-    constexpr int kPrepSplit = (NWG == 1) ? 0 : (NWG == 2) ? 12 : C;
-
     float zk = 0.0f;  // running sum of phi(k), column g
     if (from_handoff) {
       if (p.zT) zk = __ldcg(p.zT + size_t(unit) * D + g);
@@ -558,12 +570,15 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
     const int rfP = rf_on ? p.refresh_period : 1;
     int ph = rf_on ? int((p.step_offset + t_begin) % rfP) : 0;
 
-    if (nchunks > 0) prep_inputs(0, 0, NWG);
-    group_bar(1, NG);
-    if (g == 0 && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
+    if constexpr (!Cfg::PREPW) {
+      if (nchunks > 0) prep_inputs(0, 0, NWG);
+      group_bar(1, NG);
+      if (g == 0 && NSTAGE < nchunks) issue(NSTAGE);   // raw stage 0 is free again
+    }
 
     for (int c = 0; c < nchunks; ++c) {
       const int slot = c % RING;
+      if constexpr (Cfg::PREPW) wait(&kfull[c % KRING], (c / KRING) & 1);   // the prep warp has widened chunk c
       const float* Kh = kring + size_t(c % KRING) * Cfg::kslot_floats;
       const float* Qf = Kh + C * D;
       float* Zs = zring + size_t(slot) * Cfg::slot_floats;
@@ -620,6 +635,9 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
       // Group S must be done with chunk c - RING: that frees Z slot `slot` and, because
       // KRING = RING + 1, the input slot that chunk c + 1 is about to overwrite.
       if (c >= RING) wait(&ring_empty[slot], ((c / RING) + 1) & 1);
+      if constexpr (Cfg::PREPW) {
+        if (g == 0) mbar_arrive(kgo);    // the prep warp may widen chunk c + 1 into that input slot
+      }
       if (gw == NWG - 1 && lane < C) {   // denominators of this chunk into the (now free) slot
         float dd = 0.f;
 #pragma unroll
@@ -687,14 +705,18 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
         VLA_MARK(8)
         // the factorising warp takes the tail of the prep where the other warps would
         // otherwise finish after it (one other warp at d = 64, none at d = 32)
-        if (c + 1 < nchunks && kPrepSplit < C) prep_inputs(c + 1, 0, 1, kPrepSplit, C);
+        if constexpr (!Cfg::PREPW) {
+          if (c + 1 < nchunks && kPrepSplit < C) prep_inputs(c + 1, 0, 1, kPrepSplit, C);
+        }
       } else {
         if (c + 1 < nchunks) prep_inputs(c + 1, 1, NWG - 1, 0, kPrepSplit);
         VLA_MARK(8)
       }
       group_bar(1, NG);
       // the raw stage of chunk c + 1 has been consumed: refill it
-      if (g == 0 && c + 1 + NSTAGE < nchunks) issue(c + 1 + NSTAGE);
+      if constexpr (!Cfg::PREPW) {
+        if (g == 0 && c + 1 + NSTAGE < nchunks) issue(c + 1 + NSTAGE);
+      }
       VLA_MARK(4)
 
       // ---- row g of Z by forward substitution: z_t = z0_t - sum_{s<t} L[t][s] z_s
@@ -778,11 +800,14 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
         if (!HAS_U) {
           const float scd = sc_r * d_r;   // multiplies column r of L
           // lane (r, h) writes GuT[r][h*8 .. h*8+7]: GuT[r][s] = scd_s L[r][s]
+          float lr[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) lr[j] = Ls[r * CP + h * 8 + j];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const int s2 = h * 8 + j;
             const float scd_s = __shfl_sync(0xffffffffu, scd, s2);
-            GuT[r * CP + s2] = (s2 < r) ? scd_s * Ls[r * CP + s2] : 0.0f;
+            GuT[r * CP + s2] = (s2 < r) ? scd_s * lr[j] : 0.0f;
           }
         }
       }
@@ -823,6 +848,19 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
         for (int m = 0; m < NV; ++m)
           reinterpret_cast<float4*>(p.A_T + (size_t(unit) * D + row) * D)[m * LPR + cg] =
               make_float4(st[r][2 * m].x, st[r][2 * m].y, st[r][2 * m + 1].x, st[r][2 * m + 1].y);
+      }
+    }
+  } else if (is_P) {
+    // =====================================================================  prep warp (d = 32)
+    // Chunk c + 1 is widened once group A, in chunk c, has seen group S finish the chunk whose
+    // input slot it takes; the raw stage it consumed is refilled straight away.
+    for (int c = 0; c < nchunks; ++c) {
+      if (c > 0) wait(kgo, (c - 1) & 1);
+      prep_inputs(c, 0, 1);
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&kfull[c % KRING]);
+        if (c + NSTAGE < nchunks) issue(c + NSTAGE);
       }
     }
   } else {
@@ -872,10 +910,17 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
       //       Gu[s][t] e_s = Gm[t][s] e'_s)
       float o[16];
       {
-        float e[16], ep[16];
+        // (every shared-memory load of a loop ahead of its stores: the compiler cannot tell the
+        // arrays apart, and a load that follows a store in program order waits for it)
+        float e[16], ep[16], scv[16];
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
-          float a0 = VS[t * D + g], a1 = 0.f;
+          e[t] = VS[t * D + g];
+          scv[t] = scs[t];
+        }
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          float a0 = e[t], a1 = 0.f;
 #pragma unroll
           for (int s4 = 0; s4 * 4 < t; ++s4) {
             const float4 g4 = reinterpret_cast<const float4*>(Gm + t * CP)[s4];
@@ -885,8 +930,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
             if (4 * s4 + 3 < t) a1 = fmaf(-g4.w, HAS_U ? ep[4 * s4 + 3] : e[4 * s4 + 3], a1);
           }
           e[t] = a0 + a1;
-          ep[t] = e[t] * scs[t];
-          Eps[t * D + g] = ep[t];
+          ep[t] = e[t] * scv[t];
         }
         if (STASH && p.stash_e) {
           float* es = p.stash_e + (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C) * D + g;
@@ -907,12 +951,16 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
           }
           o[t] = a0 + a1;
         }
+#pragma unroll
+        for (int t = 0; t < 16; ++t) o[t] *= inv_den[t];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) Eps[t * D + g] = ep[t];
       }
       group_bar(sbar, NG);  // bulk_wait_read above is ordered before the stage is rewritten
       {
         float* ost = ostage + size_t(c & 1) * C * D;
 #pragma unroll
-        for (int t = 0; t < 16; ++t) ost[t * D + g] = o[t] * inv_den[t];
+        for (int t = 0; t < 16; ++t) ost[t * D + g] = o[t];
       }
       fence_async_smem();
       group_bar(sbar, NG);  // Eps and the out stage complete

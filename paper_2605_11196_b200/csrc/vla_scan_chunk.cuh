@@ -340,6 +340,9 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   // (the caller's limit is read from the parameters where it is needed: no register is spent on
   // it in the FMA loops)
   auto wait = [&](uint64_t* bar, uint32_t parity) {
+    // (a probe costs some 170 clk even when the phase is complete, a look at the abort flag 90
+    // more: the common case pays for the probe only)
+    if (mbar_try_wait(bar, parity)) return;
     if (*abort_flag) return;
     const bool done = p.wait_limit == 0 ? mbar_wait_bounded(bar, parity)
                                         : mbar_wait_bounded(bar, parity, p.wait_limit);

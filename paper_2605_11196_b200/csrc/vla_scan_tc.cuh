@@ -269,6 +269,9 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
 
   const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitProbeLimit;
   auto wait = [&](uint64_t* bar, uint32_t parity) {
+    // one probe costs some 170 clk even when the phase is complete, a look at the abort flag
+    // 90 more: the common case (complete) pays for the probe only
+    if (mbar_try_wait(bar, parity)) return;
     if (*abort_flag) return;
     if (!mbar_wait_bounded(bar, parity, wait_limit)) {
       *abort_flag = 1;
@@ -472,7 +475,6 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       // A is final once the update of the previous chunk has completed
       if (c > 0) wait(b_aupd, (c - 1) & 1);
       VLA_MARK(0)
-      wait(&k_full[ks], (c / KRING) & 1);
       // the lo scratch is free once group S's products of the previous chunk have read it
       if (c > 0) wait(b_lo_a, (c - 1) & 1);
       tc_fence_after();
@@ -482,6 +484,7 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       group_bar(1, NG);
       if (g == 0) mbar_arrive(b_lo_rdy_a);
       VLA_MARK(1)
+      wait(&k_full[ks], (c / KRING) & 1);   // (here it costs nothing: the products are still running)
       wait(b_z0, c & 1);
       tc_fence_after();
       VLA_MARK(2)

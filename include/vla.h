@@ -87,7 +87,7 @@ typedef enum {
   VLA_KERNEL_CHUNK_TC = 4 /* the chunk algebra on the tensor cores (Section 3.4: the chunked recurrence
                            is a chain of dense products): states in tensor memory, TF32 products in
                            hi/lo pairs with fp32 accumulation.  d = 128, u = k_hat, no refresh,
-                           [B,H,T,d] tensors, T >= 1; VLA_ERR_UNSUPPORTED otherwise.  AUTO picks it
+                           [B,H,T,d] or [B,T,H,d] tensors, T >= 1; VLA_ERR_UNSUPPORTED otherwise.  AUTO picks it
                            where it applies (and VLA_KERNEL_CHUNK then forces the fp32-FMA form) */
 } vla_kernel_t;
 

@@ -78,9 +78,9 @@ bool decode_covers(const ScanParams& p, int d) {
   return p.T == 1 && d >= 32 && p.S0 && p.A0 && p.S_T && p.A_T && !p.u && p.refresh_period <= 0;
 }
 
-// The tensor-core form of the chunk kernel: d = 128, u = k_hat, no refresh, head-major tensors.
+// The tensor-core form of the chunk kernel: d = 128, u = k_hat, no refresh; [B,H,T,d] or [B,T,H,d].
 bool chunk_tc_covers(const ScanParams& p, int d) {
-  return d == 128 && !p.u && p.refresh_period <= 0 && !(p.flags & VLA_FLAG_TOKEN_MAJOR) && p.T > 0;
+  return d == 128 && !p.u && p.refresh_period <= 0 && p.T > 0;
 }
 
 int launch(const ScanParams& p, int d, int dtype, int kernel, cudaStream_t st) {

@@ -7,7 +7,9 @@ namespace vla {
 
 int launch_chunk_tc(int d, int dtype, const ScanParams& p, cudaStream_t st) {
   if (d != 128) return VLA_ERR_UNSUPPORTED;
-  return dtype == VLA_F32 ? launch_chunk_tc_t<float>(p, st) : launch_chunk_tc_t<uint16_t>(p, st);
+  if (p.flags & VLA_FLAG_TOKEN_MAJOR)
+    return dtype == VLA_F32 ? launch_chunk_tc_t<float, true>(p, st) : launch_chunk_tc_t<uint16_t, true>(p, st);
+  return dtype == VLA_F32 ? launch_chunk_tc_t<float, false>(p, st) : launch_chunk_tc_t<uint16_t, false>(p, st);
 }
 
 }  // namespace vla

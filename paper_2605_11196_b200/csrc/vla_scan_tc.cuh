@@ -155,7 +155,7 @@ struct TcCfg {
   static constexpr size_t kslot_bytes = kq_bytes + kp_bytes + size_t(C) * VP * 4 + 4 * C * 4;   // + v, nrm, 1/den, means of k_hat and q_f
   static constexpr size_t op16_bytes = size_t(D) * C * 4;           // [4][128] float4: a 128 x 16 operand
   static constexpr size_t zslot_bytes = 2 * op16_bytes + (2 * C * CP + 2 * C) * 4;  // Z, lo(Z), GuT, HT, sc, sums of z_t
-  static constexpr size_t a_bytes = 2 * op16_bytes + size_t(C) * D * 4 + (2 * C * CP + 8 * C + 3 * C) * 4;
+  static constexpr size_t a_bytes = 2 * op16_bytes + size_t(C) * D * 4 + (2 * C * CP + 8 * C + 3 * C) * 4 + 64;   // (+ 64: keeps what follows 128-byte aligned)
   //   -Z/delta, lo | Z0 / Z rows [C][D] | W, L | N2p[4][C], ZSp[4][C] | delta, 1/delta, -1/delta
   static constexpr size_t s_bytes = 2 * op16_bytes + 2 * size_t(C) * D * 4;         // E', lo(E') | out stage [2]
   static constexpr size_t p_bytes = 2 * C * 4;                                      // denp[2][C]
@@ -214,8 +214,11 @@ static __device__ unsigned int g_tc_sched_flags[kSchedSlots * kSchedMaxUnits];
 // cut into equal pieces, and a unit that straddles a cut is started by one CTA (first thing it
 // does) and finished by the next (last thing it does), with S, A, the key sum handed over through
 // the caller's S_T / A_T / zT and a release/acquire flag per unit.
-template <typename TIn, bool BALANCED>
-__global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const ScanParams p, const SchedParams sp) {
+// TM: q, k, v, out are [B, T, H, d]: the 16 rows of a chunk are H * d apart and move as one tiled
+// TMA request per array (rows past T arrive as zeros; the store clips them).
+template <typename TIn, bool BALANCED, bool TM = false>
+__global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(
+    const ScanParams p, const SchedParams sp, const __grid_constant__ typename ChunkMapsArg<TM>::type maps) {
   using Cfg = TcCfg<TIn>;
   constexpr int D = Cfg::D, C = Cfg::C, NG = Cfg::NG, NP = Cfg::NP, CP = Cfg::CP, VP = Cfg::VP;
   constexpr int NSTAGE = Cfg::NSTAGE, KRING = Cfg::KRING, RING = Cfg::RING;
@@ -761,8 +764,13 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       group_bar(2, NG);
       if (g == 0) {
         mbar_arrive(&k_empty[ks]);
-        bulk_store(p.out + (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C) * D, ostage + size_t(c & 1) * C * D,
-                   uint32_t(n) * D * sizeof(float));
+        if constexpr (!TM) {
+          bulk_store(p.out + (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C) * D,
+                     ostage + size_t(c & 1) * C * D, uint32_t(n) * D * sizeof(float));
+        } else {   // rows past T are clipped by the tensor map
+          const int b = unit / p.heads, h = unit - b * p.heads;
+          tma_store_4d(&maps.out, 0, h, t_begin + c * C, b, ostage + size_t(c & 1) * C * D);
+        }
         bulk_commit();
         mbar_arrive(b_ep_rdy);
       }
@@ -782,11 +790,21 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
       const int n = min(C, T - c * C);
       const uint32_t bytes = uint32_t(n) * D * sizeof(TIn);
       TIn* dst = raw + size_t(s) * 3 * C * D;
-      mbar_arrive_expect_tx(&raw_full[s], 3 * bytes);
-      const size_t tok = size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
-      bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &raw_full[s]);
-      bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &raw_full[s]);
-      bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &raw_full[s]);
+      if constexpr (!TM) {
+        mbar_arrive_expect_tx(&raw_full[s], 3 * bytes);
+        const size_t tok = size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C;
+        bulk_load(dst + 0 * C * D, static_cast<const TIn*>(p.q) + tok * D, bytes, &raw_full[s]);
+        bulk_load(dst + 1 * C * D, static_cast<const TIn*>(p.k) + tok * D, bytes, &raw_full[s]);
+        bulk_load(dst + 2 * C * D, static_cast<const TIn*>(p.v) + tok * D, bytes, &raw_full[s]);
+      } else {
+        // rows past T arrive as zeros and count towards the bytes like any other
+        const int b = unit / p.heads, h = unit - b * p.heads, t0 = t_begin + c * C;
+        mbar_arrive_expect_tx(&raw_full[s], 3 * uint32_t(C * D * sizeof(TIn)));
+        tma_load_4d(dst + 0 * C * D, &maps.q, 0, h, t0, b, &raw_full[s]);
+        tma_load_4d(dst + 1 * C * D, &maps.k, 0, h, t0, b, &raw_full[s]);
+        tma_load_4d(dst + 2 * C * D, &maps.v, 0, h, t0, b, &raw_full[s]);
+        (void)bytes;
+      }
     };
     if (g == 0)
       for (int c = 0; c < NSTAGE && c < nchunks; ++c) issue(c);
@@ -1026,16 +1044,25 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(const Sc
   }
 }
 
-template <typename TIn>
+int encode_token_major_maps(const ScanParams& p, int d, int dtype, bool has_u, TokenMajorMaps* maps);
+
+template <typename TIn, bool TM>
 int launch_chunk_tc_t(const ScanParams& p, cudaStream_t st) {
   using Cfg = TcCfg<TIn>;
   static_assert(Cfg::smem_bytes <= 227 * 1024, "tensor-core chunk kernel exceeds the shared memory of one CTA");
-  auto kern = vla_scan_tc_kernel<TIn, false>;       // one CTA per unit
-  auto kern_bal = vla_scan_tc_kernel<TIn, true>;    // persistent grid, units cut at chunks
+  auto kern = vla_scan_tc_kernel<TIn, false, TM>;       // one CTA per unit
+  auto kern_bal = vla_scan_tc_kernel<TIn, true, TM>;    // persistent grid, units cut at chunks
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess ||
       cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess) {
     cudaGetLastError();
     return VLA_ERR_CUDA;
+  }
+  typename ChunkMapsArg<TM>::type maps;
+  if constexpr (TM) {
+    const int rc = encode_token_major_maps(p, Cfg::D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, false, &maps);
+    if (rc != VLA_OK) return rc;
+  } else {
+    maps.unused = 0;
   }
   SchedParams sp;
   sp.balanced = 0;
@@ -1066,10 +1093,10 @@ int launch_chunk_tc_t(const ScanParams& p, cudaStream_t st) {
     cudaGetLastError();
   }
   if (sp.balanced) {
-    kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+    kern_bal<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
     sched_slot_mark(sp.epoch, st);
   } else {
-    kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp);
+    kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
   }
   note_launch("vla_scan_tc_kernel", Cfg::D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, sp.grid, sp.balanced);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;

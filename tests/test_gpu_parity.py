@@ -418,11 +418,12 @@ def test_token_major_long_units_and_where_it_is_refused():
     assert rel_err(r.out.permute(0, 2, 1, 3), ref.out) <= 1e-4
     wb = W.Workload("t", 1, 151, 128, 256 + 5, "bf16", 79)      # more units than resident CTAs
     q, k, v = W.make_inputs(wb)
-    plain = run_gpu(q, k, v, wb.lam, kernel=vla.VLA_KERNEL_CHUNK)   # the same (FMA) kernel, head-major
-    r = vla.vla_forward(tm(q), tm(k), tm(v), wb.lam, flags=TOKEN_MAJOR)
-    torch.cuda.synchronize()
-    assert int(r.status.item()) == 0
-    assert torch.equal(r.out.permute(0, 2, 1, 3), plain.out) and torch.equal(r.A_T, plain.A_T)
+    for kern in (vla.VLA_KERNEL_CHUNK, vla.VLA_KERNEL_AUTO):        # the FMA form, and the library's choice
+        plain = run_gpu(q, k, v, wb.lam, kernel=kern)               # the same kernel, head-major
+        r = vla.vla_forward(tm(q), tm(k), tm(v), wb.lam, flags=TOKEN_MAJOR, kernel=kern)
+        torch.cuda.synchronize()
+        assert int(r.status.item()) == 0
+        assert torch.equal(r.out.permute(0, 2, 1, 3), plain.out) and torch.equal(r.A_T, plain.A_T)
     assert vla.vla_query_support(64, 64, vla.VLA_BF16, TOKEN_MAJOR) == vla.VLA_OK
     w2 = W.Workload("t", 1, 2, 64, 64, "f32", 78)
     q, k, v = [x.to(dev) for x in W.make_inputs(w2)]

@@ -158,6 +158,50 @@ def test_tc_units_cut_across_ctas_match_the_oracle():
             assert e <= 1e-4, "unit %d %s: %.3e" % (u, name, e)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("T", [16, 83, 400])
+def test_tc_token_major_tensors(dtype, T):
+    """[B,T,H,d] tensors (tiled TMA loads and stores; the rows of a ragged last chunk arrive as
+    zeros and are clipped on the way out): bit-identical to the head-major call, and within 1e-4
+    of the oracle; nothing is written outside `out`."""
+    dev = torch.device("cuda:0")
+    w = W.Workload("tc", 2, 3, 128, T, dtype, 60 + T)
+    q, k, v = W.make_inputs(w)
+    tm = lambda x: x.transpose(1, 2).contiguous().to(dev)          # [B,T,H,d]
+    pad = 256
+    buf = torch.full((w.B * T * w.H * 128 + 2 * pad,), -3.5, device=dev)
+    out = buf[pad:-pad].view(w.B, T, w.H, 128)
+    r = vla.vla_forward(tm(q), tm(k), tm(v), 1.0, flags=vla.VLA_FLAG_TOKEN_MAJOR, kernel=TC, out=out)
+    h = run_gpu(q, k, v, 1.0, kernel=TC)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    assert torch.all(buf[:pad] == -3.5) and torch.all(buf[-pad:] == -3.5)
+    assert torch.equal(r.out.transpose(1, 2), h.out)
+    assert torch.equal(r.S_T, h.S_T) and torch.equal(r.A_T, h.A_T) and torch.equal(r.z_T, h.z_T)
+    ref = run_oracle(q, k, v, 1.0)
+    assert rel_err(r.out.transpose(1, 2), ref.out) <= 1e-4 and rel_err(r.S_T, ref.S_T) <= 1e-4
+
+
+def test_tc_token_major_units_cut_across_ctas():
+    """[B,T,H,d] tensors on the persistent grid (more units than SMs): a sample of units against
+    the oracle."""
+    dev = torch.device("cuda:0")
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    H = sms + 21
+    w = W.Workload("tc", 1, H, 128, 1024, "bf16", 61)
+    q, k, v = W.make_inputs(w)
+    tm = lambda x: x.transpose(1, 2).contiguous().to(dev)
+    r = vla.vla_forward(tm(q), tm(k), tm(v), 1.0, flags=vla.VLA_FLAG_TOKEN_MAJOR)
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    assert vla.last_launch().startswith("vla_scan_tc_kernel<128,bf16>") and "balanced" in vla.last_launch()
+    sel = [0, 1, 77, sms - 1, sms, H - 1]
+    ref = run_oracle(q[:, sel].contiguous(), k[:, sel].contiguous(), v[:, sel].contiguous(), 1.0)
+    for i, u in enumerate(sel):
+        assert rel_err(r.out[0, :, u], ref.out[0, i]) <= 1e-4, u
+        assert rel_err(r.S_T[0, u], ref.S_T[0, i]) <= 1e-4 and rel_err(r.A_T[0, u], ref.A_T[0, i]) <= 1e-4
+
+
 def test_tc_very_long_sequence():
     """T = 65536 at d = 128, one unit, both readings: within the 1e-3 of long sequences (measured
     A_T 1.6e-4: the rank-16 updates accumulate into the state with truncation)."""
@@ -169,7 +213,7 @@ def test_tc_very_long_sequence():
 
 def test_auto_picks_the_tc_kernel_where_it_applies():
     """The library's own choice at d = 128 (u = k_hat, no refresh, [B,H,T,d]) is the tensor-core
-    kernel; an explicit u, the refresh or token-major tensors go to the FMA chunk kernel."""
+    kernel ([B,H,T,d] or [B,T,H,d] tensors); an explicit u or the refresh go to the FMA chunk kernel."""
     dev = torch.device("cuda:0")
     w = W.Workload("tc", 1, 3, 128, 96, "bf16", 8)
     q, k, v = [x.to(dev) for x in W.make_inputs(w)]

@@ -64,9 +64,10 @@ struct ChunkCfg {
   static constexpr int NV = TW / 4;              // float4 operand groups per thread
   static constexpr int NG = D;                   // threads per warp group
   static constexpr int NGROUPS = TRI ? 3 : 2;    // A, S [, transfer scan]
-  // d = 32: group A is a single warp, and widening the next chunk's inputs after the
-  // factorisation was a fifth of its chain; there a warp of its own does it
-  static constexpr bool PREPW = D == 32;
+  // d <= 64: group A is one or two warps, and widening the next chunk's inputs around the
+  // factorisation was an eighth to a fifth of its chain; there a warp of its own does it (not in
+  // the three-group kernel at d = 64, whose two CTAs per SM leave it no registers)
+  static constexpr bool PREPW = D == 32 || (D == 64 && !TRI);
   static constexpr int NT = NGROUPS * D + (PREPW ? 32 : 0);   // threads per CTA
   static constexpr int NWG = D / 32;             // warps per group
   static constexpr int NIN = UT ? 4 : 3;         // q, k, v[, u]
@@ -118,7 +119,7 @@ __device__ __forceinline__ void reduce_scatter(float (&v)[NTOK][LPR], int cg) {
 // For every token t of the chunk: sink(t, row g of (state tile) . op[t]).  Two tokens per
 // pass so that the shuffle rounds of the reduce-scatter are paid once per pair, and the
 // reduce-scatter of one pair is issued alongside the FMAs of the next (software pipeline).
-template <int TR, int TW, int LPR, int D, int C, typename Sink>
+template <int TR, int TW, int LPR, int D, int C, bool UNR = false, typename Sink>
 __device__ __forceinline__ void tile_matvec_chunk(const float2 (&st)[TR][TW / 2], const float* op,
                                                   int cg, Sink sink) {
   constexpr int NV = TW / 4;
@@ -150,7 +151,11 @@ __device__ __forceinline__ void tile_matvec_chunk(const float2 (&st)[TR][TW / 2]
   };
   float v[2][LPR];
   pair_partial(0, v);
-#pragma unroll 1
+  // rolled, except (UNR) in the two-group kernel at d = 64: there a group is two warps, one per
+  // scheduler, and what the rolled loop cannot overlap (operand loads behind the previous pair's
+  // stores, the reduce-scatter) was a quarter of group S's chain; at d = 32 and d = 128, and in the
+  // three-group kernel (two CTAs per SM, 146 registers a thread), the longer code costs more than it saves
+#pragma unroll(UNR ? C / 2 : 1)
   for (int t = 2; t < C; t += 2) {
     float vn[2][LPR];
     pair_partial(t, vn);          // independent of the shuffles below: issued together
@@ -270,6 +275,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
   static_assert(!TRI || (D <= 64 && !BALANCED), "three groups: d <= 64, one CTA per unit");
   static_assert(!STASH || !TRI, "the stash: not with the three-group kernel");
   constexpr bool HAS_U = Cfg::GEN;   // general path: a_t = A_t k_hat_t formed explicitly
+  constexpr bool kUnrollMatvec = D == 64 && !TRI;
   constexpr bool UT = Cfg::UT;       // u comes from the caller's tensor
   constexpr int NIN = Cfg::NIN;
   constexpr int C = Cfg::C, TW = Cfg::TW, TR = Cfg::TR, LPR = Cfg::LPR, NV = Cfg::NV;
@@ -619,9 +625,9 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
 
       // ---- Z0 = A U^T (U = K when no u is given); with an explicit u also W0 = A K^T
       const float* Uf = UT ? (Ufs + size_t(c & 1) * C * D) : Kh;
-      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Uf, cg, [&](int t, float x) { Z0s[t * D + g] = x; });
+      tile_matvec_chunk<TR, TW, LPR, D, C, kUnrollMatvec>(st, Uf, cg, [&](int t, float x) { Z0s[t * D + g] = x; });
       if (UT)
-        tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) { W0s[t * D + g] = x; });
+        tile_matvec_chunk<TR, TW, LPR, D, C, kUnrollMatvec>(st, Kh, cg, [&](int t, float x) { W0s[t * D + g] = x; });
       group_bar(1, NG);
       VLA_MARK(1)
 
@@ -712,7 +718,9 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
           if (c + 1 < nchunks && kPrepSplit < C) prep_inputs(c + 1, 0, 1, kPrepSplit, C);
         }
       } else {
-        if (c + 1 < nchunks) prep_inputs(c + 1, 1, NWG - 1, 0, kPrepSplit);
+        if constexpr (!Cfg::PREPW) {
+          if (c + 1 < nchunks) prep_inputs(c + 1, 1, NWG - 1, 0, kPrepSplit);
+        }
         VLA_MARK(8)
       }
       group_bar(1, NG);
@@ -854,7 +862,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
       }
     }
   } else if (is_P) {
-    // =====================================================================  prep warp (d = 32)
+    // =====================================================================  prep warp (d <= 64)
     // Chunk c + 1 is widened once group A, in chunk c, has seen group S finish the chunk whose
     // input slot it takes; the raw stage it consumed is refilled straight away.
     for (int c = 0; c < nchunks; ++c) {
@@ -885,10 +893,10 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
       VLA_MARK(1)
 
       // ---- B = V^T - S K^T and R0 = S Q^T, row g of each
-      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Kh, cg, [&](int t, float x) {
+      tile_matvec_chunk<TR, TW, LPR, D, C, kUnrollMatvec>(st, Kh, cg, [&](int t, float x) {
         VS[t * D + g] = (TRI && pscan ? 0.0f : Vf[t * D + g]) - x;
       });
-      tile_matvec_chunk<TR, TW, LPR, D, C>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
+      tile_matvec_chunk<TR, TW, LPR, D, C, kUnrollMatvec>(st, Qf, cg, [&](int t, float x) { R0s[t * D + g] = x; });
       if (g == 0) bulk_wait_read<1>();  // the out stage of chunk c-2 has left shared memory
       // explicit u: the ring's Z slot carries a_t = A_t k_hat_t; the two small matrices
       // k_hat_t . a_s and q_t . a_s are formed here (for u = k_hat they come from group A)

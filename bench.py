@@ -211,7 +211,7 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def bench_one(vla, w, dev, q, k, v, steps, warmup, stream):
+def bench_one(vla, w, dev, q, k, v, steps, warmup, stream, kernel="auto"):
     """Device-resident timing of `steps` launches; returns (seconds for all steps, per-launch ms list)."""
     qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
     out = torch.empty((w.B, w.H, w.T, w.d), dtype=torch.float32, device=dev)
@@ -219,8 +219,10 @@ def bench_one(vla, w, dev, q, k, v, steps, warmup, stream):
     A_T = torch.empty_like(S_T)
     z_T = torch.empty((w.B, w.H, w.d), dtype=torch.float32, device=dev)
     status = torch.zeros((), dtype=torch.int32, device=dev)
+    kern = {"auto": vla.VLA_KERNEL_AUTO, "token": vla.VLA_KERNEL_TOKEN, "chunk": vla.VLA_KERNEL_CHUNK,
+            "chunk_tc": vla.VLA_KERNEL_CHUNK_TC}[kernel]
     call = lambda: vla.vla_forward(qd, kd, vd, w.lam, out=out, S_T=S_T, A_T=A_T, z_T=z_T,
-                                   status=status, stream=stream)
+                                   status=status, stream=stream, kernel=kern)
     return (qd, kd, vd, out, S_T, A_T, z_T, status), call
 
 
@@ -239,6 +241,8 @@ def main():
     ap.add_argument("--B", type=int, default=None, help="override the workload's batch (profiling cases)")
     ap.add_argument("--H", type=int, default=None, help="override the workload's heads")
     ap.add_argument("--T", type=int, default=None, help="override the workload's sequence length")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "token", "chunk", "chunk_tc"],
+                    help="force a kernel for the headline call (profiling; the default is the library's own choice)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -281,7 +285,7 @@ def main():
         w_full = w
         q, k, v = W.make_inputs(w, rank=rank)
     stream = torch.cuda.Stream(dev)
-    bufs, call = bench_one(vla, w, dev, q, k, v, args.steps, args.warmup, stream)
+    bufs, call = bench_one(vla, w, dev, q, k, v, args.steps, args.warmup, stream, args.kernel)
     qd, kd, vd, out, S_T, A_T, z_T, status = bufs
     in_bytes = 2 if w.dtype == "bf16" else 4
     working_set = 3 * w.tokens * w.d * in_bytes + w.tokens * w.d * 4
@@ -469,7 +473,8 @@ def main():
                        "parallelism": "dp%d over (batch, head) units, no collective%s"
                                       % (world, ", B split %s per rank" % (w.B,) if strong else ""),
                        "l2": ("inputs+outputs %.0f MB > L2" % (working_set / 1e6)) if flush is None
-                             else "L2 flushed between timed steps (256 MB write)"},
+                             else "L2 flushed between timed steps (256 MB write)",
+                       **({"kernel_forced": args.kernel} if args.kernel != "auto" else {})},
             "ns_per_scan_step": 1e6 * launch_ms / w.T,
             "roofline": roof, "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks}
 

@@ -66,6 +66,39 @@ def test_forward_random_calls(seed):
         assert e <= 1e-4, "%s %s rel err %.3e" % (label, name, e)
 
 
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("VLA_FUZZ_TC_SEEDS", "24"))))
+def test_tc_random_calls(seed):
+    """The tensor-core kernel, forced: unit counts on both schedules, ragged lengths, both input
+    types and readings, carried states, either layout."""
+    rng = np.random.default_rng(3000 + seed)
+    B, H = (int(rng.integers(1, 4)), int(rng.integers(1, 6))) if rng.random() < 0.6 else (1, int(rng.choice([149, 163, 301])))
+    T = int(rng.choice([1, 5, 16, 17, 47, 64, 130, 257, 600]))
+    if B * H > 100:
+        T = min(T, 130)
+    dtype = str(rng.choice(["f32", "bf16"]))
+    flags = int(rng.choice([0, vla.VLA_FLAG_IDENTITY_MAP]))
+    lam = float(rng.choice([0.1, 0.5, 1.0, 3.0]))
+    w = W.Workload("f", B, H, 128, T, dtype, 7000 + seed)
+    q, k, v = W.make_inputs(w)
+    S0, A0, z0 = _states(rng, B, H, 128, seed)
+    tmaj = rng.random() < 0.4
+    sel = list(range(H)) if B * H <= 100 else sorted(set(int(x) for x in rng.integers(0, H, 6)) | {0, H - 1})
+    pick = lambda x: None if x is None else x[:, sel].contiguous()
+    ref = run_oracle(pick(q), pick(k), pick(v), lam, S0=pick(S0), A0=pick(A0), z0=pick(z0), flags=flags)
+    mv = lambda x: None if x is None else x.to(DEV)
+    tm = (lambda x: None if x is None else x.permute(0, 2, 1, 3).contiguous().to(DEV)) if tmaj else mv
+    r = vla.vla_forward(tm(q), tm(k), tm(v), lam, S0=mv(S0), A0=mv(A0), z0=mv(z0), kernel=vla.VLA_KERNEL_CHUNK_TC,
+                        flags=flags | (vla.VLA_FLAG_TOKEN_MAJOR if tmaj else 0))
+    torch.cuda.synchronize()
+    assert int(r.status.item()) == 0
+    out = r.out.permute(0, 2, 1, 3) if tmaj else r.out
+    label = "seed %d: B=%d H=%d T=%d %s flags=%d lam=%g tm=%s %s" % (seed, B, H, T, dtype, flags, lam, tmaj, vla.last_launch())
+    for name, got, want in (("o", out[:, sel], ref.out), ("S_T", r.S_T[:, sel], ref.S_T), ("A_T", r.A_T[:, sel], ref.A_T),
+                            ("z_T", r.z_T[:, sel], ref.z_T)):
+        e = rel_err(got, want)
+        assert e <= 1e-4, "%s %s rel err %.3e" % (label, name, e)
+
+
 @pytest.mark.parametrize("seed", range(30))
 def test_backward_random_calls(seed):
     rng = np.random.default_rng(2000 + seed)

@@ -174,12 +174,15 @@ __device__ __forceinline__ void tile_matvec_chunk(const float2 (&st)[TR][TW / 2]
 
 // tile += sum_s scale[s] * coef[s][rows of the tile] (x) vec[s][cols of the tile]   (rank-16
 // update; scale == nullptr means 1)
-template <int TR, int TW, int LPR, int D, int C>
+template <int TR, int TW, int LPR, int D, int C, bool UNR = false>
 __device__ __forceinline__ void tile_rank_update(float2 (&st)[TR][TW / 2], const float* coef,
                                                  const float* vec, const float* scale, int rb,
                                                  int cg) {
   constexpr int NV = TW / 4;
-#pragma unroll 2
+  // (UNR: the two-group kernel at d = 64, as for the mat-vec: eight tokens' operand loads in
+  // flight instead of two; at d = 32 and d = 128 deeper unrolling was slower)
+  constexpr int kRuUnroll = UNR ? 8 : 2;
+#pragma unroll(kRuUnroll)
   for (int s2 = 0; s2 < C; ++s2) {
     const float sc = scale ? scale[s2] : 1.0f;
     float cf[TR];
@@ -833,7 +836,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
       // ---- A <- A - Z diag(1/delta) Z^T
       {
         const float* Zown = HAS_U ? Z0s : Zs;
-        tile_rank_update<TR, TW, LPR, D, C>(st, Zown, Zown, nidl, rb, cg);
+        tile_rank_update<TR, TW, LPR, D, C, kUnrollMatvec>(st, Zown, Zown, nidl, rb, cg);
         if (rf_chunk) {   // + eta I per refresh: the diagonal entries that fall in this tile
 #pragma unroll
           for (int r = 0; r < TR; ++r)
@@ -992,7 +995,7 @@ vla_scan_chunk_kernel(const ScanParams p, const SchedParams sp,
       VLA_MARK(3)
 
       // ---- S <- S + E' Z^T
-      tile_rank_update<TR, TW, LPR, D, C>(st, Eps, Zs, nullptr, rb, cg);
+      tile_rank_update<TR, TW, LPR, D, C, kUnrollMatvec>(st, Eps, Zs, nullptr, rb, cg);
       group_bar(sbar, NG);
       if (g == 0) mbar_arrive(&ring_empty[slot]);
       VLA_MARK(4)

@@ -244,24 +244,34 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
 #pragma unroll
         for (int e = 0; e < EPL; ++e) zkx[e] = nz[e] - nk2[e];
       }
-      ss = warp_sum(ss);
-      zz = warp_sum(zz);
-      og = warp_sum(og);
-      const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
-      const float idl = 1.0f / pdelta;
-      const float sc = UX ? 1.0f / fmaxf(sqrtf(zz), eps) : idl / fmaxf(sqrtf(zz) * idl, eps);
-      float dn = 0.f, qa = 0.f;
+      // This warp sets the pace of the CTA (its token takes 2700 of the 2800 clk a token takes at
+      // d = 128): all five sums go through the shuffles together, and the reciprocals and square
+      // roots are the hardware estimates plus one Newton step, as in the forward kernels.
+      float dn = 0.f, qz = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        dn = fmaf(zkx[e], qx[e], dn);
+        qz = fmaf(qx[e], pz[e], qz);
+      }
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) {
+        ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        zz += __shfl_xor_sync(0xffffffffu, zz, off);
+        og += __shfl_xor_sync(0xffffffffu, og, off);
+        dn += __shfl_xor_sync(0xffffffffu, dn, off);
+        qz += __shfl_xor_sync(0xffffffffu, qz, off);
+      }
+      const float ink = rcp_nr(fmaxf(sqrt_approx(ss), eps));
+      const float idl = rcp_nr(pdelta);
+      const float sc = UX ? rcp_nr(fmaxf(sqrt_approx(zz), eps)) : idl * rcp_nr(fmaxf(sqrt_approx(zz) * idl, eps));
+      const float qa = sc * qz;      // qf . alpha
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
         khx[e] = kx[e] * ink;
         alx[e] = sc * pz[e];
-        dn = fmaf(zkx[e], qx[e], dn);
-        qa = fmaf(qx[e], alx[e], qa);
       }
-      dn = warp_sum(dn);
-      qa = warp_sum(qa);
       const float den = ident ? 1.0f : fmaxf(dn, eps);
-      const float iden = 1.0f / den;
+      const float iden = rcp_nr(den);
 #pragma unroll
       for (int e = 0; e < EPL; ++e) dyx[e] = pg[e] * iden;
       bwd_st<EPL>(cvec(t, cKf) + c0, kx);
@@ -633,7 +643,7 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
     // k_hat, alpha, da = (dalpha - alpha (alpha.dalpha)) / ||a|| and the scalars of token t
     auto open_token = [&](int t) {
       float kx[EPL], khx[EPL], dax[EPL];
-      float ss = 0.f, zz = 0.f, zpa = 0.f, kz = 0.f, uz = 0.f;
+      float ss = 0.f, zz = 0.f, zpa = 0.f, kz = 0.f, uz = 0.f, papz = 0.f, avpz = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
         float kk = pk[e];
@@ -644,31 +654,43 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
         zz = fmaf(av, av, zz);
         zpa = fmaf(av, pa[e], zpa);
         kz = fmaf(kk, pz[e], kz);
+        papz = fmaf(pa[e], pz[e], papz);             // for da . z below, so that no second round of sums is needed
+        if (UX) avpz = fmaf(av, pz[e], avpz);
         if (UX && gu) uz = fmaf(pu[e], pz[e], uz);
       }
-      ss = warp_sum(ss); zz = warp_sum(zz); zpa = warp_sum(zpa); kz = warp_sum(kz);
-      if (UX && gu) uz = warp_sum(uz);
-      const float ink = 1.0f / fmaxf(sqrtf(ss), eps);
+      // (this warp sets the pace of the CTA: every sum of the token in one pass through the
+      // shuffles, reciprocals and square roots as in the forward kernels)
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) {
+        ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        zz += __shfl_xor_sync(0xffffffffu, zz, off);
+        zpa += __shfl_xor_sync(0xffffffffu, zpa, off);
+        kz += __shfl_xor_sync(0xffffffffu, kz, off);
+        papz += __shfl_xor_sync(0xffffffffu, papz, off);
+        if (UX) avpz += __shfl_xor_sync(0xffffffffu, avpz, off);
+        if (UX && gu) uz += __shfl_xor_sync(0xffffffffu, uz, off);
+      }
+      if (!UX) avpz = zz;
+      const float ink = rcp_nr(fmaxf(sqrt_approx(ss), eps));
       if (UX && !gu) {
 #pragma unroll
         for (int e = 0; e < EPL; ++e) pu[e] = kx[e] * ink;
         uz = kz * ink;
       }
-      const float idl = 1.0f / pdelta;
-      const float na = UX ? sqrtf(zz) : sqrtf(zz) * idl;   // ||a||  (a = z / delta when u = k_hat)
-      const float sc = (UX ? 1.0f : idl) / fmaxf(na, eps);
+      const float idl = rcp_nr(pdelta);
+      const float na = UX ? sqrt_approx(zz) : sqrt_approx(zz) * idl;   // ||a||  (a = z / delta when u = k_hat)
+      const float sc = (UX ? 1.0f : idl) * rcp_nr(fmaxf(na, eps));
       const float adal = sc * zpa;                   // alpha . dalpha
       const float khz = kz * ink;
-      const float ina = na > eps ? 1.0f / na : 1.0f / eps;
-      float daz = 0.f;
+      const float ina = rcp_nr(fmaxf(na, eps));
 #pragma unroll
       for (int e = 0; e < EPL; ++e) {
         const float al = sc * (UX ? pat[e] : pz[e]);
         dax[e] = na > eps ? (pa[e] - al * adal) * ina : pa[e] * ina;
         khx[e] = kx[e] * ink;
-        daz = fmaf(dax[e], pz[e], daz);
       }
-      daz = warp_sum(daz);
+      // da . z from the sums above: (dalpha . z - (alpha . dalpha) (alpha . z)) / ||a||, alpha . z = sc (a . z)
+      const float daz = na > eps ? (papz - adal * sc * avpz) * ina : papz * ina;
       bwd_st<EPL>(cvec(t, cKf) + c0, kx);
       bwd_st<EPL>(cvec(t, cKh) + c0, khx);
       bwd_st<EPL>(cvec(t, cZt) + c0, pz);
@@ -678,7 +700,7 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
       if constexpr (UX) bwd_st<EPL>(cvec(t, cU) + c0, pu);
       if (lane == 0) {
         float* os = cscl[t & (NCTX - 1)];
-        os[sDelta] = pdelta; os[sKhz] = khz; os[sDaz] = daz; os[sNk] = sqrtf(ss);
+        os[sDelta] = pdelta; os[sKhz] = khz; os[sDaz] = daz; os[sNk] = sqrt_approx(ss);
         os[sUz] = UX ? uz : khz;
       }
     };

@@ -333,7 +333,7 @@ __device__ __forceinline__ void vla_backward_s_body(const BackwardSplitParams& p
         }
         bwd_ld<EPL>(cvec(t, cQf) + c0, qf);
         bwd_ld<EPL>(cvec(t, cZk) + c0, zkt);
-        const float dden = den_live ? -og / den : 0.0f;   // -(S_t qf . dO) / den^2 with S_t qf = den o_t
+        const float dden = den_live ? -og * rcp_nr(den) : 0.0f;   // -(S_t qf . dO) / den^2 with S_t qf = den o_t
         float gzc[EPL], dq[EPL], gzo[EPL];
         bwd_ld<EPL>(gz + c0, gzc);
 #pragma unroll
@@ -598,7 +598,7 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
     const float* sc = cscl[t & (NCTX - 1)];
     MidScalars m;
     m.khz = sc[sKhz];
-    m.idl = 1.0f / sc[sDelta];
+    m.idl = rcp_nr(sc[sDelta]);   // (on every matrix warp's path, once a token)
     m.zg = zg;
     const bool delta_live = (1.0f + sc[sUz]) >= eps;
     m.ddelta = delta_live ? fmaf(sc[sDaz], m.khz, zg) * m.idl * m.idl : 0.0f;
@@ -737,7 +737,7 @@ __device__ __forceinline__ void vla_backward_a_body(const BackwardSplitParams& p
       bwd_ld<EPL>(rowv[t % 3][2] + c0, r3);
       const float nkraw = cscl[t & (NCTX - 1)][sNk], daz = cscl[t & (NCTX - 1)][sDaz];
       const float uz = cscl[t & (NCTX - 1)][sUz];
-      const float ink = nkraw > eps ? 1.0f / nkraw : 1.0f / eps;
+      const float ink = rcp_nr(fmaxf(nkraw, eps));
       // z . dz = cU u.z + cK khz - idl (2 z.g + khz daz);  A dz = A' dz + z (z.dz) / delta
       const float zdz = fmaf(ms.cU, uz, fmaf(ms.cK, ms.khz, -ms.idl * fmaf(ms.khz, daz, 2.0f * ms.zg)));
       const float zs = fmaf(zdz, ms.idl, ms.ddelta);

@@ -651,7 +651,9 @@ int vla_backward(const void* q, const void* k, const void* v, float lambda_, int
   f.stash_z = zst; f.stash_e = est; f.stash_delta = dst; f.stash_zk = zkcw; f.stash_a = general ? astw : nullptr;
   f.heads = H;
   f.wait_limit = o.wait_probe_limit;
-  rc = vla::launch_chunk_stash(d_k, o.qkv_dtype, f, st);
+  // d = 128, u = k_hat, no refresh: the tensor-core form of the chunk kernel leaves the same stash
+  if (chunk_tc_covers(f, d_k)) rc = vla::launch_chunk_tc_stash(d_k, o.qkv_dtype, f, st);
+  else rc = vla::launch_chunk_stash(d_k, o.qkv_dtype, f, st);
   if (rc != VLA_OK) return rc;
   // 2. the S-side and A-side reverse scans
   vla::BackwardSplitParams p;

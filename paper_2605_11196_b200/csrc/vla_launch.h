@@ -30,6 +30,8 @@ int launch_chunk_tc(int d, int dtype, const ScanParams& p, cudaStream_t st);
 
 // Chunk kernel as the forward of a backward pass: leaves z_t, e_t, delta_t per token (p.stash_*).
 int launch_chunk_stash(int d, int dtype, const ScanParams& p, cudaStream_t st);
+// The tensor-core form of the same (d = 128, u = k_hat, no refresh).
+int launch_chunk_tc_stash(int d, int dtype, const ScanParams& p, cudaStream_t st);
 
 // Chunk kernel with three warp groups per CTA (d in {32, 64}; sequence-parallel launches).
 int launch_chunk_tri(int d, int dtype, const ScanParams& p, cudaStream_t st);

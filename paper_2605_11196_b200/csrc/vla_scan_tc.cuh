@@ -216,7 +216,10 @@ static __device__ unsigned int g_tc_sched_flags[kSchedSlots * kSchedMaxUnits];
 // the caller's S_T / A_T / zT and a release/acquire flag per unit.
 // TM: q, k, v, out are [B, T, H, d]: the 16 rows of a chunk are H * d apart and move as one tiled
 // TMA request per array (rows past T arrive as zeros; the store clips them).
-template <typename TIn, bool BALANCED, bool TM = false>
+// STASH: the launch also leaves z_t, e_t, delta_t of every token and the key sum after every
+// chunk in global memory (the forward of a backward pass); an instantiation of its own, so that
+// the plain forward carries none of it.
+template <typename TIn, bool BALANCED, bool TM = false, bool STASH = false>
 __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(
     const ScanParams p, const SchedParams sp, const __grid_constant__ typename ChunkMapsArg<TM>::type maps) {
   using Cfg = TcCfg<TIn>;
@@ -604,10 +607,16 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(
         for (int t = 0; t < 16; ++t) sq[t] = z[t];
         const float tot1 = warp_reduce_scatter16(sq, lane);
         if ((lane & 1) == 0) ZSp[gw * C + (lane >> 1)] = tot1;
-#ifdef VLA_TC_DUMP
-        if (p.stash_z) for (int t = 0; t < 16; ++t) p.stash_z[(size_t(unit) * p.T + t_begin + c * C + t) * D + g] = z[t];
-        if (p.stash_delta && g < 16) p.stash_delta[size_t(unit) * p.T + t_begin + c * C + g] = dlt[g];
-#endif
+        if constexpr (STASH) {   // the backward pass walks the tokens back with these
+          const int nv = min(C, T - c * C);
+          if (p.stash_z) {
+            float* zs = p.stash_z + (size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C) * D + g;
+#pragma unroll
+            for (int t = 0; t < 16; ++t)
+              if (t < nv) zs[size_t(t) * D] = z[t];
+          }
+          if (p.stash_delta && g < nv) p.stash_delta[size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C + g] = dlt[g];
+        }
       }
       group_bar(1, NG);
       VLA_MARK(6)
@@ -728,9 +737,9 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(
         e[t] = a0 + a1;
         ep[t] = e[t] * scs[t];
         s1 = fmaf(ep[t], ssm[t], s1);          // S 1 after this chunk: += e'_t (z_t . 1)
-#ifdef VLA_TC_DUMP
-        if (p.stash_e) p.stash_e[(size_t(unit) * p.T + t_begin + c * C + t) * D + g] = e[t];
-#endif
+        if constexpr (STASH) {
+          if (p.stash_e && t < n) p.stash_e[(size_t(unit) * size_t(p.T) + size_t(t_begin) + size_t(c) * C + t) * D + g] = e[t];
+        }
       }
 #pragma unroll
       for (int t = 0; t < 16; ++t) {
@@ -916,6 +925,12 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(
         }
         const float tot = warp_reduce_scatter16(pr, lane);
         if ((lane & 1) == 0) denp[pw * C + (lane >> 1)] = tot;
+        if constexpr (STASH) {
+          // the backward pass restarts its walk back of the key sum from these (a walk from the
+          // final sum alone would cancel catastrophically at the early tokens)
+          if (p.stash_zk)
+            *reinterpret_cast<float2*>(p.stash_zk + (size_t(unit) * size_t(nch_unit) + size_t(t_begin / C + c)) * D + 2 * g) = zk;
+        }
         group_bar(3, NP);
         if (g < C) inv_den[g] = rcp_nr(fmaxf(denp[g] + denp[C + g], eps));
       } else {
@@ -1046,12 +1061,12 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(
 
 int encode_token_major_maps(const ScanParams& p, int d, int dtype, bool has_u, TokenMajorMaps* maps);
 
-template <typename TIn, bool TM>
+template <typename TIn, bool TM, bool STASH = false>
 int launch_chunk_tc_t(const ScanParams& p, cudaStream_t st) {
   using Cfg = TcCfg<TIn>;
   static_assert(Cfg::smem_bytes <= 227 * 1024, "tensor-core chunk kernel exceeds the shared memory of one CTA");
-  auto kern = vla_scan_tc_kernel<TIn, false, TM>;       // one CTA per unit
-  auto kern_bal = vla_scan_tc_kernel<TIn, true, TM>;    // persistent grid, units cut at chunks
+  auto kern = vla_scan_tc_kernel<TIn, false, TM, STASH>;       // one CTA per unit
+  auto kern_bal = vla_scan_tc_kernel<TIn, true, TM, STASH>;    // persistent grid, units cut at chunks
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess ||
       cudaFuncSetAttribute(kern_bal, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) != cudaSuccess) {
     cudaGetLastError();
@@ -1098,7 +1113,8 @@ int launch_chunk_tc_t(const ScanParams& p, cudaStream_t st) {
   } else {
     kern<<<sp.grid, Cfg::NT, Cfg::smem_bytes, st>>>(p, sp, maps);
   }
-  note_launch("vla_scan_tc_kernel", Cfg::D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, sp.grid, sp.balanced);
+  note_launch(STASH ? "vla_scan_tc_kernel(stash)" : "vla_scan_tc_kernel", Cfg::D, sizeof(TIn) == 2 ? VLA_BF16 : VLA_F32, sp.grid,
+              sp.balanced);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
 

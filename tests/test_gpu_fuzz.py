@@ -13,6 +13,12 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
+def _seeds(default):
+    """Seeds per test; VLA_FUZZ_SEEDS=N runs N of each (a longer hunt, by hand)."""
+    import os
+    return int(os.environ.get("VLA_FUZZ_SEEDS", default))
+
+
 def _draw(rng):
     d = int(rng.choice([16, 32, 64, 128]))
     B, H = int(rng.integers(1, 4)), int(rng.integers(1, 6))
@@ -36,7 +42,7 @@ def _states(rng, B, H, d, seed):
     return S0, A0, z0
 
 
-@pytest.mark.parametrize("seed", range(40))
+@pytest.mark.parametrize("seed", range(_seeds(40)))
 def test_forward_random_calls(seed):
     rng = np.random.default_rng(1000 + seed)
     d, B, H, T, dtype, flags, lam = _draw(rng)
@@ -66,7 +72,7 @@ def test_forward_random_calls(seed):
         assert e <= 1e-4, "%s %s rel err %.3e" % (label, name, e)
 
 
-@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("VLA_FUZZ_TC_SEEDS", "24"))))
+@pytest.mark.parametrize("seed", range(_seeds(24)))
 def test_tc_random_calls(seed):
     """The tensor-core kernel, forced: unit counts on both schedules, ragged lengths, both input
     types and readings, carried states, either layout."""
@@ -99,7 +105,7 @@ def test_tc_random_calls(seed):
         assert e <= 1e-4, "%s %s rel err %.3e" % (label, name, e)
 
 
-@pytest.mark.parametrize("seed", range(30))
+@pytest.mark.parametrize("seed", range(_seeds(30)))
 def test_backward_random_calls(seed):
     rng = np.random.default_rng(2000 + seed)
     d, B, H, T, dtype, flags, lam = _draw(rng)
@@ -143,7 +149,7 @@ def test_backward_random_calls(seed):
         assert e <= 3e-4, "%s %s rel err %.3e" % (label, name, e)
 
 
-@pytest.mark.parametrize("seed", range(20))
+@pytest.mark.parametrize("seed", range(_seeds(20)))
 def test_seqpar_random_calls(seed):
     rng = np.random.default_rng(3000 + seed)
     d = int(rng.choice([32, 64, 128]))

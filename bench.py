@@ -546,8 +546,11 @@ def main():
         # u formed on the device from a projection (Algorithm 1: u = L2norm(W_u k) / sqrt(d_h))
         Wu = (torch.randn((w.H, w.d, w.d), generator=torch.Generator().manual_seed(11)) / w.d ** 0.5).to(dev)
         ms_mk = timed_ms(lambda: vla.vla_make_u(kd, Wu, out=uu, stream=stream), stream, dev, 1, 3)
-        per[w.name + "_make_u"] = {"ms": ms_mk, "tokens_per_s": w.tokens / (ms_mk * 1e-3), "kernel": "vla_make_u_kernel",
-                                   "fp32_tflops": 2.0 * w.d * w.d * w.tokens / (ms_mk * 1e-3) / 1e12}
+        in_b = 2 if w.dtype == "bf16" else 4
+        per[w.name + "_make_u"] = {"ms": ms_mk, "tokens_per_s": w.tokens / (ms_mk * 1e-3),
+                                   "kernel": "vla_make_u_tc_kernel (tcgen05, TF32 hi/lo)" if w.d == 128 else "vla_make_u_kernel",
+                                   "tflops": 2.0 * w.d * w.d * w.tokens / (ms_mk * 1e-3) / 1e12,
+                                   "hbm_frac": 2.0 * w.tokens * w.d * in_b / (ms_mk * 1e-3) / 1e9 / hbm_peak}
         def wcall():
             vla.vla_make_u(kd, Wu, out=uu, stream=stream)
             vla.vla_forward(qd, kd, vd, w.lam, u=uu, **fwd)

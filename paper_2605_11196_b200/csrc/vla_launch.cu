@@ -5,6 +5,7 @@
 #include "vla_backward.cuh"
 #include "vla_backward_split.cuh"
 #include "vla_make_u.cuh"
+#include "vla_make_u_tc.cuh"
 #include "vla_decode.cuh"
 #include "vla_scan_token.cuh"
 #include "vla_seqpar.cuh"
@@ -254,6 +255,28 @@ int launch_make_u_t(const MakeUParams& p, cudaStream_t st) {
   kern<<<unsigned(ctas), 256, Cfg::smem_bytes, st>>>(p);
   return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
 }
+// d = 128: the product runs on the tensor cores
+template <typename TIn, typename TOut>
+int launch_make_u_tc_t(const MakeUParams& p, cudaStream_t st) {
+  using Cfg = MakeUTcCfg;
+  auto kern = vla_make_u_tc_kernel<TIn, TOut>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(Cfg::smem_bytes)) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return VLA_ERR_CUDA;
+  }
+  const long long ctas = (long long)p.units * ((p.T + kMakeUTokensPerCta - 1) / kMakeUTokensPerCta);
+  if (ctas <= 0) return VLA_OK;
+  if (ctas > 0x7fffffffLL) return VLA_ERR_INVALID_ARG;
+  kern<<<unsigned(ctas), Cfg::TILE, Cfg::smem_bytes, st>>>(p);
+  return cudaGetLastError() == cudaSuccess ? VLA_OK : VLA_ERR_CUDA;
+}
+int launch_make_u_tc(int in_dtype, int out_dtype, const MakeUParams& p, cudaStream_t st) {
+  const bool fi = in_dtype == VLA_F32, fo = out_dtype == VLA_F32;
+  if (fi) return fo ? launch_make_u_tc_t<float, float>(p, st) : launch_make_u_tc_t<float, uint16_t>(p, st);
+  return fo ? launch_make_u_tc_t<uint16_t, float>(p, st) : launch_make_u_tc_t<uint16_t, uint16_t>(p, st);
+}
+
 template <int D>
 int launch_make_u_d(int in_dtype, int out_dtype, const MakeUParams& p, cudaStream_t st) {
   const bool fi = in_dtype == VLA_F32, fo = out_dtype == VLA_F32;
@@ -267,7 +290,7 @@ int launch_make_u(int d, int in_dtype, int out_dtype, const MakeUParams& p, cuda
     case 16: return launch_make_u_d<16>(in_dtype, out_dtype, p, st);
     case 32: return launch_make_u_d<32>(in_dtype, out_dtype, p, st);
     case 64: return launch_make_u_d<64>(in_dtype, out_dtype, p, st);
-    case 128: return launch_make_u_d<128>(in_dtype, out_dtype, p, st);
+    case 128: return launch_make_u_tc(in_dtype, out_dtype, p, st);
     default: return VLA_ERR_UNSUPPORTED;
   }
 }

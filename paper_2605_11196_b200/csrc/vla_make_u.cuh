@@ -1,9 +1,10 @@
 // Penalty directions from a projection (Algorithm 1, the step u_t = L2norm(W_u k_t) / sqrt(d_h)):
 //   y_t = W_u[h] k_t,   u_t = scale * y_t / max(||y_t||, eps)
 // for every token of every (batch, head) unit, written in the layout and element type the scan
-// kernels read explicit directions in.  A dense [tokens, d] x [d, d] product per head, kept on
-// the fp32 FMA pipe: u feeds the recurrence, whose 1e-4 bound leaves no room for a
-// reduced-precision product, and it is 2 d^2 of the scan's ~12 d^2 flops per token.
+// kernels read explicit directions in.  A dense [tokens, d] x [d, d] product per head.  This
+// file: the fp32-FMA form, used for d < 128 (d = 128 runs on the tensor cores, vla_make_u_tc.cuh):
+// u feeds the recurrence, whose 1e-4 bound leaves no room for a reduced-precision product, and
+// it is 2 d^2 of the scan's ~12 d^2 flops per token.
 //
 // One CTA of 256 threads takes kTokensPerCta consecutive tokens of one unit, W_u[h]^T staged
 // once in shared memory; per tile of 64 tokens thread (ty, tx) of a 16 x 16 grid forms 4

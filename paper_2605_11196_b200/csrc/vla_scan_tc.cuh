@@ -36,15 +36,13 @@
 
 namespace vla {
 
-#ifndef VLA_TC_GRAM_UNROLL
-#define VLA_TC_GRAM_UNROLL 4
-#endif
-#ifndef VLA_TC_PREP_UNROLL
-#define VLA_TC_PREP_UNROLL 2
-#endif
-#ifndef VLA_TC_LOOP_UNROLL
-#define VLA_TC_LOOP_UNROLL 1
-#endif
+// Unrolling, as measured: the chunk loop of the four roles is straight-line code that is fetched
+// anew every chunk, so code size counts.  The Gram loops stay fully unrolled (rolled: 5 KB less,
+// 25 % slower), the prep group's passes take two steps at a time (it has time to spare), the chunk
+// loops themselves are not unrolled (twice: same work, 40 % slower).
+constexpr int kTcGramUnroll = 4;
+constexpr int kTcPrepUnroll = 2;
+constexpr int kTcLoopUnroll = 1;
 // ---------------------------------------------------------------- configuration
 template <typename TIn>
 struct TcCfg {
@@ -84,7 +82,7 @@ struct TcCfg {
 template <int CP, int XS>
 __device__ __forceinline__ void gram16_tc(const float* X, const float* Y, float* G, int g) {
   constexpr int P = 8;
-  constexpr int kGramUnroll = VLA_TC_GRAM_UNROLL;
+  constexpr int kGramUnroll = kTcGramUnroll;
   const int tile = g / P, part = g % P;
   const int i0 = (tile >> 2) * 4, j0 = (tile & 3) * 4;
   float2 w2[16];
@@ -140,8 +138,8 @@ __global__ void __launch_bounds__(TcCfg<TIn>::NT, 1) vla_scan_tc_kernel(
   using Cfg = TcCfg<TIn>;
   constexpr int D = Cfg::D, C = Cfg::C, NG = Cfg::NG, NP = Cfg::NP, CP = Cfg::CP, VP = Cfg::VP;
   constexpr int NSTAGE = Cfg::NSTAGE, KRING = Cfg::KRING, RING = Cfg::RING;
-  constexpr int kLoopUnroll = VLA_TC_LOOP_UNROLL;
-  constexpr int kPrepUnroll = VLA_TC_PREP_UNROLL;
+  constexpr int kLoopUnroll = kTcLoopUnroll;
+  constexpr int kPrepUnroll = kTcPrepUnroll;
 
   extern __shared__ __align__(128) unsigned char smem[];
   TIn* raw = reinterpret_cast<TIn*>(smem);

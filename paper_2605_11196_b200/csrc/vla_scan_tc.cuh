@@ -108,16 +108,8 @@ __device__ __forceinline__ void gram16_tc(const float* X, const float* Y, float*
   float w[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) w[i] = w2[i].x + w2[i].y;
-#pragma unroll
-  for (int off = P / 2; off >= 1; off >>= 1)
-#pragma unroll
-    for (int i = 0; i < 16; ++i) w[i] += __shfl_xor_sync(0xffffffffu, w[i], off);
-  if (part == 0) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      *reinterpret_cast<float4*>(G + (i0 + i) * CP + j0) =
-          make_float4(w[4 * i + 0], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
-  }
+  const int base = tile16_reduce_scatter<P>(w, part);
+  tile16_store<P, CP>(G, i0, j0, w, base);
 }
 
 // Hand-over flags of the balanced schedule (see SchedParams): one word per unit and slot.

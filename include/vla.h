@@ -267,7 +267,8 @@ size_t vla_backward_workspace_bytes(int B, int H, int T, int d_k);
  *
  *     y_t = W_u[h] k_t,     u_t = scale * y_t / max(||y_t||_2, eps)
  *
- * for every token of every (b, h), in fp32 on the device.  k [B,H,T,d_k] (k_dtype, the raw keys:
+ * for every token of every (b, h), to fp32 accuracy on the device (d_k = 128: on the tensor cores,
+ * TF32 products in hi/lo pairs with fp32 accumulation; below that on the fp32 pipe).  k [B,H,T,d_k] (k_dtype, the raw keys:
  * no feature map is applied), W_u [H,d_k,d_k] fp32 row-major (one matrix per head; y = W k),
  * u [B,H,T,d_k] (u_dtype: VLA_F32, or VLA_BF16 rounded to nearest even) -- the buffer a later
  * vla_forward takes as opts->u (with opts->qkv_dtype == u_dtype).  scale is used as given
